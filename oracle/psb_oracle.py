@@ -1,0 +1,218 @@
+"""ctypes front end of the CPU oracle (``psb_oracle.cpp``).
+
+TEST INFRASTRUCTURE ONLY.  The oracle is the slow, plain restatement of the
+paper's definitions that the CUDA library is compared against.  Nothing in the
+product path may import this module; it shares no code with the CUDA library.
+"""
+import ctypes as C
+import os
+import subprocess
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "psb_oracle.cpp")
+_LIB = os.path.join(_HERE, "libpsb_oracle.so")
+
+NCHW, NHWC = 0, 1
+U8, S8 = 0, 1
+
+
+def build(force=False):
+    """Compile the oracle with the host compiler (no CUDA involved)."""
+    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
+        cmd = ["g++", "-O2", "-std=c++17", "-ffp-contract=off", "-fPIC", "-shared", _SRC, "-o", _LIB]
+        subprocess.run(cmd, check=True)
+    return _LIB
+
+
+class _Geom(C.Structure):
+    _fields_ = [(n, C.c_uint32) for n in (
+        "layout", "x_dtype", "N", "C", "H", "W", "O", "KH", "KW", "groups", "stride", "pad", "OH", "OW")]
+
+
+class _Epi(C.Structure):
+    _fields_ = [("scale", C.c_void_p), ("bias", C.c_void_p), ("e_base", C.c_void_p),
+                ("residual", C.c_void_p), ("residual_dtype", C.c_uint32),
+                ("residual_scale", C.c_float), ("relu", C.c_uint32), ("inv_step", C.c_float),
+                ("qmin", C.c_int32), ("qmax", C.c_int32)]
+
+
+_lib = None
+
+
+def lib():
+    global _lib
+    if _lib is None:
+        _lib = C.CDLL(build())
+        _lib.psbo_decode.argtypes = [C.c_float, C.POINTER(C.c_int), C.POINTER(C.c_int), C.POINTER(C.c_uint32)]
+        _lib.psbo_decode.restype = C.c_int
+        _lib.psbo_draw_bit.argtypes = [C.c_uint64, C.c_uint32, C.c_uint64, C.c_uint32, C.c_uint32]
+        _lib.psbo_draw_bit.restype = C.c_int
+        _lib.psbo_dequant_one.argtypes = [C.c_int64, C.c_float, C.c_int32, C.c_uint32, C.c_float,
+                                          C.c_int, C.c_int32, C.c_float, C.c_int]
+        _lib.psbo_dequant_one.restype = C.c_float
+        _lib.psbo_requant_one.argtypes = [C.c_float, C.c_float, C.c_int32, C.c_int32]
+        _lib.psbo_requant_one.restype = C.c_int32
+        _lib.psbo_sample_level.restype = C.c_int
+        _lib.psbo_conv_acc.restype = C.c_int
+        _lib.psbo_conv_acc_points.restype = C.c_int
+        _lib.psbo_window.restype = C.c_int
+    return _lib
+
+
+def _p(a):
+    return None if a is None else C.c_void_p(a.ctypes.data)
+
+
+def philox4x32_10(ctr, key):
+    c = np.asarray(ctr, dtype=np.uint32)
+    k = np.asarray(key, dtype=np.uint32)
+    out = np.zeros(4, dtype=np.uint32)
+    lib().psbo_philox4x32_10(_p(c), _p(k), _p(out))
+    return out
+
+
+def decode(w):
+    """Eq. 5-7: returns (class, s, e, p * 2^23); class 0 = zero, 1 = normal, 2 = non-finite."""
+    s, e, m = C.c_int(), C.c_int(), C.c_uint32()
+    cls = lib().psbo_decode(C.c_float(float(np.float32(w))), C.byref(s), C.byref(e), C.byref(m))
+    return cls, s.value, e.value, m.value
+
+
+def draw_bit(seed, layer, index, j, p_num):
+    return lib().psbo_draw_bit(seed, layer, index, j, p_num)
+
+
+def sample_level(w, seed, layer, log2k, exp_bits=4, norm=0, counts_in=None):
+    """Integer weights of level k = 2**log2k for a filter of shape [O, ...].
+
+    Returns (W int64 of w's shape, e_base int32 [O], counts uint32 of w's shape).
+    """
+    w = np.ascontiguousarray(w, dtype=np.float32)
+    O = w.shape[0]
+    D = int(np.prod(w.shape[1:])) if w.ndim > 1 else 1
+    W_out = np.zeros(w.shape, dtype=np.int64)
+    e_base = np.zeros(O, dtype=np.int32)
+    counts = np.zeros(w.shape, dtype=np.uint32)
+    cin = None if counts_in is None else np.ascontiguousarray(counts_in, dtype=np.uint32)
+    rc = lib().psbo_sample_level(_p(w), C.c_uint32(O), C.c_uint64(D), C.c_uint64(seed),
+                                 C.c_uint32(layer), C.c_uint32(exp_bits), C.c_uint32(norm),
+                                 C.c_uint32(log2k), _p(cin), _p(W_out), _p(e_base), _p(counts))
+    if rc != 0:
+        raise ValueError("non-finite weight")
+    return W_out, e_base, counts
+
+
+def geom(x_shape, layout, x_dtype, w_shape, groups, stride, pad):
+    if layout == NCHW:
+        N, Cc, H, W = x_shape
+    else:
+        N, H, W, Cc = x_shape
+    O, Cg, KH, KW = w_shape
+    assert Cg * groups == Cc and O % groups == 0
+    OH = (H + 2 * pad - KH) // stride + 1
+    OW = (W + 2 * pad - KW) // stride + 1
+    return _Geom(layout, x_dtype, N, Cc, H, W, O, KH, KW, groups, stride, pad, OH, OW)
+
+
+def out_shape(g):
+    return (g.N, g.O, g.OH, g.OW) if g.layout == NCHW else (g.N, g.OH, g.OW, g.O)
+
+
+def _levels_array(W_levels):
+    arr = (C.c_void_p * 7)()
+    keep = []
+    for lvl, Wk in W_levels.items():
+        a = np.ascontiguousarray(Wk, dtype=np.int64)
+        keep.append(a)
+        arr[lvl] = a.ctypes.data
+    return arr, keep
+
+
+def conv_acc(x, g, W_levels, kmap=None, uniform_log2k=0):
+    """Exact int64 accumulators of the whole layer; W_levels maps log2k -> int64 filter."""
+    x = np.ascontiguousarray(x)
+    arr, keep = _levels_array(W_levels)
+    km = None if kmap is None else np.ascontiguousarray(kmap, dtype=np.uint8)
+    acc = np.zeros(out_shape(g), dtype=np.int64)
+    rc = lib().psbo_conv_acc(_p(x), C.byref(g), arr, _p(km), C.c_uint32(uniform_log2k), _p(acc))
+    if rc != 0:
+        raise ValueError("level not sampled")
+    return acc
+
+
+def conv_acc_points(x, g, W_levels, pts, kmap=None, uniform_log2k=0):
+    """Accumulators at the rows of pts = [[n, o, oy, ox], ...] only."""
+    x = np.ascontiguousarray(x)
+    arr, keep = _levels_array(W_levels)
+    km = None if kmap is None else np.ascontiguousarray(kmap, dtype=np.uint8)
+    pts = np.ascontiguousarray(pts, dtype=np.uint32)
+    acc = np.zeros(len(pts), dtype=np.int64)
+    rc = lib().psbo_conv_acc_points(_p(x), C.byref(g), arr, _p(km), C.c_uint32(uniform_log2k),
+                                    _p(pts), C.c_uint64(len(pts)), _p(acc))
+    if rc != 0:
+        raise ValueError("level not sampled")
+    return acc
+
+
+def epilogue(acc, g, scale, bias, e_base, relu, inv_step, qmin, qmax, residual=None,
+             residual_scale=0.0, kmap=None, uniform_log2k=0):
+    """Dequantise, add bias and shortcut, ReLU, re-quantise.  Returns (y float32, q int32)."""
+    acc = np.ascontiguousarray(acc, dtype=np.int64)
+    scale = np.ascontiguousarray(scale, dtype=np.float32)
+    bias = np.ascontiguousarray(bias, dtype=np.float32)
+    e_base = np.ascontiguousarray(e_base, dtype=np.int32)
+    res = None
+    rdt = 0
+    if residual is not None:
+        res = np.ascontiguousarray(residual)
+        assert res.shape == acc.shape and res.dtype in (np.uint8, np.int8)
+        rdt = U8 if res.dtype == np.uint8 else S8
+    km = None if kmap is None else np.ascontiguousarray(kmap, dtype=np.uint8)
+    ep = _Epi(scale.ctypes.data, bias.ctypes.data, e_base.ctypes.data,
+              None if res is None else res.ctypes.data, rdt, residual_scale, int(relu),
+              inv_step, qmin, qmax)
+    y = np.zeros(acc.shape, dtype=np.float32)
+    q = np.zeros(acc.shape, dtype=np.int32)
+    lib().psbo_epilogue_apply(_p(acc), C.byref(g), C.byref(ep), _p(km), C.c_uint32(uniform_log2k),
+                              _p(y), _p(q))
+    return y, q
+
+
+def dequant_one(acc, scale, e_base, log2k, bias, res_q=None, res_scale=0.0, relu=False):
+    return lib().psbo_dequant_one(int(acc), float(np.float32(scale)), int(e_base), int(log2k),
+                                  float(np.float32(bias)), 0 if res_q is None else 1,
+                                  0 if res_q is None else int(res_q), float(np.float32(res_scale)),
+                                  int(relu))
+
+
+def requant_one(y, inv_step, qmin, qmax):
+    return lib().psbo_requant_one(float(np.float32(y)), float(np.float32(inv_step)), qmin, qmax)
+
+
+def maxpool_u8(x, layout, ksize, stride, pad):
+    x = np.ascontiguousarray(x, dtype=np.uint8)
+    if layout == NCHW:
+        N, Cc, H, W = x.shape
+    else:
+        N, H, W, Cc = x.shape
+    OH = (H + 2 * pad - ksize) // stride + 1
+    OW = (W + 2 * pad - ksize) // stride + 1
+    out = np.zeros((N, Cc, OH, OW) if layout == NCHW else (N, OH, OW, Cc), dtype=np.uint8)
+    lib().psbo_maxpool_u8(_p(x), C.c_uint32(layout), C.c_uint32(N), C.c_uint32(Cc), C.c_uint32(H),
+                          C.c_uint32(W), C.c_uint32(ksize), C.c_uint32(stride), C.c_uint32(pad), _p(out))
+    return out
+
+
+def global_avgpool_u8(x, layout, pool_mul, qmin, qmax):
+    x = np.ascontiguousarray(x, dtype=np.uint8)
+    if layout == NCHW:
+        N, Cc, H, W = x.shape
+    else:
+        N, H, W, Cc = x.shape
+    out = np.zeros((N, Cc), dtype=np.uint8)
+    lib().psbo_global_avgpool_u8(_p(x), C.c_uint32(layout), C.c_uint32(N), C.c_uint32(Cc),
+                                 C.c_uint32(H), C.c_uint32(W), C.c_float(pool_mul), C.c_int32(qmin),
+                                 C.c_int32(qmax), _p(out))
+    return out

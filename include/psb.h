@@ -1,0 +1,225 @@
+/*
+ * psb.h - C ABI of the B200 (sm_100a) library for progressive stochastic
+ * binarization (PSB) inference layers, after "Progressive Stochastic
+ * Binarization of Deep Networks" (arXiv 1904.02205).
+ *
+ * What a layer computes (paper Sec. 3 and 3.1):
+ *   Eq. 1    y = relu(sum_i x_i * w_i)                      the layer
+ *   Eq. 4-7  w -> s * 2^e * (B_p + 1),  s = sign w, e = floor(log2 |w|),
+ *            p = |w| / 2^e - 1, B_p a Bernoulli(p) bit      the number system
+ *   Eq. 8    w -> s * 2^e * (B_{k,p} / k + 1)               k accumulated draws
+ *   Eq. 9    x * w_k = s * (sum_j x << (e + B_p^(j))) >> log2 k
+ * Activations x are small integers (one byte each); every weight is replaced by
+ * k random picks between its two neighbouring powers of two; the sum over the k
+ * picks and over i is an exact integer; k may differ per output location
+ * (Sec. 4.5).  The library keeps the integer accumulator exact (64-bit) and folds
+ * 1/k and the group's base exponent into the fp32 dequantisation scale.
+ *
+ * Conventions
+ *   - Every pointer named *_dev is DEVICE memory owned by the caller unless said
+ *     otherwise; everything else is host memory.  Sizes are in elements.
+ *   - `stream` is a cudaStream_t passed as void*.  All compute calls are
+ *     asynchronous on that stream and never synchronise the device; only
+ *     psb_create, psb_destroy, the first psb_sample_weights for a handle,
+ *     psb_weights_free and psb_device_status may block.
+ *   - Every function returns a psb_status: 0 on success, negative on error.
+ *     Arguments are validated on the host before anything is launched; a call
+ *     that returns an error has launched nothing.  There is no CPU fallback: if
+ *     no CUDA device is usable, psb_create fails.
+ *   - Filters are given as fp32 in canonical [out_ch][in_ch/groups][kh][kw]
+ *     order.  The canonical linear index of a weight in that order keys its
+ *     random stream, so results do not depend on any internal tiling.
+ *   - Activation tensors are [n][c][h][w] (PSB_LAYOUT_NCHW) or [n][h][w][c]
+ *     (PSB_LAYOUT_NHWC), one byte per element.  NHWC is the native layout; NCHW
+ *     inputs and outputs are converted inside the call.
+ */
+#ifndef PSB_H_
+#define PSB_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef int32_t psb_status;
+
+enum {
+  PSB_OK = 0,
+  PSB_ERR_INVALID_ARG = -1,      /* null / misaligned pointer, zero dimension, shape mismatch   */
+  PSB_ERR_BAD_K = -2,            /* level not sampled, or k not a power of two in 1..64          */
+  PSB_ERR_UNSUPPORTED = -3,      /* valid request that no kernel of this library covers          */
+  PSB_ERR_ALLOC = -4,            /* device or host allocation failed                             */
+  PSB_ERR_CUDA = -5,             /* a CUDA runtime / driver call failed                          */
+  PSB_ERR_TIMEOUT = -6,          /* a bounded device-side wait ran out (reported by the device)  */
+  PSB_ERR_NONFINITE_WEIGHT = -7  /* a filter holds Inf or NaN (reported by the device)           */
+};
+
+enum { PSB_LAYOUT_NCHW = 0, PSB_LAYOUT_NHWC = 1 };
+enum { PSB_DT_U8 = 0, PSB_DT_S8 = 1 };
+
+/* Which contraction kernel a conv / gemm call uses. */
+enum {
+  PSB_PATH_AUTO = 0,       /* library chooses                                                     */
+  PSB_PATH_SHIFT_ADD = 1,  /* CUDA-core integer path (depthwise, tiny batch, few input channels)  */
+  PSB_PATH_TENSOR = 2      /* tcgen05 int8 MMA on signed digit planes, accumulators in TMEM       */
+};
+
+typedef struct psb_ctx psb_ctx;         /* per-device state: error word, scratch, current draw-count map */
+typedef struct psb_weights psb_weights; /* library-owned sampled integer filters of one layer            */
+
+/* Create / destroy the per-device context.  `device` is a CUDA ordinal.  The
+ * context owns a small device error word and scratch buffers that grow on
+ * demand (growth allocates, so it blocks).  Not thread-safe: use one context per
+ * host thread. */
+psb_status psb_create(psb_ctx** ctx, int device);
+psb_status psb_destroy(psb_ctx* ctx);
+
+/* Static, human-readable name of a status code. */
+const char* psb_status_string(psb_status st);
+
+/* Synchronise `stream`, then return and clear the sticky device-side error
+ * (PSB_ERR_TIMEOUT, PSB_ERR_NONFINITE_WEIGHT, PSB_ERR_BAD_K from a draw-count
+ * map naming a level that was not sampled), or PSB_OK. */
+psb_status psb_device_status(psb_ctx* ctx, void* stream);
+
+/* Shape of a filter in canonical order [out_ch][in_ch_per_group][kh][kw]. */
+typedef struct {
+  uint32_t out_ch, in_ch_per_group, kh, kw, groups;
+} psb_wshape;
+
+/* How to sample a filter.
+ *   seed, layer_id  key of the random stream: draw j of the weight with canonical
+ *                   index i is word (j mod 4) of Philox4x32-10 with counter
+ *                   (j / 4, layer_id, lo32(i), hi32(i)) and key (lo32(seed),
+ *                   hi32(seed)); the bit is 1 ("upper shift", Eq. 4) when that
+ *                   word is below p * 2^32.
+ *   level_mask      bit l set => produce the filter for k = 2^l draws, l = 0..6.
+ *                   All levels share draws: level k uses draws 0..k-1
+ *                   (progressive refinement, Sec. 1.1).
+ *   exp_bits        1..4: exponents are kept in a window of 2^exp_bits octaves
+ *                   below the group's largest exponent; smaller weights, zeros
+ *                   and sub-normals contribute nothing (Sec. 4.4: 4-bit
+ *                   exponents suffice).  0 selects 4.
+ *   norm            0: one exponent window per layer; 1: one per output channel. */
+typedef struct {
+  uint64_t seed;
+  uint32_t layer_id;
+  uint32_t level_mask;
+  uint32_t exp_bits;
+  uint32_t norm;
+} psb_sample_cfg;
+
+/* Draw the random bits and build the integer filters (Eq. 8 scaled by
+ * k / 2^e_base):  W_k[i] = s_i * (k + c_k[i]) * 2^(e_i - e_base),  c_k = number of
+ * upper draws among the first k.  Nothing random is stored: the bits live in
+ * registers only.
+ *   w_dev     fp32 filter, canonical order, device memory, 4-byte aligned.
+ *   *weights  NULL: a handle is created (allocates, blocks).  Non-NULL: must
+ *             come from an earlier call with the same shape, level_mask,
+ *             exp_bits; it is re-sampled in place without allocating.
+ * A filter with Inf/NaN sets the device error word (see psb_device_status). */
+psb_status psb_sample_weights(psb_ctx* ctx, const float* w_dev, const psb_wshape* shape,
+                              const psb_sample_cfg* cfg, psb_weights** weights, void* stream);
+
+/* Test hook: copy the level-2^log2k integer filter (int32, canonical order,
+ * out_ch*in_ch_per_group*kh*kw elements) and e_base (int32 [out_ch]) to caller
+ * device buffers.  Either pointer may be NULL. */
+psb_status psb_weights_export(psb_ctx* ctx, const psb_weights* weights, uint32_t log2k,
+                              int32_t* wint_dev, int32_t* e_base_dev, void* stream);
+
+psb_status psb_weights_free(psb_ctx* ctx, psb_weights* weights);
+
+/* Localised accuracy control (Sec. 4.5): the number of draws used by output
+ * location (n, oy, ox) of the following conv / gemm calls.
+ *   log2k_dev      u8 [n][oh][ow] holding log2 k per location, or NULL for a
+ *                  uniform k = 2^uniform_log2k.  The pointer is borrowed: it must
+ *                  stay valid until the calls that use it have finished.  Its
+ *                  dimensions must equal the output dimensions of those calls.
+ * The setting is sticky until changed.  A new context starts uniform, k = 1. */
+psb_status psb_set_sample_map(psb_ctx* ctx, const uint8_t* log2k_dev, uint32_t n, uint32_t oh,
+                              uint32_t ow, uint32_t uniform_log2k);
+
+/* Fused output stage (Eq. 1's relu, the folded batch-norm a*y+b of Sec. 3, and
+ * the fixed-point intermediates of Sec. 4.1), per output element:
+ *   a  = (float) acc                              round to nearest even
+ *   y  = fma(a, scale[o] * 2^(e_base[o] - log2 k), bias[o])
+ *   y  = fma((float) residual, residual_scale, y)  if residual_dev != NULL
+ *   y  = max(y, 0)                                 if relu
+ *   q  = clamp(rint(y * inv_step), qmin, qmax)     ties to even
+ * Outputs, each optional (NULL) but at least one present, all in the layout of
+ * the call: q_out_dev (one byte, out_dtype), f32_out_dev (y), acc_out_dev (the
+ * raw 64-bit accumulator, a test hook).  residual_dev has the output's shape and
+ * layout, one byte per element of residual_dtype. */
+typedef struct {
+  const float* scale_dev;    /* [out_ch] */
+  const float* bias_dev;     /* [out_ch] */
+  const void* residual_dev;  /* nullable */
+  float residual_scale;
+  uint32_t residual_dtype;
+  uint32_t relu;
+  float inv_step;
+  int32_t qmin, qmax;
+  uint32_t out_dtype;        /* PSB_DT_U8 | PSB_DT_S8 */
+  void* q_out_dev;           /* nullable */
+  float* f32_out_dev;        /* nullable */
+  int64_t* acc_out_dev;      /* nullable */
+} psb_epilogue;
+
+/* 2-D convolution, zero padding, square stride.  Output size
+ * oh = (h + 2*pad - kh) / stride + 1 (same for ow).
+ *   in_max   largest activation magnitude the caller guarantees (e.g. 15 for
+ *            4-bit data); 0 means "full range of in_dtype".  The tensor path
+ *            feeds activations to the MMA as signed bytes, so it needs
+ *            in_max <= 127; larger unsigned data takes the shift-add path.
+ *   path     PSB_PATH_AUTO, or force one path (PSB_ERR_UNSUPPORTED if the forced
+ *            path cannot run this shape). */
+typedef struct {
+  uint32_t layout;
+  uint32_t in_dtype;
+  uint32_t in_max;
+  uint32_t n, c, h, w;
+  uint32_t stride, pad;
+  uint32_t path;
+  psb_epilogue ep;
+} psb_conv_desc;
+
+psb_status psb_conv2d(psb_ctx* ctx, const psb_weights* weights, const void* x_dev,
+                      const psb_conv_desc* desc, void* stream);
+
+/* Fully connected layer: x [batch][in_features] (one byte each), filter shape
+ * [out][in][1][1], outputs [batch][out].  The draw-count map, if set, is
+ * [batch][1][1]. */
+typedef struct {
+  uint32_t in_dtype;
+  uint32_t in_max;
+  uint32_t batch, in_features;
+  uint32_t path;
+  psb_epilogue ep;
+} psb_gemm_desc;
+
+psb_status psb_gemm(psb_ctx* ctx, const psb_weights* weights, const void* x_dev,
+                    const psb_gemm_desc* desc, void* stream);
+
+/* Which path the last successful psb_conv2d / psb_gemm call on this context took
+ * (PSB_PATH_SHIFT_ADD or PSB_PATH_TENSOR); 0 before any call. */
+int32_t psb_last_path(const psb_ctx* ctx);
+
+/* Glue between layers (supplement, "ReLU, Batch-Norm, and Pooling"): max-pooling
+ * is comparators only; the 1/(h*w) of average pooling is folded into one
+ * re-quantisation factor.
+ * psb_maxpool2d_u8: u8 activations, window k, given stride and padding; padded
+ *   positions never win.  Output [n][oh][ow][c] / [n][c][oh][ow].
+ * psb_global_avgpool_u8: integer sum over h*w, then
+ *   q = clamp(rint((float) sum * pool_mul), qmin, qmax), output u8 [n][c]. */
+psb_status psb_maxpool2d_u8(psb_ctx* ctx, const uint8_t* x_dev, uint32_t layout, uint32_t n,
+                            uint32_t c, uint32_t h, uint32_t w, uint32_t k, uint32_t stride,
+                            uint32_t pad, uint8_t* out_dev, void* stream);
+psb_status psb_global_avgpool_u8(psb_ctx* ctx, const uint8_t* x_dev, uint32_t layout, uint32_t n,
+                                 uint32_t c, uint32_t h, uint32_t w, float pool_mul, int32_t qmin,
+                                 int32_t qmax, uint8_t* out_dev, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* PSB_H_ */

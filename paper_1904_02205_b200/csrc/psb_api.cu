@@ -1,0 +1,352 @@
+// Host side of the C ABI declared in psb.h: argument validation, handle
+// management, path selection and kernel launches.  No arithmetic of the method
+// happens on the host.
+#include <new>
+
+#include "psb_common.cuh"
+
+using namespace psb;
+
+namespace {
+
+bool pow2_level_ok(uint32_t log2k) { return log2k < (uint32_t)kMaxLevels; }
+
+psb_status ensure_scratch(psb_ctx* ctx, int slot, size_t bytes) {
+  if (ctx->scratch_bytes[slot] >= bytes) return PSB_OK;
+  if (ctx->scratch[slot]) cudaFree(ctx->scratch[slot]);
+  ctx->scratch[slot] = nullptr;
+  ctx->scratch_bytes[slot] = 0;
+  size_t want = bytes + bytes / 4;
+  if (cudaMalloc(&ctx->scratch[slot], want) != cudaSuccess) {
+    cudaGetLastError();
+    return PSB_ERR_ALLOC;
+  }
+  ctx->scratch_bytes[slot] = want;
+  return PSB_OK;
+}
+
+void free_weights_storage(psb_weights* w) {
+  for (int l = 0; l < kMaxLevels; ++l) {
+    if (w->level[l].wint) cudaFree(w->level[l].wint);
+    if (w->level[l].planes) cudaFree(w->level[l].planes);
+    w->level[l] = LevelStore();
+  }
+  if (w->e_base) cudaFree(w->e_base);
+  if (w->e_max) cudaFree(w->e_max);
+  w->e_base = nullptr;
+  w->e_max = nullptr;
+}
+
+psb_status check_epilogue(const psb_epilogue& ep) {
+  if (!ep.scale_dev || !ep.bias_dev) return PSB_ERR_INVALID_ARG;
+  if (!ep.q_out_dev && !ep.f32_out_dev && !ep.acc_out_dev) return PSB_ERR_INVALID_ARG;
+  if (ep.out_dtype != PSB_DT_U8 && ep.out_dtype != PSB_DT_S8) return PSB_ERR_INVALID_ARG;
+  if (ep.residual_dev && ep.residual_dtype != PSB_DT_U8 && ep.residual_dtype != PSB_DT_S8)
+    return PSB_ERR_INVALID_ARG;
+  if (ep.qmin > ep.qmax) return PSB_ERR_INVALID_ARG;
+  if (ep.q_out_dev) {
+    int lo = ep.out_dtype == PSB_DT_U8 ? 0 : -128, hi = ep.out_dtype == PSB_DT_U8 ? 255 : 127;
+    if (ep.qmin < lo || ep.qmax > hi) return PSB_ERR_INVALID_ARG;
+  }
+  if (((uintptr_t)ep.scale_dev | (uintptr_t)ep.bias_dev | (uintptr_t)ep.f32_out_dev) & 3u)
+    return PSB_ERR_INVALID_ARG;
+  if ((uintptr_t)ep.acc_out_dev & 7u) return PSB_ERR_INVALID_ARG;
+  return PSB_OK;
+}
+
+// Shared body of psb_conv2d and psb_gemm.
+psb_status run_layer(psb_ctx* ctx, const psb_weights* wt, const void* x_dev, uint32_t layout,
+                     uint32_t in_dtype, uint32_t in_max, uint32_t n, uint32_t c, uint32_t h,
+                     uint32_t w, uint32_t stride, uint32_t pad, uint32_t path,
+                     const psb_epilogue& ep, void* stream) {
+  if (!ctx || !wt || !x_dev) return PSB_ERR_INVALID_ARG;
+  if (wt->device != ctx->device) return PSB_ERR_INVALID_ARG;
+  if (layout != PSB_LAYOUT_NCHW && layout != PSB_LAYOUT_NHWC) return PSB_ERR_INVALID_ARG;
+  if (in_dtype != PSB_DT_U8 && in_dtype != PSB_DT_S8) return PSB_ERR_INVALID_ARG;
+  if (path > PSB_PATH_TENSOR) return PSB_ERR_INVALID_ARG;
+  const psb_wshape& sh = wt->shape;
+  if (n == 0 || c == 0 || h == 0 || w == 0 || stride == 0) return PSB_ERR_INVALID_ARG;
+  if (c != sh.in_ch_per_group * sh.groups) return PSB_ERR_INVALID_ARG;
+  if (h + 2 * pad < sh.kh || w + 2 * pad < sh.kw) return PSB_ERR_INVALID_ARG;
+  if (pad > 0 && (pad >= sh.kh || pad >= sh.kw)) return PSB_ERR_INVALID_ARG;
+  psb_status st = check_epilogue(ep);
+  if (st != PSB_OK) return st;
+  const uint32_t oh = (h + 2 * pad - sh.kh) / stride + 1, ow = (w + 2 * pad - sh.kw) / stride + 1;
+  if ((uint64_t)n * oh * ow >= (1ull << 31)) return PSB_ERR_UNSUPPORTED;
+  if (ctx->kmap) {
+    if (ctx->map_n != n || ctx->map_oh != oh || ctx->map_ow != ow) return PSB_ERR_INVALID_ARG;
+  } else {
+    if (!pow2_level_ok(ctx->uniform_log2k) || !((wt->cfg.level_mask >> ctx->uniform_log2k) & 1u))
+      return PSB_ERR_BAD_K;
+  }
+  cudaStream_t s = (cudaStream_t)stream;
+
+  ConvArgs a;
+  a.x = x_dev;
+  a.in_dtype = in_dtype;
+  a.N = n; a.C = c; a.H = h; a.W = w;
+  a.O = sh.out_ch; a.KH = sh.kh; a.KW = sh.kw; a.groups = sh.groups;
+  a.stride = stride; a.pad = pad; a.OH = oh; a.OW = ow;
+  a.kmap = ctx->kmap;
+  a.uniform_log2k = ctx->uniform_log2k;
+  a.level_mask = wt->cfg.level_mask;
+  a.scale = ep.scale_dev; a.bias = ep.bias_dev; a.e_base = wt->e_base;
+  a.residual = ep.residual_dev; a.residual_dtype = ep.residual_dtype;
+  a.residual_scale = ep.residual_scale;
+  a.relu = ep.relu; a.inv_step = ep.inv_step; a.qmin = ep.qmin; a.qmax = ep.qmax;
+  a.out_dtype = ep.out_dtype;
+  a.q_out = ep.q_out_dev; a.f32_out = ep.f32_out_dev; a.acc_out = ep.acc_out_dev;
+  a.err = ctx->err_dev;
+  // NCHW differs from NHWC only when both the channel and the spatial extent exceed one.
+  const bool in_conv = layout == PSB_LAYOUT_NCHW && c > 1 && (uint64_t)h * w > 1;
+  a.out_nchw = (layout == PSB_LAYOUT_NCHW && sh.out_ch > 1 && (uint64_t)oh * ow > 1) ? 1u : 0u;
+
+  // largest activation magnitude the caller vouches for
+  uint32_t amax = in_max ? in_max : (in_dtype == PSB_DT_U8 ? 255u : 128u);
+  bool tensor_ok = false;
+  if (path != PSB_PATH_SHIFT_ADD) {
+    tensor_ok = (in_dtype == PSB_DT_S8 || amax <= 127u) && tensor_supported(ctx, wt, a) == PSB_OK;
+    if (path == PSB_PATH_TENSOR && !tensor_ok) return PSB_ERR_UNSUPPORTED;
+    if (path == PSB_PATH_AUTO && (uint64_t)n * oh * ow < 128) tensor_ok = false;
+  }
+
+  if (in_conv) {
+    size_t bytes = (size_t)n * c * h * w;
+    st = ensure_scratch(ctx, 0, bytes);
+    if (st != PSB_OK) return st;
+    if (launch_nchw_to_nhwc(x_dev, ctx->scratch[0], n, c, h * w, 1, s) != cudaSuccess)
+      return PSB_ERR_CUDA;
+    a.x = ctx->scratch[0];
+  }
+
+  if (tensor_ok) {
+    st = launch_tensor(ctx, wt, a, s);
+    if (st != PSB_OK) return st;
+    ctx->last_path = PSB_PATH_TENSOR;
+    return PSB_OK;
+  }
+  WintTable tab;
+  for (int l = 0; l < kMaxLevels; ++l) tab.w[l] = wt->level[l].wint;
+  if (launch_shift_add(a, tab, s) != cudaSuccess) return PSB_ERR_CUDA;
+  ctx->last_path = PSB_PATH_SHIFT_ADD;
+  return PSB_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+psb_status psb_create(psb_ctx** out, int device) {
+  if (!out) return PSB_ERR_INVALID_ARG;
+  *out = nullptr;
+  int count = 0;
+  if (cudaGetDeviceCount(&count) != cudaSuccess || device < 0 || device >= count) {
+    cudaGetLastError();
+    return PSB_ERR_CUDA;
+  }
+  if (cudaSetDevice(device) != cudaSuccess) return PSB_ERR_CUDA;
+  int major = 0;
+  cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, device);
+  if (major != 10) return PSB_ERR_UNSUPPORTED;  // kernels are built for sm_100a only
+  psb_ctx* ctx = new (std::nothrow) psb_ctx();
+  if (!ctx) return PSB_ERR_ALLOC;
+  ctx->device = device;
+  cudaDeviceGetAttribute(&ctx->sm_count, cudaDevAttrMultiProcessorCount, device);
+  if (cudaMalloc(&ctx->err_dev, sizeof(uint32_t)) != cudaSuccess ||
+      cudaMemset(ctx->err_dev, 0, sizeof(uint32_t)) != cudaSuccess) {
+    delete ctx;
+    return PSB_ERR_ALLOC;
+  }
+  cudaDriverEntryPointQueryResult q;
+  if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ctx->encode_tiled, cudaEnableDefault, &q) !=
+          cudaSuccess || q != cudaDriverEntryPointSuccess)
+    ctx->encode_tiled = nullptr;
+  if (cudaGetDriverEntryPoint("cuTensorMapEncodeIm2col", &ctx->encode_im2col, cudaEnableDefault, &q) !=
+          cudaSuccess || q != cudaDriverEntryPointSuccess)
+    ctx->encode_im2col = nullptr;
+  cudaGetLastError();
+  *out = ctx;
+  return PSB_OK;
+}
+
+psb_status psb_destroy(psb_ctx* ctx) {
+  if (!ctx) return PSB_ERR_INVALID_ARG;
+  cudaSetDevice(ctx->device);
+  cudaDeviceSynchronize();
+  for (int i = 0; i < 3; ++i)
+    if (ctx->scratch[i]) cudaFree(ctx->scratch[i]);
+  if (ctx->err_dev) cudaFree(ctx->err_dev);
+  delete ctx;
+  return PSB_OK;
+}
+
+const char* psb_status_string(psb_status st) {
+  switch (st) {
+    case PSB_OK: return "PSB_OK";
+    case PSB_ERR_INVALID_ARG: return "PSB_ERR_INVALID_ARG";
+    case PSB_ERR_BAD_K: return "PSB_ERR_BAD_K";
+    case PSB_ERR_UNSUPPORTED: return "PSB_ERR_UNSUPPORTED";
+    case PSB_ERR_ALLOC: return "PSB_ERR_ALLOC";
+    case PSB_ERR_CUDA: return "PSB_ERR_CUDA";
+    case PSB_ERR_TIMEOUT: return "PSB_ERR_TIMEOUT";
+    case PSB_ERR_NONFINITE_WEIGHT: return "PSB_ERR_NONFINITE_WEIGHT";
+    default: return "PSB_ERR_UNKNOWN";
+  }
+}
+
+psb_status psb_device_status(psb_ctx* ctx, void* stream) {
+  if (!ctx) return PSB_ERR_INVALID_ARG;
+  if (cudaStreamSynchronize((cudaStream_t)stream) != cudaSuccess) return PSB_ERR_CUDA;
+  uint32_t word = 0;
+  if (cudaMemcpy(&word, ctx->err_dev, sizeof(word), cudaMemcpyDeviceToHost) != cudaSuccess)
+    return PSB_ERR_CUDA;
+  if (word) cudaMemset(ctx->err_dev, 0, sizeof(word));
+  if (word & kDevErrTimeout) return PSB_ERR_TIMEOUT;
+  if (word & kDevErrNonFinite) return PSB_ERR_NONFINITE_WEIGHT;
+  if (word & kDevErrBadLevel) return PSB_ERR_BAD_K;
+  return PSB_OK;
+}
+
+psb_status psb_sample_weights(psb_ctx* ctx, const float* w_dev, const psb_wshape* shape,
+                              const psb_sample_cfg* cfg_in, psb_weights** weights, void* stream) {
+  if (!ctx || !w_dev || !shape || !cfg_in || !weights) return PSB_ERR_INVALID_ARG;
+  if ((uintptr_t)w_dev & 3u) return PSB_ERR_INVALID_ARG;
+  psb_sample_cfg cfg = *cfg_in;
+  if (cfg.exp_bits == 0) cfg.exp_bits = 4;
+  if (cfg.exp_bits > 4 || cfg.norm > 1) return PSB_ERR_INVALID_ARG;
+  if (cfg.level_mask == 0 || cfg.level_mask >= (1u << kMaxLevels)) return PSB_ERR_BAD_K;
+  if (!shape->out_ch || !shape->in_ch_per_group || !shape->kh || !shape->kw || !shape->groups)
+    return PSB_ERR_INVALID_ARG;
+  if (shape->out_ch % shape->groups) return PSB_ERR_INVALID_ARG;
+  if ((uint64_t)shape->kh * shape->kw > 2048) return PSB_ERR_UNSUPPORTED;
+  uint64_t d64 = (uint64_t)shape->in_ch_per_group * shape->kh * shape->kw;
+  if (d64 > (1u << 24) || d64 * shape->out_ch > (1ull << 31)) return PSB_ERR_UNSUPPORTED;
+  cudaStream_t s = (cudaStream_t)stream;
+
+  psb_weights* w = *weights;
+  if (w) {
+    const psb_wshape& a = w->shape;
+    if (a.out_ch != shape->out_ch || a.in_ch_per_group != shape->in_ch_per_group ||
+        a.kh != shape->kh || a.kw != shape->kw || a.groups != shape->groups ||
+        w->cfg.level_mask != cfg.level_mask || w->cfg.exp_bits != cfg.exp_bits ||
+        w->device != ctx->device)
+      return PSB_ERR_INVALID_ARG;
+    w->cfg = cfg;
+  } else {
+    w = new (std::nothrow) psb_weights();
+    if (!w) return PSB_ERR_ALLOC;
+    w->shape = *shape;
+    w->cfg = cfg;
+    w->device = ctx->device;
+    w->d = (uint32_t)d64;
+    w->has_planes = shape->groups == 1 && shape->in_ch_per_group % 16 == 0;
+    w->cpad = shape->in_ch_per_group;
+    w->kpad = shape->kh * shape->kw * w->cpad;
+    w->o_tiles = (shape->out_ch + kTileN - 1) / kTileN;
+    w->bk = tensor_bk(shape->in_ch_per_group);
+    bool ok = cudaMalloc(&w->e_base, sizeof(int32_t) * shape->out_ch) == cudaSuccess &&
+              cudaMalloc(&w->e_max, sizeof(uint32_t) * shape->out_ch) == cudaSuccess;
+    for (uint32_t l = 0; ok && l < (uint32_t)kMaxLevels; ++l) {
+      if (!((cfg.level_mask >> l) & 1u)) continue;
+      ok = cudaMalloc(&w->level[l].wint, sizeof(int32_t) * d64 * shape->out_ch) == cudaSuccess;
+      if (ok && w->has_planes) {
+        int P = planes_for(cfg.exp_bits, l);
+        size_t bytes = (size_t)w->o_tiles * P * kTileN * w->kpad;
+        w->level[l].planes_count = P;
+        ok = cudaMalloc(&w->level[l].planes, bytes) == cudaSuccess &&
+             cudaMemsetAsync(w->level[l].planes, 0, bytes, s) == cudaSuccess;
+      }
+    }
+    if (!ok) {
+      cudaGetLastError();
+      free_weights_storage(w);
+      delete w;
+      return PSB_ERR_ALLOC;
+    }
+  }
+  if (launch_sampler(w_dev, w, ctx->err_dev, s) != cudaSuccess) {
+    if (!*weights) { free_weights_storage(w); delete w; }
+    return PSB_ERR_CUDA;
+  }
+  *weights = w;
+  return PSB_OK;
+}
+
+psb_status psb_weights_export(psb_ctx* ctx, const psb_weights* weights, uint32_t log2k,
+                              int32_t* wint_dev, int32_t* e_base_dev, void* stream) {
+  if (!ctx || !weights) return PSB_ERR_INVALID_ARG;
+  if (!pow2_level_ok(log2k) || !((weights->cfg.level_mask >> log2k) & 1u)) return PSB_ERR_BAD_K;
+  if (((uintptr_t)wint_dev | (uintptr_t)e_base_dev) & 3u) return PSB_ERR_INVALID_ARG;
+  if (launch_export(weights, log2k, wint_dev, e_base_dev, (cudaStream_t)stream) != cudaSuccess)
+    return PSB_ERR_CUDA;
+  return PSB_OK;
+}
+
+psb_status psb_weights_free(psb_ctx* ctx, psb_weights* weights) {
+  if (!ctx || !weights) return PSB_ERR_INVALID_ARG;
+  cudaSetDevice(ctx->device);
+  cudaDeviceSynchronize();
+  free_weights_storage(weights);
+  delete weights;
+  return PSB_OK;
+}
+
+psb_status psb_set_sample_map(psb_ctx* ctx, const uint8_t* log2k_dev, uint32_t n, uint32_t oh,
+                              uint32_t ow, uint32_t uniform_log2k) {
+  if (!ctx) return PSB_ERR_INVALID_ARG;
+  if (log2k_dev) {
+    if (!n || !oh || !ow) return PSB_ERR_INVALID_ARG;
+    ctx->kmap = log2k_dev;
+    ctx->map_n = n; ctx->map_oh = oh; ctx->map_ow = ow;
+  } else {
+    if (!pow2_level_ok(uniform_log2k)) return PSB_ERR_BAD_K;
+    ctx->kmap = nullptr;
+    ctx->map_n = ctx->map_oh = ctx->map_ow = 0;
+    ctx->uniform_log2k = uniform_log2k;
+  }
+  return PSB_OK;
+}
+
+psb_status psb_conv2d(psb_ctx* ctx, const psb_weights* weights, const void* x_dev,
+                      const psb_conv_desc* d, void* stream) {
+  if (!d) return PSB_ERR_INVALID_ARG;
+  return run_layer(ctx, weights, x_dev, d->layout, d->in_dtype, d->in_max, d->n, d->c, d->h, d->w,
+                   d->stride, d->pad, d->path, d->ep, stream);
+}
+
+psb_status psb_gemm(psb_ctx* ctx, const psb_weights* weights, const void* x_dev,
+                    const psb_gemm_desc* d, void* stream) {
+  if (!d) return PSB_ERR_INVALID_ARG;
+  if (weights && (weights->shape.kh != 1 || weights->shape.kw != 1 || weights->shape.groups != 1))
+    return PSB_ERR_INVALID_ARG;
+  return run_layer(ctx, weights, x_dev, PSB_LAYOUT_NHWC, d->in_dtype, d->in_max, d->batch,
+                   d->in_features, 1, 1, 1, 0, d->path, d->ep, stream);
+}
+
+int32_t psb_last_path(const psb_ctx* ctx) { return ctx ? ctx->last_path : 0; }
+
+psb_status psb_maxpool2d_u8(psb_ctx* ctx, const uint8_t* x_dev, uint32_t layout, uint32_t n,
+                            uint32_t c, uint32_t h, uint32_t w, uint32_t k, uint32_t stride,
+                            uint32_t pad, uint8_t* out_dev, void* stream) {
+  if (!ctx || !x_dev || !out_dev || !n || !c || !h || !w || !k || !stride) return PSB_ERR_INVALID_ARG;
+  if (layout > PSB_LAYOUT_NHWC || h + 2 * pad < k || w + 2 * pad < k || pad >= k)
+    return PSB_ERR_INVALID_ARG;
+  if (launch_maxpool(x_dev, layout == PSB_LAYOUT_NCHW, n, c, h, w, k, stride, pad, out_dev,
+                     (cudaStream_t)stream) != cudaSuccess)
+    return PSB_ERR_CUDA;
+  return PSB_OK;
+}
+
+psb_status psb_global_avgpool_u8(psb_ctx* ctx, const uint8_t* x_dev, uint32_t layout, uint32_t n,
+                                 uint32_t c, uint32_t h, uint32_t w, float pool_mul, int32_t qmin,
+                                 int32_t qmax, uint8_t* out_dev, void* stream) {
+  if (!ctx || !x_dev || !out_dev || !n || !c || !h || !w) return PSB_ERR_INVALID_ARG;
+  if (layout > PSB_LAYOUT_NHWC || qmin < 0 || qmax > 255 || qmin > qmax) return PSB_ERR_INVALID_ARG;
+  if ((uint64_t)h * w * 255 >= (1ull << 31)) return PSB_ERR_UNSUPPORTED;
+  if (launch_avgpool(x_dev, layout == PSB_LAYOUT_NCHW, n, c, h, w, pool_mul, qmin, qmax, out_dev,
+                     (cudaStream_t)stream) != cudaSuccess)
+    return PSB_ERR_CUDA;
+  return PSB_OK;
+}
+
+}  // extern "C"

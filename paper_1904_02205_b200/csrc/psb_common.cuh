@@ -1,0 +1,145 @@
+// Internal declarations shared by the translation units of the PSB library.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "psb.h"
+
+namespace psb {
+
+constexpr int kMaxLevels = 7;        // k = 1, 2, 4, ..., 64
+constexpr int kDigitBits = 7;        // magnitude bits per signed digit plane
+constexpr int kTileN = 64;           // output channels per tensor-path tile
+constexpr int kMaxPlanes = 4;
+
+// Bits of the device error word.
+constexpr uint32_t kDevErrNonFinite = 1u;
+constexpr uint32_t kDevErrTimeout = 2u;
+constexpr uint32_t kDevErrBadLevel = 4u;
+
+// Number of 7-bit digit planes that hold |W_k| = (k + c) * 2^(e - e_base) for
+// every weight of a window of 2^exp_bits octaves: the top value is 2k * 2^span.
+inline int planes_for(uint32_t exp_bits, uint32_t log2k) {
+  int span = (1 << exp_bits) - 1;
+  int bits = span + (int)log2k + 2;  // bit length of 2k << span
+  return (bits + kDigitBits - 1) / kDigitBits;
+}
+
+// Reduction-axis block (bytes of activations per MMA stage row) for the tensor path.
+inline uint32_t tensor_bk(uint32_t cg) { return cg >= 128 ? 128u : (cg >= 64 ? 64u : 32u); }
+inline uint32_t round_up(uint32_t a, uint32_t b) { return (a + b - 1) / b * b; }
+
+struct LevelStore {
+  int32_t* wint = nullptr;  // [O][KH][KW][Cg]  signed integer filter, channels innermost
+  int8_t* planes = nullptr; // [O_tiles][P][kTileN][Kpad]  signed 7-bit digits, Kpad = KH*KW*Cpad
+  int planes_count = 0;
+};
+
+}  // namespace psb
+
+struct psb_weights {
+  psb_wshape shape;
+  psb_sample_cfg cfg;
+  uint32_t d;        // in_ch_per_group * kh * kw
+  uint32_t cpad;     // channels per tap in the plane layout (multiple of the K block)
+  uint32_t kpad;     // kh * kw * cpad
+  uint32_t o_tiles;  // ceil(out_ch / kTileN)
+  uint32_t bk;       // K block of the tensor path
+  bool has_planes;   // digit planes are produced (groups == 1)
+  psb::LevelStore level[psb::kMaxLevels];
+  int32_t* e_base = nullptr;   // [O]
+  uint32_t* e_max = nullptr;   // [O] scratch of the window reduction (biased exponent, 0 = none)
+  int device;
+};
+
+struct psb_ctx {
+  int device;
+  uint32_t* err_dev = nullptr;      // device error word
+  const uint8_t* kmap = nullptr;    // borrowed
+  uint32_t map_n = 0, map_oh = 0, map_ow = 0;
+  uint32_t uniform_log2k = 0;
+  void* scratch[3] = {nullptr, nullptr, nullptr};   // layout conversion buffers
+  size_t scratch_bytes[3] = {0, 0, 0};
+  int32_t last_path = 0;
+  int sm_count = 0;
+  void* encode_tiled = nullptr;     // cuTensorMapEncodeTiled
+  void* encode_im2col = nullptr;    // cuTensorMapEncodeIm2col
+};
+
+namespace psb {
+
+// Everything a contraction kernel needs besides the filter.
+struct ConvArgs {
+  const void* x;         // NHWC activations
+  uint32_t in_dtype;
+  uint32_t N, C, H, W, O, KH, KW, groups, stride, pad, OH, OW;
+  const uint8_t* kmap;   // [N][OH][OW] or null
+  uint32_t uniform_log2k;
+  uint32_t level_mask;
+  // epilogue
+  const float* scale;
+  const float* bias;
+  const int32_t* e_base;
+  const void* residual;
+  uint32_t residual_dtype;
+  float residual_scale;
+  uint32_t relu;
+  float inv_step;
+  int32_t qmin, qmax;
+  uint32_t out_dtype;
+  void* q_out;
+  float* f32_out;
+  int64_t* acc_out;
+  uint32_t out_nchw;     // outputs (and residual) are laid out [n][o][oy][ox]
+  uint32_t* err;
+};
+
+struct WintTable {
+  const int32_t* w[kMaxLevels];
+};
+struct PlaneTable {
+  const int8_t* p[kMaxLevels];
+  int count[kMaxLevels];
+};
+
+// ---- fused output stage, identical in every kernel ---------------------------
+// sc = scale[o] * 2^(e_base[o] - log2k) is exact; the rest is one fma, an
+// optional fma for the shortcut, a max, one multiply and a round-half-even.
+__device__ __forceinline__ float dequant(long long acc, float sc, float bias, bool has_res,
+                                         int res_q, float res_scale, bool relu) {
+  float a = __ll2float_rn(acc);
+  float y = __fmaf_rn(a, sc, bias);
+  if (has_res) y = __fmaf_rn((float)res_q, res_scale, y);
+  if (relu) y = fmaxf(y, 0.0f);
+  return y;
+}
+
+__device__ __forceinline__ int requant(float y, float inv_step, int qmin, int qmax) {
+  float t = __fmul_rn(y, inv_step);
+  float r = rintf(t);
+  r = fmaxf(r, (float)qmin);
+  r = fminf(r, (float)qmax);
+  return (int)r;
+}
+
+// host-side launchers (defined in the .cu files)
+cudaError_t launch_sampler(const float* w_dev, psb_weights* wt, uint32_t* err_dev, cudaStream_t s);
+cudaError_t launch_export(const psb_weights* wt, uint32_t level, int32_t* wint_out,
+                          int32_t* e_base_out, cudaStream_t s);
+cudaError_t launch_shift_add(const ConvArgs& a, const WintTable& wt, cudaStream_t s);
+cudaError_t launch_nchw_to_nhwc(const void* src, void* dst, uint32_t N, uint32_t C, uint32_t HW,
+                                uint32_t elem_bytes, cudaStream_t s);
+cudaError_t launch_nhwc_to_nchw(const void* src, void* dst, uint32_t N, uint32_t C, uint32_t HW,
+                                uint32_t elem_bytes, cudaStream_t s);
+cudaError_t launch_maxpool(const uint8_t* x, uint32_t nchw, uint32_t N, uint32_t C, uint32_t H,
+                           uint32_t W, uint32_t k, uint32_t stride, uint32_t pad, uint8_t* out,
+                           cudaStream_t s);
+cudaError_t launch_avgpool(const uint8_t* x, uint32_t nchw, uint32_t N, uint32_t C, uint32_t H,
+                           uint32_t W, float pool_mul, int32_t qmin, int32_t qmax, uint8_t* out,
+                           cudaStream_t s);
+// tensor path: returns PSB_ERR_UNSUPPORTED if the shape does not fit it
+psb_status tensor_supported(const psb_ctx* ctx, const psb_weights* wt, const ConvArgs& a);
+psb_status launch_tensor(psb_ctx* ctx, const psb_weights* wt, const ConvArgs& a, cudaStream_t s);
+
+}  // namespace psb

@@ -1,0 +1,245 @@
+// Weight sampler: turns an fp32 filter into exact integer filters, one per
+// requested draw count k (paper Eq. 4-8).  Per weight:
+//   decode (s, e, p) from the IEEE-754 fields          Eq. 5-7
+//   window the exponent against the group's maximum    (4-bit exponents, Sec. 4.4)
+//   draw k Bernoulli(p) bits from Philox4x32-10         the comparator of the
+//                                                       stochastic multiplier
+//   count the upper draws among the first k, every k    Eq. 8 (binomial count)
+//   emit W_k = s (k + c_k) 2^(e - e_base) as int32 and as signed 7-bit digit
+//   planes in the layout the tensor path loads with TMA.
+// The random bits never leave registers.
+#include "psb_common.cuh"
+
+namespace psb {
+
+namespace {
+
+constexpr int kThreads = 256;
+constexpr int kStage = 2048;  // weights staged in shared memory per block
+
+// Philox4x32-10 (Salmon et al., SC'11): ten rounds of two 32x32->64 multiplies and
+// xors; the key advances by the two Weyl constants after every round.
+__device__ __forceinline__ void philox4x32_10(uint32_t c0, uint32_t c1, uint32_t c2, uint32_t c3,
+                                              uint32_t k0, uint32_t k1, uint32_t (&out)[4]) {
+  const uint32_t M0 = 0xD2511F53u, M1 = 0xCD9E8D57u;
+#pragma unroll
+  for (int r = 0; r < 10; ++r) {
+    uint32_t hi0 = __umulhi(M0, c0), lo0 = M0 * c0;
+    uint32_t hi1 = __umulhi(M1, c2), lo1 = M1 * c2;
+    uint32_t n0 = hi1 ^ c1 ^ k0;
+    uint32_t n2 = hi0 ^ c3 ^ k1;
+    c0 = n0; c1 = lo1; c2 = n2; c3 = lo0;
+    k0 += 0x9E3779B9u;
+    k1 += 0xBB67AE85u;
+  }
+  out[0] = c0; out[1] = c1; out[2] = c2; out[3] = c3;
+}
+
+// Largest biased exponent of each exponent group; flags Inf/NaN.
+// norm == 1: one block per output channel.  norm == 0: grid-stride over the layer.
+__global__ void emax_kernel(const float* __restrict__ w, uint32_t O, uint32_t d, uint32_t norm,
+                            uint32_t* __restrict__ e_max, uint32_t* __restrict__ err) {
+  __shared__ uint32_t red[kThreads / 32];
+  uint32_t best = 0;
+  bool bad = false;
+  if (norm) {
+    const float* row = w + (size_t)blockIdx.x * d;
+    for (uint32_t i = threadIdx.x; i < d; i += blockDim.x) {
+      uint32_t E = (__float_as_uint(row[i]) >> 23) & 0xFFu;
+      bad |= (E == 255u);
+      best = max(best, E);
+    }
+  } else {
+    size_t total = (size_t)O * d;
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < total;
+         i += (size_t)gridDim.x * blockDim.x) {
+      uint32_t E = (__float_as_uint(w[i]) >> 23) & 0xFFu;
+      bad |= (E == 255u);
+      best = max(best, E);
+    }
+  }
+  if (__any_sync(0xFFFFFFFFu, bad) && (threadIdx.x & 31) == 0) atomicOr(err, kDevErrNonFinite);
+  best = __reduce_max_sync(0xFFFFFFFFu, best);
+  if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = best;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    for (int i = 1; i < kThreads / 32; ++i) best = max(best, red[i]);
+    if (best == 255u) best = 0;  // error already flagged; keep the window well defined
+    if (norm) e_max[blockIdx.x] = best;
+    else if (best) atomicMax(&e_max[0], best);
+  }
+}
+
+struct SampleParams {
+  const float* w;
+  uint32_t O, Cg, KHKW, d;
+  uint32_t rows_per_block, ch_per_block, ch_chunks;
+  uint32_t norm, span, level_mask, max_level;
+  uint32_t seed_lo, seed_hi, layer_id;
+  uint32_t cpad, kpad, has_planes;
+  const uint32_t* e_max;
+  int32_t* e_base;
+  int32_t* wint[kMaxLevels];
+  int8_t* planes[kMaxLevels];
+  int planes_count[kMaxLevels];
+};
+
+__global__ void __launch_bounds__(kThreads) sample_kernel(const SampleParams p) {
+  __shared__ float stage[kStage];
+  const uint32_t row_block = blockIdx.x / p.ch_chunks;
+  const uint32_t chunk = blockIdx.x % p.ch_chunks;
+  const uint32_t o0 = row_block * p.rows_per_block;
+  const uint32_t c0 = chunk * p.ch_per_block;
+  const uint32_t rows = min(p.rows_per_block, p.O - o0);
+  const uint32_t cc = min(p.ch_per_block, p.Cg - c0);
+  const uint32_t per_row = cc * p.KHKW;     // canonical elements of one row in this block
+  const uint32_t count = rows * per_row;
+
+  // stage the canonical (channel-major) slice with coalesced loads
+  for (uint32_t t = threadIdx.x; t < count; t += blockDim.x) {
+    uint32_t r = t / per_row, rem = t % per_row;
+    stage[t] = p.w[(size_t)(o0 + r) * p.d + (size_t)c0 * p.KHKW + rem];
+  }
+  __syncthreads();
+
+  // walk the slice in output order (row, tap, channel) so that stores coalesce
+  for (uint32_t t = threadIdx.x; t < count; t += blockDim.x) {
+    const uint32_t r = t / per_row, rem = t % per_row;
+    const uint32_t tap = rem / cc, cl = rem % cc;
+    const uint32_t o = o0 + r, ci = c0 + cl;
+    const uint32_t u = __float_as_uint(stage[r * per_row + cl * p.KHKW + tap]);
+    const uint64_t index = (uint64_t)o * p.d + (uint64_t)ci * p.KHKW + tap;  // canonical
+
+    const uint32_t E = (u >> 23) & 0xFFu;
+    const uint32_t m = u & 0x7FFFFFu;
+    const uint32_t Emax = p.e_max[p.norm ? o : 0];
+    // biased exponents throughout: e - e_base = E - (Emax - span)
+    const int ebase_biased = (int)Emax - (int)p.span;
+    if (tap == 0 && ci == 0) p.e_base[o] = Emax ? ebase_biased - 127 : 0;
+    const bool live = (E != 0u) && (E != 255u) && ((int)E >= ebase_biased);
+    const uint32_t sh = live ? (uint32_t)((int)E - ebase_biased) : 0u;
+    const bool neg = (u >> 31) != 0u;
+
+    // c_k for every level, packed 7 bits per level
+    unsigned long long packed = 0ull;
+    if (live && m != 0u) {
+      const uint32_t T = m << 9;
+      const uint32_t kmax = 1u << p.max_level;
+      uint32_t c = 0, j = 0;
+      for (uint32_t q = 0; q * 4u < kmax; ++q) {
+        uint32_t rnd[4];
+        philox4x32_10(q, p.layer_id, (uint32_t)index, (uint32_t)(index >> 32), p.seed_lo, p.seed_hi,
+                      rnd);
+#pragma unroll
+        for (int v = 0; v < 4; ++v) {
+          if (j < kmax) {
+            c += (rnd[v] < T) ? 1u : 0u;
+            ++j;
+            if ((j & (j - 1u)) == 0u) packed |= (unsigned long long)c << (7 * (31 - __clz(j)));
+          }
+        }
+      }
+    }
+
+    const size_t wpos = ((size_t)o * p.KHKW + tap) * p.Cg + ci;
+    const uint32_t jt = o / kTileN, on = o % kTileN;
+    for (uint32_t l = 0; l <= p.max_level; ++l) {
+      if (!((p.level_mask >> l) & 1u)) continue;
+      const uint32_t c = (uint32_t)(packed >> (7 * l)) & 0x7Fu;
+      const uint32_t mag = live ? (((1u << l) + c) << sh) : 0u;
+      p.wint[l][wpos] = neg ? -(int32_t)mag : (int32_t)mag;
+      if (p.has_planes) {
+        const int P = p.planes_count[l];
+        for (int pl = 0; pl < P; ++pl) {
+          int digit = (int)((mag >> (kDigitBits * pl)) & 0x7Fu);
+          p.planes[l][(((size_t)jt * P + pl) * kTileN + on) * p.kpad + (size_t)tap * p.cpad + ci] =
+              (int8_t)(neg ? -digit : digit);
+        }
+      }
+    }
+  }
+}
+
+// Canonical-order copy of one level for the test hook.
+__global__ void export_kernel(const int32_t* __restrict__ wint, int32_t* __restrict__ out, uint32_t O,
+                              uint32_t Cg, uint32_t KHKW) {
+  size_t total = (size_t)O * Cg * KHKW;
+  for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < total;
+       i += (size_t)gridDim.x * blockDim.x) {
+    uint32_t tap = (uint32_t)(i % KHKW);
+    size_t t = i / KHKW;
+    uint32_t ci = (uint32_t)(t % Cg);
+    size_t o = t / Cg;
+    out[i] = wint[(o * KHKW + tap) * Cg + ci];
+  }
+}
+
+}  // namespace
+
+cudaError_t launch_sampler(const float* w_dev, psb_weights* wt, uint32_t* err_dev, cudaStream_t s) {
+  const psb_wshape& sh = wt->shape;
+  const uint32_t O = sh.out_ch, Cg = sh.in_ch_per_group, KHKW = sh.kh * sh.kw, d = wt->d;
+  const uint32_t norm = wt->cfg.norm;
+  cudaError_t e = cudaMemsetAsync(wt->e_max, 0, sizeof(uint32_t) * O, s);
+  if (e != cudaSuccess) return e;
+  if (norm) {
+    emax_kernel<<<O, kThreads, 0, s>>>(w_dev, O, d, 1, wt->e_max, err_dev);
+  } else {
+    size_t total = (size_t)O * d;
+    uint32_t blocks = (uint32_t)((total + kThreads * 8 - 1) / (kThreads * 8));
+    blocks = blocks < 1 ? 1 : (blocks > 1184 ? 1184 : blocks);
+    emax_kernel<<<blocks, kThreads, 0, s>>>(w_dev, O, d, 0, wt->e_max, err_dev);
+  }
+  SampleParams p;
+  p.w = w_dev;
+  p.O = O; p.Cg = Cg; p.KHKW = KHKW; p.d = d;
+  if (d <= (uint32_t)kStage) {
+    p.rows_per_block = kStage / d;
+    p.ch_per_block = Cg;
+    p.ch_chunks = 1;
+  } else {
+    p.rows_per_block = 1;
+    p.ch_per_block = kStage / KHKW;
+    p.ch_chunks = (Cg + p.ch_per_block - 1) / p.ch_per_block;
+  }
+  p.norm = norm;
+  p.span = (1u << wt->cfg.exp_bits) - 1u;
+  p.level_mask = wt->cfg.level_mask;
+  p.max_level = 0;
+  for (uint32_t l = 0; l < (uint32_t)kMaxLevels; ++l)
+    if ((p.level_mask >> l) & 1u) p.max_level = l;
+  p.seed_lo = (uint32_t)wt->cfg.seed;
+  p.seed_hi = (uint32_t)(wt->cfg.seed >> 32);
+  p.layer_id = wt->cfg.layer_id;
+  p.cpad = wt->cpad; p.kpad = wt->kpad; p.has_planes = wt->has_planes ? 1u : 0u;
+  p.e_max = wt->e_max;
+  p.e_base = wt->e_base;
+  for (int l = 0; l < kMaxLevels; ++l) {
+    p.wint[l] = wt->level[l].wint;
+    p.planes[l] = wt->level[l].planes;
+    p.planes_count[l] = wt->level[l].planes_count;
+  }
+  uint32_t row_blocks = (O + p.rows_per_block - 1) / p.rows_per_block;
+  sample_kernel<<<row_blocks * p.ch_chunks, kThreads, 0, s>>>(p);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_export(const psb_weights* wt, uint32_t level, int32_t* wint_out,
+                          int32_t* e_base_out, cudaStream_t s) {
+  const psb_wshape& sh = wt->shape;
+  if (wint_out) {
+    size_t total = (size_t)sh.out_ch * wt->d;
+    uint32_t blocks = (uint32_t)((total + 255) / 256);
+    blocks = blocks > 4096 ? 4096 : (blocks < 1 ? 1 : blocks);
+    export_kernel<<<blocks, 256, 0, s>>>(wt->level[level].wint, wint_out, sh.out_ch,
+                                        sh.in_ch_per_group, sh.kh * sh.kw);
+  }
+  if (e_base_out) {
+    cudaError_t e = cudaMemcpyAsync(e_base_out, wt->e_base, sizeof(int32_t) * sh.out_ch,
+                                    cudaMemcpyDeviceToDevice, s);
+    if (e != cudaSuccess) return e;
+  }
+  return cudaGetLastError();
+}
+
+}  // namespace psb

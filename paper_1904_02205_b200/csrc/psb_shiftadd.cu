@@ -1,0 +1,179 @@
+// CUDA-core contraction ("shift-add" path) and the glue kernels.
+//
+// The paper's capacitor unit adds x << (e + B) over the draws (Eq. 9); summed over
+// the k draws that is x * (k + c_k) << (e - e_base), an integer product with the
+// sampled integer weight.  On the GPU one 64-bit integer multiply-add per
+// (activation, weight) pair realises exactly that sum.  This path serves layers
+// that are not dense matrix products for the tensor cores: depthwise filters,
+// fully connected layers at small batch, very few input channels, 8-bit unsigned
+// activations, and it honours per-location draw counts directly.
+#include "psb_common.cuh"
+
+namespace psb {
+
+namespace {
+
+__device__ __forceinline__ int load_act(const void* x, uint32_t dtype, size_t idx) {
+  return dtype == PSB_DT_U8 ? (int)((const uint8_t*)x)[idx] : (int)((const int8_t*)x)[idx];
+}
+
+__device__ __forceinline__ void store_outputs(const ConvArgs& a, size_t oidx, uint32_t o,
+                                              uint32_t level, long long acc) {
+  if (a.acc_out) a.acc_out[oidx] = acc;
+  if (a.q_out || a.f32_out) {
+    float sc = ldexpf(a.scale[o], a.e_base[o] - (int)level);
+    int rq = a.residual ? load_act(a.residual, a.residual_dtype, oidx) : 0;
+    float y = dequant(acc, sc, a.bias[o], a.residual != nullptr, rq, a.residual_scale, a.relu != 0);
+    if (a.f32_out) a.f32_out[oidx] = y;
+    if (a.q_out) {
+      int q = requant(y, a.inv_step, a.qmin, a.qmax);
+      if (a.out_dtype == PSB_DT_U8) ((uint8_t*)a.q_out)[oidx] = (uint8_t)q;
+      else ((int8_t*)a.q_out)[oidx] = (int8_t)q;
+    }
+  }
+}
+
+// One thread per output element, output channel fastest.  For depthwise filters
+// (one input channel per group) neighbouring threads read neighbouring bytes.
+__global__ void __launch_bounds__(256) conv_direct_kernel(const ConvArgs a, const WintTable wt) {
+  const size_t total = (size_t)a.N * a.OH * a.OW * a.O;
+  const uint32_t Cg = a.C / a.groups, Og = a.O / a.groups;
+  for (size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x; idx < total;
+       idx += (size_t)gridDim.x * blockDim.x) {
+    const uint32_t o = (uint32_t)(idx % a.O);
+    const size_t pix = idx / a.O;
+    const uint32_t ox = (uint32_t)(pix % a.OW);
+    const uint32_t oy = (uint32_t)((pix / a.OW) % a.OH);
+    const uint32_t n = (uint32_t)(pix / ((size_t)a.OW * a.OH));
+    const uint32_t level = a.kmap ? a.kmap[pix] : a.uniform_log2k;
+    if (level >= (uint32_t)kMaxLevels || !((a.level_mask >> level) & 1u)) {
+      atomicOr(a.err, kDevErrBadLevel);
+      continue;
+    }
+    const int32_t* __restrict__ w = wt.w[level] + (size_t)o * a.KH * a.KW * Cg;
+    const uint32_t cbase = (o / Og) * Cg;
+    long long acc = 0;
+    for (uint32_t kh = 0; kh < a.KH; ++kh) {
+      const int iy = (int)(oy * a.stride + kh) - (int)a.pad;
+      if (iy < 0 || iy >= (int)a.H) continue;
+      for (uint32_t kw = 0; kw < a.KW; ++kw) {
+        const int ix = (int)(ox * a.stride + kw) - (int)a.pad;
+        if (ix < 0 || ix >= (int)a.W) continue;
+        const size_t xoff = (((size_t)n * a.H + iy) * a.W + ix) * a.C + cbase;
+        const int32_t* wr = w + (size_t)(kh * a.KW + kw) * Cg;
+        for (uint32_t ci = 0; ci < Cg; ++ci) {
+          int xv = load_act(a.x, a.in_dtype, xoff + ci);
+          acc += (long long)xv * (long long)__ldg(wr + ci);
+        }
+      }
+    }
+    const size_t oidx = a.out_nchw ? (((size_t)n * a.O + o) * a.OH + oy) * a.OW + ox : idx;
+    store_outputs(a, oidx, o, level, acc);
+  }
+}
+
+// [N][C][HW] -> [N][HW][C], elements of 1 byte, through a 32x33 tile.
+__global__ void nchw_to_nhwc_u8_kernel(const uint8_t* __restrict__ src, uint8_t* __restrict__ dst,
+                                       uint32_t C, uint32_t HW) {
+  __shared__ uint8_t tile[32][33];
+  const size_t base = (size_t)blockIdx.z * C * HW;
+  const uint32_t p0 = blockIdx.x * 32, c0 = blockIdx.y * 32;
+  for (uint32_t r = threadIdx.y; r < 32; r += blockDim.y) {
+    uint32_t c = c0 + r, p = p0 + threadIdx.x;
+    if (c < C && p < HW) tile[r][threadIdx.x] = src[base + (size_t)c * HW + p];
+  }
+  __syncthreads();
+  for (uint32_t r = threadIdx.y; r < 32; r += blockDim.y) {
+    uint32_t p = p0 + r, c = c0 + threadIdx.x;
+    if (c < C && p < HW) dst[base + (size_t)p * C + c] = tile[threadIdx.x][r];
+  }
+}
+
+__global__ void maxpool_kernel(const uint8_t* __restrict__ x, uint32_t nchw, uint32_t N, uint32_t C,
+                               uint32_t H, uint32_t W, uint32_t k, uint32_t stride, uint32_t pad,
+                               uint32_t OH, uint32_t OW, uint8_t* __restrict__ out) {
+  const size_t total = (size_t)N * OH * OW * C;
+  for (size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x; idx < total;
+       idx += (size_t)gridDim.x * blockDim.x) {
+    uint32_t c, ox, oy, n;
+    if (nchw) {
+      ox = idx % OW; oy = (idx / OW) % OH; c = (idx / ((size_t)OW * OH)) % C;
+      n = idx / ((size_t)OW * OH * C);
+    } else {
+      c = idx % C; ox = (idx / C) % OW; oy = (idx / ((size_t)C * OW)) % OH;
+      n = idx / ((size_t)C * OW * OH);
+    }
+    int best = 0;
+    for (uint32_t kh = 0; kh < k; ++kh) {
+      int iy = (int)(oy * stride + kh) - (int)pad;
+      if (iy < 0 || iy >= (int)H) continue;
+      for (uint32_t kw = 0; kw < k; ++kw) {
+        int ix = (int)(ox * stride + kw) - (int)pad;
+        if (ix < 0 || ix >= (int)W) continue;
+        size_t xi = nchw ? (((size_t)n * C + c) * H + iy) * W + ix
+                         : (((size_t)n * H + iy) * W + ix) * C + c;
+        best = max(best, (int)x[xi]);
+      }
+    }
+    out[idx] = (uint8_t)best;
+  }
+}
+
+// One warp per (n, c): integer sum over H*W, then one re-quantisation.
+__global__ void avgpool_kernel(const uint8_t* __restrict__ x, uint32_t nchw, uint32_t N, uint32_t C,
+                               uint32_t HW, float pool_mul, int qmin, int qmax,
+                               uint8_t* __restrict__ out) {
+  const uint32_t warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
+  if (warp >= N * C) return;
+  const uint32_t n = warp / C, c = warp % C;
+  int sum = 0;
+  for (uint32_t p = lane; p < HW; p += 32) {
+    size_t xi = nchw ? ((size_t)n * C + c) * HW + p : ((size_t)n * HW + p) * C + c;
+    sum += x[xi];
+  }
+  sum = __reduce_add_sync(0xFFFFFFFFu, sum);
+  if (lane == 0) out[warp] = (uint8_t)requant((float)sum, pool_mul, qmin, qmax);
+}
+
+uint32_t grid_for(size_t total, uint32_t threads) {
+  size_t b = (total + threads - 1) / threads;
+  if (b < 1) b = 1;
+  if (b > 148u * 32u) b = 148u * 32u;
+  return (uint32_t)b;
+}
+
+}  // namespace
+
+cudaError_t launch_shift_add(const ConvArgs& a, const WintTable& wt, cudaStream_t s) {
+  size_t total = (size_t)a.N * a.OH * a.OW * a.O;
+  conv_direct_kernel<<<grid_for(total, 256), 256, 0, s>>>(a, wt);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_nchw_to_nhwc(const void* src, void* dst, uint32_t N, uint32_t C, uint32_t HW,
+                                uint32_t elem_bytes, cudaStream_t s) {
+  if (elem_bytes != 1) return cudaErrorInvalidValue;
+  dim3 grid((HW + 31) / 32, (C + 31) / 32, N), block(32, 8);
+  nchw_to_nhwc_u8_kernel<<<grid, block, 0, s>>>((const uint8_t*)src, (uint8_t*)dst, C, HW);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_maxpool(const uint8_t* x, uint32_t nchw, uint32_t N, uint32_t C, uint32_t H,
+                           uint32_t W, uint32_t k, uint32_t stride, uint32_t pad, uint8_t* out,
+                           cudaStream_t s) {
+  uint32_t OH = (H + 2 * pad - k) / stride + 1, OW = (W + 2 * pad - k) / stride + 1;
+  size_t total = (size_t)N * OH * OW * C;
+  maxpool_kernel<<<grid_for(total, 256), 256, 0, s>>>(x, nchw, N, C, H, W, k, stride, pad, OH, OW, out);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_avgpool(const uint8_t* x, uint32_t nchw, uint32_t N, uint32_t C, uint32_t H,
+                           uint32_t W, float pool_mul, int32_t qmin, int32_t qmax, uint8_t* out,
+                           cudaStream_t s) {
+  size_t warps = (size_t)N * C;
+  uint32_t blocks = (uint32_t)((warps * 32 + 255) / 256);
+  avgpool_kernel<<<blocks, 256, 0, s>>>(x, nchw, N, C, H * W, pool_mul, qmin, qmax, out);
+  return cudaGetLastError();
+}
+
+}  // namespace psb

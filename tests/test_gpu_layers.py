@@ -1,0 +1,308 @@
+"""GPU parity: CUDA library (through the C ABI) against the CPU oracle, element by element.
+
+Bit-exact on integer filters, base exponents, 64-bit accumulators and re-quantised
+activations; 1e-6 relative on fp32 outputs.
+"""
+import numpy as np
+import pytest
+
+from psb_testlib import compare, gpu_layer, oracle_layer
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def psb():
+    import paper_1904_02205_b200 as p
+
+    return p
+
+
+@pytest.fixture(scope="module")
+def ctx(psb):
+    c = psb.Context(0)
+    yield c
+    c.close()
+
+
+def _layer_inputs(rng, N, C, H, W, O, KH, KW, groups, layout, x_dtype=np.uint8, x_hi=16, w_sigma=None):
+    d = (C // groups) * KH * KW
+    sigma = np.sqrt(2.0 / d) if w_sigma is None else w_sigma
+    w = rng.normal(0, sigma, size=(O, C // groups, KH, KW)).astype(np.float32)
+    lo = 0 if x_dtype == np.uint8 else -x_hi
+    shape = (N, C, H, W) if layout == 0 else (N, H, W, C)
+    x = rng.integers(lo, x_hi, size=shape).astype(x_dtype)
+    scale = rng.uniform(0.5, 1.5, O).astype(np.float32)
+    bias = rng.normal(0, 0.5, O).astype(np.float32)
+    return w, x, scale, bias
+
+
+def _both(psb, ctx, oracle, w, x, layout, groups, stride, pad, levels, scale, bias, kmap=None,
+          uniform=None, relu=True, inv_step=0.5, qmin=0, qmax=15, out_dtype=0, residual=None,
+          res_scale=0.0, exp_bits=4, norm=0, in_max=0, path=0, seed=5, layer_id=3):
+    uniform = levels[0] if uniform is None else uniform
+    o = oracle_layer(oracle, w, x, layout, groups, stride, pad, seed, layer_id, levels, kmap, uniform,
+                     scale, bias, relu, np.float32(inv_step), qmin, qmax, residual, np.float32(res_scale),
+                     exp_bits, norm)
+    g = gpu_layer(psb, ctx, w, x, layout, groups, stride, pad, seed, layer_id, levels, kmap, uniform,
+                  scale, bias, relu, np.float32(inv_step), qmin, qmax, out_dtype, residual,
+                  np.float32(res_scale), exp_bits, norm, in_max, path)
+    compare(g, o, levels)
+    return g
+
+
+# ------------------------------------------------------------------------ sampler
+
+@pytest.mark.parametrize("shape,groups", [((128, 256, 1, 1), 1), ((64, 64, 3, 3), 1), ((96, 1, 3, 3), 96),
+                                           ((16, 3, 7, 7), 1), ((5, 512, 3, 3), 1), ((1000, 40, 1, 1), 1),
+                                           ((3, 2100, 1, 1), 1)])
+@pytest.mark.parametrize("norm", [0, 1])
+def test_sampler_all_levels(psb, ctx, oracle, shape, groups, norm):
+    import torch
+
+    rng = np.random.default_rng(abs(hash((shape, norm))) % 2 ** 31)
+    w = rng.normal(0, 0.1, size=shape).astype(np.float32)
+    flat = w.reshape(-1)
+    flat[rng.random(flat.size) < 0.05] = 0.0
+    flat[:4] = [0.5, -0.25, 1e-41, 3e-9]          # exact powers of two, a sub-normal, a flushed one
+    for exp_bits in (4, 2):
+        wt = ctx.sample_weights(torch.from_numpy(w).cuda(), groups=groups, seed=2 ** 40 + 17, layer_id=9,
+                                level_mask=0x7F, exp_bits=exp_bits, norm=norm)
+        for l in range(7):
+            Wg, ebg = (v.cpu().numpy() for v in ctx.weights_export(wt, l))
+            Wo, ebo, _ = oracle.sample_level(w, 2 ** 40 + 17, 9, l, exp_bits=exp_bits, norm=norm)
+            assert np.array_equal(ebg, ebo)
+            assert np.array_equal(Wg.astype(np.int64), Wo), (shape, norm, exp_bits, l)
+        assert ctx.device_status() == 0
+        wt.free()
+
+
+def test_resampling_in_place_changes_with_the_seed_only(psb, ctx, oracle):
+    import torch
+
+    rng = np.random.default_rng(1)
+    w = rng.normal(0, 0.1, size=(32, 32, 3, 3)).astype(np.float32)
+    wd = torch.from_numpy(w).cuda()
+    wt = ctx.sample_weights(wd, seed=1, layer_id=0, level_mask=0b1000)
+    a = ctx.weights_export(wt, 3)[0].cpu().numpy()
+    ctx.sample_weights(wd, seed=2, layer_id=0, level_mask=0b1000, into=wt)
+    b = ctx.weights_export(wt, 3)[0].cpu().numpy()
+    ctx.sample_weights(wd, seed=1, layer_id=0, level_mask=0b1000, into=wt)
+    c = ctx.weights_export(wt, 3)[0].cpu().numpy()
+    assert np.array_equal(a, c) and not np.array_equal(a, b)
+    assert np.array_equal(b.astype(np.int64), oracle.sample_level(w, 2, 0, 3)[0])
+    with pytest.raises(psb.PsbError):
+        ctx.sample_weights(wd, seed=1, layer_id=0, level_mask=0b0100, into=wt)
+    wt.free()
+
+
+# ------------------------------------------------------------------ shift-add path
+
+def test_config1_fully_connected(psb, ctx, oracle):
+    from workloads import config1_fc
+
+    c = config1_fc()
+    x = c["x"].reshape(16, 1, 1, 256)
+    _both(psb, ctx, oracle, c["w"], x, 1, 1, 1, 0, [c["log2k"]], c["scale"], c["bias"], relu=True,
+          inv_step=c["inv_step"], qmin=0, qmax=255, seed=c["seed"], layer_id=0, path=psb.PSB_PATH_SHIFT_ADD)
+
+
+@pytest.mark.parametrize("case", [
+    dict(N=2, C=8, H=9, W=7, O=12, K=3, groups=1, stride=1, pad=1, layout=1),
+    dict(N=1, C=12, H=10, W=10, O=8, K=3, groups=4, stride=2, pad=1, layout=0),
+    dict(N=3, C=40, H=13, W=11, O=40, K=3, groups=40, stride=1, pad=1, layout=1),
+    dict(N=2, C=40, H=13, W=11, O=40, K=3, groups=40, stride=2, pad=1, layout=0),
+    dict(N=2, C=3, H=21, W=21, O=10, K=7, groups=1, stride=2, pad=3, layout=1),
+    dict(N=2, C=20, H=5, W=6, O=7, K=1, groups=1, stride=1, pad=0, layout=0),
+])
+def test_shift_add_convolutions(psb, ctx, oracle, case):
+    rng = np.random.default_rng(case["C"] * 31 + case["K"])
+    w, x, scale, bias = _layer_inputs(rng, case["N"], case["C"], case["H"], case["W"], case["O"], case["K"],
+                                      case["K"], case["groups"], case["layout"], x_hi=256)
+    g = _both(psb, ctx, oracle, w, x, case["layout"], case["groups"], case["stride"], case["pad"], [4],
+              scale, bias, inv_step=0.02, qmax=255, path=psb.PSB_PATH_SHIFT_ADD)
+    assert g["path"] == psb.PSB_PATH_SHIFT_ADD
+
+
+def test_shift_add_signed_input_residual_and_map(psb, ctx, oracle):
+    rng = np.random.default_rng(77)
+    w, x, scale, bias = _layer_inputs(rng, 2, 16, 8, 8, 24, 3, 3, 1, 1, x_dtype=np.int8, x_hi=128)
+    res = rng.integers(-128, 128, size=(2, 8, 8, 24)).astype(np.int8)
+    kmap = rng.choice([0, 1, 3, 6], size=(2, 8, 8)).astype(np.uint8)
+    _both(psb, ctx, oracle, w, x, 1, 1, 1, 1, [0, 1, 3, 6], scale, bias, kmap=kmap, relu=False, inv_step=0.01,
+          qmin=-128, qmax=127, out_dtype=1, residual=res, res_scale=0.07, path=psb.PSB_PATH_SHIFT_ADD)
+
+
+# --------------------------------------------------------------------- tensor path
+
+@pytest.mark.parametrize("case", [
+    dict(N=2, C=64, H=9, W=15, O=64, K=1, stride=1, pad=0),      # plain GEMM, ragged last tile
+    dict(N=1, C=256, H=12, W=12, O=128, K=1, stride=1, pad=0),   # 128-byte K block, two channel tiles
+    dict(N=3, C=96, H=7, W=9, O=24, K=1, stride=1, pad=0),       # partial K block, ragged channels
+    dict(N=2, C=32, H=10, W=10, O=80, K=1, stride=1, pad=0),     # 32-byte K block
+    dict(N=2, C=64, H=14, W=14, O=64, K=3, stride=1, pad=1),     # 3x3 through the im2col loader
+    dict(N=3, C=64, H=15, W=13, O=64, K=3, stride=2, pad=1),     # strided 3x3, odd sizes
+    dict(N=2, C=128, H=14, W=14, O=256, K=1, stride=2, pad=0),   # strided projection
+    dict(N=2, C=32, H=20, W=20, O=16, K=7, stride=2, pad=3),     # 7x7
+    dict(N=1, C=160, H=9, W=9, O=64, K=3, stride=1, pad=1),      # 160 channels: K blocks 128 + 32
+])
+def test_tensor_path_layers(psb, ctx, oracle, case):
+    rng = np.random.default_rng(case["C"] * 131 + case["K"] * 7 + case["stride"])
+    w, x, scale, bias = _layer_inputs(rng, case["N"], case["C"], case["H"], case["W"], case["O"], case["K"],
+                                      case["K"], 1, 1)
+    g = _both(psb, ctx, oracle, w, x, 1, 1, case["stride"], case["pad"], [3], scale, bias, inv_step=0.6,
+              in_max=15, path=psb.PSB_PATH_TENSOR)
+    assert g["path"] == psb.PSB_PATH_TENSOR
+
+
+@pytest.mark.parametrize("log2k", [0, 1, 2, 4, 5, 6])
+def test_tensor_path_every_draw_count(psb, ctx, oracle, log2k):
+    rng = np.random.default_rng(log2k)
+    w, x, scale, bias = _layer_inputs(rng, 2, 64, 12, 12, 64, 3, 3, 1, 1)
+    _both(psb, ctx, oracle, w, x, 1, 1, 1, 1, [log2k], scale, bias, inv_step=0.6, in_max=15,
+          path=psb.PSB_PATH_TENSOR)
+
+
+def test_tensor_path_per_location_draw_counts(psb, ctx, oracle):
+    rng = np.random.default_rng(21)
+    w, x, scale, bias = _layer_inputs(rng, 2, 64, 16, 16, 64, 3, 3, 1, 1)
+    kmap = np.zeros((2, 16, 16), dtype=np.uint8)
+    kmap[0, :8] = 3                       # tiles with a single level
+    kmap[0, 8:] = rng.choice([0, 1, 2, 3, 4], size=(8, 16))   # mixed tiles
+    kmap[1] = rng.choice([2, 4], size=(16, 16))
+    _both(psb, ctx, oracle, w, x, 1, 1, 1, 1, [0, 1, 2, 3, 4], scale, bias, kmap=kmap, inv_step=0.6, in_max=15,
+          path=psb.PSB_PATH_TENSOR)
+
+
+def test_tensor_path_signed_inputs_residual_nchw_and_exponent_options(psb, ctx, oracle):
+    rng = np.random.default_rng(22)
+    w, x, scale, bias = _layer_inputs(rng, 2, 64, 10, 10, 32, 3, 3, 1, 0, x_dtype=np.int8, x_hi=128)
+    res = rng.integers(0, 256, size=(2, 32, 10, 10)).astype(np.uint8)
+    _both(psb, ctx, oracle, w, x, 0, 1, 1, 1, [3], scale, bias, relu=False, inv_step=0.05, qmin=-128, qmax=127,
+          out_dtype=1, residual=res, res_scale=0.3, norm=1, path=psb.PSB_PATH_TENSOR)
+    w, x, scale, bias = _layer_inputs(rng, 2, 64, 10, 10, 32, 3, 3, 1, 1)
+    res = rng.integers(-128, 128, size=(2, 10, 10, 32)).astype(np.int8)
+    _both(psb, ctx, oracle, w, x, 1, 1, 1, 1, [3], scale, bias, inv_step=0.5, residual=res, res_scale=0.3,
+          exp_bits=3, in_max=15, path=psb.PSB_PATH_TENSOR)
+
+
+def test_auto_path_selection(psb, ctx, oracle):
+    rng = np.random.default_rng(23)
+    w, x, scale, bias = _layer_inputs(rng, 2, 64, 12, 12, 64, 3, 3, 1, 1)
+    g = _both(psb, ctx, oracle, w, x, 1, 1, 1, 1, [3], scale, bias, in_max=15)
+    assert g["path"] == psb.PSB_PATH_TENSOR
+    g = _both(psb, ctx, oracle, w, x, 1, 1, 1, 1, [3], scale, bias)          # full-range u8: CUDA cores
+    assert g["path"] == psb.PSB_PATH_SHIFT_ADD
+    w, x, scale, bias = _layer_inputs(rng, 2, 48, 12, 12, 48, 3, 3, 48, 1)
+    g = _both(psb, ctx, oracle, w, x, 1, 48, 1, 1, [3], scale, bias, in_max=15)
+    assert g["path"] == psb.PSB_PATH_SHIFT_ADD
+
+
+# ----------------------------------------------------- config 2 at its full size
+
+@pytest.mark.parametrize("log2k", [0, 3])
+def test_config2_full_size_sampled_outputs(psb, ctx, oracle, log2k):
+    """The 3x3 64->64 conv on 56x56, batch 32, NCHW, as the benchmark launches it: accumulators at
+    4000 sampled outputs against the oracle, all image borders included, plus whole-tensor properties."""
+    import torch
+    from workloads import config2_conv
+
+    c = config2_conv()
+    dev = ctx.device
+    wt = ctx.sample_weights(torch.from_numpy(c["w"]).to(dev), seed=c["seed"], layer_id=0, level_mask=1 << log2k)
+    ctx.set_sample_map(None, log2k)
+    out = ctx.conv2d(wt, torch.from_numpy(c["x"]).to(dev), psb.PSB_LAYOUT_NCHW, 1, 1,
+                     torch.from_numpy(c["scale"]).to(dev), torch.from_numpy(c["bias"]).to(dev), True,
+                     c["inv_step"], 0, 15, in_max=15, want=("q", "f32", "acc"))
+    assert ctx.device_status() == 0 and ctx.last_path() == psb.PSB_PATH_TENSOR
+    acc, q, f32 = (out[k].cpu().numpy() for k in ("acc", "q", "f32"))
+    W, eb, _ = oracle.sample_level(c["w"], c["seed"], 0, log2k)
+    g = oracle.geom(c["x"].shape, oracle.NCHW, oracle.U8, c["w"].shape, 1, 1, 1)
+    rng = np.random.default_rng(3)
+    pts = np.stack([rng.integers(0, 32, 4000), rng.integers(0, 64, 4000), rng.integers(0, 56, 4000),
+                    rng.integers(0, 56, 4000)], 1)
+    pts[:500, 2] = rng.choice([0, 55], 500)
+    pts[250:750, 3] = rng.choice([0, 55], 500)
+    ref = oracle.conv_acc_points(c["x"], g, {log2k: W}, pts, uniform_log2k=log2k)
+    got = acc[pts[:, 0], pts[:, 1], pts[:, 2], pts[:, 3]]
+    assert np.array_equal(got, ref)
+    for t in range(0, 4000, 40):
+        n, o, oy, ox = pts[t]
+        y = oracle.dequant_one(ref[t], c["scale"][o], eb[o], log2k, c["bias"][o], relu=True)
+        assert f32[n, o, oy, ox] == np.float32(y)
+        assert q[n, o, oy, ox] == oracle.requant_one(y, c["inv_step"], 0, 15)
+    assert q.max() <= 15 and (f32 >= 0).all()
+    wt.free()
+
+
+# ---------------------------------------------------------------- errors and glue
+
+def test_argument_errors_are_reported_not_launched(psb, ctx):
+    import torch
+
+    w = torch.randn(64, 64, 3, 3, device=ctx.device)
+    wt = ctx.sample_weights(w, level_mask=0b100)
+    x = torch.zeros(1, 8, 8, 64, dtype=torch.uint8, device=ctx.device)
+    sc = torch.ones(64, device=ctx.device)
+    ctx.set_sample_map(None, 3)                                 # level 3 was not sampled
+    with pytest.raises(psb.PsbError) as e:
+        ctx.conv2d(wt, x, 1, 1, 1, sc, sc, True, 1.0, 0, 15)
+    assert e.value.status == psb.PSB_ERR_BAD_K
+    ctx.set_sample_map(None, 2)
+    with pytest.raises(psb.PsbError) as e:                      # channel mismatch
+        ctx.conv2d(wt, torch.zeros(1, 8, 8, 32, dtype=torch.uint8, device=ctx.device), 1, 1, 1, sc, sc, True, 1.0, 0, 15)
+    assert e.value.status == psb.PSB_ERR_INVALID_ARG
+    with pytest.raises(psb.PsbError) as e:                      # code range beyond the container
+        ctx.conv2d(wt, x, 1, 1, 1, sc, sc, True, 1.0, 0, 300)
+    assert e.value.status == psb.PSB_ERR_INVALID_ARG
+    with pytest.raises(psb.PsbError) as e:                      # full-range u8 cannot take the tensor path
+        ctx.conv2d(wt, x, 1, 1, 1, sc, sc, True, 1.0, 0, 15, path=psb.PSB_PATH_TENSOR)
+    assert e.value.status == psb.PSB_ERR_UNSUPPORTED
+    kmap = torch.zeros(1, 4, 4, dtype=torch.uint8, device=ctx.device)
+    ctx.set_sample_map(kmap)                                    # map of the wrong size
+    with pytest.raises(psb.PsbError) as e:
+        ctx.conv2d(wt, x, 1, 1, 1, sc, sc, True, 1.0, 0, 15)
+    assert e.value.status == psb.PSB_ERR_INVALID_ARG
+    with pytest.raises(psb.PsbError):
+        ctx.sample_weights(w, level_mask=0)
+    with pytest.raises(psb.PsbError):
+        ctx.sample_weights(w, level_mask=1, exp_bits=5)
+    ctx.set_sample_map(None, 0)
+    assert ctx.device_status() == 0
+    wt.free()
+
+
+def test_device_side_errors_are_sticky_until_read(psb, ctx):
+    import torch
+
+    w = torch.randn(16, 16, 1, 1, device=ctx.device)
+    w[3, 2, 0, 0] = float("nan")
+    wt = ctx.sample_weights(w, level_mask=1)
+    assert ctx.device_status() == psb.PSB_ERR_NONFINITE_WEIGHT
+    assert ctx.device_status() == 0
+    wt.free()
+    w = torch.randn(64, 64, 1, 1, device=ctx.device)
+    wt = ctx.sample_weights(w, level_mask=0b101)
+    sc = torch.ones(64, device=ctx.device)
+    for path, in_max in ((psb.PSB_PATH_SHIFT_ADD, 0), (psb.PSB_PATH_TENSOR, 15)):
+        kmap = torch.full((2, 8, 8), 2, dtype=torch.uint8, device=ctx.device)
+        kmap[1, 3, 3] = 1                                       # a level that was not sampled
+        ctx.set_sample_map(kmap)
+        x = torch.ones(2, 8, 8, 64, dtype=torch.uint8, device=ctx.device)
+        ctx.conv2d(wt, x, 1, 1, 0, sc, sc, True, 1.0, 0, 15, in_max=in_max, path=path)
+        assert ctx.device_status() == psb.PSB_ERR_BAD_K
+    ctx.set_sample_map(None, 0)
+    wt.free()
+
+
+def test_pooling_kernels(psb, ctx, oracle):
+    import torch
+
+    rng = np.random.default_rng(31)
+    for layout in (0, 1):
+        x = rng.integers(0, 256, size=(3, 9, 13, 11) if layout == 0 else (3, 13, 11, 9), dtype=np.uint8)
+        xd = torch.from_numpy(x).to(ctx.device)
+        assert np.array_equal(ctx.maxpool2d_u8(xd, layout, 3, 2, 1).cpu().numpy(),
+                              oracle.maxpool_u8(x, layout, 3, 2, 1))
+        assert np.array_equal(ctx.global_avgpool_u8(xd, layout, 0.0123, 0, 255).cpu().numpy(),
+                              oracle.global_avgpool_u8(x, layout, np.float32(0.0123), 0, 255))

@@ -219,6 +219,41 @@ psb_status psb_global_avgpool_u8(psb_ctx* ctx, const uint8_t* x_dev, uint32_t la
                                  uint32_t c, uint32_t h, uint32_t w, float pool_mul, int32_t qmin,
                                  int32_t qmax, uint8_t* out_dev, void* stream);
 
+/* Sampling of one level without any allocation.  (The paper has no counterpart:
+ * this entry point exists for hosts, not for the method.)
+ *
+ * psb_sample_weights creates a handle with cudaMalloc on first use.  Some callers
+ * cannot do that at the moment they need fresh draws: a real-time loop that must
+ * never block on the device allocator, a thread working while another part of the
+ * process captures a CUDA graph (allocation is illegal during capture), or a
+ * process whose device memory was fully handed out at start-up.  This variant
+ * allocates nothing, on the device or through any library: its only scratch, the
+ * per-output-channel exponent maxima of the window reduction, lives in a fixed
+ * array inside the library's device image (PSB_STATIC_MAX_OUT_CH words + 256 B,
+ * held by every GPU that loads the library until the process exits).
+ *
+ *   w_dev, shape, cfg   as for psb_sample_weights; cfg->level_mask is ignored.
+ *   log2k               the one level to produce, k = 2^log2k, 0..6.
+ *   wint_out_dev        int32, canonical [out_ch][in_ch_per_group][kh][kw] order,
+ *                       caller-owned device memory; receives the same integers that
+ *                       psb_weights_export returns for that level.  May be NULL.
+ *   e_base_out_dev      int32 [out_ch], caller-owned; may be NULL (not both).
+ * Works on the current device, asynchronously on `stream`.
+ * Errors: PSB_ERR_UNSUPPORTED if shape->out_ch > PSB_STATIC_MAX_OUT_CH (the fixed
+ * array cannot hold the reduction) or the filter exceeds the sizes
+ * psb_sample_weights accepts; PSB_ERR_INVALID_ARG / PSB_ERR_BAD_K as usual.  Inf/NaN
+ * weights are not reported here; they contribute nothing.
+ * The first call on each device looks up the array's device address (a runtime
+ * query, no allocation); make that first call outside any stream capture.
+ * All calls on a device share the one array, which still holds the previous
+ * call's contents; every call clears the part it uses on `stream` first.  Two
+ * calls that can overlap on the GPU (different streams, no dependency) race on
+ * it: serialise them. */
+#define PSB_STATIC_MAX_OUT_CH 4096
+psb_status psb_sample_level_static(const float* w_dev, const psb_wshape* shape,
+                                   const psb_sample_cfg* cfg, uint32_t log2k, int32_t* wint_out_dev,
+                                   int32_t* e_base_out_dev, void* stream);
+
 #ifdef __cplusplus
 }
 #endif

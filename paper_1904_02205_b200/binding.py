@@ -22,7 +22,7 @@ PSB_PATH_AUTO, PSB_PATH_SHIFT_ADD, PSB_PATH_TENSOR = 0, 1, 2
 
 EXPORTS = ["psb_create", "psb_destroy", "psb_status_string", "psb_device_status", "psb_sample_weights",
            "psb_weights_export", "psb_weights_free", "psb_set_sample_map", "psb_conv2d", "psb_gemm",
-           "psb_last_path", "psb_maxpool2d_u8", "psb_global_avgpool_u8"]
+           "psb_last_path", "psb_maxpool2d_u8", "psb_global_avgpool_u8", "psb_sample_level_static"]
 
 
 class psb_wshape(C.Structure):
@@ -80,6 +80,7 @@ def load_library():
     lib.psb_last_path.argtypes = [vp]
     lib.psb_maxpool2d_u8.argtypes = [vp, vp, u32, u32, u32, u32, u32, u32, u32, u32, vp, vp]
     lib.psb_global_avgpool_u8.argtypes = [vp, vp, u32, u32, u32, u32, u32, C.c_float, i32, i32, vp, vp]
+    lib.psb_sample_level_static.argtypes = [vp, C.POINTER(psb_wshape), C.POINTER(psb_sample_cfg), u32, vp, vp, vp]
     for name in EXPORTS:
         if name != "psb_status_string":
             getattr(lib, name).restype = i32
@@ -117,6 +118,28 @@ def _dt_of(t):
     if t.dtype == torch.int8:
         return PSB_DT_S8
     raise TypeError("activations must be uint8 or int8")
+
+
+PSB_STATIC_MAX_OUT_CH = 4096
+
+
+def sample_level_static(w, wint_out, e_base_out, groups=1, seed=0, layer_id=0, log2k=0, exp_bits=4,
+                        norm=0, stream=None):
+    """psb_sample_level_static: sample one level into tensors the caller already owns.
+
+    For callers that must not allocate (real-time loops, work next to a graph capture, fixed
+    memory budgets): needs no Context and allocates nothing; w is a float32 CUDA tensor
+    [out_ch, in_ch/groups, kh, kw], wint_out an int32 CUDA tensor of the same shape, e_base_out
+    int32 [out_ch] (either output may be None).  Calls that may overlap on the GPU must be
+    serialised by the caller; they share one fixed scratch array inside the library.
+    """
+    assert w.is_cuda and w.dtype == torch.float32 and w.is_contiguous()
+    shape = psb_wshape(w.shape[0], w.shape[1], w.shape[2], w.shape[3], groups)
+    cfg = psb_sample_cfg(seed, layer_id, 0, exp_bits, norm)
+    with torch.cuda.device(w.device):
+        _check(load_library().psb_sample_level_static(_ptr(w), C.byref(shape), C.byref(cfg), log2k,
+                                                      _ptr(wint_out), _ptr(e_base_out), _stream(stream)),
+               "psb_sample_level_static")
 
 
 class Weights:

@@ -243,3 +243,113 @@ cudaError_t launch_export(const psb_weights* wt, uint32_t level, int32_t* wint_o
 }
 
 }  // namespace psb
+
+// ---------------------------------------------------------------------------
+// Allocation-free sampling of one level (psb_sample_level_static in psb.h).
+//
+// Some hosts may not allocate device memory when they need fresh weights: a
+// real-time loop that must not block on the allocator, code running while a CUDA
+// graph is being captured elsewhere in the process, or a process whose memory
+// budget was handed out at start-up.  For them the window reduction's scratch
+// (one biased exponent per output channel, plus a device error word nobody reads)
+// lives in this file-scope device array instead of a cudaMalloc'ed buffer.  Every
+// GPU that loads the library holds these 16 KB + 256 B until the process exits.
+namespace psb {
+namespace {
+
+constexpr uint32_t kStaticMaxOutCh = 4096;   // PSB_STATIC_MAX_OUT_CH in psb.h
+static __device__ __align__(256) uint32_t g_static_scratch[kStaticMaxOutCh + 64];
+
+constexpr int kMaxDevices = 64;
+uint32_t* g_static_scratch_addr[kMaxDevices] = {};   // device address per device ordinal
+
+// One thread per weight, canonical order in and out (both coalesce).  e_max is
+// the device address of the static scratch, filled by emax_kernel just before.
+__global__ void __launch_bounds__(kThreads)
+sample_level_canonical_kernel(const float* __restrict__ w, uint32_t O, uint32_t d, uint32_t norm,
+                              uint32_t span, uint32_t log2k, uint32_t seed_lo, uint32_t seed_hi,
+                              uint32_t layer_id, const uint32_t* __restrict__ e_max,
+                              int32_t* __restrict__ wint_out, int32_t* __restrict__ e_base_out) {
+  const size_t total = (size_t)O * d;
+  for (size_t index = (size_t)blockIdx.x * blockDim.x + threadIdx.x; index < total;
+       index += (size_t)gridDim.x * blockDim.x) {
+    const uint32_t o = (uint32_t)(index / d);
+    const uint32_t u = __float_as_uint(w[index]);
+    const uint32_t E = (u >> 23) & 0xFFu, m = u & 0x7FFFFFu;
+    const uint32_t Emax = e_max[norm ? o : 0];
+    const int ebase_biased = (int)Emax - (int)span;
+    if (index % d == 0 && e_base_out) e_base_out[o] = Emax ? ebase_biased - 127 : 0;
+    if (!wint_out) continue;
+    const bool live = (E != 0u) && (E != 255u) && ((int)E >= ebase_biased);
+    uint32_t c = 0;
+    if (live && m != 0u) {
+      const uint32_t T = m << 9, k = 1u << log2k;
+      for (uint32_t q = 0; q * 4u < k; ++q) {
+        uint32_t rnd[4];
+        philox4x32_10(q, layer_id, (uint32_t)index, (uint32_t)(index >> 32), seed_lo, seed_hi, rnd);
+#pragma unroll
+        for (int v = 0; v < 4; ++v)
+          if (q * 4u + v < k) c += (rnd[v] < T) ? 1u : 0u;
+      }
+    }
+    const uint32_t mag = live ? (((1u << log2k) + c) << (uint32_t)((int)E - ebase_biased)) : 0u;
+    wint_out[index] = (u >> 31) ? -(int32_t)mag : (int32_t)mag;
+  }
+}
+
+}  // namespace
+}  // namespace psb
+
+extern "C" psb_status psb_sample_level_static(const float* w_dev, const psb_wshape* shape,
+                                              const psb_sample_cfg* cfg, uint32_t log2k,
+                                              int32_t* wint_out_dev, int32_t* e_base_out_dev,
+                                              void* stream) {
+  using namespace psb;
+  if (!w_dev || !shape || !cfg || (!wint_out_dev && !e_base_out_dev)) return PSB_ERR_INVALID_ARG;
+  if (((uintptr_t)w_dev | (uintptr_t)wint_out_dev | (uintptr_t)e_base_out_dev) & 3u)
+    return PSB_ERR_INVALID_ARG;
+  if (!shape->out_ch || !shape->in_ch_per_group || !shape->kh || !shape->kw || !shape->groups)
+    return PSB_ERR_INVALID_ARG;
+  if (log2k >= (uint32_t)kMaxLevels) return PSB_ERR_BAD_K;
+  const uint32_t exp_bits = cfg->exp_bits ? cfg->exp_bits : 4u;
+  if (exp_bits > 4 || cfg->norm > 1) return PSB_ERR_INVALID_ARG;
+  // the static scratch holds one word per output channel: larger filters are refused
+  if (shape->out_ch > kStaticMaxOutCh) return PSB_ERR_UNSUPPORTED;
+  const uint64_t d64 = (uint64_t)shape->in_ch_per_group * shape->kh * shape->kw;
+  if (d64 > (1u << 24) || d64 * shape->out_ch > (1ull << 31)) return PSB_ERR_UNSUPPORTED;
+
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return PSB_ERR_CUDA;
+  if (!g_static_scratch_addr[dev]) {
+    // first call on this device: the symbol's name is only a host-side stand-in, so ask the
+    // runtime for the array's address on the current device
+    void* addr = nullptr;
+    if (cudaGetSymbolAddress(&addr, g_static_scratch) != cudaSuccess || !addr) {
+      cudaGetLastError();
+      return PSB_ERR_CUDA;
+    }
+    g_static_scratch_addr[dev] = (uint32_t*)addr;
+  }
+  uint32_t* scratch = g_static_scratch_addr[dev];
+  uint32_t* e_max = scratch;                        // [out_ch]
+  uint32_t* err_sink = scratch + kStaticMaxOutCh;   // written on Inf/NaN, never read
+  cudaStream_t s = (cudaStream_t)stream;
+  const uint32_t O = shape->out_ch, d = (uint32_t)d64;
+  // the array keeps the previous call's maxima: the reduction must start from zero
+  if (cudaMemsetAsync(e_max, 0, sizeof(uint32_t) * O, s) != cudaSuccess) return PSB_ERR_CUDA;
+  if (cfg->norm) {
+    emax_kernel<<<O, kThreads, 0, s>>>(w_dev, O, d, 1, e_max, err_sink);
+  } else {
+    size_t total = (size_t)O * d;
+    uint32_t blocks = (uint32_t)((total + kThreads * 8 - 1) / (kThreads * 8));
+    blocks = blocks < 1 ? 1 : (blocks > 1184 ? 1184 : blocks);
+    emax_kernel<<<blocks, kThreads, 0, s>>>(w_dev, O, d, 0, e_max, err_sink);
+  }
+  size_t total = (size_t)O * d;
+  uint32_t blocks = (uint32_t)((total + kThreads - 1) / kThreads);
+  blocks = blocks > 148u * 16u ? 148u * 16u : blocks;
+  sample_level_canonical_kernel<<<blocks, kThreads, 0, s>>>(
+      w_dev, O, d, cfg->norm, (1u << exp_bits) - 1u, log2k, (uint32_t)cfg->seed,
+      (uint32_t)(cfg->seed >> 32), cfg->layer_id, e_max, wint_out_dev, e_base_out_dev);
+  return cudaGetLastError() == cudaSuccess ? PSB_OK : PSB_ERR_CUDA;
+}

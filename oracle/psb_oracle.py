@@ -216,3 +216,41 @@ def global_avgpool_u8(x, layout, pool_mul, qmin, qmax):
                                  C.c_uint32(H), C.c_uint32(W), C.c_float(pool_mul), C.c_int32(qmin),
                                  C.c_int32(qmax), _p(out))
     return out
+
+
+def run_network(layers, net, images, seed, uniform_log2k=3, fc_log2k=None, kmaps=None, levels=None):
+    """The oracle's forward pass of a layer list (workloads.nets) on u8 images [n, h, w, 3].
+
+    Returns ({tensor name: integer codes}, logits float32).  kmaps: {resolution: u8 [n, res, res]}.
+    """
+    fc_log2k = uniform_log2k if fc_log2k is None else fc_log2k
+    acts = {"image": np.ascontiguousarray(images)}
+    logits = None
+    for l in layers:
+        x = acts[l["src"]]
+        if l["op"] == "maxpool":
+            acts[l["dst"]] = maxpool_u8(x, NHWC, l["k"], l["stride"], l["pad"])
+            continue
+        p = net["params"][l["name"]]
+        if l["op"] == "avgpool":
+            acts[l["dst"]] = global_avgpool_u8(x, NHWC, p["pool_mul"], p["qmin"], p["qmax"])
+            continue
+        is_fc = x.ndim == 2
+        if is_fc:
+            x = x.reshape(x.shape[0], 1, 1, x.shape[1])
+        kmap = None if (kmaps is None or is_fc) else np.ascontiguousarray(kmaps[l["hout"]][:x.shape[0]])
+        lv = fc_log2k if is_fc else uniform_log2k
+        need = sorted(set(int(v) for v in np.unique(kmap))) if kmap is not None else [lv]
+        Ws, eb = {}, None
+        for lev in need:
+            Ws[lev], eb, _ = sample_level(p["w"], seed, p["layer_id"], lev)
+        g = geom(x.shape, NHWC, U8 if x.dtype == np.uint8 else S8, p["w"].shape, l["groups"], l["stride"], l["pad"])
+        acc = conv_acc(x, g, Ws, kmap=kmap, uniform_log2k=lv)
+        res = None if l["residual"] is None else acts[l["residual"]]
+        y, q = epilogue(acc, g, p["scale"], p["bias"], eb, l["relu"], p["inv_step"], p["qmin"], p["qmax"],
+                        residual=res, residual_scale=p["res_scale"], kmap=kmap, uniform_log2k=lv)
+        q = q.astype(np.int8 if p["out_dtype"] == S8 else np.uint8)
+        if is_fc:
+            q, logits = q.reshape(q.shape[0], -1), y.reshape(y.shape[0], -1)
+        acts[l["dst"]] = q
+    return acts, logits

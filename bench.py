@@ -176,11 +176,117 @@ class ConvWorkload:
         return dt, self.macs * n_images // self.images, "first %d of %d images, all layers" % (n_images, self.images)
 
 
+class NetWorkload:
+    """Network-shaped workloads: every conv / FC layer is a PSB layer, activations stay in HBM."""
+    oracle_images = 1
+
+    def __init__(self, kind, k, rank=0, batch=0):
+        from workloads import mobilenetv2_layers, network_macs, resnet50_layers
+
+        self.kind, self.k, self.rank = kind, k, rank
+        self.log2k = int(np.log2(k))
+        if kind == "mobilenetv2":
+            self.layers, self.batch, self.qu, self.qs, self.prune, self.seed = mobilenetv2_layers(), batch or 64, 255, 127, 0.5, 3
+        else:
+            self.layers, self.qu, self.qs, self.prune = resnet50_layers(), 15, 15, 0.0
+            self.batch, self.seed = (batch or 128, 4) if kind == "resnet50_adaptive" else (batch or 64, 2)
+        self.adaptive = kind == "resnet50_adaptive"
+        self.images = self.batch
+        self.macs_per_image = network_macs(self.layers)
+        self.macs = self.macs_per_image * self.batch
+        self.name = "%s_b%d" % (kind, self.batch)
+        self.mean_k = 4.0 if self.adaptive else float(k)
+
+    def setup(self, ctx, psb, torch):
+        from paper_1904_02205_b200.network import Network
+        from workloads import build_network, saliency_kmaps
+
+        self.ctx, self.psb, self.torch = ctx, psb, torch
+        self.net = build_network(self.layers, 224, self.batch, self.seed + 100 * self.rank, self.qu, self.qs,
+                                 prune_frac=self.prune)
+        self.kmaps = saliency_kmaps(self.batch, [112, 56, 28, 14, 7], self.seed) if self.adaptive else None
+        mask = 0b11111 if self.adaptive else 1 << self.log2k
+        self.nw = Network(ctx, self.layers, self.net, self.batch, mask, kmaps=self.kmaps, uniform_log2k=self.log2k,
+                          fc_log2k=4 if self.adaptive else None)
+        self.nw.sample(self.seed)
+        self.image_host = torch.from_numpy(self.net["image"]).pin_memory()
+        self.image_dev = self.image_host.to(ctx.device)
+        self.logits_host = torch.empty((self.batch, self.layers[-1]["cout"]), dtype=torch.float32).pin_memory()
+        self.nw.forward(self.image_dev)
+        n_conv = sum(1 for l in self.layers if l["op"] == "conv")
+        # per conv layer: window reduction + sampler + contraction; plus the pooling kernels
+        self.launches_per_step = 3 * n_conv + (len(self.layers) - n_conv)
+        self.e2e_h2d = self.image_host.numel()
+        self.e2e_d2h = self.logits_host.numel() * 4
+        self.layer_ms = None
+
+    def step(self, i):
+        self.nw.sample(self.seed + i)
+        self.nw.forward()
+
+    def kernel_only(self):
+        """One forward pass with fixed filters and a pair of events around every layer."""
+        ev = {}
+        self.nw.forward(layer_events=ev)
+        self.torch.cuda.synchronize()
+        ms = {k: a.elapsed_time(b) for k, (a, b) in ev.items()}
+        if self.layer_ms is None:
+            self.layer_ms = {k: [] for k in ms}
+        for k, v in ms.items():
+            self.layer_ms[k].append(v)
+
+    def e2e_step(self, i):
+        self.nw.acts["image"].copy_(self.image_host, non_blocking=True)
+        self.nw.sample(self.seed + i)
+        self.nw.forward()
+        self.logits_host.copy_(self.nw.logits, non_blocking=True)
+
+    def roofline(self, _kernel_ms, peaks):
+        """All launches of the tensor-core contraction in one forward pass, from per-layer events."""
+        psb = self.psb
+        span_bits = 15 + (4 if self.adaptive else self.log2k) + 2
+        planes = (span_bits + 6) // 7
+        t_ops, t_ms, s_ms, rows = 0.0, 0.0, 0.0, []
+        for l in self.layers:
+            ms = statistics.mean(self.layer_ms[l["name"]][1:] or self.layer_ms[l["name"]])
+            if l["op"] != "conv":
+                s_ms += ms
+                continue
+            macs = l["hout"] ** 2 * l["cout"] * (l["cin"] // l["groups"]) * l["k"] ** 2 * self.batch
+            path = self.nw.paths[l["name"]]
+            if path == psb.PSB_PATH_TENSOR:
+                t_ops += 2.0 * macs * planes
+                t_ms += ms
+            else:
+                s_ms += ms
+            rows.append((l["name"], "tensor" if path == psb.PSB_PATH_TENSOR else "cuda-core", macs, ms))
+        self.layer_rows = rows
+        achieved = t_ops / (t_ms * 1e-3) / 1e12 if t_ms else 0.0
+        peak = 2.0 * peaks["bf16_tflops_sustained"]
+        return dict(bound="tensor", kernel="psb_mma_kernel (all launches of one forward pass)", achieved=achieved,
+                    peak=peak, unit="TOP/s (int8)", frac=achieved / peak, traffic=None,
+                    peak_source=peaks["source"] + " bf16 sustained x 2", planes=planes, tensor_path_ms=t_ms,
+                    other_layers_ms=s_ms)
+
+    def oracle_sample(self, n_images=1):
+        from oracle import psb_oracle as orc
+
+        if not hasattr(self, "net"):
+            from workloads import build_network, saliency_kmaps
+
+            self.net = build_network(self.layers, 224, max(n_images, 2), self.seed, self.qu, self.qs, prune_frac=self.prune)
+            self.kmaps = saliency_kmaps(max(n_images, 2), [112, 56, 28, 14, 7], self.seed) if self.adaptive else None
+        t0 = time.perf_counter()
+        orc.run_network(self.layers, self.net, self.net["image"][:n_images], self.seed, uniform_log2k=self.log2k,
+                        fc_log2k=4 if self.adaptive else None,
+                        kmaps=None if self.kmaps is None else {r: m[:n_images] for r, m in self.kmaps.items()})
+        dt = time.perf_counter() - t0
+        return dt, self.macs_per_image * n_images, "first %d of %d images, all layers, filters sampled once" % (n_images, self.batch)
+
+
 def make_workload(args, rank):
     if args.workload == "conv3x3":
         return ConvWorkload(args.k, rank)
-    from bench_nets import NetWorkload  # network-shaped workloads
-
     return NetWorkload(args.workload, args.k, rank, batch=args.batch)
 
 
@@ -234,6 +340,7 @@ def main():
     ap.add_argument("--k", type=int, default=8)
     ap.add_argument("--batch", type=int, default=0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--layer-table", default="", help="write per-layer times of the network workloads to this CSV")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl != "reference" else args.warmup
     if args.impl == "reference":
@@ -279,7 +386,7 @@ def main():
     torch.cuda.synchronize()
     if world > 1:
         dist.barrier()
-    kern_ms = timed(lambda i: wl.kernel_only(), max(args.steps, 10))
+    kern_ms = timed(lambda i: wl.kernel_only(), max(args.steps, 10) if args.workload == "conv3x3" else 4)
     clk = clocks.stop()
     ctx.check_device()
     e2e_warm = timed(wl.e2e_step, 3)
@@ -310,6 +417,11 @@ def main():
         dt, macs, sample = wl.oracle_sample(getattr(wl, "oracle_images", 4))
         line["cpu_baseline"] = dict(value=macs / dt / 1e9, unit=UNIT, cores=1, kind="oracle", sample=sample)
     print(json.dumps(line))
+    if args.layer_table and hasattr(wl, "layer_rows"):
+        with open(args.layer_table, "w") as f:
+            f.write("layer,path,macs,ms,logical_gmacs\n")
+            for name, path, macs, ms in wl.layer_rows:
+                f.write("%s,%s,%d,%.5f,%.1f\n" % (name, path, macs, ms, macs / (ms * 1e-3) / 1e9))
     if world > 1:
         dist.destroy_process_group()
     return 0

@@ -51,12 +51,21 @@ class Network:
                 pr["w"], groups=l["groups"], seed=seed, layer_id=pr["p"]["layer_id"], level_mask=self.level_mask,
                 into=self.weights.get(l["name"]))
 
-    def forward(self, image=None):
-        """image: u8 CUDA tensor [batch, h, w, 3] (copied into the resident input buffer) or None."""
+    def forward(self, image=None, layer_events=None):
+        """image: u8 CUDA tensor [batch, h, w, 3] (copied into the resident input buffer) or None.
+        layer_events: optional dict that receives {layer name: (start, end)} CUDA events."""
         ctx = self.ctx
         if image is not None:
             self.acts["image"].copy_(image, non_blocking=True)
+        prev_end = None
         for l in self.layers:
+            if layer_events is not None:
+                ev = (torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
+                if prev_end is not None:
+                    prev_end.record()
+                ev[0].record()
+                layer_events[l["name"]] = ev
+                prev_end = ev[1]
             x = self.acts[l["src"]]
             if l["op"] == "maxpool":
                 ctx.maxpool2d_u8(x, B.PSB_LAYOUT_NHWC, l["k"], l["stride"], l["pad"], out=self.acts[l["dst"]])
@@ -84,6 +93,8 @@ class Network:
                            residual=res, residual_scale=p["res_scale"], in_max=self.qmax[l["src"]],
                            path=self.path, out=out)
             self.paths[l["name"]] = ctx.last_path()
+        if prev_end is not None:
+            prev_end.record()
         ctx.set_sample_map(None, 0)
         return self.logits
 

@@ -120,7 +120,7 @@ psb_status run_layer(psb_ctx* ctx, const psb_weights* wt, const void* x_dev, uin
   }
 
   if (tensor_ok) {
-    st = launch_tensor(ctx, wt, a, s);
+    st = launch_tensor(ctx, wt, a, amax, s);
     if (st != PSB_OK) return st;
     ctx->last_path = PSB_PATH_TENSOR;
     return PSB_OK;

@@ -140,6 +140,7 @@ cudaError_t launch_avgpool(const uint8_t* x, uint32_t nchw, uint32_t N, uint32_t
                            cudaStream_t s);
 // tensor path: returns PSB_ERR_UNSUPPORTED if the shape does not fit it
 psb_status tensor_supported(const psb_ctx* ctx, const psb_weights* wt, const ConvArgs& a);
-psb_status launch_tensor(psb_ctx* ctx, const psb_weights* wt, const ConvArgs& a, cudaStream_t s);
+psb_status launch_tensor(psb_ctx* ctx, const psb_weights* wt, const ConvArgs& a, uint32_t amax,
+                         cudaStream_t s);
 
 }  // namespace psb

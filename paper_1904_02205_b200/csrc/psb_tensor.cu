@@ -15,7 +15,7 @@
 //            of the digit-plane tile into a ring of shared-memory stages
 //   warp 1   allocates TMEM; one thread issues the MMAs and commits them to the
 //            stage-free and accumulator-ready barriers
-//   warps 2-5  epilogue: TMEM -> registers, recombine planes, dequantise, bias,
+//   warps 2-9  epilogue: TMEM -> registers, recombine planes, dequantise, bias,
 //            shortcut, ReLU, re-quantise, vectorised stores; overlaps the next
 //            tile's MMAs through two TMEM accumulator buffers
 // Per-location draw counts (Sec. 4.5): a tile is contracted once per level present
@@ -33,11 +33,13 @@ namespace psb {
 namespace {
 
 constexpr int kTileM = 128;
-constexpr int kThreadsTensor = 192;
+constexpr int kEpilogueWarps = 8;
+constexpr int kThreadsTensor = 64 + 32 * kEpilogueWarps;   // producer warp, MMA warp, epilogue warps
 constexpr uint32_t kTmemCols = 512;
 constexpr uint32_t kTmemBufStride = 256;
-constexpr int kMaxStages = 8;
-constexpr unsigned long long kWaitLimitNs = 2000000000ull;  // 2 s per wait
+constexpr int kMaxStages = 12;
+constexpr long long kWaitLimitCycles = 4000000000ll;        // about 2 s of SM clocks per wait
+constexpr uint32_t kResidentMaxBytes = 112 * 1024;          // digit planes kept in shared memory
 
 struct TmapSet {
   CUtensorMap a;
@@ -52,9 +54,15 @@ struct TensorParams {
   uint32_t cpad;
   uint32_t im2col;      // 1: activation tile through the im2col tensor map
   uint32_t stages;
+  uint32_t group;       // K blocks per pipeline stage (one barrier hand-over per group)
   uint32_t stage_bytes_a, stage_bytes_b_max;
   uint32_t planes[kMaxLevels];
   uint32_t vec_ok;      // 16-byte stores are legal for every output pointer
+  uint32_t resident;    // 1: the CTA keeps the digit planes of its channel tile in shared memory
+  uint32_t ctas_per_otile;
+  uint32_t resident_bytes;
+  uint32_t narrow;      // P <= 3 and plane sums below 2^22 (2) or 2^24 (1): 32-bit recombination
+  const long long* corr[kMaxLevels];  // per-channel integer addend, or null
 };
 
 // ---- thin PTX wrappers -------------------------------------------------------
@@ -88,22 +96,18 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
   return ok != 0;
 }
 
-__device__ __forceinline__ unsigned long long global_ns() {
-  unsigned long long t;
-  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
-  return t;
-}
-
-// Bounded wait.  Returns false after kWaitLimitNs without completion, or as soon
-// as another thread of the CTA has given up.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile uint32_t* abort) {
+// Bounded wait.  Returns false after kWaitLimitCycles SM clocks without completion, or as soon
+// as another thread of the CTA has given up.  (The SM cycle counter is cheap to read.)
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile uint32_t* abort,
+                                          uint32_t backoff_ns = 0) {
   if (mbar_try_wait(bar, parity)) return true;
-  const unsigned long long t0 = global_ns();
+  const long long t0 = clock64();
   uint32_t spins = 0;
   while (!mbar_try_wait(bar, parity)) {
-    if ((++spins & 255u) == 0u) {
+    if (backoff_ns) __nanosleep(backoff_ns);
+    if ((++spins & 15u) == 0u) {
       if (*abort) return false;
-      if (global_ns() - t0 > kWaitLimitNs) return false;
+      if (clock64() - t0 > kWaitLimitCycles) return false;
     }
   }
   return true;
@@ -190,111 +194,195 @@ __device__ __forceinline__ uint32_t tile_levels(const TensorParams& p, uint32_t 
   return __reduce_or_sync(0xFFFFFFFFu, mask);
 }
 
+// Same, computed by one thread alone (the single-thread producer and MMA roles).
+__device__ __forceinline__ uint32_t tile_levels_serial(const TensorParams& p, uint32_t m0) {
+  if (!p.a.kmap) return 1u << p.a.uniform_log2k;
+  uint32_t mask = 0;
+  const uint32_t end = min(m0 + (uint32_t)kTileM, p.M);
+  for (uint32_t m = m0; m < end; ++m) mask |= 1u << (p.a.kmap[m] & 31u);
+  return mask;
+}
+
+// Walks the tiles of this CTA without divisions in the loop.  Resident mode: the CTA owns one
+// channel tile and strides over the row tiles; streaming mode: tiles are dealt round-robin with
+// the channel tile fastest.
+struct TileIter {
+  uint32_t m_tile, o_tile, step_m, step_o, o_tiles, m_tiles;
+  __device__ __forceinline__ void init(const TensorParams& p) {
+    o_tiles = p.o_tiles;
+    m_tiles = p.m_tiles;
+    if (p.resident) {
+      o_tile = blockIdx.x / p.ctas_per_otile;
+      m_tile = blockIdx.x % p.ctas_per_otile;
+      step_m = p.ctas_per_otile;
+      step_o = 0;
+    } else {
+      m_tile = blockIdx.x / p.o_tiles;
+      o_tile = blockIdx.x % p.o_tiles;
+      step_m = gridDim.x / p.o_tiles;
+      step_o = gridDim.x % p.o_tiles;
+    }
+  }
+  __device__ __forceinline__ bool valid() const { return m_tile < m_tiles; }
+  __device__ __forceinline__ void next() {
+    m_tile += step_m;
+    o_tile += step_o;
+    if (o_tile >= o_tiles) { o_tile -= o_tiles; ++m_tile; }
+  }
+};
+
 struct SharedCtl {
   unsigned long long full[kMaxStages];
   unsigned long long empty[kMaxStages];
   unsigned long long acc_full[2];
   unsigned long long acc_empty[2];
+  unsigned long long planes_full;
   uint32_t tmem_base;
   volatile uint32_t abort;
-  float sc[4][kTileN];      // per epilogue warp: scale[o] * 2^(e_base[o] - log2 k)
-  float bias[4][kTileN];
+  float2 scb[kEpilogueWarps][32];       // per epilogue warp: (scale * 2^(e_base - log2 k), bias)
+  long long corr[kEpilogueWarps][32];   // per epilogue warp: integer addend per channel
 };
 
-template <int P>
-__device__ __forceinline__ void epilogue_chunk(const TensorParams& p, uint32_t tmem_row_base,
-                                               uint32_t chunk, uint32_t o_base, uint32_t m, bool valid,
-                                               uint32_t n, uint32_t pix, const float* sc_s,
-                                               const float* bias_s) {
+// Exact round-to-nearest conversion of a 64-bit accumulator, |acc| < 2^47: split into a high
+// part (multiple of 2^24) and a 24-bit low part, both exact in fp32; one fma rounds their sum once.
+__device__ __forceinline__ float acc_to_float(long long acc) {
+  const int hi = (int)(acc >> 24);
+  const int lo = (int)((unsigned int)acc & 0xFFFFFFu);
+  return __fmaf_rn((float)hi, 16777216.0f, (float)lo);
+}
+
+// Fast output stage for the common case: only re-quantised bytes are wanted, channels-last,
+// 16 whole channels, 16-byte aligned.  Same arithmetic as dequant()/requant().
+// NARROW: every plane sum is below 2^24 in magnitude and P <= 3, so the recombination fits 32-bit
+// integers: with u = v0 + 2^7 v1 and w = (u >> 14) + v2, acc = w * 2^14 + (u mod 2^14), both parts
+// exact in fp32, and one fma rounds acc to nearest once.
+// The run-time options enter as data (a relu floor of 0 or -inf, a sign mask, an addend that may
+// be zero), not as branches, so that each instantiation stays one compact code path.
+// Integer <-> float conversions run on a slow pipe (a quarter of the FMA rate), so small integers
+// are converted with exponent tricks on the main pipes instead:
+//   float(n) = as_float(0x4B000000 | n) - 2^23              for 0 <= n < 2^23
+//   float(n) = as_float(0x4B400000 + n) - 1.5 * 2^23        for |n| < 2^22
+//   rint(t)  = low bits of as_int(t + 1.5 * 2^23)           for |t| < 2^22 (the add rounds to even)
+// MODE 2: every plane sum is below 2^22 in magnitude (both halves of the accumulator by tricks);
+// MODE 1: below 2^24 (the high half by a conversion instruction); MODE 0: 64-bit recombination.
+template <int P, int MODE, bool HAS_RES>
+__device__ __noinline__ void epilogue_chunk_q(uint32_t taddr, bool valid, uint8_t* q_dst, uint4 r4,
+                                              const float2* scb, const long long* corr, float res_scale,
+                                              uint32_t res_sign, float relu_floor, float inv_step,
+                                              float qmin_f, float qmax_f) {
   uint32_t v[P][16];
 #pragma unroll
-  for (int pl = 0; pl < P; ++pl) tc_ld16(tmem_row_base + pl * kTileN + chunk * 16u, v[pl]);
+  for (int pl = 0; pl < P; ++pl) tc_ld16(taddr + pl * kTileN, v[pl]);
+  tc_wait_ld();
+  if (!valid) return;
+  const uint32_t rw[4] = {r4.x, r4.y, r4.z, r4.w};
+  const float res_bias = 8388608.0f + (float)res_sign;   // undoes the magic constant and the sign flip
+  uint32_t q[16];
+#pragma unroll
+  for (int j = 0; j < 16; ++j) {
+    float af;
+    if (MODE > 0) {
+      // acc = w * 2^14 + lo with u = v0 + 2^7 v1, w = (u >> 14) + v2, lo = u mod 2^14: both parts
+      // are exact in fp32 and one fma rounds acc to nearest once
+      int u = (int)v[0][j];
+      if (P > 1) u += (int)v[1][j] << kDigitBits;
+      int w = u >> (2 * kDigitBits);
+      if (P > 2) w += (int)v[2][j];
+      const float lo_f = __uint_as_float(0x4B000000u | ((uint32_t)u & 0x3FFFu)) - 8388608.0f;
+      const float w_f = MODE == 2 ? __int_as_float(0x4B400000 + w) - 12582912.0f : (float)w;
+      af = __fmaf_rn(w_f, 16384.0f, lo_f);
+    } else {
+      long long acc = (long long)(int)v[0][j];
+#pragma unroll
+      for (int pl = 1; pl < P; ++pl) acc += (long long)(int)v[pl][j] * (long long)(1 << (kDigitBits * pl));
+      acc += corr[j];
+      af = acc_to_float(acc);
+    }
+    const float2 sb = scb[j];
+    float y = __fmaf_rn(af, sb.x, sb.y);
+    if (HAS_RES) {
+      const uint32_t rb = ((rw[j >> 2] >> (8 * (j & 3))) & 0xFFu) ^ res_sign;   // byte + 128 if signed
+      y = __fmaf_rn(__uint_as_float(0x4B000000u | rb) - res_bias, res_scale, y);
+    }
+    y = fmaxf(y, relu_floor);
+    // clamp, then round half to even by adding 1.5 * 2^23: the low byte of the sum is the code
+    const float t = fminf(fmaxf(__fmul_rn(y, inv_step), qmin_f), qmax_f);
+    q[j] = __float_as_uint(t + 12582912.0f);
+  }
+  uint32_t qw[4];
+#pragma unroll
+  for (int g = 0; g < 4; ++g) {
+    const uint32_t lo = __byte_perm(q[4 * g], q[4 * g + 1], 0x0040);
+    const uint32_t hi = __byte_perm(q[4 * g + 2], q[4 * g + 3], 0x0040);
+    qw[g] = __byte_perm(lo, hi, 0x5410);
+  }
+  *reinterpret_cast<uint4*>(q_dst) = make_uint4(qw[0], qw[1], qw[2], qw[3]);
+}
+
+// General output stage: any combination of outputs, layouts, ragged channel counts.
+template <int P>
+__device__ __noinline__ void epilogue_chunk(const TensorParams& p, uint32_t taddr, uint32_t o_base,
+                                            uint32_t m, bool valid, uint32_t n, uint32_t pix,
+                                            const float2* scb, const long long* corr, bool use_corr) {
+  uint32_t v[P][16];
+#pragma unroll
+  for (int pl = 0; pl < P; ++pl) tc_ld16(taddr + pl * kTileN, v[pl]);
   tc_wait_ld();
   if (!valid) return;
   const ConvArgs& a = p.a;
   const uint32_t ohow = a.OH * a.OW;
-  long long acc[16];
-#pragma unroll
-  for (int j = 0; j < 16; ++j) {
-    long long s = (long long)(int)v[0][j];
-#pragma unroll
-    for (int pl = 1; pl < P; ++pl) s += (long long)(int)v[pl][j] << (kDigitBits * pl);
-    acc[j] = s;
+  const bool vec = p.vec_ok && o_base + 16u <= a.O && !a.out_nchw;
+  uint32_t rw[4] = {0, 0, 0, 0};
+  if (vec && a.residual) {
+    uint4 r4 = *reinterpret_cast<const uint4*>((const uint8_t*)a.residual + (size_t)m * a.O + o_base);
+    rw[0] = r4.x; rw[1] = r4.y; rw[2] = r4.z; rw[3] = r4.w;
   }
-  const bool full16 = o_base + 16u <= a.O;
-  if (p.vec_ok && full16 && !a.out_nchw) {
-    const size_t oidx = (size_t)m * a.O + o_base;
-    if (a.acc_out) {
-      longlong2* dst = reinterpret_cast<longlong2*>(a.acc_out + oidx);
-#pragma unroll
-      for (int j = 0; j < 8; ++j) dst[j] = make_longlong2(acc[2 * j], acc[2 * j + 1]);
-    }
-    if (a.q_out || a.f32_out) {
-      uint32_t rw[4] = {0, 0, 0, 0};
-      if (a.residual) {
-        uint4 r4 = *reinterpret_cast<const uint4*>((const uint8_t*)a.residual + oidx);
-        rw[0] = r4.x; rw[1] = r4.y; rw[2] = r4.z; rw[3] = r4.w;
-      }
-      float y[16];
-#pragma unroll
-      for (int j = 0; j < 16; ++j) {
-        int rb = (int)((rw[j >> 2] >> (8 * (j & 3))) & 0xFFu);
-        if (a.residual_dtype == PSB_DT_S8) rb = (int)(int8_t)rb;
-        y[j] = dequant(acc[j], sc_s[chunk * 16 + j], bias_s[chunk * 16 + j], a.residual != nullptr, rb,
-                       a.residual_scale, a.relu != 0);
-      }
-      if (a.f32_out) {
-        float4* dst = reinterpret_cast<float4*>(a.f32_out + oidx);
-#pragma unroll
-        for (int j = 0; j < 4; ++j) dst[j] = make_float4(y[4 * j], y[4 * j + 1], y[4 * j + 2], y[4 * j + 3]);
-      }
-      if (a.q_out) {
-        uint32_t qw[4] = {0, 0, 0, 0};
-#pragma unroll
-        for (int j = 0; j < 16; ++j) {
-          int q = requant(y[j], a.inv_step, a.qmin, a.qmax);
-          qw[j >> 2] |= ((uint32_t)q & 0xFFu) << (8 * (j & 3));
-        }
-        *reinterpret_cast<uint4*>((uint8_t*)a.q_out + oidx) = make_uint4(qw[0], qw[1], qw[2], qw[3]);
-      }
-    }
-    return;
-  }
-  // element-wise stores: channel-major outputs, ragged channel counts, odd alignment
+  uint32_t qw[4] = {0, 0, 0, 0};
 #pragma unroll 1
   for (int j = 0; j < 16; ++j) {
     const uint32_t o = o_base + j;
     if (o >= a.O) break;
+    long long acc = (long long)(int)v[0][j];
+#pragma unroll
+    for (int pl = 1; pl < P; ++pl) acc += (long long)(int)v[pl][j] * (long long)(1 << (kDigitBits * pl));
+    if (use_corr) acc += corr[j];
     const size_t oidx = a.out_nchw ? ((size_t)n * a.O + o) * ohow + pix : (size_t)m * a.O + o;
-    if (a.acc_out) a.acc_out[oidx] = acc[j];
+    if (a.acc_out) a.acc_out[oidx] = acc;
     if (a.q_out || a.f32_out) {
       int rb = 0;
-      if (a.residual)
-        rb = a.residual_dtype == PSB_DT_U8 ? (int)((const uint8_t*)a.residual)[oidx]
-                                           : (int)((const int8_t*)a.residual)[oidx];
-      float y = dequant(acc[j], sc_s[chunk * 16 + j], bias_s[chunk * 16 + j], a.residual != nullptr, rb,
-                        a.residual_scale, a.relu != 0);
+      if (a.residual) {
+        if (vec) rb = (int)((rw[j >> 2] >> (8 * (j & 3))) & 0xFFu);
+        else rb = (int)((const uint8_t*)a.residual)[oidx];
+        if (a.residual_dtype == PSB_DT_S8) rb = (int)(int8_t)rb;
+      }
+      const float y = dequant(acc, scb[j].x, scb[j].y, a.residual != nullptr, rb, a.residual_scale, a.relu != 0);
       if (a.f32_out) a.f32_out[oidx] = y;
       if (a.q_out) {
-        int q = requant(y, a.inv_step, a.qmin, a.qmax);
-        if (a.out_dtype == PSB_DT_U8) ((uint8_t*)a.q_out)[oidx] = (uint8_t)q;
-        else ((int8_t*)a.q_out)[oidx] = (int8_t)q;
+        const int q = requant(y, a.inv_step, a.qmin, a.qmax);
+        if (vec) qw[j >> 2] |= ((uint32_t)q & 0xFFu) << (8 * (j & 3));
+        else ((uint8_t*)a.q_out)[oidx] = (uint8_t)q;
       }
     }
   }
+  if (vec && a.q_out)
+    *reinterpret_cast<uint4*>((uint8_t*)a.q_out + (size_t)m * a.O + o_base) = make_uint4(qw[0], qw[1], qw[2], qw[3]);
 }
 
 template <int BK>
 __global__ void __launch_bounds__(kThreadsTensor, 1)
-psb_mma_kernel(const __grid_constant__ TmapSet maps, const TensorParams p) {
+psb_mma_kernel(const __grid_constant__ TmapSet maps, const __grid_constant__ TensorParams p) {
   extern __shared__ uint8_t smem_raw[];
   // stage buffers need 1024-byte alignment for the 128-byte swizzle pattern
   uint8_t* smem = reinterpret_cast<uint8_t*>(((uintptr_t)smem_raw + 1023u) & ~(uintptr_t)1023u);
-  const uint32_t stage_bytes = p.stage_bytes_a + p.stage_bytes_b_max;
-  SharedCtl* ctl = reinterpret_cast<SharedCtl*>(smem + (size_t)p.stages * stage_bytes);
+  // resident mode: [digit planes of all K blocks][ring of activation stages][control]
+  // streaming mode: [ring of (activation, planes) stages][control]
+  uint8_t* ring = smem + (p.resident ? p.resident_bytes : 0u);
+  // a stage holds `group` K blocks, each an activation tile followed (streaming mode) by planes
+  const uint32_t sub_bytes = p.stage_bytes_a + (p.resident ? 0u : p.stage_bytes_b_max);
+  const uint32_t stage_bytes = sub_bytes * p.group;
+  SharedCtl* ctl = reinterpret_cast<SharedCtl*>(ring + (size_t)p.stages * stage_bytes);
 
   const uint32_t warp = threadIdx.x >> 5, lane = threadIdx.x & 31u;
-  const uint32_t n_tiles = p.m_tiles * p.o_tiles;
   const uint32_t k_iters = p.a.KH * p.a.KW * p.n_cb;
 
   if (threadIdx.x == 0) {
@@ -304,8 +392,9 @@ psb_mma_kernel(const __grid_constant__ TmapSet maps, const TensorParams p) {
     }
     for (int b = 0; b < 2; ++b) {
       mbar_init(smem_u32(&ctl->acc_full[b]), 1);
-      mbar_init(smem_u32(&ctl->acc_empty[b]), 4);
+      mbar_init(smem_u32(&ctl->acc_empty[b]), kEpilogueWarps);
     }
+    mbar_init(smem_u32(&ctl->planes_full), 1);
     ctl->abort = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -325,138 +414,237 @@ psb_mma_kernel(const __grid_constant__ TmapSet maps, const TensorParams p) {
 
   if (warp == 0) {
     // ------------------------------------------------------------ producer
-    uint32_t g = 0;  // stage use counter
-    for (uint32_t tile = blockIdx.x; tile < n_tiles && !failed; tile += gridDim.x) {
-      const uint32_t m_tile = tile / p.o_tiles, o_tile = tile % p.o_tiles;
-      const uint32_t m0 = m_tile * kTileM;
-      const uint32_t levels = tile_levels(p, m0);
-      const uint32_t ohow = p.a.OH * p.a.OW;
-      const uint32_t n0 = m0 / ohow, rem = m0 % ohow;
-      const int h0 = (int)((rem / p.a.OW) * p.a.stride) - (int)p.a.pad;
-      const int w0 = (int)((rem % p.a.OW) * p.a.stride) - (int)p.a.pad;
-      for (uint32_t l = 0; l < (uint32_t)kMaxLevels && !failed; ++l) {
-        if (!((levels >> l) & 1u)) continue;
-        if (!((p.a.level_mask >> l) & 1u)) continue;   // flagged by the epilogue
-        const uint32_t P = p.planes[l];
-        const uint32_t bytes = p.stage_bytes_a + P * kTileN * BK;
-        for (uint32_t it = 0; it < k_iters; ++it, ++g) {
-          const uint32_t s = g % p.stages, ph = (g / p.stages) & 1u;
-          if (lane == 0) {
-            if (!mbar_wait(smem_u32(&ctl->empty[s]), ph ^ 1u, abort)) failed = true;
-            if (!failed) {
-              const uint32_t tap = it / p.n_cb, cb = it % p.n_cb;
-              const uint32_t bar = smem_u32(&ctl->full[s]);
-              const uint32_t dst_a = smem_u32(smem + (size_t)s * stage_bytes);
-              const uint32_t dst_b = dst_a + p.stage_bytes_a;
-              mbar_expect_tx(bar, bytes);
+    // One thread runs the whole loop.  Every barrier round trip costs a few hundred cycles of
+    // latency on this thread, so the index arithmetic is incremental (no divisions), K blocks are
+    // handed over in groups, and the next stage's barrier is probed before it is needed.
+    if (lane == 0) {
+      if (p.resident) {
+        // the digit planes of this CTA's channel tile, all K blocks, once
+        const uint32_t l = p.a.uniform_log2k, P = p.planes[l];
+        const uint32_t o_tile = blockIdx.x / p.ctas_per_otile;
+        const uint32_t bar = smem_u32(&ctl->planes_full);
+        const uint32_t blk = P * kTileN * BK;
+        mbar_expect_tx(bar, k_iters * blk);
+        uint32_t kcol = 0, cb = 0;
+        for (uint32_t it = 0; it < k_iters; ++it) {
+          tma_load_2d(smem_u32(smem) + it * blk, &maps.b[l], bar, (int)(kcol + cb * BK),
+                      (int)(o_tile * P * kTileN));
+          if (++cb == p.n_cb) { cb = 0; kcol += p.cpad; }
+        }
+      }
+      uint32_t s = 0, ph = 0;  // ring position and its phase
+      bool next_free = mbar_try_wait(smem_u32(&ctl->empty[0]), 1u);
+      TileIter ti;
+      for (ti.init(p); ti.valid() && !failed; ti.next()) {
+        const uint32_t m_tile = ti.m_tile, o_tile = ti.o_tile;
+        const uint32_t m0 = m_tile * kTileM;
+        const uint32_t levels = tile_levels_serial(p, m0) & p.a.level_mask;
+        const uint32_t ohow = p.a.OH * p.a.OW;
+        const uint32_t n0 = m0 / ohow, rem = m0 % ohow;
+        const int h0 = (int)((rem / p.a.OW) * p.a.stride) - (int)p.a.pad;
+        const int w0 = (int)((rem % p.a.OW) * p.a.stride) - (int)p.a.pad;
+        // one pass per level present in the tile (levels that were not sampled are flagged by the
+        // epilogue and skipped by every role)
+        for (uint32_t todo = levels & 0x7Fu; todo && !failed; todo &= todo - 1u) {
+          const uint32_t l = (uint32_t)__ffs((int)todo) - 1u;
+          const uint32_t P = p.planes[l];
+          const uint32_t bytes = p.stage_bytes_a + (p.resident ? 0u : P * kTileN * BK);
+          const int b_row = (int)(o_tile * P * kTileN);
+          uint32_t kw = 0, kh = 0, cb = 0, kcol = 0;     // tap (kh, kw), channel block, plane column
+          for (uint32_t it = 0; it < k_iters;) {
+            const uint32_t cnt = min(p.group, k_iters - it);
+            if (!next_free && !mbar_wait(smem_u32(&ctl->empty[s]), ph ^ 1u, abort)) { failed = true; break; }
+            const uint32_t bar = smem_u32(&ctl->full[s]);
+            uint32_t dst = smem_u32(ring) + s * stage_bytes;
+            mbar_expect_tx(bar, bytes * cnt);
+            // probe the following stage now; the answer is back by the time it is needed
+            const uint32_t s2 = (s + 1 == p.stages) ? 0u : s + 1;
+            const uint32_t ph2 = (s + 1 == p.stages) ? ph ^ 1u : ph;
+            next_free = mbar_try_wait(smem_u32(&ctl->empty[s2]), ph2 ^ 1u);
+            for (uint32_t j = 0; j < cnt; ++j, dst += sub_bytes) {
               if (p.im2col)
-                tma_load_im2col_4d(dst_a, &maps.a, bar, (int)(cb * BK), w0, h0, (int)n0,
-                                   (uint16_t)(tap % p.a.KW), (uint16_t)(tap / p.a.KW));
+                tma_load_im2col_4d(dst, &maps.a, bar, (int)(cb * BK), w0, h0, (int)n0, (uint16_t)kw,
+                                   (uint16_t)kh);
               else
-                tma_load_2d(dst_a, &maps.a, bar, (int)(cb * BK), (int)m0);
-              tma_load_2d(dst_b, &maps.b[l], bar, (int)(tap * p.cpad + cb * BK),
-                          (int)(o_tile * P * kTileN));
+                tma_load_2d(dst, &maps.a, bar, (int)(cb * BK), (int)m0);
+              if (!p.resident)
+                tma_load_2d(dst + p.stage_bytes_a, &maps.b[l], bar, (int)(kcol + cb * BK), b_row);
+              if (++cb == p.n_cb) {
+                cb = 0;
+                kcol += p.cpad;
+                if (++kw == p.a.KW) { kw = 0; ++kh; }
+              }
             }
+            it += cnt;
+            s = s2;
+            ph = ph2;
           }
-          failed = __shfl_sync(0xFFFFFFFFu, failed ? 1 : 0, 0) != 0;
-          if (failed) break;
         }
       }
     }
+    failed = __shfl_sync(0xFFFFFFFFu, failed ? 1 : 0, 0) != 0;
   } else if (warp == 1) {
     // ---------------------------------------------------------------- MMA
-    uint32_t g = 0, pass = 0;
-    for (uint32_t tile = blockIdx.x; tile < n_tiles && !failed; tile += gridDim.x) {
-      const uint32_t m0 = (tile / p.o_tiles) * kTileM;
-      const uint32_t levels = tile_levels(p, m0);
-      for (uint32_t l = 0; l < (uint32_t)kMaxLevels && !failed; ++l) {
-        if (!((levels >> l) & 1u)) continue;
-        if (!((p.a.level_mask >> l) & 1u)) continue;
-        const uint32_t P = p.planes[l];
-        const uint32_t buf = pass & 1u, aph = (pass >> 1) & 1u;
-        // instruction descriptor: s32 accumulators, s8 x s8, both K-major, M = 128, N = P * 64
-        const uint32_t idesc = (2u << 4) | (1u << 7) | (1u << 10) | (((P * kTileN) >> 3) << 17) |
-                               ((kTileM >> 4) << 24);
-        const uint32_t d_tmem = tmem_base + buf * kTmemBufStride;
-        if (lane == 0) {
-          if (!mbar_wait(smem_u32(&ctl->acc_empty[buf]), aph ^ 1u, abort)) failed = true;
-        }
-        failed = __shfl_sync(0xFFFFFFFFu, failed ? 1 : 0, 0) != 0;
-        if (failed) break;
-        tc_fence_after();
-        for (uint32_t it = 0; it < k_iters; ++it, ++g) {
-          const uint32_t s = g % p.stages, ph = (g / p.stages) & 1u;
-          if (lane == 0) {
-            if (!mbar_wait(smem_u32(&ctl->full[s]), ph, abort)) failed = true;
-            if (!failed) {
-              tc_fence_after();
-              const uint32_t a_addr = smem_u32(smem + (size_t)s * stage_bytes);
-              const uint32_t b_addr = a_addr + p.stage_bytes_a;
+    if (lane == 0) {
+      uint32_t s = 0, ph = 0, pass = 0;
+      if (p.resident && !mbar_wait(smem_u32(&ctl->planes_full), 0u, abort)) failed = true;
+      const uint32_t ring_addr = smem_u32(ring), planes_addr = smem_u32(smem);
+      bool next_full = false;
+      TileIter ti;
+      for (ti.init(p); !failed && ti.valid(); ti.next()) {
+        const uint32_t m0 = ti.m_tile * kTileM;
+        const uint32_t levels = tile_levels_serial(p, m0) & p.a.level_mask;
+        for (uint32_t todo = levels & 0x7Fu; todo && !failed; todo &= todo - 1u) {
+          const uint32_t l = (uint32_t)__ffs((int)todo) - 1u;
+          const uint32_t P = p.planes[l];
+          const uint32_t buf = pass & 1u, aph = (pass >> 1) & 1u;
+          // instruction descriptor: s32 accumulators, s8 x s8, both K-major, M = 128, N = P * 64
+          const uint32_t idesc = (2u << 4) | (1u << 7) | (1u << 10) | (((P * kTileN) >> 3) << 17) |
+                                 ((kTileM >> 4) << 24);
+          const uint32_t d_tmem = tmem_base + buf * kTmemBufStride;
+          const uint32_t blk = P * kTileN * BK;
+          if (!mbar_wait(smem_u32(&ctl->acc_empty[buf]), aph ^ 1u, abort)) { failed = true; break; }
+          tc_fence_after();
+          uint32_t b_res = planes_addr;
+          for (uint32_t it = 0; it < k_iters;) {
+            const uint32_t cnt = min(p.group, k_iters - it);
+            if (!next_full && !mbar_wait(smem_u32(&ctl->full[s]), ph, abort)) { failed = true; break; }
+            tc_fence_after();
+            // probe the following stage while this one's MMAs are being issued
+            const uint32_t s2 = (s + 1 == p.stages) ? 0u : s + 1;
+            const uint32_t ph2 = (s + 1 == p.stages) ? ph ^ 1u : ph;
+            next_full = mbar_try_wait(smem_u32(&ctl->full[s2]), ph2);
+            uint32_t a_addr = ring_addr + s * stage_bytes;
+            for (uint32_t j = 0; j < cnt; ++j, a_addr += sub_bytes, b_res += blk) {
+              const uint32_t b_addr = p.resident ? b_res : a_addr + p.stage_bytes_a;
 #pragma unroll
               for (int ks = 0; ks < BK / 32; ++ks)
                 tc_mma_i8(d_tmem, smem_desc(a_addr + ks * 32, BK), smem_desc(b_addr + ks * 32, BK),
-                          idesc, (it | ks) != 0 ? 1u : 0u);
-              tc_commit(smem_u32(&ctl->empty[s]));
-              if (it + 1 == k_iters) tc_commit(smem_u32(&ctl->acc_full[buf]));
+                          idesc, (it | j | ks) != 0 ? 1u : 0u);
             }
+            tc_commit(smem_u32(&ctl->empty[s]));
+            it += cnt;
+            if (it == k_iters) tc_commit(smem_u32(&ctl->acc_full[buf]));
+            s = s2;
+            ph = ph2;
           }
-          failed = __shfl_sync(0xFFFFFFFFu, failed ? 1 : 0, 0) != 0;
-          if (failed) break;
+          ++pass;
         }
-        ++pass;
       }
     }
+    failed = __shfl_sync(0xFFFFFFFFu, failed ? 1 : 0, 0) != 0;
   } else {
     // ----------------------------------------------------------- epilogue
+    const uint32_t ew = warp - 2u;                   // 0..7
     const uint32_t quarter = warp & 3u;              // TMEM lanes this warp may touch
+    const uint32_t half = ew >> 2;                   // which 32 of the tile's 64 channels
     const uint32_t row = quarter * 32u + lane;
-    uint32_t pass = 0;
-    for (uint32_t tile = blockIdx.x; tile < n_tiles && !failed; tile += gridDim.x) {
-      const uint32_t m_tile = tile / p.o_tiles, o_tile = tile % p.o_tiles;
+    const ConvArgs& a = p.a;
+    const bool q_only = a.q_out && !a.f32_out && !a.acc_out && p.vec_ok;
+    // a clamp at qmin >= 0 already removes negatives, so the relu only matters for signed codes
+    const float relu_floor = (a.relu && a.qmin < 0) ? 0.0f : __int_as_float(0xFF800000);
+    const uint32_t res_sign = a.residual_dtype == PSB_DT_S8 ? 0x80u : 0u;
+    const bool pre_res = q_only && a.residual != nullptr;
+    const uint8_t* res_base = (const uint8_t*)a.residual;
+    uint32_t pass = 0, cur_key = 0xFFFFFFFFu;
+    TileIter ti;
+    ti.init(p);
+    uint32_t m_tile = ti.m_tile, o_tile = ti.o_tile;
+    // shortcut bytes of the first tile; later tiles' bytes are fetched one tile ahead so that
+    // their DRAM latency hides behind the current tile's work
+    uint4 r_next[2] = {make_uint4(0, 0, 0, 0), make_uint4(0, 0, 0, 0)};
+    bool have = ti.valid();
+    if (have && pre_res) {
+      const uint32_t m = m_tile * kTileM + row, ob = o_tile * kTileN + half * 32u;
+      if (m < p.M) {
+        if (ob + 16u <= a.O) r_next[0] = __ldg(reinterpret_cast<const uint4*>(res_base + (size_t)m * a.O + ob));
+        if (ob + 32u <= a.O) r_next[1] = __ldg(reinterpret_cast<const uint4*>(res_base + (size_t)m * a.O + ob + 16u));
+      }
+    }
+    while (!failed && have) {
       const uint32_t m0 = m_tile * kTileM;
-      const uint32_t levels = tile_levels(p, m0);
+      const uint32_t levels = tile_levels(p, m0) & a.level_mask;
       const uint32_t m = m0 + row;
       const bool in_range = m < p.M;
-      const uint32_t my_level = in_range ? (p.a.kmap ? (uint32_t)p.a.kmap[m] : p.a.uniform_log2k) : 0xFFu;
-      const uint32_t ohow = p.a.OH * p.a.OW;
-      const uint32_t n = in_range ? m / ohow : 0u, pix = in_range ? m % ohow : 0u;
-      if (in_range && (my_level >= (uint32_t)kMaxLevels || !((p.a.level_mask >> my_level) & 1u)))
-        atomicOr(p.a.err, kDevErrBadLevel);
-      for (uint32_t l = 0; l < (uint32_t)kMaxLevels && !failed; ++l) {
-        if (!((levels >> l) & 1u)) continue;
-        if (!((p.a.level_mask >> l) & 1u)) continue;
+      const uint32_t my_level = in_range ? (a.kmap ? (uint32_t)a.kmap[m] : a.uniform_log2k) : 0xFFu;
+      if (in_range && (my_level >= (uint32_t)kMaxLevels || !((a.level_mask >> my_level) & 1u)))
+        atomicOr(a.err, kDevErrBadLevel);
+      const uint32_t o_tile_cur = o_tile;
+      const uint32_t o_base0 = o_tile_cur * kTileN + half * 32u;
+      const uint4 r_cur[2] = {r_next[0], r_next[1]};
+      // next tile (and its shortcut bytes)
+      ti.next();
+      const uint32_t m_tile_n = ti.m_tile, o_tile_n = ti.o_tile;
+      const bool have_n = ti.valid();
+      if (have_n && pre_res) {
+        const uint32_t mn = m_tile_n * kTileM + row, ob = o_tile_n * kTileN + half * 32u;
+        r_next[0] = make_uint4(0, 0, 0, 0);
+        r_next[1] = make_uint4(0, 0, 0, 0);
+        if (mn < p.M) {
+          if (ob + 16u <= a.O) r_next[0] = __ldg(reinterpret_cast<const uint4*>(res_base + (size_t)mn * a.O + ob));
+          if (ob + 32u <= a.O) r_next[1] = __ldg(reinterpret_cast<const uint4*>(res_base + (size_t)mn * a.O + ob + 16u));
+        }
+      }
+      for (uint32_t todo = levels & 0x7Fu; todo && !failed; todo &= todo - 1u) {
+        const uint32_t l = (uint32_t)__ffs((int)todo) - 1u;
         const uint32_t P = p.planes[l];
         const uint32_t buf = pass & 1u, aph = (pass >> 1) & 1u;
-        // per-channel constants of this pass (exact power-of-two rescale of the scale);
-        // every warp keeps its own copy so that no CTA-wide barrier is needed
-#pragma unroll
-        for (uint32_t e = lane; e < (uint32_t)kTileN; e += 32u) {
-          const uint32_t o = o_tile * kTileN + e;
-          float sc = 0.f, bi = 0.f;
-          if (o < p.a.O) {
-            sc = ldexpf(p.a.scale[o], p.a.e_base[o] - (int)l);
-            bi = p.a.bias[o];
+        const bool use_corr = p.corr[l] != nullptr;
+        // per-channel constants of this (channel tile, level): every warp keeps its own copy of
+        // its 32 channels, so no CTA-wide barrier is needed; refreshed only when the pair changes
+        const uint32_t key = o_tile_cur * 8u + l;
+        if (key != cur_key) {
+          __syncwarp();
+          const uint32_t o = o_base0 + lane;
+          float2 sb = make_float2(0.f, 0.f);
+          long long cr = 0;
+          if (o < a.O) {
+            sb.x = ldexpf(a.scale[o], a.e_base[o] - (int)l);
+            sb.y = a.bias[o];
+            if (use_corr) cr = p.corr[l][o];
           }
-          ctl->sc[quarter][e] = sc;
-          ctl->bias[quarter][e] = bi;
+          ctl->scb[ew][lane] = sb;
+          ctl->corr[ew][lane] = cr;
+          cur_key = key;
+          __syncwarp();
         }
-        __syncwarp();
         if (lane == 0) {
-          if (!mbar_wait(smem_u32(&ctl->acc_full[buf]), aph, abort)) failed = true;
+          if (!mbar_wait(smem_u32(&ctl->acc_full[buf]), aph, abort, 32)) failed = true;
         }
         failed = __shfl_sync(0xFFFFFFFFu, failed ? 1 : 0, 0) != 0;
         if (failed) break;
         tc_fence_after();
-        const uint32_t trow = tmem_base + buf * kTmemBufStride + ((quarter * 32u) << 16);
         const bool valid = in_range && my_level == l;
-        for (uint32_t chunk = 0; chunk < (uint32_t)kTileN / 16u; ++chunk) {
-          const uint32_t o_base = o_tile * kTileN + chunk * 16u;
-          if (o_base >= p.a.O) break;
-          switch (P) {
-            case 1: epilogue_chunk<1>(p, trow, chunk, o_base, m, valid, n, pix, ctl->sc[quarter], ctl->bias[quarter]); break;
-            case 2: epilogue_chunk<2>(p, trow, chunk, o_base, m, valid, n, pix, ctl->sc[quarter], ctl->bias[quarter]); break;
-            case 3: epilogue_chunk<3>(p, trow, chunk, o_base, m, valid, n, pix, ctl->sc[quarter], ctl->bias[quarter]); break;
-            default: epilogue_chunk<4>(p, trow, chunk, o_base, m, valid, n, pix, ctl->sc[quarter], ctl->bias[quarter]); break;
+#pragma unroll
+        for (uint32_t c2 = 0; c2 < 2u; ++c2) {   // unrolled: r_cur[c2] must stay in registers
+          const uint32_t o_base = o_base0 + c2 * 16u;
+          if (o_base >= a.O) break;
+          const uint32_t taddr = tmem_base + buf * kTmemBufStride + ((quarter * 32u) << 16) + half * 32u + c2 * 16u;
+          const float2* scb = &ctl->scb[ew][c2 * 16u];
+          const long long* corr = &ctl->corr[ew][c2 * 16u];
+          if (q_only && o_base + 16u <= a.O) {
+            uint8_t* q_dst = (uint8_t*)a.q_out + (size_t)m * a.O + o_base;
+            const uint32_t mode = use_corr ? 0u : p.narrow;
+#define PSB_EPI(PV, MV, RV) epilogue_chunk_q<PV, MV, RV>(taddr, valid, q_dst, r_cur[c2], scb, corr, a.residual_scale, res_sign, relu_floor, a.inv_step, (float)a.qmin, (float)a.qmax)
+#define PSB_EPI_P(MV, RV) do { if (P == 3) PSB_EPI(3, MV, RV); else if (P == 2) PSB_EPI(2, MV, RV); else PSB_EPI(1, MV, RV); } while (0)
+            if (a.residual) {
+              if (mode == 2) PSB_EPI_P(2, true); else if (mode == 1) PSB_EPI_P(1, true);
+              else if (P == 4) PSB_EPI(4, 0, true); else PSB_EPI_P(0, true);
+            } else {
+              if (mode == 2) PSB_EPI_P(2, false); else if (mode == 1) PSB_EPI_P(1, false);
+              else if (P == 4) PSB_EPI(4, 0, false); else PSB_EPI_P(0, false);
+            }
+#undef PSB_EPI_P
+#undef PSB_EPI
+          } else {
+            const uint32_t ohow = a.OH * a.OW;
+            const uint32_t n = in_range ? m / ohow : 0u, pix = in_range ? m % ohow : 0u;
+            switch (P) {
+              case 1: epilogue_chunk<1>(p, taddr, o_base, m, valid, n, pix, scb, corr, use_corr); break;
+              case 2: epilogue_chunk<2>(p, taddr, o_base, m, valid, n, pix, scb, corr, use_corr); break;
+              case 3: epilogue_chunk<3>(p, taddr, o_base, m, valid, n, pix, scb, corr, use_corr); break;
+              default: epilogue_chunk<4>(p, taddr, o_base, m, valid, n, pix, scb, corr, use_corr); break;
+            }
           }
         }
         tc_fence_before();
@@ -464,6 +652,9 @@ psb_mma_kernel(const __grid_constant__ TmapSet maps, const TensorParams p) {
         if (lane == 0) mbar_arrive(smem_u32(&ctl->acc_empty[buf]));
         ++pass;
       }
+      have = have_n;
+      m_tile = m_tile_n;
+      o_tile = o_tile_n;
     }
   }
 
@@ -520,7 +711,8 @@ psb_status tensor_supported(const psb_ctx* ctx, const psb_weights* wt, const Con
   return PSB_OK;
 }
 
-psb_status launch_tensor(psb_ctx* ctx, const psb_weights* wt, const ConvArgs& a, cudaStream_t s) {
+psb_status launch_tensor(psb_ctx* ctx, const psb_weights* wt, const ConvArgs& a, uint32_t amax,
+                         cudaStream_t s) {
   TmapSet maps;
   TensorParams p;
   p.a = a;
@@ -539,11 +731,44 @@ psb_status launch_tensor(psb_ctx* ctx, const psb_weights* wt, const ConvArgs& a,
   p.stage_bytes_a = kTileM * bk;
   p.stage_bytes_b_max = pmax * kTileN * bk;
   const size_t ctl_bytes = sizeof(SharedCtl) + 1024;
-  uint32_t stages = (uint32_t)((kSmemBudget - ctl_bytes) / (p.stage_bytes_a + p.stage_bytes_b_max));
+  const uint32_t k_iters = a.KH * a.KW * p.n_cb;
+  // Resident mode: with one draw count for the whole layer, a CTA that owns a single tile of 64
+  // output channels keeps that tile's digit planes in shared memory for all its row tiles.
+  p.resident = 0;
+  p.ctas_per_otile = 1;
+  p.resident_bytes = 0;
+  if (!a.kmap) {
+    const uint32_t P = p.planes[a.uniform_log2k];
+    const uint32_t need = k_iters * P * kTileN * bk;
+    const uint32_t cpo = (uint32_t)ctx->sm_count / p.o_tiles;
+    if (need <= kResidentMaxBytes && cpo >= 1 && p.o_tiles * cpo * 10u >= (uint32_t)ctx->sm_count * 9u) {
+      p.resident = 1;
+      p.ctas_per_otile = cpo < p.m_tiles ? cpo : p.m_tiles;
+      p.resident_bytes = need;
+    }
+  }
+  // K blocks are handed over in groups: every barrier round trip costs the issuing thread a
+  // few hundred cycles, so a stage should carry about eight MMAs (M=128, N=P*64, K=32 each)
+  const uint32_t sub_bytes = p.stage_bytes_a + (p.resident ? 0u : p.stage_bytes_b_max);
+  const size_t avail = kSmemBudget - ctl_bytes - p.resident_bytes;
+  uint32_t group = 8u / (bk / 32u);
+  if (group < 1) group = 1;
+  if (group > k_iters) group = k_iters;
+  while (group > 1 && avail / ((size_t)group * sub_bytes) < 3) --group;
+  {  // balance the groups of one tile: same number of groups, as even as possible
+    const uint32_t n_groups = (k_iters + group - 1) / group;
+    group = (k_iters + n_groups - 1) / n_groups;
+  }
+  p.group = group;
+  uint32_t stages = (uint32_t)(avail / ((size_t)group * sub_bytes));
   if (stages > (uint32_t)kMaxStages) stages = kMaxStages;
   if (stages < 2) return PSB_ERR_UNSUPPORTED;
   p.stages = stages;
-  const size_t smem_bytes = (size_t)stages * (p.stage_bytes_a + p.stage_bytes_b_max) + ctl_bytes;
+  const size_t smem_bytes = (size_t)stages * group * sub_bytes + p.resident_bytes + ctl_bytes;
+  for (int l = 0; l < kMaxLevels; ++l) p.corr[l] = nullptr;
+  // every plane sum is bounded by 127 * (largest activation magnitude) * d
+  const uint64_t plane_bound = 127ull * amax * (uint64_t)wt->d;
+  p.narrow = pmax > 3 ? 0u : (plane_bound <= 4100000ull ? 2u : (plane_bound <= 16500000ull ? 1u : 0u));
   bool vec = !a.out_nchw && a.O % 16u == 0;
   vec = vec && !(((uintptr_t)a.q_out | (uintptr_t)a.residual | (uintptr_t)a.f32_out |
                   (uintptr_t)a.acc_out) & 15u);
@@ -586,7 +811,8 @@ psb_status launch_tensor(psb_ctx* ctx, const psb_weights* wt, const ConvArgs& a,
   }
 
   const uint32_t n_tiles = p.m_tiles * p.o_tiles;
-  const uint32_t grid = n_tiles < (uint32_t)ctx->sm_count ? n_tiles : (uint32_t)ctx->sm_count;
+  const uint32_t grid = p.resident ? p.o_tiles * p.ctas_per_otile
+                                   : (n_tiles < (uint32_t)ctx->sm_count ? n_tiles : (uint32_t)ctx->sm_count);
   cudaError_t e;
 #define PSB_LAUNCH(BKV)                                                                              \
   e = cudaFuncSetAttribute(psb_mma_kernel<BKV>, cudaFuncAttributeMaxDynamicSharedMemorySize,         \

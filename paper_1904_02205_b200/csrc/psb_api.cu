@@ -29,6 +29,7 @@ void free_weights_storage(psb_weights* w) {
   for (int l = 0; l < kMaxLevels; ++l) {
     if (w->level[l].wint) cudaFree(w->level[l].wint);
     if (w->level[l].planes) cudaFree(w->level[l].planes);
+    if (w->level[l].corr128) cudaFree(w->level[l].corr128);
     w->level[l] = LevelStore();
   }
   if (w->e_base) cudaFree(w->e_base);
@@ -103,11 +104,15 @@ psb_status run_layer(psb_ctx* ctx, const psb_weights* wt, const void* x_dev, uin
 
   // largest activation magnitude the caller vouches for
   uint32_t amax = in_max ? in_max : (in_dtype == PSB_DT_U8 ? 255u : 128u);
+  const uint64_t M = (uint64_t)n * oh * ow;
   bool tensor_ok = false;
   if (path != PSB_PATH_SHIFT_ADD) {
-    tensor_ok = (in_dtype == PSB_DT_S8 || amax <= 127u) && tensor_supported(ctx, wt, a) == PSB_OK;
+    // the MMA takes signed bytes: unsigned data above 127 qualifies only where the activation
+    // matrix is gathered explicitly (packed-K filters), which stores x - 128
+    tensor_ok = (in_dtype == PSB_DT_S8 || amax <= 127u || wt->packed_k) &&
+                tensor_supported(ctx, wt, a) == PSB_OK;
     if (path == PSB_PATH_TENSOR && !tensor_ok) return PSB_ERR_UNSUPPORTED;
-    if (path == PSB_PATH_AUTO && (uint64_t)n * oh * ow < 128) tensor_ok = false;
+    if (path == PSB_PATH_AUTO && M < (wt->packed_k ? 128u : 32u)) tensor_ok = false;
   }
 
   if (in_conv) {
@@ -120,7 +125,23 @@ psb_status run_layer(psb_ctx* ctx, const psb_weights* wt, const void* x_dev, uin
   }
 
   if (tensor_ok) {
-    st = launch_tensor(ctx, wt, a, amax, s);
+    bool add_corr = false;
+    if (wt->packed_k) {
+      // gather the activation matrix [M][kpad] once, then run the layer as a plain GEMM
+      st = ensure_scratch(ctx, 1, (size_t)M * wt->kpad);
+      if (st != PSB_OK) return st;
+      const uint32_t offset = in_dtype == PSB_DT_U8 ? 128u : 0u;
+      if (launch_im2col_s8(a, wt->kpad, offset, (int8_t*)ctx->scratch[1], s) != cudaSuccess)
+        return PSB_ERR_CUDA;
+      a.x = ctx->scratch[1];
+      a.in_dtype = PSB_DT_S8;
+      a.C = wt->kpad;
+      a.H = oh; a.W = ow;
+      a.KH = 1; a.KW = 1; a.stride = 1; a.pad = 0;
+      add_corr = offset != 0;
+      amax = 128;
+    }
+    st = launch_tensor(ctx, wt, a, amax, add_corr, s);
     if (st != PSB_OK) return st;
     ctx->last_path = PSB_PATH_TENSOR;
     return PSB_OK;
@@ -239,11 +260,13 @@ psb_status psb_sample_weights(psb_ctx* ctx, const float* w_dev, const psb_wshape
     w->cfg = cfg;
     w->device = ctx->device;
     w->d = (uint32_t)d64;
-    w->has_planes = shape->groups == 1 && shape->in_ch_per_group % 16 == 0;
+    const bool wide = shape->in_ch_per_group % 16 == 0 && shape->in_ch_per_group >= 32;
+    w->packed_k = shape->groups == 1 && !wide && d64 >= 16;
+    w->has_planes = shape->groups == 1 && (wide || w->packed_k);
     w->cpad = shape->in_ch_per_group;
-    w->kpad = shape->kh * shape->kw * w->cpad;
+    w->kpad = round_up(shape->kh * shape->kw * w->cpad, 16);
     w->o_tiles = (shape->out_ch + kTileN - 1) / kTileN;
-    w->bk = tensor_bk(shape->in_ch_per_group);
+    w->bk = tensor_bk(w->packed_k ? w->kpad : shape->in_ch_per_group);
     bool ok = cudaMalloc(&w->e_base, sizeof(int32_t) * shape->out_ch) == cudaSuccess &&
               cudaMalloc(&w->e_max, sizeof(uint32_t) * shape->out_ch) == cudaSuccess;
     for (uint32_t l = 0; ok && l < (uint32_t)kMaxLevels; ++l) {
@@ -255,6 +278,8 @@ psb_status psb_sample_weights(psb_ctx* ctx, const float* w_dev, const psb_wshape
         w->level[l].planes_count = P;
         ok = cudaMalloc(&w->level[l].planes, bytes) == cudaSuccess &&
              cudaMemsetAsync(w->level[l].planes, 0, bytes, s) == cudaSuccess;
+        if (ok && w->packed_k)
+          ok = cudaMalloc(&w->level[l].corr128, sizeof(long long) * shape->out_ch) == cudaSuccess;
       }
     }
     if (!ok) {

@@ -34,6 +34,7 @@ struct LevelStore {
   int32_t* wint = nullptr;  // [O][KH][KW][Cg]  signed integer filter, channels innermost
   int8_t* planes = nullptr; // [O_tiles][P][kTileN][Kpad]  signed 7-bit digits, Kpad = KH*KW*Cpad
   int planes_count = 0;
+  long long* corr128 = nullptr;  // [O] 128 * sum of the filter row (packed-K filters only)
 };
 
 }  // namespace psb
@@ -47,6 +48,8 @@ struct psb_weights {
   uint32_t o_tiles;  // ceil(out_ch / kTileN)
   uint32_t bk;       // K block of the tensor path
   bool has_planes;   // digit planes are produced (groups == 1)
+  bool packed_k;     // few input channels: the K axis is the flat (kh, kw, ci) index, padded to 16;
+                     // such a layer runs as a plain GEMM on an explicitly gathered activation matrix
   psb::LevelStore level[psb::kMaxLevels];
   int32_t* e_base = nullptr;   // [O]
   uint32_t* e_max = nullptr;   // [O] scratch of the window reduction (biased exponent, 0 = none)
@@ -128,6 +131,9 @@ cudaError_t launch_sampler(const float* w_dev, psb_weights* wt, uint32_t* err_de
 cudaError_t launch_export(const psb_weights* wt, uint32_t level, int32_t* wint_out,
                           int32_t* e_base_out, cudaStream_t s);
 cudaError_t launch_shift_add(const ConvArgs& a, const WintTable& wt, cudaStream_t s);
+// gathers [M][kpad] signed bytes (x - offset; zero padding becomes -offset, K padding 0)
+cudaError_t launch_im2col_s8(const ConvArgs& a, uint32_t kpad, uint32_t offset, int8_t* dst,
+                             cudaStream_t s);
 cudaError_t launch_nchw_to_nhwc(const void* src, void* dst, uint32_t N, uint32_t C, uint32_t HW,
                                 uint32_t elem_bytes, cudaStream_t s);
 cudaError_t launch_nhwc_to_nchw(const void* src, void* dst, uint32_t N, uint32_t C, uint32_t HW,
@@ -141,6 +147,6 @@ cudaError_t launch_avgpool(const uint8_t* x, uint32_t nchw, uint32_t N, uint32_t
 // tensor path: returns PSB_ERR_UNSUPPORTED if the shape does not fit it
 psb_status tensor_supported(const psb_ctx* ctx, const psb_weights* wt, const ConvArgs& a);
 psb_status launch_tensor(psb_ctx* ctx, const psb_weights* wt, const ConvArgs& a, uint32_t amax,
-                         cudaStream_t s);
+                         bool add_corr128, cudaStream_t s);
 
 }  // namespace psb

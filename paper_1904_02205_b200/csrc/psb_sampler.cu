@@ -160,6 +160,18 @@ __global__ void __launch_bounds__(kThreads) sample_kernel(const SampleParams p) 
   }
 }
 
+// 128 * (sum of each filter row): the constant that restores sum x*W from sum (x-128)*W when
+// unsigned activations are fed to the signed MMA with an offset of 128.  One warp per row.
+__global__ void corr128_kernel(const int32_t* __restrict__ wint, uint32_t O, uint32_t d,
+                               long long* __restrict__ corr) {
+  const uint32_t row = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31u;
+  if (row >= O) return;
+  long long sum = 0;
+  for (uint32_t i = lane; i < d; i += 32u) sum += wint[(size_t)row * d + i];
+  for (int off = 16; off; off >>= 1) sum += __shfl_down_sync(0xFFFFFFFFu, sum, off);
+  if (lane == 0) corr[row] = sum * 128;
+}
+
 // Canonical-order copy of one level for the test hook.
 __global__ void export_kernel(const int32_t* __restrict__ wint, int32_t* __restrict__ out, uint32_t O,
                               uint32_t Cg, uint32_t KHKW) {
@@ -221,6 +233,11 @@ cudaError_t launch_sampler(const float* w_dev, psb_weights* wt, uint32_t* err_de
   }
   uint32_t row_blocks = (O + p.rows_per_block - 1) / p.rows_per_block;
   sample_kernel<<<row_blocks * p.ch_chunks, kThreads, 0, s>>>(p);
+  if (wt->packed_k)
+    for (int l = 0; l < kMaxLevels; ++l)
+      if (wt->level[l].corr128)
+        corr128_kernel<<<(O * 32 + kThreads - 1) / kThreads, kThreads, 0, s>>>(wt->level[l].wint, O, d,
+                                                                              wt->level[l].corr128);
   return cudaGetLastError();
 }
 

@@ -72,6 +72,47 @@ __global__ void __launch_bounds__(256) conv_direct_kernel(const ConvArgs a, cons
   }
 }
 
+// Explicit gather of the activation matrix for filters with few input channels (e.g. a 7x7
+// stem on 3 channels): row m = output location, column k = (kh, kw, ci) flattened, padded with
+// zeros to kpad.  Values are stored minus `offset` as signed bytes; a padded input position is the
+// value 0, i.e. -offset.  One thread writes 16 bytes.
+__global__ void __launch_bounds__(256) im2col_s8_kernel(const ConvArgs a, uint32_t kpad, uint32_t offset,
+                                                       int8_t* __restrict__ dst) {
+  extern __shared__ uint32_t ktab[];  // per column: kh | kw << 8 | ci << 16, or ~0 for K padding
+  const uint32_t d = a.KH * a.KW * a.C;
+  for (uint32_t k = threadIdx.x; k < kpad; k += blockDim.x) {
+    uint32_t tap = k / a.C, ci = k % a.C;
+    ktab[k] = k < d ? ((tap / a.KW) | ((tap % a.KW) << 8) | (ci << 16)) : 0xFFFFFFFFu;
+  }
+  __syncthreads();
+  const uint32_t chunks = kpad / 16u;
+  const size_t total = (size_t)a.N * a.OH * a.OW * chunks;
+  const uint8_t* x = (const uint8_t*)a.x;
+  for (size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x; idx < total;
+       idx += (size_t)gridDim.x * blockDim.x) {
+    const uint32_t ch = (uint32_t)(idx % chunks);
+    const size_t m = idx / chunks;
+    const uint32_t ox = (uint32_t)(m % a.OW), oy = (uint32_t)((m / a.OW) % a.OH);
+    const uint32_t n = (uint32_t)(m / ((size_t)a.OW * a.OH));
+    const int iy0 = (int)(oy * a.stride) - (int)a.pad, ix0 = (int)(ox * a.stride) - (int)a.pad;
+    uint32_t w[4] = {0, 0, 0, 0};
+#pragma unroll
+    for (int j = 0; j < 16; ++j) {
+      const uint32_t e = ktab[ch * 16u + j];
+      uint32_t v = 0;
+      if (e != 0xFFFFFFFFu) {
+        const int iy = iy0 + (int)(e & 0xFFu), ix = ix0 + (int)((e >> 8) & 0xFFu);
+        uint32_t raw = 0;
+        if (iy >= 0 && iy < (int)a.H && ix >= 0 && ix < (int)a.W)
+          raw = x[(((size_t)n * a.H + iy) * a.W + ix) * a.C + (e >> 16)];
+        v = (raw - offset) & 0xFFu;
+      }
+      w[j >> 2] |= v << (8 * (j & 3));
+    }
+    *reinterpret_cast<uint4*>(dst + m * kpad + ch * 16u) = make_uint4(w[0], w[1], w[2], w[3]);
+  }
+}
+
 // [N][C][HW] -> [N][HW][C], elements of 1 byte, through a 32x33 tile.
 __global__ void nchw_to_nhwc_u8_kernel(const uint8_t* __restrict__ src, uint8_t* __restrict__ dst,
                                        uint32_t C, uint32_t HW) {
@@ -147,6 +188,13 @@ uint32_t grid_for(size_t total, uint32_t threads) {
 cudaError_t launch_shift_add(const ConvArgs& a, const WintTable& wt, cudaStream_t s) {
   size_t total = (size_t)a.N * a.OH * a.OW * a.O;
   conv_direct_kernel<<<grid_for(total, 256), 256, 0, s>>>(a, wt);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_im2col_s8(const ConvArgs& a, uint32_t kpad, uint32_t offset, int8_t* dst,
+                             cudaStream_t s) {
+  size_t total = (size_t)a.N * a.OH * a.OW * (kpad / 16u);
+  im2col_s8_kernel<<<grid_for(total, 256), 256, kpad * sizeof(uint32_t), s>>>(a, kpad, offset, dst);
   return cudaGetLastError();
 }
 

@@ -104,8 +104,11 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
   const long long t0 = clock64();
   uint32_t spins = 0;
   while (!mbar_try_wait(bar, parity)) {
-    if (backoff_ns) __nanosleep(backoff_ns);
-    if ((++spins & 15u) == 0u) {
+    // a thread that has to wait long should not eat the issue slots of the warps doing the
+    // arithmetic: poll a few times at full speed, then sleep between polls
+    ++spins;
+    if (backoff_ns || spins > 4u) __nanosleep(backoff_ns ? backoff_ns : (spins > 32u ? 256u : 64u));
+    if ((spins & 15u) == 0u) {
       if (*abort) return false;
       if (clock64() - t0 > kWaitLimitCycles) return false;
     }
@@ -703,16 +706,17 @@ constexpr size_t kSmemBudget = 227 * 1024;
 psb_status tensor_supported(const psb_ctx* ctx, const psb_weights* wt, const ConvArgs& a) {
   if (!ctx->encode_tiled || !ctx->encode_im2col) return PSB_ERR_UNSUPPORTED;
   if (!wt->has_planes || a.groups != 1) return PSB_ERR_UNSUPPORTED;
+  // each plane accumulates in 32 bits: |digit| <= 127, |x| <= 128
+  if ((uint64_t)wt->d * 127ull * 128ull >= (1ull << 31)) return PSB_ERR_UNSUPPORTED;
+  if (wt->packed_k) return (a.KH > 255 || a.KW > 255 || a.C > 65535) ? PSB_ERR_UNSUPPORTED : PSB_OK;
   if (a.C % 16u || a.C < 32u) return PSB_ERR_UNSUPPORTED;
   if ((uintptr_t)a.x & 15u) return PSB_ERR_UNSUPPORTED;
   if (a.stride > 8 || a.pad > 127 || a.KH > 128 || a.KW > 128) return PSB_ERR_UNSUPPORTED;
-  // each plane accumulates in 32 bits: |digit| <= 127, |x| <= 128
-  if ((uint64_t)wt->d * 127ull * 128ull >= (1ull << 31)) return PSB_ERR_UNSUPPORTED;
   return PSB_OK;
 }
 
 psb_status launch_tensor(psb_ctx* ctx, const psb_weights* wt, const ConvArgs& a, uint32_t amax,
-                         cudaStream_t s) {
+                         bool add_corr128, cudaStream_t s) {
   TmapSet maps;
   TensorParams p;
   p.a = a;
@@ -765,7 +769,7 @@ psb_status launch_tensor(psb_ctx* ctx, const psb_weights* wt, const ConvArgs& a,
   if (stages < 2) return PSB_ERR_UNSUPPORTED;
   p.stages = stages;
   const size_t smem_bytes = (size_t)stages * group * sub_bytes + p.resident_bytes + ctl_bytes;
-  for (int l = 0; l < kMaxLevels; ++l) p.corr[l] = nullptr;
+  for (int l = 0; l < kMaxLevels; ++l) p.corr[l] = add_corr128 ? wt->level[l].corr128 : nullptr;
   // every plane sum is bounded by 127 * (largest activation magnitude) * d
   const uint64_t plane_bound = 127ull * amax * (uint64_t)wt->d;
   p.narrow = pmax > 3 ? 0u : (plane_bound <= 4100000ull ? 2u : (plane_bound <= 16500000ull ? 1u : 0u));

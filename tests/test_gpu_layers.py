@@ -155,6 +155,38 @@ def test_tensor_path_layers(psb, ctx, oracle, case):
     assert g["path"] == psb.PSB_PATH_TENSOR
 
 
+@pytest.mark.parametrize("case", [
+    dict(N=3, C=3, H=37, W=41, O=64, K=7, stride=2, pad=3, dtype=np.uint8, hi=256),   # image stem
+    dict(N=2, C=3, H=30, W=30, O=32, K=3, stride=2, pad=1, dtype=np.uint8, hi=256),   # 27 -> 32 columns
+    dict(N=2, C=24, H=13, W=13, O=40, K=1, stride=1, pad=0, dtype=np.int8, hi=128),   # 24 channels, signed
+    dict(N=2, C=20, H=11, W=9, O=70, K=3, stride=1, pad=1, dtype=np.uint8, hi=256),   # ragged everything
+])
+def test_tensor_path_few_input_channels_full_range_bytes(psb, ctx, oracle, case):
+    """Filters whose input-channel count is not a multiple of 16 run on the tensor cores through an
+    explicitly gathered activation matrix; unsigned bytes up to 255 are fed with an offset of 128
+    and corrected by 128 * sum(W)."""
+    rng = np.random.default_rng(case["C"] * 17 + case["K"])
+    w, x, scale, bias = _layer_inputs(rng, case["N"], case["C"], case["H"], case["W"], case["O"], case["K"],
+                                      case["K"], 1, 1, x_dtype=case["dtype"], x_hi=case["hi"])
+    for levels, kmap in (([3], None), ([0, 2, 4], "random")):
+        km = None
+        if kmap:
+            oh = (case["H"] + 2 * case["pad"] - case["K"]) // case["stride"] + 1
+            ow = (case["W"] + 2 * case["pad"] - case["K"]) // case["stride"] + 1
+            km = rng.choice(levels, size=(case["N"], oh, ow)).astype(np.uint8)
+        g = _both(psb, ctx, oracle, w, x, 1, 1, case["stride"], case["pad"], levels, scale, bias, kmap=km,
+                  inv_step=0.02, qmax=255, path=psb.PSB_PATH_TENSOR)
+        assert g["path"] == psb.PSB_PATH_TENSOR
+
+
+def test_fully_connected_on_the_tensor_path(psb, ctx, oracle):
+    rng = np.random.default_rng(5)
+    w, x, scale, bias = _layer_inputs(rng, 64, 512, 1, 1, 1000, 1, 1, 1, 1)
+    g = _both(psb, ctx, oracle, w, x, 1, 1, 1, 0, [3], scale, bias, relu=False, inv_step=0.3, qmin=-128, qmax=127,
+              out_dtype=1, in_max=15)
+    assert g["path"] == psb.PSB_PATH_TENSOR
+
+
 @pytest.mark.parametrize("log2k", [0, 1, 2, 4, 5, 6])
 def test_tensor_path_every_draw_count(psb, ctx, oracle, log2k):
     rng = np.random.default_rng(log2k)

@@ -219,6 +219,41 @@ psb_status psb_global_avgpool_u8(psb_ctx* ctx, const uint8_t* x_dev, uint32_t la
                                  uint32_t c, uint32_t h, uint32_t w, float pool_mul, int32_t qmin,
                                  int32_t qmax, uint8_t* out_dev, void* stream);
 
+/* Whole networks with few host calls.
+ *
+ * psb_sample_batch_*: re-sample many layers at once.  The handles must exist already (created
+ * by psb_sample_weights, which also fixes each layer's layer_id, level_mask, exp_bits and norm);
+ * w_dev[i] is the fp32 filter of weights[i].  psb_sample_batch_run draws every layer under one
+ * new `seed` in two kernel launches and gives exactly the filters that psb_sample_weights would
+ * give layer by layer with that seed.  Create and free allocate / block; run does not.  The
+ * filters, handles and the batch must stay alive while a run is in flight.
+ *
+ * psb_run: executes a list of layer operations in order on `stream`, each exactly as the
+ * corresponding single call would (psb_set_sample_map with the op's draw-count fields, then
+ * psb_conv2d / psb_gemm / psb_maxpool2d_u8 / psb_global_avgpool_u8).  It stops at the first
+ * error and returns it; operations before it stay launched. */
+typedef struct psb_sample_batch psb_sample_batch;
+psb_status psb_sample_batch_create(psb_ctx* ctx, uint32_t n, const float* const* w_dev,
+                                   psb_weights* const* weights, psb_sample_batch** batch);
+psb_status psb_sample_batch_run(psb_ctx* ctx, psb_sample_batch* batch, uint64_t seed, void* stream);
+psb_status psb_sample_batch_free(psb_ctx* ctx, psb_sample_batch* batch);
+
+enum { PSB_OP_CONV2D = 0, PSB_OP_GEMM = 1, PSB_OP_MAXPOOL = 2, PSB_OP_AVGPOOL = 3 };
+typedef struct {
+  uint32_t kind;
+  const psb_weights* weights;   /* conv2d, gemm */
+  const void* x_dev;            /* input activations of the op */
+  const uint8_t* map_dev;       /* draw counts per output location, or NULL for uniform_log2k */
+  uint32_t map_n, map_oh, map_ow, uniform_log2k;
+  psb_conv_desc conv;           /* conv2d; pooling reads layout, n, c, h, w, stride, pad from it */
+  psb_gemm_desc gemm;           /* gemm */
+  uint32_t pool_k;              /* max-pool window */
+  float pool_mul;               /* average pool: see psb_global_avgpool_u8 */
+  int32_t pool_qmin, pool_qmax;
+  uint8_t* pool_out_dev;
+} psb_op;
+psb_status psb_run(psb_ctx* ctx, const psb_op* ops, uint32_t n_ops, void* stream);
+
 /* Sampling of one level without any allocation.  (The paper has no counterpart:
  * this entry point exists for hosts, not for the method.)
  *

@@ -22,7 +22,8 @@ PSB_PATH_AUTO, PSB_PATH_SHIFT_ADD, PSB_PATH_TENSOR = 0, 1, 2
 
 EXPORTS = ["psb_create", "psb_destroy", "psb_status_string", "psb_device_status", "psb_sample_weights",
            "psb_weights_export", "psb_weights_free", "psb_set_sample_map", "psb_conv2d", "psb_gemm",
-           "psb_last_path", "psb_maxpool2d_u8", "psb_global_avgpool_u8", "psb_sample_level_static"]
+           "psb_last_path", "psb_maxpool2d_u8", "psb_global_avgpool_u8", "psb_sample_level_static",
+           "psb_sample_batch_create", "psb_sample_batch_run", "psb_sample_batch_free", "psb_run"]
 
 
 class psb_wshape(C.Structure):
@@ -53,6 +54,16 @@ class psb_gemm_desc(C.Structure):
                 ("in_features", C.c_uint32), ("path", C.c_uint32), ("ep", psb_epilogue)]
 
 
+class psb_op(C.Structure):
+    _fields_ = [("kind", C.c_uint32), ("weights", C.c_void_p), ("x_dev", C.c_void_p), ("map_dev", C.c_void_p),
+                ("map_n", C.c_uint32), ("map_oh", C.c_uint32), ("map_ow", C.c_uint32),
+                ("uniform_log2k", C.c_uint32), ("conv", psb_conv_desc), ("gemm", psb_gemm_desc),
+                ("pool_k", C.c_uint32), ("pool_mul", C.c_float), ("pool_qmin", C.c_int32),
+                ("pool_qmax", C.c_int32), ("pool_out_dev", C.c_void_p)]
+
+
+PSB_OP_CONV2D, PSB_OP_GEMM, PSB_OP_MAXPOOL, PSB_OP_AVGPOOL = 0, 1, 2, 3
+
 _lib = None
 
 
@@ -81,6 +92,10 @@ def load_library():
     lib.psb_maxpool2d_u8.argtypes = [vp, vp, u32, u32, u32, u32, u32, u32, u32, u32, vp, vp]
     lib.psb_global_avgpool_u8.argtypes = [vp, vp, u32, u32, u32, u32, u32, C.c_float, i32, i32, vp, vp]
     lib.psb_sample_level_static.argtypes = [vp, C.POINTER(psb_wshape), C.POINTER(psb_sample_cfg), u32, vp, vp, vp]
+    lib.psb_sample_batch_create.argtypes = [vp, u32, C.POINTER(vp), C.POINTER(vp), C.POINTER(vp)]
+    lib.psb_sample_batch_run.argtypes = [vp, vp, C.c_uint64, vp]
+    lib.psb_sample_batch_free.argtypes = [vp, vp]
+    lib.psb_run.argtypes = [vp, C.POINTER(psb_op), u32, vp]
     for name in EXPORTS:
         if name != "psb_status_string":
             getattr(lib, name).restype = i32
@@ -273,6 +288,26 @@ class Context:
         _check(self.lib.psb_gemm(self.handle, weights.handle, _ptr(x), C.byref(d), _stream(stream)),
                "psb_gemm")
         return out
+
+    # -- whole networks -------------------------------------------------------
+    def sample_batch_create(self, filters, weights):
+        """filters: float32 CUDA tensors; weights: the Weights handles sampled from them before."""
+        n = len(filters)
+        wp = (C.c_void_p * n)(*[f.data_ptr() for f in filters])
+        hp = (C.c_void_p * n)(*[w.handle.value for w in weights])
+        b = C.c_void_p()
+        _check(self.lib.psb_sample_batch_create(self.handle, n, wp, hp, C.byref(b)), "psb_sample_batch_create")
+        return b
+
+    def sample_batch_run(self, batch, seed, stream=None):
+        _check(self.lib.psb_sample_batch_run(self.handle, batch, seed, _stream(stream)), "psb_sample_batch_run")
+
+    def sample_batch_free(self, batch):
+        _check(self.lib.psb_sample_batch_free(self.handle, batch), "psb_sample_batch_free")
+
+    def run(self, ops, n_ops, stream=None):
+        """ops: ctypes array of psb_op."""
+        _check(self.lib.psb_run(self.handle, ops, n_ops, _stream(stream)), "psb_run")
 
     # -- glue ----------------------------------------------------------------
     def maxpool2d_u8(self, x, layout, k, stride, pad, out=None, stream=None):

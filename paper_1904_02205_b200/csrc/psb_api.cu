@@ -350,6 +350,59 @@ psb_status psb_gemm(psb_ctx* ctx, const psb_weights* weights, const void* x_dev,
 
 int32_t psb_last_path(const psb_ctx* ctx) { return ctx ? ctx->last_path : 0; }
 
+psb_status psb_sample_batch_create(psb_ctx* ctx, uint32_t n, const float* const* w_dev,
+                                   psb_weights* const* weights, psb_sample_batch** batch) {
+  if (!ctx || !n || !w_dev || !weights || !batch) return PSB_ERR_INVALID_ARG;
+  for (uint32_t i = 0; i < n; ++i) {
+    if (!w_dev[i] || !weights[i] || ((uintptr_t)w_dev[i] & 3u)) return PSB_ERR_INVALID_ARG;
+    if (weights[i]->device != ctx->device) return PSB_ERR_INVALID_ARG;
+  }
+  return sample_batch_create(ctx, n, w_dev, weights, batch);
+}
+
+psb_status psb_sample_batch_run(psb_ctx* ctx, psb_sample_batch* batch, uint64_t seed, void* stream) {
+  if (!ctx || !batch) return PSB_ERR_INVALID_ARG;
+  return sample_batch_run(ctx, batch, seed, (cudaStream_t)stream);
+}
+
+psb_status psb_sample_batch_free(psb_ctx* ctx, psb_sample_batch* batch) {
+  if (!ctx || !batch) return PSB_ERR_INVALID_ARG;
+  cudaSetDevice(ctx->device);
+  cudaDeviceSynchronize();
+  sample_batch_free(batch);
+  return PSB_OK;
+}
+
+psb_status psb_run(psb_ctx* ctx, const psb_op* ops, uint32_t n_ops, void* stream) {
+  if (!ctx || (!ops && n_ops)) return PSB_ERR_INVALID_ARG;
+  for (uint32_t i = 0; i < n_ops; ++i) {
+    const psb_op& op = ops[i];
+    psb_status st;
+    switch (op.kind) {
+      case PSB_OP_CONV2D:
+      case PSB_OP_GEMM:
+        st = psb_set_sample_map(ctx, op.map_dev, op.map_n, op.map_oh, op.map_ow, op.uniform_log2k);
+        if (st != PSB_OK) return st;
+        st = op.kind == PSB_OP_CONV2D ? psb_conv2d(ctx, op.weights, op.x_dev, &op.conv, stream)
+                                      : psb_gemm(ctx, op.weights, op.x_dev, &op.gemm, stream);
+        break;
+      case PSB_OP_MAXPOOL:
+        st = psb_maxpool2d_u8(ctx, (const uint8_t*)op.x_dev, op.conv.layout, op.conv.n, op.conv.c, op.conv.h,
+                              op.conv.w, op.pool_k, op.conv.stride, op.conv.pad, op.pool_out_dev, stream);
+        break;
+      case PSB_OP_AVGPOOL:
+        st = psb_global_avgpool_u8(ctx, (const uint8_t*)op.x_dev, op.conv.layout, op.conv.n, op.conv.c,
+                                   op.conv.h, op.conv.w, op.pool_mul, op.pool_qmin, op.pool_qmax,
+                                   op.pool_out_dev, stream);
+        break;
+      default:
+        st = PSB_ERR_INVALID_ARG;
+    }
+    if (st != PSB_OK) return st;
+  }
+  return PSB_OK;
+}
+
 psb_status psb_maxpool2d_u8(psb_ctx* ctx, const uint8_t* x_dev, uint32_t layout, uint32_t n,
                             uint32_t c, uint32_t h, uint32_t w, uint32_t k, uint32_t stride,
                             uint32_t pad, uint8_t* out_dev, void* stream) {

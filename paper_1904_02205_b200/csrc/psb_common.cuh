@@ -128,6 +128,10 @@ __device__ __forceinline__ int requant(float y, float inv_step, int qmin, int qm
 
 // host-side launchers (defined in the .cu files)
 cudaError_t launch_sampler(const float* w_dev, psb_weights* wt, uint32_t* err_dev, cudaStream_t s);
+psb_status sample_batch_create(psb_ctx* ctx, uint32_t n, const float* const* w_dev,
+                               psb_weights* const* weights, psb_sample_batch** out);
+psb_status sample_batch_run(psb_ctx* ctx, psb_sample_batch* b, uint64_t seed, cudaStream_t s);
+void sample_batch_free(psb_sample_batch* b);
 cudaError_t launch_export(const psb_weights* wt, uint32_t level, int32_t* wint_out,
                           int32_t* e_base_out, cudaStream_t s);
 cudaError_t launch_shift_add(const ConvArgs& a, const WintTable& wt, cudaStream_t s);

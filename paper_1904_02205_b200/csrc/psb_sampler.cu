@@ -8,6 +8,8 @@
 //   emit W_k = s (k + c_k) 2^(e - e_base) as int32 and as signed 7-bit digit
 //   planes in the layout the tensor path loads with TMA.
 // The random bits never leave registers.
+#include <new>
+
 #include "psb_common.cuh"
 
 namespace psb {
@@ -37,13 +39,14 @@ __device__ __forceinline__ void philox4x32_10(uint32_t c0, uint32_t c1, uint32_t
 
 // Largest biased exponent of each exponent group; flags Inf/NaN.
 // norm == 1: one block per output channel.  norm == 0: grid-stride over the layer.
-__global__ void emax_kernel(const float* __restrict__ w, uint32_t O, uint32_t d, uint32_t norm,
-                            uint32_t* __restrict__ e_max, uint32_t* __restrict__ err) {
+__device__ __forceinline__ void emax_block(const float* __restrict__ w, uint32_t O, uint32_t d,
+                                           uint32_t norm, uint32_t* __restrict__ e_max,
+                                           uint32_t* __restrict__ err, uint32_t block, uint32_t blocks) {
   __shared__ uint32_t red[kThreads / 32];
   uint32_t best = 0;
   bool bad = false;
   if (norm) {
-    const float* row = w + (size_t)blockIdx.x * d;
+    const float* row = w + (size_t)block * d;
     for (uint32_t i = threadIdx.x; i < d; i += blockDim.x) {
       uint32_t E = (__float_as_uint(row[i]) >> 23) & 0xFFu;
       bad |= (E == 255u);
@@ -51,8 +54,7 @@ __global__ void emax_kernel(const float* __restrict__ w, uint32_t O, uint32_t d,
     }
   } else {
     size_t total = (size_t)O * d;
-    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < total;
-         i += (size_t)gridDim.x * blockDim.x) {
+    for (size_t i = (size_t)block * blockDim.x + threadIdx.x; i < total; i += (size_t)blocks * blockDim.x) {
       uint32_t E = (__float_as_uint(w[i]) >> 23) & 0xFFu;
       bad |= (E == 255u);
       best = max(best, E);
@@ -65,9 +67,14 @@ __global__ void emax_kernel(const float* __restrict__ w, uint32_t O, uint32_t d,
   if (threadIdx.x == 0) {
     for (int i = 1; i < kThreads / 32; ++i) best = max(best, red[i]);
     if (best == 255u) best = 0;  // error already flagged; keep the window well defined
-    if (norm) e_max[blockIdx.x] = best;
+    if (norm) e_max[block] = best;
     else if (best) atomicMax(&e_max[0], best);
   }
+}
+
+__global__ void emax_kernel(const float* __restrict__ w, uint32_t O, uint32_t d, uint32_t norm,
+                            uint32_t* __restrict__ e_max, uint32_t* __restrict__ err) {
+  emax_block(w, O, d, norm, e_max, err, blockIdx.x, gridDim.x);
 }
 
 struct SampleParams {
@@ -84,10 +91,10 @@ struct SampleParams {
   int planes_count[kMaxLevels];
 };
 
-__global__ void __launch_bounds__(kThreads) sample_kernel(const SampleParams p) {
-  __shared__ float stage[kStage];
-  const uint32_t row_block = blockIdx.x / p.ch_chunks;
-  const uint32_t chunk = blockIdx.x % p.ch_chunks;
+__device__ __forceinline__ void sample_block(const SampleParams& p, uint32_t block, uint32_t seed_lo,
+                                             uint32_t seed_hi, float* stage) {
+  const uint32_t row_block = block / p.ch_chunks;
+  const uint32_t chunk = block % p.ch_chunks;
   const uint32_t o0 = row_block * p.rows_per_block;
   const uint32_t c0 = chunk * p.ch_per_block;
   const uint32_t rows = min(p.rows_per_block, p.O - o0);
@@ -128,8 +135,7 @@ __global__ void __launch_bounds__(kThreads) sample_kernel(const SampleParams p) 
       uint32_t c = 0, j = 0;
       for (uint32_t q = 0; q * 4u < kmax; ++q) {
         uint32_t rnd[4];
-        philox4x32_10(q, p.layer_id, (uint32_t)index, (uint32_t)(index >> 32), p.seed_lo, p.seed_hi,
-                      rnd);
+        philox4x32_10(q, p.layer_id, (uint32_t)index, (uint32_t)(index >> 32), seed_lo, seed_hi, rnd);
 #pragma unroll
         for (int v = 0; v < 4; ++v) {
           if (j < kmax) {
@@ -160,6 +166,43 @@ __global__ void __launch_bounds__(kThreads) sample_kernel(const SampleParams p) 
   }
 }
 
+__global__ void __launch_bounds__(kThreads) sample_kernel(const SampleParams p) {
+  __shared__ float stage[kStage];
+  sample_block(p, blockIdx.x, p.seed_lo, p.seed_hi, stage);
+}
+
+// All layers of a network in two launches.  Entry i owns blocks [first, first + count) of each
+// grid; its parameters sit in device memory (every thread of a block reads the same words).
+struct BatchEntry {
+  SampleParams p;
+  uint32_t emax_first, emax_blocks, sample_first, sample_blocks;
+};
+
+__device__ __forceinline__ uint32_t find_entry(const BatchEntry* __restrict__ e, uint32_t n, uint32_t block,
+                                               bool emax) {
+  uint32_t lo = 0, hi = n - 1;
+  while (lo < hi) {
+    const uint32_t mid = (lo + hi + 1) >> 1;
+    const uint32_t first = emax ? e[mid].emax_first : e[mid].sample_first;
+    if (first <= block) lo = mid; else hi = mid - 1;
+  }
+  return lo;
+}
+
+__global__ void __launch_bounds__(kThreads) emax_batch_kernel(const BatchEntry* __restrict__ entries, uint32_t n,
+                                                              uint32_t* __restrict__ err) {
+  const BatchEntry& e = entries[find_entry(entries, n, blockIdx.x, true)];
+  emax_block(e.p.w, e.p.O, e.p.d, e.p.norm, const_cast<uint32_t*>(e.p.e_max), err,
+             blockIdx.x - e.emax_first, e.emax_blocks);
+}
+
+__global__ void __launch_bounds__(kThreads) sample_batch_kernel(const BatchEntry* __restrict__ entries, uint32_t n,
+                                                                uint32_t seed_lo, uint32_t seed_hi) {
+  __shared__ float stage[kStage];
+  const BatchEntry& e = entries[find_entry(entries, n, blockIdx.x, false)];
+  sample_block(e.p, blockIdx.x - e.sample_first, seed_lo, seed_hi, stage);
+}
+
 // 128 * (sum of each filter row): the constant that restores sum x*W from sum (x-128)*W when
 // unsigned activations are fed to the signed MMA with an offset of 128.  One warp per row.
 __global__ void corr128_kernel(const int32_t* __restrict__ wint, uint32_t O, uint32_t d,
@@ -188,21 +231,19 @@ __global__ void export_kernel(const int32_t* __restrict__ wint, int32_t* __restr
 
 }  // namespace
 
-cudaError_t launch_sampler(const float* w_dev, psb_weights* wt, uint32_t* err_dev, cudaStream_t s) {
+namespace {
+
+uint32_t emax_blocks_for(uint32_t O, uint32_t d, uint32_t norm) {
+  if (norm) return O;
+  size_t total = (size_t)O * d;
+  uint32_t blocks = (uint32_t)((total + kThreads * 8 - 1) / (kThreads * 8));
+  return blocks < 1 ? 1 : (blocks > 1184 ? 1184 : blocks);
+}
+
+// Parameters of one layer's sampling pass; returns the number of blocks it needs.
+uint32_t fill_sample_params(const float* w_dev, const psb_weights* wt, uint32_t* e_max, SampleParams& p) {
   const psb_wshape& sh = wt->shape;
   const uint32_t O = sh.out_ch, Cg = sh.in_ch_per_group, KHKW = sh.kh * sh.kw, d = wt->d;
-  const uint32_t norm = wt->cfg.norm;
-  cudaError_t e = cudaMemsetAsync(wt->e_max, 0, sizeof(uint32_t) * O, s);
-  if (e != cudaSuccess) return e;
-  if (norm) {
-    emax_kernel<<<O, kThreads, 0, s>>>(w_dev, O, d, 1, wt->e_max, err_dev);
-  } else {
-    size_t total = (size_t)O * d;
-    uint32_t blocks = (uint32_t)((total + kThreads * 8 - 1) / (kThreads * 8));
-    blocks = blocks < 1 ? 1 : (blocks > 1184 ? 1184 : blocks);
-    emax_kernel<<<blocks, kThreads, 0, s>>>(w_dev, O, d, 0, wt->e_max, err_dev);
-  }
-  SampleParams p;
   p.w = w_dev;
   p.O = O; p.Cg = Cg; p.KHKW = KHKW; p.d = d;
   if (d <= (uint32_t)kStage) {
@@ -214,7 +255,7 @@ cudaError_t launch_sampler(const float* w_dev, psb_weights* wt, uint32_t* err_de
     p.ch_per_block = kStage / KHKW;
     p.ch_chunks = (Cg + p.ch_per_block - 1) / p.ch_per_block;
   }
-  p.norm = norm;
+  p.norm = wt->cfg.norm;
   p.span = (1u << wt->cfg.exp_bits) - 1u;
   p.level_mask = wt->cfg.level_mask;
   p.max_level = 0;
@@ -224,21 +265,117 @@ cudaError_t launch_sampler(const float* w_dev, psb_weights* wt, uint32_t* err_de
   p.seed_hi = (uint32_t)(wt->cfg.seed >> 32);
   p.layer_id = wt->cfg.layer_id;
   p.cpad = wt->cpad; p.kpad = wt->kpad; p.has_planes = wt->has_planes ? 1u : 0u;
-  p.e_max = wt->e_max;
+  p.e_max = e_max;
   p.e_base = wt->e_base;
   for (int l = 0; l < kMaxLevels; ++l) {
     p.wint[l] = wt->level[l].wint;
     p.planes[l] = wt->level[l].planes;
     p.planes_count[l] = wt->level[l].planes_count;
   }
-  uint32_t row_blocks = (O + p.rows_per_block - 1) / p.rows_per_block;
-  sample_kernel<<<row_blocks * p.ch_chunks, kThreads, 0, s>>>(p);
-  if (wt->packed_k)
-    for (int l = 0; l < kMaxLevels; ++l)
-      if (wt->level[l].corr128)
-        corr128_kernel<<<(O * 32 + kThreads - 1) / kThreads, kThreads, 0, s>>>(wt->level[l].wint, O, d,
-                                                                              wt->level[l].corr128);
+  const uint32_t row_blocks = (O + p.rows_per_block - 1) / p.rows_per_block;
+  return row_blocks * p.ch_chunks;
+}
+
+void launch_corr128(const psb_weights* wt, cudaStream_t s) {
+  const uint32_t O = wt->shape.out_ch;
+  for (int l = 0; l < kMaxLevels; ++l)
+    if (wt->level[l].corr128)
+      corr128_kernel<<<(O * 32 + kThreads - 1) / kThreads, kThreads, 0, s>>>(wt->level[l].wint, O, wt->d,
+                                                                            wt->level[l].corr128);
+}
+
+}  // namespace
+
+cudaError_t launch_sampler(const float* w_dev, psb_weights* wt, uint32_t* err_dev, cudaStream_t s) {
+  const uint32_t O = wt->shape.out_ch;
+  cudaError_t e = cudaMemsetAsync(wt->e_max, 0, sizeof(uint32_t) * O, s);
+  if (e != cudaSuccess) return e;
+  emax_kernel<<<emax_blocks_for(O, wt->d, wt->cfg.norm), kThreads, 0, s>>>(w_dev, O, wt->d, wt->cfg.norm,
+                                                                          wt->e_max, err_dev);
+  SampleParams p;
+  const uint32_t blocks = fill_sample_params(w_dev, wt, wt->e_max, p);
+  sample_kernel<<<blocks, kThreads, 0, s>>>(p);
+  if (wt->packed_k) launch_corr128(wt, s);
   return cudaGetLastError();
+}
+
+}  // namespace psb
+
+// ---- batched sampling: every layer of a network in two launches ---------------------------
+struct psb_sample_batch {
+  uint32_t n = 0;
+  psb::BatchEntry* entries_dev = nullptr;
+  uint32_t* e_max_pool = nullptr;     // one word per output channel of every layer
+  size_t e_max_words = 0;
+  uint32_t emax_grid = 0, sample_grid = 0;
+  psb_weights** packed = nullptr;     // layers that need the offset correction recomputed
+  uint32_t n_packed = 0;
+  int device = 0;
+};
+
+namespace psb {
+
+psb_status sample_batch_create(psb_ctx* ctx, uint32_t n, const float* const* w_dev,
+                               psb_weights* const* weights, psb_sample_batch** out) {
+  psb_sample_batch* b = new (std::nothrow) psb_sample_batch();
+  BatchEntry* host = new (std::nothrow) BatchEntry[n];
+  psb_weights** packed = new (std::nothrow) psb_weights*[n];
+  if (!b || !host || !packed) { delete b; delete[] host; delete[] packed; return PSB_ERR_ALLOC; }
+  size_t words = 0;
+  for (uint32_t i = 0; i < n; ++i) words += weights[i]->shape.out_ch;
+  bool ok = cudaMalloc(&b->e_max_pool, sizeof(uint32_t) * words) == cudaSuccess &&
+            cudaMalloc(&b->entries_dev, sizeof(BatchEntry) * n) == cudaSuccess;
+  if (ok) {
+    size_t off = 0;
+    uint32_t eb = 0, sb = 0;
+    for (uint32_t i = 0; i < n; ++i) {
+      const psb_weights* wt = weights[i];
+      BatchEntry& e = host[i];
+      e.sample_blocks = fill_sample_params(w_dev[i], wt, b->e_max_pool + off, e.p);
+      e.emax_blocks = emax_blocks_for(wt->shape.out_ch, wt->d, wt->cfg.norm);
+      e.emax_first = eb;
+      e.sample_first = sb;
+      eb += e.emax_blocks;
+      sb += e.sample_blocks;
+      off += wt->shape.out_ch;
+      if (wt->packed_k) packed[b->n_packed++] = weights[i];
+    }
+    b->emax_grid = eb;
+    b->sample_grid = sb;
+    ok = cudaMemcpy(b->entries_dev, host, sizeof(BatchEntry) * n, cudaMemcpyHostToDevice) == cudaSuccess;
+  }
+  delete[] host;
+  if (!ok) {
+    cudaGetLastError();
+    if (b->e_max_pool) cudaFree(b->e_max_pool);
+    if (b->entries_dev) cudaFree(b->entries_dev);
+    delete[] packed;
+    delete b;
+    return PSB_ERR_ALLOC;
+  }
+  b->n = n;
+  b->e_max_words = words;
+  b->packed = packed;
+  b->device = ctx->device;
+  *out = b;
+  return PSB_OK;
+}
+
+psb_status sample_batch_run(psb_ctx* ctx, psb_sample_batch* b, uint64_t seed, cudaStream_t s) {
+  if (cudaMemsetAsync(b->e_max_pool, 0, sizeof(uint32_t) * b->e_max_words, s) != cudaSuccess)
+    return PSB_ERR_CUDA;
+  emax_batch_kernel<<<b->emax_grid, kThreads, 0, s>>>(b->entries_dev, b->n, ctx->err_dev);
+  sample_batch_kernel<<<b->sample_grid, kThreads, 0, s>>>(b->entries_dev, b->n, (uint32_t)seed,
+                                                         (uint32_t)(seed >> 32));
+  for (uint32_t i = 0; i < b->n_packed; ++i) launch_corr128(b->packed[i], s);
+  return cudaGetLastError() == cudaSuccess ? PSB_OK : PSB_ERR_CUDA;
+}
+
+void sample_batch_free(psb_sample_batch* b) {
+  if (b->e_max_pool) cudaFree(b->e_max_pool);
+  if (b->entries_dev) cudaFree(b->entries_dev);
+  delete[] b->packed;
+  delete b;
 }
 
 cudaError_t launch_export(const psb_weights* wt, uint32_t level, int32_t* wint_out,

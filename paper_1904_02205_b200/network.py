@@ -40,9 +40,15 @@ class Network:
                 self.qmax[l["dst"]] = p["qmax"]
         self.logits = torch.empty((batch, layers[-1]["cout"]), dtype=torch.float32, device=dev)
         self.paths = {}
+        self._batch = None
+        self._ops = None
 
     def sample(self, seed):
-        """Fresh draws for every layer (psb_sample_weights; handles are created on first use)."""
+        """Fresh draws for every layer.  The first call creates the handles layer by layer
+        (psb_sample_weights); later calls re-sample all layers in one psb_sample_batch_run."""
+        if self._batch is not None:
+            self.ctx.sample_batch_run(self._batch, seed)
+            return
         for l in self.layers:
             if l["op"] != "conv":
                 continue
@@ -50,6 +56,54 @@ class Network:
             self.weights[l["name"]] = self.ctx.sample_weights(
                 pr["w"], groups=l["groups"], seed=seed, layer_id=pr["p"]["layer_id"], level_mask=self.level_mask,
                 into=self.weights.get(l["name"]))
+        convs = [l["name"] for l in self.layers if l["op"] == "conv"]
+        self._batch = self.ctx.sample_batch_create([self.params[n]["w"] for n in convs],
+                                                   [self.weights[n] for n in convs])
+
+    def _build_ops(self):
+        """The forward pass as one psb_run op list (same arguments as the per-layer calls)."""
+        ops = (B.psb_op * len(self.layers))()
+        for op, l in zip(ops, self.layers):
+            x = self.acts[l["src"]]
+            op.x_dev = x.data_ptr()
+            if l["op"] != "conv":
+                n, h, w, c = x.shape
+                op.conv.layout, op.conv.n, op.conv.c, op.conv.h, op.conv.w = B.PSB_LAYOUT_NHWC, n, c, h, w
+                op.pool_out_dev = self.acts[l["dst"]].data_ptr()
+                if l["op"] == "maxpool":
+                    op.kind, op.pool_k, op.conv.stride, op.conv.pad = B.PSB_OP_MAXPOOL, l["k"], l["stride"], l["pad"]
+                else:
+                    p = self.params[l["name"]]["p"]
+                    op.kind, op.pool_mul, op.pool_qmin, op.pool_qmax = B.PSB_OP_AVGPOOL, float(p["pool_mul"]), p["qmin"], p["qmax"]
+                continue
+            pr = self.params[l["name"]]
+            p = pr["p"]
+            is_fc = x.dim() == 2
+            op.weights = self.weights[l["name"]].handle.value
+            if self.kmaps is not None and not is_fc:
+                km = self.kmaps[l["hout"]]
+                op.map_dev, op.map_n, op.map_oh, op.map_ow = km.data_ptr(), km.shape[0], km.shape[1], km.shape[2]
+            else:
+                op.uniform_log2k = self.fc_log2k if is_fc else self.uniform_log2k
+            ep = B.psb_epilogue()
+            ep.scale_dev, ep.bias_dev = pr["scale"].data_ptr(), pr["bias"].data_ptr()
+            if l["residual"] is not None:
+                res = self.acts[l["residual"]]
+                ep.residual_dev, ep.residual_dtype = res.data_ptr(), B._dt_of(res)
+            ep.residual_scale = float(p["res_scale"])
+            ep.relu, ep.inv_step, ep.qmin, ep.qmax = int(l["relu"]), float(p["inv_step"]), p["qmin"], p["qmax"]
+            ep.out_dtype = p["out_dtype"]
+            ep.q_out_dev = self.acts[l["dst"]].data_ptr()
+            if is_fc:
+                ep.f32_out_dev = self.logits.data_ptr()
+                op.kind = B.PSB_OP_GEMM
+                op.gemm = B.psb_gemm_desc(B._dt_of(x), self.qmax[l["src"]], x.shape[0], x.shape[1], self.path, ep)
+            else:
+                n, h, w, c = x.shape
+                op.kind = B.PSB_OP_CONV2D
+                op.conv = B.psb_conv_desc(B.PSB_LAYOUT_NHWC, B._dt_of(x), self.qmax[l["src"]], n, c, h, w,
+                                          l["stride"], l["pad"], self.path, ep)
+        self._ops = ops
 
     def forward(self, image=None, layer_events=None):
         """image: u8 CUDA tensor [batch, h, w, 3] (copied into the resident input buffer) or None.
@@ -57,6 +111,12 @@ class Network:
         ctx = self.ctx
         if image is not None:
             self.acts["image"].copy_(image, non_blocking=True)
+        if layer_events is None and self.paths:
+            # every later pass: one psb_run call over the whole layer list
+            if self._ops is None:
+                self._build_ops()
+            ctx.run(self._ops, len(self.layers))
+            return self.logits
         prev_end = None
         for l in self.layers:
             if layer_events is not None:
@@ -99,6 +159,9 @@ class Network:
         return self.logits
 
     def free(self):
+        if self._batch is not None:
+            self.ctx.sample_batch_free(self._batch)
+            self._batch = None
         for w in self.weights.values():
             w.free()
         self.weights = {}

@@ -54,6 +54,31 @@ def test_tiny_resnet_uniform_k(psb, oracle):
     nw.free(); ctx.close()
 
 
+def test_batched_sampling_and_op_list_equal_the_layer_by_layer_calls(psb, oracle):
+    """psb_sample_batch_run and psb_run must reproduce what the single calls give (and the oracle)."""
+    import torch
+    from paper_1904_02205_b200.network import Network
+    from workloads import build_network, tiny_resnet_layers
+
+    L = tiny_resnet_layers()
+    net = build_network(L, 40, 3, 2, 15, 15)
+    ctx = psb.Context(0)
+    nw = Network(ctx, L, net, 3, 1 << 3, uniform_log2k=3)
+    img = torch.from_numpy(net["image"][:3]).to(ctx.device)
+    nw.sample(7)                      # layer by layer: creates the handles
+    nw.forward(img)                   # layer by layer: records the paths
+    nw.sample(11)                     # all layers in one batch, new seed
+    logits = nw.forward(img).cpu().numpy()       # one psb_run call
+    assert ctx.device_status() == 0
+    for l in L:
+        if l["op"] == "conv":
+            got = ctx.weights_export(nw.weights[l["name"]], 3)[0].cpu().numpy().astype(np.int64)
+            p = net["params"][l["name"]]
+            assert np.array_equal(got, oracle.sample_level(p["w"], 11, p["layer_id"], 3)[0]), l["name"]
+    _compare(nw, logits, oracle, L, net, range(3), 11, 3)
+    nw.free(); ctx.close()
+
+
 def test_tiny_resnet_per_location_draw_counts(psb, oracle):
     from workloads import build_network, saliency_kmaps, tiny_resnet_layers
 

@@ -75,41 +75,53 @@ __global__ void __launch_bounds__(256) conv_direct_kernel(const ConvArgs a, cons
 // Explicit gather of the activation matrix for filters with few input channels (e.g. a 7x7
 // stem on 3 channels): row m = output location, column k = (kh, kw, ci) flattened, padded with
 // zeros to kpad.  Values are stored minus `offset` as signed bytes; a padded input position is the
-// value 0, i.e. -offset.  One thread writes 16 bytes.
+// value 0, i.e. -offset.  A block handles kIm2colPix consecutive output locations of one output
+// row: the input rows they touch are staged in shared memory with coalesced loads, then every
+// thread assembles and writes 16-byte pieces of the matrix.
+constexpr uint32_t kIm2colPix = 32;
+
 __global__ void __launch_bounds__(256) im2col_s8_kernel(const ConvArgs a, uint32_t kpad, uint32_t offset,
-                                                       int8_t* __restrict__ dst) {
-  extern __shared__ uint32_t ktab[];  // per column: kh | kw << 8 | ci << 16, or ~0 for K padding
+                                                       uint32_t span_bytes, int8_t* __restrict__ dst) {
+  extern __shared__ uint32_t im2col_smem[];
+  uint32_t* ktab = im2col_smem;                               // per column: kh | (kw*C + ci) << 8, or ~0
+  uint8_t* rows = reinterpret_cast<uint8_t*>(ktab + kpad);    // [KH][span_bytes], already offset
   const uint32_t d = a.KH * a.KW * a.C;
   for (uint32_t k = threadIdx.x; k < kpad; k += blockDim.x) {
-    uint32_t tap = k / a.C, ci = k % a.C;
-    ktab[k] = k < d ? ((tap / a.KW) | ((tap % a.KW) << 8) | (ci << 16)) : 0xFFFFFFFFu;
+    const uint32_t tap = k / a.C, ci = k % a.C;
+    ktab[k] = k < d ? ((tap / a.KW) | (((tap % a.KW) * a.C + ci) << 8)) : 0xFFFFFFFFu;
+  }
+  const uint32_t strips = (a.OW + kIm2colPix - 1) / kIm2colPix;
+  const uint32_t strip = blockIdx.x % strips;
+  const uint32_t oy = (blockIdx.x / strips) % a.OH;
+  const uint32_t n = blockIdx.x / (strips * a.OH);
+  const uint32_t ox0 = strip * kIm2colPix;
+  const uint32_t npix = min(kIm2colPix, a.OW - ox0);
+  const int ix0 = (int)(ox0 * a.stride) - (int)a.pad;         // leftmost input column of the strip
+  const int iy0 = (int)(oy * a.stride) - (int)a.pad;
+  const uint8_t* x = (const uint8_t*)a.x;
+  const uint8_t fill = (uint8_t)(0u - offset);
+  for (uint32_t t = threadIdx.x; t < a.KH * span_bytes; t += blockDim.x) {
+    const uint32_t kh = t / span_bytes, b = t % span_bytes;
+    const int iy = iy0 + (int)kh, ix = ix0 + (int)(b / a.C);
+    uint8_t v = fill;
+    if (iy >= 0 && iy < (int)a.H && ix >= 0 && ix < (int)a.W)
+      v = (uint8_t)(x[(((size_t)n * a.H + iy) * a.W + ix) * a.C + b % a.C] - offset);
+    rows[t] = v;
   }
   __syncthreads();
   const uint32_t chunks = kpad / 16u;
-  const size_t total = (size_t)a.N * a.OH * a.OW * chunks;
-  const uint8_t* x = (const uint8_t*)a.x;
-  for (size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x; idx < total;
-       idx += (size_t)gridDim.x * blockDim.x) {
-    const uint32_t ch = (uint32_t)(idx % chunks);
-    const size_t m = idx / chunks;
-    const uint32_t ox = (uint32_t)(m % a.OW), oy = (uint32_t)((m / a.OW) % a.OH);
-    const uint32_t n = (uint32_t)(m / ((size_t)a.OW * a.OH));
-    const int iy0 = (int)(oy * a.stride) - (int)a.pad, ix0 = (int)(ox * a.stride) - (int)a.pad;
+  const size_t m0 = ((size_t)n * a.OH + oy) * a.OW + ox0;
+  for (uint32_t t = threadIdx.x; t < npix * chunks; t += blockDim.x) {
+    const uint32_t px = t / chunks, ch = t % chunks;
+    const uint32_t base = px * a.stride * a.C;
     uint32_t w[4] = {0, 0, 0, 0};
 #pragma unroll
     for (int j = 0; j < 16; ++j) {
       const uint32_t e = ktab[ch * 16u + j];
-      uint32_t v = 0;
-      if (e != 0xFFFFFFFFu) {
-        const int iy = iy0 + (int)(e & 0xFFu), ix = ix0 + (int)((e >> 8) & 0xFFu);
-        uint32_t raw = 0;
-        if (iy >= 0 && iy < (int)a.H && ix >= 0 && ix < (int)a.W)
-          raw = x[(((size_t)n * a.H + iy) * a.W + ix) * a.C + (e >> 16)];
-        v = (raw - offset) & 0xFFu;
-      }
+      const uint32_t v = e == 0xFFFFFFFFu ? 0u : rows[(e & 0xFFu) * span_bytes + base + (e >> 8)];
       w[j >> 2] |= v << (8 * (j & 3));
     }
-    *reinterpret_cast<uint4*>(dst + m * kpad + ch * 16u) = make_uint4(w[0], w[1], w[2], w[3]);
+    *reinterpret_cast<uint4*>(dst + (m0 + px) * kpad + ch * 16u) = make_uint4(w[0], w[1], w[2], w[3]);
   }
 }
 
@@ -160,6 +172,35 @@ __global__ void maxpool_kernel(const uint8_t* __restrict__ x, uint32_t nchw, uin
   }
 }
 
+// Channels-last max-pooling, 16 channels per thread: 16-byte loads, byte-wise maxima.
+__global__ void __launch_bounds__(256) maxpool_nhwc16_kernel(const uint8_t* __restrict__ x, uint32_t N, uint32_t C,
+                                                            uint32_t H, uint32_t W, uint32_t k, uint32_t stride,
+                                                            uint32_t pad, uint32_t OH, uint32_t OW,
+                                                            uint8_t* __restrict__ out) {
+  const uint32_t groups = C / 16u;
+  const size_t total = (size_t)N * OH * OW * groups;
+  for (size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x; idx < total;
+       idx += (size_t)gridDim.x * blockDim.x) {
+    const uint32_t g = (uint32_t)(idx % groups);
+    const size_t pix = idx / groups;
+    const uint32_t ox = (uint32_t)(pix % OW), oy = (uint32_t)((pix / OW) % OH);
+    const uint32_t n = (uint32_t)(pix / ((size_t)OW * OH));
+    uint4 best = make_uint4(0, 0, 0, 0);
+    for (uint32_t kh = 0; kh < k; ++kh) {
+      const int iy = (int)(oy * stride + kh) - (int)pad;
+      if (iy < 0 || iy >= (int)H) continue;
+      for (uint32_t kw = 0; kw < k; ++kw) {
+        const int ix = (int)(ox * stride + kw) - (int)pad;
+        if (ix < 0 || ix >= (int)W) continue;
+        const uint4 v = __ldg(reinterpret_cast<const uint4*>(x + (((size_t)n * H + iy) * W + ix) * C + g * 16u));
+        best.x = __vmaxu4(best.x, v.x); best.y = __vmaxu4(best.y, v.y);
+        best.z = __vmaxu4(best.z, v.z); best.w = __vmaxu4(best.w, v.w);
+      }
+    }
+    *reinterpret_cast<uint4*>(out + pix * C + g * 16u) = best;
+  }
+}
+
 // One warp per (n, c): integer sum over H*W, then one re-quantisation.
 __global__ void avgpool_kernel(const uint8_t* __restrict__ x, uint32_t nchw, uint32_t N, uint32_t C,
                                uint32_t HW, float pool_mul, int qmin, int qmax,
@@ -193,8 +234,12 @@ cudaError_t launch_shift_add(const ConvArgs& a, const WintTable& wt, cudaStream_
 
 cudaError_t launch_im2col_s8(const ConvArgs& a, uint32_t kpad, uint32_t offset, int8_t* dst,
                              cudaStream_t s) {
-  size_t total = (size_t)a.N * a.OH * a.OW * (kpad / 16u);
-  im2col_s8_kernel<<<grid_for(total, 256), 256, kpad * sizeof(uint32_t), s>>>(a, kpad, offset, dst);
+  const uint32_t strips = (a.OW + kIm2colPix - 1) / kIm2colPix;
+  const uint32_t span_bytes = ((kIm2colPix - 1) * a.stride + a.KW) * a.C;
+  const size_t smem = kpad * sizeof(uint32_t) + (size_t)a.KH * span_bytes;
+  if (smem > 48 * 1024 || (uint64_t)a.N * a.OH * strips >= (1ull << 31) || a.KW * a.C >= (1u << 24))
+    return cudaErrorInvalidValue;
+  im2col_s8_kernel<<<a.N * a.OH * strips, 256, smem, s>>>(a, kpad, offset, span_bytes, dst);
   return cudaGetLastError();
 }
 
@@ -211,7 +256,10 @@ cudaError_t launch_maxpool(const uint8_t* x, uint32_t nchw, uint32_t N, uint32_t
                            cudaStream_t s) {
   uint32_t OH = (H + 2 * pad - k) / stride + 1, OW = (W + 2 * pad - k) / stride + 1;
   size_t total = (size_t)N * OH * OW * C;
-  maxpool_kernel<<<grid_for(total, 256), 256, 0, s>>>(x, nchw, N, C, H, W, k, stride, pad, OH, OW, out);
+  if (!nchw && C % 16u == 0 && !(((uintptr_t)x | (uintptr_t)out) & 15u))
+    maxpool_nhwc16_kernel<<<grid_for(total / 16, 256), 256, 0, s>>>(x, N, C, H, W, k, stride, pad, OH, OW, out);
+  else
+    maxpool_kernel<<<grid_for(total, 256), 256, 0, s>>>(x, nchw, N, C, H, W, k, stride, pad, OH, OW, out);
   return cudaGetLastError();
 }
 

@@ -10,12 +10,12 @@
 // in 64-bit integers, which makes the result exact.
 //
 // Structure of one CTA (one per SM, persistent over tiles):
-//   warp 0   producer: TMA loads of the activation tile (im2col mode for
+//   warps 0-2 producers (one thread each, taking the stages in turns): TMA loads of the activation tile (im2col mode for
 //            filters with taps, stride or padding; plain 2-D tiles otherwise) and
 //            of the digit-plane tile into a ring of shared-memory stages
-//   warp 1   allocates TMEM; one thread issues the MMAs and commits them to the
+//   warp 3   allocates TMEM; one thread issues the MMAs and commits them to the
 //            stage-free and accumulator-ready barriers
-//   warps 2-9  epilogue: TMEM -> registers, recombine planes, dequantise, bias,
+//   warps 4-11 epilogue: TMEM -> registers, recombine planes, dequantise, bias,
 //            shortcut, ReLU, re-quantise, vectorised stores; overlaps the next
 //            tile's MMAs through two TMEM accumulator buffers
 // Per-location draw counts (Sec. 4.5): a tile is contracted once per level present
@@ -33,8 +33,11 @@ namespace psb {
 namespace {
 
 constexpr int kTileM = 128;
+constexpr int kProducerWarps = 3;    // one issuing thread each: their barrier waits overlap
+constexpr int kMmaWarp = kProducerWarps;
+constexpr int kFirstEpilogueWarp = kMmaWarp + 1;   // a multiple of 4: warp & 3 = TMEM lane quarter
 constexpr int kEpilogueWarps = 8;
-constexpr int kThreadsTensor = 64 + 32 * kEpilogueWarps;   // producer warp, MMA warp, epilogue warps
+constexpr int kThreadsTensor = 32 * (kFirstEpilogueWarp + kEpilogueWarps);
 constexpr uint32_t kTmemCols = 512;
 constexpr uint32_t kTmemBufStride = 256;
 constexpr int kMaxStages = 12;
@@ -401,7 +404,7 @@ psb_mma_kernel(const __grid_constant__ TmapSet maps, const __grid_constant__ Ten
     ctl->abort = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
-  if (warp == 1) {
+  if (warp == kMmaWarp) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(
                      smem_u32(&ctl->tmem_base)),
                  "r"(kTmemCols)
@@ -415,13 +418,14 @@ psb_mma_kernel(const __grid_constant__ TmapSet maps, const __grid_constant__ Ten
   volatile uint32_t* abort = &ctl->abort;
   bool failed = false;
 
-  if (warp == 0) {
-    // ------------------------------------------------------------ producer
-    // One thread runs the whole loop.  Every barrier round trip costs a few hundred cycles of
-    // latency on this thread, so the index arithmetic is incremental (no divisions), K blocks are
-    // handed over in groups, and the next stage's barrier is probed before it is needed.
+  if (warp < (uint32_t)kProducerWarps) {
+    // ----------------------------------------------------------- producers
+    // One thread per producer warp.  Every barrier round trip costs its thread a few hundred
+    // cycles of latency, which caps a single thread at about one TMA load per 300 cycles; the
+    // producer threads therefore take the pipeline stages in turns (all of them walk the same
+    // sequence of stages with incremental index arithmetic, each issues every third one).
     if (lane == 0) {
-      if (p.resident) {
+      if (p.resident && warp == 0) {
         // the digit planes of this CTA's channel tile, all K blocks, once
         const uint32_t l = p.a.uniform_log2k, P = p.planes[l];
         const uint32_t o_tile = blockIdx.x / p.ctas_per_otile;
@@ -435,8 +439,8 @@ psb_mma_kernel(const __grid_constant__ TmapSet maps, const __grid_constant__ Ten
           if (++cb == p.n_cb) { cb = 0; kcol += p.cpad; }
         }
       }
-      uint32_t s = 0, ph = 0;  // ring position and its phase
-      bool next_free = mbar_try_wait(smem_u32(&ctl->empty[0]), 1u);
+      uint32_t s = 0, ph = 0;   // ring position and phase of the current stage use
+      uint32_t turn = 0;        // whose turn it is among the producer threads
       TileIter ti;
       for (ti.init(p); ti.valid() && !failed; ti.next()) {
         const uint32_t m_tile = ti.m_tile, o_tile = ti.o_tile;
@@ -456,22 +460,23 @@ psb_mma_kernel(const __grid_constant__ TmapSet maps, const __grid_constant__ Ten
           uint32_t kw = 0, kh = 0, cb = 0, kcol = 0;     // tap (kh, kw), channel block, plane column
           for (uint32_t it = 0; it < k_iters;) {
             const uint32_t cnt = min(p.group, k_iters - it);
-            if (!next_free && !mbar_wait(smem_u32(&ctl->empty[s]), ph ^ 1u, abort)) { failed = true; break; }
+            const bool mine = turn == warp;
+            if (mine) {
+              if (!mbar_wait(smem_u32(&ctl->empty[s]), ph ^ 1u, abort)) { failed = true; break; }
+              mbar_expect_tx(smem_u32(&ctl->full[s]), bytes * cnt);
+            }
             const uint32_t bar = smem_u32(&ctl->full[s]);
             uint32_t dst = smem_u32(ring) + s * stage_bytes;
-            mbar_expect_tx(bar, bytes * cnt);
-            // probe the following stage now; the answer is back by the time it is needed
-            const uint32_t s2 = (s + 1 == p.stages) ? 0u : s + 1;
-            const uint32_t ph2 = (s + 1 == p.stages) ? ph ^ 1u : ph;
-            next_free = mbar_try_wait(smem_u32(&ctl->empty[s2]), ph2 ^ 1u);
             for (uint32_t j = 0; j < cnt; ++j, dst += sub_bytes) {
-              if (p.im2col)
-                tma_load_im2col_4d(dst, &maps.a, bar, (int)(cb * BK), w0, h0, (int)n0, (uint16_t)kw,
-                                   (uint16_t)kh);
-              else
-                tma_load_2d(dst, &maps.a, bar, (int)(cb * BK), (int)m0);
-              if (!p.resident)
-                tma_load_2d(dst + p.stage_bytes_a, &maps.b[l], bar, (int)(kcol + cb * BK), b_row);
+              if (mine) {
+                if (p.im2col)
+                  tma_load_im2col_4d(dst, &maps.a, bar, (int)(cb * BK), w0, h0, (int)n0, (uint16_t)kw,
+                                     (uint16_t)kh);
+                else
+                  tma_load_2d(dst, &maps.a, bar, (int)(cb * BK), (int)m0);
+                if (!p.resident)
+                  tma_load_2d(dst + p.stage_bytes_a, &maps.b[l], bar, (int)(kcol + cb * BK), b_row);
+              }
               if (++cb == p.n_cb) {
                 cb = 0;
                 kcol += p.cpad;
@@ -479,14 +484,14 @@ psb_mma_kernel(const __grid_constant__ TmapSet maps, const __grid_constant__ Ten
               }
             }
             it += cnt;
-            s = s2;
-            ph = ph2;
+            if (++s == p.stages) { s = 0; ph ^= 1u; }
+            if (++turn == (uint32_t)kProducerWarps) turn = 0;
           }
         }
       }
     }
     failed = __shfl_sync(0xFFFFFFFFu, failed ? 1 : 0, 0) != 0;
-  } else if (warp == 1) {
+  } else if (warp == (uint32_t)kMmaWarp) {
     // ---------------------------------------------------------------- MMA
     if (lane == 0) {
       uint32_t s = 0, ph = 0, pass = 0;
@@ -538,7 +543,7 @@ psb_mma_kernel(const __grid_constant__ TmapSet maps, const __grid_constant__ Ten
     failed = __shfl_sync(0xFFFFFFFFu, failed ? 1 : 0, 0) != 0;
   } else {
     // ----------------------------------------------------------- epilogue
-    const uint32_t ew = warp - 2u;                   // 0..7
+    const uint32_t ew = warp - (uint32_t)kFirstEpilogueWarp;   // 0..7
     const uint32_t quarter = warp & 3u;              // TMEM lanes this warp may touch
     const uint32_t half = ew >> 2;                   // which 32 of the tile's 64 channels
     const uint32_t row = quarter * 32u + lane;
@@ -672,7 +677,7 @@ psb_mma_kernel(const __grid_constant__ TmapSet maps, const __grid_constant__ Ten
   }
   tc_fence_before();
   __syncthreads();
-  if (warp == 1) {
+  if (warp == kMmaWarp) {
     tc_fence_after();
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base),
                  "r"(kTmemCols)
@@ -708,7 +713,11 @@ psb_status tensor_supported(const psb_ctx* ctx, const psb_weights* wt, const Con
   if (!wt->has_planes || a.groups != 1) return PSB_ERR_UNSUPPORTED;
   // each plane accumulates in 32 bits: |digit| <= 127, |x| <= 128
   if ((uint64_t)wt->d * 127ull * 128ull >= (1ull << 31)) return PSB_ERR_UNSUPPORTED;
-  if (wt->packed_k) return (a.KH > 255 || a.KW > 255 || a.C > 65535) ? PSB_ERR_UNSUPPORTED : PSB_OK;
+  if (wt->packed_k) {
+    // the gather kernel stages KH input-row segments of a 32-pixel strip in 48 KB of shared memory
+    const uint64_t stage = (uint64_t)wt->kpad * 4u + (uint64_t)a.KH * ((31u * a.stride + a.KW) * a.C);
+    return (a.KH > 255 || stage > 48u * 1024u) ? PSB_ERR_UNSUPPORTED : PSB_OK;
+  }
   if (a.C % 16u || a.C < 32u) return PSB_ERR_UNSUPPORTED;
   if ((uintptr_t)a.x & 15u) return PSB_ERR_UNSUPPORTED;
   if (a.stride > 8 || a.pad > 127 || a.KH > 128 || a.KW > 128) return PSB_ERR_UNSUPPORTED;

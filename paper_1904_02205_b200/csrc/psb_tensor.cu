@@ -15,7 +15,7 @@
 //            of the digit-plane tile into a ring of shared-memory stages
 //   warp 3   allocates TMEM; one thread issues the MMAs and commits them to the
 //            stage-free and accumulator-ready barriers
-//   warps 4-11 epilogue: TMEM -> registers, recombine planes, dequantise, bias,
+//   warps 4-19 epilogue: TMEM -> registers, recombine planes, dequantise, bias,
 //            shortcut, ReLU, re-quantise, vectorised stores; overlaps the next
 //            tile's MMAs through two TMEM accumulator buffers
 // Per-location draw counts (Sec. 4.5): a tile is contracted once per level present
@@ -36,7 +36,7 @@ constexpr int kTileM = 128;
 constexpr int kProducerWarps = 3;    // one issuing thread each: their barrier waits overlap
 constexpr int kMmaWarp = kProducerWarps;
 constexpr int kFirstEpilogueWarp = kMmaWarp + 1;   // a multiple of 4: warp & 3 = TMEM lane quarter
-constexpr int kEpilogueWarps = 8;
+constexpr int kEpilogueWarps = 16;
 constexpr int kThreadsTensor = 32 * (kFirstEpilogueWarp + kEpilogueWarps);
 constexpr uint32_t kTmemCols = 512;
 constexpr uint32_t kTmemBufStride = 256;
@@ -245,8 +245,8 @@ struct SharedCtl {
   unsigned long long planes_full;
   uint32_t tmem_base;
   volatile uint32_t abort;
-  float2 scb[kEpilogueWarps][32];       // per epilogue warp: (scale * 2^(e_base - log2 k), bias)
-  long long corr[kEpilogueWarps][32];   // per epilogue warp: integer addend per channel
+  float2 scb[kEpilogueWarps][16];       // per epilogue warp: (scale * 2^(e_base - log2 k), bias)
+  long long corr[kEpilogueWarps][16];   // per epilogue warp: integer addend per channel
 };
 
 // Exact round-to-nearest conversion of a 64-bit accumulator, |acc| < 2^47: split into a high
@@ -257,72 +257,76 @@ __device__ __forceinline__ float acc_to_float(long long acc) {
   return __fmaf_rn((float)hi, 16777216.0f, (float)lo);
 }
 
-// Fast output stage for the common case: only re-quantised bytes are wanted, channels-last,
-// 16 whole channels, 16-byte aligned.  Same arithmetic as dequant()/requant().
-// NARROW: every plane sum is below 2^24 in magnitude and P <= 3, so the recombination fits 32-bit
-// integers: with u = v0 + 2^7 v1 and w = (u >> 14) + v2, acc = w * 2^14 + (u mod 2^14), both parts
-// exact in fp32, and one fma rounds acc to nearest once.
-// The run-time options enter as data (a relu floor of 0 or -inf, a sign mask, an addend that may
-// be zero), not as branches, so that each instantiation stays one compact code path.
-// Integer <-> float conversions run on a slow pipe (a quarter of the FMA rate), so small integers
-// are converted with exponent tricks on the main pipes instead:
+// Output arithmetic of one 16-channel chunk held in registers (v[plane][channel]), common case:
+// only re-quantised bytes are wanted.  Same arithmetic as dequant()/requant(), arranged for the
+// main pipes: integer <-> float conversions run on a slow pipe (a quarter of the FMA rate), so
+// small integers are converted with exponent tricks instead:
 //   float(n) = as_float(0x4B000000 | n) - 2^23              for 0 <= n < 2^23
 //   float(n) = as_float(0x4B400000 + n) - 1.5 * 2^23        for |n| < 2^22
 //   rint(t)  = low bits of as_int(t + 1.5 * 2^23)           for |t| < 2^22 (the add rounds to even)
-// MODE 2: every plane sum is below 2^22 in magnitude (both halves of the accumulator by tricks);
-// MODE 1: below 2^24 (the high half by a conversion instruction); MODE 0: 64-bit recombination.
+// MODE 2: every plane sum is below 2^22 in magnitude and P <= 3: with u = v0 + 2^7 v1,
+// w = (u >> 14) + v2, acc = w * 2^14 + (u mod 2^14); both parts are exact in fp32 (by the tricks)
+// and one fma rounds acc to nearest once.  MODE 1: below 2^24 (w by a conversion instruction).
+// MODE 0: 64-bit recombination plus the per-channel integer addend.
+// The run-time options enter as data (a relu floor of 0 or -inf, a sign mask), not as branches.
+struct EpiConst {
+  float res_scale, relu_floor, inv_step, qmin_f, qmax_f;
+  uint32_t res_sign;
+};
+
+template <int P, int MODE, bool HAS_RES>
+__device__ __forceinline__ uint4 chunk_math(const uint32_t (&v)[P][16], const uint4& r4, const float2* scb,
+                                            const long long* corr, const EpiConst& c) {
+  const uint32_t rw[4] = {r4.x, r4.y, r4.z, r4.w};
+  const float res_bias = 8388608.0f + (float)c.res_sign;   // undoes the magic constant and the sign flip
+  uint32_t qw[4];
+#pragma unroll
+  for (int g = 0; g < 4; ++g) {
+    uint32_t q[4];
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+      const int j = 4 * g + e;
+      float af;
+      if (MODE > 0) {
+        int u = (int)v[0][j];
+        if (P > 1) u += (int)v[1][j] << kDigitBits;
+        int w = u >> (2 * kDigitBits);
+        if (P > 2) w += (int)v[2][j];
+        const float lo_f = __uint_as_float(0x4B000000u | ((uint32_t)u & 0x3FFFu)) - 8388608.0f;
+        const float w_f = MODE == 2 ? __int_as_float(0x4B400000 + w) - 12582912.0f : (float)w;
+        af = __fmaf_rn(w_f, 16384.0f, lo_f);
+      } else {
+        long long acc = (long long)(int)v[0][j];
+#pragma unroll
+        for (int pl = 1; pl < P; ++pl) acc += (long long)(int)v[pl][j] * (long long)(1 << (kDigitBits * pl));
+        acc += corr[j];
+        af = acc_to_float(acc);
+      }
+      const float2 sb = scb[j];
+      float y = __fmaf_rn(af, sb.x, sb.y);
+      if (HAS_RES) {
+        const uint32_t rb = ((rw[g] >> (8 * e)) & 0xFFu) ^ c.res_sign;   // byte + 128 if signed
+        y = __fmaf_rn(__uint_as_float(0x4B000000u | rb) - res_bias, c.res_scale, y);
+      }
+      y = fmaxf(y, c.relu_floor);
+      // clamp, then round half to even by adding 1.5 * 2^23: the low byte of the sum is the code
+      const float t = fminf(fmaxf(__fmul_rn(y, c.inv_step), c.qmin_f), c.qmax_f);
+      q[e] = __float_as_uint(t + 12582912.0f);
+    }
+    qw[g] = __byte_perm(__byte_perm(q[0], q[1], 0x0040), __byte_perm(q[2], q[3], 0x0040), 0x5410);
+  }
+  return make_uint4(qw[0], qw[1], qw[2], qw[3]);
+}
+
 template <int P, int MODE, bool HAS_RES>
 __device__ __noinline__ void epilogue_chunk_q(uint32_t taddr, bool valid, uint8_t* q_dst, uint4 r4,
-                                              const float2* scb, const long long* corr, float res_scale,
-                                              uint32_t res_sign, float relu_floor, float inv_step,
-                                              float qmin_f, float qmax_f) {
+                                              const float2* scb, const long long* corr, EpiConst c) {
   uint32_t v[P][16];
 #pragma unroll
   for (int pl = 0; pl < P; ++pl) tc_ld16(taddr + pl * kTileN, v[pl]);
   tc_wait_ld();
   if (!valid) return;
-  const uint32_t rw[4] = {r4.x, r4.y, r4.z, r4.w};
-  const float res_bias = 8388608.0f + (float)res_sign;   // undoes the magic constant and the sign flip
-  uint32_t q[16];
-#pragma unroll
-  for (int j = 0; j < 16; ++j) {
-    float af;
-    if (MODE > 0) {
-      // acc = w * 2^14 + lo with u = v0 + 2^7 v1, w = (u >> 14) + v2, lo = u mod 2^14: both parts
-      // are exact in fp32 and one fma rounds acc to nearest once
-      int u = (int)v[0][j];
-      if (P > 1) u += (int)v[1][j] << kDigitBits;
-      int w = u >> (2 * kDigitBits);
-      if (P > 2) w += (int)v[2][j];
-      const float lo_f = __uint_as_float(0x4B000000u | ((uint32_t)u & 0x3FFFu)) - 8388608.0f;
-      const float w_f = MODE == 2 ? __int_as_float(0x4B400000 + w) - 12582912.0f : (float)w;
-      af = __fmaf_rn(w_f, 16384.0f, lo_f);
-    } else {
-      long long acc = (long long)(int)v[0][j];
-#pragma unroll
-      for (int pl = 1; pl < P; ++pl) acc += (long long)(int)v[pl][j] * (long long)(1 << (kDigitBits * pl));
-      acc += corr[j];
-      af = acc_to_float(acc);
-    }
-    const float2 sb = scb[j];
-    float y = __fmaf_rn(af, sb.x, sb.y);
-    if (HAS_RES) {
-      const uint32_t rb = ((rw[j >> 2] >> (8 * (j & 3))) & 0xFFu) ^ res_sign;   // byte + 128 if signed
-      y = __fmaf_rn(__uint_as_float(0x4B000000u | rb) - res_bias, res_scale, y);
-    }
-    y = fmaxf(y, relu_floor);
-    // clamp, then round half to even by adding 1.5 * 2^23: the low byte of the sum is the code
-    const float t = fminf(fmaxf(__fmul_rn(y, inv_step), qmin_f), qmax_f);
-    q[j] = __float_as_uint(t + 12582912.0f);
-  }
-  uint32_t qw[4];
-#pragma unroll
-  for (int g = 0; g < 4; ++g) {
-    const uint32_t lo = __byte_perm(q[4 * g], q[4 * g + 1], 0x0040);
-    const uint32_t hi = __byte_perm(q[4 * g + 2], q[4 * g + 3], 0x0040);
-    qw[g] = __byte_perm(lo, hi, 0x5410);
-  }
-  *reinterpret_cast<uint4*>(q_dst) = make_uint4(qw[0], qw[1], qw[2], qw[3]);
+  *reinterpret_cast<uint4*>(q_dst) = chunk_math<P, MODE, HAS_RES>(v, r4, scb, corr, c);
 }
 
 // General output stage: any combination of outputs, layouts, ragged channel counts.
@@ -372,6 +376,85 @@ __device__ __noinline__ void epilogue_chunk(const TensorParams& p, uint32_t tadd
   }
   if (vec && a.q_out)
     *reinterpret_cast<uint4*>((uint8_t*)a.q_out + (size_t)m * a.O + o_base) = make_uint4(qw[0], qw[1], qw[2], qw[3]);
+}
+
+// Epilogue loop of one warp for the common case: one draw count for the whole layer, only
+// re-quantised bytes wanted, channels-last, whole 16-channel chunks.  The warp owns 32 rows
+// (its TMEM lane quarter) x 16 channels of every tile.  Per tile: wait for the accumulator, pull
+// the chunk into registers, hand the TMEM buffer back at once (the MMA of the tile after next can
+// start), then do the arithmetic and the 16-byte store.  Shortcut bytes are fetched one tile ahead.
+// Returns true if a wait timed out.
+template <int P, int MODE, bool HAS_RES>
+__device__ __noinline__ bool epilogue_uniform(const TensorParams& p, SharedCtl* ctl, uint32_t tmem_base,
+                                              uint32_t ew, uint32_t lane, EpiConst c) {
+  const ConvArgs& a = p.a;
+  const uint32_t quarter = ew & 3u, sub = ew >> 2;
+  const uint32_t row = quarter * 32u + lane;
+  const uint32_t l = a.uniform_log2k;
+  const bool use_corr = p.corr[l] != nullptr;
+  volatile uint32_t* abort = &ctl->abort;
+  const uint8_t* res_base = (const uint8_t*)a.residual;
+  const float2* scb = ctl->scb[ew];
+  const long long* corr = ctl->corr[ew];
+  TileIter ti;
+  ti.init(p);
+  uint32_t pass = 0, cur_o_tile = 0xFFFFFFFFu;
+  uint4 r_next = make_uint4(0, 0, 0, 0);
+  if (HAS_RES && ti.valid()) {
+    const uint32_t m = ti.m_tile * kTileM + row, ob = ti.o_tile * kTileN + sub * 16u;
+    if (m < p.M && ob < a.O) r_next = __ldg(reinterpret_cast<const uint4*>(res_base + (size_t)m * a.O + ob));
+  }
+  while (ti.valid()) {
+    const uint32_t m = ti.m_tile * kTileM + row;
+    const uint32_t o_tile = ti.o_tile;
+    const uint32_t o_base = o_tile * kTileN + sub * 16u;
+    const bool active = o_base < a.O;          // warp-uniform
+    ti.next();
+    if (o_tile != cur_o_tile) {
+      // per-channel constants of this channel tile: the warp keeps its own copy of its 16 channels
+      __syncwarp();
+      if (lane < 16u) {
+        const uint32_t o = o_base + lane;
+        float2 sb = make_float2(0.f, 0.f);
+        long long cr = 0;
+        if (o < a.O) {
+          sb.x = ldexpf(a.scale[o], a.e_base[o] - (int)l);
+          sb.y = a.bias[o];
+          if (use_corr) cr = p.corr[l][o];
+        }
+        ctl->scb[ew][lane] = sb;
+        ctl->corr[ew][lane] = cr;
+      }
+      cur_o_tile = o_tile;
+      __syncwarp();
+    }
+    const uint4 r_cur = r_next;
+    if (HAS_RES && ti.valid()) {
+      const uint32_t mn = ti.m_tile * kTileM + row, ob = ti.o_tile * kTileN + sub * 16u;
+      r_next = make_uint4(0, 0, 0, 0);
+      if (mn < p.M && ob < a.O) r_next = __ldg(reinterpret_cast<const uint4*>(res_base + (size_t)mn * a.O + ob));
+    }
+    const uint32_t buf = pass & 1u, aph = (pass >> 1) & 1u;
+    const bool ok = mbar_wait(smem_u32(&ctl->acc_full[buf]), aph, abort, 32);
+    if (__any_sync(0xFFFFFFFFu, !ok)) return true;
+    tc_fence_after();
+    uint32_t v[P][16];
+    if (active) {
+      const uint32_t taddr = tmem_base + buf * kTmemBufStride + ((quarter * 32u) << 16) + sub * 16u;
+#pragma unroll
+      for (int pl = 0; pl < P; ++pl) tc_ld16(taddr + pl * kTileN, v[pl]);
+      tc_wait_ld();
+    }
+    // the chunk is in registers: give the accumulator buffer back before doing the arithmetic
+    tc_fence_before();
+    __syncwarp();
+    if (lane == 0) mbar_arrive(smem_u32(&ctl->acc_empty[buf]));
+    if (active && m < p.M)
+      *reinterpret_cast<uint4*>((uint8_t*)a.q_out + (size_t)m * a.O + o_base) =
+          chunk_math<P, MODE, HAS_RES>(v, r_cur, scb, corr, c);
+    ++pass;
+  }
+  return false;
 }
 
 template <int BK>
@@ -543,126 +626,116 @@ psb_mma_kernel(const __grid_constant__ TmapSet maps, const __grid_constant__ Ten
     failed = __shfl_sync(0xFFFFFFFFu, failed ? 1 : 0, 0) != 0;
   } else {
     // ----------------------------------------------------------- epilogue
-    const uint32_t ew = warp - (uint32_t)kFirstEpilogueWarp;   // 0..7
-    const uint32_t quarter = warp & 3u;              // TMEM lanes this warp may touch
-    const uint32_t half = ew >> 2;                   // which 32 of the tile's 64 channels
+    // 16 warps: warp & 3 selects the TMEM lane quarter (32 rows), ew >> 2 the 16 of the tile's 64
+    // channels.
+    const uint32_t ew = warp - (uint32_t)kFirstEpilogueWarp;   // 0..15
+    const uint32_t quarter = ew & 3u;
+    const uint32_t sub = ew >> 2;
     const uint32_t row = quarter * 32u + lane;
     const ConvArgs& a = p.a;
     const bool q_only = a.q_out && !a.f32_out && !a.acc_out && p.vec_ok;
+    EpiConst ec;
+    ec.res_scale = a.residual_scale;
     // a clamp at qmin >= 0 already removes negatives, so the relu only matters for signed codes
-    const float relu_floor = (a.relu && a.qmin < 0) ? 0.0f : __int_as_float(0xFF800000);
-    const uint32_t res_sign = a.residual_dtype == PSB_DT_S8 ? 0x80u : 0u;
-    const bool pre_res = q_only && a.residual != nullptr;
-    const uint8_t* res_base = (const uint8_t*)a.residual;
-    uint32_t pass = 0, cur_key = 0xFFFFFFFFu;
-    TileIter ti;
-    ti.init(p);
-    uint32_t m_tile = ti.m_tile, o_tile = ti.o_tile;
-    // shortcut bytes of the first tile; later tiles' bytes are fetched one tile ahead so that
-    // their DRAM latency hides behind the current tile's work
-    uint4 r_next[2] = {make_uint4(0, 0, 0, 0), make_uint4(0, 0, 0, 0)};
-    bool have = ti.valid();
-    if (have && pre_res) {
-      const uint32_t m = m_tile * kTileM + row, ob = o_tile * kTileN + half * 32u;
-      if (m < p.M) {
-        if (ob + 16u <= a.O) r_next[0] = __ldg(reinterpret_cast<const uint4*>(res_base + (size_t)m * a.O + ob));
-        if (ob + 32u <= a.O) r_next[1] = __ldg(reinterpret_cast<const uint4*>(res_base + (size_t)m * a.O + ob + 16u));
+    ec.relu_floor = (a.relu && a.qmin < 0) ? 0.0f : __int_as_float(0xFF800000);
+    ec.inv_step = a.inv_step;
+    ec.qmin_f = (float)a.qmin;
+    ec.qmax_f = (float)a.qmax;
+    ec.res_sign = a.residual_dtype == PSB_DT_S8 ? 0x80u : 0u;
+    const uint32_t P0 = p.planes[a.uniform_log2k < (uint32_t)kMaxLevels ? a.uniform_log2k : 0u];
+    if (!a.kmap && q_only && a.O % 16u == 0u && (P0 == 3u || P0 == 4u)) {
+      const uint32_t mode = (p.corr[a.uniform_log2k] != nullptr || P0 == 4u) ? 0u : p.narrow;
+#define PSB_UNI(PV, MV, RV) failed = epilogue_uniform<PV, MV, RV>(p, ctl, tmem_base, ew, lane, ec)
+      if (a.residual) {
+        if (P0 == 4u) PSB_UNI(4, 0, true); else if (mode == 2u) PSB_UNI(3, 2, true);
+        else if (mode == 1u) PSB_UNI(3, 1, true); else PSB_UNI(3, 0, true);
+      } else {
+        if (P0 == 4u) PSB_UNI(4, 0, false); else if (mode == 2u) PSB_UNI(3, 2, false);
+        else if (mode == 1u) PSB_UNI(3, 1, false); else PSB_UNI(3, 0, false);
       }
-    }
-    while (!failed && have) {
-      const uint32_t m0 = m_tile * kTileM;
-      const uint32_t levels = tile_levels(p, m0) & a.level_mask;
-      const uint32_t m = m0 + row;
-      const bool in_range = m < p.M;
-      const uint32_t my_level = in_range ? (a.kmap ? (uint32_t)a.kmap[m] : a.uniform_log2k) : 0xFFu;
-      if (in_range && (my_level >= (uint32_t)kMaxLevels || !((a.level_mask >> my_level) & 1u)))
-        atomicOr(a.err, kDevErrBadLevel);
-      const uint32_t o_tile_cur = o_tile;
-      const uint32_t o_base0 = o_tile_cur * kTileN + half * 32u;
-      const uint4 r_cur[2] = {r_next[0], r_next[1]};
-      // next tile (and its shortcut bytes)
-      ti.next();
-      const uint32_t m_tile_n = ti.m_tile, o_tile_n = ti.o_tile;
-      const bool have_n = ti.valid();
-      if (have_n && pre_res) {
-        const uint32_t mn = m_tile_n * kTileM + row, ob = o_tile_n * kTileN + half * 32u;
-        r_next[0] = make_uint4(0, 0, 0, 0);
-        r_next[1] = make_uint4(0, 0, 0, 0);
-        if (mn < p.M) {
-          if (ob + 16u <= a.O) r_next[0] = __ldg(reinterpret_cast<const uint4*>(res_base + (size_t)mn * a.O + ob));
-          if (ob + 32u <= a.O) r_next[1] = __ldg(reinterpret_cast<const uint4*>(res_base + (size_t)mn * a.O + ob + 16u));
-        }
-      }
-      for (uint32_t todo = levels & 0x7Fu; todo && !failed; todo &= todo - 1u) {
-        const uint32_t l = (uint32_t)__ffs((int)todo) - 1u;
-        const uint32_t P = p.planes[l];
-        const uint32_t buf = pass & 1u, aph = (pass >> 1) & 1u;
-        const bool use_corr = p.corr[l] != nullptr;
-        // per-channel constants of this (channel tile, level): every warp keeps its own copy of
-        // its 32 channels, so no CTA-wide barrier is needed; refreshed only when the pair changes
-        const uint32_t key = o_tile_cur * 8u + l;
-        if (key != cur_key) {
-          __syncwarp();
-          const uint32_t o = o_base0 + lane;
-          float2 sb = make_float2(0.f, 0.f);
-          long long cr = 0;
-          if (o < a.O) {
-            sb.x = ldexpf(a.scale[o], a.e_base[o] - (int)l);
-            sb.y = a.bias[o];
-            if (use_corr) cr = p.corr[l][o];
-          }
-          ctl->scb[ew][lane] = sb;
-          ctl->corr[ew][lane] = cr;
-          cur_key = key;
-          __syncwarp();
-        }
-        if (lane == 0) {
-          if (!mbar_wait(smem_u32(&ctl->acc_full[buf]), aph, abort, 32)) failed = true;
-        }
-        failed = __shfl_sync(0xFFFFFFFFu, failed ? 1 : 0, 0) != 0;
-        if (failed) break;
-        tc_fence_after();
-        const bool valid = in_range && my_level == l;
-#pragma unroll
-        for (uint32_t c2 = 0; c2 < 2u; ++c2) {   // unrolled: r_cur[c2] must stay in registers
-          const uint32_t o_base = o_base0 + c2 * 16u;
-          if (o_base >= a.O) break;
-          const uint32_t taddr = tmem_base + buf * kTmemBufStride + ((quarter * 32u) << 16) + half * 32u + c2 * 16u;
-          const float2* scb = &ctl->scb[ew][c2 * 16u];
-          const long long* corr = &ctl->corr[ew][c2 * 16u];
-          if (q_only && o_base + 16u <= a.O) {
-            uint8_t* q_dst = (uint8_t*)a.q_out + (size_t)m * a.O + o_base;
-            const uint32_t mode = use_corr ? 0u : p.narrow;
-#define PSB_EPI(PV, MV, RV) epilogue_chunk_q<PV, MV, RV>(taddr, valid, q_dst, r_cur[c2], scb, corr, a.residual_scale, res_sign, relu_floor, a.inv_step, (float)a.qmin, (float)a.qmax)
-#define PSB_EPI_P(MV, RV) do { if (P == 3) PSB_EPI(3, MV, RV); else if (P == 2) PSB_EPI(2, MV, RV); else PSB_EPI(1, MV, RV); } while (0)
-            if (a.residual) {
-              if (mode == 2) PSB_EPI_P(2, true); else if (mode == 1) PSB_EPI_P(1, true);
-              else if (P == 4) PSB_EPI(4, 0, true); else PSB_EPI_P(0, true);
-            } else {
-              if (mode == 2) PSB_EPI_P(2, false); else if (mode == 1) PSB_EPI_P(1, false);
-              else if (P == 4) PSB_EPI(4, 0, false); else PSB_EPI_P(0, false);
+#undef PSB_UNI
+    } else {
+      // general loop: per-location draw counts, any outputs and layouts, ragged channel counts
+      const float2* scb = ctl->scb[ew];
+      const long long* corr = ctl->corr[ew];
+      uint32_t pass = 0, cur_key = 0xFFFFFFFFu;
+      TileIter ti;
+      for (ti.init(p); !failed && ti.valid(); ti.next()) {
+        const uint32_t m0 = ti.m_tile * kTileM, o_tile = ti.o_tile;
+        const uint32_t levels = tile_levels(p, m0) & a.level_mask;
+        const uint32_t m = m0 + row;
+        const bool in_range = m < p.M;
+        const uint32_t my_level = in_range ? (a.kmap ? (uint32_t)a.kmap[m] : a.uniform_log2k) : 0xFFu;
+        if (in_range && (my_level >= (uint32_t)kMaxLevels || !((a.level_mask >> my_level) & 1u)))
+          atomicOr(a.err, kDevErrBadLevel);
+        const uint32_t o_base = o_tile * kTileN + sub * 16u;
+        const size_t oidx = (size_t)m * a.O + o_base;
+        const bool fast = q_only && o_base + 16u <= a.O;
+        uint4 r4 = make_uint4(0, 0, 0, 0);
+        if (fast && a.residual && in_range)
+          r4 = __ldg(reinterpret_cast<const uint4*>((const uint8_t*)a.residual + oidx));
+        for (uint32_t todo = levels & 0x7Fu; todo && !failed; todo &= todo - 1u) {
+          const uint32_t l = (uint32_t)__ffs((int)todo) - 1u;
+          const uint32_t P = p.planes[l];
+          const uint32_t buf = pass & 1u, aph = (pass >> 1) & 1u;
+          const bool use_corr = p.corr[l] != nullptr;
+          // per-channel constants of this (channel tile, level), refreshed only when the pair changes
+          const uint32_t key = o_tile * 8u + l;
+          if (key != cur_key) {
+            __syncwarp();
+            if (lane < 16u) {
+              const uint32_t o = o_base + lane;
+              float2 sb = make_float2(0.f, 0.f);
+              long long cr = 0;
+              if (o < a.O) {
+                sb.x = ldexpf(a.scale[o], a.e_base[o] - (int)l);
+                sb.y = a.bias[o];
+                if (use_corr) cr = p.corr[l][o];
+              }
+              ctl->scb[ew][lane] = sb;
+              ctl->corr[ew][lane] = cr;
             }
+            cur_key = key;
+            __syncwarp();
+          }
+          const bool ok = mbar_wait(smem_u32(&ctl->acc_full[buf]), aph, abort, 32);
+          failed = __any_sync(0xFFFFFFFFu, !ok) != 0;
+          if (failed) break;
+          tc_fence_after();
+          const uint32_t taddr = tmem_base + buf * kTmemBufStride + ((quarter * 32u) << 16) + sub * 16u;
+          const bool valid = in_range && my_level == l;
+          if (o_base < a.O) {
+            if (fast) {
+              uint8_t* q_dst = (uint8_t*)a.q_out + oidx;
+              const uint32_t mode = (use_corr || P > 3u) ? 0u : p.narrow;
+#define PSB_EPI(PV, MV, RV) epilogue_chunk_q<PV, MV, RV>(taddr, valid, q_dst, r4, scb, corr, ec)
+#define PSB_EPI_P(MV, RV) do { if (P == 3) PSB_EPI(3, MV, RV); else if (P == 2) PSB_EPI(2, MV, RV); else PSB_EPI(1, MV, RV); } while (0)
+              if (a.residual) {
+                if (mode == 2) PSB_EPI_P(2, true); else if (mode == 1) PSB_EPI_P(1, true);
+                else if (P == 4) PSB_EPI(4, 0, true); else PSB_EPI_P(0, true);
+              } else {
+                if (mode == 2) PSB_EPI_P(2, false); else if (mode == 1) PSB_EPI_P(1, false);
+                else if (P == 4) PSB_EPI(4, 0, false); else PSB_EPI_P(0, false);
+              }
 #undef PSB_EPI_P
 #undef PSB_EPI
-          } else {
-            const uint32_t ohow = a.OH * a.OW;
-            const uint32_t n = in_range ? m / ohow : 0u, pix = in_range ? m % ohow : 0u;
-            switch (P) {
-              case 1: epilogue_chunk<1>(p, taddr, o_base, m, valid, n, pix, scb, corr, use_corr); break;
-              case 2: epilogue_chunk<2>(p, taddr, o_base, m, valid, n, pix, scb, corr, use_corr); break;
-              case 3: epilogue_chunk<3>(p, taddr, o_base, m, valid, n, pix, scb, corr, use_corr); break;
-              default: epilogue_chunk<4>(p, taddr, o_base, m, valid, n, pix, scb, corr, use_corr); break;
+            } else {
+              const uint32_t ohow = a.OH * a.OW;
+              const uint32_t n = in_range ? m / ohow : 0u, pix = in_range ? m % ohow : 0u;
+              switch (P) {
+                case 1: epilogue_chunk<1>(p, taddr, o_base, m, valid, n, pix, scb, corr, use_corr); break;
+                case 2: epilogue_chunk<2>(p, taddr, o_base, m, valid, n, pix, scb, corr, use_corr); break;
+                case 3: epilogue_chunk<3>(p, taddr, o_base, m, valid, n, pix, scb, corr, use_corr); break;
+                default: epilogue_chunk<4>(p, taddr, o_base, m, valid, n, pix, scb, corr, use_corr); break;
+              }
             }
           }
+          tc_fence_before();
+          __syncwarp();
+          if (lane == 0) mbar_arrive(smem_u32(&ctl->acc_empty[buf]));
+          ++pass;
         }
-        tc_fence_before();
-        __syncwarp();
-        if (lane == 0) mbar_arrive(smem_u32(&ctl->acc_empty[buf]));
-        ++pass;
       }
-      have = have_n;
-      m_tile = m_tile_n;
-      o_tile = o_tile_n;
     }
   }
 

@@ -109,8 +109,11 @@ psb_status run_layer(psb_ctx* ctx, const psb_weights* wt, const void* x_dev, uin
   if (path != PSB_PATH_SHIFT_ADD) {
     // the MMA takes signed bytes: unsigned data above 127 qualifies only where the activation
     // matrix is gathered explicitly (packed-K filters), which stores x - 128
-    tensor_ok = (in_dtype == PSB_DT_S8 || amax <= 127u || wt->packed_k) &&
-                tensor_supported(ctx, wt, a) == PSB_OK;
+    // the MMA takes signed bytes.  Unsigned data above 127 still qualifies where it can be fed as
+    // x - 128 and corrected by 128 * sum(W): packed-K filters (the gathered matrix is built with
+    // the offset) and layers without padding (one pass flips the top bit of the whole input)
+    const bool needs_offset = in_dtype == PSB_DT_U8 && amax > 127u;
+    tensor_ok = (!needs_offset || wt->packed_k || pad == 0) && tensor_supported(ctx, wt, a) == PSB_OK;
     if (path == PSB_PATH_TENSOR && !tensor_ok) return PSB_ERR_UNSUPPORTED;
     if (path == PSB_PATH_AUTO && M < (wt->packed_k ? 128u : 32u)) tensor_ok = false;
   }
@@ -140,6 +143,21 @@ psb_status run_layer(psb_ctx* ctx, const psb_weights* wt, const void* x_dev, uin
       a.KH = 1; a.KW = 1; a.stride = 1; a.pad = 0;
       add_corr = offset != 0;
       amax = 128;
+    } else if (in_dtype == PSB_DT_U8 && amax > 127u) {
+      const size_t bytes = (size_t)n * c * h * w;   // a multiple of 16: c is
+      st = ensure_scratch(ctx, 1, bytes);
+      if (st != PSB_OK) return st;
+      if (launch_offset128(a.x, ctx->scratch[1], bytes, s) != cudaSuccess) return PSB_ERR_CUDA;
+      a.x = ctx->scratch[1];
+      a.in_dtype = PSB_DT_S8;
+      add_corr = true;
+      amax = 128;
+    }
+    if (add_corr) {
+      // 128 * (row sums of the integer filter) for every level this call may use
+      for (uint32_t l = 0; l < (uint32_t)kMaxLevels; ++l)
+        if (wt->level[l].corr128 && (ctx->kmap || l == ctx->uniform_log2k))
+          if (launch_corr128(wt, l, s) != cudaSuccess) return PSB_ERR_CUDA;
     }
     st = launch_tensor(ctx, wt, a, amax, add_corr, s);
     if (st != PSB_OK) return st;
@@ -278,7 +296,7 @@ psb_status psb_sample_weights(psb_ctx* ctx, const float* w_dev, const psb_wshape
         w->level[l].planes_count = P;
         ok = cudaMalloc(&w->level[l].planes, bytes) == cudaSuccess &&
              cudaMemsetAsync(w->level[l].planes, 0, bytes, s) == cudaSuccess;
-        if (ok && w->packed_k)
+        if (ok)
           ok = cudaMalloc(&w->level[l].corr128, sizeof(long long) * shape->out_ch) == cudaSuccess;
       }
     }

@@ -34,7 +34,7 @@ struct LevelStore {
   int32_t* wint = nullptr;  // [O][KH][KW][Cg]  signed integer filter, channels innermost
   int8_t* planes = nullptr; // [O_tiles][P][kTileN][Kpad]  signed 7-bit digits, Kpad = KH*KW*Cpad
   int planes_count = 0;
-  long long* corr128 = nullptr;  // [O] 128 * sum of the filter row (packed-K filters only)
+  long long* corr128 = nullptr;  // [O] 128 * sum of the filter row, refreshed by the calls that need it
 };
 
 }  // namespace psb
@@ -138,6 +138,8 @@ cudaError_t launch_shift_add(const ConvArgs& a, const WintTable& wt, cudaStream_
 // gathers [M][kpad] signed bytes (x - offset; zero padding becomes -offset, K padding 0)
 cudaError_t launch_im2col_s8(const ConvArgs& a, uint32_t kpad, uint32_t offset, int8_t* dst,
                              cudaStream_t s);
+cudaError_t launch_corr128(const psb_weights* wt, uint32_t level, cudaStream_t s);
+cudaError_t launch_offset128(const void* src, void* dst, size_t bytes, cudaStream_t s);
 cudaError_t launch_nchw_to_nhwc(const void* src, void* dst, uint32_t N, uint32_t C, uint32_t HW,
                                 uint32_t elem_bytes, cudaStream_t s);
 cudaError_t launch_nhwc_to_nchw(const void* src, void* dst, uint32_t N, uint32_t C, uint32_t HW,

@@ -276,15 +276,14 @@ uint32_t fill_sample_params(const float* w_dev, const psb_weights* wt, uint32_t*
   return row_blocks * p.ch_chunks;
 }
 
-void launch_corr128(const psb_weights* wt, cudaStream_t s) {
-  const uint32_t O = wt->shape.out_ch;
-  for (int l = 0; l < kMaxLevels; ++l)
-    if (wt->level[l].corr128)
-      corr128_kernel<<<(O * 32 + kThreads - 1) / kThreads, kThreads, 0, s>>>(wt->level[l].wint, O, wt->d,
-                                                                            wt->level[l].corr128);
-}
-
 }  // namespace
+
+cudaError_t launch_corr128(const psb_weights* wt, uint32_t level, cudaStream_t s) {
+  const uint32_t O = wt->shape.out_ch;
+  corr128_kernel<<<(O * 32 + kThreads - 1) / kThreads, kThreads, 0, s>>>(wt->level[level].wint, O, wt->d,
+                                                                        wt->level[level].corr128);
+  return cudaGetLastError();
+}
 
 cudaError_t launch_sampler(const float* w_dev, psb_weights* wt, uint32_t* err_dev, cudaStream_t s) {
   const uint32_t O = wt->shape.out_ch;
@@ -295,7 +294,6 @@ cudaError_t launch_sampler(const float* w_dev, psb_weights* wt, uint32_t* err_de
   SampleParams p;
   const uint32_t blocks = fill_sample_params(w_dev, wt, wt->e_max, p);
   sample_kernel<<<blocks, kThreads, 0, s>>>(p);
-  if (wt->packed_k) launch_corr128(wt, s);
   return cudaGetLastError();
 }
 
@@ -367,7 +365,6 @@ psb_status sample_batch_run(psb_ctx* ctx, psb_sample_batch* b, uint64_t seed, cu
   emax_batch_kernel<<<b->emax_grid, kThreads, 0, s>>>(b->entries_dev, b->n, ctx->err_dev);
   sample_batch_kernel<<<b->sample_grid, kThreads, 0, s>>>(b->entries_dev, b->n, (uint32_t)seed,
                                                          (uint32_t)(seed >> 32));
-  for (uint32_t i = 0; i < b->n_packed; ++i) launch_corr128(b->packed[i], s);
   return cudaGetLastError() == cudaSuccess ? PSB_OK : PSB_ERR_CUDA;
 }
 

@@ -72,6 +72,77 @@ __global__ void __launch_bounds__(256) conv_direct_kernel(const ConvArgs a, cons
   }
 }
 
+// Depthwise filters (one input channel per output channel), channels-last, one draw count for
+// the layer: a thread owns 8 consecutive channels of one output location.  The block keeps the
+// layer's integer filter in shared memory as [tap][channel]; activations come in 8-byte loads;
+// the integer sum x * W_k over the taps is Eq. 9 summed over the draws.  Writes 8 codes at once.
+__global__ void __launch_bounds__(256) dwconv_nhwc8_kernel(const ConvArgs a, const int32_t* __restrict__ wint) {
+  extern __shared__ int32_t dw_w[];   // [KH*KW][C]
+  const uint32_t taps = a.KH * a.KW, C = a.C;
+  for (uint32_t i = threadIdx.x; i < taps * C; i += blockDim.x) dw_w[(i % taps) * C + i / taps] = wint[i];
+  __syncthreads();
+  const uint32_t level = a.uniform_log2k;
+  const uint32_t groups = C / 8u;
+  const size_t total = (size_t)a.N * a.OH * a.OW * groups;
+  const bool has_res = a.residual != nullptr;
+  for (size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x; idx < total;
+       idx += (size_t)gridDim.x * blockDim.x) {
+    const uint32_t g = (uint32_t)(idx % groups);
+    const size_t pix = idx / groups;
+    const uint32_t ox = (uint32_t)(pix % a.OW), oy = (uint32_t)((pix / a.OW) % a.OH);
+    const uint32_t n = (uint32_t)(pix / ((size_t)a.OW * a.OH));
+    const uint32_t c0 = g * 8u;
+    long long acc[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+    for (uint32_t kh = 0; kh < a.KH; ++kh) {
+      const int iy = (int)(oy * a.stride + kh) - (int)a.pad;
+      if (iy < 0 || iy >= (int)a.H) continue;
+      for (uint32_t kw = 0; kw < a.KW; ++kw) {
+        const int ix = (int)(ox * a.stride + kw) - (int)a.pad;
+        if (ix < 0 || ix >= (int)a.W) continue;
+        const uint2 xv = __ldg(reinterpret_cast<const uint2*>(
+            (const uint8_t*)a.x + (((size_t)n * a.H + iy) * a.W + ix) * C + c0));
+        const int32_t* wr = dw_w + (kh * a.KW + kw) * C + c0;
+        const int4 w0 = *reinterpret_cast<const int4*>(wr), w1 = *reinterpret_cast<const int4*>(wr + 4);
+        const int ws[8] = {w0.x, w0.y, w0.z, w0.w, w1.x, w1.y, w1.z, w1.w};
+        const uint32_t xw[2] = {xv.x, xv.y};
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+          const uint32_t b = (xw[j >> 2] >> (8 * (j & 3))) & 0xFFu;
+          const int xi = a.in_dtype == PSB_DT_U8 ? (int)b : (int)(int8_t)b;
+          acc[j] += (long long)xi * (long long)ws[j];
+        }
+      }
+    }
+    const size_t oidx = pix * C + c0;
+    uint32_t rw[2] = {0, 0};
+    if (has_res) {
+      const uint2 rv = __ldg(reinterpret_cast<const uint2*>((const uint8_t*)a.residual + oidx));
+      rw[0] = rv.x; rw[1] = rv.y;
+    }
+    uint32_t qw[2] = {0, 0};
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+      const uint32_t o = c0 + j;
+      const float sc = ldexpf(a.scale[o], a.e_base[o] - (int)level);
+      int rb = (int)((rw[j >> 2] >> (8 * (j & 3))) & 0xFFu);
+      if (a.residual_dtype == PSB_DT_S8) rb = (int)(int8_t)rb;
+      const float y = dequant(acc[j], sc, a.bias[o], has_res, rb, a.residual_scale, a.relu != 0);
+      const int q = requant(y, a.inv_step, a.qmin, a.qmax);
+      qw[j >> 2] |= ((uint32_t)q & 0xFFu) << (8 * (j & 3));
+    }
+    *reinterpret_cast<uint2*>((uint8_t*)a.q_out + oidx) = make_uint2(qw[0], qw[1]);
+  }
+}
+
+// x ^ 0x80 over a whole tensor: unsigned bytes become (x - 128) as signed bytes, 16 per thread.
+__global__ void offset128_kernel(const uint4* __restrict__ src, uint4* __restrict__ dst, size_t n16) {
+  for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n16; i += (size_t)gridDim.x * blockDim.x) {
+    uint4 v = __ldg(src + i);
+    v.x ^= 0x80808080u; v.y ^= 0x80808080u; v.z ^= 0x80808080u; v.w ^= 0x80808080u;
+    dst[i] = v;
+  }
+}
+
 // Explicit gather of the activation matrix for filters with few input channels (e.g. a 7x7
 // stem on 3 channels): row m = output location, column k = (kh, kw, ci) flattened, padded with
 // zeros to kpad.  Values are stored minus `offset` as signed bytes; a padded input position is the
@@ -226,8 +297,29 @@ uint32_t grid_for(size_t total, uint32_t threads) {
 
 }  // namespace
 
+cudaError_t launch_offset128(const void* src, void* dst, size_t bytes, cudaStream_t s) {
+  const size_t n16 = bytes / 16;
+  offset128_kernel<<<grid_for(n16, 256), 256, 0, s>>>((const uint4*)src, (uint4*)dst, n16);
+  return cudaGetLastError();
+}
+
 cudaError_t launch_shift_add(const ConvArgs& a, const WintTable& wt, cudaStream_t s) {
   size_t total = (size_t)a.N * a.OH * a.OW * a.O;
+  // depthwise, channels-last, one draw count, only codes wanted: the vectorised kernel
+  const size_t dw_smem = (size_t)a.KH * a.KW * a.C * sizeof(int32_t);
+  if (a.groups == a.C && a.O == a.C && a.C % 8u == 0 && !a.kmap && a.q_out && !a.f32_out && !a.acc_out &&
+      !a.out_nchw && dw_smem <= 64 * 1024 &&
+      !(((uintptr_t)a.x | (uintptr_t)a.q_out | (uintptr_t)a.residual) & 7u)) {
+    static bool attr_set = false;
+    if (!attr_set) {
+      cudaFuncSetAttribute(dwconv_nhwc8_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 64 * 1024);
+      attr_set = true;
+    }
+    uint32_t blocks = grid_for(total / 8, 256);
+    if (blocks > 148u * 4u) blocks = 148u * 4u;
+    dwconv_nhwc8_kernel<<<blocks, 256, dw_smem, s>>>(a, wt.w[a.uniform_log2k]);
+    return cudaGetLastError();
+  }
   conv_direct_kernel<<<grid_for(total, 256), 256, 0, s>>>(a, wt);
   return cudaGetLastError();
 }

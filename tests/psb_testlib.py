@@ -19,7 +19,7 @@ def oracle_layer(orc, w, x, layout, groups, stride, pad, seed, layer_id, levels,
 
 def gpu_layer(psb, ctx, w, x, layout, groups, stride, pad, seed, layer_id, levels, kmap, uniform_log2k,
               scale, bias, relu, inv_step, qmin, qmax, out_dtype, residual=None, res_scale=0.0,
-              exp_bits=4, norm=0, in_max=0, path=0, guard=True):
+              exp_bits=4, norm=0, in_max=0, path=0, guard=True, want=("q", "f32", "acc")):
     import torch
 
     dev = ctx.device
@@ -44,11 +44,10 @@ def gpu_layer(psb, ctx, w, x, layout, groups, stride, pad, seed, layer_id, level
     bufs = {"q": torch.full((numel + 2 * G,), 0x5A, dtype=qdt, device=dev),
             "f32": torch.full((numel + 2 * G,), -777.0, dtype=torch.float32, device=dev),
             "acc": torch.full((numel + 2 * G,), -(1 << 60) + 7, dtype=torch.int64, device=dev)}
-    out = {k: v[G:G + numel].view(oshape) for k, v in bufs.items()}
+    out = {k: v[G:G + numel].view(oshape) for k, v in bufs.items() if k in want}
     res = ctx.conv2d(wt, t(x), layout, stride, pad, t(scale), t(bias), relu, inv_step, qmin, qmax,
                      out_dtype=out_dtype, residual=None if residual is None else t(residual),
-                     residual_scale=res_scale, in_max=in_max, path=path, want=("q", "f32", "acc"),
-                     out=out)
+                     residual_scale=res_scale, in_max=in_max, path=path, want=want, out=out)
     status = ctx.device_status()
     used = ctx.last_path()
     host = {k: v.cpu().numpy() for k, v in res.items()}
@@ -60,8 +59,8 @@ def gpu_layer(psb, ctx, w, x, layout, groups, stride, pad, seed, layer_id, level
             assert np.all(full[:G] == fill) and np.all(full[G + numel:] == fill), "guard band of %s overwritten" % k
     ctx.set_sample_map(None, 0)
     wt.free()
-    return dict(W={l: exported[l][0] for l in levels}, e_base=exported[levels[0]][1], acc=host["acc"],
-                f32=host["f32"], q=host["q"], status=status, path=used)
+    return dict(W={l: exported[l][0] for l in levels}, e_base=exported[levels[0]][1], acc=host.get("acc"),
+                f32=host.get("f32"), q=host.get("q"), status=status, path=used)
 
 
 def compare(g, o, levels):
@@ -69,8 +68,12 @@ def compare(g, o, levels):
     assert np.array_equal(g["e_base"], o["e_base"]), "e_base"
     for l in levels:
         assert np.array_equal(g["W"][l].astype(np.int64), o["W"][l]), "integer filter, level %d" % l
-    assert np.array_equal(g["acc"], o["acc"]), "accumulators: %d of %d differ" % (
-        int((g["acc"] != o["acc"]).sum()), o["acc"].size)
-    assert np.array_equal(g["q"].astype(np.int32), o["q"]), "re-quantised activations"
+    if g["acc"] is not None:
+        assert np.array_equal(g["acc"], o["acc"]), "accumulators: %d of %d differ" % (
+            int((g["acc"] != o["acc"]).sum()), o["acc"].size)
+    if g["q"] is not None:
+        bad = int((g["q"].astype(np.int32) != o["q"]).sum())
+        assert bad == 0, "re-quantised activations: %d of %d differ" % (bad, o["q"].size)
     # fp32: 1e-6 relative (both sides use correctly rounded IEEE operations, so expect equality)
-    assert np.allclose(g["f32"], o["f32"], rtol=1e-6, atol=0.0), "fp32 outputs"
+    if g["f32"] is not None:
+        assert np.allclose(g["f32"], o["f32"], rtol=1e-6, atol=0.0), "fp32 outputs"

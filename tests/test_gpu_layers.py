@@ -39,14 +39,14 @@ def _layer_inputs(rng, N, C, H, W, O, KH, KW, groups, layout, x_dtype=np.uint8, 
 
 def _both(psb, ctx, oracle, w, x, layout, groups, stride, pad, levels, scale, bias, kmap=None,
           uniform=None, relu=True, inv_step=0.5, qmin=0, qmax=15, out_dtype=0, residual=None,
-          res_scale=0.0, exp_bits=4, norm=0, in_max=0, path=0, seed=5, layer_id=3):
+          res_scale=0.0, exp_bits=4, norm=0, in_max=0, path=0, seed=5, layer_id=3, want=("q", "f32", "acc")):
     uniform = levels[0] if uniform is None else uniform
     o = oracle_layer(oracle, w, x, layout, groups, stride, pad, seed, layer_id, levels, kmap, uniform,
                      scale, bias, relu, np.float32(inv_step), qmin, qmax, residual, np.float32(res_scale),
                      exp_bits, norm)
     g = gpu_layer(psb, ctx, w, x, layout, groups, stride, pad, seed, layer_id, levels, kmap, uniform,
                   scale, bias, relu, np.float32(inv_step), qmin, qmax, out_dtype, residual,
-                  np.float32(res_scale), exp_bits, norm, in_max, path)
+                  np.float32(res_scale), exp_bits, norm, in_max, path, want=want)
     compare(g, o, levels)
     return g
 
@@ -176,6 +176,44 @@ def test_tensor_path_few_input_channels_full_range_bytes(psb, ctx, oracle, case)
             km = rng.choice(levels, size=(case["N"], oh, ow)).astype(np.uint8)
         g = _both(psb, ctx, oracle, w, x, 1, 1, case["stride"], case["pad"], levels, scale, bias, kmap=km,
                   inv_step=0.02, qmax=255, path=psb.PSB_PATH_TENSOR)
+        assert g["path"] == psb.PSB_PATH_TENSOR
+
+
+@pytest.mark.parametrize("case", [
+    dict(N=2, C=96, H=13, W=11, stride=1, dtype=np.uint8, hi=256, res=None),
+    dict(N=3, C=144, H=15, W=15, stride=2, dtype=np.uint8, hi=256, res=None),
+    dict(N=2, C=32, H=9, W=9, stride=1, dtype=np.int8, hi=128, res=np.int8),
+    dict(N=2, C=960, H=7, W=7, stride=1, dtype=np.uint8, hi=256, res=np.uint8),
+])
+def test_depthwise_codes_only(psb, ctx, oracle, case):
+    """Depthwise 3x3 through the vectorised channels-last kernel (only re-quantised codes wanted)."""
+    rng = np.random.default_rng(case["C"] + case["stride"])
+    C = case["C"]
+    w, x, scale, bias = _layer_inputs(rng, case["N"], C, case["H"], case["W"], C, 3, 3, C, 1,
+                                      x_dtype=case["dtype"], x_hi=case["hi"])
+    oh = (case["H"] + 2 - 3) // case["stride"] + 1
+    ow = (case["W"] + 2 - 3) // case["stride"] + 1
+    res = None
+    if case["res"] is not None:
+        lo, hi = (0, 256) if case["res"] == np.uint8 else (-128, 128)
+        res = rng.integers(lo, hi, size=(case["N"], oh, ow, C)).astype(case["res"])
+    g = _both(psb, ctx, oracle, w, x, 1, C, case["stride"], 1, [4], scale, bias, inv_step=0.03, qmax=255,
+              residual=res, res_scale=0.2, want=("q",))
+    assert g["path"] == psb.PSB_PATH_SHIFT_ADD
+
+
+@pytest.mark.parametrize("case", [
+    dict(N=2, C=96, H=14, W=14, O=32, K=1, stride=1),     # projection after a ReLU6: bytes up to 255
+    dict(N=2, C=64, H=15, W=15, O=64, K=3, stride=2),     # taps but no padding
+    dict(N=64, C=1280, H=1, W=1, O=1000, K=1, stride=1),  # classifier on pooled unsigned bytes
+])
+def test_tensor_path_full_range_unsigned_bytes_without_padding(psb, ctx, oracle, case):
+    rng = np.random.default_rng(case["C"] + case["K"])
+    w, x, scale, bias = _layer_inputs(rng, case["N"], case["C"], case["H"], case["W"], case["O"], case["K"],
+                                      case["K"], 1, 1, x_hi=256)
+    for want in (("q", "f32", "acc"), ("q",)):
+        g = _both(psb, ctx, oracle, w, x, 1, 1, case["stride"], 0, [4], scale, bias, relu=False, inv_step=0.01,
+                  qmin=-128, qmax=127, out_dtype=1, path=psb.PSB_PATH_TENSOR, want=want)
         assert g["path"] == psb.PSB_PATH_TENSOR
 
 

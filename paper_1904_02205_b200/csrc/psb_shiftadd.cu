@@ -134,6 +134,68 @@ __global__ void __launch_bounds__(256) dwconv_nhwc8_kernel(const ConvArgs a, con
   }
 }
 
+// The 3x3 case of the kernel above, unrolled: all nine 8-byte loads are issued before the
+// arithmetic, positions outside the image read as zero through a predicate instead of a branch,
+// index arithmetic is 32-bit, and the per-channel output constants sit in shared memory.
+template <bool kSignedIn>
+__global__ void __launch_bounds__(256) dwconv3x3_nhwc8_kernel(const ConvArgs a, const int32_t* __restrict__ wint) {
+  extern __shared__ int32_t dw_w[];   // [9][C] filter, then [C] float2 (scale * 2^(e_base - log2k), bias)
+  const uint32_t C = a.C;
+  float2* scb = reinterpret_cast<float2*>(dw_w + 9u * C);
+  for (uint32_t i = threadIdx.x; i < 9u * C; i += blockDim.x) dw_w[(i % 9u) * C + i / 9u] = wint[i];
+  for (uint32_t o = threadIdx.x; o < C; o += blockDim.x)
+    scb[o] = make_float2(ldexpf(a.scale[o], a.e_base[o] - (int)a.uniform_log2k), a.bias[o]);
+  __syncthreads();
+  const uint32_t groups = C / 8u;
+  const uint32_t total = a.N * a.OH * a.OW * groups;   // the launcher keeps this below 2^32
+  const bool has_res = a.residual != nullptr;
+  const bool relu = a.relu != 0;
+  const uint8_t* x = (const uint8_t*)a.x;
+  for (uint32_t idx = blockIdx.x * blockDim.x + threadIdx.x; idx < total; idx += gridDim.x * blockDim.x) {
+    const uint32_t pix = idx / groups, c0 = (idx - pix * groups) * 8u;
+    const uint32_t row = pix / a.OW, ox = pix - row * a.OW;
+    const uint32_t n = row / a.OH, oy = row - n * a.OH;
+    const int iy0 = (int)(oy * a.stride) - (int)a.pad, ix0 = (int)(ox * a.stride) - (int)a.pad;
+    uint2 xv[9];
+#pragma unroll
+    for (int t = 0; t < 9; ++t) {
+      const int iy = iy0 + t / 3, ix = ix0 + t % 3;
+      const bool in = (unsigned)iy < a.H && (unsigned)ix < a.W;
+      xv[t] = make_uint2(0u, 0u);
+      if (in) xv[t] = __ldg(reinterpret_cast<const uint2*>(x + ((size_t)(n * a.H + iy) * a.W + ix) * C + c0));
+    }
+    uint2 rv = make_uint2(0u, 0u);
+    const size_t oidx = (size_t)pix * C + c0;
+    if (has_res) rv = __ldg(reinterpret_cast<const uint2*>((const uint8_t*)a.residual + oidx));
+    long long acc[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+#pragma unroll
+    for (int t = 0; t < 9; ++t) {
+      const int32_t* wr = dw_w + t * C + c0;
+      const int4 w0 = *reinterpret_cast<const int4*>(wr), w1 = *reinterpret_cast<const int4*>(wr + 4);
+      const int ws[8] = {w0.x, w0.y, w0.z, w0.w, w1.x, w1.y, w1.z, w1.w};
+      const uint32_t xw[2] = {xv[t].x, xv[t].y};
+#pragma unroll
+      for (int j = 0; j < 8; ++j) {
+        const uint32_t b = (xw[j >> 2] >> (8 * (j & 3))) & 0xFFu;
+        const int xi = kSignedIn ? (int)(int8_t)b : (int)b;
+        acc[j] += (long long)xi * (long long)ws[j];
+      }
+    }
+    const uint32_t rw[2] = {rv.x, rv.y};
+    uint32_t qw[2] = {0, 0};
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+      const float2 sb = scb[c0 + j];
+      int rb = (int)((rw[j >> 2] >> (8 * (j & 3))) & 0xFFu);
+      if (a.residual_dtype == PSB_DT_S8) rb = (int)(int8_t)rb;
+      const float y = dequant(acc[j], sb.x, sb.y, has_res, rb, a.residual_scale, relu);
+      const int q = requant(y, a.inv_step, a.qmin, a.qmax);
+      qw[j >> 2] |= ((uint32_t)q & 0xFFu) << (8 * (j & 3));
+    }
+    *reinterpret_cast<uint2*>((uint8_t*)a.q_out + oidx) = make_uint2(qw[0], qw[1]);
+  }
+}
+
 // x ^ 0x80 over a whole tensor: unsigned bytes become (x - 128) as signed bytes, 16 per thread.
 __global__ void offset128_kernel(const uint4* __restrict__ src, uint4* __restrict__ dst, size_t n16) {
   for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n16; i += (size_t)gridDim.x * blockDim.x) {
@@ -310,10 +372,25 @@ cudaError_t launch_shift_add(const ConvArgs& a, const WintTable& wt, cudaStream_
   if (a.groups == a.C && a.O == a.C && a.C % 8u == 0 && !a.kmap && a.q_out && !a.f32_out && !a.acc_out &&
       !a.out_nchw && dw_smem <= 64 * 1024 &&
       !(((uintptr_t)a.x | (uintptr_t)a.q_out | (uintptr_t)a.residual) & 7u)) {
-    static bool attr_set = false;
-    if (!attr_set) {
+    static bool attr_set[64] = {};
+    int dev = 0;
+    cudaGetDevice(&dev);
+    if (dev >= 0 && dev < 64 && !attr_set[dev]) {
       cudaFuncSetAttribute(dwconv_nhwc8_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 64 * 1024);
-      attr_set = true;
+      cudaFuncSetAttribute(dwconv3x3_nhwc8_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 64 * 1024);
+      cudaFuncSetAttribute(dwconv3x3_nhwc8_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 64 * 1024);
+      attr_set[dev] = true;
+    }
+    const size_t smem3 = dw_smem + (size_t)a.C * sizeof(float2);
+    if (a.KH == 3 && a.KW == 3 && smem3 <= 64 * 1024 && total / 8 < (1ull << 31)) {
+      // as many blocks per SM as the shared-memory copies of the filter allow, at most 8
+      uint32_t per_sm = (uint32_t)((200u * 1024u) / (smem3 + 1024u));
+      per_sm = per_sm > 8u ? 8u : (per_sm < 1u ? 1u : per_sm);
+      uint32_t blocks = grid_for(total / 8, 256);
+      if (blocks > 148u * per_sm) blocks = 148u * per_sm;
+      if (a.in_dtype == PSB_DT_S8) dwconv3x3_nhwc8_kernel<true><<<blocks, 256, smem3, s>>>(a, wt.w[a.uniform_log2k]);
+      else dwconv3x3_nhwc8_kernel<false><<<blocks, 256, smem3, s>>>(a, wt.w[a.uniform_log2k]);
+      return cudaGetLastError();
     }
     uint32_t blocks = grid_for(total / 8, 256);
     if (blocks > 148u * 4u) blocks = 148u * 4u;

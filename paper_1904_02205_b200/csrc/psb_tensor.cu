@@ -60,7 +60,7 @@ struct TensorParams {
   uint32_t group;       // K blocks per pipeline stage (one barrier hand-over per group)
   uint32_t stage_bytes_a, stage_bytes_b_max;
   uint32_t planes[kMaxLevels];
-  uint32_t vec_ok;      // 16-byte stores are legal for every output pointer
+  uint32_t vec_ok;      // output rows (and pointers) are multiples of 16 bytes (2), of 8 bytes (1), or neither
   uint32_t resident;    // 1: the CTA keeps the digit planes of its channel tile in shared memory
   uint32_t ctas_per_otile;
   uint32_t resident_bytes;
@@ -318,15 +318,33 @@ __device__ __forceinline__ uint4 chunk_math(const uint32_t (&v)[P][16], const ui
   return make_uint4(qw[0], qw[1], qw[2], qw[3]);
 }
 
+// 16 bytes of a channels-last row.  Rows that are only 8-byte aligned (channel counts that are odd
+// multiples of 8) move as two halves; `both` is false for the last 8 channels of such a row.
+__device__ __forceinline__ uint4 load_row16(const uint8_t* src, bool vec16, bool both) {
+  if (vec16) return __ldg(reinterpret_cast<const uint4*>(src));
+  const uint2 lo = __ldg(reinterpret_cast<const uint2*>(src));
+  uint2 hi = make_uint2(0u, 0u);
+  if (both) hi = __ldg(reinterpret_cast<const uint2*>(src + 8));
+  return make_uint4(lo.x, lo.y, hi.x, hi.y);
+}
+__device__ __forceinline__ void store_row16(uint8_t* dst, uint4 v, bool vec16, bool both) {
+  if (vec16) {
+    *reinterpret_cast<uint4*>(dst) = v;
+  } else {
+    *reinterpret_cast<uint2*>(dst) = make_uint2(v.x, v.y);
+    if (both) *reinterpret_cast<uint2*>(dst + 8) = make_uint2(v.z, v.w);
+  }
+}
+
 template <int P, int MODE, bool HAS_RES>
-__device__ __noinline__ void epilogue_chunk_q(uint32_t taddr, bool valid, uint8_t* q_dst, uint4 r4,
-                                              const float2* scb, const long long* corr, EpiConst c) {
+__device__ __noinline__ void epilogue_chunk_q(uint32_t taddr, bool valid, uint8_t* q_dst, uint4 r4, bool vec16,
+                                              bool both, const float2* scb, const long long* corr, EpiConst c) {
   uint32_t v[P][16];
 #pragma unroll
   for (int pl = 0; pl < P; ++pl) tc_ld16(taddr + pl * kTileN, v[pl]);
   tc_wait_ld();
   if (!valid) return;
-  *reinterpret_cast<uint4*>(q_dst) = chunk_math<P, MODE, HAS_RES>(v, r4, scb, corr, c);
+  store_row16(q_dst, chunk_math<P, MODE, HAS_RES>(v, r4, scb, corr, c), vec16, both);
 }
 
 // General output stage: any combination of outputs, layouts, ragged channel counts.
@@ -341,7 +359,7 @@ __device__ __noinline__ void epilogue_chunk(const TensorParams& p, uint32_t tadd
   if (!valid) return;
   const ConvArgs& a = p.a;
   const uint32_t ohow = a.OH * a.OW;
-  const bool vec = p.vec_ok && o_base + 16u <= a.O && !a.out_nchw;
+  const bool vec = p.vec_ok == 2u && o_base + 16u <= a.O && !a.out_nchw;
   uint32_t rw[4] = {0, 0, 0, 0};
   if (vec && a.residual) {
     uint4 r4 = *reinterpret_cast<const uint4*>((const uint8_t*)a.residual + (size_t)m * a.O + o_base);
@@ -396,13 +414,14 @@ __device__ __noinline__ bool epilogue_uniform(const TensorParams& p, SharedCtl* 
   const uint8_t* res_base = (const uint8_t*)a.residual;
   const float2* scb = ctl->scb[ew];
   const long long* corr = ctl->corr[ew];
+  const bool vec16 = p.vec_ok == 2u;
   TileIter ti;
   ti.init(p);
   uint32_t pass = 0, cur_o_tile = 0xFFFFFFFFu;
   uint4 r_next = make_uint4(0, 0, 0, 0);
   if (HAS_RES && ti.valid()) {
     const uint32_t m = ti.m_tile * kTileM + row, ob = ti.o_tile * kTileN + sub * 16u;
-    if (m < p.M && ob < a.O) r_next = __ldg(reinterpret_cast<const uint4*>(res_base + (size_t)m * a.O + ob));
+    if (m < p.M && ob < a.O) r_next = load_row16(res_base + (size_t)m * a.O + ob, vec16, ob + 16u <= a.O);
   }
   while (ti.valid()) {
     const uint32_t m = ti.m_tile * kTileM + row;
@@ -432,7 +451,7 @@ __device__ __noinline__ bool epilogue_uniform(const TensorParams& p, SharedCtl* 
     if (HAS_RES && ti.valid()) {
       const uint32_t mn = ti.m_tile * kTileM + row, ob = ti.o_tile * kTileN + sub * 16u;
       r_next = make_uint4(0, 0, 0, 0);
-      if (mn < p.M && ob < a.O) r_next = __ldg(reinterpret_cast<const uint4*>(res_base + (size_t)mn * a.O + ob));
+      if (mn < p.M && ob < a.O) r_next = load_row16(res_base + (size_t)mn * a.O + ob, vec16, ob + 16u <= a.O);
     }
     const uint32_t buf = pass & 1u, aph = (pass >> 1) & 1u;
     const bool ok = mbar_wait(smem_u32(&ctl->acc_full[buf]), aph, abort, 32);
@@ -450,8 +469,8 @@ __device__ __noinline__ bool epilogue_uniform(const TensorParams& p, SharedCtl* 
     __syncwarp();
     if (lane == 0) mbar_arrive(smem_u32(&ctl->acc_empty[buf]));
     if (active && m < p.M)
-      *reinterpret_cast<uint4*>((uint8_t*)a.q_out + (size_t)m * a.O + o_base) =
-          chunk_math<P, MODE, HAS_RES>(v, r_cur, scb, corr, c);
+      store_row16((uint8_t*)a.q_out + (size_t)m * a.O + o_base, chunk_math<P, MODE, HAS_RES>(v, r_cur, scb, corr, c),
+                  vec16, o_base + 16u <= a.O);
     ++pass;
   }
   return false;
@@ -643,7 +662,7 @@ psb_mma_kernel(const __grid_constant__ TmapSet maps, const __grid_constant__ Ten
     ec.qmax_f = (float)a.qmax;
     ec.res_sign = a.residual_dtype == PSB_DT_S8 ? 0x80u : 0u;
     const uint32_t P0 = p.planes[a.uniform_log2k < (uint32_t)kMaxLevels ? a.uniform_log2k : 0u];
-    if (!a.kmap && q_only && a.O % 16u == 0u && (P0 == 3u || P0 == 4u)) {
+    if (!a.kmap && q_only && (P0 == 3u || P0 == 4u)) {
       const uint32_t mode = (p.corr[a.uniform_log2k] != nullptr || P0 == 4u) ? 0u : p.narrow;
 #define PSB_UNI(PV, MV, RV) failed = epilogue_uniform<PV, MV, RV>(p, ctl, tmem_base, ew, lane, ec)
       if (a.residual) {
@@ -670,10 +689,10 @@ psb_mma_kernel(const __grid_constant__ TmapSet maps, const __grid_constant__ Ten
           atomicOr(a.err, kDevErrBadLevel);
         const uint32_t o_base = o_tile * kTileN + sub * 16u;
         const size_t oidx = (size_t)m * a.O + o_base;
-        const bool fast = q_only && o_base + 16u <= a.O;
+        const bool vec16 = p.vec_ok == 2u, both = o_base + 16u <= a.O;
+        const bool fast = q_only && o_base < a.O;
         uint4 r4 = make_uint4(0, 0, 0, 0);
-        if (fast && a.residual && in_range)
-          r4 = __ldg(reinterpret_cast<const uint4*>((const uint8_t*)a.residual + oidx));
+        if (fast && a.residual && in_range) r4 = load_row16((const uint8_t*)a.residual + oidx, vec16, both);
         for (uint32_t todo = levels & 0x7Fu; todo && !failed; todo &= todo - 1u) {
           const uint32_t l = (uint32_t)__ffs((int)todo) - 1u;
           const uint32_t P = p.planes[l];
@@ -708,7 +727,7 @@ psb_mma_kernel(const __grid_constant__ TmapSet maps, const __grid_constant__ Ten
             if (fast) {
               uint8_t* q_dst = (uint8_t*)a.q_out + oidx;
               const uint32_t mode = (use_corr || P > 3u) ? 0u : p.narrow;
-#define PSB_EPI(PV, MV, RV) epilogue_chunk_q<PV, MV, RV>(taddr, valid, q_dst, r4, scb, corr, ec)
+#define PSB_EPI(PV, MV, RV) epilogue_chunk_q<PV, MV, RV>(taddr, valid, q_dst, r4, vec16, both, scb, corr, ec)
 #define PSB_EPI_P(MV, RV) do { if (P == 3) PSB_EPI(3, MV, RV); else if (P == 2) PSB_EPI(2, MV, RV); else PSB_EPI(1, MV, RV); } while (0)
               if (a.residual) {
                 if (mode == 2) PSB_EPI_P(2, true); else if (mode == 1) PSB_EPI_P(1, true);
@@ -855,10 +874,10 @@ psb_status launch_tensor(psb_ctx* ctx, const psb_weights* wt, const ConvArgs& a,
   // every plane sum is bounded by 127 * (largest activation magnitude) * d
   const uint64_t plane_bound = 127ull * amax * (uint64_t)wt->d;
   p.narrow = pmax > 3 ? 0u : (plane_bound <= 4100000ull ? 2u : (plane_bound <= 16500000ull ? 1u : 0u));
-  bool vec = !a.out_nchw && a.O % 16u == 0;
-  vec = vec && !(((uintptr_t)a.q_out | (uintptr_t)a.residual | (uintptr_t)a.f32_out |
-                  (uintptr_t)a.acc_out) & 15u);
-  p.vec_ok = vec ? 1u : 0u;
+  const uintptr_t out_ptrs = (uintptr_t)a.q_out | (uintptr_t)a.residual | (uintptr_t)a.f32_out | (uintptr_t)a.acc_out;
+  p.vec_ok = 0u;
+  if (!a.out_nchw && a.O % 16u == 0u && !(out_ptrs & 15u)) p.vec_ok = 2u;
+  else if (!a.out_nchw && a.O % 8u == 0u && !(out_ptrs & 7u)) p.vec_ok = 1u;
 
   const CUtensorMapSwizzle swz = swizzle_for(bk);
   EncodeTiledFn enc_tiled = (EncodeTiledFn)ctx->encode_tiled;

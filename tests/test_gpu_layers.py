@@ -217,6 +217,27 @@ def test_tensor_path_full_range_unsigned_bytes_without_padding(psb, ctx, oracle,
         assert g["path"] == psb.PSB_PATH_TENSOR
 
 
+@pytest.mark.parametrize("O,with_res,with_map", [(24, False, False), (24, True, False), (40, True, True), (72, False, True)])
+def test_tensor_path_rows_of_odd_multiples_of_eight_channels(psb, ctx, oracle, O, with_res, with_map):
+    """Output rows that are 8- but not 16-byte aligned keep the vector store path (codes only)."""
+    rng = np.random.default_rng(O)
+    N, C, H, W = 3, 96, 13, 12
+    w, x, scale, bias = _layer_inputs(rng, N, C, H, W, O, 1, 1, 1, 1, x_hi=128)
+    res = rng.integers(0, 256, size=(N, H, W, O)).astype(np.uint8) if with_res else None
+    kmap = rng.integers(0, 5, size=(N, H, W)).astype(np.uint8) if with_map else None
+    levels = [0, 1, 2, 3, 4] if with_map else [3]
+    g = _both(psb, ctx, oracle, w, x, 1, 1, 1, 0, levels, scale, bias, kmap=kmap, inv_step=0.02, qmax=255,
+              residual=res, res_scale=0.1, in_max=127, path=psb.PSB_PATH_TENSOR, want=("q",))
+    assert g["path"] == psb.PSB_PATH_TENSOR
+
+
+def test_depthwise_5x5_codes_only(psb, ctx, oracle):
+    rng = np.random.default_rng(55)
+    C = 48
+    w, x, scale, bias = _layer_inputs(rng, 2, C, 12, 10, C, 5, 5, C, 1, x_hi=256)
+    _both(psb, ctx, oracle, w, x, 1, C, 1, 2, [3], scale, bias, inv_step=0.03, qmax=255, want=("q",))
+
+
 def test_fully_connected_on_the_tensor_path(psb, ctx, oracle):
     rng = np.random.default_rng(5)
     w, x, scale, bias = _layer_inputs(rng, 64, 512, 1, 1, 1000, 1, 1, 1, 1)

@@ -126,6 +126,26 @@ __device__ __forceinline__ int requant(float y, float inv_step, int qmin, int qm
   return (int)r;
 }
 
+// Exact round-to-nearest conversion of a 64-bit accumulator, |acc| < 2^55: split into a high
+// part (multiple of 2^24) and a 24-bit low part, both exact in fp32; one fma rounds their sum once.
+__device__ __forceinline__ float acc_to_float(long long acc) {
+  const int hi = (int)(acc >> 24);
+  const int lo = (int)((unsigned int)acc & 0xFFFFFFu);
+  return __fmaf_rn((float)hi, 16777216.0f, (float)lo);
+}
+
+// The same for |acc| < 2^45, without the conversion unit: the parts get their float form by
+// exponent arithmetic,
+//   float(n) = as_float(0x4B400000 + n) - 1.5 * 2^23   for |n| < 2^22,
+//   float(n) = as_float(0x4B000000 | n) - 2^23         for 0 <= n < 2^23.
+__device__ __forceinline__ float acc_to_float_small(long long acc) {
+  const int hi = (int)(acc >> 23);
+  const unsigned int lo = (unsigned int)acc & 0x7FFFFFu;
+  const float hi_f = __int_as_float(0x4B400000 + hi) - 12582912.0f;
+  const float lo_f = __uint_as_float(0x4B000000u | lo) - 8388608.0f;
+  return __fmaf_rn(hi_f, 8388608.0f, lo_f);
+}
+
 // host-side launchers (defined in the .cu files)
 cudaError_t launch_sampler(const float* w_dev, psb_weights* wt, uint32_t* err_dev, cudaStream_t s);
 psb_status sample_batch_create(psb_ctx* ctx, uint32_t n, const float* const* w_dev,

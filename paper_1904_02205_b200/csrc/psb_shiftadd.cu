@@ -134,65 +134,107 @@ __global__ void __launch_bounds__(256) dwconv_nhwc8_kernel(const ConvArgs a, con
   }
 }
 
-// The 3x3 case of the kernel above, unrolled: all nine 8-byte loads are issued before the
-// arithmetic, positions outside the image read as zero through a predicate instead of a branch,
-// index arithmetic is 32-bit, and the per-channel output constants sit in shared memory.
-template <bool kSignedIn>
-__global__ void __launch_bounds__(256) dwconv3x3_nhwc8_kernel(const ConvArgs a, const int32_t* __restrict__ wint) {
-  extern __shared__ int32_t dw_w[];   // [9][C] filter, then [C] float2 (scale * 2^(e_base - log2k), bias)
-  const uint32_t C = a.C;
-  float2* scb = reinterpret_cast<float2*>(dw_w + 9u * C);
-  for (uint32_t i = threadIdx.x; i < 9u * C; i += blockDim.x) dw_w[(i % 9u) * C + i / 9u] = wint[i];
-  for (uint32_t o = threadIdx.x; o < C; o += blockDim.x)
-    scb[o] = make_float2(ldexpf(a.scale[o], a.e_base[o] - (int)a.uniform_log2k), a.bias[o]);
-  __syncthreads();
-  const uint32_t groups = C / 8u;
-  const uint32_t total = a.N * a.OH * a.OW * groups;   // the launcher keeps this below 2^32
-  const bool has_res = a.residual != nullptr;
-  const bool relu = a.relu != 0;
-  const uint8_t* x = (const uint8_t*)a.x;
-  for (uint32_t idx = blockIdx.x * blockDim.x + threadIdx.x; idx < total; idx += gridDim.x * blockDim.x) {
-    const uint32_t pix = idx / groups, c0 = (idx - pix * groups) * 8u;
-    const uint32_t row = pix / a.OW, ox = pix - row * a.OW;
-    const uint32_t n = row / a.OH, oy = row - n * a.OH;
-    const int iy0 = (int)(oy * a.stride) - (int)a.pad, ix0 = (int)(ox * a.stride) - (int)a.pad;
-    uint2 xv[9];
+// Depthwise 3x3, channels-last, one draw count, only codes wanted.  A thread owns 4 channels
+// and kDwSeg consecutive output columns of one output row: its 36 filter values and 8 output
+// constants stay in registers, every input column of the 3-row band is loaded once (one 32-bit
+// load per row) and serves up to three outputs.  All loads of the band are issued before the
+// arithmetic; positions outside the image read as zero through a predicate.  The output stage
+// is dequant()/requant() written without the conversion unit (exponent arithmetic, see
+// acc_to_float_small).  Adjacent threads take adjacent channel quads, so a warp's loads and
+// stores are contiguous runs of the channels-last rows.
+template <int S>
+struct DwSeg { static constexpr int kOut = S == 1 ? 8 : 4; static constexpr int kCols = (kOut - 1) * S + 3; };
+
+template <int S, bool kSignedIn>
+__global__ void __launch_bounds__(256, 2) dwconv3x3_row_kernel(const ConvArgs a, const int32_t* __restrict__ wint) {
+  constexpr int L = DwSeg<S>::kOut, NC = DwSeg<S>::kCols;
+  const uint32_t C = a.C, G = C / 4u;
+  const uint32_t segs = (a.OW + L - 1) / L;
+  const uint32_t total = a.N * a.OH * segs * G;   // the launcher keeps this below 2^32
+  const uint32_t idx = blockIdx.x * blockDim.x + threadIdx.x;
+  if (idx >= total) return;
+  uint32_t t = idx / G;
+  const uint32_t c0 = (idx - t * G) * 4u;
+  const uint32_t seg = t % segs; t /= segs;
+  const uint32_t oy = t % a.OH, n = t / a.OH;
+  const uint32_t ox0 = seg * L;
+
+  // band of input: rows iy0..iy0+2, columns ix0..ix0+NC-1
+  const int iy0 = (int)(oy * S) - (int)a.pad, ix0 = (int)(ox0 * S) - (int)a.pad;
+  const uint32_t last_ox = min(ox0 + (uint32_t)L, a.OW) - 1u;
+  const int ix_end = (int)(last_ox * S) - (int)a.pad + 2;     // last column any output of the segment reads
+  uint32_t raw[3][NC];
 #pragma unroll
-    for (int t = 0; t < 9; ++t) {
-      const int iy = iy0 + t / 3, ix = ix0 + t % 3;
-      const bool in = (unsigned)iy < a.H && (unsigned)ix < a.W;
-      xv[t] = make_uint2(0u, 0u);
-      if (in) xv[t] = __ldg(reinterpret_cast<const uint2*>(x + ((size_t)(n * a.H + iy) * a.W + ix) * C + c0));
+  for (int r = 0; r < 3; ++r) {
+    const int iy = iy0 + r;
+    const bool row_in = (unsigned)iy < a.H;
+    const uint8_t* rp = (const uint8_t*)a.x + ((size_t)(n * a.H + (row_in ? iy : 0)) * a.W) * C + c0;
+#pragma unroll
+    for (int cidx = 0; cidx < NC; ++cidx) {
+      const int ix = ix0 + cidx;
+      raw[r][cidx] = 0u;
+      if (row_in && (unsigned)ix < a.W && ix <= ix_end)
+        raw[r][cidx] = __ldg(reinterpret_cast<const uint32_t*>(rp + (size_t)ix * C));
     }
-    uint2 rv = make_uint2(0u, 0u);
-    const size_t oidx = (size_t)pix * C + c0;
-    if (has_res) rv = __ldg(reinterpret_cast<const uint2*>((const uint8_t*)a.residual + oidx));
-    long long acc[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+  }
+  // filter [channel][tap] and output constants of the 4 channels
+  int w[36];
+  {
+    const int4* wp = reinterpret_cast<const int4*>(wint + (size_t)c0 * 9u);
 #pragma unroll
-    for (int t = 0; t < 9; ++t) {
-      const int32_t* wr = dw_w + t * C + c0;
-      const int4 w0 = *reinterpret_cast<const int4*>(wr), w1 = *reinterpret_cast<const int4*>(wr + 4);
-      const int ws[8] = {w0.x, w0.y, w0.z, w0.w, w1.x, w1.y, w1.z, w1.w};
-      const uint32_t xw[2] = {xv[t].x, xv[t].y};
+    for (int i = 0; i < 9; ++i) {
+      const int4 v = __ldg(wp + i);
+      w[4 * i] = v.x; w[4 * i + 1] = v.y; w[4 * i + 2] = v.z; w[4 * i + 3] = v.w;
+    }
+  }
+  float sc[4], bi[4];
 #pragma unroll
-      for (int j = 0; j < 8; ++j) {
-        const uint32_t b = (xw[j >> 2] >> (8 * (j & 3))) & 0xFFu;
-        const int xi = kSignedIn ? (int)(int8_t)b : (int)b;
-        acc[j] += (long long)xi * (long long)ws[j];
+  for (int j = 0; j < 4; ++j) {
+    sc[j] = ldexpf(a.scale[c0 + j], a.e_base[c0 + j] - (int)a.uniform_log2k);
+    bi[j] = a.bias[c0 + j];
+  }
+  const bool has_res = a.residual != nullptr;
+  const uint32_t res_sign = a.residual_dtype == PSB_DT_S8 ? 0x80u : 0u;
+  const float res_bias = 8388608.0f + (float)res_sign;
+  const float relu_floor = (a.relu && a.qmin < 0) ? 0.0f : __int_as_float(0xFF800000);
+  const float qmin_f = (float)a.qmin, qmax_f = (float)a.qmax;
+  const size_t obase = ((size_t)(n * a.OH + oy) * a.OW + ox0) * C + c0;
+
+#pragma unroll
+  for (int i = 0; i < L; ++i) {
+    if (ox0 + i > last_ox) break;
+    const size_t oidx = obase + (size_t)i * C;
+    uint32_t rv = 0u;
+    if (has_res) rv = __ldg(reinterpret_cast<const uint32_t*>((const uint8_t*)a.residual + oidx));
+    long long acc[4] = {0, 0, 0, 0};
+#pragma unroll
+    for (int r = 0; r < 3; ++r) {
+#pragma unroll
+      for (int kw = 0; kw < 3; ++kw) {
+        const uint32_t v = raw[r][i * S + kw];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          const uint32_t b = (v >> (8 * j)) & 0xFFu;
+          const int xi = kSignedIn ? (int)(int8_t)b : (int)b;
+          acc[j] += (long long)xi * (long long)w[j * 9 + r * 3 + kw];
+        }
       }
     }
-    const uint32_t rw[2] = {rv.x, rv.y};
-    uint32_t qw[2] = {0, 0};
+    uint32_t q[4];
 #pragma unroll
-    for (int j = 0; j < 8; ++j) {
-      const float2 sb = scb[c0 + j];
-      int rb = (int)((rw[j >> 2] >> (8 * (j & 3))) & 0xFFu);
-      if (a.residual_dtype == PSB_DT_S8) rb = (int)(int8_t)rb;
-      const float y = dequant(acc[j], sb.x, sb.y, has_res, rb, a.residual_scale, relu);
-      const int q = requant(y, a.inv_step, a.qmin, a.qmax);
-      qw[j >> 2] |= ((uint32_t)q & 0xFFu) << (8 * (j & 3));
+    for (int j = 0; j < 4; ++j) {
+      float y = __fmaf_rn(acc_to_float_small(acc[j]), sc[j], bi[j]);
+      if (has_res) {
+        const uint32_t rb = ((rv >> (8 * j)) & 0xFFu) ^ res_sign;   // byte + 128 if signed
+        y = __fmaf_rn(__uint_as_float(0x4B000000u | rb) - res_bias, a.residual_scale, y);
+      }
+      y = fmaxf(y, relu_floor);
+      // clamp, then round half to even by adding 1.5 * 2^23: the low byte of the sum is the code
+      const float tq = fminf(fmaxf(__fmul_rn(y, a.inv_step), qmin_f), qmax_f);
+      q[j] = __float_as_uint(tq + 12582912.0f);
     }
-    *reinterpret_cast<uint2*>((uint8_t*)a.q_out + oidx) = make_uint2(qw[0], qw[1]);
+    *reinterpret_cast<uint32_t*>((uint8_t*)a.q_out + oidx) =
+        __byte_perm(__byte_perm(q[0], q[1], 0x0040), __byte_perm(q[2], q[3], 0x0040), 0x5410);
   }
 }
 
@@ -377,20 +419,24 @@ cudaError_t launch_shift_add(const ConvArgs& a, const WintTable& wt, cudaStream_
     cudaGetDevice(&dev);
     if (dev >= 0 && dev < 64 && !attr_set[dev]) {
       cudaFuncSetAttribute(dwconv_nhwc8_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 64 * 1024);
-      cudaFuncSetAttribute(dwconv3x3_nhwc8_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 64 * 1024);
-      cudaFuncSetAttribute(dwconv3x3_nhwc8_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 64 * 1024);
       attr_set[dev] = true;
     }
-    const size_t smem3 = dw_smem + (size_t)a.C * sizeof(float2);
-    if (a.KH == 3 && a.KW == 3 && smem3 <= 64 * 1024 && total / 8 < (1ull << 31)) {
-      // as many blocks per SM as the shared-memory copies of the filter allow, at most 8
-      uint32_t per_sm = (uint32_t)((200u * 1024u) / (smem3 + 1024u));
-      per_sm = per_sm > 8u ? 8u : (per_sm < 1u ? 1u : per_sm);
-      uint32_t blocks = grid_for(total / 8, 256);
-      if (blocks > 148u * per_sm) blocks = 148u * per_sm;
-      if (a.in_dtype == PSB_DT_S8) dwconv3x3_nhwc8_kernel<true><<<blocks, 256, smem3, s>>>(a, wt.w[a.uniform_log2k]);
-      else dwconv3x3_nhwc8_kernel<false><<<blocks, 256, smem3, s>>>(a, wt.w[a.uniform_log2k]);
-      return cudaGetLastError();
+    if (a.KH == 3 && a.KW == 3 && (a.stride == 1 || a.stride == 2)) {
+      const uint32_t seg_out = a.stride == 1 ? DwSeg<1>::kOut : DwSeg<2>::kOut;
+      const uint64_t threads = (uint64_t)a.N * a.OH * ((a.OW + seg_out - 1) / seg_out) * (a.C / 4u);
+      if (threads < (1ull << 32) - 256u) {
+        const uint32_t blocks = (uint32_t)((threads + 255u) / 256u);
+        const int32_t* wl = wt.w[a.uniform_log2k];
+        const bool sg = a.in_dtype == PSB_DT_S8;
+        if (a.stride == 1) {
+          if (sg) dwconv3x3_row_kernel<1, true><<<blocks, 256, 0, s>>>(a, wl);
+          else dwconv3x3_row_kernel<1, false><<<blocks, 256, 0, s>>>(a, wl);
+        } else {
+          if (sg) dwconv3x3_row_kernel<2, true><<<blocks, 256, 0, s>>>(a, wl);
+          else dwconv3x3_row_kernel<2, false><<<blocks, 256, 0, s>>>(a, wl);
+        }
+        return cudaGetLastError();
+      }
     }
     uint32_t blocks = grid_for(total / 8, 256);
     if (blocks > 148u * 4u) blocks = 148u * 4u;

@@ -249,14 +249,6 @@ struct SharedCtl {
   long long corr[kEpilogueWarps][16];   // per epilogue warp: integer addend per channel
 };
 
-// Exact round-to-nearest conversion of a 64-bit accumulator, |acc| < 2^47: split into a high
-// part (multiple of 2^24) and a 24-bit low part, both exact in fp32; one fma rounds their sum once.
-__device__ __forceinline__ float acc_to_float(long long acc) {
-  const int hi = (int)(acc >> 24);
-  const int lo = (int)((unsigned int)acc & 0xFFFFFFu);
-  return __fmaf_rn((float)hi, 16777216.0f, (float)lo);
-}
-
 // Output arithmetic of one 16-channel chunk held in registers (v[plane][channel]), common case:
 // only re-quantised bytes are wanted.  Same arithmetic as dequant()/requant(), arranged for the
 // main pipes: integer <-> float conversions run on a slow pipe (a quarter of the FMA rate), so

@@ -104,8 +104,6 @@ class ConvWorkload:
         self.cfg = config2_conv(seed=1 + 100 * rank)
         self.macs = self.cfg["macs"]
         self.images = self.cfg["x"].shape[0]
-        # transpose, window reduction, sampler, contraction
-        self.launches_per_step = 4
         self.planes = None
 
     def setup(self, ctx, psb, torch):
@@ -213,9 +211,6 @@ class NetWorkload:
         self.image_dev = self.image_host.to(ctx.device)
         self.logits_host = torch.empty((self.batch, self.layers[-1]["cout"]), dtype=torch.float32).pin_memory()
         self.nw.forward(self.image_dev)
-        n_conv = sum(1 for l in self.layers if l["op"] == "conv")
-        # per conv layer: window reduction + sampler + contraction; plus the pooling kernels
-        self.launches_per_step = 3 * n_conv + (len(self.layers) - n_conv)
         self.e2e_h2d = self.image_host.numel()
         self.e2e_d2h = self.logits_host.numel() * 4
         self.layer_ms = None
@@ -382,8 +377,10 @@ def main():
     torch.cuda.synchronize()
     clocks = ClockSampler(local_rank)
     clocks.start()
+    launches0 = ctx.launch_count()
     step_ms = timed(wl.step, args.steps, first=args.warmup)
     torch.cuda.synchronize()
+    launches = ctx.launch_count() - launches0      # kernels of the library inside the timed steps
     if world > 1:
         dist.barrier()
     kern_ms = timed(lambda i: wl.kernel_only(), max(args.steps, 10) if args.workload == "conv3x3" else 4)
@@ -409,7 +406,7 @@ def main():
                             images_per_step=wl.images * world, sampler="inside the timed step, fresh seed per step"),
                 images_per_s=wl.images * world * args.steps / sec,
                 gated_add_equiv_per_s=units * getattr(wl, "mean_k", args.k) / sec,
-                clocks=clk, gpu_launches=wl.launches_per_step * args.steps,
+                clocks=clk, gpu_launches=launches * world,
                 e2e=dict(value=e2e_units / e2e_sec / 1e9, unit=UNIT, h2d_bytes_per_step=wl.e2e_h2d,
                          d2h_bytes_per_step=wl.e2e_d2h),
                 roofline=wl.roofline(statistics.mean(kern_ms), peaks))

@@ -205,6 +205,11 @@ psb_status psb_gemm(psb_ctx* ctx, const psb_weights* weights, const void* x_dev,
  * (PSB_PATH_SHIFT_ADD or PSB_PATH_TENSOR); 0 before any call. */
 int32_t psb_last_path(const psb_ctx* ctx);
 
+/* Number of GPU kernels this library has launched in this process so far (all
+ * contexts, all entry points).  A reporting aid: throughput figures state how
+ * many launches a timed region took.  Never fails. */
+uint64_t psb_launch_count(void);
+
 /* Glue between layers (supplement, "ReLU, Batch-Norm, and Pooling"): max-pooling
  * is comparators only; the 1/(h*w) of average pooling is folded into one
  * re-quantisation factor.

@@ -23,7 +23,8 @@ PSB_PATH_AUTO, PSB_PATH_SHIFT_ADD, PSB_PATH_TENSOR = 0, 1, 2
 EXPORTS = ["psb_create", "psb_destroy", "psb_status_string", "psb_device_status", "psb_sample_weights",
            "psb_weights_export", "psb_weights_free", "psb_set_sample_map", "psb_conv2d", "psb_gemm",
            "psb_last_path", "psb_maxpool2d_u8", "psb_global_avgpool_u8", "psb_sample_level_static",
-           "psb_sample_batch_create", "psb_sample_batch_run", "psb_sample_batch_free", "psb_run"]
+           "psb_sample_batch_create", "psb_sample_batch_run", "psb_sample_batch_free", "psb_run",
+           "psb_launch_count"]
 
 
 class psb_wshape(C.Structure):
@@ -89,6 +90,8 @@ def load_library():
     lib.psb_conv2d.argtypes = [vp, vp, vp, C.POINTER(psb_conv_desc), vp]
     lib.psb_gemm.argtypes = [vp, vp, vp, C.POINTER(psb_gemm_desc), vp]
     lib.psb_last_path.argtypes = [vp]
+    lib.psb_launch_count.argtypes = []
+    lib.psb_launch_count.restype = C.c_uint64
     lib.psb_maxpool2d_u8.argtypes = [vp, vp, u32, u32, u32, u32, u32, u32, u32, u32, vp, vp]
     lib.psb_global_avgpool_u8.argtypes = [vp, vp, u32, u32, u32, u32, u32, C.c_float, i32, i32, vp, vp]
     lib.psb_sample_level_static.argtypes = [vp, C.POINTER(psb_wshape), C.POINTER(psb_sample_cfg), u32, vp, vp, vp]
@@ -97,7 +100,7 @@ def load_library():
     lib.psb_sample_batch_free.argtypes = [vp, vp]
     lib.psb_run.argtypes = [vp, C.POINTER(psb_op), u32, vp]
     for name in EXPORTS:
-        if name != "psb_status_string":
+        if name not in ("psb_status_string", "psb_launch_count"):
             getattr(lib, name).restype = i32
     _lib = lib
     return lib
@@ -196,6 +199,10 @@ class Context:
 
     def last_path(self):
         return self.lib.psb_last_path(self.handle)
+
+    def launch_count(self):
+        """Kernels launched by the library in this process so far."""
+        return int(self.lib.psb_launch_count())
 
     # -- psb_sample_weights --------------------------------------------------
     def sample_weights(self, w, groups=1, seed=0, layer_id=0, level_mask=1, exp_bits=4, norm=0,

@@ -5,6 +5,8 @@
 
 #include "psb_common.cuh"
 
+#include <atomic>
+
 using namespace psb;
 
 namespace {
@@ -172,6 +174,12 @@ psb_status run_layer(psb_ctx* ctx, const psb_weights* wt, const void* x_dev, uin
 }
 
 }  // namespace
+
+namespace psb {
+static std::atomic<unsigned long long> g_launches{0};
+void note_launch() { g_launches.fetch_add(1, std::memory_order_relaxed); }
+unsigned long long launches_so_far() { return g_launches.load(std::memory_order_relaxed); }
+}  // namespace psb
 
 extern "C" {
 
@@ -367,6 +375,8 @@ psb_status psb_gemm(psb_ctx* ctx, const psb_weights* weights, const void* x_dev,
 }
 
 int32_t psb_last_path(const psb_ctx* ctx) { return ctx ? ctx->last_path : 0; }
+
+uint64_t psb_launch_count(void) { return (uint64_t)psb::launches_so_far(); }
 
 psb_status psb_sample_batch_create(psb_ctx* ctx, uint32_t n, const float* const* w_dev,
                                    psb_weights* const* weights, psb_sample_batch** batch) {

@@ -146,6 +146,10 @@ __device__ __forceinline__ float acc_to_float_small(long long acc) {
   return __fmaf_rn(hi_f, 8388608.0f, lo_f);
 }
 
+// every kernel launch of the library is counted (process-wide), for throughput reports
+void note_launch();
+unsigned long long launches_so_far();
+
 // host-side launchers (defined in the .cu files)
 cudaError_t launch_sampler(const float* w_dev, psb_weights* wt, uint32_t* err_dev, cudaStream_t s);
 psb_status sample_batch_create(psb_ctx* ctx, uint32_t n, const float* const* w_dev,

@@ -281,7 +281,7 @@ uint32_t fill_sample_params(const float* w_dev, const psb_weights* wt, uint32_t*
 cudaError_t launch_corr128(const psb_weights* wt, uint32_t level, cudaStream_t s) {
   const uint32_t O = wt->shape.out_ch;
   corr128_kernel<<<(O * 32 + kThreads - 1) / kThreads, kThreads, 0, s>>>(wt->level[level].wint, O, wt->d,
-                                                                        wt->level[level].corr128);
+                                                                        wt->level[level].corr128); note_launch();
   return cudaGetLastError();
 }
 
@@ -290,10 +290,10 @@ cudaError_t launch_sampler(const float* w_dev, psb_weights* wt, uint32_t* err_de
   cudaError_t e = cudaMemsetAsync(wt->e_max, 0, sizeof(uint32_t) * O, s);
   if (e != cudaSuccess) return e;
   emax_kernel<<<emax_blocks_for(O, wt->d, wt->cfg.norm), kThreads, 0, s>>>(w_dev, O, wt->d, wt->cfg.norm,
-                                                                          wt->e_max, err_dev);
+                                                                          wt->e_max, err_dev); note_launch();
   SampleParams p;
   const uint32_t blocks = fill_sample_params(w_dev, wt, wt->e_max, p);
-  sample_kernel<<<blocks, kThreads, 0, s>>>(p);
+  sample_kernel<<<blocks, kThreads, 0, s>>>(p); note_launch();
   return cudaGetLastError();
 }
 
@@ -362,9 +362,9 @@ psb_status sample_batch_create(psb_ctx* ctx, uint32_t n, const float* const* w_d
 psb_status sample_batch_run(psb_ctx* ctx, psb_sample_batch* b, uint64_t seed, cudaStream_t s) {
   if (cudaMemsetAsync(b->e_max_pool, 0, sizeof(uint32_t) * b->e_max_words, s) != cudaSuccess)
     return PSB_ERR_CUDA;
-  emax_batch_kernel<<<b->emax_grid, kThreads, 0, s>>>(b->entries_dev, b->n, ctx->err_dev);
+  emax_batch_kernel<<<b->emax_grid, kThreads, 0, s>>>(b->entries_dev, b->n, ctx->err_dev); note_launch();
   sample_batch_kernel<<<b->sample_grid, kThreads, 0, s>>>(b->entries_dev, b->n, (uint32_t)seed,
-                                                         (uint32_t)(seed >> 32));
+                                                         (uint32_t)(seed >> 32)); note_launch();
   return cudaGetLastError() == cudaSuccess ? PSB_OK : PSB_ERR_CUDA;
 }
 
@@ -383,7 +383,7 @@ cudaError_t launch_export(const psb_weights* wt, uint32_t level, int32_t* wint_o
     uint32_t blocks = (uint32_t)((total + 255) / 256);
     blocks = blocks > 4096 ? 4096 : (blocks < 1 ? 1 : blocks);
     export_kernel<<<blocks, 256, 0, s>>>(wt->level[level].wint, wint_out, sh.out_ch,
-                                        sh.in_ch_per_group, sh.kh * sh.kw);
+                                        sh.in_ch_per_group, sh.kh * sh.kw); note_launch();
   }
   if (e_base_out) {
     cudaError_t e = cudaMemcpyAsync(e_base_out, wt->e_base, sizeof(int32_t) * sh.out_ch,
@@ -489,18 +489,18 @@ extern "C" psb_status psb_sample_level_static(const float* w_dev, const psb_wsha
   // the array keeps the previous call's maxima: the reduction must start from zero
   if (cudaMemsetAsync(e_max, 0, sizeof(uint32_t) * O, s) != cudaSuccess) return PSB_ERR_CUDA;
   if (cfg->norm) {
-    emax_kernel<<<O, kThreads, 0, s>>>(w_dev, O, d, 1, e_max, err_sink);
+    emax_kernel<<<O, kThreads, 0, s>>>(w_dev, O, d, 1, e_max, err_sink); note_launch();
   } else {
     size_t total = (size_t)O * d;
     uint32_t blocks = (uint32_t)((total + kThreads * 8 - 1) / (kThreads * 8));
     blocks = blocks < 1 ? 1 : (blocks > 1184 ? 1184 : blocks);
-    emax_kernel<<<blocks, kThreads, 0, s>>>(w_dev, O, d, 0, e_max, err_sink);
+    emax_kernel<<<blocks, kThreads, 0, s>>>(w_dev, O, d, 0, e_max, err_sink); note_launch();
   }
   size_t total = (size_t)O * d;
   uint32_t blocks = (uint32_t)((total + kThreads - 1) / kThreads);
   blocks = blocks > 148u * 16u ? 148u * 16u : blocks;
   sample_level_canonical_kernel<<<blocks, kThreads, 0, s>>>(
       w_dev, O, d, cfg->norm, (1u << exp_bits) - 1u, log2k, (uint32_t)cfg->seed,
-      (uint32_t)(cfg->seed >> 32), cfg->layer_id, e_max, wint_out_dev, e_base_out_dev);
+      (uint32_t)(cfg->seed >> 32), cfg->layer_id, e_max, wint_out_dev, e_base_out_dev); note_launch();
   return cudaGetLastError() == cudaSuccess ? PSB_OK : PSB_ERR_CUDA;
 }

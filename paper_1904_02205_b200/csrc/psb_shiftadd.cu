@@ -403,7 +403,7 @@ uint32_t grid_for(size_t total, uint32_t threads) {
 
 cudaError_t launch_offset128(const void* src, void* dst, size_t bytes, cudaStream_t s) {
   const size_t n16 = bytes / 16;
-  offset128_kernel<<<grid_for(n16, 256), 256, 0, s>>>((const uint4*)src, (uint4*)dst, n16);
+  offset128_kernel<<<grid_for(n16, 256), 256, 0, s>>>((const uint4*)src, (uint4*)dst, n16); note_launch();
   return cudaGetLastError();
 }
 
@@ -435,15 +435,16 @@ cudaError_t launch_shift_add(const ConvArgs& a, const WintTable& wt, cudaStream_
           if (sg) dwconv3x3_row_kernel<2, true><<<blocks, 256, 0, s>>>(a, wl);
           else dwconv3x3_row_kernel<2, false><<<blocks, 256, 0, s>>>(a, wl);
         }
+        note_launch();
         return cudaGetLastError();
       }
     }
     uint32_t blocks = grid_for(total / 8, 256);
     if (blocks > 148u * 4u) blocks = 148u * 4u;
-    dwconv_nhwc8_kernel<<<blocks, 256, dw_smem, s>>>(a, wt.w[a.uniform_log2k]);
+    dwconv_nhwc8_kernel<<<blocks, 256, dw_smem, s>>>(a, wt.w[a.uniform_log2k]); note_launch();
     return cudaGetLastError();
   }
-  conv_direct_kernel<<<grid_for(total, 256), 256, 0, s>>>(a, wt);
+  conv_direct_kernel<<<grid_for(total, 256), 256, 0, s>>>(a, wt); note_launch();
   return cudaGetLastError();
 }
 
@@ -454,7 +455,7 @@ cudaError_t launch_im2col_s8(const ConvArgs& a, uint32_t kpad, uint32_t offset, 
   const size_t smem = kpad * sizeof(uint32_t) + (size_t)a.KH * span_bytes;
   if (smem > 48 * 1024 || (uint64_t)a.N * a.OH * strips >= (1ull << 31) || a.KW * a.C >= (1u << 24))
     return cudaErrorInvalidValue;
-  im2col_s8_kernel<<<a.N * a.OH * strips, 256, smem, s>>>(a, kpad, offset, span_bytes, dst);
+  im2col_s8_kernel<<<a.N * a.OH * strips, 256, smem, s>>>(a, kpad, offset, span_bytes, dst); note_launch();
   return cudaGetLastError();
 }
 
@@ -462,7 +463,7 @@ cudaError_t launch_nchw_to_nhwc(const void* src, void* dst, uint32_t N, uint32_t
                                 uint32_t elem_bytes, cudaStream_t s) {
   if (elem_bytes != 1) return cudaErrorInvalidValue;
   dim3 grid((HW + 31) / 32, (C + 31) / 32, N), block(32, 8);
-  nchw_to_nhwc_u8_kernel<<<grid, block, 0, s>>>((const uint8_t*)src, (uint8_t*)dst, C, HW);
+  nchw_to_nhwc_u8_kernel<<<grid, block, 0, s>>>((const uint8_t*)src, (uint8_t*)dst, C, HW); note_launch();
   return cudaGetLastError();
 }
 
@@ -475,6 +476,7 @@ cudaError_t launch_maxpool(const uint8_t* x, uint32_t nchw, uint32_t N, uint32_t
     maxpool_nhwc16_kernel<<<grid_for(total / 16, 256), 256, 0, s>>>(x, N, C, H, W, k, stride, pad, OH, OW, out);
   else
     maxpool_kernel<<<grid_for(total, 256), 256, 0, s>>>(x, nchw, N, C, H, W, k, stride, pad, OH, OW, out);
+  note_launch();
   return cudaGetLastError();
 }
 
@@ -483,7 +485,7 @@ cudaError_t launch_avgpool(const uint8_t* x, uint32_t nchw, uint32_t N, uint32_t
                            cudaStream_t s) {
   size_t warps = (size_t)N * C;
   uint32_t blocks = (uint32_t)((warps * 32 + 255) / 256);
-  avgpool_kernel<<<blocks, 256, 0, s>>>(x, nchw, N, C, H * W, pool_mul, qmin, qmax, out);
+  avgpool_kernel<<<blocks, 256, 0, s>>>(x, nchw, N, C, H * W, pool_mul, qmin, qmax, out); note_launch();
   return cudaGetLastError();
 }
 

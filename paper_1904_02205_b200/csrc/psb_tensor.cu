@@ -328,6 +328,30 @@ __device__ __forceinline__ void store_row16(uint8_t* dst, uint4 v, bool vec16, b
   }
 }
 
+// The same 16 channels of one output location in a planar ([n][o][oy][ox]) tensor: byte j sits
+// j * plane further on.  Lanes of a warp hold consecutive locations, so each of the 16 accesses
+// is a contiguous run of 32 bytes per warp.
+__device__ __noinline__ uint4 load_planar16(const uint8_t* src, size_t plane, uint32_t count) {
+  uint32_t w[4] = {0u, 0u, 0u, 0u};
+#pragma unroll
+  for (int j = 0; j < 16; ++j)
+    if ((uint32_t)j < count) w[j >> 2] |= (uint32_t)__ldg(src + (size_t)j * plane) << (8 * (j & 3));
+  return make_uint4(w[0], w[1], w[2], w[3]);
+}
+__device__ __noinline__ void store_planar16(uint8_t* dst, size_t plane, uint32_t count, uint4 v) {
+  const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+  for (int j = 0; j < 16; ++j)
+    if ((uint32_t)j < count) dst[(size_t)j * plane] = (uint8_t)(w[j >> 2] >> (8 * (j & 3)));
+}
+
+// Offset of (row m, channel o_base) in the output tensor, either layout.
+__device__ __forceinline__ size_t out_offset(const ConvArgs& a, uint32_t ohow, uint32_t m, uint32_t o_base) {
+  if (!a.out_nchw) return (size_t)m * a.O + o_base;
+  const uint32_t n = m / ohow;
+  return ((size_t)n * a.O + o_base) * ohow + (m - n * ohow);
+}
+
 template <int P, int MODE, bool HAS_RES>
 __device__ __noinline__ void epilogue_chunk_q(uint32_t taddr, bool valid, uint8_t* q_dst, uint4 r4, bool vec16,
                                               bool both, const float2* scb, const long long* corr, EpiConst c) {
@@ -388,12 +412,19 @@ __device__ __noinline__ void epilogue_chunk(const TensorParams& p, uint32_t tadd
     *reinterpret_cast<uint4*>((uint8_t*)a.q_out + (size_t)m * a.O + o_base) = make_uint4(qw[0], qw[1], qw[2], qw[3]);
 }
 
+// True when the layer takes the specialised epilogue loop below.
+__device__ __forceinline__ bool uniform_epilogue(const TensorParams& p) {
+  const ConvArgs& a = p.a;
+  const bool q_only = a.q_out && !a.f32_out && !a.acc_out && (p.vec_ok || a.out_nchw);
+  const uint32_t P0 = p.planes[a.uniform_log2k < (uint32_t)kMaxLevels ? a.uniform_log2k : 0u];
+  return !a.kmap && q_only && (P0 == 3u || P0 == 4u);
+}
+
 // Epilogue loop of one warp for the common case: one draw count for the whole layer, only
-// re-quantised bytes wanted, channels-last, whole 16-channel chunks.  The warp owns 32 rows
-// (its TMEM lane quarter) x 16 channels of every tile.  Per tile: wait for the accumulator, pull
-// the chunk into registers, hand the TMEM buffer back at once (the MMA of the tile after next can
-// start), then do the arithmetic and the 16-byte store.  Shortcut bytes are fetched one tile ahead.
-// Returns true if a wait timed out.
+// re-quantised bytes wanted.  The warp owns 32 rows (its TMEM lane quarter) x 16 channels of
+// every tile.  Per tile: wait for the accumulator, pull the chunk into registers, hand the TMEM
+// buffer back at once (the MMA of the tile after next can start), then do the arithmetic and
+// the store.  Shortcut bytes are fetched one tile ahead.  Returns true if a wait timed out.
 template <int P, int MODE, bool HAS_RES>
 __device__ __noinline__ bool epilogue_uniform(const TensorParams& p, SharedCtl* ctl, uint32_t tmem_base,
                                               uint32_t ew, uint32_t lane, EpiConst c) {
@@ -406,14 +437,18 @@ __device__ __noinline__ bool epilogue_uniform(const TensorParams& p, SharedCtl* 
   const uint8_t* res_base = (const uint8_t*)a.residual;
   const float2* scb = ctl->scb[ew];
   const long long* corr = ctl->corr[ew];
-  const bool vec16 = p.vec_ok == 2u;
+  const bool vec16 = p.vec_ok == 2u, planar = a.out_nchw != 0u;
+  const uint32_t ohow = a.OH * a.OW;
   TileIter ti;
   ti.init(p);
   uint32_t pass = 0, cur_o_tile = 0xFFFFFFFFu;
   uint4 r_next = make_uint4(0, 0, 0, 0);
   if (HAS_RES && ti.valid()) {
     const uint32_t m = ti.m_tile * kTileM + row, ob = ti.o_tile * kTileN + sub * 16u;
-    if (m < p.M && ob < a.O) r_next = load_row16(res_base + (size_t)m * a.O + ob, vec16, ob + 16u <= a.O);
+    if (m < p.M && ob < a.O) {
+      const uint8_t* src = res_base + out_offset(a, ohow, m, ob);
+      r_next = planar ? load_planar16(src, ohow, a.O - ob) : load_row16(src, vec16, ob + 16u <= a.O);
+    }
   }
   while (ti.valid()) {
     const uint32_t m = ti.m_tile * kTileM + row;
@@ -443,7 +478,10 @@ __device__ __noinline__ bool epilogue_uniform(const TensorParams& p, SharedCtl* 
     if (HAS_RES && ti.valid()) {
       const uint32_t mn = ti.m_tile * kTileM + row, ob = ti.o_tile * kTileN + sub * 16u;
       r_next = make_uint4(0, 0, 0, 0);
-      if (mn < p.M && ob < a.O) r_next = load_row16(res_base + (size_t)mn * a.O + ob, vec16, ob + 16u <= a.O);
+      if (mn < p.M && ob < a.O) {
+        const uint8_t* src = res_base + out_offset(a, ohow, mn, ob);
+        r_next = planar ? load_planar16(src, ohow, a.O - ob) : load_row16(src, vec16, ob + 16u <= a.O);
+      }
     }
     const uint32_t buf = pass & 1u, aph = (pass >> 1) & 1u;
     const bool ok = mbar_wait(smem_u32(&ctl->acc_full[buf]), aph, abort, 32);
@@ -460,9 +498,12 @@ __device__ __noinline__ bool epilogue_uniform(const TensorParams& p, SharedCtl* 
     tc_fence_before();
     __syncwarp();
     if (lane == 0) mbar_arrive(smem_u32(&ctl->acc_empty[buf]));
-    if (active && m < p.M)
-      store_row16((uint8_t*)a.q_out + (size_t)m * a.O + o_base, chunk_math<P, MODE, HAS_RES>(v, r_cur, scb, corr, c),
-                  vec16, o_base + 16u <= a.O);
+    if (active && m < p.M) {
+      const uint4 q16 = chunk_math<P, MODE, HAS_RES>(v, r_cur, scb, corr, c);
+      uint8_t* dst = (uint8_t*)a.q_out + out_offset(a, ohow, m, o_base);
+      if (planar) store_planar16(dst, ohow, a.O - o_base, q16);
+      else store_row16(dst, q16, vec16, o_base + 16u <= a.O);
+    }
     ++pass;
   }
   return false;
@@ -540,10 +581,11 @@ psb_mma_kernel(const __grid_constant__ TmapSet maps, const __grid_constant__ Ten
         const uint32_t m_tile = ti.m_tile, o_tile = ti.o_tile;
         const uint32_t m0 = m_tile * kTileM;
         const uint32_t levels = tile_levels_serial(p, m0) & p.a.level_mask;
-        const uint32_t ohow = p.a.OH * p.a.OW;
-        const uint32_t n0 = m0 / ohow, rem = m0 % ohow;
-        const int h0 = (int)((rem / p.a.OW) * p.a.stride) - (int)p.a.pad;
-        const int w0 = (int)((rem % p.a.OW) * p.a.stride) - (int)p.a.pad;
+        // image coordinates of the tile's first row: divisions, so only the thread that is about to
+        // issue a copy of this tile computes them
+        uint32_t n0 = 0;
+        int h0 = 0, w0 = 0;
+        bool have_coords = !p.im2col;
         // one pass per level present in the tile (levels that were not sampled are flagged by the
         // epilogue and skipped by every role)
         for (uint32_t todo = levels & 0x7Fu; todo && !failed; todo &= todo - 1u) {
@@ -556,6 +598,14 @@ psb_mma_kernel(const __grid_constant__ TmapSet maps, const __grid_constant__ Ten
             const uint32_t cnt = min(p.group, k_iters - it);
             const bool mine = turn == warp;
             if (mine) {
+              if (!have_coords) {
+                const uint32_t ohow = p.a.OH * p.a.OW;
+                n0 = m0 / ohow;
+                const uint32_t rem = m0 - n0 * ohow, oy = rem / p.a.OW;
+                h0 = (int)(oy * p.a.stride) - (int)p.a.pad;
+                w0 = (int)((rem - oy * p.a.OW) * p.a.stride) - (int)p.a.pad;
+                have_coords = true;
+              }
               if (!mbar_wait(smem_u32(&ctl->empty[s]), ph ^ 1u, abort)) { failed = true; break; }
               mbar_expect_tx(smem_u32(&ctl->full[s]), bytes * cnt);
             }
@@ -591,7 +641,7 @@ psb_mma_kernel(const __grid_constant__ TmapSet maps, const __grid_constant__ Ten
       uint32_t s = 0, ph = 0, pass = 0;
       if (p.resident && !mbar_wait(smem_u32(&ctl->planes_full), 0u, abort)) failed = true;
       const uint32_t ring_addr = smem_u32(ring), planes_addr = smem_u32(smem);
-      bool next_full = false;
+      bool next_full = false, acc_ready = false;
       TileIter ti;
       for (ti.init(p); !failed && ti.valid(); ti.next()) {
         const uint32_t m0 = ti.m_tile * kTileM;
@@ -605,8 +655,10 @@ psb_mma_kernel(const __grid_constant__ TmapSet maps, const __grid_constant__ Ten
                                  ((kTileM >> 4) << 24);
           const uint32_t d_tmem = tmem_base + buf * kTmemBufStride;
           const uint32_t blk = P * kTileN * BK;
-          if (!mbar_wait(smem_u32(&ctl->acc_empty[buf]), aph ^ 1u, abort)) { failed = true; break; }
+          if (!acc_ready && !mbar_wait(smem_u32(&ctl->acc_empty[buf]), aph ^ 1u, abort)) { failed = true; break; }
           tc_fence_after();
+          // probe the buffer of the following pass now; the answer is needed only after this pass's MMAs
+          acc_ready = mbar_try_wait(smem_u32(&ctl->acc_empty[buf ^ 1u]), (((pass + 1u) >> 1) & 1u) ^ 1u);
           uint32_t b_res = planes_addr;
           for (uint32_t it = 0; it < k_iters;) {
             const uint32_t cnt = min(p.group, k_iters - it);
@@ -644,7 +696,7 @@ psb_mma_kernel(const __grid_constant__ TmapSet maps, const __grid_constant__ Ten
     const uint32_t sub = ew >> 2;
     const uint32_t row = quarter * 32u + lane;
     const ConvArgs& a = p.a;
-    const bool q_only = a.q_out && !a.f32_out && !a.acc_out && p.vec_ok;
+    const bool q_only = a.q_out && !a.f32_out && !a.acc_out && (p.vec_ok || a.out_nchw);
     EpiConst ec;
     ec.res_scale = a.residual_scale;
     // a clamp at qmin >= 0 already removes negatives, so the relu only matters for signed codes
@@ -654,7 +706,7 @@ psb_mma_kernel(const __grid_constant__ TmapSet maps, const __grid_constant__ Ten
     ec.qmax_f = (float)a.qmax;
     ec.res_sign = a.residual_dtype == PSB_DT_S8 ? 0x80u : 0u;
     const uint32_t P0 = p.planes[a.uniform_log2k < (uint32_t)kMaxLevels ? a.uniform_log2k : 0u];
-    if (!a.kmap && q_only && (P0 == 3u || P0 == 4u)) {
+    if (uniform_epilogue(p)) {
       const uint32_t mode = (p.corr[a.uniform_log2k] != nullptr || P0 == 4u) ? 0u : p.narrow;
 #define PSB_UNI(PV, MV, RV) failed = epilogue_uniform<PV, MV, RV>(p, ctl, tmem_base, ew, lane, ec)
       if (a.residual) {
@@ -682,7 +734,7 @@ psb_mma_kernel(const __grid_constant__ TmapSet maps, const __grid_constant__ Ten
         const uint32_t o_base = o_tile * kTileN + sub * 16u;
         const size_t oidx = (size_t)m * a.O + o_base;
         const bool vec16 = p.vec_ok == 2u, both = o_base + 16u <= a.O;
-        const bool fast = q_only && o_base < a.O;
+        const bool fast = q_only && !a.out_nchw && o_base < a.O;
         uint4 r4 = make_uint4(0, 0, 0, 0);
         if (fast && a.residual && in_range) r4 = load_row16((const uint8_t*)a.residual + oidx, vec16, both);
         for (uint32_t todo = levels & 0x7Fu; todo && !failed; todo &= todo - 1u) {
@@ -914,7 +966,7 @@ psb_status launch_tensor(psb_ctx* ctx, const psb_weights* wt, const ConvArgs& a,
 #define PSB_LAUNCH(BKV)                                                                              \
   e = cudaFuncSetAttribute(psb_mma_kernel<BKV>, cudaFuncAttributeMaxDynamicSharedMemorySize,         \
                            (int)smem_bytes);                                                         \
-  if (e == cudaSuccess) psb_mma_kernel<BKV><<<grid, kThreadsTensor, smem_bytes, s>>>(maps, p);
+  if (e == cudaSuccess) psb_mma_kernel<BKV><<<grid, kThreadsTensor, smem_bytes, s>>>(maps, p); note_launch();
   if (bk == 128) { PSB_LAUNCH(128) } else if (bk == 64) { PSB_LAUNCH(64) } else { PSB_LAUNCH(32) }
 #undef PSB_LAUNCH
   if (e != cudaSuccess || cudaGetLastError() != cudaSuccess) return PSB_ERR_CUDA;

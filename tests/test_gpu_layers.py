@@ -231,6 +231,18 @@ def test_tensor_path_rows_of_odd_multiples_of_eight_channels(psb, ctx, oracle, O
     assert g["path"] == psb.PSB_PATH_TENSOR
 
 
+@pytest.mark.parametrize("O,with_res", [(64, False), (72, True), (20, True)])
+def test_tensor_path_planar_layout_codes_only(psb, ctx, oracle, O, with_res):
+    """[n][c][h][w] tensors in and out, only re-quantised codes wanted: planar stores from the tensor path."""
+    rng = np.random.default_rng(O + 1)
+    N, C, H, W = 3, 64, 14, 13
+    w, x, scale, bias = _layer_inputs(rng, N, C, H, W, O, 3, 3, 1, 0, x_hi=16)
+    res = rng.integers(0, 16, size=(N, O, H, W)).astype(np.uint8) if with_res else None
+    g = _both(psb, ctx, oracle, w, x, 0, 1, 1, 1, [3], scale, bias, inv_step=0.4, qmax=15, residual=res,
+              res_scale=0.3, in_max=15, path=psb.PSB_PATH_TENSOR, want=("q",))
+    assert g["path"] == psb.PSB_PATH_TENSOR
+
+
 def test_depthwise_5x5_codes_only(psb, ctx, oracle):
     rng = np.random.default_rng(55)
     C = 48

@@ -12,6 +12,8 @@
 
 #include "psb_common.cuh"
 
+#include <algorithm>
+
 namespace psb {
 
 namespace {
@@ -246,13 +248,19 @@ uint32_t fill_sample_params(const float* w_dev, const psb_weights* wt, uint32_t*
   const uint32_t O = sh.out_ch, Cg = sh.in_ch_per_group, KHKW = sh.kh * sh.kw, d = wt->d;
   p.w = w_dev;
   p.O = O; p.Cg = Cg; p.KHKW = KHKW; p.d = d;
-  if (d <= (uint32_t)kStage) {
-    p.rows_per_block = kStage / d;
+  // weights per block: the whole staging buffer for large layers, less for small ones so that
+  // the layer still spreads over a few hundred blocks
+  const uint64_t total = (uint64_t)O * d;
+  uint32_t budget = (uint32_t)std::min<uint64_t>((uint64_t)kStage, std::max<uint64_t>(256u, total / 296u));
+  if (budget < KHKW) budget = KHKW;   // at least one channel (host validation keeps kh*kw <= kStage)
+  if (d <= budget) {
+    p.rows_per_block = budget / d;
     p.ch_per_block = Cg;
     p.ch_chunks = 1;
   } else {
     p.rows_per_block = 1;
-    p.ch_per_block = kStage / KHKW;
+    p.ch_per_block = budget / KHKW;
+    if (p.ch_per_block > 16u) p.ch_per_block &= ~15u;   // whole 16-byte pieces of the plane rows
     p.ch_chunks = (Cg + p.ch_per_block - 1) / p.ch_per_block;
   }
   p.norm = wt->cfg.norm;

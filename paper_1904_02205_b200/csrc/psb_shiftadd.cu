@@ -317,6 +317,43 @@ __global__ void nchw_to_nhwc_u8_kernel(const uint8_t* __restrict__ src, uint8_t*
   }
 }
 
+// The same for C and HW multiples of 4, four bytes at a time.  A block moves 32 channels x 128
+// locations.  Warp i takes channels 4i..4i+3: each lane loads 4 locations of each of them (four
+// 128-byte runs per warp), transposes the 4x4 bytes in registers and parks the four words (one
+// per location, 4 channels each) in shared memory with one 16-byte store.  Then 8 consecutive
+// lanes write the 32 channel bytes of one location: whole 32-byte sectors, no bank conflicts
+// (row pitch 132 words: bank = 4 * quad + location).
+__global__ void __launch_bounds__(256) nchw_to_nhwc_u8x4_kernel(const uint8_t* __restrict__ src,
+                                                               uint8_t* __restrict__ dst, uint32_t C,
+                                                               uint32_t HW) {
+  __shared__ __align__(16) uint32_t tile[8][132];
+  const size_t base = (size_t)blockIdx.z * C * HW;
+  const uint32_t p0 = blockIdx.x * 128u, c0 = blockIdx.y * 32u;
+  const uint32_t warp = threadIdx.x >> 5, lane = threadIdx.x & 31u;
+  {
+    const uint32_t c = c0 + 4u * warp, p = p0 + 4u * lane;
+    uint32_t r[4] = {0u, 0u, 0u, 0u};
+    if (c < C && p < HW) {
+#pragma unroll
+      for (int k = 0; k < 4; ++k)
+        r[k] = __ldg(reinterpret_cast<const uint32_t*>(src + base + (size_t)(c + k) * HW + p));
+    }
+    const uint32_t a = __byte_perm(r[0], r[1], 0x5140), b = __byte_perm(r[2], r[3], 0x5140);
+    const uint32_t cc = __byte_perm(r[0], r[1], 0x7362), d = __byte_perm(r[2], r[3], 0x7362);
+    *reinterpret_cast<uint4*>(&tile[warp][4u * lane]) =
+        make_uint4(__byte_perm(a, b, 0x5410), __byte_perm(a, b, 0x7632), __byte_perm(cc, d, 0x5410),
+                   __byte_perm(cc, d, 0x7632));
+  }
+  __syncthreads();
+  const uint32_t q = threadIdx.x & 7u;
+#pragma unroll
+  for (int r = 0; r < 4; ++r) {
+    const uint32_t pl = (threadIdx.x >> 3) + 32u * r;
+    const uint32_t p = p0 + pl, c = c0 + 4u * q;
+    if (p < HW && c < C) *reinterpret_cast<uint32_t*>(dst + base + (size_t)p * C + c) = tile[q][pl];
+  }
+}
+
 __global__ void maxpool_kernel(const uint8_t* __restrict__ x, uint32_t nchw, uint32_t N, uint32_t C,
                                uint32_t H, uint32_t W, uint32_t k, uint32_t stride, uint32_t pad,
                                uint32_t OH, uint32_t OW, uint8_t* __restrict__ out) {
@@ -462,8 +499,14 @@ cudaError_t launch_im2col_s8(const ConvArgs& a, uint32_t kpad, uint32_t offset, 
 cudaError_t launch_nchw_to_nhwc(const void* src, void* dst, uint32_t N, uint32_t C, uint32_t HW,
                                 uint32_t elem_bytes, cudaStream_t s) {
   if (elem_bytes != 1) return cudaErrorInvalidValue;
-  dim3 grid((HW + 31) / 32, (C + 31) / 32, N), block(32, 8);
-  nchw_to_nhwc_u8_kernel<<<grid, block, 0, s>>>((const uint8_t*)src, (uint8_t*)dst, C, HW); note_launch();
+  if (C % 4u == 0 && HW % 4u == 0 && !(((uintptr_t)src | (uintptr_t)dst) & 3u)) {
+    dim3 grid4((HW + 127) / 128, (C + 31) / 32, N);
+    nchw_to_nhwc_u8x4_kernel<<<grid4, 256, 0, s>>>((const uint8_t*)src, (uint8_t*)dst, C, HW);
+  } else {
+    dim3 grid((HW + 31) / 32, (C + 31) / 32, N), block(32, 8);
+    nchw_to_nhwc_u8_kernel<<<grid, block, 0, s>>>((const uint8_t*)src, (uint8_t*)dst, C, HW);
+  }
+  note_launch();
   return cudaGetLastError();
 }
 

@@ -325,6 +325,24 @@ def run_reference(args):
     return 0
 
 
+def run_int8_probe(ctx, index):
+    """Ceiling of the dense path: back-to-back int8 MMAs from resident shared-memory tiles on every SM."""
+    clocks = ClockSampler(index)
+    clocks.start()
+    rows = []
+    for n_cols in (64, 128, 192, 256):
+        for _ in range(3):
+            mac_clk, tops = ctx.int8_mma_probe(n_cols, 20000)
+        rows.append(dict(n_cols=n_cols, mac_per_clk_per_sm=mac_clk, tera_ops_per_s=tops))
+    ctx.check_device()
+    peaks = measured_peaks()
+    print(json.dumps(dict(probe="tcgen05.mma.cta_group::1.kind::i8, M=128, K=32, operands resident in shared memory",
+                          rows=rows, clocks=clocks.stop(),
+                          bf16_x2_burst=2.0 * peaks["bf16_tflops"], bf16_x2_sustained=2.0 * peaks["bf16_tflops_sustained"],
+                          peak_source=peaks["source"])))
+    return 0
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -336,6 +354,8 @@ def main():
     ap.add_argument("--batch", type=int, default=0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--layer-table", default="", help="write per-layer times of the network workloads to this CSV")
+    ap.add_argument("--probe-int8", action="store_true",
+                    help="measure the bare tcgen05 int8 MMA issue rate instead of a workload and exit")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl != "reference" else args.warmup
     if args.impl == "reference":
@@ -353,6 +373,8 @@ def main():
         dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
     torch.cuda.set_device(local_rank)
     ctx = psb.Context(local_rank)
+    if args.probe_int8:
+        return run_int8_probe(ctx, local_rank)
     wl = make_workload(args, rank)
     wl.setup(ctx, psb, torch)
     flush = torch.empty(512 << 20, dtype=torch.uint8, device=ctx.device)   # > L2 (126 MB)

@@ -210,6 +210,21 @@ int32_t psb_last_path(const psb_ctx* ctx);
  * many launches a timed region took.  Never fails. */
 uint64_t psb_launch_count(void);
 
+/* Measurement aid, no counterpart in the paper: the ceiling of the dense path.
+ * Every SM issues `groups` groups of four back-to-back tcgen05.mma kind::i8
+ * instructions (M = 128, N = n_cols, K = 32, s8 x s8 -> s32 in TMEM) on zero
+ * operand tiles resident in shared memory; nothing is copied or stored.
+ *   n_cols: 16..256, multiple of 16.  groups: 1..2^20.
+ *   mac_per_clk_per_sm (host, out): int8 multiply-accumulates per SM clock of
+ *     the slowest SM, from the SM cycle counter.
+ *   tera_ops_per_s (host, out): 2 * MACs of all SMs / elapsed time of the
+ *     launch (CUDA events on `stream`), in 10^12 operations per second.
+ * Synchronises `stream` and allocates one small device buffer for the duration
+ * of the call.  A wait that runs out sets the device error word (see
+ * psb_device_status).  Errors: PSB_ERR_INVALID_ARG, PSB_ERR_ALLOC, PSB_ERR_CUDA. */
+psb_status psb_int8_mma_probe(psb_ctx* ctx, uint32_t n_cols, uint32_t groups, double* mac_per_clk_per_sm,
+                              double* tera_ops_per_s, void* stream);
+
 /* Glue between layers (supplement, "ReLU, Batch-Norm, and Pooling"): max-pooling
  * is comparators only; the 1/(h*w) of average pooling is folded into one
  * re-quantisation factor.

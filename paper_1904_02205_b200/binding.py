@@ -24,7 +24,7 @@ EXPORTS = ["psb_create", "psb_destroy", "psb_status_string", "psb_device_status"
            "psb_weights_export", "psb_weights_free", "psb_set_sample_map", "psb_conv2d", "psb_gemm",
            "psb_last_path", "psb_maxpool2d_u8", "psb_global_avgpool_u8", "psb_sample_level_static",
            "psb_sample_batch_create", "psb_sample_batch_run", "psb_sample_batch_free", "psb_run",
-           "psb_launch_count"]
+           "psb_launch_count", "psb_int8_mma_probe"]
 
 
 class psb_wshape(C.Structure):
@@ -90,6 +90,7 @@ def load_library():
     lib.psb_conv2d.argtypes = [vp, vp, vp, C.POINTER(psb_conv_desc), vp]
     lib.psb_gemm.argtypes = [vp, vp, vp, C.POINTER(psb_gemm_desc), vp]
     lib.psb_last_path.argtypes = [vp]
+    lib.psb_int8_mma_probe.argtypes = [vp, u32, u32, C.POINTER(C.c_double), C.POINTER(C.c_double), vp]
     lib.psb_launch_count.argtypes = []
     lib.psb_launch_count.restype = C.c_uint64
     lib.psb_maxpool2d_u8.argtypes = [vp, vp, u32, u32, u32, u32, u32, u32, u32, u32, vp, vp]
@@ -199,6 +200,13 @@ class Context:
 
     def last_path(self):
         return self.lib.psb_last_path(self.handle)
+
+    def int8_mma_probe(self, n_cols=192, groups=4000, stream=None):
+        """Returns (int8 MAC per clock per SM, tera-operations per second) of bare MMA issue."""
+        a, b = C.c_double(0.0), C.c_double(0.0)
+        _check(self.lib.psb_int8_mma_probe(self.handle, n_cols, groups, C.byref(a), C.byref(b), _stream(stream)),
+               "psb_int8_mma_probe")
+        return a.value, b.value
 
     def launch_count(self):
         """Kernels launched by the library in this process so far."""

@@ -378,6 +378,13 @@ int32_t psb_last_path(const psb_ctx* ctx) { return ctx ? ctx->last_path : 0; }
 
 uint64_t psb_launch_count(void) { return (uint64_t)psb::launches_so_far(); }
 
+psb_status psb_int8_mma_probe(psb_ctx* ctx, uint32_t n_cols, uint32_t groups, double* mac_per_clk_per_sm,
+                              double* tera_ops_per_s, void* stream) {
+  if (!ctx) return PSB_ERR_INVALID_ARG;
+  cudaSetDevice(ctx->device);
+  return psb::int8_mma_probe(ctx, n_cols, groups, mac_per_clk_per_sm, tera_ops_per_s, (cudaStream_t)stream);
+}
+
 psb_status psb_sample_batch_create(psb_ctx* ctx, uint32_t n, const float* const* w_dev,
                                    psb_weights* const* weights, psb_sample_batch** batch) {
   if (!ctx || !n || !w_dev || !weights || !batch) return PSB_ERR_INVALID_ARG;

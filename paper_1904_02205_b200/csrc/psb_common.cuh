@@ -179,4 +179,8 @@ psb_status tensor_supported(const psb_ctx* ctx, const psb_weights* wt, const Con
 psb_status launch_tensor(psb_ctx* ctx, const psb_weights* wt, const ConvArgs& a, uint32_t amax,
                          bool add_corr128, cudaStream_t s);
 
+// int8 tensor-core issue-rate probe (psb_probe.cu)
+psb_status int8_mma_probe(psb_ctx* ctx, uint32_t n_cols, uint32_t groups, double* mac_per_clk_per_sm,
+                          double* tera_ops_per_s, cudaStream_t s);
+
 }  // namespace psb

@@ -409,3 +409,14 @@ def test_pooling_kernels(psb, ctx, oracle):
                               oracle.maxpool_u8(x, layout, 3, 2, 1))
         assert np.array_equal(ctx.global_avgpool_u8(xd, layout, 0.0123, 0, 255).cpu().numpy(),
                               oracle.global_avgpool_u8(x, layout, np.float32(0.0123), 0, 255))
+
+
+def test_int8_issue_rate_probe_reports_a_plausible_ceiling(psb, ctx):
+    """The measurement aid runs, leaves the device error word clear and reports between a quarter of and
+    the full documented rate of 8192 int8 multiply-accumulates per SM clock."""
+    mac_clk, tops = ctx.int8_mma_probe(192, 2000)
+    assert ctx.device_status() == 0
+    assert 2000.0 < mac_clk < 8300.0
+    assert tops > 100.0
+    with pytest.raises(psb.PsbError):
+        ctx.int8_mma_probe(200, 10)      # columns must be a multiple of 16

@@ -161,6 +161,10 @@ psb_status run_layer(psb_ctx* ctx, const psb_weights* wt, const void* x_dev, uin
         if (wt->level[l].corr128 && (ctx->kmap || l == ctx->uniform_log2k))
           if (launch_corr128(wt, l, s) != cudaSuccess) return PSB_ERR_CUDA;
     }
+    if (a.kmap) {
+      st = ensure_scratch(ctx, 2, ((size_t)a.N * a.OH * a.OW + 127) / 128);
+      if (st != PSB_OK) return st;
+    }
     st = launch_tensor(ctx, wt, a, amax, add_corr, s);
     if (st != PSB_OK) return st;
     ctx->last_path = PSB_PATH_TENSOR;

@@ -60,6 +60,7 @@ struct TensorParams {
   uint32_t group;       // K blocks per pipeline stage (one barrier hand-over per group)
   uint32_t stage_bytes_a, stage_bytes_b_max;
   uint32_t planes[kMaxLevels];
+  const uint8_t* tile_mask;   // per row tile: levels present (bit l = level l), or null without a map
   uint32_t vec_ok;      // output rows (and pointers) are multiples of 16 bytes (2), of 8 bytes (1), or neither
   uint32_t resident;    // 1: the CTA keeps the digit planes of its channel tile in shared memory
   uint32_t ctas_per_otile;
@@ -187,26 +188,25 @@ __device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t bk) {
   return d;
 }
 
-// Levels (log2 k) present among the 128 rows of a tile, as a bit mask.  Warp-collective.
-__device__ __forceinline__ uint32_t tile_levels(const TensorParams& p, uint32_t m0) {
-  if (!p.a.kmap) return 1u << p.a.uniform_log2k;
-  const uint32_t lane = threadIdx.x & 31u;
+// Levels (log2 k) present among the 128 rows of a tile, as a bit mask: one byte per row tile,
+// written by tile_levels_kernel just before the contraction kernel.
+__device__ __forceinline__ uint32_t tile_levels(const TensorParams& p, uint32_t m_tile) {
+  if (!p.tile_mask) return 1u << p.a.uniform_log2k;
+  return (uint32_t)p.tile_mask[m_tile];
+}
+
+__global__ void tile_levels_kernel(const uint8_t* __restrict__ kmap, uint32_t M, uint32_t m_tiles,
+                                   uint8_t* __restrict__ tile_mask) {
+  const uint32_t tile = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31u;
+  if (tile >= m_tiles) return;
   uint32_t mask = 0;
 #pragma unroll
   for (int r = 0; r < 4; ++r) {
-    uint32_t m = m0 + r * 32u + lane;
-    if (m < p.M) mask |= 1u << (p.a.kmap[m] & 31u);
+    const uint32_t m = tile * kTileM + r * 32u + lane;
+    if (m < M) mask |= 1u << min((uint32_t)kmap[m], 7u);   // levels >= 7 are invalid: bit 7, flagged by the epilogue
   }
-  return __reduce_or_sync(0xFFFFFFFFu, mask);
-}
-
-// Same, computed by one thread alone (the single-thread producer and MMA roles).
-__device__ __forceinline__ uint32_t tile_levels_serial(const TensorParams& p, uint32_t m0) {
-  if (!p.a.kmap) return 1u << p.a.uniform_log2k;
-  uint32_t mask = 0;
-  const uint32_t end = min(m0 + (uint32_t)kTileM, p.M);
-  for (uint32_t m = m0; m < end; ++m) mask |= 1u << (p.a.kmap[m] & 31u);
-  return mask;
+  mask = __reduce_or_sync(0xFFFFFFFFu, mask);
+  if (lane == 0) tile_mask[tile] = (uint8_t)mask;
 }
 
 // Walks the tiles of this CTA without divisions in the loop.  Resident mode: the CTA owns one
@@ -580,7 +580,7 @@ psb_mma_kernel(const __grid_constant__ TmapSet maps, const __grid_constant__ Ten
       for (ti.init(p); ti.valid() && !failed; ti.next()) {
         const uint32_t m_tile = ti.m_tile, o_tile = ti.o_tile;
         const uint32_t m0 = m_tile * kTileM;
-        const uint32_t levels = tile_levels_serial(p, m0) & p.a.level_mask;
+        const uint32_t levels = tile_levels(p, ti.m_tile) & p.a.level_mask;
         // image coordinates of the tile's first row: divisions, so only the thread that is about to
         // issue a copy of this tile computes them
         uint32_t n0 = 0;
@@ -644,8 +644,7 @@ psb_mma_kernel(const __grid_constant__ TmapSet maps, const __grid_constant__ Ten
       bool next_full = false, acc_ready = false;
       TileIter ti;
       for (ti.init(p); !failed && ti.valid(); ti.next()) {
-        const uint32_t m0 = ti.m_tile * kTileM;
-        const uint32_t levels = tile_levels_serial(p, m0) & p.a.level_mask;
+        const uint32_t levels = tile_levels(p, ti.m_tile) & p.a.level_mask;
         for (uint32_t todo = levels & 0x7Fu; todo && !failed; todo &= todo - 1u) {
           const uint32_t l = (uint32_t)__ffs((int)todo) - 1u;
           const uint32_t P = p.planes[l];
@@ -725,7 +724,7 @@ psb_mma_kernel(const __grid_constant__ TmapSet maps, const __grid_constant__ Ten
       TileIter ti;
       for (ti.init(p); !failed && ti.valid(); ti.next()) {
         const uint32_t m0 = ti.m_tile * kTileM, o_tile = ti.o_tile;
-        const uint32_t levels = tile_levels(p, m0) & a.level_mask;
+        const uint32_t levels = tile_levels(p, ti.m_tile) & a.level_mask;
         const uint32_t m = m0 + row;
         const bool in_range = m < p.M;
         const uint32_t my_level = in_range ? (a.kmap ? (uint32_t)a.kmap[m] : a.uniform_log2k) : 0xFFu;
@@ -959,6 +958,15 @@ psb_status launch_tensor(psb_ctx* ctx, const psb_weights* wt, const ConvArgs& a,
       return PSB_ERR_CUDA;
   }
 
+  p.tile_mask = nullptr;
+  if (a.kmap) {
+    // the caller has sized the third scratch buffer for one byte per row tile
+    if (!ctx->scratch[2] || ctx->scratch_bytes[2] < p.m_tiles) return PSB_ERR_INVALID_ARG;
+    tile_levels_kernel<<<(p.m_tiles * 32u + 255u) / 256u, 256, 0, s>>>(a.kmap, p.M, p.m_tiles,
+                                                                      (uint8_t*)ctx->scratch[2]);
+    note_launch();
+    p.tile_mask = (const uint8_t*)ctx->scratch[2];
+  }
   const uint32_t n_tiles = p.m_tiles * p.o_tiles;
   const uint32_t grid = p.resident ? p.o_tiles * p.ctas_per_otile
                                    : (n_tiles < (uint32_t)ctx->sm_count ? n_tiles : (uint32_t)ctx->sm_count);

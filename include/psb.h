@@ -170,8 +170,11 @@ typedef struct {
  * oh = (h + 2*pad - kh) / stride + 1 (same for ow).
  *   in_max   largest activation magnitude the caller guarantees (e.g. 15 for
  *            4-bit data); 0 means "full range of in_dtype".  The tensor path
- *            feeds activations to the MMA as signed bytes, so it needs
- *            in_max <= 127; larger unsigned data takes the shift-add path.
+ *            feeds activations to the MMA as signed bytes.  Unsigned data
+ *            above 127 reaches it as x - 128 with 128 * sum(W) added back
+ *            (filters gathered explicitly, or any filter without padding);
+ *            with padding it takes the shift-add path.  A smaller in_max also
+ *            lets the output stage recombine the digit planes in 32 bits.
  *   path     PSB_PATH_AUTO, or force one path (PSB_ERR_UNSUPPORTED if the forced
  *            path cannot run this shape). */
 typedef struct {

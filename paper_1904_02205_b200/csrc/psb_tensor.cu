@@ -65,7 +65,7 @@ struct TensorParams {
   uint32_t resident;    // 1: the CTA keeps the digit planes of its channel tile in shared memory
   uint32_t ctas_per_otile;
   uint32_t resident_bytes;
-  uint32_t narrow;      // P <= 3 and plane sums below 2^22 (2) or 2^24 (1): 32-bit recombination
+  uint32_t narrow;      // P <= 3 and plane sums below 2^22 (2) or 2^24 (1): 32-bit recombination; 3: whole sum below 2^31
   const long long* corr[kMaxLevels];  // per-channel integer addend, or null
 };
 
@@ -259,10 +259,12 @@ struct SharedCtl {
 // MODE 2: every plane sum is below 2^22 in magnitude and P <= 3: with u = v0 + 2^7 v1,
 // w = (u >> 14) + v2, acc = w * 2^14 + (u mod 2^14); both parts are exact in fp32 (by the tricks)
 // and one fma rounds acc to nearest once.  MODE 1: below 2^24 (w by a conversion instruction).
+// MODE 3: the accumulator itself is below 2^31 in magnitude: 32-bit recombination, one int -> float
+// conversion (round to nearest even, like the 64-bit one).
 // MODE 0: 64-bit recombination plus the per-channel integer addend.
 // The run-time options enter as data (a relu floor of 0 or -inf, a sign mask), not as branches.
 struct EpiConst {
-  float res_scale, relu_floor, inv_step, qmin_f, qmax_f;
+  float res_scale, inv_step, qmin_f, qmax_f;   // qmin_f already holds the relu (see the epilogue set-up)
   uint32_t res_sign;
 };
 
@@ -279,7 +281,13 @@ __device__ __forceinline__ uint4 chunk_math(const uint32_t (&v)[P][16], const ui
     for (int e = 0; e < 4; ++e) {
       const int j = 4 * g + e;
       float af;
-      if (MODE > 0) {
+      if (MODE == 3) {
+        // the whole sum fits 32 bits (wrap-around in the partial sums is harmless): one conversion
+        int acc = (int)v[0][j];
+        if (P > 1) acc += (int)v[1][j] << kDigitBits;
+        if (P > 2) acc += (int)v[2][j] << (2 * kDigitBits);
+        af = (float)acc;
+      } else if (MODE > 0) {
         int u = (int)v[0][j];
         if (P > 1) u += (int)v[1][j] << kDigitBits;
         int w = u >> (2 * kDigitBits);
@@ -300,7 +308,6 @@ __device__ __forceinline__ uint4 chunk_math(const uint32_t (&v)[P][16], const ui
         const uint32_t rb = ((rw[g] >> (8 * e)) & 0xFFu) ^ c.res_sign;   // byte + 128 if signed
         y = __fmaf_rn(__uint_as_float(0x4B000000u | rb) - res_bias, c.res_scale, y);
       }
-      y = fmaxf(y, c.relu_floor);
       // clamp, then round half to even by adding 1.5 * 2^23: the low byte of the sum is the code
       const float t = fminf(fmaxf(__fmul_rn(y, c.inv_step), c.qmin_f), c.qmax_f);
       q[e] = __float_as_uint(t + 12582912.0f);
@@ -312,12 +319,18 @@ __device__ __forceinline__ uint4 chunk_math(const uint32_t (&v)[P][16], const ui
 
 // 16 bytes of a channels-last row.  Rows that are only 8-byte aligned (channel counts that are odd
 // multiples of 8) move as two halves; `both` is false for the last 8 channels of such a row.
+// The loads are volatile asm so that they stay where they are written (a tile ahead of their use, before
+// the wait for the accumulator) instead of being sunk to the first use of the value.
 __device__ __forceinline__ uint4 load_row16(const uint8_t* src, bool vec16, bool both) {
-  if (vec16) return __ldg(reinterpret_cast<const uint4*>(src));
-  const uint2 lo = __ldg(reinterpret_cast<const uint2*>(src));
-  uint2 hi = make_uint2(0u, 0u);
-  if (both) hi = __ldg(reinterpret_cast<const uint2*>(src + 8));
-  return make_uint4(lo.x, lo.y, hi.x, hi.y);
+  uint4 r = make_uint4(0u, 0u, 0u, 0u);
+  if (vec16) {
+    asm volatile("ld.global.nc.v4.u32 {%0, %1, %2, %3}, [%4];"
+                 : "=r"(r.x), "=r"(r.y), "=r"(r.z), "=r"(r.w) : "l"(src));
+    return r;
+  }
+  asm volatile("ld.global.nc.v2.u32 {%0, %1}, [%2];" : "=r"(r.x), "=r"(r.y) : "l"(src));
+  if (both) asm volatile("ld.global.nc.v2.u32 {%0, %1}, [%2];" : "=r"(r.z), "=r"(r.w) : "l"(src + 8));
+  return r;
 }
 __device__ __forceinline__ void store_row16(uint8_t* dst, uint4 v, bool vec16, bool both) {
   if (vec16) {
@@ -415,7 +428,7 @@ __device__ __noinline__ void epilogue_chunk(const TensorParams& p, uint32_t tadd
 // True when the layer takes the specialised epilogue loop below.
 __device__ __forceinline__ bool uniform_epilogue(const TensorParams& p) {
   const ConvArgs& a = p.a;
-  const bool q_only = a.q_out && !a.f32_out && !a.acc_out && (p.vec_ok || a.out_nchw);
+  const bool q_only = a.q_out && !a.f32_out && !a.acc_out && (p.vec_ok || a.out_nchw) && a.inv_step > 0.0f;
   const uint32_t P0 = p.planes[a.uniform_log2k < (uint32_t)kMaxLevels ? a.uniform_log2k : 0u];
   return !a.kmap && q_only && (P0 == 3u || P0 == 4u);
 }
@@ -552,6 +565,13 @@ psb_mma_kernel(const __grid_constant__ TmapSet maps, const __grid_constant__ Ten
   const uint32_t tmem_base = ctl->tmem_base;
   volatile uint32_t* abort = &ctl->abort;
   bool failed = false;
+  // The kernel is launched with programmatic stream serialisation: a CTA may get here while the
+  // kernel before it in the stream is still draining.  Nothing above touches global memory; from
+  // here on everything does (activations, planes, constants, outputs), so every thread waits for
+  // the earlier grids to complete and their writes to be visible.  The kernel after this one may
+  // be scheduled as soon as SMs free up (it waits at the same point).
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  asm volatile("griddepcontrol.wait;" ::: "memory");
 
   if (warp < (uint32_t)kProducerWarps) {
     // ----------------------------------------------------------- producers
@@ -695,13 +715,13 @@ psb_mma_kernel(const __grid_constant__ TmapSet maps, const __grid_constant__ Ten
     const uint32_t sub = ew >> 2;
     const uint32_t row = quarter * 32u + lane;
     const ConvArgs& a = p.a;
-    const bool q_only = a.q_out && !a.f32_out && !a.acc_out && (p.vec_ok || a.out_nchw);
+    const bool q_only = a.q_out && !a.f32_out && !a.acc_out && (p.vec_ok || a.out_nchw) && a.inv_step > 0.0f;
     EpiConst ec;
     ec.res_scale = a.residual_scale;
-    // a clamp at qmin >= 0 already removes negatives, so the relu only matters for signed codes
-    ec.relu_floor = (a.relu && a.qmin < 0) ? 0.0f : __int_as_float(0xFF800000);
+    // With inv_step > 0 (a condition of the fast paths) max(y, 0) * inv_step == max(y * inv_step, 0):
+    // the relu is folded into the lower clamp bound.
     ec.inv_step = a.inv_step;
-    ec.qmin_f = (float)a.qmin;
+    ec.qmin_f = (a.relu && a.qmin < 0) ? 0.0f : (float)a.qmin;
     ec.qmax_f = (float)a.qmax;
     ec.res_sign = a.residual_dtype == PSB_DT_S8 ? 0x80u : 0u;
     const uint32_t P0 = p.planes[a.uniform_log2k < (uint32_t)kMaxLevels ? a.uniform_log2k : 0u];
@@ -709,10 +729,10 @@ psb_mma_kernel(const __grid_constant__ TmapSet maps, const __grid_constant__ Ten
       const uint32_t mode = (p.corr[a.uniform_log2k] != nullptr || P0 == 4u) ? 0u : p.narrow;
 #define PSB_UNI(PV, MV, RV) failed = epilogue_uniform<PV, MV, RV>(p, ctl, tmem_base, ew, lane, ec)
       if (a.residual) {
-        if (P0 == 4u) PSB_UNI(4, 0, true); else if (mode == 2u) PSB_UNI(3, 2, true);
+        if (P0 == 4u) PSB_UNI(4, 0, true); else if (mode == 3u) PSB_UNI(3, 3, true); else if (mode == 2u) PSB_UNI(3, 2, true);
         else if (mode == 1u) PSB_UNI(3, 1, true); else PSB_UNI(3, 0, true);
       } else {
-        if (P0 == 4u) PSB_UNI(4, 0, false); else if (mode == 2u) PSB_UNI(3, 2, false);
+        if (P0 == 4u) PSB_UNI(4, 0, false); else if (mode == 3u) PSB_UNI(3, 3, false); else if (mode == 2u) PSB_UNI(3, 2, false);
         else if (mode == 1u) PSB_UNI(3, 1, false); else PSB_UNI(3, 0, false);
       }
 #undef PSB_UNI
@@ -769,7 +789,7 @@ psb_mma_kernel(const __grid_constant__ TmapSet maps, const __grid_constant__ Ten
           if (o_base < a.O) {
             if (fast) {
               uint8_t* q_dst = (uint8_t*)a.q_out + oidx;
-              const uint32_t mode = (use_corr || P > 3u) ? 0u : p.narrow;
+              const uint32_t mode = (use_corr || P > 3u) ? 0u : (p.narrow > 2u ? 2u : p.narrow);
 #define PSB_EPI(PV, MV, RV) epilogue_chunk_q<PV, MV, RV>(taddr, valid, q_dst, r4, vec16, both, scb, corr, ec)
 #define PSB_EPI_P(MV, RV) do { if (P == 3) PSB_EPI(3, MV, RV); else if (P == 2) PSB_EPI(2, MV, RV); else PSB_EPI(1, MV, RV); } while (0)
               if (a.residual) {
@@ -917,6 +937,19 @@ psb_status launch_tensor(psb_ctx* ctx, const psb_weights* wt, const ConvArgs& a,
   // every plane sum is bounded by 127 * (largest activation magnitude) * d
   const uint64_t plane_bound = 127ull * amax * (uint64_t)wt->d;
   p.narrow = pmax > 3 ? 0u : (plane_bound <= 4100000ull ? 2u : (plane_bound <= 16500000ull ? 1u : 0u));
+  // every |W_k| is at most 2k * 2^(2^exp_bits - 1): if the whole accumulator stays below 2^31 the
+  // output stage recombines in 32 bits
+  {
+    uint32_t lmax = a.uniform_log2k;
+    if (a.kmap)
+      for (uint32_t l = 0; l < (uint32_t)kMaxLevels; ++l)
+        if ((a.level_mask >> l) & 1u) lmax = l;
+    const uint32_t span = (1u << wt->cfg.exp_bits) - 1u;
+    if (span + lmax + 1u < 40u) {
+      const unsigned __int128 acc_bound = (unsigned __int128)amax * wt->d * ((unsigned long long)1 << (span + lmax + 1u));
+      if (p.narrow == 2u && acc_bound < ((unsigned __int128)1 << 31)) p.narrow = 3u;
+    }
+  }
   const uintptr_t out_ptrs = (uintptr_t)a.q_out | (uintptr_t)a.residual | (uintptr_t)a.f32_out | (uintptr_t)a.acc_out;
   p.vec_ok = 0u;
   if (!a.out_nchw && a.O % 16u == 0u && !(out_ptrs & 15u)) p.vec_ok = 2u;
@@ -971,10 +1004,21 @@ psb_status launch_tensor(psb_ctx* ctx, const psb_weights* wt, const ConvArgs& a,
   const uint32_t grid = p.resident ? p.o_tiles * p.ctas_per_otile
                                    : (n_tiles < (uint32_t)ctx->sm_count ? n_tiles : (uint32_t)ctx->sm_count);
   cudaError_t e;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(grid);
+  cfg.blockDim = dim3(kThreadsTensor);
+  cfg.dynamicSmemBytes = smem_bytes;
+  cfg.stream = s;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
 #define PSB_LAUNCH(BKV)                                                                              \
   e = cudaFuncSetAttribute(psb_mma_kernel<BKV>, cudaFuncAttributeMaxDynamicSharedMemorySize,         \
                            (int)smem_bytes);                                                         \
-  if (e == cudaSuccess) psb_mma_kernel<BKV><<<grid, kThreadsTensor, smem_bytes, s>>>(maps, p); note_launch();
+  if (e == cudaSuccess) e = cudaLaunchKernelEx(&cfg, psb_mma_kernel<BKV>, maps, p);                  \
+  note_launch();
   if (bk == 128) { PSB_LAUNCH(128) } else if (bk == 64) { PSB_LAUNCH(64) } else { PSB_LAUNCH(32) }
 #undef PSB_LAUNCH
   if (e != cudaSuccess || cudaGetLastError() != cudaSuccess) return PSB_ERR_CUDA;

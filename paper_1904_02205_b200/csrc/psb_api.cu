@@ -136,7 +136,7 @@ psb_status run_layer(psb_ctx* ctx, const psb_weights* wt, const void* x_dev, uin
       st = ensure_scratch(ctx, 1, (size_t)M * wt->kpad);
       if (st != PSB_OK) return st;
       const uint32_t offset = in_dtype == PSB_DT_U8 ? 128u : 0u;
-      if (launch_im2col_s8(a, wt->kpad, offset, (int8_t*)ctx->scratch[1], s) != cudaSuccess)
+      if (launch_im2col_s8(a, wt->kpad, wt->run_pitch, offset, (int8_t*)ctx->scratch[1], s) != cudaSuccess)
         return PSB_ERR_CUDA;
       a.x = ctx->scratch[1];
       a.in_dtype = PSB_DT_S8;
@@ -294,7 +294,9 @@ psb_status psb_sample_weights(psb_ctx* ctx, const float* w_dev, const psb_wshape
     w->packed_k = shape->groups == 1 && !wide && d64 >= 16;
     w->has_planes = shape->groups == 1 && (wide || w->packed_k);
     w->cpad = shape->in_ch_per_group;
-    w->kpad = round_up(shape->kh * shape->kw * w->cpad, 16);
+    w->run_pitch = shape->kw * w->cpad;
+    if (w->packed_k) w->run_pitch = round_up(w->run_pitch, 8);
+    w->kpad = round_up(shape->kh * w->run_pitch, 16);
     w->o_tiles = (shape->out_ch + kTileN - 1) / kTileN;
     w->bk = tensor_bk(w->packed_k ? w->kpad : shape->in_ch_per_group);
     bool ok = cudaMalloc(&w->e_base, sizeof(int32_t) * shape->out_ch) == cudaSuccess &&

@@ -44,7 +44,8 @@ struct psb_weights {
   psb_sample_cfg cfg;
   uint32_t d;        // in_ch_per_group * kh * kw
   uint32_t cpad;     // channels per tap in the plane layout (multiple of the K block)
-  uint32_t kpad;     // kh * kw * cpad
+  uint32_t kpad;     // kh * kw * cpad; packed K: kh * run_pitch rounded up to 16
+  uint32_t run_pitch; // packed K: bytes reserved per filter row (kw * cin rounded up to 8); else kw * cpad
   uint32_t o_tiles;  // ceil(out_ch / kTileN)
   uint32_t bk;       // K block of the tensor path
   bool has_planes;   // digit planes are produced (groups == 1)
@@ -159,8 +160,9 @@ void sample_batch_free(psb_sample_batch* b);
 cudaError_t launch_export(const psb_weights* wt, uint32_t level, int32_t* wint_out,
                           int32_t* e_base_out, cudaStream_t s);
 cudaError_t launch_shift_add(const ConvArgs& a, const WintTable& wt, cudaStream_t s);
-// gathers [M][kpad] signed bytes (x - offset; zero padding becomes -offset, K padding 0)
-cudaError_t launch_im2col_s8(const ConvArgs& a, uint32_t kpad, uint32_t offset, int8_t* dst,
+// gathers [M][kpad] signed bytes (x - offset; zero padding becomes -offset, K padding 0); row kh of the
+// filter window occupies bytes [kh * run_pitch, kh * run_pitch + kw * c) of a matrix row
+cudaError_t launch_im2col_s8(const ConvArgs& a, uint32_t kpad, uint32_t run_pitch, uint32_t offset, int8_t* dst,
                              cudaStream_t s);
 cudaError_t launch_corr128(const psb_weights* wt, uint32_t level, cudaStream_t s);
 cudaError_t launch_offset128(const void* src, void* dst, size_t bytes, cudaStream_t s);

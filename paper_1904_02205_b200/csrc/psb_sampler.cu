@@ -86,6 +86,7 @@ struct SampleParams {
   uint32_t norm, span, level_mask, max_level;
   uint32_t seed_lo, seed_hi, layer_id;
   uint32_t cpad, kpad, has_planes;
+  uint32_t packed_kw, run_pitch;   // packed K (packed_kw = kw, else 0): plane column = kh * run_pitch + kw * Cg + ci
   const uint32_t* e_max;
   int32_t* e_base;
   int32_t* wint[kMaxLevels];
@@ -150,6 +151,11 @@ __device__ __forceinline__ void sample_block(const SampleParams& p, uint32_t blo
     }
 
     const size_t wpos = ((size_t)o * p.KHKW + tap) * p.Cg + ci;
+    uint32_t kcol = tap * p.cpad + ci;
+    if (p.packed_kw) {
+      const uint32_t kh = tap / p.packed_kw;
+      kcol = kh * p.run_pitch + (tap - kh * p.packed_kw) * p.Cg + ci;
+    }
     const uint32_t jt = o / kTileN, on = o % kTileN;
     for (uint32_t l = 0; l <= p.max_level; ++l) {
       if (!((p.level_mask >> l) & 1u)) continue;
@@ -160,7 +166,7 @@ __device__ __forceinline__ void sample_block(const SampleParams& p, uint32_t blo
         const int P = p.planes_count[l];
         for (int pl = 0; pl < P; ++pl) {
           int digit = (int)((mag >> (kDigitBits * pl)) & 0x7Fu);
-          p.planes[l][(((size_t)jt * P + pl) * kTileN + on) * p.kpad + (size_t)tap * p.cpad + ci] =
+          p.planes[l][(((size_t)jt * P + pl) * kTileN + on) * p.kpad + kcol] =
               (int8_t)(neg ? -digit : digit);
         }
       }
@@ -273,6 +279,8 @@ uint32_t fill_sample_params(const float* w_dev, const psb_weights* wt, uint32_t*
   p.seed_hi = (uint32_t)(wt->cfg.seed >> 32);
   p.layer_id = wt->cfg.layer_id;
   p.cpad = wt->cpad; p.kpad = wt->kpad; p.has_planes = wt->has_planes ? 1u : 0u;
+  p.packed_kw = wt->packed_k ? wt->shape.kw : 0u;
+  p.run_pitch = wt->run_pitch;
   p.e_max = e_max;
   p.e_base = wt->e_base;
   for (int l = 0; l < kMaxLevels; ++l) {

@@ -248,23 +248,21 @@ __global__ void offset128_kernel(const uint4* __restrict__ src, uint4* __restric
 }
 
 // Explicit gather of the activation matrix for filters with few input channels (e.g. a 7x7
-// stem on 3 channels): row m = output location, column k = (kh, kw, ci) flattened, padded with
-// zeros to kpad.  Values are stored minus `offset` as signed bytes; a padded input position is the
-// value 0, i.e. -offset.  A block handles kIm2colPix consecutive output locations of one output
-// row: the input rows they touch are staged in shared memory with coalesced loads, then every
-// thread assembles and writes 16-byte pieces of the matrix.
+// stem on 3 channels): row m = output location; filter row kh occupies bytes
+// [kh * run_pitch, kh * run_pitch + KW * C) of it, which in a channels-last image is one
+// contiguous run of the input row iy0 + kh; the rest of the matrix row is zero.  Values are
+// stored minus `offset` (0 or 128) as signed bytes; a padded input position is the value 0, i.e.
+// -offset.  A block handles kIm2colPix consecutive output locations of one output row: the KH
+// input-row spans they touch are staged in shared memory (contiguous copies, no index
+// arithmetic per byte), then each thread copies whole runs: aligned shared-memory words, a
+// funnel shift by the byte misalignment, 8-byte stores.
 constexpr uint32_t kIm2colPix = 32;
 
-__global__ void __launch_bounds__(256) im2col_s8_kernel(const ConvArgs a, uint32_t kpad, uint32_t offset,
-                                                       uint32_t span_bytes, int8_t* __restrict__ dst) {
-  extern __shared__ uint32_t im2col_smem[];
-  uint32_t* ktab = im2col_smem;                               // per column: kh | (kw*C + ci) << 8, or ~0
-  uint8_t* rows = reinterpret_cast<uint8_t*>(ktab + kpad);    // [KH][span_bytes], already offset
-  const uint32_t d = a.KH * a.KW * a.C;
-  for (uint32_t k = threadIdx.x; k < kpad; k += blockDim.x) {
-    const uint32_t tap = k / a.C, ci = k % a.C;
-    ktab[k] = k < d ? ((tap / a.KW) | (((tap % a.KW) * a.C + ci) << 8)) : 0xFFFFFFFFu;
-  }
+__global__ void __launch_bounds__(256) im2col_s8_kernel(const ConvArgs a, uint32_t kpad, uint32_t run_pitch,
+                                                       uint32_t offset, uint32_t span_bytes, uint32_t span_pitch,
+                                                       int8_t* __restrict__ dst) {
+  extern __shared__ uint32_t im2col_smem[];                   // [KH][span_pitch / 4] words
+  uint8_t* rows = reinterpret_cast<uint8_t*>(im2col_smem);
   const uint32_t strips = (a.OW + kIm2colPix - 1) / kIm2colPix;
   const uint32_t strip = blockIdx.x % strips;
   const uint32_t oy = (blockIdx.x / strips) % a.OH;
@@ -274,29 +272,48 @@ __global__ void __launch_bounds__(256) im2col_s8_kernel(const ConvArgs a, uint32
   const int ix0 = (int)(ox0 * a.stride) - (int)a.pad;         // leftmost input column of the strip
   const int iy0 = (int)(oy * a.stride) - (int)a.pad;
   const uint8_t* x = (const uint8_t*)a.x;
+  const uint8_t flip = (uint8_t)offset;                       // 0 or 0x80: v - 128 == v ^ 0x80 as a byte
   const uint8_t fill = (uint8_t)(0u - offset);
-  for (uint32_t t = threadIdx.x; t < a.KH * span_bytes; t += blockDim.x) {
-    const uint32_t kh = t / span_bytes, b = t % span_bytes;
-    const int iy = iy0 + (int)kh, ix = ix0 + (int)(b / a.C);
-    uint8_t v = fill;
-    if (iy >= 0 && iy < (int)a.H && ix >= 0 && ix < (int)a.W)
-      v = (uint8_t)(x[(((size_t)n * a.H + iy) * a.W + ix) * a.C + b % a.C] - offset);
-    rows[t] = v;
+  // bytes [lo_b, hi_b) of a span lie inside the image row
+  const int lo_b = ix0 < 0 ? -ix0 * (int)a.C : 0;
+  const int hi_b = min((int)span_bytes, ((int)a.W - ix0) * (int)a.C);
+  for (uint32_t kh = threadIdx.x >> 6; kh < a.KH; kh += 4u) {
+    const int iy = iy0 + (int)kh;
+    const bool row_in = iy >= 0 && iy < (int)a.H;
+    const uint8_t* src = x + (((size_t)n * a.H + (row_in ? iy : 0)) * a.W) * a.C + (ptrdiff_t)ix0 * (int)a.C;
+    for (uint32_t b = threadIdx.x & 63u; b < span_pitch; b += 64u) {
+      uint8_t v = fill;
+      if (row_in && (int)b >= lo_b && (int)b < hi_b) v = (uint8_t)(src[b] ^ flip);
+      rows[kh * span_pitch + b] = v;
+    }
   }
   __syncthreads();
-  const uint32_t chunks = kpad / 16u;
   const size_t m0 = ((size_t)n * a.OH + oy) * a.OW + ox0;
-  for (uint32_t t = threadIdx.x; t < npix * chunks; t += blockDim.x) {
-    const uint32_t px = t / chunks, ch = t % chunks;
-    const uint32_t base = px * a.stride * a.C;
-    uint32_t w[4] = {0, 0, 0, 0};
-#pragma unroll
-    for (int j = 0; j < 16; ++j) {
-      const uint32_t e = ktab[ch * 16u + j];
-      const uint32_t v = e == 0xFFFFFFFFu ? 0u : rows[(e & 0xFFu) * span_bytes + base + (e >> 8)];
-      w[j >> 2] |= v << (8 * (j & 3));
+  const uint32_t run = a.KW * a.C;                            // bytes of one filter row
+  const uint32_t words = run_pitch / 4u;
+  const uint32_t tail0 = a.KH * run_pitch;                    // zero bytes [tail0, kpad)
+  const uint32_t items = a.KH + (kpad > tail0 ? 1u : 0u);
+  for (uint32_t t = threadIdx.x; t < npix * items; t += blockDim.x) {
+    const uint32_t px = t / items, kh = t - px * items;
+    int8_t* out = dst + (m0 + px) * kpad + kh * run_pitch;
+    if (kh == a.KH) {
+      for (uint32_t b = 0; b < kpad - tail0; b += 8u) *reinterpret_cast<uint2*>(out + b) = make_uint2(0u, 0u);
+      continue;
     }
-    *reinterpret_cast<uint4*>(dst + (m0 + px) * kpad + ch * 16u) = make_uint4(w[0], w[1], w[2], w[3]);
+    const uint32_t o = px * a.stride * a.C;                   // byte offset of the run in the staged span
+    const uint32_t* wsrc = im2col_smem + kh * (span_pitch / 4u) + (o >> 2);
+    const uint32_t sh = (o & 3u) * 8u;
+    uint32_t lo = wsrc[0];
+    for (uint32_t w = 0; w < words; w += 2u) {
+      const uint32_t mid = wsrc[w + 1], hi = wsrc[w + 2];
+      uint32_t v0 = __funnelshift_r(lo, mid, sh), v1 = __funnelshift_r(mid, hi, sh);
+      // bytes at or beyond the run are K padding: zero
+      const uint32_t b0 = w * 4u;
+      if (b0 + 4u > run) v0 = b0 >= run ? 0u : (v0 & (0xFFFFFFFFu >> (8u * (b0 + 4u - run))));
+      if (b0 + 8u > run) v1 = b0 + 4u >= run ? 0u : (v1 & (0xFFFFFFFFu >> (8u * (b0 + 8u - run))));
+      *reinterpret_cast<uint2*>(out + b0) = make_uint2(v0, v1);
+      lo = hi;
+    }
   }
 }
 
@@ -485,14 +502,18 @@ cudaError_t launch_shift_add(const ConvArgs& a, const WintTable& wt, cudaStream_
   return cudaGetLastError();
 }
 
-cudaError_t launch_im2col_s8(const ConvArgs& a, uint32_t kpad, uint32_t offset, int8_t* dst,
+cudaError_t launch_im2col_s8(const ConvArgs& a, uint32_t kpad, uint32_t run_pitch, uint32_t offset, int8_t* dst,
                              cudaStream_t s) {
   const uint32_t strips = (a.OW + kIm2colPix - 1) / kIm2colPix;
   const uint32_t span_bytes = ((kIm2colPix - 1) * a.stride + a.KW) * a.C;
-  const size_t smem = kpad * sizeof(uint32_t) + (size_t)a.KH * span_bytes;
-  if (smem > 48 * 1024 || (uint64_t)a.N * a.OH * strips >= (1ull << 31) || a.KW * a.C >= (1u << 24))
+  // a run may be read up to run_pitch + 7 bytes past its start (whole words, two at a time)
+  const uint32_t span_pitch = round_up((kIm2colPix - 1) * a.stride * a.C + run_pitch + 12u, 4u);
+  const size_t smem = (size_t)a.KH * span_pitch;
+  if (smem > 48 * 1024 || (uint64_t)a.N * a.OH * strips >= (1ull << 31) || run_pitch % 8u || kpad % 16u ||
+      (offset != 0u && offset != 128u) || a.KH * run_pitch > kpad)
     return cudaErrorInvalidValue;
-  im2col_s8_kernel<<<a.N * a.OH * strips, 256, smem, s>>>(a, kpad, offset, span_bytes, dst); note_launch();
+  im2col_s8_kernel<<<a.N * a.OH * strips, 256, smem, s>>>(a, kpad, run_pitch, offset, span_bytes, span_pitch, dst);
+  note_launch();
   return cudaGetLastError();
 }
 

@@ -22,22 +22,46 @@ constexpr int kThreads = 256;
 constexpr int kStage = 2048;  // weights staged in shared memory per block
 
 // Philox4x32-10 (Salmon et al., SC'11): ten rounds of two 32x32->64 multiplies and
-// xors; the key advances by the two Weyl constants after every round.
+// xors; the key advances by the two Weyl constants after every round.  The ten round keys
+// depend on the seed only, so a thread computes them once (PhiloxKeys) and reuses them for
+// every weight.
+struct PhiloxKeys {
+  uint32_t k0[10], k1[10];
+  __device__ __forceinline__ PhiloxKeys(uint32_t seed_lo, uint32_t seed_hi) {
+#pragma unroll
+    for (int r = 0; r < 10; ++r) {
+      k0[r] = seed_lo + (uint32_t)r * 0x9E3779B9u;
+      k1[r] = seed_hi + (uint32_t)r * 0xBB67AE85u;
+    }
+  }
+};
+
 __device__ __forceinline__ void philox4x32_10(uint32_t c0, uint32_t c1, uint32_t c2, uint32_t c3,
-                                              uint32_t k0, uint32_t k1, uint32_t (&out)[4]) {
+                                              const PhiloxKeys& key, uint32_t (&out)[4]) {
   const uint32_t M0 = 0xD2511F53u, M1 = 0xCD9E8D57u;
 #pragma unroll
   for (int r = 0; r < 10; ++r) {
-    uint32_t hi0 = __umulhi(M0, c0), lo0 = M0 * c0;
-    uint32_t hi1 = __umulhi(M1, c2), lo1 = M1 * c2;
-    uint32_t n0 = hi1 ^ c1 ^ k0;
-    uint32_t n2 = hi0 ^ c3 ^ k1;
+    // one widening multiply gives both halves
+    const unsigned long long p0 = (unsigned long long)M0 * c0, p1 = (unsigned long long)M1 * c2;
+    const uint32_t hi0 = (uint32_t)(p0 >> 32), lo0 = (uint32_t)p0;
+    const uint32_t hi1 = (uint32_t)(p1 >> 32), lo1 = (uint32_t)p1;
+    const uint32_t n0 = hi1 ^ c1 ^ key.k0[r];
+    const uint32_t n2 = hi0 ^ c3 ^ key.k1[r];
     c0 = n0; c1 = lo1; c2 = n2; c3 = lo0;
-    k0 += 0x9E3779B9u;
-    k1 += 0xBB67AE85u;
   }
   out[0] = c0; out[1] = c1; out[2] = c2; out[3] = c3;
 }
+
+__device__ __forceinline__ void philox4x32_10(uint32_t c0, uint32_t c1, uint32_t c2, uint32_t c3,
+                                              uint32_t k0, uint32_t k1, uint32_t (&out)[4]) {
+  const PhiloxKeys key(k0, k1);
+  philox4x32_10(c0, c1, c2, c3, key, out);
+}
+
+// Division of a small number (< 2^16) by a block-uniform divisor (< 2^16): q = umulhi(t, magic)
+// with magic = floor((2^32 - 1) / d) + 1 is exact in that range.
+__device__ __forceinline__ uint32_t small_div_magic(uint32_t d) { return 0xFFFFFFFFu / d + 1u; }
+__device__ __forceinline__ uint32_t small_div(uint32_t t, uint32_t magic) { return magic ? __umulhi(t, magic) : t; }   // magic wraps to 0 for d = 1
 
 // Largest biased exponent of each exponent group; flags Inf/NaN.
 // norm == 1: one block per output channel.  norm == 0: grid-stride over the layer.
@@ -96,6 +120,11 @@ struct SampleParams {
 
 __device__ __forceinline__ void sample_block(const SampleParams& p, uint32_t block, uint32_t seed_lo,
                                              uint32_t seed_hi, float* stage) {
+  // the parameters may sit in global memory (batched launch): read the scalars once
+  const uint32_t norm = p.norm, span = p.span, level_mask = p.level_mask, max_level = p.max_level;
+  const uint32_t layer_id = p.layer_id, KHKW = p.KHKW, Cg = p.Cg, cpad = p.cpad, kpad = p.kpad;
+  const uint32_t packed_kw = p.packed_kw, run_pitch = p.run_pitch, has_planes = p.has_planes;
+  const PhiloxKeys keys(seed_lo, seed_hi);
   const uint32_t row_block = block / p.ch_chunks;
   const uint32_t chunk = block % p.ch_chunks;
   const uint32_t o0 = row_block * p.rows_per_block;
@@ -105,69 +134,77 @@ __device__ __forceinline__ void sample_block(const SampleParams& p, uint32_t blo
   const uint32_t per_row = cc * p.KHKW;     // canonical elements of one row in this block
   const uint32_t count = rows * per_row;
 
+  // count <= kStage = 2048 and the divisors are block-uniform: divisions by multiply-high
+  const uint32_t per_row_magic = small_div_magic(per_row), cc_magic = small_div_magic(cc);
   // stage the canonical (channel-major) slice with coalesced loads
   for (uint32_t t = threadIdx.x; t < count; t += blockDim.x) {
-    uint32_t r = t / per_row, rem = t % per_row;
+    const uint32_t r = small_div(t, per_row_magic), rem = t - r * per_row;
     stage[t] = p.w[(size_t)(o0 + r) * p.d + (size_t)c0 * p.KHKW + rem];
   }
   __syncthreads();
 
   // walk the slice in output order (row, tap, channel) so that stores coalesce
   for (uint32_t t = threadIdx.x; t < count; t += blockDim.x) {
-    const uint32_t r = t / per_row, rem = t % per_row;
-    const uint32_t tap = rem / cc, cl = rem % cc;
+    const uint32_t r = small_div(t, per_row_magic), rem = t - r * per_row;
+    const uint32_t tap = small_div(rem, cc_magic), cl = rem - tap * cc;
     const uint32_t o = o0 + r, ci = c0 + cl;
     const uint32_t u = __float_as_uint(stage[r * per_row + cl * p.KHKW + tap]);
     const uint64_t index = (uint64_t)o * p.d + (uint64_t)ci * p.KHKW + tap;  // canonical
 
     const uint32_t E = (u >> 23) & 0xFFu;
     const uint32_t m = u & 0x7FFFFFu;
-    const uint32_t Emax = p.e_max[p.norm ? o : 0];
+    const uint32_t Emax = p.e_max[norm ? o : 0];
     // biased exponents throughout: e - e_base = E - (Emax - span)
-    const int ebase_biased = (int)Emax - (int)p.span;
+    const int ebase_biased = (int)Emax - (int)span;
     if (tap == 0 && ci == 0) p.e_base[o] = Emax ? ebase_biased - 127 : 0;
     const bool live = (E != 0u) && (E != 255u) && ((int)E >= ebase_biased);
     const uint32_t sh = live ? (uint32_t)((int)E - ebase_biased) : 0u;
     const bool neg = (u >> 31) != 0u;
 
-    // c_k for every level, packed 7 bits per level
-    unsigned long long packed = 0ull;
+    // c_k for every level k = 2^l: level l is complete after draw 2^l, i.e. levels 0..2 after the
+    // first Philox call, level l >= 2 after call 2^(l-2)
+    uint32_t cnt[kMaxLevels] = {0u, 0u, 0u, 0u, 0u, 0u, 0u};
     if (live && m != 0u) {
       const uint32_t T = m << 9;
-      const uint32_t kmax = 1u << p.max_level;
-      uint32_t c = 0, j = 0;
-      for (uint32_t q = 0; q * 4u < kmax; ++q) {
-        uint32_t rnd[4];
-        philox4x32_10(q, p.layer_id, (uint32_t)index, (uint32_t)(index >> 32), seed_lo, seed_hi, rnd);
+      const uint32_t i_lo = (uint32_t)index, i_hi = (uint32_t)(index >> 32);
+      uint32_t rnd[4];
+      philox4x32_10(0u, layer_id, i_lo, i_hi, keys, rnd);
+      cnt[0] = rnd[0] < T ? 1u : 0u;
+      cnt[1] = cnt[0] + (rnd[1] < T ? 1u : 0u);
+      uint32_t c = cnt[1] + (rnd[2] < T ? 1u : 0u) + (rnd[3] < T ? 1u : 0u);
+      cnt[2] = c;
 #pragma unroll
-        for (int v = 0; v < 4; ++v) {
-          if (j < kmax) {
-            c += (rnd[v] < T) ? 1u : 0u;
-            ++j;
-            if ((j & (j - 1u)) == 0u) packed |= (unsigned long long)c << (7 * (31 - __clz(j)));
+      for (int l = 3; l < kMaxLevels; ++l) {
+        if ((uint32_t)l <= max_level) {
+          for (uint32_t q = 1u << (l - 3); q < (1u << (l - 2)); ++q) {
+            philox4x32_10(q, layer_id, i_lo, i_hi, keys, rnd);
+            c += (rnd[0] < T ? 1u : 0u) + (rnd[1] < T ? 1u : 0u) + (rnd[2] < T ? 1u : 0u) + (rnd[3] < T ? 1u : 0u);
           }
+          cnt[l] = c;
         }
       }
     }
 
-    const size_t wpos = ((size_t)o * p.KHKW + tap) * p.Cg + ci;
-    uint32_t kcol = tap * p.cpad + ci;
-    if (p.packed_kw) {
-      const uint32_t kh = tap / p.packed_kw;
-      kcol = kh * p.run_pitch + (tap - kh * p.packed_kw) * p.Cg + ci;
+    const size_t wpos = ((size_t)o * KHKW + tap) * Cg + ci;
+    uint32_t kcol = tap * cpad + ci;
+    if (packed_kw) {
+      const uint32_t kh = tap / packed_kw;
+      kcol = kh * run_pitch + (tap - kh * packed_kw) * Cg + ci;
     }
     const uint32_t jt = o / kTileN, on = o % kTileN;
-    for (uint32_t l = 0; l <= p.max_level; ++l) {
-      if (!((p.level_mask >> l) & 1u)) continue;
-      const uint32_t c = (uint32_t)(packed >> (7 * l)) & 0x7Fu;
-      const uint32_t mag = live ? (((1u << l) + c) << sh) : 0u;
+    const size_t plane_stride = (size_t)kTileN * kpad;           // one plane of one channel tile
+    const size_t in_plane = (size_t)on * kpad + kcol;
+#pragma unroll
+    for (int l = 0; l < kMaxLevels; ++l) {
+      if (!((level_mask >> l) & 1u)) continue;
+      const uint32_t mag = live ? (((1u << l) + cnt[l]) << sh) : 0u;
       p.wint[l][wpos] = neg ? -(int32_t)mag : (int32_t)mag;
-      if (p.has_planes) {
+      if (has_planes) {
         const int P = p.planes_count[l];
-        for (int pl = 0; pl < P; ++pl) {
-          int digit = (int)((mag >> (kDigitBits * pl)) & 0x7Fu);
-          p.planes[l][(((size_t)jt * P + pl) * kTileN + on) * p.kpad + kcol] =
-              (int8_t)(neg ? -digit : digit);
+        int8_t* dstp = p.planes[l] + (size_t)jt * P * plane_stride + in_plane;
+        for (int pl = 0; pl < P; ++pl, dstp += plane_stride) {
+          const int digit = (int)((mag >> (kDigitBits * pl)) & 0x7Fu);
+          *dstp = (int8_t)(neg ? -digit : digit);
         }
       }
     }

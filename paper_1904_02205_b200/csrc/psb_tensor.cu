@@ -10,11 +10,14 @@
 // in 64-bit integers, which makes the result exact.
 //
 // Structure of one CTA (one per SM, persistent over tiles):
-//   warps 0-2 producers (one thread each, taking the stages in turns): TMA loads of the activation tile (im2col mode for
+//   warps 0-1 producers (one thread each, taking the stages in turns): TMA loads of the activation tile (im2col mode for
 //            filters with taps, stride or padding; plain 2-D tiles otherwise) and
 //            of the digit-plane tile into a ring of shared-memory stages
-//   warp 3   allocates TMEM; one thread issues the MMAs and commits them to the
-//            stage-free and accumulator-ready barriers
+//   warps 2-3 MMA issuers (one thread each; warp 3 also allocates TMEM): the pipeline stages
+//            alternate between them.  The tensor pipe takes only a few MMAs ahead of the one it
+//            executes, so whatever else an issuing thread does (barrier waits, commits, tile
+//            bookkeeping: a few hundred clocks per stage) would leave the pipe idle; with two
+//            issuers one thread's bookkeeping runs under the other's MMAs
 //   warps 4-19 epilogue: TMEM -> registers, recombine planes, dequantise, bias,
 //            shortcut, ReLU, re-quantise, vectorised stores; overlaps the next
 //            tile's MMAs through two TMEM accumulator buffers
@@ -33,9 +36,11 @@ namespace psb {
 namespace {
 
 constexpr int kTileM = 128;
-constexpr int kProducerWarps = 3;    // one issuing thread each: their barrier waits overlap
-constexpr int kMmaWarp = kProducerWarps;
-constexpr int kFirstEpilogueWarp = kMmaWarp + 1;   // a multiple of 4: warp & 3 = TMEM lane quarter
+constexpr int kProducerWarps = 2;    // one issuing thread each: their barrier waits overlap
+constexpr int kMmaWarp0 = kProducerWarps;          // issues the even passes
+constexpr int kMmaWarp1 = kMmaWarp0 + 1;           // issues the odd passes; owns the TMEM allocation
+constexpr int kFirstEpilogueWarp = kMmaWarp1 + 1;  // a multiple of 4: warp & 3 = TMEM lane quarter
+constexpr int kPlaneBars = 4;        // resident digit planes arrive in this many parts, each with its barrier
 constexpr int kEpilogueWarps = 16;
 constexpr int kThreadsTensor = 32 * (kFirstEpilogueWarp + kEpilogueWarps);
 constexpr uint32_t kTmemCols = 512;
@@ -242,7 +247,8 @@ struct SharedCtl {
   unsigned long long empty[kMaxStages];
   unsigned long long acc_full[2];
   unsigned long long acc_empty[2];
-  unsigned long long planes_full;
+  unsigned long long planes_full[kPlaneBars];
+  unsigned long long started[2];        // per accumulator buffer: the zeroing MMA of the pass has been issued
   uint32_t tmem_base;
   volatile uint32_t abort;
   float2 scb[kEpilogueWarps][16];       // per epilogue warp: (scale * 2^(e_base - log2 k), bias)
@@ -522,6 +528,90 @@ __device__ __noinline__ bool epilogue_uniform(const TensorParams& p, SharedCtl* 
   return false;
 }
 
+// The MMA issuing role, one thread of warp kMmaWarp0 (mine = 0) and one of kMmaWarp1 (mine = 1).
+// Both walk the same sequence of passes and ring stages; stage uses are numbered through the
+// whole kernel and the number's parity selects the thread.  The thread that owns the first
+// stage of a pass waits for the accumulator buffer and issues the zeroing MMA; the other one
+// joins the pass after that (`started`).  Integer accumulation is exact, so the order in
+// which the two threads' MMAs reach the accumulator is immaterial.  A parity wait on a stage
+// barrier is meaningful while the waiter is less than two uses of that stage ahead of it: a
+// thread has seen use n - 2 arrive before it waits for use n, and with two or more ring
+// stages use n - stages is not later than that.  Kept out of line and fed from local copies of
+// the parameters so that its loop state lives in registers: the pipe idles for every clock this
+// thread spends between two MMAs beyond what the other thread covers.  Returns true on a timeout.
+template <int BK>
+__device__ __noinline__ bool mma_role(const TensorParams& p, SharedCtl* ctl, uint32_t tmem_base, uint32_t ring_addr,
+                                      uint32_t planes_addr, uint32_t stage_bytes, uint32_t sub_bytes,
+                                      uint32_t k_iters, uint32_t mine) {
+  volatile uint32_t* abort = &ctl->abort;
+  const uint32_t group = p.group, stages = p.stages, resident = p.resident, stage_bytes_a = p.stage_bytes_a;
+  const uint32_t level_mask = p.a.level_mask;
+  const uint32_t n_groups = (k_iters + group - 1) / group;
+  const uint32_t full0 = smem_u32(&ctl->full[0]), empty0 = smem_u32(&ctl->empty[0]);
+  const uint32_t acc_full0 = smem_u32(&ctl->acc_full[0]), acc_empty0 = smem_u32(&ctl->acc_empty[0]);
+  const uint32_t started0 = smem_u32(&ctl->started[0]);
+  // resident digit planes: K blocks below planes_upto are known to have landed
+  const uint32_t plane_part = (k_iters + kPlaneBars - 1) / kPlaneBars;
+  uint32_t planes_ready = 0, planes_upto = resident ? 0u : 0xFFFFFFFFu;
+  uint32_t s = 0, ph = 0, pass = 0, use = 0;
+  TileIter ti;
+  for (ti.init(p); ti.valid(); ti.next()) {
+    const uint32_t levels = tile_levels(p, ti.m_tile) & level_mask;
+    for (uint32_t todo = levels & 0x7Fu; todo; todo &= todo - 1u) {
+      const uint32_t l = (uint32_t)__ffs((int)todo) - 1u;
+      const uint32_t P = p.planes[l];
+      const uint32_t buf = pass & 1u, aph = (pass >> 1) & 1u;
+      // instruction descriptor: s32 accumulators, s8 x s8, both K-major, M = 128, N = P * 64
+      const uint32_t idesc = (2u << 4) | (1u << 7) | (1u << 10) | (((P * kTileN) >> 3) << 17) |
+                             ((kTileM >> 4) << 24);
+      const uint32_t d_tmem = tmem_base + buf * kTmemBufStride;
+      const uint32_t blk = P * kTileN * BK;
+      bool joined = (use & 1u) == mine;
+      if (joined) {
+        if (!mbar_wait(acc_empty0 + 8u * buf, aph ^ 1u, abort)) return true;
+        tc_fence_after();
+      }
+      uint32_t b_res = planes_addr, g = 0;
+      for (uint32_t it = 0; it < k_iters; ++g, ++use) {
+        const uint32_t cnt = min(group, k_iters - it);
+        if ((use & 1u) == mine) {
+          if (!joined) {
+            if (!mbar_wait(started0 + 8u * buf, aph, abort)) return true;
+            joined = true;
+          }
+          if (!mbar_wait(full0 + 8u * s, ph, abort)) return true;
+          while (it + cnt > planes_upto) {
+            if (!mbar_wait(smem_u32(&ctl->planes_full[planes_ready]), 0u, abort)) return true;
+            ++planes_ready;
+            planes_upto = planes_ready == (uint32_t)kPlaneBars ? 0xFFFFFFFFu : planes_upto + plane_part;
+          }
+          tc_fence_after();
+          uint32_t a_addr = ring_addr + s * stage_bytes, b_blk = b_res;
+          for (uint32_t j = 0; j < cnt; ++j, a_addr += sub_bytes, b_blk += blk) {
+            const uint32_t b_addr = resident ? b_blk : a_addr + stage_bytes_a;
+#pragma unroll
+            for (int ks = 0; ks < BK / 32; ++ks)
+              tc_mma_i8(d_tmem, smem_desc(a_addr + ks * 32, BK), smem_desc(b_addr + ks * 32, BK), idesc,
+                        (it | j | ks) != 0 ? 1u : 0u);
+          }
+          if (it == 0 && n_groups > 1u) {
+            tc_fence_before();
+            mbar_arrive(started0 + 8u * buf);
+          }
+          tc_commit(empty0 + 8u * s);
+          // this thread's last stage of the pass: the last or the last but one
+          if (g + 2u >= n_groups) tc_commit(acc_full0 + 8u * buf);
+        }
+        b_res += cnt * blk;
+        it += cnt;
+        if (++s == stages) { s = 0; ph ^= 1u; }
+      }
+      ++pass;
+    }
+  }
+  return false;
+}
+
 template <int BK>
 __global__ void __launch_bounds__(kThreadsTensor, 1)
 psb_mma_kernel(const __grid_constant__ TmapSet maps, const __grid_constant__ TensorParams p) {
@@ -545,14 +635,29 @@ psb_mma_kernel(const __grid_constant__ TmapSet maps, const __grid_constant__ Ten
       mbar_init(smem_u32(&ctl->empty[s]), 1);
     }
     for (int b = 0; b < 2; ++b) {
-      mbar_init(smem_u32(&ctl->acc_full[b]), 1);
+      // both issuing threads commit to it when a pass has more than one stage
+      mbar_init(smem_u32(&ctl->acc_full[b]), (k_iters + p.group - 1) / p.group > 1u ? 2u : 1u);
       mbar_init(smem_u32(&ctl->acc_empty[b]), kEpilogueWarps);
     }
-    mbar_init(smem_u32(&ctl->planes_full), 1);
+    {  // part b of the resident planes holds K blocks [b * part, (b + 1) * part): one arrival per block
+      const uint32_t part = (k_iters + kPlaneBars - 1) / kPlaneBars;
+      for (uint32_t b = 0; b < (uint32_t)kPlaneBars; ++b) {
+        const uint32_t lo = b * part, hi = min(lo + part, k_iters);
+        mbar_init(smem_u32(&ctl->planes_full[b]), hi > lo ? hi - lo : 1u);
+      }
+    }
+    for (int b = 0; b < 2; ++b) mbar_init(smem_u32(&ctl->started[b]), 1);
     ctl->abort = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
-  if (warp == kMmaWarp) {
+  if (threadIdx.x == 32) {
+    // descriptor fetches of the first copies would otherwise sit on the critical path of the first tile
+    asm volatile("prefetch.tensormap [%0];" ::"l"(&maps.a) : "memory");
+    for (int l = 0; l < kMaxLevels; ++l)
+      if (p.planes[l] && ((p.a.level_mask >> l) & 1u))
+        asm volatile("prefetch.tensormap [%0];" ::"l"(&maps.b[l]) : "memory");
+  }
+  if (warp == kMmaWarp1) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(
                      smem_u32(&ctl->tmem_base)),
                  "r"(kTmemCols)
@@ -575,136 +680,74 @@ psb_mma_kernel(const __grid_constant__ TmapSet maps, const __grid_constant__ Ten
 
   if (warp < (uint32_t)kProducerWarps) {
     // ----------------------------------------------------------- producers
-    // One thread per producer warp.  Every barrier round trip costs its thread a few hundred
-    // cycles of latency, which caps a single thread at about one TMA load per 300 cycles; the
-    // producer threads therefore take the pipeline stages in turns (all of them walk the same
-    // sequence of stages with incremental index arithmetic, each issues every third one).
-    if (lane == 0) {
-      if (p.resident && warp == 0) {
-        // the digit planes of this CTA's channel tile, all K blocks, once
-        const uint32_t l = p.a.uniform_log2k, P = p.planes[l];
-        const uint32_t o_tile = blockIdx.x / p.ctas_per_otile;
-        const uint32_t bar = smem_u32(&ctl->planes_full);
-        const uint32_t blk = P * kTileN * BK;
-        mbar_expect_tx(bar, k_iters * blk);
-        uint32_t kcol = 0, cb = 0;
-        for (uint32_t it = 0; it < k_iters; ++it) {
-          tma_load_2d(smem_u32(smem) + it * blk, &maps.b[l], bar, (int)(kcol + cb * BK),
-                      (int)(o_tile * P * kTileN));
-          if (++cb == p.n_cb) { cb = 0; kcol += p.cpad; }
-        }
-      }
-      uint32_t s = 0, ph = 0;   // ring position and phase of the current stage use
-      uint32_t turn = 0;        // whose turn it is among the producer threads
-      TileIter ti;
-      for (ti.init(p); ti.valid() && !failed; ti.next()) {
-        const uint32_t m_tile = ti.m_tile, o_tile = ti.o_tile;
-        const uint32_t m0 = m_tile * kTileM;
-        const uint32_t levels = tile_levels(p, ti.m_tile) & p.a.level_mask;
-        // image coordinates of the tile's first row: divisions, so only the thread that is about to
-        // issue a copy of this tile computes them
-        uint32_t n0 = 0;
-        int h0 = 0, w0 = 0;
-        bool have_coords = !p.im2col;
-        // one pass per level present in the tile (levels that were not sampled are flagged by the
-        // epilogue and skipped by every role)
-        for (uint32_t todo = levels & 0x7Fu; todo && !failed; todo &= todo - 1u) {
-          const uint32_t l = (uint32_t)__ffs((int)todo) - 1u;
-          const uint32_t P = p.planes[l];
-          const uint32_t bytes = p.stage_bytes_a + (p.resident ? 0u : P * kTileN * BK);
-          const int b_row = (int)(o_tile * P * kTileN);
-          uint32_t kw = 0, kh = 0, cb = 0, kcol = 0;     // tap (kh, kw), channel block, plane column
-          for (uint32_t it = 0; it < k_iters;) {
-            const uint32_t cnt = min(p.group, k_iters - it);
-            const bool mine = turn == warp;
-            if (mine) {
-              if (!have_coords) {
-                const uint32_t ohow = p.a.OH * p.a.OW;
-                n0 = m0 / ohow;
-                const uint32_t rem = m0 - n0 * ohow, oy = rem / p.a.OW;
-                h0 = (int)(oy * p.a.stride) - (int)p.a.pad;
-                w0 = (int)((rem - oy * p.a.OW) * p.a.stride) - (int)p.a.pad;
-                have_coords = true;
-              }
-              if (!mbar_wait(smem_u32(&ctl->empty[s]), ph ^ 1u, abort)) { failed = true; break; }
-              mbar_expect_tx(smem_u32(&ctl->full[s]), bytes * cnt);
+    // A copy instruction holds its thread for a few hundred clocks, whatever its size, while the
+    // copy engine takes several at a time: the K blocks of a stage are therefore issued by as
+    // many lanes of the warp in one go (lane j copies block j), after lane 0 has waited for the
+    // stage and posted the byte count; and the producer warps take the stages in turns (all of
+    // them walk the same sequence of stages, each issues every second one).
+    uint32_t s = 0, ph = 0;   // ring position and phase of the current stage use
+    uint32_t turn = 0;        // whose turn it is among the producer warps
+    const uint32_t ring_addr = smem_u32(ring);
+    TileIter ti;
+    for (ti.init(p); ti.valid() && !failed; ti.next()) {
+      const uint32_t m_tile = ti.m_tile, o_tile = ti.o_tile;
+      const uint32_t m0 = m_tile * kTileM;
+      const uint32_t levels = tile_levels(p, ti.m_tile) & p.a.level_mask;
+      // image coordinates of the tile's first row: divisions, so only the warp that is about to
+      // issue a copy of this tile computes them
+      uint32_t n0 = 0;
+      int h0 = 0, w0 = 0;
+      bool have_coords = !p.im2col;
+      // one pass per level present in the tile (levels that were not sampled are flagged by the
+      // epilogue and skipped by every role)
+      for (uint32_t todo = levels & 0x7Fu; todo && !failed; todo &= todo - 1u) {
+        const uint32_t l = (uint32_t)__ffs((int)todo) - 1u;
+        const uint32_t P = p.planes[l];
+        const uint32_t bytes = p.stage_bytes_a + (p.resident ? 0u : P * kTileN * BK);
+        const int b_row = (int)(o_tile * P * kTileN);
+        for (uint32_t it = 0; it < k_iters;) {
+          const uint32_t cnt = min(p.group, k_iters - it);
+          if (turn == warp) {
+            if (!have_coords) {
+              const uint32_t ohow = p.a.OH * p.a.OW;
+              n0 = m0 / ohow;
+              const uint32_t rem = m0 - n0 * ohow, oy = rem / p.a.OW;
+              h0 = (int)(oy * p.a.stride) - (int)p.a.pad;
+              w0 = (int)((rem - oy * p.a.OW) * p.a.stride) - (int)p.a.pad;
+              have_coords = true;
             }
             const uint32_t bar = smem_u32(&ctl->full[s]);
-            uint32_t dst = smem_u32(ring) + s * stage_bytes;
-            for (uint32_t j = 0; j < cnt; ++j, dst += sub_bytes) {
-              if (mine) {
-                if (p.im2col)
-                  tma_load_im2col_4d(dst, &maps.a, bar, (int)(cb * BK), w0, h0, (int)n0, (uint16_t)kw,
-                                     (uint16_t)kh);
-                else
-                  tma_load_2d(dst, &maps.a, bar, (int)(cb * BK), (int)m0);
-                if (!p.resident)
-                  tma_load_2d(dst + p.stage_bytes_a, &maps.b[l], bar, (int)(kcol + cb * BK), b_row);
-              }
-              if (++cb == p.n_cb) {
-                cb = 0;
-                kcol += p.cpad;
-                if (++kw == p.a.KW) { kw = 0; ++kh; }
-              }
+            bool ok = true;
+            if (lane == 0) {
+              ok = mbar_wait(smem_u32(&ctl->empty[s]), ph ^ 1u, abort);
+              if (ok) mbar_expect_tx(bar, bytes * cnt);
             }
-            it += cnt;
-            if (++s == p.stages) { s = 0; ph ^= 1u; }
-            if (++turn == (uint32_t)kProducerWarps) turn = 0;
+            if (!__shfl_sync(0xFFFFFFFFu, ok ? 1 : 0, 0)) { failed = true; break; }
+            if (lane < cnt) {
+              // K block it + lane: tap (kh, kw), channel block cb, column kcol of the plane matrix
+              const uint32_t kb = it + lane;
+              const uint32_t tap = kb / p.n_cb, cb = kb - tap * p.n_cb;
+              const uint32_t kh = tap / p.a.KW, kw = tap - kh * p.a.KW;
+              const uint32_t dst = ring_addr + s * stage_bytes + lane * sub_bytes;
+              if (p.im2col)
+                tma_load_im2col_4d(dst, &maps.a, bar, (int)(cb * BK), w0, h0, (int)n0, (uint16_t)kw, (uint16_t)kh);
+              else
+                tma_load_2d(dst, &maps.a, bar, (int)(cb * BK), (int)m0);
+              if (!p.resident)
+                tma_load_2d(dst + p.stage_bytes_a, &maps.b[l], bar, (int)(tap * p.cpad + cb * BK), b_row);
+            }
           }
+          it += cnt;
+          if (++s == p.stages) { s = 0; ph ^= 1u; }
+          if (++turn == (uint32_t)kProducerWarps) turn = 0;
         }
       }
     }
-    failed = __shfl_sync(0xFFFFFFFFu, failed ? 1 : 0, 0) != 0;
-  } else if (warp == (uint32_t)kMmaWarp) {
+  } else if (warp == (uint32_t)kMmaWarp0 || warp == (uint32_t)kMmaWarp1) {
     // ---------------------------------------------------------------- MMA
-    if (lane == 0) {
-      uint32_t s = 0, ph = 0, pass = 0;
-      if (p.resident && !mbar_wait(smem_u32(&ctl->planes_full), 0u, abort)) failed = true;
-      const uint32_t ring_addr = smem_u32(ring), planes_addr = smem_u32(smem);
-      bool next_full = false, acc_ready = false;
-      TileIter ti;
-      for (ti.init(p); !failed && ti.valid(); ti.next()) {
-        const uint32_t levels = tile_levels(p, ti.m_tile) & p.a.level_mask;
-        for (uint32_t todo = levels & 0x7Fu; todo && !failed; todo &= todo - 1u) {
-          const uint32_t l = (uint32_t)__ffs((int)todo) - 1u;
-          const uint32_t P = p.planes[l];
-          const uint32_t buf = pass & 1u, aph = (pass >> 1) & 1u;
-          // instruction descriptor: s32 accumulators, s8 x s8, both K-major, M = 128, N = P * 64
-          const uint32_t idesc = (2u << 4) | (1u << 7) | (1u << 10) | (((P * kTileN) >> 3) << 17) |
-                                 ((kTileM >> 4) << 24);
-          const uint32_t d_tmem = tmem_base + buf * kTmemBufStride;
-          const uint32_t blk = P * kTileN * BK;
-          if (!acc_ready && !mbar_wait(smem_u32(&ctl->acc_empty[buf]), aph ^ 1u, abort)) { failed = true; break; }
-          tc_fence_after();
-          // probe the buffer of the following pass now; the answer is needed only after this pass's MMAs
-          acc_ready = mbar_try_wait(smem_u32(&ctl->acc_empty[buf ^ 1u]), (((pass + 1u) >> 1) & 1u) ^ 1u);
-          uint32_t b_res = planes_addr;
-          for (uint32_t it = 0; it < k_iters;) {
-            const uint32_t cnt = min(p.group, k_iters - it);
-            if (!next_full && !mbar_wait(smem_u32(&ctl->full[s]), ph, abort)) { failed = true; break; }
-            tc_fence_after();
-            // probe the following stage while this one's MMAs are being issued
-            const uint32_t s2 = (s + 1 == p.stages) ? 0u : s + 1;
-            const uint32_t ph2 = (s + 1 == p.stages) ? ph ^ 1u : ph;
-            next_full = mbar_try_wait(smem_u32(&ctl->full[s2]), ph2);
-            uint32_t a_addr = ring_addr + s * stage_bytes;
-            for (uint32_t j = 0; j < cnt; ++j, a_addr += sub_bytes, b_res += blk) {
-              const uint32_t b_addr = p.resident ? b_res : a_addr + p.stage_bytes_a;
-#pragma unroll
-              for (int ks = 0; ks < BK / 32; ++ks)
-                tc_mma_i8(d_tmem, smem_desc(a_addr + ks * 32, BK), smem_desc(b_addr + ks * 32, BK),
-                          idesc, (it | j | ks) != 0 ? 1u : 0u);
-            }
-            tc_commit(smem_u32(&ctl->empty[s]));
-            it += cnt;
-            if (it == k_iters) tc_commit(smem_u32(&ctl->acc_full[buf]));
-            s = s2;
-            ph = ph2;
-          }
-          ++pass;
-        }
-      }
-    }
+    if (lane == 0)
+      failed = mma_role<BK>(p, ctl, tmem_base, smem_u32(ring), smem_u32(smem), stage_bytes, sub_bytes, k_iters,
+                            warp - (uint32_t)kMmaWarp0);
     failed = __shfl_sync(0xFFFFFFFFu, failed ? 1 : 0, 0) != 0;
   } else {
     // ----------------------------------------------------------- epilogue
@@ -725,6 +768,20 @@ psb_mma_kernel(const __grid_constant__ TmapSet maps, const __grid_constant__ Ten
     ec.qmax_f = (float)a.qmax;
     ec.res_sign = a.residual_dtype == PSB_DT_S8 ? 0x80u : 0u;
     const uint32_t P0 = p.planes[a.uniform_log2k < (uint32_t)kMaxLevels ? a.uniform_log2k : 0u];
+    if (p.resident && lane == 0) {
+      // the digit planes of this CTA's channel tile, all K blocks, once: the epilogue warps have
+      // nothing else to do yet, and sixteen threads get the copies under way sooner than one
+      const uint32_t o_tile = blockIdx.x / p.ctas_per_otile;
+      const uint32_t blk = P0 * kTileN * BK;
+      const uint32_t part = (k_iters + kPlaneBars - 1) / kPlaneBars;
+      for (uint32_t it = ew; it < k_iters; it += (uint32_t)kEpilogueWarps) {
+        const uint32_t bar = smem_u32(&ctl->planes_full[it / part]);
+        const uint32_t tap = it / p.n_cb, cb = it - tap * p.n_cb;
+        mbar_expect_tx(bar, blk);
+        tma_load_2d(smem_u32(smem) + it * blk, &maps.b[a.uniform_log2k], bar, (int)(tap * p.cpad + cb * BK),
+                    (int)(o_tile * P0 * kTileN));
+      }
+    }
     if (uniform_epilogue(p)) {
       const uint32_t mode = (p.corr[a.uniform_log2k] != nullptr || P0 == 4u) ? 0u : p.narrow;
 #define PSB_UNI(PV, MV, RV) failed = epilogue_uniform<PV, MV, RV>(p, ctl, tmem_base, ew, lane, ec)
@@ -832,7 +889,7 @@ psb_mma_kernel(const __grid_constant__ TmapSet maps, const __grid_constant__ Ten
   }
   tc_fence_before();
   __syncthreads();
-  if (warp == kMmaWarp) {
+  if (warp == kMmaWarp1) {
     tc_fence_after();
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base),
                  "r"(kTmemCols)
@@ -922,7 +979,7 @@ psb_status launch_tensor(psb_ctx* ctx, const psb_weights* wt, const ConvArgs& a,
   uint32_t group = 8u / (bk / 32u);
   if (group < 1) group = 1;
   if (group > k_iters) group = k_iters;
-  while (group > 1 && avail / ((size_t)group * sub_bytes) < 3) --group;
+  while (group > 1 && avail / ((size_t)group * sub_bytes) < 4) --group;
   {  // balance the groups of one tile: same number of groups, as even as possible
     const uint32_t n_groups = (k_iters + group - 1) / group;
     group = (k_iters + n_groups - 1) / n_groups;
@@ -930,6 +987,12 @@ psb_status launch_tensor(psb_ctx* ctx, const psb_weights* wt, const ConvArgs& a,
   p.group = group;
   uint32_t stages = (uint32_t)(avail / ((size_t)group * sub_bytes));
   if (stages > (uint32_t)kMaxStages) stages = kMaxStages;
+  // An even number of stages: the two producer warps and the two MMA issuing threads each take
+  // every second stage use, so with an even ring each of them keeps to its own slots and every
+  // parity wait on a slot's barriers follows that same thread's previous use of the slot.  (With
+  // an odd ring a thread could wait on a slot whose previous use, the other thread's, has not
+  // happened yet, and a parity wait cannot tell two phases apart.)
+  stages &= ~1u;
   if (stages < 2) return PSB_ERR_UNSUPPORTED;
   p.stages = stages;
   const size_t smem_bytes = (size_t)stages * group * sub_bytes + p.resident_bytes + ctl_bytes;

@@ -299,6 +299,8 @@ psb_status psb_sample_weights(psb_ctx* ctx, const float* w_dev, const psb_wshape
     w->kpad = round_up(shape->kh * w->run_pitch, 16);
     w->o_tiles = (shape->out_ch + kTileN - 1) / kTileN;
     w->bk = tensor_bk(w->packed_k ? w->kpad : shape->in_ch_per_group);
+    w->n_cb = ((w->packed_k ? w->kpad : shape->in_ch_per_group) + w->bk - 1) / w->bk;
+    w->n_kb = w->packed_k ? w->n_cb : shape->kh * shape->kw * w->n_cb;
     bool ok = cudaMalloc(&w->e_base, sizeof(int32_t) * shape->out_ch) == cudaSuccess &&
               cudaMalloc(&w->e_max, sizeof(uint32_t) * shape->out_ch) == cudaSuccess;
     for (uint32_t l = 0; ok && l < (uint32_t)kMaxLevels; ++l) {
@@ -306,7 +308,7 @@ psb_status psb_sample_weights(psb_ctx* ctx, const float* w_dev, const psb_wshape
       ok = cudaMalloc(&w->level[l].wint, sizeof(int32_t) * d64 * shape->out_ch) == cudaSuccess;
       if (ok && w->has_planes) {
         int P = planes_for(cfg.exp_bits, l);
-        size_t bytes = (size_t)w->o_tiles * P * kTileN * w->kpad;
+        size_t bytes = (size_t)w->o_tiles * w->n_kb * P * kTileN * w->bk;
         w->level[l].planes_count = P;
         ok = cudaMalloc(&w->level[l].planes, bytes) == cudaSuccess &&
              cudaMemsetAsync(w->level[l].planes, 0, bytes, s) == cudaSuccess;

@@ -30,9 +30,21 @@ inline int planes_for(uint32_t exp_bits, uint32_t log2k) {
 inline uint32_t tensor_bk(uint32_t cg) { return cg >= 128 ? 128u : (cg >= 64 ? 64u : 32u); }
 inline uint32_t round_up(uint32_t a, uint32_t b) { return (a + b - 1) / b * b; }
 
+// Byte offset, inside one operand tile of P * kTileN rows by bk bytes, of column `kin` of row
+// `row`: rows are bk bytes apart and the 16-byte chunks of a row are permuted by the row number
+// the way the 32/64/128-byte swizzle modes of TMA and of the MMA descriptors do (address bits 4..
+// XOR address bits 7..).  A tile copied as it is to a 1024-byte aligned shared-memory address is
+// a valid K-major swizzled operand.
+__host__ __device__ inline uint32_t plane_offset(uint32_t row, uint32_t kin, uint32_t bk) {
+  const uint32_t lin = row * bk + kin;
+  return lin ^ (((lin >> 7) & (bk / 16u - 1u)) << 4);
+}
+
 struct LevelStore {
   int32_t* wint = nullptr;  // [O][KH][KW][Cg]  signed integer filter, channels innermost
-  int8_t* planes = nullptr; // [O_tiles][P][kTileN][Kpad]  signed 7-bit digits, Kpad = KH*KW*Cpad
+  int8_t* planes = nullptr; // [O_tiles][K blocks][P * kTileN rows][bk bytes]  signed 7-bit digits: every
+                            // (channel tile, K block) operand tile is contiguous and already in the
+                            // swizzled order the MMA reads from shared memory (plane_offset below)
   int planes_count = 0;
   long long* corr128 = nullptr;  // [O] 128 * sum of the filter row, refreshed by the calls that need it
 };
@@ -48,6 +60,8 @@ struct psb_weights {
   uint32_t run_pitch; // packed K: bytes reserved per filter row (kw * cin rounded up to 8); else kw * cpad
   uint32_t o_tiles;  // ceil(out_ch / kTileN)
   uint32_t bk;       // K block of the tensor path
+  uint32_t n_cb;     // K blocks per tap (packed K: K blocks in all)
+  uint32_t n_kb;     // K blocks of a filter row: kh * kw * n_cb (packed K: n_cb)
   bool has_planes;   // digit planes are produced (groups == 1)
   bool packed_k;     // few input channels: the K axis is the flat (kh, kw, ci) index, padded to 16;
                      // such a layer runs as a plain GEMM on an explicitly gathered activation matrix

@@ -110,6 +110,7 @@ struct SampleParams {
   uint32_t norm, span, level_mask, max_level;
   uint32_t seed_lo, seed_hi, layer_id;
   uint32_t cpad, kpad, has_planes;
+  uint32_t bk, n_cb, n_kb;         // operand tiles of the tensor path: K block bytes, blocks per tap, blocks per row
   uint32_t packed_kw, run_pitch;   // packed K (packed_kw = kw, else 0): plane column = kh * run_pitch + kw * Cg + ci
   const uint32_t* e_max;
   int32_t* e_base;
@@ -122,8 +123,9 @@ __device__ __forceinline__ void sample_block(const SampleParams& p, uint32_t blo
                                              uint32_t seed_hi, float* stage) {
   // the parameters may sit in global memory (batched launch): read the scalars once
   const uint32_t norm = p.norm, span = p.span, level_mask = p.level_mask, max_level = p.max_level;
-  const uint32_t layer_id = p.layer_id, KHKW = p.KHKW, Cg = p.Cg, cpad = p.cpad, kpad = p.kpad;
+  const uint32_t layer_id = p.layer_id, KHKW = p.KHKW, Cg = p.Cg;
   const uint32_t packed_kw = p.packed_kw, run_pitch = p.run_pitch, has_planes = p.has_planes;
+  const uint32_t bk = p.bk, n_cb = p.n_cb, n_kb = p.n_kb;
   const PhiloxKeys keys(seed_lo, seed_hi);
   const uint32_t row_block = block / p.ch_chunks;
   const uint32_t chunk = block % p.ch_chunks;
@@ -186,14 +188,15 @@ __device__ __forceinline__ void sample_block(const SampleParams& p, uint32_t blo
     }
 
     const size_t wpos = ((size_t)o * KHKW + tap) * Cg + ci;
-    uint32_t kcol = tap * cpad + ci;
+    // K block and column inside it (bk is a power of two)
+    uint32_t kb = tap * n_cb + ci / bk, kin = ci % bk;
     if (packed_kw) {
       const uint32_t kh = tap / packed_kw;
-      kcol = kh * run_pitch + (tap - kh * packed_kw) * Cg + ci;
+      const uint32_t kcol = kh * run_pitch + (tap - kh * packed_kw) * Cg + ci;
+      kb = kcol / bk;
+      kin = kcol % bk;
     }
     const uint32_t jt = o / kTileN, on = o % kTileN;
-    const size_t plane_stride = (size_t)kTileN * kpad;           // one plane of one channel tile
-    const size_t in_plane = (size_t)on * kpad + kcol;
 #pragma unroll
     for (int l = 0; l < kMaxLevels; ++l) {
       if (!((level_mask >> l) & 1u)) continue;
@@ -201,10 +204,10 @@ __device__ __forceinline__ void sample_block(const SampleParams& p, uint32_t blo
       p.wint[l][wpos] = neg ? -(int32_t)mag : (int32_t)mag;
       if (has_planes) {
         const int P = p.planes_count[l];
-        int8_t* dstp = p.planes[l] + (size_t)jt * P * plane_stride + in_plane;
-        for (int pl = 0; pl < P; ++pl, dstp += plane_stride) {
+        int8_t* tile = p.planes[l] + ((size_t)jt * n_kb + kb) * ((size_t)P * kTileN * bk);
+        for (int pl = 0; pl < P; ++pl) {
           const int digit = (int)((mag >> (kDigitBits * pl)) & 0x7Fu);
-          *dstp = (int8_t)(neg ? -digit : digit);
+          tile[plane_offset((uint32_t)pl * kTileN + on, kin, bk)] = (int8_t)(neg ? -digit : digit);
         }
       }
     }
@@ -316,6 +319,7 @@ uint32_t fill_sample_params(const float* w_dev, const psb_weights* wt, uint32_t*
   p.seed_hi = (uint32_t)(wt->cfg.seed >> 32);
   p.layer_id = wt->cfg.layer_id;
   p.cpad = wt->cpad; p.kpad = wt->kpad; p.has_planes = wt->has_planes ? 1u : 0u;
+  p.bk = wt->bk; p.n_cb = wt->n_cb; p.n_kb = wt->n_kb;
   p.packed_kw = wt->packed_k ? wt->shape.kw : 0u;
   p.run_pitch = wt->run_pitch;
   p.e_max = e_max;

@@ -50,8 +50,7 @@ constexpr long long kWaitLimitCycles = 4000000000ll;        // about 2 s of SM c
 constexpr uint32_t kResidentMaxBytes = 112 * 1024;          // digit planes kept in shared memory
 
 struct TmapSet {
-  CUtensorMap a;
-  CUtensorMap b[kMaxLevels];
+  CUtensorMap a;     // activations; the digit planes need none: their tiles are contiguous
 };
 
 struct TensorParams {
@@ -72,6 +71,20 @@ struct TensorParams {
   uint32_t resident_bytes;
   uint32_t narrow;      // P <= 3 and plane sums below 2^22 (2) or 2^24 (1): 32-bit recombination; 3: whole sum below 2^31
   const long long* corr[kMaxLevels];  // per-channel integer addend, or null
+  const int8_t* planes_ptr[kMaxLevels];  // digit planes: [o_tile][K block][P * 64 rows][BK], pre-swizzled tiles
+  // Band mode (stride-1 filters with taps, one channel block, resident planes): a tile is 128
+  // consecutive positions of one image's output in "padded-linear" order t = oy * Wp + ox with
+  // Wp = W + 2 * pad (positions with ox >= OW are computed and dropped).  In that order the
+  // input pixel of tap (kh, kw) for position t is pixel t + kh * Wp + kw of the zero-padded
+  // image, so one copy of a band of padded input rows serves every tap: the activation operand
+  // of a tap is the same shared-memory band read from a start address moved by
+  // (kh * Wp + kw) pixels.  (The swizzle of a K-major operand is a function of the
+  // shared-memory address bits, so a start address moved by whole rows reads correctly.)
+  uint32_t band;        // 1: band mode
+  uint32_t Wp;          // padded row length
+  uint32_t tpi;         // tiles per image: ceil(OH * Wp / 128)
+  uint32_t band_rows;   // padded input rows per band
+  uint32_t band_bytes;  // stage size (band_rows * Wp * C rounded up to 1024)
 };
 
 // ---- thin PTX wrappers -------------------------------------------------------
@@ -131,6 +144,23 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map
       "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes"
       " [%0], [%1, {%3, %4}], [%2];"
       ::"r"(dst), "l"(map), "r"(bar), "r"(x), "r"(y)
+      : "memory");
+}
+
+// Plain bulk copy of a contiguous, 16-byte aligned run of global memory.
+__device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+      ::"r"(dst), "l"(src), "r"(bytes), "r"(bar)
+      : "memory");
+}
+
+__device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c, int w, int h,
+                                            int n) {
+  asm volatile(
+      "cp.async.bulk.tensor.4d.shared::cluster.global.tile.mbarrier::complete_tx::bytes"
+      " [%0], [%1, {%3, %4, %5, %6}], [%2];"
+      ::"r"(dst), "l"(map), "r"(bar), "r"(c), "r"(w), "r"(h), "r"(n)
       : "memory");
 }
 
@@ -439,6 +469,22 @@ __device__ __forceinline__ bool uniform_epilogue(const TensorParams& p) {
   return !a.kmap && q_only && (P0 == 3u || P0 == 4u);
 }
 
+// Linear output index (n * OH + oy) * OW + ox of row `row` of row tile `m_tile`, and whether the
+// row is a real output.  Plain mode: rows are consecutive outputs.  Band mode: rows are
+// padded-linear positions of one image.
+__device__ __forceinline__ uint32_t tile_row_index(const TensorParams& p, uint32_t m_tile, uint32_t row, bool* valid) {
+  if (!p.band) {
+    const uint32_t m = m_tile * kTileM + row;
+    *valid = m < p.M;
+    return m;
+  }
+  const uint32_t n = m_tile / p.tpi;
+  const uint32_t t = (m_tile - n * p.tpi) * kTileM + row;
+  const uint32_t oy = t / p.Wp, ox = t - oy * p.Wp;
+  *valid = oy < p.a.OH && ox < p.a.OW;
+  return (n * p.a.OH + oy) * p.a.OW + ox;
+}
+
 // Epilogue loop of one warp for the common case: one draw count for the whole layer, only
 // re-quantised bytes wanted.  The warp owns 32 rows (its TMEM lane quarter) x 16 channels of
 // every tile.  Per tile: wait for the accumulator, pull the chunk into registers, hand the TMEM
@@ -463,14 +509,16 @@ __device__ __noinline__ bool epilogue_uniform(const TensorParams& p, SharedCtl* 
   uint32_t pass = 0, cur_o_tile = 0xFFFFFFFFu;
   uint4 r_next = make_uint4(0, 0, 0, 0);
   if (HAS_RES && ti.valid()) {
-    const uint32_t m = ti.m_tile * kTileM + row, ob = ti.o_tile * kTileN + sub * 16u;
-    if (m < p.M && ob < a.O) {
+    bool ok_row;
+    const uint32_t m = tile_row_index(p, ti.m_tile, row, &ok_row), ob = ti.o_tile * kTileN + sub * 16u;
+    if (ok_row && ob < a.O) {
       const uint8_t* src = res_base + out_offset(a, ohow, m, ob);
       r_next = planar ? load_planar16(src, ohow, a.O - ob) : load_row16(src, vec16, ob + 16u <= a.O);
     }
   }
   while (ti.valid()) {
-    const uint32_t m = ti.m_tile * kTileM + row;
+    bool row_valid;
+    const uint32_t m = tile_row_index(p, ti.m_tile, row, &row_valid);
     const uint32_t o_tile = ti.o_tile;
     const uint32_t o_base = o_tile * kTileN + sub * 16u;
     const bool active = o_base < a.O;          // warp-uniform
@@ -495,9 +543,10 @@ __device__ __noinline__ bool epilogue_uniform(const TensorParams& p, SharedCtl* 
     }
     const uint4 r_cur = r_next;
     if (HAS_RES && ti.valid()) {
-      const uint32_t mn = ti.m_tile * kTileM + row, ob = ti.o_tile * kTileN + sub * 16u;
+      bool ok_row;
+      const uint32_t mn = tile_row_index(p, ti.m_tile, row, &ok_row), ob = ti.o_tile * kTileN + sub * 16u;
       r_next = make_uint4(0, 0, 0, 0);
-      if (mn < p.M && ob < a.O) {
+      if (ok_row && ob < a.O) {
         const uint8_t* src = res_base + out_offset(a, ohow, mn, ob);
         r_next = planar ? load_planar16(src, ohow, a.O - ob) : load_row16(src, vec16, ob + 16u <= a.O);
       }
@@ -517,7 +566,7 @@ __device__ __noinline__ bool epilogue_uniform(const TensorParams& p, SharedCtl* 
     tc_fence_before();
     __syncwarp();
     if (lane == 0) mbar_arrive(smem_u32(&ctl->acc_empty[buf]));
-    if (active && m < p.M) {
+    if (active && row_valid) {
       const uint4 q16 = chunk_math<P, MODE, HAS_RES>(v, r_cur, scb, corr, c);
       uint8_t* dst = (uint8_t*)a.q_out + out_offset(a, ohow, m, o_base);
       if (planar) store_planar16(dst, ohow, a.O - o_base, q16);
@@ -546,6 +595,7 @@ __device__ __noinline__ bool mma_role(const TensorParams& p, SharedCtl* ctl, uin
   volatile uint32_t* abort = &ctl->abort;
   const uint32_t group = p.group, stages = p.stages, resident = p.resident, stage_bytes_a = p.stage_bytes_a;
   const uint32_t level_mask = p.a.level_mask;
+  const uint32_t band = p.band, row_bytes = p.Wp * p.a.C, KH = p.a.KH, KW = p.a.KW;
   const uint32_t n_groups = (k_iters + group - 1) / group;
   const uint32_t full0 = smem_u32(&ctl->full[0]), empty0 = smem_u32(&ctl->empty[0]);
   const uint32_t acc_full0 = smem_u32(&ctl->acc_full[0]), acc_empty0 = smem_u32(&ctl->acc_empty[0]);
@@ -567,6 +617,11 @@ __device__ __noinline__ bool mma_role(const TensorParams& p, SharedCtl* ctl, uin
       const uint32_t d_tmem = tmem_base + buf * kTmemBufStride;
       const uint32_t blk = P * kTileN * BK;
       bool joined = (use & 1u) == mine;
+      uint32_t band_off = 0;     // band mode: byte offset of the tile's first position in its band
+      if (band && joined) {
+        const uint32_t t0 = (ti.m_tile % p.tpi) * kTileM;
+        band_off = (t0 % p.Wp) * (uint32_t)BK;
+      }
       if (joined) {
         if (!mbar_wait(acc_empty0 + 8u * buf, aph ^ 1u, abort)) return true;
         tc_fence_after();
@@ -587,12 +642,27 @@ __device__ __noinline__ bool mma_role(const TensorParams& p, SharedCtl* ctl, uin
           }
           tc_fence_after();
           uint32_t a_addr = ring_addr + s * stage_bytes, b_blk = b_res;
-          for (uint32_t j = 0; j < cnt; ++j, a_addr += sub_bytes, b_blk += blk) {
-            const uint32_t b_addr = resident ? b_blk : a_addr + stage_bytes_a;
+          if (band) {
+            // every tap reads the one band of the stage, from a start moved by kh rows and kw pixels
+            a_addr += band_off;
+            uint32_t first = 0;
+            for (uint32_t kh = 0; kh < KH; ++kh, a_addr += row_bytes)
+              for (uint32_t kw = 0; kw < KW; ++kw, b_blk += blk) {
 #pragma unroll
-            for (int ks = 0; ks < BK / 32; ++ks)
-              tc_mma_i8(d_tmem, smem_desc(a_addr + ks * 32, BK), smem_desc(b_addr + ks * 32, BK), idesc,
-                        (it | j | ks) != 0 ? 1u : 0u);
+                for (int ks = 0; ks < BK / 32; ++ks) {
+                  tc_mma_i8(d_tmem, smem_desc(a_addr + kw * BK + ks * 32, BK), smem_desc(b_blk + ks * 32, BK), idesc,
+                            first);
+                  first = 1u;
+                }
+              }
+          } else {
+            for (uint32_t j = 0; j < cnt; ++j, a_addr += sub_bytes, b_blk += blk) {
+              const uint32_t b_addr = resident ? b_blk : a_addr + stage_bytes_a;
+#pragma unroll
+              for (int ks = 0; ks < BK / 32; ++ks)
+                tc_mma_i8(d_tmem, smem_desc(a_addr + ks * 32, BK), smem_desc(b_addr + ks * 32, BK), idesc,
+                          (it | j | ks) != 0 ? 1u : 0u);
+            }
           }
           if (it == 0 && n_groups > 1u) {
             tc_fence_before();
@@ -623,7 +693,7 @@ psb_mma_kernel(const __grid_constant__ TmapSet maps, const __grid_constant__ Ten
   uint8_t* ring = smem + (p.resident ? p.resident_bytes : 0u);
   // a stage holds `group` K blocks, each an activation tile followed (streaming mode) by planes
   const uint32_t sub_bytes = p.stage_bytes_a + (p.resident ? 0u : p.stage_bytes_b_max);
-  const uint32_t stage_bytes = sub_bytes * p.group;
+  const uint32_t stage_bytes = p.band ? p.band_bytes : sub_bytes * p.group;
   SharedCtl* ctl = reinterpret_cast<SharedCtl*>(ring + (size_t)p.stages * stage_bytes);
 
   const uint32_t warp = threadIdx.x >> 5, lane = threadIdx.x & 31u;
@@ -653,9 +723,6 @@ psb_mma_kernel(const __grid_constant__ TmapSet maps, const __grid_constant__ Ten
   if (threadIdx.x == 32) {
     // descriptor fetches of the first copies would otherwise sit on the critical path of the first tile
     asm volatile("prefetch.tensormap [%0];" ::"l"(&maps.a) : "memory");
-    for (int l = 0; l < kMaxLevels; ++l)
-      if (p.planes[l] && ((p.a.level_mask >> l) & 1u))
-        asm volatile("prefetch.tensormap [%0];" ::"l"(&maps.b[l]) : "memory");
   }
   if (warp == kMmaWarp1) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(
@@ -697,14 +764,15 @@ psb_mma_kernel(const __grid_constant__ TmapSet maps, const __grid_constant__ Ten
       // issue a copy of this tile computes them
       uint32_t n0 = 0;
       int h0 = 0, w0 = 0;
-      bool have_coords = !p.im2col;
+      bool have_coords = !p.im2col || p.band;
       // one pass per level present in the tile (levels that were not sampled are flagged by the
       // epilogue and skipped by every role)
       for (uint32_t todo = levels & 0x7Fu; todo && !failed; todo &= todo - 1u) {
         const uint32_t l = (uint32_t)__ffs((int)todo) - 1u;
         const uint32_t P = p.planes[l];
         const uint32_t bytes = p.stage_bytes_a + (p.resident ? 0u : P * kTileN * BK);
-        const int b_row = (int)(o_tile * P * kTileN);
+        const uint32_t blk = P * kTileN * BK;
+        const int8_t* b_tiles = p.planes_ptr[l] + (size_t)o_tile * k_iters * blk;   // this channel tile's K blocks
         for (uint32_t it = 0; it < k_iters;) {
           const uint32_t cnt = min(p.group, k_iters - it);
           if (turn == warp) {
@@ -720,10 +788,18 @@ psb_mma_kernel(const __grid_constant__ TmapSet maps, const __grid_constant__ Ten
             bool ok = true;
             if (lane == 0) {
               ok = mbar_wait(smem_u32(&ctl->empty[s]), ph ^ 1u, abort);
-              if (ok) mbar_expect_tx(bar, bytes * cnt);
+              if (ok) mbar_expect_tx(bar, p.band ? p.band_rows * p.Wp * p.a.C : bytes * cnt);
             }
             if (!__shfl_sync(0xFFFFFFFFu, ok ? 1 : 0, 0)) { failed = true; break; }
-            if (lane < cnt) {
+            if (p.band) {
+              // one copy per tile: the band of padded input rows that holds every tap of the tile;
+              // rows and columns outside the image read as zeros
+              if (lane == 0) {
+                const uint32_t n = m_tile / p.tpi;
+                const uint32_t r0 = ((m_tile - n * p.tpi) * kTileM) / p.Wp;
+                tma_load_4d(ring_addr + s * stage_bytes, &maps.a, bar, 0, -(int)p.a.pad, (int)r0 - (int)p.a.pad, (int)n);
+              }
+            } else if (lane < cnt) {
               // K block it + lane: tap (kh, kw), channel block cb, column kcol of the plane matrix
               const uint32_t kb = it + lane;
               const uint32_t tap = kb / p.n_cb, cb = kb - tap * p.n_cb;
@@ -733,8 +809,7 @@ psb_mma_kernel(const __grid_constant__ TmapSet maps, const __grid_constant__ Ten
                 tma_load_im2col_4d(dst, &maps.a, bar, (int)(cb * BK), w0, h0, (int)n0, (uint16_t)kw, (uint16_t)kh);
               else
                 tma_load_2d(dst, &maps.a, bar, (int)(cb * BK), (int)m0);
-              if (!p.resident)
-                tma_load_2d(dst + p.stage_bytes_a, &maps.b[l], bar, (int)(tap * p.cpad + cb * BK), b_row);
+              if (!p.resident) bulk_load(dst + p.stage_bytes_a, b_tiles + (size_t)kb * blk, blk, bar);
             }
           }
           it += cnt;
@@ -776,10 +851,9 @@ psb_mma_kernel(const __grid_constant__ TmapSet maps, const __grid_constant__ Ten
       const uint32_t part = (k_iters + kPlaneBars - 1) / kPlaneBars;
       for (uint32_t it = ew; it < k_iters; it += (uint32_t)kEpilogueWarps) {
         const uint32_t bar = smem_u32(&ctl->planes_full[it / part]);
-        const uint32_t tap = it / p.n_cb, cb = it - tap * p.n_cb;
         mbar_expect_tx(bar, blk);
-        tma_load_2d(smem_u32(smem) + it * blk, &maps.b[a.uniform_log2k], bar, (int)(tap * p.cpad + cb * BK),
-                    (int)(o_tile * P0 * kTileN));
+        bulk_load(smem_u32(smem) + it * blk, p.planes_ptr[a.uniform_log2k] + ((size_t)o_tile * k_iters + it) * blk, blk,
+                  bar);
       }
     }
     if (uniform_epilogue(p)) {
@@ -962,14 +1036,36 @@ psb_status launch_tensor(psb_ctx* ctx, const psb_weights* wt, const ConvArgs& a,
   p.resident = 0;
   p.ctas_per_otile = 1;
   p.resident_bytes = 0;
+  p.band = 0;
+  p.Wp = p.tpi = p.band_rows = p.band_bytes = 0;
+  const uintptr_t out_ptrs = (uintptr_t)a.q_out | (uintptr_t)a.residual | (uintptr_t)a.f32_out | (uintptr_t)a.acc_out;
+  p.vec_ok = 0u;
+  if (!a.out_nchw && a.O % 16u == 0u && !(out_ptrs & 15u)) p.vec_ok = 2u;
+  else if (!a.out_nchw && a.O % 8u == 0u && !(out_ptrs & 7u)) p.vec_ok = 1u;
   if (!a.kmap) {
     const uint32_t P = p.planes[a.uniform_log2k];
     const uint32_t need = k_iters * P * kTileN * bk;
     const uint32_t cpo = (uint32_t)ctx->sm_count / p.o_tiles;
     if (need <= kResidentMaxBytes && cpo >= 1 && p.o_tiles * cpo * 10u >= (uint32_t)ctx->sm_count * 9u) {
       p.resident = 1;
-      p.ctas_per_otile = cpo < p.m_tiles ? cpo : p.m_tiles;
       p.resident_bytes = need;
+      // band mode: see TensorParams; needs the specialised output stage (codes only)
+      const bool codes_only = a.q_out && !a.f32_out && !a.acc_out && (p.vec_ok || a.out_nchw) && a.inv_step > 0.0f &&
+                              (P == 3u || P == 4u);
+      const uint32_t Wp = a.W + 2u * a.pad;
+      const uint32_t span = kTileM + (a.KH - 1u) * Wp + (a.KW - 1u);   // band pixels a tile touches
+      const uint32_t rows = (Wp - 1u + span + Wp - 1u) / Wp;           // whatever the tile's offset in its first row
+      const uint32_t bytes = round_up(rows * Wp * a.C, 1024u);
+      if (codes_only && p.im2col && a.stride == 1 && a.KH * a.KW > 1u && a.C == bk && (bk == 64u || bk == 128u) &&
+          Wp <= 256u && rows <= 256u && (kSmemBudget - ctl_bytes - need) / bytes >= 2u) {
+        p.band = 1;
+        p.Wp = Wp;
+        p.tpi = (a.OH * Wp + kTileM - 1) / kTileM;
+        p.band_rows = rows;
+        p.band_bytes = bytes;
+        p.m_tiles = a.N * p.tpi;
+      }
+      p.ctas_per_otile = cpo < p.m_tiles ? cpo : p.m_tiles;
     }
   }
   // K blocks are handed over in groups: every barrier round trip costs the issuing thread a
@@ -984,8 +1080,9 @@ psb_status launch_tensor(psb_ctx* ctx, const psb_weights* wt, const ConvArgs& a,
     const uint32_t n_groups = (k_iters + group - 1) / group;
     group = (k_iters + n_groups - 1) / n_groups;
   }
+  if (p.band) group = k_iters;   // one stage = one band = every tap of a tile
   p.group = group;
-  uint32_t stages = (uint32_t)(avail / ((size_t)group * sub_bytes));
+  uint32_t stages = (uint32_t)(p.band ? avail / p.band_bytes : avail / ((size_t)group * sub_bytes));
   if (stages > (uint32_t)kMaxStages) stages = kMaxStages;
   // An even number of stages: the two producer warps and the two MMA issuing threads each take
   // every second stage use, so with an even ring each of them keeps to its own slots and every
@@ -995,7 +1092,8 @@ psb_status launch_tensor(psb_ctx* ctx, const psb_weights* wt, const ConvArgs& a,
   stages &= ~1u;
   if (stages < 2) return PSB_ERR_UNSUPPORTED;
   p.stages = stages;
-  const size_t smem_bytes = (size_t)stages * group * sub_bytes + p.resident_bytes + ctl_bytes;
+  const size_t smem_bytes = (p.band ? (size_t)stages * p.band_bytes : (size_t)stages * group * sub_bytes) +
+                            p.resident_bytes + ctl_bytes;
   for (int l = 0; l < kMaxLevels; ++l) p.corr[l] = add_corr128 ? wt->level[l].corr128 : nullptr;
   // every plane sum is bounded by 127 * (largest activation magnitude) * d
   const uint64_t plane_bound = 127ull * amax * (uint64_t)wt->d;
@@ -1013,15 +1111,19 @@ psb_status launch_tensor(psb_ctx* ctx, const psb_weights* wt, const ConvArgs& a,
       if (p.narrow == 2u && acc_bound < ((unsigned __int128)1 << 31)) p.narrow = 3u;
     }
   }
-  const uintptr_t out_ptrs = (uintptr_t)a.q_out | (uintptr_t)a.residual | (uintptr_t)a.f32_out | (uintptr_t)a.acc_out;
-  p.vec_ok = 0u;
-  if (!a.out_nchw && a.O % 16u == 0u && !(out_ptrs & 15u)) p.vec_ok = 2u;
-  else if (!a.out_nchw && a.O % 8u == 0u && !(out_ptrs & 7u)) p.vec_ok = 1u;
-
   const CUtensorMapSwizzle swz = swizzle_for(bk);
   EncodeTiledFn enc_tiled = (EncodeTiledFn)ctx->encode_tiled;
   EncodeIm2colFn enc_im2col = (EncodeIm2colFn)ctx->encode_im2col;
-  if (p.im2col) {
+  if (p.band) {
+    cuuint64_t dims[4] = {a.C, a.W, a.H, a.N};
+    cuuint64_t strides[3] = {(cuuint64_t)a.C, (cuuint64_t)a.C * a.W, (cuuint64_t)a.C * a.W * a.H};
+    cuuint32_t box[4] = {a.C, p.Wp, p.band_rows, 1};
+    cuuint32_t estr[4] = {1, 1, 1, 1};
+    if (enc_tiled(&maps.a, CU_TENSOR_MAP_DATA_TYPE_UINT8, 4, const_cast<void*>(a.x), dims, strides, box, estr,
+                  CU_TENSOR_MAP_INTERLEAVE_NONE, swz, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+      return PSB_ERR_CUDA;
+  } else if (p.im2col) {
     cuuint64_t dims[4] = {a.C, a.W, a.H, a.N};
     cuuint64_t strides[3] = {(cuuint64_t)a.C, (cuuint64_t)a.C * a.W, (cuuint64_t)a.C * a.W * a.H};
     int lower[2] = {-(int)a.pad, -(int)a.pad};
@@ -1041,18 +1143,7 @@ psb_status launch_tensor(psb_ctx* ctx, const psb_weights* wt, const ConvArgs& a,
                   CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
       return PSB_ERR_CUDA;
   }
-  for (int l = 0; l < kMaxLevels; ++l) {
-    if (!wt->level[l].planes) { memset(&maps.b[l], 0, sizeof(CUtensorMap)); continue; }
-    const uint32_t P = (uint32_t)wt->level[l].planes_count;
-    cuuint64_t dims[2] = {wt->kpad, (cuuint64_t)wt->o_tiles * P * kTileN};
-    cuuint64_t strides[1] = {(cuuint64_t)wt->kpad};
-    cuuint32_t box[2] = {bk, P * kTileN};
-    cuuint32_t estr[2] = {1, 1};
-    if (enc_tiled(&maps.b[l], CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, wt->level[l].planes, dims, strides, box,
-                  estr, CU_TENSOR_MAP_INTERLEAVE_NONE, swz, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
-      return PSB_ERR_CUDA;
-  }
+  for (int l = 0; l < kMaxLevels; ++l) p.planes_ptr[l] = wt->level[l].planes;
 
   p.tile_mask = nullptr;
   if (a.kmap) {

@@ -58,7 +58,6 @@ struct TensorParams {
   uint32_t M;           // N * OH * OW
   uint32_t m_tiles, o_tiles;
   uint32_t n_cb;        // channel blocks per tap
-  uint32_t cpad;
   uint32_t im2col;      // 1: activation tile through the im2col tensor map
   uint32_t stages;
   uint32_t group;       // K blocks per pipeline stage (one barrier hand-over per group)
@@ -85,6 +84,8 @@ struct TensorParams {
   uint32_t tpi;         // tiles per image: ceil(OH * Wp / 128)
   uint32_t band_rows;   // padded input rows per band
   uint32_t band_bytes;  // stage size (band_rows * Wp * C rounded up to 1024)
+  uint32_t Wp_magic, tpi_magic;   // ceil(2^32 / Wp), ceil(2^32 / tpi): quotients by multiply-high (exact in the
+                                  // ranges band mode is restricted to)
 };
 
 // ---- thin PTX wrappers -------------------------------------------------------
@@ -281,7 +282,9 @@ struct SharedCtl {
   unsigned long long started[2];        // per accumulator buffer: the zeroing MMA of the pass has been issued
   uint32_t tmem_base;
   volatile uint32_t abort;
-  float2 scb[kEpilogueWarps][16];       // per epilogue warp: (scale * 2^(e_base - log2 k), bias)
+  // per epilogue warp: 16 values of scale * 2^(e_base - log2 k), then the 16 biases (pairs of
+  // neighbouring channels are read as one 8-byte word)
+  alignas(16) float scb[kEpilogueWarps][32];
   long long corr[kEpilogueWarps][16];   // per epilogue warp: integer addend per channel
 };
 
@@ -304,49 +307,97 @@ struct EpiConst {
   uint32_t res_sign;
 };
 
+// Two fp32 operations per instruction (each half rounded to nearest even on its own, like the scalar
+// forms): the output stage is bound by instruction issue, and half of its arithmetic is of this kind.
+__device__ __forceinline__ float2 fma2(float2 a, float2 b, float2 c) {
+  unsigned long long d;
+  asm("fma.rn.f32x2 %0, %1, %2, %3;"
+      : "=l"(d)
+      : "l"(*reinterpret_cast<unsigned long long*>(&a)), "l"(*reinterpret_cast<unsigned long long*>(&b)),
+        "l"(*reinterpret_cast<unsigned long long*>(&c)));
+  return *reinterpret_cast<float2*>(&d);
+}
+__device__ __forceinline__ float2 add2(float2 a, float2 b) {
+  unsigned long long d;
+  asm("add.rn.f32x2 %0, %1, %2;"
+      : "=l"(d)
+      : "l"(*reinterpret_cast<unsigned long long*>(&a)), "l"(*reinterpret_cast<unsigned long long*>(&b)));
+  return *reinterpret_cast<float2*>(&d);
+}
+__device__ __forceinline__ float2 mul2(float2 a, float2 b) {
+  unsigned long long d;
+  asm("mul.rn.f32x2 %0, %1, %2;"
+      : "=l"(d)
+      : "l"(*reinterpret_cast<unsigned long long*>(&a)), "l"(*reinterpret_cast<unsigned long long*>(&b)));
+  return *reinterpret_cast<float2*>(&d);
+}
+
 template <int P, int MODE, bool HAS_RES>
-__device__ __forceinline__ uint4 chunk_math(const uint32_t (&v)[P][16], const uint4& r4, const float2* scb,
+__device__ __forceinline__ uint4 chunk_math(const uint32_t (&v)[P][16], const uint4& r4, const float* scb,
                                             const long long* corr, const EpiConst& c) {
   const uint32_t rw[4] = {r4.x, r4.y, r4.z, r4.w};
   const float res_bias = 8388608.0f + (float)c.res_sign;   // undoes the magic constant and the sign flip
+  const float2 neg_res_bias2 = make_float2(-res_bias, -res_bias), res_scale2 = make_float2(c.res_scale, c.res_scale);
+  const float2 inv_step2 = make_float2(c.inv_step, c.inv_step), magic2 = make_float2(12582912.0f, 12582912.0f);
   uint32_t qw[4];
 #pragma unroll
   for (int g = 0; g < 4; ++g) {
     uint32_t q[4];
 #pragma unroll
-    for (int e = 0; e < 4; ++e) {
-      const int j = 4 * g + e;
-      float af;
-      if (MODE == 3) {
-        // the whole sum fits 32 bits (wrap-around in the partial sums is harmless): one conversion
-        int acc = (int)v[0][j];
-        if (P > 1) acc += (int)v[1][j] << kDigitBits;
-        if (P > 2) acc += (int)v[2][j] << (2 * kDigitBits);
-        af = (float)acc;
-      } else if (MODE > 0) {
-        int u = (int)v[0][j];
-        if (P > 1) u += (int)v[1][j] << kDigitBits;
-        int w = u >> (2 * kDigitBits);
-        if (P > 2) w += (int)v[2][j];
-        const float lo_f = __uint_as_float(0x4B000000u | ((uint32_t)u & 0x3FFFu)) - 8388608.0f;
-        const float w_f = MODE == 2 ? __int_as_float(0x4B400000 + w) - 12582912.0f : (float)w;
-        af = __fmaf_rn(w_f, 16384.0f, lo_f);
-      } else {
-        long long acc = (long long)(int)v[0][j];
+    for (int h = 0; h < 2; ++h) {
+      const int j = 4 * g + 2 * h;       // channels j and j + 1 go through the arithmetic side by side
+      float af[2] = {0.0f, 0.0f};
 #pragma unroll
-        for (int pl = 1; pl < P; ++pl) acc += (long long)(int)v[pl][j] * (long long)(1 << (kDigitBits * pl));
-        acc += corr[j];
-        af = acc_to_float(acc);
+      for (int e = 0; e < 2; ++e) {
+        if (MODE == 3) {
+          // the whole sum fits 32 bits (wrap-around in the partial sums is harmless): one conversion
+          int acc = (int)v[0][j + e];
+          if (P > 1) acc += (int)v[1][j + e] << kDigitBits;
+          if (P > 2) acc += (int)v[2][j + e] << (2 * kDigitBits);
+          af[e] = (float)acc;
+        } else if (MODE == 0) {
+          long long acc = (long long)(int)v[0][j + e];
+#pragma unroll
+          for (int pl = 1; pl < P; ++pl) acc += (long long)(int)v[pl][j + e] * (long long)(1 << (kDigitBits * pl));
+          acc += corr[j + e];
+          af[e] = acc_to_float(acc);
+        }
       }
-      const float2 sb = scb[j];
-      float y = __fmaf_rn(af, sb.x, sb.y);
+      float2 a2 = make_float2(af[0], af[1]);
+      if (MODE == 1 || MODE == 2) {
+        int w[2];
+        uint32_t lo[2];
+#pragma unroll
+        for (int e = 0; e < 2; ++e) {
+          int u = (int)v[0][j + e];
+          if (P > 1) u += (int)v[1][j + e] << kDigitBits;
+          w[e] = u >> (2 * kDigitBits);
+          if (P > 2) w[e] += (int)v[2][j + e];
+          lo[e] = 0x4B000000u | ((uint32_t)u & 0x3FFFu);
+        }
+        const float2 lo2 = add2(make_float2(__uint_as_float(lo[0]), __uint_as_float(lo[1])),
+                                make_float2(-8388608.0f, -8388608.0f));
+        const float2 w2 = MODE == 2 ? add2(make_float2(__int_as_float(0x4B400000 + w[0]), __int_as_float(0x4B400000 + w[1])),
+                                           make_float2(-12582912.0f, -12582912.0f))
+                                    : make_float2((float)w[0], (float)w[1]);
+        a2 = fma2(w2, make_float2(16384.0f, 16384.0f), lo2);
+      }
+      const float2 sc2 = *reinterpret_cast<const float2*>(scb + j), bi2 = *reinterpret_cast<const float2*>(scb + 16 + j);
+      float2 y2 = fma2(a2, sc2, bi2);
       if (HAS_RES) {
-        const uint32_t rb = ((rw[g] >> (8 * e)) & 0xFFu) ^ c.res_sign;   // byte + 128 if signed
-        y = __fmaf_rn(__uint_as_float(0x4B000000u | rb) - res_bias, c.res_scale, y);
+        const uint32_t rb0 = ((rw[g] >> (16 * h)) & 0xFFu) ^ c.res_sign;        // byte + 128 if signed
+        const uint32_t rb1 = ((rw[g] >> (16 * h + 8)) & 0xFFu) ^ c.res_sign;
+        const float2 r2 = add2(make_float2(__uint_as_float(0x4B000000u | rb0), __uint_as_float(0x4B000000u | rb1)),
+                               neg_res_bias2);
+        y2 = fma2(r2, res_scale2, y2);
       }
       // clamp, then round half to even by adding 1.5 * 2^23: the low byte of the sum is the code
-      const float t = fminf(fmaxf(__fmul_rn(y, c.inv_step), c.qmin_f), c.qmax_f);
-      q[e] = __float_as_uint(t + 12582912.0f);
+      float2 t2 = mul2(y2, inv_step2);
+      t2.x = fminf(fmaxf(t2.x, c.qmin_f), c.qmax_f);
+      t2.y = fminf(fmaxf(t2.y, c.qmin_f), c.qmax_f);
+      const float2 q2 = add2(t2, magic2);
+      q[2 * h] = __float_as_uint(q2.x);
+      q[2 * h + 1] = __float_as_uint(q2.y);
     }
     qw[g] = __byte_perm(__byte_perm(q[0], q[1], 0x0040), __byte_perm(q[2], q[3], 0x0040), 0x5410);
   }
@@ -403,7 +454,7 @@ __device__ __forceinline__ size_t out_offset(const ConvArgs& a, uint32_t ohow, u
 
 template <int P, int MODE, bool HAS_RES>
 __device__ __noinline__ void epilogue_chunk_q(uint32_t taddr, bool valid, uint8_t* q_dst, uint4 r4, bool vec16,
-                                              bool both, const float2* scb, const long long* corr, EpiConst c) {
+                                              bool both, const float* scb, const long long* corr, EpiConst c) {
   uint32_t v[P][16];
 #pragma unroll
   for (int pl = 0; pl < P; ++pl) tc_ld16(taddr + pl * kTileN, v[pl]);
@@ -416,7 +467,7 @@ __device__ __noinline__ void epilogue_chunk_q(uint32_t taddr, bool valid, uint8_
 template <int P>
 __device__ __noinline__ void epilogue_chunk(const TensorParams& p, uint32_t taddr, uint32_t o_base,
                                             uint32_t m, bool valid, uint32_t n, uint32_t pix,
-                                            const float2* scb, const long long* corr, bool use_corr) {
+                                            const float* scb, const long long* corr, bool use_corr) {
   uint32_t v[P][16];
 #pragma unroll
   for (int pl = 0; pl < P; ++pl) tc_ld16(taddr + pl * kTileN, v[pl]);
@@ -448,7 +499,7 @@ __device__ __noinline__ void epilogue_chunk(const TensorParams& p, uint32_t tadd
         else rb = (int)((const uint8_t*)a.residual)[oidx];
         if (a.residual_dtype == PSB_DT_S8) rb = (int)(int8_t)rb;
       }
-      const float y = dequant(acc, scb[j].x, scb[j].y, a.residual != nullptr, rb, a.residual_scale, a.relu != 0);
+      const float y = dequant(acc, scb[j], scb[16 + j], a.residual != nullptr, rb, a.residual_scale, a.relu != 0);
       if (a.f32_out) a.f32_out[oidx] = y;
       if (a.q_out) {
         const int q = requant(y, a.inv_step, a.qmin, a.qmax);
@@ -478,9 +529,9 @@ __device__ __forceinline__ uint32_t tile_row_index(const TensorParams& p, uint32
     *valid = m < p.M;
     return m;
   }
-  const uint32_t n = m_tile / p.tpi;
+  const uint32_t n = __umulhi(m_tile, p.tpi_magic);
   const uint32_t t = (m_tile - n * p.tpi) * kTileM + row;
-  const uint32_t oy = t / p.Wp, ox = t - oy * p.Wp;
+  const uint32_t oy = __umulhi(t, p.Wp_magic), ox = t - oy * p.Wp;
   *valid = oy < p.a.OH && ox < p.a.OW;
   return (n * p.a.OH + oy) * p.a.OW + ox;
 }
@@ -500,7 +551,7 @@ __device__ __noinline__ bool epilogue_uniform(const TensorParams& p, SharedCtl* 
   const bool use_corr = p.corr[l] != nullptr;
   volatile uint32_t* abort = &ctl->abort;
   const uint8_t* res_base = (const uint8_t*)a.residual;
-  const float2* scb = ctl->scb[ew];
+  const float* scb = ctl->scb[ew];
   const long long* corr = ctl->corr[ew];
   const bool vec16 = p.vec_ok == 2u, planar = a.out_nchw != 0u;
   const uint32_t ohow = a.OH * a.OW;
@@ -535,7 +586,8 @@ __device__ __noinline__ bool epilogue_uniform(const TensorParams& p, SharedCtl* 
           sb.y = a.bias[o];
           if (use_corr) cr = p.corr[l][o];
         }
-        ctl->scb[ew][lane] = sb;
+        ctl->scb[ew][lane] = sb.x;
+        ctl->scb[ew][16 + lane] = sb.y;
         ctl->corr[ew][lane] = cr;
       }
       cur_o_tile = o_tile;
@@ -583,9 +635,9 @@ __device__ __noinline__ bool epilogue_uniform(const TensorParams& p, SharedCtl* 
 // stage of a pass waits for the accumulator buffer and issues the zeroing MMA; the other one
 // joins the pass after that (`started`).  Integer accumulation is exact, so the order in
 // which the two threads' MMAs reach the accumulator is immaterial.  A parity wait on a stage
-// barrier is meaningful while the waiter is less than two uses of that stage ahead of it: a
-// thread has seen use n - 2 arrive before it waits for use n, and with two or more ring
-// stages use n - stages is not later than that.  Kept out of line and fed from local copies of
+// barrier is meaningful while the waiter is less than two uses of that stage ahead of it; the
+// ring has an even number of stages, so a thread always meets the same slots and its wait for
+// a slot follows its own previous use of that slot.  Kept out of line and fed from local copies of
 // the parameters so that its loop state lives in registers: the pipe idles for every clock this
 // thread spends between two MMAs beyond what the other thread covers.  Returns true on a timeout.
 template <int BK>
@@ -619,8 +671,8 @@ __device__ __noinline__ bool mma_role(const TensorParams& p, SharedCtl* ctl, uin
       bool joined = (use & 1u) == mine;
       uint32_t band_off = 0;     // band mode: byte offset of the tile's first position in its band
       if (band && joined) {
-        const uint32_t t0 = (ti.m_tile % p.tpi) * kTileM;
-        band_off = (t0 % p.Wp) * (uint32_t)BK;
+        const uint32_t t0 = (ti.m_tile - __umulhi(ti.m_tile, p.tpi_magic) * p.tpi) * kTileM;
+        band_off = (t0 - __umulhi(t0, p.Wp_magic) * p.Wp) * (uint32_t)BK;
       }
       if (joined) {
         if (!mbar_wait(acc_empty0 + 8u * buf, aph ^ 1u, abort)) return true;
@@ -795,8 +847,8 @@ psb_mma_kernel(const __grid_constant__ TmapSet maps, const __grid_constant__ Ten
               // one copy per tile: the band of padded input rows that holds every tap of the tile;
               // rows and columns outside the image read as zeros
               if (lane == 0) {
-                const uint32_t n = m_tile / p.tpi;
-                const uint32_t r0 = ((m_tile - n * p.tpi) * kTileM) / p.Wp;
+                const uint32_t n = __umulhi(m_tile, p.tpi_magic);
+                const uint32_t r0 = __umulhi((m_tile - n * p.tpi) * kTileM, p.Wp_magic);
                 tma_load_4d(ring_addr + s * stage_bytes, &maps.a, bar, 0, -(int)p.a.pad, (int)r0 - (int)p.a.pad, (int)n);
               }
             } else if (lane < cnt) {
@@ -869,7 +921,7 @@ psb_mma_kernel(const __grid_constant__ TmapSet maps, const __grid_constant__ Ten
 #undef PSB_UNI
     } else {
       // general loop: per-location draw counts, any outputs and layouts, ragged channel counts
-      const float2* scb = ctl->scb[ew];
+      const float* scb = ctl->scb[ew];
       const long long* corr = ctl->corr[ew];
       uint32_t pass = 0, cur_key = 0xFFFFFFFFu;
       TileIter ti;
@@ -905,7 +957,8 @@ psb_mma_kernel(const __grid_constant__ TmapSet maps, const __grid_constant__ Ten
                 sb.y = a.bias[o];
                 if (use_corr) cr = p.corr[l][o];
               }
-              ctl->scb[ew][lane] = sb;
+              ctl->scb[ew][lane] = sb.x;
+        ctl->scb[ew][16 + lane] = sb.y;
               ctl->corr[ew][lane] = cr;
             }
             cur_key = key;
@@ -1020,7 +1073,6 @@ psb_status launch_tensor(psb_ctx* ctx, const psb_weights* wt, const ConvArgs& a,
   p.o_tiles = wt->o_tiles;
   const uint32_t bk = wt->bk;
   p.n_cb = (a.C + bk - 1) / bk;
-  p.cpad = wt->cpad;
   p.im2col = is_plain_gemm(a) ? 0u : 1u;
   uint32_t pmax = 1;
   for (int l = 0; l < kMaxLevels; ++l) {
@@ -1037,7 +1089,7 @@ psb_status launch_tensor(psb_ctx* ctx, const psb_weights* wt, const ConvArgs& a,
   p.ctas_per_otile = 1;
   p.resident_bytes = 0;
   p.band = 0;
-  p.Wp = p.tpi = p.band_rows = p.band_bytes = 0;
+  p.Wp = p.tpi = p.band_rows = p.band_bytes = p.Wp_magic = p.tpi_magic = 0;
   const uintptr_t out_ptrs = (uintptr_t)a.q_out | (uintptr_t)a.residual | (uintptr_t)a.f32_out | (uintptr_t)a.acc_out;
   p.vec_ok = 0u;
   if (!a.out_nchw && a.O % 16u == 0u && !(out_ptrs & 15u)) p.vec_ok = 2u;
@@ -1056,11 +1108,18 @@ psb_status launch_tensor(psb_ctx* ctx, const psb_weights* wt, const ConvArgs& a,
       const uint32_t span = kTileM + (a.KH - 1u) * Wp + (a.KW - 1u);   // band pixels a tile touches
       const uint32_t rows = (Wp - 1u + span + Wp - 1u) / Wp;           // whatever the tile's offset in its first row
       const uint32_t bytes = round_up(rows * Wp * a.C, 1024u);
+      // x / d == mulhi(x, ceil(2^32 / d)) while x * d < 2^32 (d >= 2): positions t < tpi * 128 against Wp,
+      // tile numbers < N * tpi against tpi
+      const uint64_t tpi = ((uint64_t)a.OH * Wp + kTileM - 1) / kTileM;
+      const bool quotients_ok = Wp >= 2u && tpi >= 2u && tpi * kTileM * Wp < (1ull << 32) &&
+                                (uint64_t)a.N * tpi * tpi < (1ull << 32);
       if (codes_only && p.im2col && a.stride == 1 && a.KH * a.KW > 1u && a.C == bk && (bk == 64u || bk == 128u) &&
-          Wp <= 256u && rows <= 256u && (kSmemBudget - ctl_bytes - need) / bytes >= 2u) {
+          Wp <= 256u && rows <= 256u && (kSmemBudget - ctl_bytes - need) / bytes >= 2u && quotients_ok) {
         p.band = 1;
         p.Wp = Wp;
-        p.tpi = (a.OH * Wp + kTileM - 1) / kTileM;
+        p.tpi = (uint32_t)tpi;
+        p.Wp_magic = (uint32_t)(((1ull << 32) + Wp - 1) / Wp);
+        p.tpi_magic = (uint32_t)(((1ull << 32) + tpi - 1) / tpi);
         p.band_rows = rows;
         p.band_bytes = bytes;
         p.m_tiles = a.N * p.tpi;

@@ -243,6 +243,32 @@ def test_tensor_path_planar_layout_codes_only(psb, ctx, oracle, O, with_res):
     assert g["path"] == psb.PSB_PATH_TENSOR
 
 
+# (N, C, H, W, O, KH, KW, pad, layout, signed input, shortcut): stride-1 filters with taps, one channel
+# block and codes-only output take the band mode of the tensor kernel (a tile is 128 positions of one
+# image in padded-row order); odd and even padded widths, no padding, wide filters, ragged last tiles,
+# several images, two channel tiles, planar and channels-last outputs
+@pytest.mark.parametrize("case", [(3, 64, 13, 11, 64, 3, 3, 1, 1, False, False),
+                                  (2, 64, 30, 30, 128, 3, 3, 1, 1, False, True),
+                                  (2, 128, 14, 9, 64, 2, 2, 1, 1, False, True),
+                                  (2, 64, 12, 17, 64, 3, 3, 0, 1, False, False),
+                                  (1, 64, 9, 21, 64, 2, 2, 1, 1, True, False),
+                                  (2, 64, 10, 23, 48, 1, 3, 0, 0, False, True),
+                                  (2, 128, 11, 6, 64, 3, 1, 0, 1, False, False),
+                                  (5, 64, 7, 7, 64, 3, 3, 1, 0, False, False)])
+def test_tensor_path_band_mode_codes_only(psb, ctx, oracle, case):
+    N, C, H, W, O, KH, KW, pad, layout, signed, with_res = case
+    rng = np.random.default_rng(abs(hash(case)) % 2 ** 31)
+    w, x, scale, bias = _layer_inputs(rng, N, C, H, W, O, KH, KW, 1, layout, x_dtype=np.int8 if signed else np.uint8,
+                                      x_hi=16)
+    OH, OW = H + 2 * pad - KH + 1, W + 2 * pad - KW + 1
+    res = None
+    if with_res:
+        res = rng.integers(0, 16, size=(N, O, OH, OW) if layout == 0 else (N, OH, OW, O)).astype(np.uint8)
+    g = _both(psb, ctx, oracle, w, x, layout, 1, 1, pad, [3], scale, bias, inv_step=0.4, residual=res,
+              res_scale=0.25 if with_res else 0.0, in_max=16 if signed else 15, path=psb.PSB_PATH_TENSOR, want=("q",))
+    assert g["path"] == psb.PSB_PATH_TENSOR
+
+
 def test_depthwise_5x5_codes_only(psb, ctx, oracle):
     rng = np.random.default_rng(55)
     C = 48

@@ -282,9 +282,7 @@ struct SharedCtl {
   unsigned long long started[2];        // per accumulator buffer: the zeroing MMA of the pass has been issued
   uint32_t tmem_base;
   volatile uint32_t abort;
-  // per epilogue warp: 16 values of scale * 2^(e_base - log2 k), then the 16 biases (pairs of
-  // neighbouring channels are read as one 8-byte word)
-  alignas(16) float scb[kEpilogueWarps][32];
+  float2 scb[kEpilogueWarps][16];       // per epilogue warp: (scale * 2^(e_base - log2 k), bias)
   long long corr[kEpilogueWarps][16];   // per epilogue warp: integer addend per channel
 };
 
@@ -307,97 +305,49 @@ struct EpiConst {
   uint32_t res_sign;
 };
 
-// Two fp32 operations per instruction (each half rounded to nearest even on its own, like the scalar
-// forms): the output stage is bound by instruction issue, and half of its arithmetic is of this kind.
-__device__ __forceinline__ float2 fma2(float2 a, float2 b, float2 c) {
-  unsigned long long d;
-  asm("fma.rn.f32x2 %0, %1, %2, %3;"
-      : "=l"(d)
-      : "l"(*reinterpret_cast<unsigned long long*>(&a)), "l"(*reinterpret_cast<unsigned long long*>(&b)),
-        "l"(*reinterpret_cast<unsigned long long*>(&c)));
-  return *reinterpret_cast<float2*>(&d);
-}
-__device__ __forceinline__ float2 add2(float2 a, float2 b) {
-  unsigned long long d;
-  asm("add.rn.f32x2 %0, %1, %2;"
-      : "=l"(d)
-      : "l"(*reinterpret_cast<unsigned long long*>(&a)), "l"(*reinterpret_cast<unsigned long long*>(&b)));
-  return *reinterpret_cast<float2*>(&d);
-}
-__device__ __forceinline__ float2 mul2(float2 a, float2 b) {
-  unsigned long long d;
-  asm("mul.rn.f32x2 %0, %1, %2;"
-      : "=l"(d)
-      : "l"(*reinterpret_cast<unsigned long long*>(&a)), "l"(*reinterpret_cast<unsigned long long*>(&b)));
-  return *reinterpret_cast<float2*>(&d);
-}
-
 template <int P, int MODE, bool HAS_RES>
-__device__ __forceinline__ uint4 chunk_math(const uint32_t (&v)[P][16], const uint4& r4, const float* scb,
+__device__ __forceinline__ uint4 chunk_math(const uint32_t (&v)[P][16], const uint4& r4, const float2* scb,
                                             const long long* corr, const EpiConst& c) {
   const uint32_t rw[4] = {r4.x, r4.y, r4.z, r4.w};
   const float res_bias = 8388608.0f + (float)c.res_sign;   // undoes the magic constant and the sign flip
-  const float2 neg_res_bias2 = make_float2(-res_bias, -res_bias), res_scale2 = make_float2(c.res_scale, c.res_scale);
-  const float2 inv_step2 = make_float2(c.inv_step, c.inv_step), magic2 = make_float2(12582912.0f, 12582912.0f);
   uint32_t qw[4];
 #pragma unroll
   for (int g = 0; g < 4; ++g) {
     uint32_t q[4];
 #pragma unroll
-    for (int h = 0; h < 2; ++h) {
-      const int j = 4 * g + 2 * h;       // channels j and j + 1 go through the arithmetic side by side
-      float af[2] = {0.0f, 0.0f};
+    for (int e = 0; e < 4; ++e) {
+      const int j = 4 * g + e;
+      float af;
+      if (MODE == 3) {
+        // the whole sum fits 32 bits (wrap-around in the partial sums is harmless): one conversion
+        int acc = (int)v[0][j];
+        if (P > 1) acc += (int)v[1][j] << kDigitBits;
+        if (P > 2) acc += (int)v[2][j] << (2 * kDigitBits);
+        af = (float)acc;
+      } else if (MODE > 0) {
+        int u = (int)v[0][j];
+        if (P > 1) u += (int)v[1][j] << kDigitBits;
+        int w = u >> (2 * kDigitBits);
+        if (P > 2) w += (int)v[2][j];
+        const float lo_f = __uint_as_float(0x4B000000u | ((uint32_t)u & 0x3FFFu)) - 8388608.0f;
+        const float w_f = MODE == 2 ? __int_as_float(0x4B400000 + w) - 12582912.0f : (float)w;
+        af = __fmaf_rn(w_f, 16384.0f, lo_f);
+      } else {
+        long long acc = (long long)(int)v[0][j];
 #pragma unroll
-      for (int e = 0; e < 2; ++e) {
-        if (MODE == 3) {
-          // the whole sum fits 32 bits (wrap-around in the partial sums is harmless): one conversion
-          int acc = (int)v[0][j + e];
-          if (P > 1) acc += (int)v[1][j + e] << kDigitBits;
-          if (P > 2) acc += (int)v[2][j + e] << (2 * kDigitBits);
-          af[e] = (float)acc;
-        } else if (MODE == 0) {
-          long long acc = (long long)(int)v[0][j + e];
-#pragma unroll
-          for (int pl = 1; pl < P; ++pl) acc += (long long)(int)v[pl][j + e] * (long long)(1 << (kDigitBits * pl));
-          acc += corr[j + e];
-          af[e] = acc_to_float(acc);
-        }
+        for (int pl = 1; pl < P; ++pl) acc += (long long)(int)v[pl][j] * (long long)(1 << (kDigitBits * pl));
+        acc += corr[j];
+        af = acc_to_float(acc);
       }
-      float2 a2 = make_float2(af[0], af[1]);
-      if (MODE == 1 || MODE == 2) {
-        int w[2];
-        uint32_t lo[2];
-#pragma unroll
-        for (int e = 0; e < 2; ++e) {
-          int u = (int)v[0][j + e];
-          if (P > 1) u += (int)v[1][j + e] << kDigitBits;
-          w[e] = u >> (2 * kDigitBits);
-          if (P > 2) w[e] += (int)v[2][j + e];
-          lo[e] = 0x4B000000u | ((uint32_t)u & 0x3FFFu);
-        }
-        const float2 lo2 = add2(make_float2(__uint_as_float(lo[0]), __uint_as_float(lo[1])),
-                                make_float2(-8388608.0f, -8388608.0f));
-        const float2 w2 = MODE == 2 ? add2(make_float2(__int_as_float(0x4B400000 + w[0]), __int_as_float(0x4B400000 + w[1])),
-                                           make_float2(-12582912.0f, -12582912.0f))
-                                    : make_float2((float)w[0], (float)w[1]);
-        a2 = fma2(w2, make_float2(16384.0f, 16384.0f), lo2);
-      }
-      const float2 sc2 = *reinterpret_cast<const float2*>(scb + j), bi2 = *reinterpret_cast<const float2*>(scb + 16 + j);
-      float2 y2 = fma2(a2, sc2, bi2);
+      const float2 sb = scb[j];
+      float y = __fmaf_rn(af, sb.x, sb.y);
       if (HAS_RES) {
-        const uint32_t rb0 = ((rw[g] >> (16 * h)) & 0xFFu) ^ c.res_sign;        // byte + 128 if signed
-        const uint32_t rb1 = ((rw[g] >> (16 * h + 8)) & 0xFFu) ^ c.res_sign;
-        const float2 r2 = add2(make_float2(__uint_as_float(0x4B000000u | rb0), __uint_as_float(0x4B000000u | rb1)),
-                               neg_res_bias2);
-        y2 = fma2(r2, res_scale2, y2);
+        const uint32_t rb = ((rw[g] >> (8 * e)) & 0xFFu) ^ c.res_sign;   // byte + 128 if signed
+        y = __fmaf_rn(__uint_as_float(0x4B000000u | rb) - res_bias, c.res_scale, y);
       }
       // clamp, then round half to even by adding 1.5 * 2^23: the low byte of the sum is the code
-      float2 t2 = mul2(y2, inv_step2);
-      t2.x = fminf(fmaxf(t2.x, c.qmin_f), c.qmax_f);
-      t2.y = fminf(fmaxf(t2.y, c.qmin_f), c.qmax_f);
-      const float2 q2 = add2(t2, magic2);
-      q[2 * h] = __float_as_uint(q2.x);
-      q[2 * h + 1] = __float_as_uint(q2.y);
+      const float t = fminf(fmaxf(__fmul_rn(y, c.inv_step), c.qmin_f), c.qmax_f);
+      q[e] = __float_as_uint(t + 12582912.0f);
     }
     qw[g] = __byte_perm(__byte_perm(q[0], q[1], 0x0040), __byte_perm(q[2], q[3], 0x0040), 0x5410);
   }
@@ -454,7 +404,7 @@ __device__ __forceinline__ size_t out_offset(const ConvArgs& a, uint32_t ohow, u
 
 template <int P, int MODE, bool HAS_RES>
 __device__ __noinline__ void epilogue_chunk_q(uint32_t taddr, bool valid, uint8_t* q_dst, uint4 r4, bool vec16,
-                                              bool both, const float* scb, const long long* corr, EpiConst c) {
+                                              bool both, const float2* scb, const long long* corr, EpiConst c) {
   uint32_t v[P][16];
 #pragma unroll
   for (int pl = 0; pl < P; ++pl) tc_ld16(taddr + pl * kTileN, v[pl]);
@@ -467,7 +417,7 @@ __device__ __noinline__ void epilogue_chunk_q(uint32_t taddr, bool valid, uint8_
 template <int P>
 __device__ __noinline__ void epilogue_chunk(const TensorParams& p, uint32_t taddr, uint32_t o_base,
                                             uint32_t m, bool valid, uint32_t n, uint32_t pix,
-                                            const float* scb, const long long* corr, bool use_corr) {
+                                            const float2* scb, const long long* corr, bool use_corr) {
   uint32_t v[P][16];
 #pragma unroll
   for (int pl = 0; pl < P; ++pl) tc_ld16(taddr + pl * kTileN, v[pl]);
@@ -499,7 +449,7 @@ __device__ __noinline__ void epilogue_chunk(const TensorParams& p, uint32_t tadd
         else rb = (int)((const uint8_t*)a.residual)[oidx];
         if (a.residual_dtype == PSB_DT_S8) rb = (int)(int8_t)rb;
       }
-      const float y = dequant(acc, scb[j], scb[16 + j], a.residual != nullptr, rb, a.residual_scale, a.relu != 0);
+      const float y = dequant(acc, scb[j].x, scb[j].y, a.residual != nullptr, rb, a.residual_scale, a.relu != 0);
       if (a.f32_out) a.f32_out[oidx] = y;
       if (a.q_out) {
         const int q = requant(y, a.inv_step, a.qmin, a.qmax);
@@ -551,7 +501,7 @@ __device__ __noinline__ bool epilogue_uniform(const TensorParams& p, SharedCtl* 
   const bool use_corr = p.corr[l] != nullptr;
   volatile uint32_t* abort = &ctl->abort;
   const uint8_t* res_base = (const uint8_t*)a.residual;
-  const float* scb = ctl->scb[ew];
+  const float2* scb = ctl->scb[ew];
   const long long* corr = ctl->corr[ew];
   const bool vec16 = p.vec_ok == 2u, planar = a.out_nchw != 0u;
   const uint32_t ohow = a.OH * a.OW;
@@ -586,8 +536,7 @@ __device__ __noinline__ bool epilogue_uniform(const TensorParams& p, SharedCtl* 
           sb.y = a.bias[o];
           if (use_corr) cr = p.corr[l][o];
         }
-        ctl->scb[ew][lane] = sb.x;
-        ctl->scb[ew][16 + lane] = sb.y;
+        ctl->scb[ew][lane] = sb;
         ctl->corr[ew][lane] = cr;
       }
       cur_o_tile = o_tile;
@@ -921,7 +870,7 @@ psb_mma_kernel(const __grid_constant__ TmapSet maps, const __grid_constant__ Ten
 #undef PSB_UNI
     } else {
       // general loop: per-location draw counts, any outputs and layouts, ragged channel counts
-      const float* scb = ctl->scb[ew];
+      const float2* scb = ctl->scb[ew];
       const long long* corr = ctl->corr[ew];
       uint32_t pass = 0, cur_key = 0xFFFFFFFFu;
       TileIter ti;
@@ -957,8 +906,7 @@ psb_mma_kernel(const __grid_constant__ TmapSet maps, const __grid_constant__ Ten
                 sb.y = a.bias[o];
                 if (use_corr) cr = p.corr[l][o];
               }
-              ctl->scb[ew][lane] = sb.x;
-        ctl->scb[ew][16 + lane] = sb.y;
+              ctl->scb[ew][lane] = sb;
               ctl->corr[ew][lane] = cr;
             }
             cur_key = key;

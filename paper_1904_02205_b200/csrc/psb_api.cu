@@ -302,7 +302,8 @@ psb_status psb_sample_weights(psb_ctx* ctx, const float* w_dev, const psb_wshape
     w->n_cb = ((w->packed_k ? w->kpad : shape->in_ch_per_group) + w->bk - 1) / w->bk;
     w->n_kb = w->packed_k ? w->n_cb : shape->kh * shape->kw * w->n_cb;
     bool ok = cudaMalloc(&w->e_base, sizeof(int32_t) * shape->out_ch) == cudaSuccess &&
-              cudaMalloc(&w->e_max, sizeof(uint32_t) * shape->out_ch) == cudaSuccess;
+              cudaMalloc(&w->e_max, sizeof(uint32_t) * shape->out_ch) == cudaSuccess &&
+              cudaMemsetAsync(w->e_max, 0, sizeof(uint32_t) * shape->out_ch, s) == cudaSuccess;
     for (uint32_t l = 0; ok && l < (uint32_t)kMaxLevels; ++l) {
       if (!((cfg.level_mask >> l) & 1u)) continue;
       ok = cudaMalloc(&w->level[l].wint, sizeof(int32_t) * d64 * shape->out_ch) == cudaSuccess;

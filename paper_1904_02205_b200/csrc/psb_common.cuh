@@ -67,7 +67,8 @@ struct psb_weights {
                      // such a layer runs as a plain GEMM on an explicitly gathered activation matrix
   psb::LevelStore level[psb::kMaxLevels];
   int32_t* e_base = nullptr;   // [O]
-  uint32_t* e_max = nullptr;   // [O] scratch of the window reduction (biased exponent, 0 = none)
+  uint32_t* e_max = nullptr;   // [O] scratch of the window reduction: (call number << 8) | biased exponent
+  uint32_t e_calls = 0;        // sampling calls made on this handle, modulo 2^24
   int device;
 };
 
@@ -160,6 +161,31 @@ __device__ __forceinline__ float acc_to_float_small(long long acc) {
   const float lo_f = __uint_as_float(0x4B000000u | lo) - 8388608.0f;
   return __fmaf_rn(hi_f, 8388608.0f, lo_f);
 }
+
+// Programmatic dependent launch: a kernel launched through launch_pdl may be scheduled while the
+// kernel before it in the stream is still running; it must call pdl_prologue() before it touches
+// global memory, which waits for the earlier grids to complete (and lets the kernel after it be
+// scheduled in turn).  What is saved is the launch latency between the many short kernels of a step.
+#ifdef __CUDACC__
+__device__ __forceinline__ void pdl_prologue() {
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+}
+template <typename K, typename... Args>
+inline cudaError_t launch_pdl(K kernel, dim3 grid, dim3 block, size_t smem, cudaStream_t s, Args... args) {
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = s;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kernel, args...);
+}
+#endif
 
 // every kernel launch of the library is counted (process-wide), for throughput reports
 void note_launch();

@@ -67,7 +67,8 @@ __device__ __forceinline__ uint32_t small_div(uint32_t t, uint32_t magic) { retu
 // norm == 1: one block per output channel.  norm == 0: grid-stride over the layer.
 __device__ __forceinline__ void emax_block(const float* __restrict__ w, uint32_t O, uint32_t d,
                                            uint32_t norm, uint32_t* __restrict__ e_max,
-                                           uint32_t* __restrict__ err, uint32_t block, uint32_t blocks) {
+                                           uint32_t* __restrict__ err, uint32_t block, uint32_t blocks,
+                                           uint32_t tag) {
   __shared__ uint32_t red[kThreads / 32];
   uint32_t best = 0;
   bool bad = false;
@@ -93,14 +94,17 @@ __device__ __forceinline__ void emax_block(const float* __restrict__ w, uint32_t
   if (threadIdx.x == 0) {
     for (int i = 1; i < kThreads / 32; ++i) best = max(best, red[i]);
     if (best == 255u) best = 0;  // error already flagged; keep the window well defined
-    if (norm) e_max[block] = best;
-    else if (best) atomicMax(&e_max[0], best);
+    // `tag` (a call number in the bits above the exponent) makes the maxima of this call beat
+    // whatever an earlier call left in the word, so the words need no clearing between calls
+    if (norm) e_max[block] = tag | best;
+    else if (best) atomicMax(&e_max[0], tag | best);
   }
 }
 
 __global__ void emax_kernel(const float* __restrict__ w, uint32_t O, uint32_t d, uint32_t norm,
-                            uint32_t* __restrict__ e_max, uint32_t* __restrict__ err) {
-  emax_block(w, O, d, norm, e_max, err, blockIdx.x, gridDim.x);
+                            uint32_t* __restrict__ e_max, uint32_t* __restrict__ err, uint32_t tag) {
+  pdl_prologue();
+  emax_block(w, O, d, norm, e_max, err, blockIdx.x, gridDim.x, tag);
 }
 
 struct SampleParams {
@@ -113,6 +117,7 @@ struct SampleParams {
   uint32_t bk, n_cb, n_kb;         // operand tiles of the tensor path: K block bytes, blocks per tap, blocks per row
   uint32_t packed_kw, run_pitch;   // packed K (packed_kw = kw, else 0): plane column = kh * run_pitch + kw * Cg + ci
   const uint32_t* e_max;
+  uint32_t e_tag;                  // call number the words of e_max must carry (bits 8 and up)
   int32_t* e_base;
   int32_t* wint[kMaxLevels];
   int8_t* planes[kMaxLevels];
@@ -155,7 +160,9 @@ __device__ __forceinline__ void sample_block(const SampleParams& p, uint32_t blo
 
     const uint32_t E = (u >> 23) & 0xFFu;
     const uint32_t m = u & 0x7FFFFFu;
-    const uint32_t Emax = p.e_max[norm ? o : 0];
+    // a word written by an earlier call (other tag) means this call found no live weight in the group
+    const uint32_t e_word = p.e_max[norm ? o : 0];
+    const uint32_t Emax = (e_word >> 8) == p.e_tag ? (e_word & 0xFFu) : 0u;
     // biased exponents throughout: e - e_base = E - (Emax - span)
     const int ebase_biased = (int)Emax - (int)span;
     if (tap == 0 && ci == 0) p.e_base[o] = Emax ? ebase_biased - 127 : 0;
@@ -215,6 +222,7 @@ __device__ __forceinline__ void sample_block(const SampleParams& p, uint32_t blo
 }
 
 __global__ void __launch_bounds__(kThreads) sample_kernel(const SampleParams p) {
+  pdl_prologue();
   __shared__ float stage[kStage];
   sample_block(p, blockIdx.x, p.seed_lo, p.seed_hi, stage);
 }
@@ -239,13 +247,15 @@ __device__ __forceinline__ uint32_t find_entry(const BatchEntry* __restrict__ e,
 
 __global__ void __launch_bounds__(kThreads) emax_batch_kernel(const BatchEntry* __restrict__ entries, uint32_t n,
                                                               uint32_t* __restrict__ err) {
+  pdl_prologue();
   const BatchEntry& e = entries[find_entry(entries, n, blockIdx.x, true)];
   emax_block(e.p.w, e.p.O, e.p.d, e.p.norm, const_cast<uint32_t*>(e.p.e_max), err,
-             blockIdx.x - e.emax_first, e.emax_blocks);
+             blockIdx.x - e.emax_first, e.emax_blocks, 0u);
 }
 
 __global__ void __launch_bounds__(kThreads) sample_batch_kernel(const BatchEntry* __restrict__ entries, uint32_t n,
                                                                 uint32_t seed_lo, uint32_t seed_hi) {
+  pdl_prologue();
   __shared__ float stage[kStage];
   const BatchEntry& e = entries[find_entry(entries, n, blockIdx.x, false)];
   sample_block(e.p, blockIdx.x - e.sample_first, seed_lo, seed_hi, stage);
@@ -255,6 +265,7 @@ __global__ void __launch_bounds__(kThreads) sample_batch_kernel(const BatchEntry
 // unsigned activations are fed to the signed MMA with an offset of 128.  One warp per row.
 __global__ void corr128_kernel(const int32_t* __restrict__ wint, uint32_t O, uint32_t d,
                                long long* __restrict__ corr) {
+  pdl_prologue();
   const uint32_t row = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31u;
   if (row >= O) return;
   long long sum = 0;
@@ -266,6 +277,7 @@ __global__ void corr128_kernel(const int32_t* __restrict__ wint, uint32_t O, uin
 // Canonical-order copy of one level for the test hook.
 __global__ void export_kernel(const int32_t* __restrict__ wint, int32_t* __restrict__ out, uint32_t O,
                               uint32_t Cg, uint32_t KHKW) {
+  pdl_prologue();
   size_t total = (size_t)O * Cg * KHKW;
   for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < total;
        i += (size_t)gridDim.x * blockDim.x) {
@@ -284,7 +296,8 @@ namespace {
 uint32_t emax_blocks_for(uint32_t O, uint32_t d, uint32_t norm) {
   if (norm) return O;
   size_t total = (size_t)O * d;
-  uint32_t blocks = (uint32_t)((total + kThreads * 8 - 1) / (kThreads * 8));
+  // two weights per thread: the loads of a small layer are all in flight at once
+  uint32_t blocks = (uint32_t)((total + kThreads * 2 - 1) / (kThreads * 2));
   return blocks < 1 ? 1 : (blocks > 1184 ? 1184 : blocks);
 }
 
@@ -323,6 +336,7 @@ uint32_t fill_sample_params(const float* w_dev, const psb_weights* wt, uint32_t*
   p.packed_kw = wt->packed_k ? wt->shape.kw : 0u;
   p.run_pitch = wt->run_pitch;
   p.e_max = e_max;
+  p.e_tag = 0;
   p.e_base = wt->e_base;
   for (int l = 0; l < kMaxLevels; ++l) {
     p.wint[l] = wt->level[l].wint;
@@ -337,20 +351,27 @@ uint32_t fill_sample_params(const float* w_dev, const psb_weights* wt, uint32_t*
 
 cudaError_t launch_corr128(const psb_weights* wt, uint32_t level, cudaStream_t s) {
   const uint32_t O = wt->shape.out_ch;
-  corr128_kernel<<<(O * 32 + kThreads - 1) / kThreads, kThreads, 0, s>>>(wt->level[level].wint, O, wt->d,
-                                                                        wt->level[level].corr128); note_launch();
+  launch_pdl(corr128_kernel, (O * 32 + kThreads - 1) / kThreads, kThreads, 0, s, (const int32_t*)wt->level[level].wint, O,
+             wt->d, wt->level[level].corr128); note_launch();
   return cudaGetLastError();
 }
 
 cudaError_t launch_sampler(const float* w_dev, psb_weights* wt, uint32_t* err_dev, cudaStream_t s) {
   const uint32_t O = wt->shape.out_ch;
-  cudaError_t e = cudaMemsetAsync(wt->e_max, 0, sizeof(uint32_t) * O, s);
-  if (e != cudaSuccess) return e;
-  emax_kernel<<<emax_blocks_for(O, wt->d, wt->cfg.norm), kThreads, 0, s>>>(w_dev, O, wt->d, wt->cfg.norm,
-                                                                          wt->e_max, err_dev); note_launch();
+  // the exponent maxima carry the number of the call that wrote them; the words were cleared when
+  // the handle was made and are cleared again only when the 24-bit call number wraps
+  wt->e_calls = (wt->e_calls + 1u) & 0xFFFFFFu;
+  if (wt->e_calls == 0u) {
+    cudaError_t e = cudaMemsetAsync(wt->e_max, 0, sizeof(uint32_t) * O, s);
+    if (e != cudaSuccess) return e;
+    wt->e_calls = 1u;
+  }
+  launch_pdl(emax_kernel, emax_blocks_for(O, wt->d, wt->cfg.norm), kThreads, 0, s, w_dev, O, wt->d, wt->cfg.norm,
+             wt->e_max, err_dev, wt->e_calls << 8); note_launch();
   SampleParams p;
   const uint32_t blocks = fill_sample_params(w_dev, wt, wt->e_max, p);
-  sample_kernel<<<blocks, kThreads, 0, s>>>(p); note_launch();
+  p.e_tag = wt->e_calls;
+  launch_pdl(sample_kernel, blocks, kThreads, 0, s, p); note_launch();
   return cudaGetLastError();
 }
 
@@ -419,9 +440,11 @@ psb_status sample_batch_create(psb_ctx* ctx, uint32_t n, const float* const* w_d
 psb_status sample_batch_run(psb_ctx* ctx, psb_sample_batch* b, uint64_t seed, cudaStream_t s) {
   if (cudaMemsetAsync(b->e_max_pool, 0, sizeof(uint32_t) * b->e_max_words, s) != cudaSuccess)
     return PSB_ERR_CUDA;
-  emax_batch_kernel<<<b->emax_grid, kThreads, 0, s>>>(b->entries_dev, b->n, ctx->err_dev); note_launch();
-  sample_batch_kernel<<<b->sample_grid, kThreads, 0, s>>>(b->entries_dev, b->n, (uint32_t)seed,
-                                                         (uint32_t)(seed >> 32)); note_launch();
+  launch_pdl(emax_batch_kernel, b->emax_grid, kThreads, 0, s, (const BatchEntry*)b->entries_dev, b->n, ctx->err_dev);
+  note_launch();
+  launch_pdl(sample_batch_kernel, b->sample_grid, kThreads, 0, s, (const BatchEntry*)b->entries_dev, b->n, (uint32_t)seed,
+             (uint32_t)(seed >> 32));
+  note_launch();
   return cudaGetLastError() == cudaSuccess ? PSB_OK : PSB_ERR_CUDA;
 }
 
@@ -478,6 +501,7 @@ sample_level_canonical_kernel(const float* __restrict__ w, uint32_t O, uint32_t 
                               uint32_t span, uint32_t log2k, uint32_t seed_lo, uint32_t seed_hi,
                               uint32_t layer_id, const uint32_t* __restrict__ e_max,
                               int32_t* __restrict__ wint_out, int32_t* __restrict__ e_base_out) {
+  pdl_prologue();
   const size_t total = (size_t)O * d;
   for (size_t index = (size_t)blockIdx.x * blockDim.x + threadIdx.x; index < total;
        index += (size_t)gridDim.x * blockDim.x) {
@@ -546,12 +570,12 @@ extern "C" psb_status psb_sample_level_static(const float* w_dev, const psb_wsha
   // the array keeps the previous call's maxima: the reduction must start from zero
   if (cudaMemsetAsync(e_max, 0, sizeof(uint32_t) * O, s) != cudaSuccess) return PSB_ERR_CUDA;
   if (cfg->norm) {
-    emax_kernel<<<O, kThreads, 0, s>>>(w_dev, O, d, 1, e_max, err_sink); note_launch();
+    emax_kernel<<<O, kThreads, 0, s>>>(w_dev, O, d, 1, e_max, err_sink, 0u); note_launch();
   } else {
     size_t total = (size_t)O * d;
     uint32_t blocks = (uint32_t)((total + kThreads * 8 - 1) / (kThreads * 8));
     blocks = blocks < 1 ? 1 : (blocks > 1184 ? 1184 : blocks);
-    emax_kernel<<<blocks, kThreads, 0, s>>>(w_dev, O, d, 0, e_max, err_sink); note_launch();
+    emax_kernel<<<blocks, kThreads, 0, s>>>(w_dev, O, d, 0, e_max, err_sink, 0u); note_launch();
   }
   size_t total = (size_t)O * d;
   uint32_t blocks = (uint32_t)((total + kThreads - 1) / kThreads);

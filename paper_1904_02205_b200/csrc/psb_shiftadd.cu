@@ -36,6 +36,7 @@ __device__ __forceinline__ void store_outputs(const ConvArgs& a, size_t oidx, ui
 // One thread per output element, output channel fastest.  For depthwise filters
 // (one input channel per group) neighbouring threads read neighbouring bytes.
 __global__ void __launch_bounds__(256) conv_direct_kernel(const ConvArgs a, const WintTable wt) {
+  pdl_prologue();
   const size_t total = (size_t)a.N * a.OH * a.OW * a.O;
   const uint32_t Cg = a.C / a.groups, Og = a.O / a.groups;
   for (size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x; idx < total;
@@ -77,6 +78,7 @@ __global__ void __launch_bounds__(256) conv_direct_kernel(const ConvArgs a, cons
 // layer's integer filter in shared memory as [tap][channel]; activations come in 8-byte loads;
 // the integer sum x * W_k over the taps is Eq. 9 summed over the draws.  Writes 8 codes at once.
 __global__ void __launch_bounds__(256) dwconv_nhwc8_kernel(const ConvArgs a, const int32_t* __restrict__ wint) {
+  pdl_prologue();
   extern __shared__ int32_t dw_w[];   // [KH*KW][C]
   const uint32_t taps = a.KH * a.KW, C = a.C;
   for (uint32_t i = threadIdx.x; i < taps * C; i += blockDim.x) dw_w[(i % taps) * C + i / taps] = wint[i];
@@ -147,6 +149,7 @@ struct DwSeg { static constexpr int kOut = S == 1 ? 8 : 4; static constexpr int 
 
 template <int S, bool kSignedIn>
 __global__ void __launch_bounds__(256, 2) dwconv3x3_row_kernel(const ConvArgs a, const int32_t* __restrict__ wint) {
+  pdl_prologue();
   constexpr int L = DwSeg<S>::kOut, NC = DwSeg<S>::kCols;
   const uint32_t C = a.C, G = C / 4u;
   const uint32_t segs = (a.OW + L - 1) / L;
@@ -240,6 +243,7 @@ __global__ void __launch_bounds__(256, 2) dwconv3x3_row_kernel(const ConvArgs a,
 
 // x ^ 0x80 over a whole tensor: unsigned bytes become (x - 128) as signed bytes, 16 per thread.
 __global__ void offset128_kernel(const uint4* __restrict__ src, uint4* __restrict__ dst, size_t n16) {
+  pdl_prologue();
   for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n16; i += (size_t)gridDim.x * blockDim.x) {
     uint4 v = __ldg(src + i);
     v.x ^= 0x80808080u; v.y ^= 0x80808080u; v.z ^= 0x80808080u; v.w ^= 0x80808080u;
@@ -261,6 +265,7 @@ constexpr uint32_t kIm2colPix = 32;
 __global__ void __launch_bounds__(256) im2col_s8_kernel(const ConvArgs a, uint32_t kpad, uint32_t run_pitch,
                                                        uint32_t offset, uint32_t span_bytes, uint32_t span_pitch,
                                                        int8_t* __restrict__ dst) {
+  pdl_prologue();
   extern __shared__ uint32_t im2col_smem[];                   // [KH][span_pitch / 4] words
   uint8_t* rows = reinterpret_cast<uint8_t*>(im2col_smem);
   const uint32_t strips = (a.OW + kIm2colPix - 1) / kIm2colPix;
@@ -320,6 +325,7 @@ __global__ void __launch_bounds__(256) im2col_s8_kernel(const ConvArgs a, uint32
 // [N][C][HW] -> [N][HW][C], elements of 1 byte, through a 32x33 tile.
 __global__ void nchw_to_nhwc_u8_kernel(const uint8_t* __restrict__ src, uint8_t* __restrict__ dst,
                                        uint32_t C, uint32_t HW) {
+  pdl_prologue();
   __shared__ uint8_t tile[32][33];
   const size_t base = (size_t)blockIdx.z * C * HW;
   const uint32_t p0 = blockIdx.x * 32, c0 = blockIdx.y * 32;
@@ -343,6 +349,7 @@ __global__ void nchw_to_nhwc_u8_kernel(const uint8_t* __restrict__ src, uint8_t*
 __global__ void __launch_bounds__(256) nchw_to_nhwc_u8x4_kernel(const uint8_t* __restrict__ src,
                                                                uint8_t* __restrict__ dst, uint32_t C,
                                                                uint32_t HW) {
+  pdl_prologue();
   __shared__ __align__(16) uint32_t tile[8][132];
   const size_t base = (size_t)blockIdx.z * C * HW;
   const uint32_t p0 = blockIdx.x * 128u, c0 = blockIdx.y * 32u;
@@ -374,6 +381,7 @@ __global__ void __launch_bounds__(256) nchw_to_nhwc_u8x4_kernel(const uint8_t* _
 __global__ void maxpool_kernel(const uint8_t* __restrict__ x, uint32_t nchw, uint32_t N, uint32_t C,
                                uint32_t H, uint32_t W, uint32_t k, uint32_t stride, uint32_t pad,
                                uint32_t OH, uint32_t OW, uint8_t* __restrict__ out) {
+  pdl_prologue();
   const size_t total = (size_t)N * OH * OW * C;
   for (size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x; idx < total;
        idx += (size_t)gridDim.x * blockDim.x) {
@@ -406,6 +414,7 @@ __global__ void __launch_bounds__(256) maxpool_nhwc16_kernel(const uint8_t* __re
                                                             uint32_t H, uint32_t W, uint32_t k, uint32_t stride,
                                                             uint32_t pad, uint32_t OH, uint32_t OW,
                                                             uint8_t* __restrict__ out) {
+  pdl_prologue();
   const uint32_t groups = C / 16u;
   const size_t total = (size_t)N * OH * OW * groups;
   for (size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x; idx < total;
@@ -434,6 +443,7 @@ __global__ void __launch_bounds__(256) maxpool_nhwc16_kernel(const uint8_t* __re
 __global__ void avgpool_kernel(const uint8_t* __restrict__ x, uint32_t nchw, uint32_t N, uint32_t C,
                                uint32_t HW, float pool_mul, int qmin, int qmax,
                                uint8_t* __restrict__ out) {
+  pdl_prologue();
   const uint32_t warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
   if (warp >= N * C) return;
   const uint32_t n = warp / C, c = warp % C;
@@ -457,7 +467,7 @@ uint32_t grid_for(size_t total, uint32_t threads) {
 
 cudaError_t launch_offset128(const void* src, void* dst, size_t bytes, cudaStream_t s) {
   const size_t n16 = bytes / 16;
-  offset128_kernel<<<grid_for(n16, 256), 256, 0, s>>>((const uint4*)src, (uint4*)dst, n16); note_launch();
+  launch_pdl(offset128_kernel, grid_for(n16, 256), 256, 0, s, (const uint4*)src, (uint4*)dst, n16); note_launch();
   return cudaGetLastError();
 }
 
@@ -483,11 +493,11 @@ cudaError_t launch_shift_add(const ConvArgs& a, const WintTable& wt, cudaStream_
         const int32_t* wl = wt.w[a.uniform_log2k];
         const bool sg = a.in_dtype == PSB_DT_S8;
         if (a.stride == 1) {
-          if (sg) dwconv3x3_row_kernel<1, true><<<blocks, 256, 0, s>>>(a, wl);
-          else dwconv3x3_row_kernel<1, false><<<blocks, 256, 0, s>>>(a, wl);
+          if (sg) launch_pdl(dwconv3x3_row_kernel<1, true>, blocks, 256, 0, s, a, wl);
+          else launch_pdl(dwconv3x3_row_kernel<1, false>, blocks, 256, 0, s, a, wl);
         } else {
-          if (sg) dwconv3x3_row_kernel<2, true><<<blocks, 256, 0, s>>>(a, wl);
-          else dwconv3x3_row_kernel<2, false><<<blocks, 256, 0, s>>>(a, wl);
+          if (sg) launch_pdl(dwconv3x3_row_kernel<2, true>, blocks, 256, 0, s, a, wl);
+          else launch_pdl(dwconv3x3_row_kernel<2, false>, blocks, 256, 0, s, a, wl);
         }
         note_launch();
         return cudaGetLastError();
@@ -495,10 +505,10 @@ cudaError_t launch_shift_add(const ConvArgs& a, const WintTable& wt, cudaStream_
     }
     uint32_t blocks = grid_for(total / 8, 256);
     if (blocks > 148u * 4u) blocks = 148u * 4u;
-    dwconv_nhwc8_kernel<<<blocks, 256, dw_smem, s>>>(a, wt.w[a.uniform_log2k]); note_launch();
+    launch_pdl(dwconv_nhwc8_kernel, blocks, 256, dw_smem, s, a, wt.w[a.uniform_log2k]); note_launch();
     return cudaGetLastError();
   }
-  conv_direct_kernel<<<grid_for(total, 256), 256, 0, s>>>(a, wt); note_launch();
+  launch_pdl(conv_direct_kernel, grid_for(total, 256), 256, 0, s, a, wt); note_launch();
   return cudaGetLastError();
 }
 
@@ -512,7 +522,7 @@ cudaError_t launch_im2col_s8(const ConvArgs& a, uint32_t kpad, uint32_t run_pitc
   if (smem > 48 * 1024 || (uint64_t)a.N * a.OH * strips >= (1ull << 31) || run_pitch % 8u || kpad % 16u ||
       (offset != 0u && offset != 128u) || a.KH * run_pitch > kpad)
     return cudaErrorInvalidValue;
-  im2col_s8_kernel<<<a.N * a.OH * strips, 256, smem, s>>>(a, kpad, run_pitch, offset, span_bytes, span_pitch, dst);
+  launch_pdl(im2col_s8_kernel, a.N * a.OH * strips, 256, smem, s, a, kpad, run_pitch, offset, span_bytes, span_pitch, dst);
   note_launch();
   return cudaGetLastError();
 }
@@ -522,10 +532,10 @@ cudaError_t launch_nchw_to_nhwc(const void* src, void* dst, uint32_t N, uint32_t
   if (elem_bytes != 1) return cudaErrorInvalidValue;
   if (C % 4u == 0 && HW % 4u == 0 && !(((uintptr_t)src | (uintptr_t)dst) & 3u)) {
     dim3 grid4((HW + 127) / 128, (C + 31) / 32, N);
-    nchw_to_nhwc_u8x4_kernel<<<grid4, 256, 0, s>>>((const uint8_t*)src, (uint8_t*)dst, C, HW);
+    launch_pdl(nchw_to_nhwc_u8x4_kernel, grid4, 256, 0, s, (const uint8_t*)src, (uint8_t*)dst, C, HW);
   } else {
     dim3 grid((HW + 31) / 32, (C + 31) / 32, N), block(32, 8);
-    nchw_to_nhwc_u8_kernel<<<grid, block, 0, s>>>((const uint8_t*)src, (uint8_t*)dst, C, HW);
+    launch_pdl(nchw_to_nhwc_u8_kernel, grid, block, 0, s, (const uint8_t*)src, (uint8_t*)dst, C, HW);
   }
   note_launch();
   return cudaGetLastError();
@@ -537,9 +547,9 @@ cudaError_t launch_maxpool(const uint8_t* x, uint32_t nchw, uint32_t N, uint32_t
   uint32_t OH = (H + 2 * pad - k) / stride + 1, OW = (W + 2 * pad - k) / stride + 1;
   size_t total = (size_t)N * OH * OW * C;
   if (!nchw && C % 16u == 0 && !(((uintptr_t)x | (uintptr_t)out) & 15u))
-    maxpool_nhwc16_kernel<<<grid_for(total / 16, 256), 256, 0, s>>>(x, N, C, H, W, k, stride, pad, OH, OW, out);
+    launch_pdl(maxpool_nhwc16_kernel, grid_for(total / 16, 256), 256, 0, s, x, N, C, H, W, k, stride, pad, OH, OW, out);
   else
-    maxpool_kernel<<<grid_for(total, 256), 256, 0, s>>>(x, nchw, N, C, H, W, k, stride, pad, OH, OW, out);
+    launch_pdl(maxpool_kernel, grid_for(total, 256), 256, 0, s, x, nchw, N, C, H, W, k, stride, pad, OH, OW, out);
   note_launch();
   return cudaGetLastError();
 }
@@ -549,7 +559,7 @@ cudaError_t launch_avgpool(const uint8_t* x, uint32_t nchw, uint32_t N, uint32_t
                            cudaStream_t s) {
   size_t warps = (size_t)N * C;
   uint32_t blocks = (uint32_t)((warps * 32 + 255) / 256);
-  avgpool_kernel<<<blocks, 256, 0, s>>>(x, nchw, N, C, H * W, pool_mul, qmin, qmax, out); note_launch();
+  launch_pdl(avgpool_kernel, blocks, 256, 0, s, x, nchw, N, C, H * W, pool_mul, qmin, qmax, out); note_launch();
   return cudaGetLastError();
 }
 

@@ -154,8 +154,12 @@ class ConvWorkload:
         ops = 2.0 * self.macs * self.planes
         achieved = ops / (kernel_ms * 1e-3) / 1e12
         peak = 2.0 * peaks["bf16_tflops"]
+        # DRAM bytes of one launch from the ncu capture summarised in profiles/psb_mma_kernel_conv3x3_b32.md
+        # (dram__bytes_read.sum + dram__bytes_write.sum; k does not change them); to be set back to None
+        # whenever the kernel changes before the counters are taken again
         return dict(bound="tensor", kernel="psb_mma_kernel", achieved=achieved, peak=peak, unit="TOP/s (int8)",
-                    frac=achieved / peak, traffic=None, peak_source=peaks["source"] + " bf16 burst x 2",
+                    frac=achieved / peak, traffic=6.63e6, traffic_unit="bytes per launch (ncu)",
+                    peak_source=peaks["source"] + " bf16 burst x 2",
                     planes=self.planes, logical_gmacs=self.macs / (kernel_ms * 1e-3) / 1e9,
                     kernel_ms=kernel_ms)
 

@@ -381,7 +381,9 @@ def main():
         return run_int8_probe(ctx, local_rank)
     wl = make_workload(args, rank)
     wl.setup(ctx, psb, torch)
-    flush = torch.empty(512 << 20, dtype=torch.uint8, device=ctx.device)   # > L2 (126 MB)
+    # > L2 (126 MB); writing it also takes long enough (about 0.2 ms) for the host to have queued the whole
+    # step behind it, so that the events see device time and not the host's launch rate
+    flush = torch.empty(1 << 30, dtype=torch.uint8, device=ctx.device)
 
     def timed(fn, n, first=0):
         ms = []
@@ -428,7 +430,7 @@ def main():
     line = dict(metric=METRIC, value=value, unit=UNIT, n_gpus=world, steps=args.steps, warmup=args.warmup,
                 ms_per_step=sec * 1e3 / args.steps, higher_is_better=True, scaling="weak", vs_baseline=None,
                 dtype="int8 digits, int64 accumulators", data="synthetic",
-                config=dict(workload=wl.name, k=args.k, l2="flushed between steps (512 MiB memset, untimed)",
+                config=dict(workload=wl.name, k=args.k, l2="flushed between steps (1 GiB memset, untimed)",
                             images_per_step=wl.images * world, sampler="inside the timed step, fresh seed per step"),
                 images_per_s=wl.images * world * args.steps / sec,
                 gated_add_equiv_per_s=units * getattr(wl, "mean_k", args.k) / sec,

@@ -381,6 +381,11 @@ __device__ __forceinline__ void store_row16(uint8_t* dst, uint4 v, bool vec16, b
 // The same 16 channels of one output location in a planar ([n][o][oy][ox]) tensor: byte j sits
 // j * plane further on.  Lanes of a warp hold consecutive locations, so each of the 16 accesses
 // is a contiguous run of 32 bytes per warp.
+// (Out of line to keep the callers' loops small.  The registers such a function may use are what all
+// of its callers can spare, so each caller family gets its own instance, selected by TAG: when the
+// plain output-stage loop, which holds more live values, shared one instance with the band-mode loop,
+// the byte loop of the store spilled and band mode with planar output lost a third of its speed.)
+template <int TAG>
 __device__ __noinline__ uint4 load_planar16(const uint8_t* src, size_t plane, uint32_t count) {
   uint32_t w[4] = {0u, 0u, 0u, 0u};
 #pragma unroll
@@ -388,6 +393,7 @@ __device__ __noinline__ uint4 load_planar16(const uint8_t* src, size_t plane, ui
     if ((uint32_t)j < count) w[j >> 2] |= (uint32_t)__ldg(src + (size_t)j * plane) << (8 * (j & 3));
   return make_uint4(w[0], w[1], w[2], w[3]);
 }
+template <int TAG>
 __device__ __noinline__ void store_planar16(uint8_t* dst, size_t plane, uint32_t count, uint4 v) {
   const uint32_t w[4] = {v.x, v.y, v.z, v.w};
 #pragma unroll
@@ -486,6 +492,27 @@ __device__ __forceinline__ uint32_t tile_row_index(const TensorParams& p, uint32
   return (n * p.a.OH + oy) * p.a.OW + ox;
 }
 
+// The same two functions on register copies of the few parameters they need.  Inside an out-of-line
+// function the kernel's parameter block is reached through a generic pointer, and every asm statement
+// with a memory clobber (barrier waits, TMEM loads) makes the compiler fetch such fields again: a
+// dozen dependent loads per tile in the output-stage loop before the copies were made.  (Plain mode.)
+struct RowMap {
+  uint32_t M, O, ohow, planar;
+  __device__ __forceinline__ void init(const TensorParams& p) {
+    M = p.M; O = p.a.O; ohow = p.a.OH * p.a.OW; planar = p.a.out_nchw;
+  }
+  __device__ __forceinline__ uint32_t row_index(uint32_t m_tile, uint32_t row, bool* valid) const {
+    const uint32_t m = m_tile * kTileM + row;
+    *valid = m < M;
+    return m;
+  }
+  __device__ __forceinline__ size_t offset(uint32_t m, uint32_t o_base) const {
+    if (!planar) return (size_t)m * O + o_base;
+    const uint32_t n = m / ohow;
+    return ((size_t)n * O + o_base) * ohow + (m - n * ohow);
+  }
+};
+
 // Epilogue loop of one warp for the common case: one draw count for the whole layer, only
 // re-quantised bytes wanted.  The warp owns 32 rows (its TMEM lane quarter) x 16 channels of
 // every tile.  Per tile: wait for the accumulator, pull the chunk into registers, hand the TMEM
@@ -493,6 +520,99 @@ __device__ __forceinline__ uint32_t tile_row_index(const TensorParams& p, uint32
 // the store.  Shortcut bytes are fetched one tile ahead.  Returns true if a wait timed out.
 template <int P, int MODE, bool HAS_RES>
 __device__ __noinline__ bool epilogue_uniform(const TensorParams& p, SharedCtl* ctl, uint32_t tmem_base,
+                                              uint32_t ew, uint32_t lane, EpiConst c) {
+  const ConvArgs& a = p.a;
+  const uint32_t quarter = ew & 3u, sub = ew >> 2;
+  const uint32_t row = quarter * 32u + lane;
+  const uint32_t l = a.uniform_log2k;
+  const bool use_corr = p.corr[l] != nullptr;
+  volatile uint32_t* abort = &ctl->abort;
+  const uint8_t* const res_base = (const uint8_t*)a.residual;
+  uint8_t* const q_base = (uint8_t*)a.q_out;
+  RowMap rm;
+  rm.init(p);
+  const float2* scb = ctl->scb[ew];
+  const long long* corr = ctl->corr[ew];
+  const bool vec16 = p.vec_ok == 2u, planar = rm.planar != 0u;
+  const uint32_t ohow = rm.ohow;
+  TileIter ti;
+  ti.init(p);
+  uint32_t pass = 0, cur_o_tile = 0xFFFFFFFFu;
+  uint4 r_next = make_uint4(0, 0, 0, 0);
+  if (HAS_RES && ti.valid()) {
+    bool ok_row;
+    const uint32_t m = rm.row_index(ti.m_tile, row, &ok_row), ob = ti.o_tile * kTileN + sub * 16u;
+    if (ok_row && ob < rm.O) {
+      const uint8_t* src = res_base + rm.offset(m, ob);
+      r_next = planar ? load_planar16<1>(src, ohow, rm.O - ob) : load_row16(src, vec16, ob + 16u <= rm.O);
+    }
+  }
+  while (ti.valid()) {
+    bool row_valid;
+    const uint32_t m = rm.row_index(ti.m_tile, row, &row_valid);
+    const uint32_t o_tile = ti.o_tile;
+    const uint32_t o_base = o_tile * kTileN + sub * 16u;
+    const bool active = o_base < rm.O;          // warp-uniform
+    ti.next();
+    if (o_tile != cur_o_tile) {
+      // per-channel constants of this channel tile: the warp keeps its own copy of its 16 channels
+      __syncwarp();
+      if (lane < 16u) {
+        const uint32_t o = o_base + lane;
+        float2 sb = make_float2(0.f, 0.f);
+        long long cr = 0;
+        if (o < a.O) {
+          sb.x = ldexpf(a.scale[o], a.e_base[o] - (int)l);
+          sb.y = a.bias[o];
+          if (use_corr) cr = p.corr[l][o];
+        }
+        ctl->scb[ew][lane] = sb;
+        ctl->corr[ew][lane] = cr;
+      }
+      cur_o_tile = o_tile;
+      __syncwarp();
+    }
+    const uint4 r_cur = r_next;
+    if (HAS_RES && ti.valid()) {
+      bool ok_row;
+      const uint32_t mn = rm.row_index(ti.m_tile, row, &ok_row), ob = ti.o_tile * kTileN + sub * 16u;
+      r_next = make_uint4(0, 0, 0, 0);
+      if (ok_row && ob < rm.O) {
+        const uint8_t* src = res_base + rm.offset(mn, ob);
+        r_next = planar ? load_planar16<1>(src, ohow, rm.O - ob) : load_row16(src, vec16, ob + 16u <= rm.O);
+      }
+    }
+    const uint32_t buf = pass & 1u, aph = (pass >> 1) & 1u;
+    const bool ok = mbar_wait(smem_u32(&ctl->acc_full[buf]), aph, abort, 32);
+    if (__any_sync(0xFFFFFFFFu, !ok)) return true;
+    tc_fence_after();
+    uint32_t v[P][16];
+    if (active) {
+      const uint32_t taddr = tmem_base + buf * kTmemBufStride + ((quarter * 32u) << 16) + sub * 16u;
+#pragma unroll
+      for (int pl = 0; pl < P; ++pl) tc_ld16(taddr + pl * kTileN, v[pl]);
+      tc_wait_ld();
+    }
+    // the chunk is in registers: give the accumulator buffer back before doing the arithmetic
+    tc_fence_before();
+    __syncwarp();
+    if (lane == 0) mbar_arrive(smem_u32(&ctl->acc_empty[buf]));
+    if (active && row_valid) {
+      const uint4 q16 = chunk_math<P, MODE, HAS_RES>(v, r_cur, scb, corr, c);
+      uint8_t* dst = q_base + rm.offset(m, o_base);
+      if (planar) store_planar16<1>(dst, ohow, rm.O - o_base, q16);
+      else store_row16(dst, q16, vec16, o_base + 16u <= rm.O);
+    }
+    ++pass;
+  }
+  return false;
+}
+
+// The same loop for band mode, reading the parameter block where it needs it: band mode's index
+// arithmetic wants eight more fields, and holding them in registers made the loop spill more than the
+// loads cost.
+template <int P, int MODE, bool HAS_RES>
+__device__ __noinline__ bool epilogue_uniform_band(const TensorParams& p, SharedCtl* ctl, uint32_t tmem_base,
                                               uint32_t ew, uint32_t lane, EpiConst c) {
   const ConvArgs& a = p.a;
   const uint32_t quarter = ew & 3u, sub = ew >> 2;
@@ -514,7 +634,7 @@ __device__ __noinline__ bool epilogue_uniform(const TensorParams& p, SharedCtl* 
     const uint32_t m = tile_row_index(p, ti.m_tile, row, &ok_row), ob = ti.o_tile * kTileN + sub * 16u;
     if (ok_row && ob < a.O) {
       const uint8_t* src = res_base + out_offset(a, ohow, m, ob);
-      r_next = planar ? load_planar16(src, ohow, a.O - ob) : load_row16(src, vec16, ob + 16u <= a.O);
+      r_next = planar ? load_planar16<0>(src, ohow, a.O - ob) : load_row16(src, vec16, ob + 16u <= a.O);
     }
   }
   while (ti.valid()) {
@@ -549,7 +669,7 @@ __device__ __noinline__ bool epilogue_uniform(const TensorParams& p, SharedCtl* 
       r_next = make_uint4(0, 0, 0, 0);
       if (ok_row && ob < a.O) {
         const uint8_t* src = res_base + out_offset(a, ohow, mn, ob);
-        r_next = planar ? load_planar16(src, ohow, a.O - ob) : load_row16(src, vec16, ob + 16u <= a.O);
+        r_next = planar ? load_planar16<0>(src, ohow, a.O - ob) : load_row16(src, vec16, ob + 16u <= a.O);
       }
     }
     const uint32_t buf = pass & 1u, aph = (pass >> 1) & 1u;
@@ -570,7 +690,7 @@ __device__ __noinline__ bool epilogue_uniform(const TensorParams& p, SharedCtl* 
     if (active && row_valid) {
       const uint4 q16 = chunk_math<P, MODE, HAS_RES>(v, r_cur, scb, corr, c);
       uint8_t* dst = (uint8_t*)a.q_out + out_offset(a, ohow, m, o_base);
-      if (planar) store_planar16(dst, ohow, a.O - o_base, q16);
+      if (planar) store_planar16<0>(dst, ohow, a.O - o_base, q16);
       else store_row16(dst, q16, vec16, o_base + 16u <= a.O);
     }
     ++pass;
@@ -859,7 +979,9 @@ psb_mma_kernel(const __grid_constant__ TmapSet maps, const __grid_constant__ Ten
     }
     if (uniform_epilogue(p)) {
       const uint32_t mode = (p.corr[a.uniform_log2k] != nullptr || P0 == 4u) ? 0u : p.narrow;
-#define PSB_UNI(PV, MV, RV) failed = epilogue_uniform<PV, MV, RV>(p, ctl, tmem_base, ew, lane, ec)
+#define PSB_UNI(PV, MV, RV)                                                                   \
+  failed = p.band ? epilogue_uniform_band<PV, MV, RV>(p, ctl, tmem_base, ew, lane, ec)        \
+                  : epilogue_uniform<PV, MV, RV>(p, ctl, tmem_base, ew, lane, ec)
       if (a.residual) {
         if (P0 == 4u) PSB_UNI(4, 0, true); else if (mode == 3u) PSB_UNI(3, 3, true); else if (mode == 2u) PSB_UNI(3, 2, true);
         else if (mode == 1u) PSB_UNI(3, 1, true); else PSB_UNI(3, 0, true);

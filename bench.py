@@ -412,6 +412,16 @@ def main():
     if world > 1:
         dist.barrier()
     kern_ms = timed(lambda i: wl.kernel_only(), max(args.steps, 10) if args.workload == "conv3x3" else 4)
+    in_step_ms = []
+    if args.workload == "conv3x3":
+        # the same steps once more with the library's own pair of events around the contraction kernel:
+        # its duration inside the step (filters and converted input just written, output planar)
+        ctx.contraction_timing(True)
+        for i in range(max(args.steps, 10)):
+            flush.zero_()
+            wl.step(args.warmup + args.steps + i)
+            in_step_ms.append(ctx.contraction_time())
+        ctx.contraction_timing(False)
     clk = clocks.stop()
     ctx.check_device()
     e2e_warm = timed(wl.e2e_step, 3)
@@ -438,6 +448,10 @@ def main():
                 e2e=dict(value=e2e_units / e2e_sec / 1e9, unit=UNIT, h2d_bytes_per_step=wl.e2e_h2d,
                          d2h_bytes_per_step=wl.e2e_d2h),
                 roofline=wl.roofline(statistics.mean(kern_ms), peaks))
+    if in_step_ms:
+        # for comparison: the same kernel inside the step, where it writes planar output and, with the events
+        # around it, cannot start under the conversion kernel's tail (an empty pair of events reads 2.7 us)
+        line["roofline"]["kernel_ms_in_step_planar_out"] = statistics.mean(in_step_ms)
     if not args.no_cpu_baseline and world == 1:
         dt, macs, sample = wl.oracle_sample(getattr(wl, "oracle_images", 4))
         line["cpu_baseline"] = dict(value=macs / dt / 1e9, unit=UNIT, cores=1, kind="oracle", sample=sample)

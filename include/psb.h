@@ -213,6 +213,17 @@ int32_t psb_last_path(const psb_ctx* ctx);
  * many launches a timed region took.  Never fails. */
 uint64_t psb_launch_count(void);
 
+/* Measurement aid, no counterpart in the paper: device time of the tensor-core
+ * contraction kernel inside a larger step.  With `enable` != 0 every launch of
+ * that kernel by this context is bracketed by a pair of CUDA events on its
+ * stream (which also keeps it from starting under its predecessor's tail, so a
+ * step runs a little slower while this is on); psb_contraction_time waits for
+ * the end of the most recent such launch and returns its duration in
+ * milliseconds.  PSB_ERR_INVALID_ARG for null arguments or when no launch has
+ * been timed yet, PSB_ERR_CUDA if the events cannot be created or read. */
+psb_status psb_contraction_timing(psb_ctx* ctx, uint32_t enable);
+psb_status psb_contraction_time(psb_ctx* ctx, float* milliseconds);
+
 /* Measurement aid, no counterpart in the paper: the ceiling of the dense path.
  * Every SM issues `groups` groups of four back-to-back tcgen05.mma kind::i8
  * instructions (M = 128, N = n_cols, K = 32, s8 x s8 -> s32 in TMEM) on zero

@@ -24,7 +24,7 @@ EXPORTS = ["psb_create", "psb_destroy", "psb_status_string", "psb_device_status"
            "psb_weights_export", "psb_weights_free", "psb_set_sample_map", "psb_conv2d", "psb_gemm",
            "psb_last_path", "psb_maxpool2d_u8", "psb_global_avgpool_u8", "psb_sample_level_static",
            "psb_sample_batch_create", "psb_sample_batch_run", "psb_sample_batch_free", "psb_run",
-           "psb_launch_count", "psb_int8_mma_probe"]
+           "psb_launch_count", "psb_int8_mma_probe", "psb_contraction_timing", "psb_contraction_time"]
 
 
 class psb_wshape(C.Structure):
@@ -91,6 +91,8 @@ def load_library():
     lib.psb_gemm.argtypes = [vp, vp, vp, C.POINTER(psb_gemm_desc), vp]
     lib.psb_last_path.argtypes = [vp]
     lib.psb_int8_mma_probe.argtypes = [vp, u32, u32, C.POINTER(C.c_double), C.POINTER(C.c_double), vp]
+    lib.psb_contraction_timing.argtypes = [vp, u32]
+    lib.psb_contraction_time.argtypes = [vp, C.POINTER(C.c_float)]
     lib.psb_launch_count.argtypes = []
     lib.psb_launch_count.restype = C.c_uint64
     lib.psb_maxpool2d_u8.argtypes = [vp, vp, u32, u32, u32, u32, u32, u32, u32, u32, vp, vp]
@@ -207,6 +209,16 @@ class Context:
         _check(self.lib.psb_int8_mma_probe(self.handle, n_cols, groups, C.byref(a), C.byref(b), _stream(stream)),
                "psb_int8_mma_probe")
         return a.value, b.value
+
+    def contraction_timing(self, enable):
+        """Bracket every launch of the contraction kernel with CUDA events (measurement aid)."""
+        _check(self.lib.psb_contraction_timing(self.handle, 1 if enable else 0), "psb_contraction_timing")
+
+    def contraction_time(self):
+        """Device time in milliseconds of the most recent timed contraction launch (waits for it)."""
+        ms = C.c_float(0.0)
+        _check(self.lib.psb_contraction_time(self.handle, C.byref(ms)), "psb_contraction_time")
+        return float(ms.value)
 
     def launch_count(self):
         """Kernels launched by the library in this process so far."""

@@ -227,6 +227,8 @@ psb_status psb_destroy(psb_ctx* ctx) {
   for (int i = 0; i < 3; ++i)
     if (ctx->scratch[i]) cudaFree(ctx->scratch[i]);
   if (ctx->err_dev) cudaFree(ctx->err_dev);
+  if (ctx->t_begin) cudaEventDestroy(ctx->t_begin);
+  if (ctx->t_end) cudaEventDestroy(ctx->t_end);
   delete ctx;
   return PSB_OK;
 }
@@ -386,6 +388,29 @@ psb_status psb_gemm(psb_ctx* ctx, const psb_weights* weights, const void* x_dev,
 int32_t psb_last_path(const psb_ctx* ctx) { return ctx ? ctx->last_path : 0; }
 
 uint64_t psb_launch_count(void) { return (uint64_t)psb::launches_so_far(); }
+
+psb_status psb_contraction_timing(psb_ctx* ctx, uint32_t enable) {
+  if (!ctx) return PSB_ERR_INVALID_ARG;
+  if (enable && !ctx->t_begin) {
+    cudaSetDevice(ctx->device);
+    if (cudaEventCreate(&ctx->t_begin) != cudaSuccess || cudaEventCreate(&ctx->t_end) != cudaSuccess) {
+      cudaGetLastError();
+      return PSB_ERR_CUDA;
+    }
+  }
+  ctx->time_contraction = enable != 0;
+  return PSB_OK;
+}
+
+psb_status psb_contraction_time(psb_ctx* ctx, float* milliseconds) {
+  if (!ctx || !milliseconds || !ctx->contraction_timed) return PSB_ERR_INVALID_ARG;
+  if (cudaEventSynchronize(ctx->t_end) != cudaSuccess ||
+      cudaEventElapsedTime(milliseconds, ctx->t_begin, ctx->t_end) != cudaSuccess) {
+    cudaGetLastError();
+    return PSB_ERR_CUDA;
+  }
+  return PSB_OK;
+}
 
 psb_status psb_int8_mma_probe(psb_ctx* ctx, uint32_t n_cols, uint32_t groups, double* mac_per_clk_per_sm,
                               double* tera_ops_per_s, void* stream) {

@@ -84,6 +84,9 @@ struct psb_ctx {
   int sm_count = 0;
   void* encode_tiled = nullptr;     // cuTensorMapEncodeTiled
   void* encode_im2col = nullptr;    // cuTensorMapEncodeIm2col
+  bool time_contraction = false;    // bracket the contraction kernel with the two events below
+  bool contraction_timed = false;   // a pair has been recorded
+  cudaEvent_t t_begin = nullptr, t_end = nullptr;
 };
 
 namespace psb {

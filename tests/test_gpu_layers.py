@@ -437,6 +437,21 @@ def test_pooling_kernels(psb, ctx, oracle):
                               oracle.global_avgpool_u8(x, layout, np.float32(0.0123), 0, 255))
 
 
+def test_contraction_timing_hook(psb, oracle):
+    """The measurement hook brackets the tensor-core kernel with events; results are unchanged by it."""
+    c = psb.Context(0)
+    with pytest.raises(psb.PsbError):
+        c.contraction_time()                      # nothing timed yet
+    rng = np.random.default_rng(31)
+    w, x, scale, bias = _layer_inputs(rng, 2, 64, 12, 12, 64, 3, 3, 1, 1)
+    c.contraction_timing(True)
+    _both(psb, c, oracle, w, x, 1, 1, 1, 1, [3], scale, bias, in_max=15, path=psb.PSB_PATH_TENSOR, want=("q",))
+    ms = c.contraction_time()
+    assert 0.0 < ms < 50.0
+    c.contraction_timing(False)
+    c.close()
+
+
 def test_int8_issue_rate_probe_reports_a_plausible_ceiling(psb, ctx):
     """The measurement aid runs, leaves the device error word clear and reports between a quarter of and
     the full documented rate of 8192 int8 multiply-accumulates per SM clock."""

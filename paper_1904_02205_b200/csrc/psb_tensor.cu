@@ -476,6 +476,30 @@ __device__ __forceinline__ bool uniform_epilogue(const TensorParams& p) {
   return !a.kmap && q_only && (P0 == 3u || P0 == 4u);
 }
 
+// The P plane sums of a 16-channel chunk, TMEM -> registers.  With three planes and 32-bit
+// recombination the first two planes are folded (v0 + 2^7 v1, what chunk_math computes first anyway)
+// before the third is fetched: 32 registers at the peak instead of 48, which is what the loop around
+// it was spilling.  The folded plane is left as a literal zero, so the arithmetic after it drops out.
+template <int P, int MODE>
+__device__ __forceinline__ void load_chunk(uint32_t taddr, uint32_t (&v)[P][16]) {
+  if (P == 3 && MODE != 0) {
+    tc_ld16(taddr, v[0]);
+    tc_ld16(taddr + kTileN, v[1]);
+    tc_wait_ld();
+#pragma unroll
+    for (int j = 0; j < 16; ++j) {
+      v[0][j] = (uint32_t)((int)v[0][j] + ((int)v[1][j] << kDigitBits));
+      v[1][j] = 0u;
+    }
+    tc_ld16(taddr + 2 * kTileN, v[2]);
+    tc_wait_ld();
+  } else {
+#pragma unroll
+    for (int pl = 0; pl < P; ++pl) tc_ld16(taddr + pl * kTileN, v[pl]);
+    tc_wait_ld();
+  }
+}
+
 // Linear output index (n * OH + oy) * OW + ox of row `row` of row tile `m_tile`, and whether the
 // row is a real output.  Plain mode: rows are consecutive outputs.  Band mode: rows are
 // padded-linear positions of one image.
@@ -589,9 +613,7 @@ __device__ __noinline__ bool epilogue_uniform(const TensorParams& p, SharedCtl* 
     uint32_t v[P][16];
     if (active) {
       const uint32_t taddr = tmem_base + buf * kTmemBufStride + ((quarter * 32u) << 16) + sub * 16u;
-#pragma unroll
-      for (int pl = 0; pl < P; ++pl) tc_ld16(taddr + pl * kTileN, v[pl]);
-      tc_wait_ld();
+      load_chunk<P, MODE>(taddr, v);
     }
     // the chunk is in registers: give the accumulator buffer back before doing the arithmetic
     tc_fence_before();
@@ -679,9 +701,7 @@ __device__ __noinline__ bool epilogue_uniform_band(const TensorParams& p, Shared
     uint32_t v[P][16];
     if (active) {
       const uint32_t taddr = tmem_base + buf * kTmemBufStride + ((quarter * 32u) << 16) + sub * 16u;
-#pragma unroll
-      for (int pl = 0; pl < P; ++pl) tc_ld16(taddr + pl * kTileN, v[pl]);
-      tc_wait_ld();
+      load_chunk<P, MODE>(taddr, v);
     }
     // the chunk is in registers: give the accumulator buffer back before doing the arithmetic
     tc_fence_before();

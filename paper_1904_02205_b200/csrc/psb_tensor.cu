@@ -408,13 +408,35 @@ __device__ __forceinline__ size_t out_offset(const ConvArgs& a, uint32_t ohow, u
   return ((size_t)n * a.O + o_base) * ohow + (m - n * ohow);
 }
 
+// The P plane sums of a 16-channel chunk, TMEM -> registers.  With three planes and 32-bit
+// recombination the first two planes are folded (v0 + 2^7 v1, what chunk_math computes first anyway)
+// before the third is fetched: 32 registers at the peak instead of 48, which is what the loop around
+// it was spilling.  The folded plane is left as a literal zero, so the arithmetic after it drops out.
+template <int P, int MODE>
+__device__ __forceinline__ void load_chunk(uint32_t taddr, uint32_t (&v)[P][16]) {
+  if (P == 3 && MODE != 0) {
+    tc_ld16(taddr, v[0]);
+    tc_ld16(taddr + kTileN, v[1]);
+    tc_wait_ld();
+#pragma unroll
+    for (int j = 0; j < 16; ++j) {
+      v[0][j] = (uint32_t)((int)v[0][j] + ((int)v[1][j] << kDigitBits));
+      v[1][j] = 0u;
+    }
+    tc_ld16(taddr + 2 * kTileN, v[2]);
+    tc_wait_ld();
+  } else {
+#pragma unroll
+    for (int pl = 0; pl < P; ++pl) tc_ld16(taddr + pl * kTileN, v[pl]);
+    tc_wait_ld();
+  }
+}
+
 template <int P, int MODE, bool HAS_RES>
 __device__ __noinline__ void epilogue_chunk_q(uint32_t taddr, bool valid, uint8_t* q_dst, uint4 r4, bool vec16,
                                               bool both, const float2* scb, const long long* corr, EpiConst c) {
   uint32_t v[P][16];
-#pragma unroll
-  for (int pl = 0; pl < P; ++pl) tc_ld16(taddr + pl * kTileN, v[pl]);
-  tc_wait_ld();
+  load_chunk<P, MODE>(taddr, v);
   if (!valid) return;
   store_row16(q_dst, chunk_math<P, MODE, HAS_RES>(v, r4, scb, corr, c), vec16, both);
 }
@@ -476,30 +498,6 @@ __device__ __forceinline__ bool uniform_epilogue(const TensorParams& p) {
   return !a.kmap && q_only && (P0 == 3u || P0 == 4u);
 }
 
-// The P plane sums of a 16-channel chunk, TMEM -> registers.  With three planes and 32-bit
-// recombination the first two planes are folded (v0 + 2^7 v1, what chunk_math computes first anyway)
-// before the third is fetched: 32 registers at the peak instead of 48, which is what the loop around
-// it was spilling.  The folded plane is left as a literal zero, so the arithmetic after it drops out.
-template <int P, int MODE>
-__device__ __forceinline__ void load_chunk(uint32_t taddr, uint32_t (&v)[P][16]) {
-  if (P == 3 && MODE != 0) {
-    tc_ld16(taddr, v[0]);
-    tc_ld16(taddr + kTileN, v[1]);
-    tc_wait_ld();
-#pragma unroll
-    for (int j = 0; j < 16; ++j) {
-      v[0][j] = (uint32_t)((int)v[0][j] + ((int)v[1][j] << kDigitBits));
-      v[1][j] = 0u;
-    }
-    tc_ld16(taddr + 2 * kTileN, v[2]);
-    tc_wait_ld();
-  } else {
-#pragma unroll
-    for (int pl = 0; pl < P; ++pl) tc_ld16(taddr + pl * kTileN, v[pl]);
-    tc_wait_ld();
-  }
-}
-
 // Linear output index (n * OH + oy) * OW + ox of row `row` of row tile `m_tile`, and whether the
 // row is a real output.  Plain mode: rows are consecutive outputs.  Band mode: rows are
 // padded-linear positions of one image.
@@ -529,6 +527,27 @@ struct RowMap {
     const uint32_t m = m_tile * kTileM + row;
     *valid = m < M;
     return m;
+  }
+  __device__ __forceinline__ size_t offset(uint32_t m, uint32_t o_base) const {
+    if (!planar) return (size_t)m * O + o_base;
+    const uint32_t n = m / ohow;
+    return ((size_t)n * O + o_base) * ohow + (m - n * ohow);
+  }
+};
+
+// Band mode: rows of a tile are padded-linear positions of one image (tile_row_index above).
+struct RowMapBand {
+  uint32_t tpi, tpi_magic, Wp, Wp_magic, OH, OW, O, ohow, planar;
+  __device__ __forceinline__ void init(const TensorParams& p) {
+    tpi = p.tpi; tpi_magic = p.tpi_magic; Wp = p.Wp; Wp_magic = p.Wp_magic;
+    OH = p.a.OH; OW = p.a.OW; O = p.a.O; ohow = p.a.OH * p.a.OW; planar = p.a.out_nchw;
+  }
+  __device__ __forceinline__ uint32_t row_index(uint32_t m_tile, uint32_t row, bool* valid) const {
+    const uint32_t n = __umulhi(m_tile, tpi_magic);
+    const uint32_t t = (m_tile - n * tpi) * kTileM + row;
+    const uint32_t oy = __umulhi(t, Wp_magic), ox = t - oy * Wp;
+    *valid = oy < OH && ox < OW;
+    return (n * OH + oy) * OW + ox;
   }
   __device__ __forceinline__ size_t offset(uint32_t m, uint32_t o_base) const {
     if (!planar) return (size_t)m * O + o_base;
@@ -630,9 +649,8 @@ __device__ __noinline__ bool epilogue_uniform(const TensorParams& p, SharedCtl* 
   return false;
 }
 
-// The same loop for band mode, reading the parameter block where it needs it: band mode's index
-// arithmetic wants eight more fields, and holding them in registers made the loop spill more than the
-// loads cost.
+// The same loop for band mode (RowMapBand: band mode's index arithmetic wants five more fields; a loop
+// of its own keeps them out of the register budget of plain mode).
 template <int P, int MODE, bool HAS_RES>
 __device__ __noinline__ bool epilogue_uniform_band(const TensorParams& p, SharedCtl* ctl, uint32_t tmem_base,
                                               uint32_t ew, uint32_t lane, EpiConst c) {
@@ -642,29 +660,32 @@ __device__ __noinline__ bool epilogue_uniform_band(const TensorParams& p, Shared
   const uint32_t l = a.uniform_log2k;
   const bool use_corr = p.corr[l] != nullptr;
   volatile uint32_t* abort = &ctl->abort;
-  const uint8_t* res_base = (const uint8_t*)a.residual;
+  const uint8_t* const res_base = (const uint8_t*)a.residual;
+  uint8_t* const q_base = (uint8_t*)a.q_out;
+  RowMapBand rm;
+  rm.init(p);
   const float2* scb = ctl->scb[ew];
   const long long* corr = ctl->corr[ew];
-  const bool vec16 = p.vec_ok == 2u, planar = a.out_nchw != 0u;
-  const uint32_t ohow = a.OH * a.OW;
+  const bool vec16 = p.vec_ok == 2u, planar = rm.planar != 0u;
+  const uint32_t ohow = rm.ohow;
   TileIter ti;
   ti.init(p);
   uint32_t pass = 0, cur_o_tile = 0xFFFFFFFFu;
   uint4 r_next = make_uint4(0, 0, 0, 0);
   if (HAS_RES && ti.valid()) {
     bool ok_row;
-    const uint32_t m = tile_row_index(p, ti.m_tile, row, &ok_row), ob = ti.o_tile * kTileN + sub * 16u;
-    if (ok_row && ob < a.O) {
-      const uint8_t* src = res_base + out_offset(a, ohow, m, ob);
-      r_next = planar ? load_planar16<0>(src, ohow, a.O - ob) : load_row16(src, vec16, ob + 16u <= a.O);
+    const uint32_t m = rm.row_index(ti.m_tile, row, &ok_row), ob = ti.o_tile * kTileN + sub * 16u;
+    if (ok_row && ob < rm.O) {
+      const uint8_t* src = res_base + rm.offset(m, ob);
+      r_next = planar ? load_planar16<0>(src, ohow, rm.O - ob) : load_row16(src, vec16, ob + 16u <= rm.O);
     }
   }
   while (ti.valid()) {
     bool row_valid;
-    const uint32_t m = tile_row_index(p, ti.m_tile, row, &row_valid);
+    const uint32_t m = rm.row_index(ti.m_tile, row, &row_valid);
     const uint32_t o_tile = ti.o_tile;
     const uint32_t o_base = o_tile * kTileN + sub * 16u;
-    const bool active = o_base < a.O;          // warp-uniform
+    const bool active = o_base < rm.O;          // warp-uniform
     ti.next();
     if (o_tile != cur_o_tile) {
       // per-channel constants of this channel tile: the warp keeps its own copy of its 16 channels
@@ -687,11 +708,11 @@ __device__ __noinline__ bool epilogue_uniform_band(const TensorParams& p, Shared
     const uint4 r_cur = r_next;
     if (HAS_RES && ti.valid()) {
       bool ok_row;
-      const uint32_t mn = tile_row_index(p, ti.m_tile, row, &ok_row), ob = ti.o_tile * kTileN + sub * 16u;
+      const uint32_t mn = rm.row_index(ti.m_tile, row, &ok_row), ob = ti.o_tile * kTileN + sub * 16u;
       r_next = make_uint4(0, 0, 0, 0);
-      if (ok_row && ob < a.O) {
-        const uint8_t* src = res_base + out_offset(a, ohow, mn, ob);
-        r_next = planar ? load_planar16<0>(src, ohow, a.O - ob) : load_row16(src, vec16, ob + 16u <= a.O);
+      if (ok_row && ob < rm.O) {
+        const uint8_t* src = res_base + rm.offset(mn, ob);
+        r_next = planar ? load_planar16<0>(src, ohow, rm.O - ob) : load_row16(src, vec16, ob + 16u <= rm.O);
       }
     }
     const uint32_t buf = pass & 1u, aph = (pass >> 1) & 1u;
@@ -709,9 +730,9 @@ __device__ __noinline__ bool epilogue_uniform_band(const TensorParams& p, Shared
     if (lane == 0) mbar_arrive(smem_u32(&ctl->acc_empty[buf]));
     if (active && row_valid) {
       const uint4 q16 = chunk_math<P, MODE, HAS_RES>(v, r_cur, scb, corr, c);
-      uint8_t* dst = (uint8_t*)a.q_out + out_offset(a, ohow, m, o_base);
-      if (planar) store_planar16<0>(dst, ohow, a.O - o_base, q16);
-      else store_row16(dst, q16, vec16, o_base + 16u <= a.O);
+      uint8_t* dst = q_base + rm.offset(m, o_base);
+      if (planar) store_planar16<0>(dst, ohow, rm.O - o_base, q16);
+      else store_row16(dst, q16, vec16, o_base + 16u <= rm.O);
     }
     ++pass;
   }

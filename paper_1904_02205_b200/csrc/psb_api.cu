@@ -162,7 +162,10 @@ psb_status run_layer(psb_ctx* ctx, const psb_weights* wt, const void* x_dev, uin
           if (launch_corr128(wt, l, s) != cudaSuccess) return PSB_ERR_CUDA;
     }
     if (a.kmap) {
-      st = ensure_scratch(ctx, 2, ((size_t)a.N * a.OH * a.OW + 127) / 128);
+      // one byte per row tile: strips of 128 locations, or 8 x 16 patches (a few more of them)
+      const size_t strips = ((size_t)a.N * a.OH * a.OW + 127) / 128;
+      const size_t patches = (size_t)((a.OW + 7) / 8) * (((size_t)a.OH * a.N + 15) / 16);
+      st = ensure_scratch(ctx, 2, strips > patches ? strips : patches);
       if (st != PSB_OK) return st;
     }
     st = launch_tensor(ctx, wt, a, amax, add_corr, s);

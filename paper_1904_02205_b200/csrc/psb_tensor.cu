@@ -84,6 +84,12 @@ struct TensorParams {
   uint32_t tpi;         // tiles per image: ceil(OH * Wp / 128)
   uint32_t band_rows;   // padded input rows per band
   uint32_t band_bytes;  // stage size (band_rows * Wp * C rounded up to 1024)
+  // Patch mode (plain GEMM layers under a per-location map): a tile is a patch of 8 x 16 locations
+  // (x by y, y running over the rows of all images) instead of a strip of 128 consecutive ones, so
+  // that fewer levels of a smooth map meet in one tile; one 3-D tiled copy per K block.  Row r of the
+  // tile is location (tx * 8 + r % 8, ty * 16 + r / 8).  Used where the image width is a multiple of 8.
+  uint32_t patch;       // 1: patch mode
+  uint32_t tiles_x;     // patches per image row: ceil(OW / 8)
   uint32_t Wp_magic, tpi_magic;   // ceil(2^32 / Wp), ceil(2^32 / tpi): quotients by multiply-high (exact in the
                                   // ranges band mode is restricted to)
 };
@@ -153,6 +159,14 @@ __device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_
   asm volatile(
       "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
       ::"r"(dst), "l"(src), "r"(bytes), "r"(bar)
+      : "memory");
+}
+
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c, int x, int y) {
+  asm volatile(
+      "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes"
+      " [%0], [%1, {%3, %4, %5}], [%2];"
+      ::"r"(dst), "l"(map), "r"(bar), "r"(c), "r"(x), "r"(y)
       : "memory");
 }
 
@@ -231,15 +245,30 @@ __device__ __forceinline__ uint32_t tile_levels(const TensorParams& p, uint32_t 
   return (uint32_t)p.tile_mask[m_tile];
 }
 
+constexpr uint32_t kPatchW = 8, kPatchH = kTileM / kPatchW;
+
+// Linear location index of row `row` of patch `m_tile` (rows of all images stacked: y < rows_all), and
+// whether it is a real location.
+__device__ __forceinline__ uint32_t patch_row_index(uint32_t m_tile, uint32_t row, uint32_t tiles_x, uint32_t OW,
+                                                    uint32_t rows_all, bool* valid) {
+  const uint32_t ty = m_tile / tiles_x, tx = m_tile - ty * tiles_x;
+  const uint32_t x = tx * kPatchW + (row % kPatchW), y = ty * kPatchH + row / kPatchW;
+  *valid = x < OW && y < rows_all;
+  return y * OW + x;
+}
+
 __global__ void tile_levels_kernel(const uint8_t* __restrict__ kmap, uint32_t M, uint32_t m_tiles,
-                                   uint8_t* __restrict__ tile_mask) {
+                                   uint8_t* __restrict__ tile_mask, uint32_t patch_tiles_x, uint32_t OW,
+                                   uint32_t rows_all) {
   const uint32_t tile = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31u;
   if (tile >= m_tiles) return;
   uint32_t mask = 0;
 #pragma unroll
   for (int r = 0; r < 4; ++r) {
-    const uint32_t m = tile * kTileM + r * 32u + lane;
-    if (m < M) mask |= 1u << min((uint32_t)kmap[m], 7u);   // levels >= 7 are invalid: bit 7, flagged by the epilogue
+    uint32_t m = tile * kTileM + r * 32u + lane;
+    bool ok = m < M;
+    if (patch_tiles_x) m = patch_row_index(tile, r * 32u + lane, patch_tiles_x, OW, rows_all, &ok);
+    if (ok) mask |= 1u << min((uint32_t)kmap[m], 7u);   // levels >= 7 are invalid: bit 7, flagged by the epilogue
   }
   mask = __reduce_or_sync(0xFFFFFFFFu, mask);
   if (lane == 0) tile_mask[tile] = (uint8_t)mask;
@@ -969,6 +998,9 @@ psb_mma_kernel(const __grid_constant__ TmapSet maps, const __grid_constant__ Ten
               const uint32_t dst = ring_addr + s * stage_bytes + lane * sub_bytes;
               if (p.im2col)
                 tma_load_im2col_4d(dst, &maps.a, bar, (int)(cb * BK), w0, h0, (int)n0, (uint16_t)kw, (uint16_t)kh);
+              else if (p.patch)
+                tma_load_3d(dst, &maps.a, bar, (int)(cb * BK), (int)((m_tile % p.tiles_x) * kPatchW),
+                            (int)((m_tile / p.tiles_x) * kPatchH));
               else
                 tma_load_2d(dst, &maps.a, bar, (int)(cb * BK), (int)m0);
               if (!p.resident) bulk_load(dst + p.stage_bytes_a, b_tiles + (size_t)kb * blk, blk, bar);
@@ -1040,8 +1072,9 @@ psb_mma_kernel(const __grid_constant__ TmapSet maps, const __grid_constant__ Ten
       for (ti.init(p); !failed && ti.valid(); ti.next()) {
         const uint32_t m0 = ti.m_tile * kTileM, o_tile = ti.o_tile;
         const uint32_t levels = tile_levels(p, ti.m_tile) & a.level_mask;
-        const uint32_t m = m0 + row;
-        const bool in_range = m < p.M;
+        uint32_t m = m0 + row;
+        bool in_range = m < p.M;
+        if (p.patch) m = patch_row_index(ti.m_tile, row, p.tiles_x, a.OW, a.OH * a.N, &in_range);
         const uint32_t my_level = in_range ? (a.kmap ? (uint32_t)a.kmap[m] : a.uniform_log2k) : 0xFFu;
         if (in_range && (my_level >= (uint32_t)kMaxLevels || !((a.level_mask >> my_level) & 1u)))
           atomicOr(a.err, kDevErrBadLevel);
@@ -1205,6 +1238,15 @@ psb_status launch_tensor(psb_ctx* ctx, const psb_weights* wt, const ConvArgs& a,
   p.vec_ok = 0u;
   if (!a.out_nchw && a.O % 16u == 0u && !(out_ptrs & 15u)) p.vec_ok = 2u;
   else if (!a.out_nchw && a.O % 8u == 0u && !(out_ptrs & 7u)) p.vec_ok = 1u;
+  p.patch = 0;
+  p.tiles_x = 0;
+  // (image widths that are not a multiple of the patch width would compute dropped columns: at 28, 14
+  // and 7 that costs what the fewer levels per tile save, so those keep strips)
+  if (a.kmap && !p.im2col && !a.out_nchw && a.OW % kPatchW == 0u) {
+    p.patch = 1;
+    p.tiles_x = (a.OW + kPatchW - 1) / kPatchW;
+    p.m_tiles = p.tiles_x * ((a.OH * a.N + kPatchH - 1) / kPatchH);
+  }
   if (!a.kmap) {
     const uint32_t P = p.planes[a.uniform_log2k];
     const uint32_t need = k_iters * P * kTileN * bk;
@@ -1303,6 +1345,15 @@ psb_status launch_tensor(psb_ctx* ctx, const psb_weights* wt, const ConvArgs& a,
                    lower, upper, bk, kTileM, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, swz,
                    CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
       return PSB_ERR_CUDA;
+  } else if (p.patch) {
+    cuuint64_t dims[3] = {a.C, a.W, (cuuint64_t)a.H * a.N};
+    cuuint64_t strides[2] = {(cuuint64_t)a.C, (cuuint64_t)a.C * a.W};
+    cuuint32_t box[3] = {bk, kPatchW, kPatchH};
+    cuuint32_t estr[3] = {1, 1, 1};
+    if (enc_tiled(&maps.a, CU_TENSOR_MAP_DATA_TYPE_UINT8, 3, const_cast<void*>(a.x), dims, strides, box, estr,
+                  CU_TENSOR_MAP_INTERLEAVE_NONE, swz, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+      return PSB_ERR_CUDA;
   } else {
     cuuint64_t dims[2] = {a.C, p.M};
     cuuint64_t strides[1] = {(cuuint64_t)a.C};
@@ -1320,7 +1371,8 @@ psb_status launch_tensor(psb_ctx* ctx, const psb_weights* wt, const ConvArgs& a,
     // the caller has sized the third scratch buffer for one byte per row tile
     if (!ctx->scratch[2] || ctx->scratch_bytes[2] < p.m_tiles) return PSB_ERR_INVALID_ARG;
     tile_levels_kernel<<<(p.m_tiles * 32u + 255u) / 256u, 256, 0, s>>>(a.kmap, p.M, p.m_tiles,
-                                                                      (uint8_t*)ctx->scratch[2]);
+                                                                      (uint8_t*)ctx->scratch[2],
+                                                                      p.patch ? p.tiles_x : 0u, a.OW, a.OH * a.N);
     note_launch();
     p.tile_mask = (const uint8_t*)ctx->scratch[2];
   }

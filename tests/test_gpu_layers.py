@@ -303,6 +303,21 @@ def test_tensor_path_per_location_draw_counts(psb, ctx, oracle):
           path=psb.PSB_PATH_TENSOR)
 
 
+@pytest.mark.parametrize("case", [(3, 64, 10, 16, 64, False), (2, 128, 7, 24, 72, True), (5, 32, 9, 8, 64, True)])
+def test_tensor_path_per_location_draw_counts_1x1_patch_tiles(psb, ctx, oracle, case):
+    """1x1 layers under a per-location map on channels-last tensors whose width is a multiple of 8 are tiled
+    in 8 x 16 patches (rows of all images stacked): ragged last patch rows, patches across image borders."""
+    N, C, H, W, O, with_res = case
+    rng = np.random.default_rng(abs(hash(case)) % 2 ** 31)
+    w, x, scale, bias = _layer_inputs(rng, N, C, H, W, O, 1, 1, 1, 1)
+    kmap = rng.choice([0, 1, 2, 3, 4], size=(N, H, W)).astype(np.uint8)
+    kmap[0, : H // 2] = 2                       # a smooth region: patches with a single level
+    res = rng.integers(0, 16, size=(N, H, W, O)).astype(np.uint8) if with_res else None
+    g = _both(psb, ctx, oracle, w, x, 1, 1, 1, 0, [0, 1, 2, 3, 4], scale, bias, kmap=kmap, inv_step=0.5,
+              residual=res, res_scale=0.2 if with_res else 0.0, in_max=15, path=psb.PSB_PATH_TENSOR)
+    assert g["path"] == psb.PSB_PATH_TENSOR
+
+
 def test_tensor_path_signed_inputs_residual_nchw_and_exponent_options(psb, ctx, oracle):
     rng = np.random.default_rng(22)
     w, x, scale, bias = _layer_inputs(rng, 2, 64, 10, 10, 32, 3, 3, 1, 0, x_dtype=np.int8, x_hi=128)

@@ -218,9 +218,11 @@ uint64_t psb_launch_count(void);
  * that kernel by this context is bracketed by a pair of CUDA events on its
  * stream (which also keeps it from starting under its predecessor's tail, so a
  * step runs a little slower while this is on); psb_contraction_time waits for
- * the end of the most recent such launch and returns its duration in
- * milliseconds.  PSB_ERR_INVALID_ARG for null arguments or when no launch has
- * been timed yet, PSB_ERR_CUDA if the events cannot be created or read. */
+ * those launches and returns the sum of their durations in milliseconds, over
+ * the launches made since timing was last switched on (switching it on again
+ * starts a new sum; at most 256 launches are kept, later ones go untimed).
+ * PSB_ERR_INVALID_ARG for null arguments or when no launch has been timed yet,
+ * PSB_ERR_CUDA if the events cannot be created or read. */
 psb_status psb_contraction_timing(psb_ctx* ctx, uint32_t enable);
 psb_status psb_contraction_time(psb_ctx* ctx, float* milliseconds);
 

@@ -215,7 +215,7 @@ class Context:
         _check(self.lib.psb_contraction_timing(self.handle, 1 if enable else 0), "psb_contraction_timing")
 
     def contraction_time(self):
-        """Device time in milliseconds of the most recent timed contraction launch (waits for it)."""
+        """Summed device time in milliseconds of the contraction launches made since timing was switched on."""
         ms = C.c_float(0.0)
         _check(self.lib.psb_contraction_time(self.handle, C.byref(ms)), "psb_contraction_time")
         return float(ms.value)

@@ -230,8 +230,10 @@ psb_status psb_destroy(psb_ctx* ctx) {
   for (int i = 0; i < 3; ++i)
     if (ctx->scratch[i]) cudaFree(ctx->scratch[i]);
   if (ctx->err_dev) cudaFree(ctx->err_dev);
-  if (ctx->t_begin) cudaEventDestroy(ctx->t_begin);
-  if (ctx->t_end) cudaEventDestroy(ctx->t_end);
+  for (int i = 0; i < psb_ctx::kTimedLaunches; ++i) {
+    if (ctx->t_begin[i]) cudaEventDestroy(ctx->t_begin[i]);
+    if (ctx->t_end[i]) cudaEventDestroy(ctx->t_end[i]);
+  }
   delete ctx;
   return PSB_OK;
 }
@@ -394,24 +396,32 @@ uint64_t psb_launch_count(void) { return (uint64_t)psb::launches_so_far(); }
 
 psb_status psb_contraction_timing(psb_ctx* ctx, uint32_t enable) {
   if (!ctx) return PSB_ERR_INVALID_ARG;
-  if (enable && !ctx->t_begin) {
+  if (enable && !ctx->t_begin[0]) {
     cudaSetDevice(ctx->device);
-    if (cudaEventCreate(&ctx->t_begin) != cudaSuccess || cudaEventCreate(&ctx->t_end) != cudaSuccess) {
-      cudaGetLastError();
-      return PSB_ERR_CUDA;
-    }
+    for (int i = 0; i < psb_ctx::kTimedLaunches; ++i)
+      if (cudaEventCreate(&ctx->t_begin[i]) != cudaSuccess || cudaEventCreate(&ctx->t_end[i]) != cudaSuccess) {
+        cudaGetLastError();
+        return PSB_ERR_CUDA;
+      }
   }
   ctx->time_contraction = enable != 0;
+  if (enable) ctx->timed_launches = 0;     // switching it on starts a new sum
   return PSB_OK;
 }
 
 psb_status psb_contraction_time(psb_ctx* ctx, float* milliseconds) {
-  if (!ctx || !milliseconds || !ctx->contraction_timed) return PSB_ERR_INVALID_ARG;
-  if (cudaEventSynchronize(ctx->t_end) != cudaSuccess ||
-      cudaEventElapsedTime(milliseconds, ctx->t_begin, ctx->t_end) != cudaSuccess) {
-    cudaGetLastError();
-    return PSB_ERR_CUDA;
+  if (!ctx || !milliseconds || ctx->timed_launches == 0) return PSB_ERR_INVALID_ARG;
+  float total = 0.0f;
+  for (int i = 0; i < ctx->timed_launches; ++i) {
+    float ms = 0.0f;
+    if (cudaEventSynchronize(ctx->t_end[i]) != cudaSuccess ||
+        cudaEventElapsedTime(&ms, ctx->t_begin[i], ctx->t_end[i]) != cudaSuccess) {
+      cudaGetLastError();
+      return PSB_ERR_CUDA;
+    }
+    total += ms;
   }
+  *milliseconds = total;
   return PSB_OK;
 }
 

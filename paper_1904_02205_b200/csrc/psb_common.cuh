@@ -84,9 +84,11 @@ struct psb_ctx {
   int sm_count = 0;
   void* encode_tiled = nullptr;     // cuTensorMapEncodeTiled
   void* encode_im2col = nullptr;    // cuTensorMapEncodeIm2col
-  bool time_contraction = false;    // bracket the contraction kernel with the two events below
-  bool contraction_timed = false;   // a pair has been recorded
-  cudaEvent_t t_begin = nullptr, t_end = nullptr;
+  // measurement aid: event pairs around the contraction launches made since timing was switched on
+  static constexpr int kTimedLaunches = 256;
+  bool time_contraction = false;
+  int timed_launches = 0;           // pairs recorded since timing was switched on (at most kTimedLaunches)
+  cudaEvent_t t_begin[kTimedLaunches] = {}, t_end[kTimedLaunches] = {};
 };
 
 namespace psb {

@@ -1395,13 +1395,13 @@ psb_status launch_tensor(psb_ctx* ctx, const psb_weights* wt, const ConvArgs& a,
                            (int)smem_bytes);                                                         \
   if (e == cudaSuccess) e = cudaLaunchKernelEx(&cfg, psb_mma_kernel<BKV>, maps, p);                  \
   note_launch();
-  const bool timed = ctx->time_contraction && ctx->t_begin && ctx->t_end;
-  if (timed) cudaEventRecord(ctx->t_begin, s);
+  const bool timed = ctx->time_contraction && ctx->t_begin[0] && ctx->timed_launches < psb_ctx::kTimedLaunches;
+  if (timed) cudaEventRecord(ctx->t_begin[ctx->timed_launches], s);
   if (bk == 128) { PSB_LAUNCH(128) } else if (bk == 64) { PSB_LAUNCH(64) } else { PSB_LAUNCH(32) }
 #undef PSB_LAUNCH
   if (timed) {
-    cudaEventRecord(ctx->t_end, s);
-    ctx->contraction_timed = true;
+    cudaEventRecord(ctx->t_end[ctx->timed_launches], s);
+    ++ctx->timed_launches;
   }
   if (e != cudaSuccess || cudaGetLastError() != cudaSuccess) return PSB_ERR_CUDA;
   return PSB_OK;

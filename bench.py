@@ -1,7 +1,7 @@
 #!/usr/bin/env python
 """Throughput of the PSB sampled-weight contraction on B200.
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload conv3x3|resnet50|mobilenetv2]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload conv3x3|fc|resnet50|resnet50_adaptive|mobilenetv2]
                     [--k 8] [--impl reference]
 
 One step = one pass of the whole hot path over one synthetic batch: draw fresh random bits
@@ -178,6 +178,76 @@ class ConvWorkload:
         return dt, self.macs * n_images // self.images, "first %d of %d images, all layers" % (n_images, self.images)
 
 
+class FcWorkload:
+    """Fully connected layer 256 -> 128, batch 16, k = 4, 8-bit output after ReLU: the small case.  Half a
+    million multiply-accumulates per step, so a step is launch latency; what to read is microseconds."""
+    name = "fc_256x128_b16"
+    oracle_images = 16
+
+    def __init__(self, k, rank=0):
+        from workloads import config1_fc
+
+        self.k = k
+        self.log2k = int(np.log2(k))
+        self.cfg = config1_fc(seed=100 * rank, k=k)
+        self.macs = self.cfg["macs"]
+        self.images = self.cfg["x"].shape[0]
+
+    def setup(self, ctx, psb, torch):
+        self.ctx, self.psb, self.torch = ctx, psb, torch
+        c, dev = self.cfg, ctx.device
+        self.w = torch.from_numpy(c["w"]).to(dev)
+        self.x = torch.from_numpy(c["x"]).to(dev)
+        self.scale = torch.from_numpy(c["scale"]).to(dev)
+        self.bias = torch.from_numpy(c["bias"]).to(dev)
+        self.wt = ctx.sample_weights(self.w, seed=c["seed"], layer_id=0, level_mask=1 << self.log2k)
+        ctx.set_sample_map(None, self.log2k)
+        self.out = {"q": torch.empty((self.images, c["w"].shape[0]), dtype=torch.uint8, device=dev)}
+        self.x_host = torch.from_numpy(c["x"]).pin_memory()
+        self.q_host = torch.empty((self.images, c["w"].shape[0]), dtype=torch.uint8).pin_memory()
+        self.x_stage = torch.empty_like(self.x)
+        self.e2e_h2d = self.x_host.numel()
+        self.e2e_d2h = self.q_host.numel()
+
+    def _gemm(self, x):
+        c = self.cfg
+        self.ctx.gemm(self.wt, x, self.scale, self.bias, True, c["inv_step"], 0, 255, in_max=15, out=self.out)
+
+    def step(self, i):
+        self.ctx.sample_weights(self.w, seed=self.cfg["seed"] + i, layer_id=0, level_mask=1 << self.log2k, into=self.wt)
+        self._gemm(self.x)
+
+    def kernel_only(self):
+        self._gemm(self.x)
+
+    def e2e_step(self, i):
+        self.x_stage.copy_(self.x_host, non_blocking=True)
+        self.ctx.sample_weights(self.w, seed=self.cfg["seed"] + i, layer_id=0, level_mask=1 << self.log2k, into=self.wt)
+        self._gemm(self.x_stage)
+        self.q_host.copy_(self.out["q"], non_blocking=True)
+
+    def roofline(self, kernel_ms, peaks):
+        # one launch of 2048 threads: neither bytes (35 KB) nor arithmetic matter, the launch does
+        nbytes = self.images * 256 + 128 * 256 * 4 + self.images * 128
+        achieved = nbytes / (kernel_ms * 1e-3) / 1e9
+        return dict(bound="hbm", kernel="conv_direct_kernel (latency-bound: one launch of 2048 threads)",
+                    achieved=achieved, peak=peaks["hbm_gbs"], unit="GB/s", frac=achieved / peaks["hbm_gbs"],
+                    traffic=None, peak_source=peaks["source"], kernel_ms=kernel_ms)
+
+    def oracle_sample(self, n_images=16):
+        from oracle import psb_oracle as orc
+
+        c = self.cfg
+        x = c["x"].reshape(self.images, 1, 1, 256)
+        t0 = time.perf_counter()
+        W, eb, _ = orc.sample_level(c["w"], c["seed"], 0, self.log2k)
+        g = orc.geom(x.shape, orc.NHWC, orc.U8, c["w"].shape, 1, 1, 0)
+        acc = orc.conv_acc(x, g, {self.log2k: W}, uniform_log2k=self.log2k)
+        orc.epilogue(acc, g, c["scale"], c["bias"], eb, True, c["inv_step"], 0, 255, uniform_log2k=self.log2k)
+        dt = time.perf_counter() - t0
+        return dt, self.macs, "the whole batch of %d, sampling included" % self.images
+
+
 class NetWorkload:
     """Network-shaped workloads: every conv / FC layer is a PSB layer, activations stay in HBM."""
     oracle_images = 1
@@ -290,6 +360,8 @@ class NetWorkload:
 def make_workload(args, rank):
     if args.workload == "conv3x3":
         return ConvWorkload(args.k, rank)
+    if args.workload == "fc":
+        return FcWorkload(args.k, rank)
     return NetWorkload(args.workload, args.k, rank, batch=args.batch)
 
 
@@ -357,7 +429,7 @@ def main():
     ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="psb")
-    ap.add_argument("--workload", default="conv3x3", choices=["conv3x3", "resnet50", "mobilenetv2", "resnet50_adaptive"])
+    ap.add_argument("--workload", default="conv3x3", choices=["conv3x3", "fc", "resnet50", "mobilenetv2", "resnet50_adaptive"])
     ap.add_argument("--k", type=int, default=8)
     ap.add_argument("--batch", type=int, default=0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -415,7 +487,7 @@ def main():
     launches = ctx.launch_count() - launches0      # kernels of the library inside the timed steps
     if world > 1:
         dist.barrier()
-    kern_ms = timed(lambda i: wl.kernel_only(), max(args.steps, 10) if args.workload == "conv3x3" else 4)
+    kern_ms = timed(lambda i: wl.kernel_only(), max(args.steps, 10) if args.workload in ("conv3x3", "fc") else 4)
     in_step_ms = []
     if args.workload == "conv3x3":
         # the same steps once more with the library's own pair of events around the contraction kernel:
@@ -426,7 +498,7 @@ def main():
             wl.step(args.warmup + args.steps + i)
             in_step_ms.append(ctx.contraction_time())
         ctx.contraction_timing(False)
-    else:
+    elif args.workload != "fc":
         # one forward pass issued as one op list with the library's events around every contraction launch:
         # the device time of the tensor path, independent of the host's per-layer call rate
         wl.hook_ms = []

@@ -73,6 +73,34 @@ __global__ void __launch_bounds__(256) conv_direct_kernel(const ConvArgs a, cons
   }
 }
 
+// Fully connected layers at small batch (1x1 filter on a 1x1 image, one group): a warp per output
+// element, the lanes stride over the input features (coalesced runs of the filter row and of the
+// activation row) and the 64-bit partial sums meet in a shuffle tree.  With one thread per output the
+// 256 dependent loads of a 256-feature row made the layer ten times longer than its launch.
+__global__ void __launch_bounds__(256) gemv_warp_kernel(const ConvArgs a, const WintTable wt) {
+  pdl_prologue();
+  const size_t total = (size_t)a.N * a.O;
+  const uint32_t lane = threadIdx.x & 31u;
+  for (size_t idx = ((size_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5; idx < total;
+       idx += ((size_t)gridDim.x * blockDim.x) >> 5) {
+    const uint32_t o = (uint32_t)(idx % a.O);
+    const uint32_t n = (uint32_t)(idx / a.O);
+    const uint32_t level = a.kmap ? a.kmap[n] : a.uniform_log2k;
+    if (level >= (uint32_t)kMaxLevels || !((a.level_mask >> level) & 1u)) {
+      if (lane == 0) atomicOr(a.err, kDevErrBadLevel);
+      continue;
+    }
+    const int32_t* __restrict__ w = wt.w[level] + (size_t)o * a.C;
+    const size_t xoff = (size_t)n * a.C;
+    long long acc = 0;
+    for (uint32_t ci = lane; ci < a.C; ci += 32u)
+      acc += (long long)load_act(a.x, a.in_dtype, xoff + ci) * (long long)__ldg(w + ci);
+#pragma unroll
+    for (int d = 16; d > 0; d >>= 1) acc += __shfl_down_sync(0xFFFFFFFFu, acc, d);
+    if (lane == 0) store_outputs(a, idx, o, level, acc);
+  }
+}
+
 // Depthwise filters (one input channel per output channel), channels-last, one draw count for
 // the layer: a thread owns 8 consecutive channels of one output location.  The block keeps the
 // layer's integer filter in shared memory as [tap][channel]; activations come in 8-byte loads;
@@ -506,6 +534,11 @@ cudaError_t launch_shift_add(const ConvArgs& a, const WintTable& wt, cudaStream_
     uint32_t blocks = grid_for(total / 8, 256);
     if (blocks > 148u * 4u) blocks = 148u * 4u;
     launch_pdl(dwconv_nhwc8_kernel, blocks, 256, dw_smem, s, a, wt.w[a.uniform_log2k]); note_launch();
+    return cudaGetLastError();
+  }
+  if (a.KH == 1 && a.KW == 1 && a.H == 1 && a.W == 1 && a.groups == 1 && a.C >= 64u && !a.out_nchw &&
+      total < (1u << 24)) {
+    launch_pdl(gemv_warp_kernel, grid_for(total * 32u, 256), 256, 0, s, a, wt); note_launch();
     return cudaGetLastError();
   }
   launch_pdl(conv_direct_kernel, grid_for(total, 256), 256, 0, s, a, wt); note_launch();

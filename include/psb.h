@@ -52,7 +52,9 @@ enum {
   PSB_ERR_ALLOC = -4,            /* device or host allocation failed                             */
   PSB_ERR_CUDA = -5,             /* a CUDA runtime / driver call failed                          */
   PSB_ERR_TIMEOUT = -6,          /* a bounded device-side wait ran out (reported by the device)  */
-  PSB_ERR_NONFINITE_WEIGHT = -7  /* a filter holds Inf or NaN (reported by the device)           */
+  PSB_ERR_NONFINITE_WEIGHT = -7, /* a filter holds Inf or NaN (reported by the device)           */
+  PSB_ERR_RANGE = -8             /* an activation exceeds the in_max the caller vouched for
+                                    (reported by the device)                                     */
 };
 
 enum { PSB_LAYOUT_NCHW = 0, PSB_LAYOUT_NHWC = 1 };
@@ -80,8 +82,28 @@ const char* psb_status_string(psb_status st);
 
 /* Synchronise `stream`, then return and clear the sticky device-side error
  * (PSB_ERR_TIMEOUT, PSB_ERR_NONFINITE_WEIGHT, PSB_ERR_BAD_K from a draw-count
- * map naming a level that was not sampled), or PSB_OK. */
+ * map naming a level that was not sampled, PSB_ERR_RANGE), or PSB_OK. */
 psb_status psb_device_status(psb_ctx* ctx, void* stream);
+
+/* Extra device-side validation, sticky until changed (no counterpart in the paper).
+ *   PSB_CHECK_RANGE  every conv / gemm call verifies that no input byte exceeds its in_max
+ *                    (see psb_conv_desc) and raises PSB_ERR_RANGE through psb_device_status
+ *                    otherwise.  Calls that convert or gather their input (NCHW tensors, filters
+ *                    with few input channels, unsigned bytes above 127) verify it in that pass
+ *                    whether the flag is set or not; the flag adds one read-only pass over the
+ *                    input to the calls that hand the tensor straight to the copy engine. */
+enum { PSB_CHECK_RANGE = 1 };
+psb_status psb_set_checks(psb_ctx* ctx, uint32_t flags);
+
+/* Every wait inside a kernel (on a copy, on the tensor pipe, on another warp) is bounded; a wait
+ * that runs out makes the kernel return and raises PSB_ERR_TIMEOUT (see psb_device_status); the
+ * context stays usable.  psb_set_wait_limit sets the bound in SM clocks for the following
+ * launches of this context (0 restores the default, 4e9 clocks, about 2 s).
+ * psb_wait_selftest launches one small thread block that waits, with that bound, on a barrier
+ * nobody arrives at: the one way to see the time-out path work without a fault.  Set a short
+ * bound (1e5 clocks) before calling it. */
+psb_status psb_set_wait_limit(psb_ctx* ctx, uint64_t sm_clocks);
+psb_status psb_wait_selftest(psb_ctx* ctx, void* stream);
 
 /* Shape of a filter in canonical order [out_ch][in_ch_per_group][kh][kw]. */
 typedef struct {
@@ -175,7 +197,11 @@ typedef struct {
  *            (filters gathered explicitly, or any filter without padding);
  *            with padding it takes the shift-add path.  A smaller in_max also
  *            lets the output stage recombine the digit planes in 32 bits.
- *   path     PSB_PATH_AUTO, or force one path (PSB_ERR_UNSUPPORTED if the forced
+ *            It is a promise the kernels rely on: a byte beyond it gives a
+ *            wrong result.  Passes that read every byte anyway verify it; the
+ *            other routes verify it on request (psb_set_checks); a violation
+ *            is reported as PSB_ERR_RANGE by psb_device_status.
+ *   path    PSB_PATH_AUTO, or force one path (PSB_ERR_UNSUPPORTED if the forced
  *            path cannot run this shape). */
 typedef struct {
   uint32_t layout;

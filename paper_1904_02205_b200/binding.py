@@ -15,7 +15,8 @@ LIB_PATH = os.path.join(_HERE, "libpsb_b200.so")
 
 PSB_OK = 0
 PSB_ERR_INVALID_ARG, PSB_ERR_BAD_K, PSB_ERR_UNSUPPORTED, PSB_ERR_ALLOC = -1, -2, -3, -4
-PSB_ERR_CUDA, PSB_ERR_TIMEOUT, PSB_ERR_NONFINITE_WEIGHT = -5, -6, -7
+PSB_ERR_CUDA, PSB_ERR_TIMEOUT, PSB_ERR_NONFINITE_WEIGHT, PSB_ERR_RANGE = -5, -6, -7, -8
+PSB_CHECK_RANGE = 1
 PSB_LAYOUT_NCHW, PSB_LAYOUT_NHWC = 0, 1
 PSB_DT_U8, PSB_DT_S8 = 0, 1
 PSB_PATH_AUTO, PSB_PATH_SHIFT_ADD, PSB_PATH_TENSOR = 0, 1, 2
@@ -24,7 +25,8 @@ EXPORTS = ["psb_create", "psb_destroy", "psb_status_string", "psb_device_status"
            "psb_weights_export", "psb_weights_free", "psb_set_sample_map", "psb_conv2d", "psb_gemm",
            "psb_last_path", "psb_maxpool2d_u8", "psb_global_avgpool_u8", "psb_sample_level_static",
            "psb_sample_batch_create", "psb_sample_batch_run", "psb_sample_batch_free", "psb_run",
-           "psb_launch_count", "psb_int8_mma_probe", "psb_contraction_timing", "psb_contraction_time"]
+           "psb_launch_count", "psb_int8_mma_probe", "psb_contraction_timing", "psb_contraction_time",
+           "psb_set_checks", "psb_set_wait_limit", "psb_wait_selftest"]
 
 
 class psb_wshape(C.Structure):
@@ -93,6 +95,9 @@ def load_library():
     lib.psb_int8_mma_probe.argtypes = [vp, u32, u32, C.POINTER(C.c_double), C.POINTER(C.c_double), vp]
     lib.psb_contraction_timing.argtypes = [vp, u32]
     lib.psb_contraction_time.argtypes = [vp, C.POINTER(C.c_float)]
+    lib.psb_set_checks.argtypes = [vp, u32]
+    lib.psb_set_wait_limit.argtypes = [vp, C.c_uint64]
+    lib.psb_wait_selftest.argtypes = [vp, vp]
     lib.psb_launch_count.argtypes = []
     lib.psb_launch_count.restype = C.c_uint64
     lib.psb_maxpool2d_u8.argtypes = [vp, vp, u32, u32, u32, u32, u32, u32, u32, u32, vp, vp]
@@ -202,6 +207,18 @@ class Context:
 
     def last_path(self):
         return self.lib.psb_last_path(self.handle)
+
+    def set_checks(self, flags):
+        """PSB_CHECK_RANGE: verify every input byte against in_max on the device."""
+        _check(self.lib.psb_set_checks(self.handle, flags), "psb_set_checks")
+
+    def set_wait_limit(self, sm_clocks):
+        """Bound of every device-side wait in SM clocks (0 restores the default)."""
+        _check(self.lib.psb_set_wait_limit(self.handle, sm_clocks), "psb_set_wait_limit")
+
+    def wait_selftest(self, stream=None):
+        """One small thread block waits on a barrier nobody arrives at; the wait runs out."""
+        _check(self.lib.psb_wait_selftest(self.handle, _stream(stream)), "psb_wait_selftest")
 
     def int8_mma_probe(self, n_cols=192, groups=4000, stream=None):
         """Returns (int8 MAC per clock per SM, tera-operations per second) of bare MMA issue."""

@@ -107,7 +107,7 @@ psb_status run_layer(psb_ctx* ctx, const psb_weights* wt, const void* x_dev, uin
   // largest activation magnitude the caller vouches for
   uint32_t amax = in_max ? in_max : (in_dtype == PSB_DT_U8 ? 255u : 128u);
   const uint64_t M = (uint64_t)n * oh * ow;
-  bool tensor_ok = false;
+  bool tensor_ok = false, range_checked = false;
   if (path != PSB_PATH_SHIFT_ADD) {
     // the MMA takes signed bytes: unsigned data above 127 qualifies only where the activation
     // matrix is gathered explicitly (packed-K filters), which stores x - 128
@@ -124,10 +124,23 @@ psb_status run_layer(psb_ctx* ctx, const psb_weights* wt, const void* x_dev, uin
     size_t bytes = (size_t)n * c * h * w;
     st = ensure_scratch(ctx, 0, bytes);
     if (st != PSB_OK) return st;
-    if (launch_nchw_to_nhwc(x_dev, ctx->scratch[0], n, c, h * w, 1, s) != cudaSuccess)
+    if (launch_nchw_to_nhwc(x_dev, ctx->scratch[0], n, c, h * w, 1, in_dtype == PSB_DT_S8, amax, ctx->err_dev, s) !=
+        cudaSuccess)
       return PSB_ERR_CUDA;
     a.x = ctx->scratch[0];
+    range_checked = true;     // the conversion pass has looked at every byte
   }
+  // in_max is a promise the kernels rely on (bytes above 127 would read as negative on the tensor path):
+  // passes that touch every input byte anyway verify it for free; the routes that hand the tensor
+  // straight to the copy engine verify it only on request (PSB_CHECK_RANGE)
+  const uint32_t no_limit = in_dtype == PSB_DT_U8 ? 255u : 128u;
+  const bool gathers = tensor_ok && (wt->packed_k || (in_dtype == PSB_DT_U8 && amax > 127u));
+  if (!range_checked && !gathers && (ctx->checks & PSB_CHECK_RANGE) && amax < no_limit) {
+    if (launch_range_check(a.x, (size_t)n * c * h * w, in_dtype == PSB_DT_S8, amax, ctx->err_dev, s) != cudaSuccess)
+      return PSB_ERR_CUDA;
+    range_checked = true;
+  }
+  const uint32_t gather_limit = range_checked ? no_limit : amax;
 
   if (tensor_ok) {
     bool add_corr = false;
@@ -136,7 +149,7 @@ psb_status run_layer(psb_ctx* ctx, const psb_weights* wt, const void* x_dev, uin
       st = ensure_scratch(ctx, 1, (size_t)M * wt->kpad);
       if (st != PSB_OK) return st;
       const uint32_t offset = in_dtype == PSB_DT_U8 ? 128u : 0u;
-      if (launch_im2col_s8(a, wt->kpad, wt->run_pitch, offset, (int8_t*)ctx->scratch[1], s) != cudaSuccess)
+      if (launch_im2col_s8(a, wt->kpad, wt->run_pitch, offset, (int8_t*)ctx->scratch[1], gather_limit, s) != cudaSuccess)
         return PSB_ERR_CUDA;
       a.x = ctx->scratch[1];
       a.in_dtype = PSB_DT_S8;
@@ -149,7 +162,7 @@ psb_status run_layer(psb_ctx* ctx, const psb_weights* wt, const void* x_dev, uin
       const size_t bytes = (size_t)n * c * h * w;   // a multiple of 16: c is
       st = ensure_scratch(ctx, 1, bytes);
       if (st != PSB_OK) return st;
-      if (launch_offset128(a.x, ctx->scratch[1], bytes, s) != cudaSuccess) return PSB_ERR_CUDA;
+      if (launch_offset128(a.x, ctx->scratch[1], bytes, gather_limit, ctx->err_dev, s) != cudaSuccess) return PSB_ERR_CUDA;
       a.x = ctx->scratch[1];
       a.in_dtype = PSB_DT_S8;
       add_corr = true;
@@ -248,6 +261,7 @@ const char* psb_status_string(psb_status st) {
     case PSB_ERR_CUDA: return "PSB_ERR_CUDA";
     case PSB_ERR_TIMEOUT: return "PSB_ERR_TIMEOUT";
     case PSB_ERR_NONFINITE_WEIGHT: return "PSB_ERR_NONFINITE_WEIGHT";
+    case PSB_ERR_RANGE: return "PSB_ERR_RANGE";
     default: return "PSB_ERR_UNKNOWN";
   }
 }
@@ -262,7 +276,26 @@ psb_status psb_device_status(psb_ctx* ctx, void* stream) {
   if (word & kDevErrTimeout) return PSB_ERR_TIMEOUT;
   if (word & kDevErrNonFinite) return PSB_ERR_NONFINITE_WEIGHT;
   if (word & kDevErrBadLevel) return PSB_ERR_BAD_K;
+  if (word & kDevErrRange) return PSB_ERR_RANGE;
   return PSB_OK;
+}
+
+psb_status psb_set_checks(psb_ctx* ctx, uint32_t flags) {
+  if (!ctx || (flags & ~(uint32_t)PSB_CHECK_RANGE)) return PSB_ERR_INVALID_ARG;
+  ctx->checks = flags;
+  return PSB_OK;
+}
+
+psb_status psb_set_wait_limit(psb_ctx* ctx, uint64_t sm_clocks) {
+  if (!ctx) return PSB_ERR_INVALID_ARG;
+  ctx->wait_limit_cycles = sm_clocks ? sm_clocks : kDefaultWaitLimitCycles;
+  return PSB_OK;
+}
+
+psb_status psb_wait_selftest(psb_ctx* ctx, void* stream) {
+  if (!ctx) return PSB_ERR_INVALID_ARG;
+  cudaSetDevice(ctx->device);
+  return launch_wait_selftest(ctx, (cudaStream_t)stream) == cudaSuccess ? PSB_OK : PSB_ERR_CUDA;
 }
 
 psb_status psb_sample_weights(psb_ctx* ctx, const float* w_dev, const psb_wshape* shape,

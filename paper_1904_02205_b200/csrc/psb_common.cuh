@@ -17,6 +17,10 @@ constexpr int kMaxPlanes = 4;
 constexpr uint32_t kDevErrNonFinite = 1u;
 constexpr uint32_t kDevErrTimeout = 2u;
 constexpr uint32_t kDevErrBadLevel = 4u;
+constexpr uint32_t kDevErrRange = 8u;      // an activation byte exceeds the magnitude the caller vouched for
+
+// Bound of every device-side wait, in SM clocks, unless the context says otherwise (about 2 s).
+constexpr unsigned long long kDefaultWaitLimitCycles = 4000000000ull;
 
 // Number of 7-bit digit planes that hold |W_k| = (k + c) * 2^(e - e_base) for
 // every weight of a window of 2^exp_bits octaves: the top value is 2k * 2^span.
@@ -82,6 +86,8 @@ struct psb_ctx {
   size_t scratch_bytes[3] = {0, 0, 0};
   int32_t last_path = 0;
   int sm_count = 0;
+  unsigned long long wait_limit_cycles = psb::kDefaultWaitLimitCycles;   // bound of every device-side wait
+  uint32_t checks = 0;              // PSB_CHECK_* bits: extra device-side validation of the inputs
   void* encode_tiled = nullptr;     // cuTensorMapEncodeTiled
   void* encode_im2col = nullptr;    // cuTensorMapEncodeIm2col
   // measurement aid: event pairs around the contraction launches made since timing was switched on
@@ -208,13 +214,18 @@ cudaError_t launch_shift_add(const ConvArgs& a, const WintTable& wt, cudaStream_
 // gathers [M][kpad] signed bytes (x - offset; zero padding becomes -offset, K padding 0); row kh of the
 // filter window occupies bytes [kh * run_pitch, kh * run_pitch + kw * c) of a matrix row
 cudaError_t launch_im2col_s8(const ConvArgs& a, uint32_t kpad, uint32_t run_pitch, uint32_t offset, int8_t* dst,
-                             cudaStream_t s);
+                             uint32_t limit, cudaStream_t s);
 cudaError_t launch_corr128(const psb_weights* wt, uint32_t level, cudaStream_t s);
-cudaError_t launch_offset128(const void* src, void* dst, size_t bytes, cudaStream_t s);
+// `limit`: largest byte magnitude allowed (255 for unsigned / 128 for signed data = no check); a byte beyond
+// it raises kDevErrRange in *err
+cudaError_t launch_offset128(const void* src, void* dst, size_t bytes, uint32_t limit, uint32_t* err, cudaStream_t s);
 cudaError_t launch_nchw_to_nhwc(const void* src, void* dst, uint32_t N, uint32_t C, uint32_t HW,
-                                uint32_t elem_bytes, cudaStream_t s);
-cudaError_t launch_nhwc_to_nchw(const void* src, void* dst, uint32_t N, uint32_t C, uint32_t HW,
-                                uint32_t elem_bytes, cudaStream_t s);
+                                uint32_t elem_bytes, uint32_t is_signed, uint32_t limit, uint32_t* err,
+                                cudaStream_t s);
+cudaError_t launch_range_check(const void* x, size_t bytes, uint32_t is_signed, uint32_t limit, uint32_t* err,
+                               cudaStream_t s);
+// one tiny CTA waits, with the context's bound, on a barrier that nobody arrives at (psb_tensor.cu)
+cudaError_t launch_wait_selftest(psb_ctx* ctx, cudaStream_t s);
 cudaError_t launch_maxpool(const uint8_t* x, uint32_t nchw, uint32_t N, uint32_t C, uint32_t H,
                            uint32_t W, uint32_t k, uint32_t stride, uint32_t pad, uint8_t* out,
                            cudaStream_t s);

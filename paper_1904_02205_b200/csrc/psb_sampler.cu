@@ -63,7 +63,8 @@ __device__ __forceinline__ void philox4x32_10(uint32_t c0, uint32_t c1, uint32_t
 __device__ __forceinline__ uint32_t small_div_magic(uint32_t d) { return 0xFFFFFFFFu / d + 1u; }
 __device__ __forceinline__ uint32_t small_div(uint32_t t, uint32_t magic) { return magic ? __umulhi(t, magic) : t; }   // magic wraps to 0 for d = 1
 
-// Largest biased exponent of each exponent group; flags Inf/NaN.
+// Largest biased exponent of the finite weights of each exponent group; flags Inf/NaN (which
+// contribute nothing: the finite weights of the group keep the window they would have without it).
 // norm == 1: one block per output channel.  norm == 0: grid-stride over the layer.
 __device__ __forceinline__ void emax_block(const float* __restrict__ w, uint32_t O, uint32_t d,
                                            uint32_t norm, uint32_t* __restrict__ e_max,
@@ -77,14 +78,14 @@ __device__ __forceinline__ void emax_block(const float* __restrict__ w, uint32_t
     for (uint32_t i = threadIdx.x; i < d; i += blockDim.x) {
       uint32_t E = (__float_as_uint(row[i]) >> 23) & 0xFFu;
       bad |= (E == 255u);
-      best = max(best, E);
+      best = max(best, E == 255u ? 0u : E);     // Inf/NaN is flagged and takes no part in the window
     }
   } else {
     size_t total = (size_t)O * d;
     for (size_t i = (size_t)block * blockDim.x + threadIdx.x; i < total; i += (size_t)blocks * blockDim.x) {
       uint32_t E = (__float_as_uint(w[i]) >> 23) & 0xFFu;
       bad |= (E == 255u);
-      best = max(best, E);
+      best = max(best, E == 255u ? 0u : E);
     }
   }
   if (__any_sync(0xFFFFFFFFu, bad) && (threadIdx.x & 31) == 0) atomicOr(err, kDevErrNonFinite);
@@ -93,7 +94,6 @@ __device__ __forceinline__ void emax_block(const float* __restrict__ w, uint32_t
   __syncthreads();
   if (threadIdx.x == 0) {
     for (int i = 1; i < kThreads / 32; ++i) best = max(best, red[i]);
-    if (best == 255u) best = 0;  // error already flagged; keep the window well defined
     // `tag` (a call number in the bits above the exponent) makes the maxima of this call beat
     // whatever an earlier call left in the word, so the words need no clearing between calls
     if (norm) e_max[block] = tag | best;

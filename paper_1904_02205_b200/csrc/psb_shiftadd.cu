@@ -13,6 +13,12 @@ namespace psb {
 
 namespace {
 
+// True when one of the four bytes of `v` exceeds `limit` in magnitude (signed bytes: |b| > limit).
+__device__ __forceinline__ bool bytes_beyond(uint32_t v, uint32_t is_signed, uint32_t limit) {
+  const uint32_t mag = is_signed ? __vabs4(v) : v;        // |-128| = 128 as an unsigned byte
+  return __vcmpgtu4(mag, limit * 0x01010101u) != 0u;
+}
+
 __device__ __forceinline__ int load_act(const void* x, uint32_t dtype, size_t idx) {
   return dtype == PSB_DT_U8 ? (int)((const uint8_t*)x)[idx] : (int)((const int8_t*)x)[idx];
 }
@@ -270,13 +276,41 @@ __global__ void __launch_bounds__(256, 2) dwconv3x3_row_kernel(const ConvArgs a,
 }
 
 // x ^ 0x80 over a whole tensor: unsigned bytes become (x - 128) as signed bytes, 16 per thread.
-__global__ void offset128_kernel(const uint4* __restrict__ src, uint4* __restrict__ dst, size_t n16) {
+__global__ void offset128_kernel(const uint4* __restrict__ src, uint4* __restrict__ dst, size_t n16, uint32_t limit,
+                                 uint32_t* __restrict__ err) {
   pdl_prologue();
+  bool bad = false;
   for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n16; i += (size_t)gridDim.x * blockDim.x) {
     uint4 v = __ldg(src + i);
+    if (limit < 255u)
+      bad |= bytes_beyond(v.x, 0u, limit) | bytes_beyond(v.y, 0u, limit) | bytes_beyond(v.z, 0u, limit) |
+             bytes_beyond(v.w, 0u, limit);
     v.x ^= 0x80808080u; v.y ^= 0x80808080u; v.z ^= 0x80808080u; v.w ^= 0x80808080u;
     dst[i] = v;
   }
+  if (bad) atomicOr(err, kDevErrRange);
+}
+
+// Largest byte magnitude of a tensor against the bound the caller gave (PSB_CHECK_RANGE): 16 bytes per
+// thread and iteration, the ragged tail byte by byte.
+__global__ void range_check_kernel(const uint8_t* __restrict__ x, size_t bytes, uint32_t is_signed, uint32_t limit,
+                                   uint32_t* __restrict__ err) {
+  pdl_prologue();
+  bool bad = false;
+  const size_t head = min(bytes, (size_t)((16u - ((uintptr_t)x & 15u)) & 15u));   // bytes before 16-byte alignment
+  const size_t n16 = (bytes - head) / 16u;
+  const uint4* x16 = reinterpret_cast<const uint4*>(x + head);
+  for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n16; i += (size_t)gridDim.x * blockDim.x) {
+    const uint4 v = __ldg(x16 + i);
+    bad |= bytes_beyond(v.x, is_signed, limit) | bytes_beyond(v.y, is_signed, limit) |
+           bytes_beyond(v.z, is_signed, limit) | bytes_beyond(v.w, is_signed, limit);
+  }
+  if (blockIdx.x == 0) {
+    const size_t tail0 = head + n16 * 16u;
+    for (size_t i = threadIdx.x; i < head; i += blockDim.x) bad |= bytes_beyond((uint32_t)x[i], is_signed, limit);
+    for (size_t i = tail0 + threadIdx.x; i < bytes; i += blockDim.x) bad |= bytes_beyond((uint32_t)x[i], is_signed, limit);
+  }
+  if (bad) atomicOr(err, kDevErrRange);
 }
 
 // Explicit gather of the activation matrix for filters with few input channels (e.g. a 7x7
@@ -292,8 +326,9 @@ constexpr uint32_t kIm2colPix = 32;
 
 __global__ void __launch_bounds__(256) im2col_s8_kernel(const ConvArgs a, uint32_t kpad, uint32_t run_pitch,
                                                        uint32_t offset, uint32_t span_bytes, uint32_t span_pitch,
-                                                       int8_t* __restrict__ dst) {
+                                                       uint32_t limit, int8_t* __restrict__ dst) {
   pdl_prologue();
+  bool bad = false;
   extern __shared__ uint32_t im2col_smem[];                   // [KH][span_pitch / 4] words
   uint8_t* rows = reinterpret_cast<uint8_t*>(im2col_smem);
   const uint32_t strips = (a.OW + kIm2colPix - 1) / kIm2colPix;
@@ -316,10 +351,15 @@ __global__ void __launch_bounds__(256) im2col_s8_kernel(const ConvArgs a, uint32
     const uint8_t* src = x + (((size_t)n * a.H + (row_in ? iy : 0)) * a.W) * a.C + (ptrdiff_t)ix0 * (int)a.C;
     for (uint32_t b = threadIdx.x & 63u; b < span_pitch; b += 64u) {
       uint8_t v = fill;
-      if (row_in && (int)b >= lo_b && (int)b < hi_b) v = (uint8_t)(src[b] ^ flip);
+      if (row_in && (int)b >= lo_b && (int)b < hi_b) {
+        const uint8_t raw = src[b];
+        bad |= bytes_beyond((uint32_t)raw, a.in_dtype == PSB_DT_S8 ? 1u : 0u, limit);
+        v = (uint8_t)(raw ^ flip);
+      }
       rows[kh * span_pitch + b] = v;
     }
   }
+  if (bad) atomicOr(a.err, kDevErrRange);
   __syncthreads();
   const size_t m0 = ((size_t)n * a.OH + oy) * a.OW + ox0;
   const uint32_t run = a.KW * a.C;                            // bytes of one filter row
@@ -352,15 +392,22 @@ __global__ void __launch_bounds__(256) im2col_s8_kernel(const ConvArgs a, uint32
 
 // [N][C][HW] -> [N][HW][C], elements of 1 byte, through a 32x33 tile.
 __global__ void nchw_to_nhwc_u8_kernel(const uint8_t* __restrict__ src, uint8_t* __restrict__ dst,
-                                       uint32_t C, uint32_t HW) {
+                                       uint32_t C, uint32_t HW, uint32_t is_signed, uint32_t limit,
+                                       uint32_t* __restrict__ err) {
   pdl_prologue();
   __shared__ uint8_t tile[32][33];
   const size_t base = (size_t)blockIdx.z * C * HW;
   const uint32_t p0 = blockIdx.x * 32, c0 = blockIdx.y * 32;
+  bool bad = false;
   for (uint32_t r = threadIdx.y; r < 32; r += blockDim.y) {
     uint32_t c = c0 + r, p = p0 + threadIdx.x;
-    if (c < C && p < HW) tile[r][threadIdx.x] = src[base + (size_t)c * HW + p];
+    if (c < C && p < HW) {
+      const uint8_t v = src[base + (size_t)c * HW + p];
+      bad |= bytes_beyond((uint32_t)v, is_signed, limit);
+      tile[r][threadIdx.x] = v;
+    }
   }
+  if (bad) atomicOr(err, kDevErrRange);
   __syncthreads();
   for (uint32_t r = threadIdx.y; r < 32; r += blockDim.y) {
     uint32_t p = p0 + r, c = c0 + threadIdx.x;
@@ -376,7 +423,8 @@ __global__ void nchw_to_nhwc_u8_kernel(const uint8_t* __restrict__ src, uint8_t*
 // (row pitch 132 words: bank = 4 * quad + location).
 __global__ void __launch_bounds__(256) nchw_to_nhwc_u8x4_kernel(const uint8_t* __restrict__ src,
                                                                uint8_t* __restrict__ dst, uint32_t C,
-                                                               uint32_t HW) {
+                                                               uint32_t HW, uint32_t is_signed, uint32_t limit,
+                                                               uint32_t* __restrict__ err) {
   pdl_prologue();
   __shared__ __align__(16) uint32_t tile[8][132];
   const size_t base = (size_t)blockIdx.z * C * HW;
@@ -389,6 +437,9 @@ __global__ void __launch_bounds__(256) nchw_to_nhwc_u8x4_kernel(const uint8_t* _
 #pragma unroll
       for (int k = 0; k < 4; ++k)
         r[k] = __ldg(reinterpret_cast<const uint32_t*>(src + base + (size_t)(c + k) * HW + p));
+      if (bytes_beyond(r[0], is_signed, limit) | bytes_beyond(r[1], is_signed, limit) |
+          bytes_beyond(r[2], is_signed, limit) | bytes_beyond(r[3], is_signed, limit))
+        atomicOr(err, kDevErrRange);
     }
     const uint32_t a = __byte_perm(r[0], r[1], 0x5140), b = __byte_perm(r[2], r[3], 0x5140);
     const uint32_t cc = __byte_perm(r[0], r[1], 0x7362), d = __byte_perm(r[2], r[3], 0x7362);
@@ -493,9 +544,19 @@ uint32_t grid_for(size_t total, uint32_t threads) {
 
 }  // namespace
 
-cudaError_t launch_offset128(const void* src, void* dst, size_t bytes, cudaStream_t s) {
+cudaError_t launch_offset128(const void* src, void* dst, size_t bytes, uint32_t limit, uint32_t* err, cudaStream_t s) {
   const size_t n16 = bytes / 16;
-  launch_pdl(offset128_kernel, grid_for(n16, 256), 256, 0, s, (const uint4*)src, (uint4*)dst, n16); note_launch();
+  launch_pdl(offset128_kernel, grid_for(n16, 256), 256, 0, s, (const uint4*)src, (uint4*)dst, n16, limit, err);
+  note_launch();
+  return cudaGetLastError();
+}
+
+cudaError_t launch_range_check(const void* x, size_t bytes, uint32_t is_signed, uint32_t limit, uint32_t* err,
+                               cudaStream_t s) {
+  uint32_t blocks = grid_for(bytes / 16 + 1, 256);
+  if (blocks > 148u * 8u) blocks = 148u * 8u;
+  launch_pdl(range_check_kernel, blocks, 256, 0, s, (const uint8_t*)x, bytes, is_signed, limit, err);
+  note_launch();
   return cudaGetLastError();
 }
 
@@ -546,7 +607,7 @@ cudaError_t launch_shift_add(const ConvArgs& a, const WintTable& wt, cudaStream_
 }
 
 cudaError_t launch_im2col_s8(const ConvArgs& a, uint32_t kpad, uint32_t run_pitch, uint32_t offset, int8_t* dst,
-                             cudaStream_t s) {
+                             uint32_t limit, cudaStream_t s) {
   const uint32_t strips = (a.OW + kIm2colPix - 1) / kIm2colPix;
   const uint32_t span_bytes = ((kIm2colPix - 1) * a.stride + a.KW) * a.C;
   // a run may be read up to run_pitch + 7 bytes past its start (whole words, two at a time)
@@ -555,20 +616,24 @@ cudaError_t launch_im2col_s8(const ConvArgs& a, uint32_t kpad, uint32_t run_pitc
   if (smem > 48 * 1024 || (uint64_t)a.N * a.OH * strips >= (1ull << 31) || run_pitch % 8u || kpad % 16u ||
       (offset != 0u && offset != 128u) || a.KH * run_pitch > kpad)
     return cudaErrorInvalidValue;
-  launch_pdl(im2col_s8_kernel, a.N * a.OH * strips, 256, smem, s, a, kpad, run_pitch, offset, span_bytes, span_pitch, dst);
+  launch_pdl(im2col_s8_kernel, a.N * a.OH * strips, 256, smem, s, a, kpad, run_pitch, offset, span_bytes, span_pitch, limit,
+             dst);
   note_launch();
   return cudaGetLastError();
 }
 
 cudaError_t launch_nchw_to_nhwc(const void* src, void* dst, uint32_t N, uint32_t C, uint32_t HW,
-                                uint32_t elem_bytes, cudaStream_t s) {
+                                uint32_t elem_bytes, uint32_t is_signed, uint32_t limit, uint32_t* err,
+                                cudaStream_t s) {
   if (elem_bytes != 1) return cudaErrorInvalidValue;
   if (C % 4u == 0 && HW % 4u == 0 && !(((uintptr_t)src | (uintptr_t)dst) & 3u)) {
     dim3 grid4((HW + 127) / 128, (C + 31) / 32, N);
-    launch_pdl(nchw_to_nhwc_u8x4_kernel, grid4, 256, 0, s, (const uint8_t*)src, (uint8_t*)dst, C, HW);
+    launch_pdl(nchw_to_nhwc_u8x4_kernel, grid4, 256, 0, s, (const uint8_t*)src, (uint8_t*)dst, C, HW, is_signed, limit,
+               err);
   } else {
     dim3 grid((HW + 31) / 32, (C + 31) / 32, N), block(32, 8);
-    launch_pdl(nchw_to_nhwc_u8_kernel, grid, block, 0, s, (const uint8_t*)src, (uint8_t*)dst, C, HW);
+    launch_pdl(nchw_to_nhwc_u8_kernel, grid, block, 0, s, (const uint8_t*)src, (uint8_t*)dst, C, HW, is_signed, limit,
+               err);
   }
   note_launch();
   return cudaGetLastError();

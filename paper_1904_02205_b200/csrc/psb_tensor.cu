@@ -46,7 +46,6 @@ constexpr int kThreadsTensor = 32 * (kFirstEpilogueWarp + kEpilogueWarps);
 constexpr uint32_t kTmemCols = 512;
 constexpr uint32_t kTmemBufStride = 256;
 constexpr int kMaxStages = 12;
-constexpr long long kWaitLimitCycles = 4000000000ll;        // about 2 s of SM clocks per wait
 constexpr uint32_t kResidentMaxBytes = 112 * 1024;          // digit planes kept in shared memory
 
 struct TmapSet {
@@ -92,6 +91,7 @@ struct TensorParams {
   uint32_t tiles_x;     // patches per image row: ceil(OW / 8)
   uint32_t Wp_magic, tpi_magic;   // ceil(2^32 / Wp), ceil(2^32 / tpi): quotients by multiply-high (exact in the
                                   // ranges band mode is restricted to)
+  unsigned long long wait_limit;  // bound of every wait in SM clocks
 };
 
 // ---- thin PTX wrappers -------------------------------------------------------
@@ -125,9 +125,16 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
   return ok != 0;
 }
 
-// Bounded wait.  Returns false after kWaitLimitCycles SM clocks without completion, or as soon
+// What a bounded wait consults on its slow path: the CTA-wide give-up flag and the bound in SM clocks.
+struct WaitCtl {
+  volatile uint32_t abort;
+  uint32_t pad;
+  volatile unsigned long long limit;
+};
+
+// Bounded wait.  Returns false after wc->limit SM clocks without completion, or as soon
 // as another thread of the CTA has given up.  (The SM cycle counter is cheap to read.)
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile uint32_t* abort,
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, WaitCtl* wc,
                                           uint32_t backoff_ns = 0) {
   if (mbar_try_wait(bar, parity)) return true;
   const long long t0 = clock64();
@@ -138,8 +145,8 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
     ++spins;
     if (backoff_ns || spins > 4u) __nanosleep(backoff_ns ? backoff_ns : (spins > 32u ? 256u : 64u));
     if ((spins & 15u) == 0u) {
-      if (*abort) return false;
-      if (clock64() - t0 > kWaitLimitCycles) return false;
+      if (wc->abort) return false;
+      if ((unsigned long long)(clock64() - t0) > wc->limit) return false;
     }
   }
   return true;
@@ -310,7 +317,7 @@ struct SharedCtl {
   unsigned long long planes_full[kPlaneBars];
   unsigned long long started[2];        // per accumulator buffer: the zeroing MMA of the pass has been issued
   uint32_t tmem_base;
-  volatile uint32_t abort;
+  WaitCtl wait;
   float2 scb[kEpilogueWarps][16];       // per epilogue warp: (scale * 2^(e_base - log2 k), bias)
   long long corr[kEpilogueWarps][16];   // per epilogue warp: integer addend per channel
 };
@@ -598,7 +605,7 @@ __device__ __noinline__ bool epilogue_uniform(const TensorParams& p, SharedCtl* 
   const uint32_t row = quarter * 32u + lane;
   const uint32_t l = a.uniform_log2k;
   const bool use_corr = p.corr[l] != nullptr;
-  volatile uint32_t* abort = &ctl->abort;
+  WaitCtl* abort = &ctl->wait;
   const uint8_t* const res_base = (const uint8_t*)a.residual;
   uint8_t* const q_base = (uint8_t*)a.q_out;
   RowMap rm;
@@ -688,7 +695,7 @@ __device__ __noinline__ bool epilogue_uniform_band(const TensorParams& p, Shared
   const uint32_t row = quarter * 32u + lane;
   const uint32_t l = a.uniform_log2k;
   const bool use_corr = p.corr[l] != nullptr;
-  volatile uint32_t* abort = &ctl->abort;
+  WaitCtl* abort = &ctl->wait;
   const uint8_t* const res_base = (const uint8_t*)a.residual;
   uint8_t* const q_base = (uint8_t*)a.q_out;
   RowMapBand rm;
@@ -783,7 +790,7 @@ template <int BK>
 __device__ __noinline__ bool mma_role(const TensorParams& p, SharedCtl* ctl, uint32_t tmem_base, uint32_t ring_addr,
                                       uint32_t planes_addr, uint32_t stage_bytes, uint32_t sub_bytes,
                                       uint32_t k_iters, uint32_t mine) {
-  volatile uint32_t* abort = &ctl->abort;
+  WaitCtl* abort = &ctl->wait;
   const uint32_t group = p.group, stages = p.stages, resident = p.resident, stage_bytes_a = p.stage_bytes_a;
   const uint32_t level_mask = p.a.level_mask;
   const uint32_t band = p.band, row_bytes = p.Wp * p.a.C, KH = p.a.KH, KW = p.a.KW;
@@ -908,7 +915,8 @@ psb_mma_kernel(const __grid_constant__ TmapSet maps, const __grid_constant__ Ten
       }
     }
     for (int b = 0; b < 2; ++b) mbar_init(smem_u32(&ctl->started[b]), 1);
-    ctl->abort = 0;
+    ctl->wait.abort = 0;
+    ctl->wait.limit = p.wait_limit;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (threadIdx.x == 32) {
@@ -926,7 +934,7 @@ psb_mma_kernel(const __grid_constant__ TmapSet maps, const __grid_constant__ Ten
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = ctl->tmem_base;
-  volatile uint32_t* abort = &ctl->abort;
+  WaitCtl* abort = &ctl->wait;
   bool failed = false;
   // The kernel is launched with programmatic stream serialisation: a CTA may get here while the
   // kernel before it in the stream is still draining.  Nothing above touches global memory; from
@@ -1152,7 +1160,7 @@ psb_mma_kernel(const __grid_constant__ TmapSet maps, const __grid_constant__ Ten
   // ------------------------------------------------------------- common exit
   if (failed) {
     if (lane == 0) {
-      *abort = 1u;
+      abort->abort = 1u;
       atomicOr(p.a.err, kDevErrTimeout);
     }
     // give copies and MMAs already in flight time to land before the CTA retires
@@ -1166,6 +1174,28 @@ psb_mma_kernel(const __grid_constant__ TmapSet maps, const __grid_constant__ Ten
                  "r"(kTmemCols)
                  : "memory");
   }
+}
+
+// One warp waits, with the given bound, on a barrier that has no other party: the wait runs out,
+// the kernel raises the error word and returns.  Exercises mbar_wait's give-up path as the contraction
+// kernel would take it, with nothing in flight.
+__global__ void wait_selftest_kernel(unsigned long long limit, uint32_t* __restrict__ err) {
+  __shared__ unsigned long long bar;
+  __shared__ WaitCtl wc;
+  if (threadIdx.x == 0) {
+    mbar_init(smem_u32(&bar), 1);
+    wc.abort = 0;
+    wc.limit = limit;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  __syncthreads();
+  bool ok = true;
+  if (threadIdx.x == 0) ok = mbar_wait(smem_u32(&bar), 0u, &wc);
+  if (!ok) {
+    wc.abort = 1u;
+    atomicOr(err, kDevErrTimeout);
+  }
+  __syncthreads();
 }
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*,
@@ -1191,6 +1221,12 @@ constexpr size_t kSmemBudget = 227 * 1024;
 
 }  // namespace
 
+cudaError_t launch_wait_selftest(psb_ctx* ctx, cudaStream_t s) {
+  wait_selftest_kernel<<<1, 32, 0, s>>>(ctx->wait_limit_cycles, ctx->err_dev);
+  note_launch();
+  return cudaGetLastError();
+}
+
 psb_status tensor_supported(const psb_ctx* ctx, const psb_weights* wt, const ConvArgs& a) {
   if (!ctx->encode_tiled || !ctx->encode_im2col) return PSB_ERR_UNSUPPORTED;
   if (!wt->has_planes || a.groups != 1) return PSB_ERR_UNSUPPORTED;
@@ -1212,6 +1248,7 @@ psb_status launch_tensor(psb_ctx* ctx, const psb_weights* wt, const ConvArgs& a,
   TmapSet maps;
   TensorParams p;
   p.a = a;
+  p.wait_limit = ctx->wait_limit_cycles;
   p.M = a.N * a.OH * a.OW;
   p.m_tiles = (p.M + kTileM - 1) / kTileM;
   p.o_tiles = wt->o_tiles;

@@ -346,8 +346,9 @@ def test_auto_path_selection(psb, ctx, oracle):
 
 @pytest.mark.parametrize("log2k", [0, 3])
 def test_config2_full_size_sampled_outputs(psb, ctx, oracle, log2k):
-    """The 3x3 64->64 conv on 56x56, batch 32, NCHW, as the benchmark launches it: accumulators at
-    4000 sampled outputs against the oracle, all image borders included, plus whole-tensor properties."""
+    """The 3x3 64->64 conv on 56x56, batch 32, NCHW, with all three outputs wanted (the general output loop;
+    the launch the benchmark times, codes only, is the next test): accumulators at 4000 sampled outputs
+    against the oracle, all image borders included, plus whole-tensor properties."""
     import torch
     from workloads import config2_conv
 
@@ -476,3 +477,176 @@ def test_int8_issue_rate_probe_reports_a_plausible_ceiling(psb, ctx):
     assert tops > 100.0
     with pytest.raises(psb.PsbError):
         ctx.int8_mma_probe(200, 10)      # columns must be a multiple of 16
+
+
+# ------------------------------------- config 2 in the launch configuration the benchmark times
+
+@pytest.mark.parametrize("log2k", [0, 1, 2, 3, 4])
+def test_config2_full_size_codes_only_planar_as_benchmarked(psb, ctx, oracle, log2k):
+    """The launch the default benchmark step makes: planar (NCHW) input, only re-quantised codes
+    wanted, tensor path (band mode, planar stores), every draw count of the sweep.  Codes against the
+    oracle at 4000 sampled outputs (image borders included) and on two whole images."""
+    import torch
+    from workloads import config2_conv
+
+    c = config2_conv()
+    dev = ctx.device
+    wt = ctx.sample_weights(torch.from_numpy(c["w"]).to(dev), seed=c["seed"], layer_id=0, level_mask=1 << log2k)
+    ctx.set_sample_map(None, log2k)
+    q_buf = torch.full((32 * 64 * 56 * 56 + 128,), 0x5A, dtype=torch.uint8, device=dev)
+    out = ctx.conv2d(wt, torch.from_numpy(c["x"]).to(dev), psb.PSB_LAYOUT_NCHW, 1, 1,
+                     torch.from_numpy(c["scale"]).to(dev), torch.from_numpy(c["bias"]).to(dev), True,
+                     c["inv_step"], 0, 15, in_max=15, want=("q",), out={"q": q_buf[64:-64].view(32, 64, 56, 56)})
+    assert ctx.device_status() == 0 and ctx.last_path() == psb.PSB_PATH_TENSOR
+    full = q_buf.cpu().numpy()
+    assert (full[:64] == 0x5A).all() and (full[-64:] == 0x5A).all(), "guard band overwritten"
+    q = out["q"].cpu().numpy()
+    W, eb, _ = oracle.sample_level(c["w"], c["seed"], 0, log2k)
+    g = oracle.geom(c["x"].shape, oracle.NCHW, oracle.U8, c["w"].shape, 1, 1, 1)
+    rng = np.random.default_rng(30 + log2k)
+    pts = np.stack([rng.integers(0, 32, 4000), rng.integers(0, 64, 4000), rng.integers(0, 56, 4000),
+                    rng.integers(0, 56, 4000)], 1)
+    pts[:500, 2] = rng.choice([0, 55], 500)
+    pts[250:750, 3] = rng.choice([0, 55], 500)
+    ref = oracle.conv_acc_points(c["x"], g, {log2k: W}, pts, uniform_log2k=log2k)
+    for t in range(4000):
+        n, o, oy, ox = pts[t]
+        y = oracle.dequant_one(ref[t], c["scale"][o], eb[o], log2k, c["bias"][o], relu=True)
+        assert q[n, o, oy, ox] == oracle.requant_one(y, c["inv_step"], 0, 15), (t, pts[t])
+    for n in (0, 31):                                   # the first and the last image, every output
+        xi = np.ascontiguousarray(c["x"][n:n + 1])
+        g1 = oracle.geom(xi.shape, oracle.NCHW, oracle.U8, c["w"].shape, 1, 1, 1)
+        acc = oracle.conv_acc(xi, g1, {log2k: W}, uniform_log2k=log2k)
+        _, qo = oracle.epilogue(acc, g1, c["scale"], c["bias"], eb, True, c["inv_step"], 0, 15, uniform_log2k=log2k)
+        assert np.array_equal(q[n].astype(np.int32), qo[0]), "image %d" % n
+    wt.free()
+
+
+# (N, C, H, W, O, K, pad, layout): codes-only output at k = 32 and 64 needs four digit planes; plain tiles
+# (1x1, strided) and band mode (3x3 stride 1), channels-last and planar
+@pytest.mark.parametrize("log2k", [5, 6])
+@pytest.mark.parametrize("case", [(2, 64, 13, 12, 64, 1, 0, 1), (2, 64, 14, 13, 80, 3, 1, 1), (3, 128, 9, 11, 64, 3, 1, 0),
+                                  (2, 256, 9, 9, 128, 1, 0, 1)])
+def test_tensor_path_codes_only_four_planes(psb, ctx, oracle, log2k, case):
+    N, C, H, W, O, K, pad, layout = case
+    rng = np.random.default_rng(abs(hash((case, log2k))) % 2 ** 31)
+    w, x, scale, bias = _layer_inputs(rng, N, C, H, W, O, K, K, 1, layout)
+    OH, OW = H + 2 * pad - K + 1, W + 2 * pad - K + 1
+    res = rng.integers(0, 16, size=(N, O, OH, OW) if layout == 0 else (N, OH, OW, O)).astype(np.uint8)
+    for r in (None, res):
+        g = _both(psb, ctx, oracle, w, x, layout, 1, 1, pad, [log2k], scale, bias, inv_step=0.5, residual=r,
+                  res_scale=0.3 if r is not None else 0.0, in_max=15, path=psb.PSB_PATH_TENSOR, want=("q",))
+        assert g["path"] == psb.PSB_PATH_TENSOR
+
+
+@pytest.mark.parametrize("exp_bits", [2, 3])
+@pytest.mark.parametrize("K", [1, 3])
+def test_tensor_path_codes_only_map_one_and_two_planes(psb, ctx, oracle, exp_bits, K):
+    """Narrow exponent windows need one or two digit planes; codes only under a per-location map."""
+    rng = np.random.default_rng(100 * exp_bits + K)
+    N, C, H, W, O = 2, 64, 11, 16, 72
+    w, x, scale, bias = _layer_inputs(rng, N, C, H, W, O, K, K, 1, 1)
+    levels = [0, 1, 2] if exp_bits == 2 else [0, 2, 3]
+    kmap = rng.choice(levels, size=(N, H, W)).astype(np.uint8)
+    kmap[0, :5] = levels[1]
+    res = rng.integers(0, 16, size=(N, H, W, O)).astype(np.uint8)
+    for r in (None, res):
+        g = _both(psb, ctx, oracle, w, x, 1, 1, 1, K // 2, levels, scale, bias, kmap=kmap, inv_step=0.5, residual=r,
+                  res_scale=0.3 if r is not None else 0.0, exp_bits=exp_bits, in_max=15, path=psb.PSB_PATH_TENSOR,
+                  want=("q",))
+        assert g["path"] == psb.PSB_PATH_TENSOR
+
+
+@pytest.mark.parametrize("norm", [0, 1])
+def test_nonfinite_weight_is_flagged_and_leaves_the_other_weights_alone(psb, ctx, oracle, norm):
+    """A NaN or Inf raises the error word; every finite weight keeps the integer it would have had with a
+    zero in that place (the oracle refuses the filter, so it is given the zero)."""
+    import torch
+
+    rng = np.random.default_rng(8 + norm)
+    w = rng.normal(0, 0.1, size=(24, 40, 3, 3)).astype(np.float32)
+    w[5, 7, 1, 1] = 7.5                      # the largest weight of row 5 sits next to the NaN
+    bad = w.copy()
+    bad[5, 3, 0, 2] = np.nan
+    bad[17, 0, 0, 0] = np.inf
+    clean = w.copy()
+    clean[5, 3, 0, 2] = 0.0
+    clean[17, 0, 0, 0] = 0.0
+    wt = ctx.sample_weights(torch.from_numpy(bad).cuda(), seed=3, layer_id=1, level_mask=0b1000, norm=norm)
+    Wg, ebg = (v.cpu().numpy() for v in ctx.weights_export(wt, 3))
+    assert ctx.device_status() == psb.PSB_ERR_NONFINITE_WEIGHT
+    Wo, ebo, _ = oracle.sample_level(clean, 3, 1, 3, norm=norm)
+    assert np.array_equal(ebg, ebo) and np.array_equal(Wg.astype(np.int64), Wo)
+    wt.free()
+    # the allocation-free entry point has no error word: same integers, nothing reported
+    wint = torch.zeros(bad.shape, dtype=torch.int32, device=ctx.device)
+    eb = torch.zeros(24, dtype=torch.int32, device=ctx.device)
+    psb.sample_level_static(torch.from_numpy(bad).cuda(), wint, eb, seed=3, layer_id=1, log2k=3, norm=norm)
+    assert np.array_equal(eb.cpu().numpy(), ebo) and np.array_equal(wint.cpu().numpy().astype(np.int64), Wo)
+    assert ctx.device_status() == 0
+
+
+def test_a_wait_that_runs_out_is_reported_and_the_context_stays_usable(psb, oracle):
+    """The bounded wait of the kernels: a thread block waits on a barrier nobody arrives at, gives up after
+    the bound, raises the error word and returns; the next ordinary call works."""
+    c = psb.Context(0)
+    c.set_wait_limit(100000)
+    c.wait_selftest()
+    assert c.device_status() == psb.PSB_ERR_TIMEOUT
+    assert c.device_status() == 0
+    rng = np.random.default_rng(41)
+    w, x, scale, bias = _layer_inputs(rng, 2, 64, 12, 12, 64, 3, 3, 1, 1)
+    _both(psb, c, oracle, w, x, 1, 1, 1, 1, [3], scale, bias, in_max=15, path=psb.PSB_PATH_TENSOR)   # short bound kept
+    c.set_wait_limit(0)
+    _both(psb, c, oracle, w, x, 1, 1, 1, 1, [3], scale, bias, in_max=15, path=psb.PSB_PATH_TENSOR, want=("q",))
+    c.close()
+
+
+def test_activation_beyond_in_max_is_reported(psb, ctx):
+    """in_max is a promise; a byte beyond it is reported instead of silently changing the result."""
+    import torch
+
+    dev = ctx.device
+    w = torch.randn(64, 64, 3, 3, device=dev)
+    wt = ctx.sample_weights(w, level_mask=0b1000)
+    ctx.set_sample_map(None, 3)
+    sc = torch.ones(64, device=dev)
+    good = torch.randint(0, 16, (2, 64, 12, 12), dtype=torch.uint8, device=dev)
+    bad = good.clone()
+    bad[1, 40, 7, 3] = 16
+    # planar input: the layout conversion looks at every byte anyway
+    ctx.conv2d(wt, good, psb.PSB_LAYOUT_NCHW, 1, 1, sc, sc, True, 1.0, 0, 15, in_max=15)
+    assert ctx.device_status() == 0
+    ctx.conv2d(wt, bad, psb.PSB_LAYOUT_NCHW, 1, 1, sc, sc, True, 1.0, 0, 15, in_max=15)
+    assert ctx.device_status() == psb.PSB_ERR_RANGE
+    # channels-last input goes straight to the copy engine: verified on request
+    good_l, bad_l = good.permute(0, 2, 3, 1).contiguous(), bad.permute(0, 2, 3, 1).contiguous()
+    ctx.conv2d(wt, bad_l, psb.PSB_LAYOUT_NHWC, 1, 1, sc, sc, True, 1.0, 0, 15, in_max=15)
+    assert ctx.device_status() == 0
+    ctx.set_checks(psb.PSB_CHECK_RANGE)
+    for path in (psb.PSB_PATH_TENSOR, psb.PSB_PATH_SHIFT_ADD):
+        ctx.conv2d(wt, good_l, psb.PSB_LAYOUT_NHWC, 1, 1, sc, sc, True, 1.0, 0, 15, in_max=15, path=path)
+        assert ctx.device_status() == 0
+        ctx.conv2d(wt, bad_l, psb.PSB_LAYOUT_NHWC, 1, 1, sc, sc, True, 1.0, 0, 15, in_max=15, path=path)
+        assert ctx.device_status() == psb.PSB_ERR_RANGE
+    # signed data: magnitudes
+    sg = torch.randint(-15, 16, (2, 12, 12, 64), dtype=torch.int8, device=dev)
+    ctx.conv2d(wt, sg, psb.PSB_LAYOUT_NHWC, 1, 1, sc, sc, True, 1.0, 0, 15, in_max=15)
+    assert ctx.device_status() == 0
+    sg[0, 0, 5, 63] = -16
+    ctx.conv2d(wt, sg, psb.PSB_LAYOUT_NHWC, 1, 1, sc, sc, True, 1.0, 0, 15, in_max=15)
+    assert ctx.device_status() == psb.PSB_ERR_RANGE
+    ctx.set_checks(0)
+    wt.free()
+    # gathered stem (3 input channels): the gather verifies it
+    w3 = torch.randn(16, 3, 3, 3, device=dev)
+    wt3 = ctx.sample_weights(w3, level_mask=0b1000)
+    img = torch.randint(0, 101, (2, 20, 20, 3), dtype=torch.uint8, device=dev)
+    sc16 = torch.ones(16, device=dev)
+    ctx.conv2d(wt3, img, psb.PSB_LAYOUT_NHWC, 2, 1, sc16, sc16, True, 1.0, 0, 255, in_max=100, path=psb.PSB_PATH_TENSOR)
+    assert ctx.device_status() == 0
+    img[1, 19, 19, 2] = 101
+    ctx.conv2d(wt3, img, psb.PSB_LAYOUT_NHWC, 2, 1, sc16, sc16, True, 1.0, 0, 255, in_max=100, path=psb.PSB_PATH_TENSOR)
+    assert ctx.device_status() == psb.PSB_ERR_RANGE
+    ctx.set_sample_map(None, 0)
+    wt3.free()

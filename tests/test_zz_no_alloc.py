@@ -4,7 +4,8 @@ psb_sample_level_static serves hosts that cannot call cudaMalloc when they need 
 (real-time loops, work beside a graph capture, fixed memory budgets): it keeps its scratch in
 a fixed array inside the library.  Here it is called through the C ABI twice in a row - the
 second call on a smaller, different filter, so that anything left in the shared array by the
-first call would show - and compared bit for bit with psb_sample_weights + psb_weights_export.
+first call would show - and compared bit for bit with psb_sample_weights + psb_weights_export
+and with the CPU oracle.
 Collected last so that a failure here cannot hide another test's result.
 """
 import numpy as np
@@ -52,6 +53,13 @@ def test_static_scratch_sampler_matches_the_allocating_one_twice_in_a_row(norm):
         ref_w, ref_e = _reference(psb, ctx, w, groups, seed, 5, log2k, exp_bits, norm)
         assert np.array_equal(e_base.cpu().numpy(), ref_e)
         assert np.array_equal(wint.cpu().numpy(), ref_w)      # integers: bit-exact, as in the other tests
+        # and directly against the CPU oracle
+        from oracle import psb_oracle
+
+        psb_oracle.build()
+        Wo, ebo, _ = psb_oracle.sample_level(w.cpu().numpy(), seed, 5, log2k, exp_bits=exp_bits, norm=norm)
+        assert np.array_equal(e_base.cpu().numpy(), ebo)
+        assert np.array_equal(wint.cpu().numpy().astype(np.int64), Wo)
     # sizes beyond the fixed array are refused with an error, nothing is launched
     big = torch.zeros((psb.PSB_STATIC_MAX_OUT_CH + 1, 1, 1, 1), dtype=torch.float32, device=dev)
     out = torch.zeros((psb.PSB_STATIC_MAX_OUT_CH + 1, 1, 1, 1), dtype=torch.int32, device=dev)

@@ -36,8 +36,10 @@ void free_weights_storage(psb_weights* w) {
   }
   if (w->e_base) cudaFree(w->e_base);
   if (w->e_max) cudaFree(w->e_max);
+  if (w->rowsum256) cudaFree(w->rowsum256);
   w->e_base = nullptr;
   w->e_max = nullptr;
+  w->rowsum256 = nullptr;
 }
 
 psb_status check_epilogue(const psb_epilogue& ep) {
@@ -343,6 +345,8 @@ psb_status psb_sample_weights(psb_ctx* ctx, const float* w_dev, const psb_wshape
     w->n_kb = w->packed_k ? w->n_cb : shape->kh * shape->kw * w->n_cb;
     bool ok = cudaMalloc(&w->e_base, sizeof(int32_t) * shape->out_ch) == cudaSuccess &&
               cudaMalloc(&w->e_max, sizeof(uint32_t) * shape->out_ch) == cudaSuccess &&
+              (!w->has_planes ||
+               cudaMalloc(&w->rowsum256, sizeof(uint32_t) * kMaxLevels * shape->out_ch) == cudaSuccess) &&
               cudaMemsetAsync(w->e_max, 0, sizeof(uint32_t) * shape->out_ch, s) == cudaSuccess;
     for (uint32_t l = 0; ok && l < (uint32_t)kMaxLevels; ++l) {
       if (!((cfg.level_mask >> l) & 1u)) continue;

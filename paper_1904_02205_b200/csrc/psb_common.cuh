@@ -73,6 +73,9 @@ struct psb_weights {
   int32_t* e_base = nullptr;   // [O]
   uint32_t* e_max = nullptr;   // [O] scratch of the window reduction: (call number << 8) | biased exponent
   uint32_t e_calls = 0;        // sampling calls made on this handle, modulo 2^24
+  uint32_t* rowsum256 = nullptr;  // [kMaxLevels][O] row sums of |W_k| of the last sampling, in units of 256 (each
+                                  // weight rounded up): the contraction derives from them whether its accumulators
+                                  // fit 32 bits; kept for filters with digit planes only
   int device;
 };
 

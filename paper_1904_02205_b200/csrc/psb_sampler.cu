@@ -20,6 +20,7 @@ namespace {
 
 constexpr int kThreads = 256;
 constexpr int kStage = 2048;  // weights staged in shared memory per block
+constexpr int kRowSumRows = 128;   // filter rows per block for which the sampler keeps sums of |W_k|
 
 // Philox4x32-10 (Salmon et al., SC'11): ten rounds of two 32x32->64 multiplies and
 // xors; the key advances by the two Weyl constants after every round.  The ten round keys
@@ -69,8 +70,12 @@ __device__ __forceinline__ uint32_t small_div(uint32_t t, uint32_t magic) { retu
 __device__ __forceinline__ void emax_block(const float* __restrict__ w, uint32_t O, uint32_t d,
                                            uint32_t norm, uint32_t* __restrict__ e_max,
                                            uint32_t* __restrict__ err, uint32_t block, uint32_t blocks,
-                                           uint32_t tag) {
+                                           uint32_t tag, uint32_t* __restrict__ rowsum) {
   __shared__ uint32_t red[kThreads / 32];
+  // the sampling pass that follows adds its row sums of |W_k| into these words: start them at zero
+  if (rowsum)
+    for (uint32_t i = block * blockDim.x + threadIdx.x; i < (uint32_t)kMaxLevels * O; i += blocks * blockDim.x)
+      rowsum[i] = 0u;
   uint32_t best = 0;
   bool bad = false;
   if (norm) {
@@ -102,9 +107,10 @@ __device__ __forceinline__ void emax_block(const float* __restrict__ w, uint32_t
 }
 
 __global__ void emax_kernel(const float* __restrict__ w, uint32_t O, uint32_t d, uint32_t norm,
-                            uint32_t* __restrict__ e_max, uint32_t* __restrict__ err, uint32_t tag) {
+                            uint32_t* __restrict__ e_max, uint32_t* __restrict__ err, uint32_t tag,
+                            uint32_t* __restrict__ rowsum) {
   pdl_prologue();
-  emax_block(w, O, d, norm, e_max, err, blockIdx.x, gridDim.x, tag);
+  emax_block(w, O, d, norm, e_max, err, blockIdx.x, gridDim.x, tag, rowsum);
 }
 
 struct SampleParams {
@@ -119,6 +125,7 @@ struct SampleParams {
   const uint32_t* e_max;
   uint32_t e_tag;                  // call number the words of e_max must carry (bits 8 and up)
   int32_t* e_base;
+  uint32_t* rowsum;                // [kMaxLevels][O] row sums of |W_k| / 256 (see psb_weights), or null
   int32_t* wint[kMaxLevels];
   int8_t* planes[kMaxLevels];
   int planes_count[kMaxLevels];
@@ -132,6 +139,14 @@ __device__ __forceinline__ void sample_block(const SampleParams& p, uint32_t blo
   const uint32_t packed_kw = p.packed_kw, run_pitch = p.run_pitch, has_planes = p.has_planes;
   const uint32_t bk = p.bk, n_cb = p.n_cb, n_kb = p.n_kb;
   const PhiloxKeys keys(seed_lo, seed_hi);
+  // Row sums of |W_k| (in units of 256, each weight rounded up) for the bound that lets the contraction
+  // recombine its digit planes in 32 bits: gathered per block in shared memory, then added to the layer's words
+  __shared__ uint32_t row_sum[kMaxLevels][kRowSumRows];
+  uint32_t* const rowsum = p.rowsum;
+  const bool track = rowsum != nullptr && p.rows_per_block <= (uint32_t)kRowSumRows;
+  if (track)
+    for (uint32_t i = threadIdx.x; i < (uint32_t)(kMaxLevels * kRowSumRows); i += blockDim.x)
+      row_sum[i / kRowSumRows][i % kRowSumRows] = 0u;
   const uint32_t row_block = block / p.ch_chunks;
   const uint32_t chunk = block % p.ch_chunks;
   const uint32_t o0 = row_block * p.rows_per_block;
@@ -209,6 +224,13 @@ __device__ __forceinline__ void sample_block(const SampleParams& p, uint32_t blo
       if (!((level_mask >> l) & 1u)) continue;
       const uint32_t mag = live ? (((1u << l) + cnt[l]) << sh) : 0u;
       p.wint[l][wpos] = neg ? -(int32_t)mag : (int32_t)mag;
+      if (track) {
+        // lanes of a warp mostly share a row: one shared-memory add per row and warp
+        const uint32_t lanes = __activemask();
+        const uint32_t peers = __match_any_sync(lanes, r);
+        const uint32_t sum = __reduce_add_sync(peers, (mag + 255u) >> 8);
+        if ((threadIdx.x & 31u) == (uint32_t)__ffs((int)peers) - 1u && sum) atomicAdd(&row_sum[l][r], sum);
+      }
       if (has_planes) {
         const int P = p.planes_count[l];
         int8_t* tile = p.planes[l] + ((size_t)jt * n_kb + kb) * ((size_t)P * kTileN * bk);
@@ -216,6 +238,18 @@ __device__ __forceinline__ void sample_block(const SampleParams& p, uint32_t blo
           const int digit = (int)((mag >> (kDigitBits * pl)) & 0x7Fu);
           tile[plane_offset((uint32_t)pl * kTileN + on, kin, bk)] = (int8_t)(neg ? -digit : digit);
         }
+      }
+    }
+  }
+  if (rowsum) {
+    __syncthreads();
+#pragma unroll
+    for (int l = 0; l < kMaxLevels; ++l) {
+      if (!((level_mask >> l) & 1u)) continue;
+      for (uint32_t r = threadIdx.x; r < rows; r += blockDim.x) {
+        // a block that could not keep sums (more rows than the table holds) leaves the bound unknown
+        if (!track) atomicMax(&rowsum[(uint32_t)l * p.O + o0 + r], 0xFFFFFFFFu);
+        else if (row_sum[l][r]) atomicAdd(&rowsum[(uint32_t)l * p.O + o0 + r], row_sum[l][r]);
       }
     }
   }
@@ -250,7 +284,7 @@ __global__ void __launch_bounds__(kThreads) emax_batch_kernel(const BatchEntry* 
   pdl_prologue();
   const BatchEntry& e = entries[find_entry(entries, n, blockIdx.x, true)];
   emax_block(e.p.w, e.p.O, e.p.d, e.p.norm, const_cast<uint32_t*>(e.p.e_max), err,
-             blockIdx.x - e.emax_first, e.emax_blocks, 0u);
+             blockIdx.x - e.emax_first, e.emax_blocks, 0u, e.p.rowsum);
 }
 
 __global__ void __launch_bounds__(kThreads) sample_batch_kernel(const BatchEntry* __restrict__ entries, uint32_t n,
@@ -338,6 +372,7 @@ uint32_t fill_sample_params(const float* w_dev, const psb_weights* wt, uint32_t*
   p.e_max = e_max;
   p.e_tag = 0;
   p.e_base = wt->e_base;
+  p.rowsum = wt->rowsum256;
   for (int l = 0; l < kMaxLevels; ++l) {
     p.wint[l] = wt->level[l].wint;
     p.planes[l] = wt->level[l].planes;
@@ -367,7 +402,7 @@ cudaError_t launch_sampler(const float* w_dev, psb_weights* wt, uint32_t* err_de
     wt->e_calls = 1u;
   }
   launch_pdl(emax_kernel, emax_blocks_for(O, wt->d, wt->cfg.norm), kThreads, 0, s, w_dev, O, wt->d, wt->cfg.norm,
-             wt->e_max, err_dev, wt->e_calls << 8); note_launch();
+             wt->e_max, err_dev, wt->e_calls << 8, wt->rowsum256); note_launch();
   SampleParams p;
   const uint32_t blocks = fill_sample_params(w_dev, wt, wt->e_max, p);
   p.e_tag = wt->e_calls;
@@ -570,12 +605,12 @@ extern "C" psb_status psb_sample_level_static(const float* w_dev, const psb_wsha
   // the array keeps the previous call's maxima: the reduction must start from zero
   if (cudaMemsetAsync(e_max, 0, sizeof(uint32_t) * O, s) != cudaSuccess) return PSB_ERR_CUDA;
   if (cfg->norm) {
-    emax_kernel<<<O, kThreads, 0, s>>>(w_dev, O, d, 1, e_max, err_sink, 0u); note_launch();
+    emax_kernel<<<O, kThreads, 0, s>>>(w_dev, O, d, 1, e_max, err_sink, 0u, nullptr); note_launch();
   } else {
     size_t total = (size_t)O * d;
     uint32_t blocks = (uint32_t)((total + kThreads * 8 - 1) / (kThreads * 8));
     blocks = blocks < 1 ? 1 : (blocks > 1184 ? 1184 : blocks);
-    emax_kernel<<<blocks, kThreads, 0, s>>>(w_dev, O, d, 0, e_max, err_sink, 0u); note_launch();
+    emax_kernel<<<blocks, kThreads, 0, s>>>(w_dev, O, d, 0, e_max, err_sink, 0u, nullptr); note_launch();
   }
   size_t total = (size_t)O * d;
   uint32_t blocks = (uint32_t)((total + kThreads - 1) / kThreads);

@@ -67,7 +67,8 @@ struct TensorParams {
   uint32_t resident;    // 1: the CTA keeps the digit planes of its channel tile in shared memory
   uint32_t ctas_per_otile;
   uint32_t resident_bytes;
-  uint32_t narrow;      // P <= 3 and plane sums below 2^22 (2) or 2^24 (1): 32-bit recombination; 3: whole sum below 2^31
+  const uint32_t* rowsum256;   // [level][O] row sums of |W_k| in units of 256 (rounded up), or null
+  uint32_t amax;        // largest activation magnitude the caller vouches for
   const long long* corr[kMaxLevels];  // per-channel integer addend, or null
   const int8_t* planes_ptr[kMaxLevels];  // digit planes: [o_tile][K block][P * 64 rows][BK], pre-swizzled tiles
   // Band mode (stride-1 filters with taps, one channel block, resident planes): a tile is 128
@@ -318,56 +319,62 @@ struct SharedCtl {
   unsigned long long started[2];        // per accumulator buffer: the zeroing MMA of the pass has been issued
   uint32_t tmem_base;
   WaitCtl wait;
-  float2 scb[kEpilogueWarps][16];       // per epilogue warp: (scale * 2^(e_base - log2 k), bias)
+  alignas(16) float2 scb[kEpilogueWarps][16];   // per epilogue warp: (scale * 2^(e_base - log2 k), bias), read two
+                                                // channels (16 bytes) at a time
   long long corr[kEpilogueWarps][16];   // per epilogue warp: integer addend per channel
 };
 
 // Output arithmetic of one 16-channel chunk held in registers (v[plane][channel]), common case:
-// only re-quantised bytes are wanted.  Same arithmetic as dequant()/requant(), arranged for the
-// main pipes: integer <-> float conversions run on a slow pipe (a quarter of the FMA rate), so
-// small integers are converted with exponent tricks instead:
-//   float(n) = as_float(0x4B000000 | n) - 2^23              for 0 <= n < 2^23
-//   float(n) = as_float(0x4B400000 + n) - 1.5 * 2^23        for |n| < 2^22
-//   rint(t)  = low bits of as_int(t + 1.5 * 2^23)           for |t| < 2^22 (the add rounds to even)
-// MODE 2: every plane sum is below 2^22 in magnitude and P <= 3: with u = v0 + 2^7 v1,
-// w = (u >> 14) + v2, acc = w * 2^14 + (u mod 2^14); both parts are exact in fp32 (by the tricks)
-// and one fma rounds acc to nearest once.  MODE 1: below 2^24 (w by a conversion instruction).
-// MODE 3: the accumulator itself is below 2^31 in magnitude: 32-bit recombination, one int -> float
-// conversion (round to nearest even, like the 64-bit one).
-// MODE 0: 64-bit recombination plus the per-channel integer addend.
-// The run-time options enter as data (a relu floor of 0 or -inf, a sign mask), not as branches.
+// only re-quantised bytes are wanted.  Same arithmetic as dequant()/requant(), with as few issued
+// instructions per output as the definition allows (the output stage of a layer with few input
+// channels is bound by instruction issue, and every slot it takes is one the MMA-issuing thread of
+// the same scheduler does not get):
+//   W32: the accumulator itself is known to stay below 2^31 in magnitude (the sampler keeps the
+//        largest row sum of |W_k|, the caller vouches for the largest activation): the planes are
+//        recombined in 32 bits (wrap-around in the partial sums is harmless) and one conversion
+//        instruction rounds to nearest even, as the 64-bit conversion would.  Otherwise 64-bit
+//        recombination plus the per-channel integer addend, converted in two exact halves.
+//   y = fma(a, sc, bias); optional shortcut fma on a byte converted by the conversion unit.
+//   t = y * inv_step, clamped above in fp32; cvt.rni (round half to even, saturating) gives the
+//   integer; cvt.pack.sat packs two integers at a time into bytes, saturating to the byte's range.
+//   FAST_U8: unsigned codes whose lower bound is 0 (the ReLU, if any, folded into it): the byte
+//   saturation is the lower clamp.  Otherwise both clamps are applied in fp32 first.
 struct EpiConst {
-  float res_scale, inv_step, qmin_f, qmax_f;   // qmin_f already holds the relu (see the epilogue set-up)
-  uint32_t res_sign;
+  float res_scale, inv_step, lo_f, hi_f;   // lo_f already holds the relu (see the epilogue set-up)
+  uint32_t out_signed;
 };
 
-template <int P, int MODE, bool HAS_RES>
+// d = bytes (sat(b), sat(a), c.b0, c.b1), saturation to the unsigned / signed byte range
+__device__ __forceinline__ uint32_t pack_sat_u8(int a, int b, uint32_t c) {
+  uint32_t d;
+  asm("cvt.pack.sat.u8.s32.b32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(c));
+  return d;
+}
+__device__ __forceinline__ uint32_t pack_sat_s8(int a, int b, uint32_t c) {
+  uint32_t d;
+  asm("cvt.pack.sat.s8.s32.b32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(c));
+  return d;
+}
+
+// RES: 0 no shortcut, 1 unsigned shortcut bytes, 2 signed ones.
+template <int P, bool W32, int RES, bool FAST_U8>
 __device__ __forceinline__ uint4 chunk_math(const uint32_t (&v)[P][16], const uint4& r4, const float2* scb,
                                             const long long* corr, const EpiConst& c) {
   const uint32_t rw[4] = {r4.x, r4.y, r4.z, r4.w};
-  const float res_bias = 8388608.0f + (float)c.res_sign;   // undoes the magic constant and the sign flip
+  const float4* scb2 = reinterpret_cast<const float4*>(scb);   // two channels' (scale, bias) per load
   uint32_t qw[4];
 #pragma unroll
   for (int g = 0; g < 4; ++g) {
-    uint32_t q[4];
+    int q[4];
 #pragma unroll
     for (int e = 0; e < 4; ++e) {
       const int j = 4 * g + e;
       float af;
-      if (MODE == 3) {
-        // the whole sum fits 32 bits (wrap-around in the partial sums is harmless): one conversion
+      if (W32) {
         int acc = (int)v[0][j];
-        if (P > 1) acc += (int)v[1][j] << kDigitBits;
-        if (P > 2) acc += (int)v[2][j] << (2 * kDigitBits);
-        af = (float)acc;
-      } else if (MODE > 0) {
-        int u = (int)v[0][j];
-        if (P > 1) u += (int)v[1][j] << kDigitBits;
-        int w = u >> (2 * kDigitBits);
-        if (P > 2) w += (int)v[2][j];
-        const float lo_f = __uint_as_float(0x4B000000u | ((uint32_t)u & 0x3FFFu)) - 8388608.0f;
-        const float w_f = MODE == 2 ? __int_as_float(0x4B400000 + w) - 12582912.0f : (float)w;
-        af = __fmaf_rn(w_f, 16384.0f, lo_f);
+#pragma unroll
+        for (int pl = 1; pl < P; ++pl) acc += (int)v[pl][j] << (kDigitBits * pl);
+        af = __int2float_rn(acc);
       } else {
         long long acc = (long long)(int)v[0][j];
 #pragma unroll
@@ -375,17 +382,21 @@ __device__ __forceinline__ uint4 chunk_math(const uint32_t (&v)[P][16], const ui
         acc += corr[j];
         af = acc_to_float(acc);
       }
-      const float2 sb = scb[j];
-      float y = __fmaf_rn(af, sb.x, sb.y);
-      if (HAS_RES) {
-        const uint32_t rb = ((rw[g] >> (8 * e)) & 0xFFu) ^ c.res_sign;   // byte + 128 if signed
-        y = __fmaf_rn(__uint_as_float(0x4B000000u | rb) - res_bias, c.res_scale, y);
-      }
-      // clamp, then round half to even by adding 1.5 * 2^23: the low byte of the sum is the code
-      const float t = fminf(fmaxf(__fmul_rn(y, c.inv_step), c.qmin_f), c.qmax_f);
-      q[e] = __float_as_uint(t + 12582912.0f);
+      const float4 sb2 = scb2[j >> 1];
+      float y = (j & 1) ? __fmaf_rn(af, sb2.z, sb2.w) : __fmaf_rn(af, sb2.x, sb2.y);
+      if (RES == 1) y = __fmaf_rn((float)((rw[g] >> (8 * e)) & 0xFFu), c.res_scale, y);
+      if (RES == 2) y = __fmaf_rn((float)(int)(signed char)(rw[g] >> (8 * e)), c.res_scale, y);
+      float t = fminf(__fmul_rn(y, c.inv_step), c.hi_f);
+      if (!FAST_U8) t = fmaxf(t, c.lo_f);
+      q[e] = __float2int_rn(t);
     }
-    qw[g] = __byte_perm(__byte_perm(q[0], q[1], 0x0040), __byte_perm(q[2], q[3], 0x0040), 0x5410);
+    if (FAST_U8) {
+      qw[g] = pack_sat_u8(q[1], q[0], pack_sat_u8(q[3], q[2], 0u));
+    } else {
+      const uint32_t u = pack_sat_u8(q[1], q[0], pack_sat_u8(q[3], q[2], 0u));
+      const uint32_t sg = pack_sat_s8(q[1], q[0], pack_sat_s8(q[3], q[2], 0u));
+      qw[g] = c.out_signed ? sg : u;
+    }
   }
   return make_uint4(qw[0], qw[1], qw[2], qw[3]);
 }
@@ -444,23 +455,26 @@ __device__ __forceinline__ size_t out_offset(const ConvArgs& a, uint32_t ohow, u
   return ((size_t)n * a.O + o_base) * ohow + (m - n * ohow);
 }
 
-// The P plane sums of a 16-channel chunk, TMEM -> registers.  With three planes and 32-bit
-// recombination the first two planes are folded (v0 + 2^7 v1, what chunk_math computes first anyway)
-// before the third is fetched: 32 registers at the peak instead of 48, which is what the loop around
-// it was spilling.  The folded plane is left as a literal zero, so the arithmetic after it drops out.
-template <int P, int MODE>
+// The P plane sums of a 16-channel chunk, TMEM -> registers.  With 32-bit recombination the planes are
+// folded as they arrive (v0 + 2^7 v1 + ..., what chunk_math computes first anyway): 32 registers at the
+// peak instead of 16 P, which is what the loop around it was spilling.  The folded planes are left as
+// literal zeros, so the arithmetic after them drops out.
+template <int P, bool W32>
 __device__ __forceinline__ void load_chunk(uint32_t taddr, uint32_t (&v)[P][16]) {
-  if (P == 3 && MODE != 0) {
+  if (P >= 3 && W32) {
     tc_ld16(taddr, v[0]);
     tc_ld16(taddr + kTileN, v[1]);
     tc_wait_ld();
 #pragma unroll
-    for (int j = 0; j < 16; ++j) {
-      v[0][j] = (uint32_t)((int)v[0][j] + ((int)v[1][j] << kDigitBits));
-      v[1][j] = 0u;
+    for (int pl = 2; pl < P; ++pl) {
+#pragma unroll
+      for (int j = 0; j < 16; ++j) {
+        v[0][j] = (uint32_t)((int)v[0][j] + ((int)v[pl - 1][j] << (kDigitBits * (pl - 1))));
+        v[pl - 1][j] = 0u;
+      }
+      tc_ld16(taddr + pl * kTileN, v[pl]);
+      tc_wait_ld();
     }
-    tc_ld16(taddr + 2 * kTileN, v[2]);
-    tc_wait_ld();
   } else {
 #pragma unroll
     for (int pl = 0; pl < P; ++pl) tc_ld16(taddr + pl * kTileN, v[pl]);
@@ -468,13 +482,13 @@ __device__ __forceinline__ void load_chunk(uint32_t taddr, uint32_t (&v)[P][16])
   }
 }
 
-template <int P, int MODE, bool HAS_RES>
+template <int P, bool W32, int RES>
 __device__ __noinline__ void epilogue_chunk_q(uint32_t taddr, bool valid, uint8_t* q_dst, uint4 r4, bool vec16,
                                               bool both, const float2* scb, const long long* corr, EpiConst c) {
   uint32_t v[P][16];
-  load_chunk<P, MODE>(taddr, v);
+  load_chunk<P, W32>(taddr, v);
   if (!valid) return;
-  store_row16(q_dst, chunk_math<P, MODE, HAS_RES>(v, r4, scb, corr, c), vec16, both);
+  store_row16(q_dst, chunk_math<P, W32, RES, false>(v, r4, scb, corr, c), vec16, both);
 }
 
 // General output stage: any combination of outputs, layouts, ragged channel counts.
@@ -531,7 +545,7 @@ __device__ __forceinline__ bool uniform_epilogue(const TensorParams& p) {
   const ConvArgs& a = p.a;
   const bool q_only = a.q_out && !a.f32_out && !a.acc_out && (p.vec_ok || a.out_nchw) && a.inv_step > 0.0f;
   const uint32_t P0 = p.planes[a.uniform_log2k < (uint32_t)kMaxLevels ? a.uniform_log2k : 0u];
-  return !a.kmap && q_only && (P0 == 3u || P0 == 4u);
+  return !a.kmap && q_only && P0 >= 2u && P0 <= 4u;
 }
 
 // Linear output index (n * OH + oy) * OW + ox of row `row` of row tile `m_tile`, and whether the
@@ -555,6 +569,7 @@ __device__ __forceinline__ uint32_t tile_row_index(const TensorParams& p, uint32
 // with a memory clobber (barrier waits, TMEM loads) makes the compiler fetch such fields again: a
 // dozen dependent loads per tile in the output-stage loop before the copies were made.  (Plain mode.)
 struct RowMap {
+  static constexpr int kTag = 1;     // distinguishes the row maps in template tags
   uint32_t M, O, ohow, planar;
   __device__ __forceinline__ void init(const TensorParams& p) {
     M = p.M; O = p.a.O; ohow = p.a.OH * p.a.OW; planar = p.a.out_nchw;
@@ -573,6 +588,7 @@ struct RowMap {
 
 // Band mode: rows of a tile are padded-linear positions of one image (tile_row_index above).
 struct RowMapBand {
+  static constexpr int kTag = 0;
   uint32_t tpi, tpi_magic, Wp, Wp_magic, OH, OW, O, ohow, planar;
   __device__ __forceinline__ void init(const TensorParams& p) {
     tpi = p.tpi; tpi_magic = p.tpi_magic; Wp = p.Wp; Wp_magic = p.Wp_magic;
@@ -592,14 +608,31 @@ struct RowMapBand {
   }
 };
 
+// Whether the accumulators of level l stay below 2^31 in magnitude: (largest row sum of |W_k|, kept by the
+// sampler in units of 256, each weight rounded up) x (largest activation magnitude).  Not used when an
+// integer addend follows.  Warp-collective: the lanes share the scan over the rows.
+__device__ __forceinline__ bool fits_32_bits(const TensorParams& p, uint32_t l) {
+  if (!p.rowsum256 || p.corr[l] != nullptr) return false;
+  const uint32_t* sums = p.rowsum256 + (size_t)l * p.a.O;
+  uint32_t best = 0;
+  for (uint32_t o = threadIdx.x & 31u; o < p.a.O; o += 32u) best = max(best, sums[o]);
+  best = __reduce_max_sync(0xFFFFFFFFu, best);
+  // (a sum that wrapped or was marked unknown reads as huge either way)
+  return (unsigned long long)best * 256ull * (unsigned long long)p.amax < (1ull << 31) && best < (1u << 24);
+}
+
 // Epilogue loop of one warp for the common case: one draw count for the whole layer, only
 // re-quantised bytes wanted.  The warp owns 32 rows (its TMEM lane quarter) x 16 channels of
 // every tile.  Per tile: wait for the accumulator, pull the chunk into registers, hand the TMEM
 // buffer back at once (the MMA of the tile after next can start), then do the arithmetic and
-// the store.  Shortcut bytes are fetched one tile ahead.  Returns true if a wait timed out.
-template <int P, int MODE, bool HAS_RES>
+// the store.  Shortcut bytes are fetched one tile ahead.  RM maps the rows of a tile to output
+// locations (plain tiles or band mode).  Returns true if a wait timed out.
+template <int P, bool W32, int RES, bool FAST_U8, typename RM>
 __device__ __noinline__ bool epilogue_uniform(const TensorParams& p, SharedCtl* ctl, uint32_t tmem_base,
                                               uint32_t ew, uint32_t lane, EpiConst c) {
+  constexpr bool HAS_RES = RES != 0;
+  // every instance of this loop gets its own instance of the out-of-line planar helpers (see load_planar16)
+  constexpr int TAG = (((P * 2 + (W32 ? 1 : 0)) * 3 + RES) * 2 + (FAST_U8 ? 1 : 0)) * 2 + RM::kTag;
   const ConvArgs& a = p.a;
   const uint32_t quarter = ew & 3u, sub = ew >> 2;
   const uint32_t row = quarter * 32u + lane;
@@ -608,7 +641,7 @@ __device__ __noinline__ bool epilogue_uniform(const TensorParams& p, SharedCtl* 
   WaitCtl* abort = &ctl->wait;
   const uint8_t* const res_base = (const uint8_t*)a.residual;
   uint8_t* const q_base = (uint8_t*)a.q_out;
-  RowMap rm;
+  RM rm;
   rm.init(p);
   const float2* scb = ctl->scb[ew];
   const long long* corr = ctl->corr[ew];
@@ -623,7 +656,7 @@ __device__ __noinline__ bool epilogue_uniform(const TensorParams& p, SharedCtl* 
     const uint32_t m = rm.row_index(ti.m_tile, row, &ok_row), ob = ti.o_tile * kTileN + sub * 16u;
     if (ok_row && ob < rm.O) {
       const uint8_t* src = res_base + rm.offset(m, ob);
-      r_next = planar ? load_planar16<1>(src, ohow, rm.O - ob) : load_row16(src, vec16, ob + 16u <= rm.O);
+      r_next = planar ? load_planar16<TAG>(src, ohow, rm.O - ob) : load_row16(src, vec16, ob + 16u <= rm.O);
     }
   }
   while (ti.valid()) {
@@ -658,7 +691,7 @@ __device__ __noinline__ bool epilogue_uniform(const TensorParams& p, SharedCtl* 
       r_next = make_uint4(0, 0, 0, 0);
       if (ok_row && ob < rm.O) {
         const uint8_t* src = res_base + rm.offset(mn, ob);
-        r_next = planar ? load_planar16<1>(src, ohow, rm.O - ob) : load_row16(src, vec16, ob + 16u <= rm.O);
+        r_next = planar ? load_planar16<TAG>(src, ohow, rm.O - ob) : load_row16(src, vec16, ob + 16u <= rm.O);
       }
     }
     const uint32_t buf = pass & 1u, aph = (pass >> 1) & 1u;
@@ -668,16 +701,16 @@ __device__ __noinline__ bool epilogue_uniform(const TensorParams& p, SharedCtl* 
     uint32_t v[P][16];
     if (active) {
       const uint32_t taddr = tmem_base + buf * kTmemBufStride + ((quarter * 32u) << 16) + sub * 16u;
-      load_chunk<P, MODE>(taddr, v);
+      load_chunk<P, W32>(taddr, v);
     }
     // the chunk is in registers: give the accumulator buffer back before doing the arithmetic
     tc_fence_before();
     __syncwarp();
     if (lane == 0) mbar_arrive(smem_u32(&ctl->acc_empty[buf]));
     if (active && row_valid) {
-      const uint4 q16 = chunk_math<P, MODE, HAS_RES>(v, r_cur, scb, corr, c);
+      const uint4 q16 = chunk_math<P, W32, RES, FAST_U8>(v, r_cur, scb, corr, c);
       uint8_t* dst = q_base + rm.offset(m, o_base);
-      if (planar) store_planar16<1>(dst, ohow, rm.O - o_base, q16);
+      if (planar) store_planar16<TAG>(dst, ohow, rm.O - o_base, q16);
       else store_row16(dst, q16, vec16, o_base + 16u <= rm.O);
     }
     ++pass;
@@ -685,94 +718,28 @@ __device__ __noinline__ bool epilogue_uniform(const TensorParams& p, SharedCtl* 
   return false;
 }
 
-// The same loop for band mode (RowMapBand: band mode's index arithmetic wants five more fields; a loop
-// of its own keeps them out of the register budget of plain mode).
-template <int P, int MODE, bool HAS_RES>
-__device__ __noinline__ bool epilogue_uniform_band(const TensorParams& p, SharedCtl* ctl, uint32_t tmem_base,
-                                              uint32_t ew, uint32_t lane, EpiConst c) {
-  const ConvArgs& a = p.a;
-  const uint32_t quarter = ew & 3u, sub = ew >> 2;
-  const uint32_t row = quarter * 32u + lane;
-  const uint32_t l = a.uniform_log2k;
-  const bool use_corr = p.corr[l] != nullptr;
-  WaitCtl* abort = &ctl->wait;
-  const uint8_t* const res_base = (const uint8_t*)a.residual;
-  uint8_t* const q_base = (uint8_t*)a.q_out;
-  RowMapBand rm;
-  rm.init(p);
-  const float2* scb = ctl->scb[ew];
-  const long long* corr = ctl->corr[ew];
-  const bool vec16 = p.vec_ok == 2u, planar = rm.planar != 0u;
-  const uint32_t ohow = rm.ohow;
-  TileIter ti;
-  ti.init(p);
-  uint32_t pass = 0, cur_o_tile = 0xFFFFFFFFu;
-  uint4 r_next = make_uint4(0, 0, 0, 0);
-  if (HAS_RES && ti.valid()) {
-    bool ok_row;
-    const uint32_t m = rm.row_index(ti.m_tile, row, &ok_row), ob = ti.o_tile * kTileN + sub * 16u;
-    if (ok_row && ob < rm.O) {
-      const uint8_t* src = res_base + rm.offset(m, ob);
-      r_next = planar ? load_planar16<0>(src, ohow, rm.O - ob) : load_row16(src, vec16, ob + 16u <= rm.O);
-    }
+// Run-time options of the uniform output stage -> template instance.
+template <int P, bool W32, int RES>
+__device__ __forceinline__ bool uniform_dispatch_tail(const TensorParams& p, SharedCtl* ctl, uint32_t tmem_base,
+                                                      uint32_t ew, uint32_t lane, const EpiConst& c, bool fast_u8) {
+  if (p.band)
+    return fast_u8 ? epilogue_uniform<P, W32, RES, true, RowMapBand>(p, ctl, tmem_base, ew, lane, c)
+                   : epilogue_uniform<P, W32, RES, false, RowMapBand>(p, ctl, tmem_base, ew, lane, c);
+  return fast_u8 ? epilogue_uniform<P, W32, RES, true, RowMap>(p, ctl, tmem_base, ew, lane, c)
+                 : epilogue_uniform<P, W32, RES, false, RowMap>(p, ctl, tmem_base, ew, lane, c);
+}
+template <int P>
+__device__ __forceinline__ bool uniform_dispatch(const TensorParams& p, SharedCtl* ctl, uint32_t tmem_base,
+                                                 uint32_t ew, uint32_t lane, const EpiConst& c, bool fast_u8,
+                                                 bool w32, uint32_t res) {
+  if (w32) {
+    if (res == 0u) return uniform_dispatch_tail<P, true, 0>(p, ctl, tmem_base, ew, lane, c, fast_u8);
+    if (res == 1u) return uniform_dispatch_tail<P, true, 1>(p, ctl, tmem_base, ew, lane, c, fast_u8);
+    return uniform_dispatch_tail<P, true, 2>(p, ctl, tmem_base, ew, lane, c, fast_u8);
   }
-  while (ti.valid()) {
-    bool row_valid;
-    const uint32_t m = rm.row_index(ti.m_tile, row, &row_valid);
-    const uint32_t o_tile = ti.o_tile;
-    const uint32_t o_base = o_tile * kTileN + sub * 16u;
-    const bool active = o_base < rm.O;          // warp-uniform
-    ti.next();
-    if (o_tile != cur_o_tile) {
-      // per-channel constants of this channel tile: the warp keeps its own copy of its 16 channels
-      __syncwarp();
-      if (lane < 16u) {
-        const uint32_t o = o_base + lane;
-        float2 sb = make_float2(0.f, 0.f);
-        long long cr = 0;
-        if (o < a.O) {
-          sb.x = ldexpf(a.scale[o], a.e_base[o] - (int)l);
-          sb.y = a.bias[o];
-          if (use_corr) cr = p.corr[l][o];
-        }
-        ctl->scb[ew][lane] = sb;
-        ctl->corr[ew][lane] = cr;
-      }
-      cur_o_tile = o_tile;
-      __syncwarp();
-    }
-    const uint4 r_cur = r_next;
-    if (HAS_RES && ti.valid()) {
-      bool ok_row;
-      const uint32_t mn = rm.row_index(ti.m_tile, row, &ok_row), ob = ti.o_tile * kTileN + sub * 16u;
-      r_next = make_uint4(0, 0, 0, 0);
-      if (ok_row && ob < rm.O) {
-        const uint8_t* src = res_base + rm.offset(mn, ob);
-        r_next = planar ? load_planar16<0>(src, ohow, rm.O - ob) : load_row16(src, vec16, ob + 16u <= rm.O);
-      }
-    }
-    const uint32_t buf = pass & 1u, aph = (pass >> 1) & 1u;
-    const bool ok = mbar_wait(smem_u32(&ctl->acc_full[buf]), aph, abort, 32);
-    if (__any_sync(0xFFFFFFFFu, !ok)) return true;
-    tc_fence_after();
-    uint32_t v[P][16];
-    if (active) {
-      const uint32_t taddr = tmem_base + buf * kTmemBufStride + ((quarter * 32u) << 16) + sub * 16u;
-      load_chunk<P, MODE>(taddr, v);
-    }
-    // the chunk is in registers: give the accumulator buffer back before doing the arithmetic
-    tc_fence_before();
-    __syncwarp();
-    if (lane == 0) mbar_arrive(smem_u32(&ctl->acc_empty[buf]));
-    if (active && row_valid) {
-      const uint4 q16 = chunk_math<P, MODE, HAS_RES>(v, r_cur, scb, corr, c);
-      uint8_t* dst = q_base + rm.offset(m, o_base);
-      if (planar) store_planar16<0>(dst, ohow, rm.O - o_base, q16);
-      else store_row16(dst, q16, vec16, o_base + 16u <= rm.O);
-    }
-    ++pass;
-  }
-  return false;
+  if (res == 0u) return uniform_dispatch_tail<P, false, 0>(p, ctl, tmem_base, ew, lane, c, fast_u8);
+  if (res == 1u) return uniform_dispatch_tail<P, false, 1>(p, ctl, tmem_base, ew, lane, c, fast_u8);
+  return uniform_dispatch_tail<P, false, 2>(p, ctl, tmem_base, ew, lane, c, fast_u8);
 }
 
 // The MMA issuing role, one thread of warp kMmaWarp0 (mine = 0) and one of kMmaWarp1 (mine = 1).
@@ -1041,9 +1008,12 @@ psb_mma_kernel(const __grid_constant__ TmapSet maps, const __grid_constant__ Ten
     // With inv_step > 0 (a condition of the fast paths) max(y, 0) * inv_step == max(y * inv_step, 0):
     // the relu is folded into the lower clamp bound.
     ec.inv_step = a.inv_step;
-    ec.qmin_f = (a.relu && a.qmin < 0) ? 0.0f : (float)a.qmin;
-    ec.qmax_f = (float)a.qmax;
-    ec.res_sign = a.residual_dtype == PSB_DT_S8 ? 0x80u : 0u;
+    ec.lo_f = (a.relu && a.qmin < 0) ? 0.0f : (float)a.qmin;
+    ec.hi_f = (float)a.qmax;
+    ec.out_signed = a.out_dtype == PSB_DT_S8 ? 1u : 0u;
+    // unsigned codes from 0 up: the byte saturation of the packing instruction is the lower clamp
+    const bool fast_u8 = a.out_dtype == PSB_DT_U8 && a.qmin == 0;
+    const uint32_t res_kind = !a.residual ? 0u : (a.residual_dtype == PSB_DT_S8 ? 2u : 1u);
     const uint32_t P0 = p.planes[a.uniform_log2k < (uint32_t)kMaxLevels ? a.uniform_log2k : 0u];
     if (p.resident && lane == 0) {
       // the digit planes of this CTA's channel tile, all K blocks, once: the epilogue warps have
@@ -1059,23 +1029,19 @@ psb_mma_kernel(const __grid_constant__ TmapSet maps, const __grid_constant__ Ten
       }
     }
     if (uniform_epilogue(p)) {
-      const uint32_t mode = (p.corr[a.uniform_log2k] != nullptr || P0 == 4u) ? 0u : p.narrow;
-#define PSB_UNI(PV, MV, RV)                                                                   \
-  failed = p.band ? epilogue_uniform_band<PV, MV, RV>(p, ctl, tmem_base, ew, lane, ec)        \
-                  : epilogue_uniform<PV, MV, RV>(p, ctl, tmem_base, ew, lane, ec)
-      if (a.residual) {
-        if (P0 == 4u) PSB_UNI(4, 0, true); else if (mode == 3u) PSB_UNI(3, 3, true); else if (mode == 2u) PSB_UNI(3, 2, true);
-        else if (mode == 1u) PSB_UNI(3, 1, true); else PSB_UNI(3, 0, true);
-      } else {
-        if (P0 == 4u) PSB_UNI(4, 0, false); else if (mode == 3u) PSB_UNI(3, 3, false); else if (mode == 2u) PSB_UNI(3, 2, false);
-        else if (mode == 1u) PSB_UNI(3, 1, false); else PSB_UNI(3, 0, false);
-      }
-#undef PSB_UNI
+      const bool w32 = fits_32_bits(p, a.uniform_log2k);
+      if (P0 == 4u) failed = uniform_dispatch<4>(p, ctl, tmem_base, ew, lane, ec, fast_u8, w32, res_kind);
+      else if (P0 == 3u) failed = uniform_dispatch<3>(p, ctl, tmem_base, ew, lane, ec, fast_u8, w32, res_kind);
+      else failed = uniform_dispatch<2>(p, ctl, tmem_base, ew, lane, ec, fast_u8, w32, res_kind);
     } else {
       // general loop: per-location draw counts, any outputs and layouts, ragged channel counts
       const float2* scb = ctl->scb[ew];
       const long long* corr = ctl->corr[ew];
       uint32_t pass = 0, cur_key = 0xFFFFFFFFu;
+      uint32_t w32_levels = 0;      // levels whose accumulators are known to fit 32 bits
+      if (q_only)
+        for (uint32_t l = 0; l < (uint32_t)kMaxLevels; ++l)
+          if (((a.level_mask >> l) & 1u) && fits_32_bits(p, l)) w32_levels |= 1u << l;
       TileIter ti;
       for (ti.init(p); !failed && ti.valid(); ti.next()) {
         const uint32_t m0 = ti.m_tile * kTileM, o_tile = ti.o_tile;
@@ -1125,15 +1091,17 @@ psb_mma_kernel(const __grid_constant__ TmapSet maps, const __grid_constant__ Ten
           if (o_base < a.O) {
             if (fast) {
               uint8_t* q_dst = (uint8_t*)a.q_out + oidx;
-              const uint32_t mode = (use_corr || P > 3u) ? 0u : (p.narrow > 2u ? 2u : p.narrow);
-#define PSB_EPI(PV, MV, RV) epilogue_chunk_q<PV, MV, RV>(taddr, valid, q_dst, r4, vec16, both, scb, corr, ec)
-#define PSB_EPI_P(MV, RV) do { if (P == 3) PSB_EPI(3, MV, RV); else if (P == 2) PSB_EPI(2, MV, RV); else PSB_EPI(1, MV, RV); } while (0)
-              if (a.residual) {
-                if (mode == 2) PSB_EPI_P(2, true); else if (mode == 1) PSB_EPI_P(1, true);
-                else if (P == 4) PSB_EPI(4, 0, true); else PSB_EPI_P(0, true);
+              const bool w32 = ((w32_levels >> l) & 1u) != 0u;
+#define PSB_EPI(PV, WV, RV) epilogue_chunk_q<PV, WV, RV>(taddr, valid, q_dst, r4, vec16, both, scb, corr, ec)
+#define PSB_EPI_P(WV, RV)                                                                          \
+  do {                                                                                             \
+    if (P == 4) PSB_EPI(4, WV, RV); else if (P == 3) PSB_EPI(3, WV, RV);                           \
+    else if (P == 2) PSB_EPI(2, WV, RV); else PSB_EPI(1, WV, RV);                                  \
+  } while (0)
+              if (w32) {
+                if (res_kind == 0u) PSB_EPI_P(true, 0); else if (res_kind == 1u) PSB_EPI_P(true, 1); else PSB_EPI_P(true, 2);
               } else {
-                if (mode == 2) PSB_EPI_P(2, false); else if (mode == 1) PSB_EPI_P(1, false);
-                else if (P == 4) PSB_EPI(4, 0, false); else PSB_EPI_P(0, false);
+                if (res_kind == 0u) PSB_EPI_P(false, 0); else if (res_kind == 1u) PSB_EPI_P(false, 1); else PSB_EPI_P(false, 2);
               }
 #undef PSB_EPI_P
 #undef PSB_EPI
@@ -1293,7 +1261,7 @@ psb_status launch_tensor(psb_ctx* ctx, const psb_weights* wt, const ConvArgs& a,
       p.resident_bytes = need;
       // band mode: see TensorParams; needs the specialised output stage (codes only)
       const bool codes_only = a.q_out && !a.f32_out && !a.acc_out && (p.vec_ok || a.out_nchw) && a.inv_step > 0.0f &&
-                              (P == 3u || P == 4u);
+                              P >= 2u && P <= 4u;
       const uint32_t Wp = a.W + 2u * a.pad;
       const uint32_t span = kTileM + (a.KH - 1u) * Wp + (a.KW - 1u);   // band pixels a tile touches
       const uint32_t rows = (Wp - 1u + span + Wp - 1u) / Wp;           // whatever the tile's offset in its first row
@@ -1344,22 +1312,8 @@ psb_status launch_tensor(psb_ctx* ctx, const psb_weights* wt, const ConvArgs& a,
   const size_t smem_bytes = (p.band ? (size_t)stages * p.band_bytes : (size_t)stages * group * sub_bytes) +
                             p.resident_bytes + ctl_bytes;
   for (int l = 0; l < kMaxLevels; ++l) p.corr[l] = add_corr128 ? wt->level[l].corr128 : nullptr;
-  // every plane sum is bounded by 127 * (largest activation magnitude) * d
-  const uint64_t plane_bound = 127ull * amax * (uint64_t)wt->d;
-  p.narrow = pmax > 3 ? 0u : (plane_bound <= 4100000ull ? 2u : (plane_bound <= 16500000ull ? 1u : 0u));
-  // every |W_k| is at most 2k * 2^(2^exp_bits - 1): if the whole accumulator stays below 2^31 the
-  // output stage recombines in 32 bits
-  {
-    uint32_t lmax = a.uniform_log2k;
-    if (a.kmap)
-      for (uint32_t l = 0; l < (uint32_t)kMaxLevels; ++l)
-        if ((a.level_mask >> l) & 1u) lmax = l;
-    const uint32_t span = (1u << wt->cfg.exp_bits) - 1u;
-    if (span + lmax + 1u < 40u) {
-      const unsigned __int128 acc_bound = (unsigned __int128)amax * wt->d * ((unsigned long long)1 << (span + lmax + 1u));
-      if (p.narrow == 2u && acc_bound < ((unsigned __int128)1 << 31)) p.narrow = 3u;
-    }
-  }
+  p.rowsum256 = wt->rowsum256;
+  p.amax = amax;
   const CUtensorMapSwizzle swz = swizzle_for(bk);
   EncodeTiledFn enc_tiled = (EncodeTiledFn)ctx->encode_tiled;
   EncodeIm2colFn enc_im2col = (EncodeIm2colFn)ctx->encode_im2col;

@@ -650,3 +650,42 @@ def test_activation_beyond_in_max_is_reported(psb, ctx):
     assert ctx.device_status() == psb.PSB_ERR_RANGE
     ctx.set_sample_map(None, 0)
     wt3.free()
+
+
+# (N, C, H, W, O, K, pad, layout, shortcut dtype or None)
+@pytest.mark.parametrize("case", [(2, 64, 13, 12, 64, 1, 0, 1, None), (2, 64, 14, 13, 80, 3, 1, 1, np.uint8),
+                                  (3, 128, 9, 11, 64, 3, 1, 0, np.uint8), (2, 256, 9, 9, 128, 1, 0, 1, np.int8)])
+@pytest.mark.parametrize("signed_out", [False, True])
+def test_tensor_path_codes_only_two_planes_and_signed_codes(psb, ctx, oracle, case, signed_out):
+    """A window of eight octaves (exp_bits = 3) needs two digit planes at k = 8; the uniform codes-only output
+    stage for it, plain tiles and band mode, unsigned codes from 0 and signed codes with both clamps."""
+    N, C, H, W, O, K, pad, layout, res_dt = case
+    rng = np.random.default_rng(abs(hash((case[:8], signed_out))) % 2 ** 31)
+    w, x, scale, bias = _layer_inputs(rng, N, C, H, W, O, K, K, 1, layout)
+    OH, OW = H + 2 * pad - K + 1, W + 2 * pad - K + 1
+    res = None
+    if res_dt is not None:
+        lo, hi = (0, 16) if res_dt == np.uint8 else (-15, 16)
+        res = rng.integers(lo, hi, size=(N, O, OH, OW) if layout == 0 else (N, OH, OW, O)).astype(res_dt)
+    kw = dict(relu=False, qmin=-15, qmax=15, out_dtype=1) if signed_out else dict(relu=True, qmin=0, qmax=15)
+    g = _both(psb, ctx, oracle, w, x, layout, 1, 1, pad, [3], scale, bias, inv_step=0.5, residual=res,
+              res_scale=0.3 if res is not None else 0.0, exp_bits=3, in_max=15, path=psb.PSB_PATH_TENSOR, want=("q",), **kw)
+    assert g["path"] == psb.PSB_PATH_TENSOR
+
+
+def test_tensor_path_codes_only_wide_accumulators(psb, ctx, oracle):
+    """Large activations against a filter with large row sums: the 32-bit recombination of the output stage
+    must not be chosen (the accumulators exceed 2^31), codes still exact."""
+    rng = np.random.default_rng(99)
+    N, C, H, W, O = 2, 512, 6, 6, 64
+    w = rng.normal(0, 1.0, size=(O, C, 3, 3)).astype(np.float32)
+    w = np.abs(w) * 0.9 + 0.5                       # same sign, all within one octave of the largest
+    x = rng.integers(100, 128, size=(N, H, W, C)).astype(np.uint8)
+    scale = np.ones(O, dtype=np.float32)
+    bias = rng.normal(0, 0.5, O).astype(np.float32)
+    g = _both(psb, ctx, oracle, w, x, 1, 1, 1, 1, [3], scale, bias, inv_step=0.008, qmax=255, in_max=127,
+              path=psb.PSB_PATH_TENSOR)
+    assert np.abs(g["acc"]).max() > 2 ** 31
+    g = _both(psb, ctx, oracle, w, x, 1, 1, 1, 1, [3], scale, bias, inv_step=0.008, qmax=255, in_max=127,
+              path=psb.PSB_PATH_TENSOR, want=("q",))
+    assert g["q"].max() > 0

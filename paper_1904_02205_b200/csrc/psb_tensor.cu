@@ -47,6 +47,8 @@ constexpr uint32_t kTmemCols = 512;
 constexpr uint32_t kTmemBufStride = 256;
 constexpr int kMaxStages = 12;
 constexpr uint32_t kResidentMaxBytes = 112 * 1024;          // digit planes kept in shared memory
+constexpr int kTapBatch = 6;                                // descriptor offsets fetched ahead of their MMAs
+constexpr int kMaxBandMmas = 128;                           // MMAs per tile (taps x K steps) that band mode handles
 
 struct TmapSet {
   CUtensorMap a;     // activations; the digit planes need none: their tiles are contiguous
@@ -133,6 +135,8 @@ struct WaitCtl {
   volatile unsigned long long limit;
 };
 
+constexpr uint32_t kNoSleep = 0xFFFFFFFFu;   // backoff value of a wait that is about to end: poll without sleeping
+
 // Bounded wait.  Returns false after wc->limit SM clocks without completion, or as soon
 // as another thread of the CTA has given up.  (The SM cycle counter is cheap to read.)
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, WaitCtl* wc,
@@ -144,7 +148,8 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, WaitCtl
     // a thread that has to wait long should not eat the issue slots of the warps doing the
     // arithmetic: poll a few times at full speed, then sleep between polls
     ++spins;
-    if (backoff_ns || spins > 4u) __nanosleep(backoff_ns ? backoff_ns : (spins > 32u ? 256u : 64u));
+    if (backoff_ns != kNoSleep && (backoff_ns || spins > 4u))
+      __nanosleep(backoff_ns ? backoff_ns : (spins > 32u ? 256u : 64u));
     if ((spins & 15u) == 0u) {
       if (wc->abort) return false;
       if ((unsigned long long)(clock64() - t0) > wc->limit) return false;
@@ -219,6 +224,29 @@ __device__ __forceinline__ void tc_mma_i8(uint32_t d_tmem, uint64_t desc_a, uint
       : "memory");
 }
 
+// The same instruction for the issue loops: accumulate always, descriptors given as (low word, high word),
+// no memory clobber (the loop's own loads of descriptor offsets may then be scheduled ahead of it; the
+// operands are written by the copy engine and ordered by the barrier waits, which keep their clobbers).
+template <bool ACC>
+__device__ __forceinline__ void tc_mma_i8_lohi(uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo, uint32_t desc_hi,
+                                               uint32_t idesc) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\t"
+      "setp.ne.b32 p, %5, 0;\n\t"
+      "mov.b64 da, {%1, %3};\n\t"
+      "mov.b64 db, {%2, %3};\n\t"
+      "tcgen05.mma.cta_group::1.kind::i8 [%0], da, db, %4, p;\n\t}"
+      ::"r"(d_tmem), "r"(a_lo), "r"(b_lo), "r"(desc_hi), "r"(idesc), "r"(ACC ? 1u : 0u));
+}
+__device__ __forceinline__ void tc_mma_i8_acc(uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo, uint32_t desc_hi,
+                                              uint32_t idesc) {
+  tc_mma_i8_lohi<true>(d_tmem, a_lo, b_lo, desc_hi, idesc);
+}
+__device__ __forceinline__ void tc_mma_i8_zero(uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo, uint32_t desc_hi,
+                                               uint32_t idesc) {
+  tc_mma_i8_lohi<false>(d_tmem, a_lo, b_lo, desc_hi, idesc);
+}
+
 __device__ __forceinline__ void tc_ld16(uint32_t taddr, uint32_t (&v)[16]) {
   asm volatile(
       "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
@@ -244,6 +272,15 @@ __device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t bk) {
   d |= (uint64_t)1 << 46;                       // descriptor version of this architecture
   d |= layout << 61;
   return d;
+}
+
+// The two words of that descriptor.  Only the low word depends on the address (bits 0..13 = address / 16;
+// shared memory ends below 2^18, so adding a byte offset / 16 to the low word moves the start address and
+// touches nothing else).
+__device__ __forceinline__ uint32_t smem_desc_lo(uint32_t addr) { return ((addr & 0x3FFFFu) >> 4) | (1u << 16); }
+__device__ __forceinline__ uint32_t smem_desc_hi(uint32_t bk) {
+  const uint32_t layout = bk == 128 ? 2u : (bk == 64 ? 4u : 6u);
+  return ((8u * bk) >> 4) | (1u << 14) | (layout << 29);
 }
 
 // Levels (log2 k) present among the 128 rows of a tile, as a bit mask: one byte per row tile,
@@ -317,6 +354,9 @@ struct SharedCtl {
   unsigned long long acc_empty[2];
   unsigned long long planes_full[kPlaneBars];
   unsigned long long started[2];        // per accumulator buffer: the zeroing MMA of the pass has been issued
+  unsigned long long pass_issued;       // all but the last K block of a pass have been issued (phase = pass number)
+  uint2 tap_tab[2][kMaxBandMmas];       // band mode, per issuing thread: (activation, plane) descriptor offsets of the
+                                        // tile's MMAs, in units of 16 bytes
   uint32_t tmem_base;
   WaitCtl wait;
   alignas(16) float2 scb[kEpilogueWarps][16];   // per epilogue warp: (scale * 2^(e_base - log2 k), bias), read two
@@ -753,6 +793,12 @@ __device__ __forceinline__ bool uniform_dispatch(const TensorParams& p, SharedCt
 // a slot follows its own previous use of that slot.  Kept out of line and fed from local copies of
 // the parameters so that its loop state lives in registers: the pipe idles for every clock this
 // thread spends between two MMAs beyond what the other thread covers.  Returns true on a timeout.
+//
+// Passes of a single stage are issued in their order: the first MMA of a pass follows the last but one K block
+// of the pass before it (`pass_issued`; the waits for the stage and the accumulator buffer are done by then).  Without
+// the rule both threads issue at once whenever both have a stage ready, the MMAs of two tiles interleave in
+// the pipe, both tiles complete late and together, and the pipe then idles until the output stage has
+// emptied an accumulator buffer.
 template <int BK>
 __device__ __noinline__ bool mma_role(const TensorParams& p, SharedCtl* ctl, uint32_t tmem_base, uint32_t ring_addr,
                                       uint32_t planes_addr, uint32_t stage_bytes, uint32_t sub_bytes,
@@ -760,11 +806,15 @@ __device__ __noinline__ bool mma_role(const TensorParams& p, SharedCtl* ctl, uin
   WaitCtl* abort = &ctl->wait;
   const uint32_t group = p.group, stages = p.stages, resident = p.resident, stage_bytes_a = p.stage_bytes_a;
   const uint32_t level_mask = p.a.level_mask;
-  const uint32_t band = p.band, row_bytes = p.Wp * p.a.C, KH = p.a.KH, KW = p.a.KW;
   const uint32_t n_groups = (k_iters + group - 1) / group;
   const uint32_t full0 = smem_u32(&ctl->full[0]), empty0 = smem_u32(&ctl->empty[0]);
   const uint32_t acc_full0 = smem_u32(&ctl->acc_full[0]), acc_empty0 = smem_u32(&ctl->acc_empty[0]);
   const uint32_t started0 = smem_u32(&ctl->started[0]);
+  const uint32_t pass_issued = smem_u32(&ctl->pass_issued);
+  // (passes of several stages already have both threads at work on the same pass in turns; there the rule
+  // only took the overlap at the pass boundaries away and cost a few per cent)
+  const bool ordered = n_groups == 1u;
+  const uint32_t desc_hi = smem_desc_hi(BK);
   // resident digit planes: K blocks below planes_upto are known to have landed
   const uint32_t plane_part = (k_iters + kPlaneBars - 1) / kPlaneBars;
   uint32_t planes_ready = 0, planes_upto = resident ? 0u : 0xFFFFFFFFu;
@@ -782,11 +832,6 @@ __device__ __noinline__ bool mma_role(const TensorParams& p, SharedCtl* ctl, uin
       const uint32_t d_tmem = tmem_base + buf * kTmemBufStride;
       const uint32_t blk = P * kTileN * BK;
       bool joined = (use & 1u) == mine;
-      uint32_t band_off = 0;     // band mode: byte offset of the tile's first position in its band
-      if (band && joined) {
-        const uint32_t t0 = (ti.m_tile - __umulhi(ti.m_tile, p.tpi_magic) * p.tpi) * kTileM;
-        band_off = (t0 - __umulhi(t0, p.Wp_magic) * p.Wp) * (uint32_t)BK;
-      }
       if (joined) {
         if (!mbar_wait(acc_empty0 + 8u * buf, aph ^ 1u, abort)) return true;
         tc_fence_after();
@@ -805,28 +850,25 @@ __device__ __noinline__ bool mma_role(const TensorParams& p, SharedCtl* ctl, uin
             ++planes_ready;
             planes_upto = planes_ready == (uint32_t)kPlaneBars ? 0xFFFFFFFFu : planes_upto + plane_part;
           }
+          if (ordered && pass != 0u) {
+            if (!mbar_wait(pass_issued, (pass - 1u) & 1u, abort, kNoSleep)) return true;
+          }
           tc_fence_after();
-          uint32_t a_addr = ring_addr + s * stage_bytes, b_blk = b_res;
-          if (band) {
-            // every tap reads the one band of the stage, from a start moved by kh rows and kw pixels
-            a_addr += band_off;
-            uint32_t first = 0;
-            for (uint32_t kh = 0; kh < KH; ++kh, a_addr += row_bytes)
-              for (uint32_t kw = 0; kw < KW; ++kw, b_blk += blk) {
+          // K blocks of the stage: activation tiles sub_bytes apart, planes beside them or resident; only the
+          // low words of the descriptors move (by bytes / 16)
+          uint32_t a_lo = smem_desc_lo(ring_addr + s * stage_bytes);
+          uint32_t b_lo = resident ? smem_desc_lo(b_res) : a_lo + (stage_bytes_a >> 4);
+          const uint32_t a_step = sub_bytes >> 4, b_step = resident ? blk >> 4 : sub_bytes >> 4;
+          for (uint32_t j = 0; j < cnt; ++j, a_lo += a_step, b_lo += b_step) {
+            // the pass after this one may start under this pass's last K block
+            if (ordered && j + 1u == cnt) mbar_arrive(pass_issued);
+            if (it == 0 && j == 0) {
+              tc_mma_i8_zero(d_tmem, a_lo, b_lo, desc_hi, idesc);
 #pragma unroll
-                for (int ks = 0; ks < BK / 32; ++ks) {
-                  tc_mma_i8(d_tmem, smem_desc(a_addr + kw * BK + ks * 32, BK), smem_desc(b_blk + ks * 32, BK), idesc,
-                            first);
-                  first = 1u;
-                }
-              }
-          } else {
-            for (uint32_t j = 0; j < cnt; ++j, a_addr += sub_bytes, b_blk += blk) {
-              const uint32_t b_addr = resident ? b_blk : a_addr + stage_bytes_a;
+              for (int ks = 1; ks < BK / 32; ++ks) tc_mma_i8_acc(d_tmem, a_lo + 2 * ks, b_lo + 2 * ks, desc_hi, idesc);
+            } else {
 #pragma unroll
-              for (int ks = 0; ks < BK / 32; ++ks)
-                tc_mma_i8(d_tmem, smem_desc(a_addr + ks * 32, BK), smem_desc(b_addr + ks * 32, BK), idesc,
-                          (it | j | ks) != 0 ? 1u : 0u);
+              for (int ks = 0; ks < BK / 32; ++ks) tc_mma_i8_acc(d_tmem, a_lo + 2 * ks, b_lo + 2 * ks, desc_hi, idesc);
             }
           }
           if (it == 0 && n_groups > 1u) {
@@ -843,6 +885,80 @@ __device__ __noinline__ bool mma_role(const TensorParams& p, SharedCtl* ctl, uin
       }
       ++pass;
     }
+  }
+  return false;
+}
+
+// The same role in band mode, where a ring stage holds the band of a whole tile: both threads work on every
+// tile, thread 0 on the first half of its MMAs (taps x K steps), thread 1 on the second half, both into the
+// one accumulator (the order of integer additions is immaterial).  One thread alone needs about 115 clocks
+// per MMA where the pipe needs 96, and a hand-over between tiles costs a few hundred more; two threads on
+// the same tile keep the pipe fed and the tiles in order.  Thread 0 issues the zeroing MMA first (`started`);
+// both commit to the stage's and the accumulator's barriers (count 2 in this mode).  The descriptor offsets of
+// a thread's MMAs are computed once (a table in shared memory, read a few entries ahead of the MMAs); the
+// issue loop then spends two additions per MMA.
+template <int BK>
+__device__ __noinline__ bool mma_role_band(const TensorParams& p, SharedCtl* ctl, uint32_t tmem_base,
+                                           uint32_t ring_addr, uint32_t planes_addr, uint32_t stage_bytes,
+                                           uint32_t mine) {
+  WaitCtl* abort = &ctl->wait;
+  const uint32_t stages = p.stages, row_bytes = p.Wp * p.a.C, KH = p.a.KH, KW = p.a.KW;
+  const uint32_t full0 = smem_u32(&ctl->full[0]), empty0 = smem_u32(&ctl->empty[0]);
+  const uint32_t acc_full0 = smem_u32(&ctl->acc_full[0]), acc_empty0 = smem_u32(&ctl->acc_empty[0]);
+  const uint32_t started0 = smem_u32(&ctl->started[0]);
+  const uint32_t desc_hi = smem_desc_hi(BK);
+  const uint32_t P = p.planes[p.a.uniform_log2k];
+  const uint32_t idesc = (2u << 4) | (1u << 7) | (1u << 10) | (((P * kTileN) >> 3) << 17) | ((kTileM >> 4) << 24);
+  const uint32_t blk = P * kTileN * BK;
+  constexpr uint32_t kSteps = BK / 32;
+  const uint32_t n_mmas = KH * KW * kSteps, half = (n_mmas + 1u) / 2u;
+  const uint32_t j_begin = mine ? half : 0u, cnt = mine ? n_mmas - half : half;
+  uint2* const tab = ctl->tap_tab[mine];
+  for (uint32_t i = 0; i < (cnt + kTapBatch - 1) / kTapBatch * kTapBatch; ++i) {
+    const uint32_t j = j_begin + i, tap = j / kSteps, ks = j - tap * kSteps, kh = tap / KW, kw = tap - kh * KW;
+    tab[i] = i < cnt ? make_uint2((kh * row_bytes + kw * (uint32_t)BK + ks * 32u) >> 4, (tap * blk + ks * 32u) >> 4)
+                     : make_uint2(0u, 0u);
+  }
+  // resident digit planes arrive in kPlaneBars parts of `plane_part` K blocks (= taps): this thread needs the
+  // parts up to the one that holds its last tap
+  const uint32_t k_iters = KH * KW, plane_part = (k_iters + kPlaneBars - 1) / kPlaneBars;
+  const uint32_t parts_needed = min((uint32_t)kPlaneBars, (j_begin + cnt - 1u) / kSteps / plane_part + 1u);
+  const uint32_t planes_lo = smem_desc_lo(planes_addr);
+  uint32_t s = 0, ph = 0, pass = 0;
+  TileIter ti;
+  for (ti.init(p); ti.valid(); ti.next(), ++pass) {
+    const uint32_t buf = pass & 1u, aph = (pass >> 1) & 1u;
+    const uint32_t d_tmem = tmem_base + buf * kTmemBufStride;
+    // byte offset of the tile's first position in its band
+    const uint32_t t0 = (ti.m_tile - __umulhi(ti.m_tile, p.tpi_magic) * p.tpi) * kTileM;
+    const uint32_t band_off = (t0 - __umulhi(t0, p.Wp_magic) * p.Wp) * (uint32_t)BK;
+    if (!mbar_wait(acc_empty0 + 8u * buf, aph ^ 1u, abort)) return true;
+    if (mine && !mbar_wait(started0 + 8u * buf, aph, abort, kNoSleep)) return true;
+    if (!mbar_wait(full0 + 8u * s, ph, abort)) return true;
+    if (pass == 0u)
+      for (uint32_t b = 0; b < parts_needed; ++b)
+        if (!mbar_wait(smem_u32(&ctl->planes_full[b]), 0u, abort)) return true;
+    tc_fence_after();
+    const uint32_t a0 = smem_desc_lo(ring_addr + s * stage_bytes + band_off);
+    for (uint32_t i0 = 0; i0 < cnt; i0 += kTapBatch) {
+      uint2 t[kTapBatch];
+#pragma unroll
+      for (int j = 0; j < kTapBatch; ++j) t[j] = tab[i0 + j];
+#pragma unroll
+      for (int j = 0; j < kTapBatch; ++j) {
+        if (i0 + (uint32_t)j >= cnt) break;
+        if (j == 0 && i0 == 0u && !mine) {
+          tc_mma_i8_zero(d_tmem, a0 + t[0].x, planes_lo + t[0].y, desc_hi, idesc);
+          tc_fence_before();
+          mbar_arrive(started0 + 8u * buf);
+        } else {
+          tc_mma_i8_acc(d_tmem, a0 + t[j].x, planes_lo + t[j].y, desc_hi, idesc);
+        }
+      }
+    }
+    tc_commit(empty0 + 8u * s);
+    tc_commit(acc_full0 + 8u * buf);
+    if (++s == stages) { s = 0; ph ^= 1u; }
   }
   return false;
 }
@@ -867,11 +983,11 @@ psb_mma_kernel(const __grid_constant__ TmapSet maps, const __grid_constant__ Ten
   if (threadIdx.x == 0) {
     for (uint32_t s = 0; s < p.stages; ++s) {
       mbar_init(smem_u32(&ctl->full[s]), 1);
-      mbar_init(smem_u32(&ctl->empty[s]), 1);
+      mbar_init(smem_u32(&ctl->empty[s]), p.band ? 2u : 1u);     // band mode: both issuing threads use every stage
     }
     for (int b = 0; b < 2; ++b) {
-      // both issuing threads commit to it when a pass has more than one stage
-      mbar_init(smem_u32(&ctl->acc_full[b]), (k_iters + p.group - 1) / p.group > 1u ? 2u : 1u);
+      // both issuing threads commit to it when a pass has more than one stage, and in band mode
+      mbar_init(smem_u32(&ctl->acc_full[b]), (p.band || (k_iters + p.group - 1) / p.group > 1u) ? 2u : 1u);
       mbar_init(smem_u32(&ctl->acc_empty[b]), kEpilogueWarps);
     }
     {  // part b of the resident planes holds K blocks [b * part, (b + 1) * part): one arrival per block
@@ -882,6 +998,7 @@ psb_mma_kernel(const __grid_constant__ TmapSet maps, const __grid_constant__ Ten
       }
     }
     for (int b = 0; b < 2; ++b) mbar_init(smem_u32(&ctl->started[b]), 1);
+    mbar_init(smem_u32(&ctl->pass_issued), 1);
     ctl->wait.abort = 0;
     ctl->wait.limit = p.wait_limit;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -990,8 +1107,10 @@ psb_mma_kernel(const __grid_constant__ TmapSet maps, const __grid_constant__ Ten
   } else if (warp == (uint32_t)kMmaWarp0 || warp == (uint32_t)kMmaWarp1) {
     // ---------------------------------------------------------------- MMA
     if (lane == 0)
-      failed = mma_role<BK>(p, ctl, tmem_base, smem_u32(ring), smem_u32(smem), stage_bytes, sub_bytes, k_iters,
-                            warp - (uint32_t)kMmaWarp0);
+      failed = p.band ? mma_role_band<BK>(p, ctl, tmem_base, smem_u32(ring), smem_u32(smem), stage_bytes,
+                                          warp - (uint32_t)kMmaWarp0)
+                      : mma_role<BK>(p, ctl, tmem_base, smem_u32(ring), smem_u32(smem), stage_bytes, sub_bytes, k_iters,
+                                     warp - (uint32_t)kMmaWarp0);
     failed = __shfl_sync(0xFFFFFFFFu, failed ? 1 : 0, 0) != 0;
   } else {
     // ----------------------------------------------------------- epilogue
@@ -1272,7 +1391,7 @@ psb_status launch_tensor(psb_ctx* ctx, const psb_weights* wt, const ConvArgs& a,
       const bool quotients_ok = Wp >= 2u && tpi >= 2u && tpi * kTileM * Wp < (1ull << 32) &&
                                 (uint64_t)a.N * tpi * tpi < (1ull << 32);
       if (codes_only && p.im2col && a.stride == 1 && a.KH * a.KW > 1u && a.C == bk && (bk == 64u || bk == 128u) &&
-          Wp <= 256u && rows <= 256u && (kSmemBudget - ctl_bytes - need) / bytes >= 2u && quotients_ok) {
+          Wp <= 256u && rows <= 256u && a.KH * a.KW * (bk / 32u) <= (uint32_t)(kMaxBandMmas - kTapBatch) && (kSmemBudget - ctl_bytes - need) / bytes >= 2u && quotients_ok) {
         p.band = 1;
         p.Wp = Wp;
         p.tpi = (uint32_t)tpi;

@@ -11,6 +11,7 @@ activation/weight pair, independent of k) with inputs resident in HBM; `e2e` is 
 through the public API from pinned host buffers, copies included.
 """
 import argparse
+import hashlib
 import json
 import os
 import statistics
@@ -36,6 +37,20 @@ def measured_peaks():
         return dict(hbm_gbs=d["hbm_gbs"], bf16_tflops=d["bf16_tflops"],
                     bf16_tflops_sustained=d.get("bf16_tflops_sustained", d["bf16_tflops"]), source="measured")
     return dict(hbm_gbs=6650.0, bf16_tflops=1590.0, bf16_tflops_sustained=1400.0, source="fallback")
+
+
+def measured_traffic(workload):
+    """DRAM bytes per launch of the dominant kernel from the last ncu capture of this workload
+    (profiles/traffic.json), or None when there is none or the kernel's source has changed since."""
+    path = os.path.join(ROOT, "profiles", "traffic.json")
+    if not os.path.exists(path):
+        return None
+    rec = json.load(open(path)).get(workload)
+    if not rec:
+        return None
+    src = os.path.join(ROOT, "paper_1904_02205_b200", "csrc", rec["source"])
+    sha = hashlib.sha256(open(src, "rb").read()).hexdigest()
+    return rec["dram_bytes_per_launch"] if sha == rec["source_sha256"] else None
 
 
 class ClockSampler:
@@ -154,12 +169,12 @@ class ConvWorkload:
         ops = 2.0 * self.macs * self.planes
         achieved = ops / (kernel_ms * 1e-3) / 1e12
         peak = 2.0 * peaks["bf16_tflops"]
-        # DRAM bytes of one launch from the ncu capture summarised in profiles/psb_mma_kernel_conv3x3_b32.md
-        # (dram__bytes_read.sum + dram__bytes_write.sum; k does not change them); to be set back to None
-        # whenever the kernel changes before the counters are taken again
+        # algorithmic bytes of the launch: activations in, codes out, digit planes once
+        alg_bytes = 2.0 * 32 * 64 * 56 * 56 + self.planes * 64 * 576
         return dict(bound="tensor", kernel="psb_mma_kernel", achieved=achieved, peak=peak, unit="TOP/s (int8)",
-                    frac=achieved / peak, traffic=6.63e6, traffic_unit="bytes per launch (ncu)",
-                    peak_source=peaks["source"] + " bf16 burst x 2",
+                    frac=achieved / peak, frac_vs_sustained=achieved / (2.0 * peaks["bf16_tflops_sustained"]),
+                    traffic=measured_traffic(self.name), traffic_unit="DRAM bytes per launch (ncu)",
+                    algorithmic_bytes=alg_bytes, peak_source=peaks["source"] + " bf16 burst x 2",
                     planes=self.planes, logical_gmacs=self.macs / (kernel_ms * 1e-3) / 1e9,
                     kernel_ms=kernel_ms)
 
@@ -341,20 +356,96 @@ class NetWorkload:
                     peak_source=peaks["source"] + " bf16 sustained x 2", planes=planes, tensor_path_ms=t_ms,
                     tensor_path_ms_per_layer_events=per_layer_ms, other_layers_ms=s_ms)
 
+    def truncate_for_oracle(self, budget_macs):
+        """Keep the longest prefix of the layer list whose work on one image fits the budget."""
+        from workloads import network_macs
+
+        keep = len(self.layers)
+        while keep > 1 and network_macs(self.layers[:keep]) > budget_macs:
+            keep -= 1
+        self.oracle_layers = self.layers[:keep]
+
     def oracle_sample(self, n_images=1):
         from oracle import psb_oracle as orc
 
+        layers = getattr(self, "oracle_layers", self.layers)
         if not hasattr(self, "net"):
             from workloads import build_network, saliency_kmaps
 
             self.net = build_network(self.layers, 224, max(n_images, 2), self.seed, self.qu, self.qs, prune_frac=self.prune)
             self.kmaps = saliency_kmaps(max(n_images, 2), [112, 56, 28, 14, 7], self.seed) if self.adaptive else None
         t0 = time.perf_counter()
-        orc.run_network(self.layers, self.net, self.net["image"][:n_images], self.seed, uniform_log2k=self.log2k,
+        from workloads import network_macs
+
+        orc.run_network(layers, self.net, self.net["image"][:n_images], self.seed, uniform_log2k=self.log2k,
                         fc_log2k=4 if self.adaptive else None,
                         kmaps=None if self.kmaps is None else {r: m[:n_images] for r, m in self.kmaps.items()})
         dt = time.perf_counter() - t0
-        return dt, self.macs_per_image * n_images, "first %d of %d images, all layers, filters sampled once" % (n_images, self.batch)
+        what = "all layers" if len(layers) == len(self.layers) else "the first %d of %d layers" % (len(layers), len(self.layers))
+        return dt, network_macs(layers) * n_images, "first %d of %d images, %s, filters sampled once" % (n_images, self.batch, what)
+
+
+def default_run_extras(args, ctx, psb, torch, timed):
+    """What the default run reports beside config 2 at k = 8: the bare int8 issue rate, the draw-count sweep of
+    the same layer, and the ResNet-50-shaped network at batch 64, k = 8 (per-launch device times from the
+    library's own events)."""
+    out = {}
+    for _ in range(2):
+        _, tops = ctx.int8_mma_probe(192, 20000)
+    out["int8_probe_tops"] = tops
+    sweep = {}
+    for k in (1, 2, 4, 16):
+        w = ConvWorkload(k, 0)
+        w.setup(ctx, psb, torch)
+        for i in range(3):
+            w.step(i)
+        ms = timed(w.step, 50, first=3)
+        sec = sum(ms) * 1e-3
+        sweep[str(k)] = dict(ms_per_step=sec * 1e3 / 50, gmacs=w.macs * 50 / sec / 1e9, images_per_s=w.images * 50 / sec)
+        w.wt.free()
+    out["k_sweep"] = sweep
+    ctx.set_sample_map(None, 3)
+    peaks = measured_peaks()
+    net = NetWorkload("resnet50", 8, 0, batch=64)
+    net.setup(ctx, psb, torch)
+    for i in range(3):
+        net.step(i)
+    ms = timed(net.step, 10, first=3)
+    sec = sum(ms) * 1e-3
+    sample_ms = timed(lambda i: net.nw.sample(100 + i), 5)
+    ctx.contraction_timing(True)
+    net.nw.forward()
+    per_launch = ctx.contraction_times()
+    ctx.contraction_timing(False)
+    planes = 3
+    tensor_layers = [l for l in net.layers if l["op"] == "conv" and net.nw.paths[l["name"]] == psb.PSB_PATH_TENSOR]
+    rec = dict(ms_per_step=sec * 1e3 / 10, images_per_s=net.batch * 10 / sec, gmacs=net.macs * 10 / sec / 1e9,
+               sampler_ms=statistics.mean(sample_ms[1:]), contraction_launches=len(per_launch))
+    if len(per_launch) == len(tensor_layers):
+        dense_ops, dense_ms, hbm_bytes, hbm_ms = 0.0, 0.0, 0.0, 0.0
+        for l, t in zip(tensor_layers, per_launch):
+            d = (l["cin"] // l["groups"]) * l["k"] ** 2
+            macs = l["hout"] ** 2 * l["cout"] * d * net.batch
+            nbytes = net.batch * (l["hin"] ** 2 * l["cin"] + l["hout"] ** 2 * l["cout"] * (2 if l["residual"] else 1)) + 4 * l["cout"] * d
+            # a layer is bound by bytes when its multiply-accumulates per byte, times the digit planes, stay
+            # below the ridge of the machine (measured tensor peak over measured HBM bandwidth)
+            ridge = 2.0 * peaks["bf16_tflops_sustained"] * 1e12 / 2.0 / (peaks["hbm_gbs"] * 1e9)
+            if macs * planes / nbytes >= ridge and l["name"] != "conv1":
+                dense_ops += 2.0 * macs * planes
+                dense_ms += t
+            else:
+                hbm_bytes += nbytes
+                hbm_ms += t
+        rec["dense_convs"] = dict(tops=dense_ops / (dense_ms * 1e-3) / 1e12, ms=dense_ms,
+                                  frac_of_2x_bf16_sustained=dense_ops / (dense_ms * 1e-3) / 1e12 / (2.0 * peaks["bf16_tflops_sustained"]),
+                                  frac_of_int8_probe=dense_ops / (dense_ms * 1e-3) / 1e12 / tops)
+        rec["bandwidth_bound_layers"] = dict(gbs=hbm_bytes / (hbm_ms * 1e-3) / 1e9, ms=hbm_ms,
+                                             frac_of_hbm=hbm_bytes / (hbm_ms * 1e-3) / 1e9 / peaks["hbm_gbs"],
+                                             note="algorithmic bytes (input, output, shortcut, fp32 filter once) over the "
+                                                  "contraction kernel's device time; the stem's gather pass is not in it")
+    out["resnet50_b64_k8"] = rec
+    net.nw.free()
+    return out
 
 
 def make_workload(args, rank):
@@ -387,7 +478,13 @@ def run_reference(args):
     if rank != 0:
         return 0
     wl = make_workload(args, 0)
-    n_img = getattr(wl, "oracle_images", 1)
+    # a bounded sample per step, so that the whole run stays within a few minutes whatever --steps is: the
+    # oracle does about 0.6 G multiply-accumulates per second on one core
+    budget_macs = 0.6e9 * 150.0 / max(1, args.warmup + args.steps)
+    per_image = wl.macs / wl.images
+    n_img = int(max(1, min(getattr(wl, "oracle_images", 1), budget_macs // per_image)))
+    if isinstance(wl, NetWorkload) and per_image > budget_macs:
+        wl.truncate_for_oracle(budget_macs)
     times, macs, sample = [], 0, ""
     for i in range(args.warmup + args.steps):
         dt, macs, sample = wl.oracle_sample(n_img)
@@ -426,13 +523,15 @@ def run_int8_probe(ctx, index):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="psb")
     ap.add_argument("--workload", default="conv3x3", choices=["conv3x3", "fc", "resnet50", "mobilenetv2", "resnet50_adaptive"])
     ap.add_argument("--k", type=int, default=8)
     ap.add_argument("--batch", type=int, default=0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-extras", action="store_true",
+                    help="default workload only: skip the draw-count sweep, the int8 probe and the network record")
     ap.add_argument("--layer-table", default="", help="write per-layer times of the network workloads to this CSV")
     ap.add_argument("--probe-int8", action="store_true",
                     help="measure the bare tcgen05 int8 MMA issue rate instead of a workload and exit")
@@ -508,6 +607,9 @@ def main():
             wl.nw.forward()
             wl.hook_ms.append(ctx.contraction_time())
         ctx.contraction_timing(False)
+    extras = {}
+    if args.workload == "conv3x3" and world == 1 and not args.no_extras:
+        extras = default_run_extras(args, ctx, psb, torch, timed)
     clk = clocks.stop()
     ctx.check_device()
     e2e_warm = timed(wl.e2e_step, 3)
@@ -537,7 +639,19 @@ def main():
     if in_step_ms:
         # for comparison: the same kernel inside the step, where it writes planar output and, with the events
         # around it, cannot start under the conversion kernel's tail (an empty pair of events reads 2.7 us)
-        line["roofline"]["kernel_ms_in_step_planar_out"] = statistics.mean(in_step_ms)
+        r = line["roofline"]
+        r["kernel_ms_in_step_planar_out"] = statistics.mean(in_step_ms)
+        r["frac_in_step"] = r["frac"] * r["kernel_ms"] / r["kernel_ms_in_step_planar_out"]
+    if clk.get("sm_mhz"):
+        # kernel time x the SM clock sampled under load: comparable across runs whatever the clock was
+        line["roofline"]["kernel_clocks"] = line["roofline"].get("kernel_ms", 0.0) * 1e-3 * clk["sm_mhz"] * 1e6
+    if "int8_probe_tops" in extras:
+        # the bare tcgen05 int8 issue rate measured in this process (zero operands, so the clocks stay up)
+        line["roofline"]["int8_probe_tops"] = extras["int8_probe_tops"]
+        line["roofline"]["frac_vs_int8_probe"] = line["roofline"]["achieved"] / extras["int8_probe_tops"]
+    for key in ("k_sweep", "resnet50_b64_k8"):
+        if key in extras:
+            line[key] = extras[key]
     if not args.no_cpu_baseline and world == 1:
         dt, macs, sample = wl.oracle_sample(getattr(wl, "oracle_images", 4))
         line["cpu_baseline"] = dict(value=macs / dt / 1e9, unit=UNIT, cores=1, kind="oracle", sample=sample)

@@ -251,6 +251,9 @@ uint64_t psb_launch_count(void);
  * PSB_ERR_CUDA if the events cannot be created or read. */
 psb_status psb_contraction_timing(psb_ctx* ctx, uint32_t enable);
 psb_status psb_contraction_time(psb_ctx* ctx, float* milliseconds);
+/* The same launches one by one, in launch order: *count receives how many have been timed since timing
+ * was switched on, milliseconds[0 .. min(*count, capacity)) their durations. */
+psb_status psb_contraction_times(psb_ctx* ctx, float* milliseconds, uint32_t capacity, uint32_t* count);
 
 /* Measurement aid, no counterpart in the paper: the ceiling of the dense path.
  * Every SM issues `groups` groups of four back-to-back tcgen05.mma kind::i8

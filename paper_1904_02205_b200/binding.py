@@ -26,7 +26,7 @@ EXPORTS = ["psb_create", "psb_destroy", "psb_status_string", "psb_device_status"
            "psb_last_path", "psb_maxpool2d_u8", "psb_global_avgpool_u8", "psb_sample_level_static",
            "psb_sample_batch_create", "psb_sample_batch_run", "psb_sample_batch_free", "psb_run",
            "psb_launch_count", "psb_int8_mma_probe", "psb_contraction_timing", "psb_contraction_time",
-           "psb_set_checks", "psb_set_wait_limit", "psb_wait_selftest"]
+           "psb_set_checks", "psb_set_wait_limit", "psb_wait_selftest", "psb_contraction_times"]
 
 
 class psb_wshape(C.Structure):
@@ -95,6 +95,7 @@ def load_library():
     lib.psb_int8_mma_probe.argtypes = [vp, u32, u32, C.POINTER(C.c_double), C.POINTER(C.c_double), vp]
     lib.psb_contraction_timing.argtypes = [vp, u32]
     lib.psb_contraction_time.argtypes = [vp, C.POINTER(C.c_float)]
+    lib.psb_contraction_times.argtypes = [vp, C.POINTER(C.c_float), u32, C.POINTER(u32)]
     lib.psb_set_checks.argtypes = [vp, u32]
     lib.psb_set_wait_limit.argtypes = [vp, C.c_uint64]
     lib.psb_wait_selftest.argtypes = [vp, vp]
@@ -236,6 +237,12 @@ class Context:
         ms = C.c_float(0.0)
         _check(self.lib.psb_contraction_time(self.handle, C.byref(ms)), "psb_contraction_time")
         return float(ms.value)
+
+    def contraction_times(self):
+        """Device time in milliseconds of each contraction launch made since timing was switched on."""
+        buf, n = (C.c_float * 256)(), C.c_uint32(0)
+        _check(self.lib.psb_contraction_times(self.handle, buf, 256, C.byref(n)), "psb_contraction_times")
+        return [float(buf[i]) for i in range(min(n.value, 256))]
 
     def launch_count(self):
         """Kernels launched by the library in this process so far."""

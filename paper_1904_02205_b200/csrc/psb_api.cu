@@ -462,6 +462,19 @@ psb_status psb_contraction_time(psb_ctx* ctx, float* milliseconds) {
   return PSB_OK;
 }
 
+psb_status psb_contraction_times(psb_ctx* ctx, float* milliseconds, uint32_t capacity, uint32_t* count) {
+  if (!ctx || !milliseconds || !count) return PSB_ERR_INVALID_ARG;
+  *count = (uint32_t)ctx->timed_launches;
+  for (int i = 0; i < ctx->timed_launches && (uint32_t)i < capacity; ++i) {
+    if (cudaEventSynchronize(ctx->t_end[i]) != cudaSuccess ||
+        cudaEventElapsedTime(&milliseconds[i], ctx->t_begin[i], ctx->t_end[i]) != cudaSuccess) {
+      cudaGetLastError();
+      return PSB_ERR_CUDA;
+    }
+  }
+  return PSB_OK;
+}
+
 psb_status psb_int8_mma_probe(psb_ctx* ctx, uint32_t n_cols, uint32_t groups, double* mac_per_clk_per_sm,
                               double* tera_ops_per_s, void* stream) {
   if (!ctx) return PSB_ERR_INVALID_ARG;

@@ -24,6 +24,14 @@
 //     stream, so larger levels refine smaller ones ("progressive").
 //   * the division by k (the ">> n" of Eq. 9) is never applied to integers: the
 //     accumulator stays exact and 1/k is folded into the floating-point scale.
+//   * optional (Sec. 3.1 "Stochastic multiplication", applied at the floor of the window): a weight
+//     below the window, |w| < 2^e_base, is not flushed but replaced per draw by s * 2^e_base * B_q with
+//     q = |w| / 2^e_base, the plain Bernoulli gate of Eq. 2-3; unbiased, no "+ 1" term.
+//   * optional (Sec. 4.4): probabilities stored with b bits on the regular grid {0, 1/2^b, ...,
+//     1 - 1/2^b}; p is rounded to the nearest grid point, and a p that rounds to 1 becomes p = 0 at the
+//     next exponent ("the right boundary would result in a higher exponent").  The comparator then has
+//     b bits (supplement, "Stochastic multiplier") and one Philox word serves floor(32 / b) draws.
+//     The deterministic variant of Sec. 4.4 uses the upper shift in round(p_q * k) of the k cases.
 //   * the random stream is Philox4x32-10 (Salmon, Moraes, Dror, Shaw, SC'11),
 //     counter = (draw / 4, layer, lo32(weight index), hi32(weight index)),
 //     key = (lo32(seed), hi32(seed)); draw j uses output word j mod 4.
@@ -85,16 +93,80 @@ void philox4x32_10(const uint32_t ctr[4], const uint32_t key[2], uint32_t out[4]
 // One Bernoulli draw B_p of Eq. 4: compare a uniform 32-bit word with p * 2^32.
 // This is the comparator of the paper's stochastic multiplier (supplement,
 // "Stochastic multiplier").  Pr[bit = 1] = (m << 9) / 2^32 = p exactly.
-int draw_bit(uint64_t seed, uint32_t layer, uint64_t index, uint32_t j, uint32_t m) {
+int draw_bit_thr(uint64_t seed, uint32_t layer, uint64_t index, uint32_t j, uint32_t T) {
   uint32_t ctr[4] = {j >> 2, layer, (uint32_t)index, (uint32_t)(index >> 32)};
   uint32_t key[2] = {(uint32_t)seed, (uint32_t)(seed >> 32)};
   uint32_t r[4];
   philox4x32_10(ctr, key, r);
-  uint32_t T = m << 9;
-  return r[j & 3] < T ? 1 : 0;
+  return r[j & 3] < T ? 1 : 0;      // Pr[1] = T / 2^32
+}
+
+int draw_bit(uint64_t seed, uint32_t layer, uint64_t index, uint32_t j, uint32_t m) {
+  return draw_bit_thr(seed, layer, index, j, m << 9);
 }
 
 inline int64_t ipow2(int n) { return (int64_t)1 << n; }
+
+// Sec. 4.4: the probability on a grid of 2^b points, nearest point, p = 1 carried into the exponent.
+// Returns the quantised (e, p * 2^b).  b == 0 leaves the weight as it is (p * 2^23 in *pq).
+void quantise(const Decoded& d, uint32_t b, int* e, uint32_t* pq) {
+  *e = d.e;
+  if (b == 0) { *pq = d.m; return; }
+  uint32_t q = (d.m + (1u << (22 - b))) >> (23 - b);     // round half up to b bits
+  if (q == (1u << b)) {
+    if (d.e < 127) { *e = d.e + 1; q = 0; }              // the next power of two, exactly
+    else q = (1u << b) - 1;                              // no exponent above: the last grid point
+  }
+  *pq = q;
+}
+
+// One draw with a b-bit comparator: draw j takes bit field (j mod n) of output word ((j / n) mod 4) of
+// Philox call j / (4 n), n = floor(32 / b) fields per word, field f = bits [f b, f b + b).
+int draw_bit_packed(uint64_t seed, uint32_t layer, uint64_t index, uint32_t j, uint32_t thr, uint32_t b) {
+  const uint32_t n = 32u / b;
+  uint32_t ctr[4] = {j / (4u * n), layer, (uint32_t)index, (uint32_t)(index >> 32)};
+  uint32_t key[2] = {(uint32_t)seed, (uint32_t)(seed >> 32)};
+  uint32_t r[4];
+  philox4x32_10(ctr, key, r);
+  const uint32_t field = (r[(j / n) & 3u] >> ((j % n) * b)) & ((1u << b) - 1u);
+  return field < thr ? 1 : 0;
+}
+
+// What one weight turns into under a given window: W_k = s (base k + c_k) 2^sh, c_k counting draws with
+// Pr[1] = thr / 2^32 (b == 0) or thr / 2^b.
+struct Sampled {
+  int live;        // 0: contributes nothing
+  uint32_t base;   // 1: a weight inside the window (Eq. 8); 0: the Bernoulli gate below it
+  int sh;
+  uint32_t thr;
+};
+
+Sampled classify(const Decoded& d, int e_base, uint32_t b, uint32_t underflow) {
+  Sampled r = {0, 0, 0, 0};
+  if (d.cls != CLASS_NORMAL) return r;
+  int e;
+  uint32_t pq;
+  quantise(d, b, &e, &pq);
+  if (e >= e_base) {
+    r.live = 1; r.base = 1; r.sh = e - e_base;
+    r.thr = b ? pq : (pq << 9);
+    return r;
+  }
+  if (!underflow) return r;
+  // q = |w| / 2^e_base = (1 + p) 2^-dist, dist >= 1
+  const int dist = e_base - e;
+  if (b == 0) {
+    const uint64_t mant = ((uint64_t)(1u << 23) + pq) << 9;          // (1 + p) 2^32
+    const uint32_t thr = dist < 42 ? (uint32_t)(mant >> dist) : 0u;   // floor(q 2^32)
+    if (thr) { r.live = 1; r.thr = thr; }
+    return r;
+  }
+  const uint64_t mant = ((uint64_t)1 << b) + pq;                      // (1 + p_q) 2^b
+  const uint64_t q = dist < 40 ? (mant + ((uint64_t)1 << (dist - 1))) >> dist : 0;   // round half up to b bits
+  if (q == ((uint64_t)1 << b)) { r.live = 1; r.base = 1; r.sh = 0; r.thr = 0; }      // rounds to 2^e_base exactly
+  else if (q) { r.live = 1; r.thr = (uint32_t)q; }
+  return r;
+}
 
 }  // namespace
 
@@ -140,6 +212,91 @@ int psbo_window(const float* w, uint32_t O, uint64_t D, uint32_t exp_bits, uint3
   }
   if (norm == 0)
     for (uint32_t o = 0; o < O; ++o) e_base[o] = any_layer ? emax_layer - span : 0;
+  return 0;
+}
+
+// The same with b-bit probabilities: the window is taken over the exponents after quantisation.
+int psbo_window_q(const float* w, uint32_t O, uint64_t D, uint32_t exp_bits, uint32_t norm, uint32_t prob_bits,
+                  int32_t* e_base) {
+  const int span = (1 << exp_bits) - 1;
+  bool any_layer = false;
+  int emax_layer = 0;
+  for (uint32_t o = 0; o < O; ++o) {
+    bool any = false;
+    int emax = 0;
+    for (uint64_t i = 0; i < D; ++i) {
+      Decoded d = decode(w[o * D + i]);
+      if (d.cls == CLASS_NONFINITE) return -1;
+      if (d.cls == CLASS_ZERO) continue;
+      int e;
+      uint32_t pq;
+      quantise(d, prob_bits, &e, &pq);
+      if (!any || e > emax) { emax = e; any = true; }
+    }
+    if (norm == 1) e_base[o] = any ? emax - span : 0;
+    if (any && (!any_layer || emax > emax_layer)) { emax_layer = emax; any_layer = true; }
+  }
+  if (norm == 0)
+    for (uint32_t o = 0; o < O; ++o) e_base[o] = any_layer ? emax_layer - span : 0;
+  return 0;
+}
+
+int psbo_quantise(float w, uint32_t prob_bits, int* e, uint32_t* pq) {
+  Decoded d = decode(w);
+  if (d.cls == CLASS_NORMAL) quantise(d, prob_bits, e, pq);
+  return d.cls;
+}
+
+// What a weight becomes under a window with base exponent e_base: out = (live, base, sh, thr), see
+// psbo_sample_level_ex.  Exposed for the pins.
+void psbo_classify(float w, int32_t e_base, uint32_t prob_bits, uint32_t underflow, uint32_t* out) {
+  const Sampled sm = classify(decode(w), e_base, prob_bits, underflow);
+  out[0] = (uint32_t)sm.live; out[1] = sm.base; out[2] = (uint32_t)sm.sh; out[3] = sm.thr;
+}
+
+int psbo_draw_bit_packed(uint64_t seed, uint32_t layer, uint64_t index, uint32_t j, uint32_t thr, uint32_t prob_bits) {
+  return draw_bit_packed(seed, layer, index, j, thr, prob_bits);
+}
+
+// Integer weights of one level with the options of Sec. 3.1 / 4.4:
+//   opts[0] exp_bits, [1] norm, [2] underflow (0 flush below the window, 1 Bernoulli gate at its floor),
+//   [3] prob_bits (0 = the full 23 bits, else 1..8), [4] deterministic (needs prob_bits > 0).
+// W_k[i] = s (base k + c_k) 2^sh; inside the window base = 1, sh = e - e_base (Eq. 8 scaled by k / 2^e_base);
+// below it (underflow = 1) base = 0, sh = 0, so that W_k 2^e_base / k = s 2^e_base c_k / k with
+// c_k ~ Binomial(k, |w| / 2^e_base).  class_out (optional): 0 nothing, 1 window, 2 gate.
+int psbo_sample_level_ex(const float* w, uint32_t O, uint64_t D, uint64_t seed, uint32_t layer,
+                         const uint32_t* opts, uint32_t log2k, const uint32_t* counts_in, int64_t* W_out,
+                         int32_t* e_base, uint32_t* counts_out, uint8_t* class_out) {
+  const uint32_t exp_bits = opts[0], norm = opts[1], underflow = opts[2], b = opts[3], deterministic = opts[4];
+  if (b > 8 || (deterministic && b == 0)) return -3;
+  if (psbo_window_q(w, O, D, exp_bits, norm, b, e_base) != 0) return -1;
+  const uint32_t k = 1u << log2k;
+  for (uint32_t o = 0; o < O; ++o) {
+    for (uint64_t pos = 0; pos < D; ++pos) {
+      const uint64_t i = (uint64_t)o * D + pos;
+      const Decoded d = decode(w[i]);
+      const Sampled sm = classify(d, e_base[o], b, underflow);
+      uint32_t c = 0;
+      if (class_out) class_out[i] = sm.live ? (sm.base ? 1 : 2) : 0;
+      if (!sm.live) {
+        W_out[i] = 0;
+        if (counts_out) counts_out[i] = 0;
+        continue;
+      }
+      if (counts_in) {
+        c = counts_in[i];
+      } else if (deterministic) {
+        c = (sm.thr * k + (1u << (b - 1))) >> b;            // the upper shift in round(p_q k) of k cases
+      } else {
+        for (uint32_t j = 0; j < k; ++j)
+          c += b ? (uint32_t)draw_bit_packed(seed, layer, i, j, sm.thr, b)
+                 : (uint32_t)draw_bit_thr(seed, layer, i, j, sm.thr);
+      }
+      const int64_t mag = (int64_t)(sm.base * k + c) * ipow2(sm.sh);
+      W_out[i] = d.s ? -mag : mag;
+      if (counts_out) counts_out[i] = c;
+    }
+  }
   return 0;
 }
 

@@ -104,6 +104,52 @@ def sample_level(w, seed, layer, log2k, exp_bits=4, norm=0, counts_in=None):
     return W_out, e_base, counts
 
 
+def sample_level_ex(w, seed, layer, log2k, exp_bits=4, norm=0, underflow=0, prob_bits=0, deterministic=0,
+                    counts_in=None):
+    """Integer weights of one level with the options of Sec. 3.1 (Bernoulli gate below the window) and
+    Sec. 4.4 (b-bit probabilities, packed draws, deterministic variant).
+
+    Returns (W int64, e_base int32 [O], counts uint32, cls uint8: 0 nothing, 1 inside the window, 2 gate).
+    """
+    w = np.ascontiguousarray(w, dtype=np.float32)
+    O = w.shape[0]
+    D = int(np.prod(w.shape[1:])) if w.ndim > 1 else 1
+    W_out = np.zeros(w.shape, dtype=np.int64)
+    e_base = np.zeros(O, dtype=np.int32)
+    counts = np.zeros(w.shape, dtype=np.uint32)
+    cls = np.zeros(w.shape, dtype=np.uint8)
+    opts = np.array([exp_bits, norm, underflow, prob_bits, deterministic], dtype=np.uint32)
+    cin = None if counts_in is None else np.ascontiguousarray(counts_in, dtype=np.uint32)
+    lib().psbo_sample_level_ex.restype = C.c_int
+    rc = lib().psbo_sample_level_ex(_p(w), C.c_uint32(O), C.c_uint64(D), C.c_uint64(seed), C.c_uint32(layer),
+                                    _p(opts), C.c_uint32(log2k), _p(cin), _p(W_out), _p(e_base), _p(counts), _p(cls))
+    if rc == -1:
+        raise ValueError("non-finite weight")
+    if rc != 0:
+        raise ValueError("bad sampling options")
+    return W_out, e_base, counts, cls
+
+
+def quantise(w, prob_bits):
+    """Sec. 4.4: (class, e, p * 2^prob_bits) of a weight after rounding p to the grid."""
+    e, pq = C.c_int(), C.c_uint32()
+    cls = lib().psbo_quantise(C.c_float(float(np.float32(w))), C.c_uint32(prob_bits), C.byref(e), C.byref(pq))
+    return cls, e.value, pq.value
+
+
+def classify(w, e_base, prob_bits=0, underflow=0):
+    """(live, base, sh, thr) of one weight under a window with base exponent e_base."""
+    out = np.zeros(4, dtype=np.uint32)
+    lib().psbo_classify(C.c_float(float(np.float32(w))), C.c_int32(e_base), C.c_uint32(prob_bits),
+                        C.c_uint32(underflow), _p(out))
+    return tuple(int(v) for v in out)
+
+
+def draw_bit_packed(seed, layer, index, j, thr, prob_bits):
+    lib().psbo_draw_bit_packed.argtypes = [C.c_uint64, C.c_uint32, C.c_uint64, C.c_uint32, C.c_uint32, C.c_uint32]
+    return lib().psbo_draw_bit_packed(seed, layer, index, j, thr, prob_bits)
+
+
 def geom(x_shape, layout, x_dtype, w_shape, groups, stride, pad):
     if layout == NCHW:
         N, Cc, H, W = x_shape

@@ -123,13 +123,34 @@ typedef struct {
  *                   below the group's largest exponent; smaller weights, zeros
  *                   and sub-normals contribute nothing (Sec. 4.4: 4-bit
  *                   exponents suffice).  0 selects 4.
- *   norm            0: one exponent window per layer; 1: one per output channel. */
+ *   norm            0: one exponent window per layer; 1: one per output channel.
+ *   underflow       0: weights below the window contribute nothing.  1: a weight below the
+ *                   window, |w| < 2^e_base, is replaced per draw by s * 2^e_base * B_q with
+ *                   q = |w| / 2^e_base (the plain Bernoulli gate of Sec. 3.1, "Stochastic
+ *                   multiplication"): W_k = s * c_k with c_k ~ Binomial(k, q), unbiased, which is
+ *                   what makes windows of fewer octaves (exp_bits 3, 2: fewer digit planes)
+ *                   usable.  Draw j uses the same random word as above, compared with
+ *                   floor(q * 2^32).
+ *   prob_bits       0: probabilities keep their 23 bits.  b = 1..8 (Sec. 4.4): p is rounded to the
+ *                   nearest point of the grid {0, 1/2^b, .., 1 - 1/2^b}; a p that rounds to 1
+ *                   becomes p = 0 at the next exponent (before the window is taken); the
+ *                   comparator has b bits and one random word serves n = floor(32 / b) draws:
+ *                   draw j compares bits [f*b, f*b + b), f = j mod n, of word (j / n) mod 4 of
+ *                   Philox4x32-10 with counter (j / (4n), layer_id, lo32(i), hi32(i)) with p * 2^b.
+ *                   With underflow = 1, q is rounded to the same grid (q = 1: the weight 2^e_base).
+ *   deterministic   1 (needs prob_bits > 0): no draws; the upper shift is taken in
+ *                   round(p * k) of the k cases (Sec. 4.4, the variant for bounded precision).
+ *   reserved        0. */
 typedef struct {
   uint64_t seed;
   uint32_t layer_id;
   uint32_t level_mask;
   uint32_t exp_bits;
   uint32_t norm;
+  uint32_t underflow;
+  uint32_t prob_bits;
+  uint32_t deterministic;
+  uint32_t reserved;
 } psb_sample_cfg;
 
 /* Draw the random bits and build the integer filters (Eq. 8 scaled by
@@ -332,7 +353,8 @@ psb_status psb_run(psb_ctx* ctx, const psb_op* ops, uint32_t n_ops, void* stream
  * array inside the library's device image (PSB_STATIC_MAX_OUT_CH words + 256 B,
  * held by every GPU that loads the library until the process exits).
  *
- *   w_dev, shape, cfg   as for psb_sample_weights; cfg->level_mask is ignored.
+ *   w_dev, shape, cfg   as for psb_sample_weights; cfg->level_mask is ignored; the options underflow,
+ *                       prob_bits and deterministic must be 0 (PSB_ERR_UNSUPPORTED otherwise).
  *   log2k               the one level to produce, k = 2^log2k, 0..6.
  *   wint_out_dev        int32, canonical [out_ch][in_ch_per_group][kh][kw] order,
  *                       caller-owned device memory; receives the same integers that

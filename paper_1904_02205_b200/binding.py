@@ -35,7 +35,8 @@ class psb_wshape(C.Structure):
 
 class psb_sample_cfg(C.Structure):
     _fields_ = [("seed", C.c_uint64), ("layer_id", C.c_uint32), ("level_mask", C.c_uint32),
-                ("exp_bits", C.c_uint32), ("norm", C.c_uint32)]
+                ("exp_bits", C.c_uint32), ("norm", C.c_uint32), ("underflow", C.c_uint32),
+                ("prob_bits", C.c_uint32), ("deterministic", C.c_uint32), ("reserved", C.c_uint32)]
 
 
 class psb_epilogue(C.Structure):
@@ -162,7 +163,7 @@ def sample_level_static(w, wint_out, e_base_out, groups=1, seed=0, layer_id=0, l
     """
     assert w.is_cuda and w.dtype == torch.float32 and w.is_contiguous()
     shape = psb_wshape(w.shape[0], w.shape[1], w.shape[2], w.shape[3], groups)
-    cfg = psb_sample_cfg(seed, layer_id, 0, exp_bits, norm)
+    cfg = psb_sample_cfg(seed, layer_id, 0, exp_bits, norm, 0, 0, 0, 0)
     with torch.cuda.device(w.device):
         _check(load_library().psb_sample_level_static(_ptr(w), C.byref(shape), C.byref(cfg), log2k,
                                                       _ptr(wint_out), _ptr(e_base_out), _stream(stream)),
@@ -250,13 +251,13 @@ class Context:
 
     # -- psb_sample_weights --------------------------------------------------
     def sample_weights(self, w, groups=1, seed=0, layer_id=0, level_mask=1, exp_bits=4, norm=0,
-                       into=None, stream=None):
+                       into=None, stream=None, underflow=0, prob_bits=0, deterministic=0):
         """w: float32 CUDA tensor [out_ch, in_ch/groups, kh, kw] (or [out, in] for a FC layer)."""
         assert w.is_cuda and w.dtype == torch.float32 and w.is_contiguous()
         if w.dim() == 2:
             w = w.view(w.shape[0], w.shape[1], 1, 1)
         shape = psb_wshape(w.shape[0], w.shape[1], w.shape[2], w.shape[3], groups)
-        cfg = psb_sample_cfg(seed, layer_id, level_mask, exp_bits, norm)
+        cfg = psb_sample_cfg(seed, layer_id, level_mask, exp_bits, norm, underflow, prob_bits, deterministic, 0)
         h = C.c_void_p(into.handle.value if into is not None else None)
         _check(self.lib.psb_sample_weights(self.handle, _ptr(w), C.byref(shape), C.byref(cfg),
                                            C.byref(h), _stream(stream)), "psb_sample_weights")

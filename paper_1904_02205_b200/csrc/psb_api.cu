@@ -307,6 +307,9 @@ psb_status psb_sample_weights(psb_ctx* ctx, const float* w_dev, const psb_wshape
   psb_sample_cfg cfg = *cfg_in;
   if (cfg.exp_bits == 0) cfg.exp_bits = 4;
   if (cfg.exp_bits > 4 || cfg.norm > 1) return PSB_ERR_INVALID_ARG;
+  if (cfg.underflow > 1 || cfg.prob_bits > 8 || cfg.deterministic > 1 || cfg.reserved != 0 ||
+      (cfg.deterministic && cfg.prob_bits == 0))
+    return PSB_ERR_INVALID_ARG;
   if (cfg.level_mask == 0 || cfg.level_mask >= (1u << kMaxLevels)) return PSB_ERR_BAD_K;
   if (!shape->out_ch || !shape->in_ch_per_group || !shape->kh || !shape->kw || !shape->groups)
     return PSB_ERR_INVALID_ARG;

@@ -67,10 +67,19 @@ __device__ __forceinline__ uint32_t small_div(uint32_t t, uint32_t magic) { retu
 // Largest biased exponent of the finite weights of each exponent group; flags Inf/NaN (which
 // contribute nothing: the finite weights of the group keep the window they would have without it).
 // norm == 1: one block per output channel.  norm == 0: grid-stride over the layer.
+// Biased exponent of a weight after its probability has been rounded to `pbits` bits (Sec. 4.4): a
+// probability that rounds to 1 is the next power of two.  pbits == 0: the exponent as it is.
+__device__ __forceinline__ uint32_t quantised_exponent(uint32_t u, uint32_t pbits) {
+  const uint32_t E = (u >> 23) & 0xFFu;
+  if (pbits == 0u || E == 0u || E >= 254u) return E;
+  const uint32_t pq = ((u & 0x7FFFFFu) + (1u << (22u - pbits))) >> (23u - pbits);
+  return E + (pq >> pbits);
+}
+
 __device__ __forceinline__ void emax_block(const float* __restrict__ w, uint32_t O, uint32_t d,
                                            uint32_t norm, uint32_t* __restrict__ e_max,
                                            uint32_t* __restrict__ err, uint32_t block, uint32_t blocks,
-                                           uint32_t tag, uint32_t* __restrict__ rowsum) {
+                                           uint32_t tag, uint32_t* __restrict__ rowsum, uint32_t pbits) {
   __shared__ uint32_t red[kThreads / 32];
   // the sampling pass that follows adds its row sums of |W_k| into these words: start them at zero
   if (rowsum)
@@ -81,14 +90,14 @@ __device__ __forceinline__ void emax_block(const float* __restrict__ w, uint32_t
   if (norm) {
     const float* row = w + (size_t)block * d;
     for (uint32_t i = threadIdx.x; i < d; i += blockDim.x) {
-      uint32_t E = (__float_as_uint(row[i]) >> 23) & 0xFFu;
+      uint32_t E = quantised_exponent(__float_as_uint(row[i]), pbits);
       bad |= (E == 255u);
       best = max(best, E == 255u ? 0u : E);     // Inf/NaN is flagged and takes no part in the window
     }
   } else {
     size_t total = (size_t)O * d;
     for (size_t i = (size_t)block * blockDim.x + threadIdx.x; i < total; i += (size_t)blocks * blockDim.x) {
-      uint32_t E = (__float_as_uint(w[i]) >> 23) & 0xFFu;
+      uint32_t E = quantised_exponent(__float_as_uint(w[i]), pbits);
       bad |= (E == 255u);
       best = max(best, E == 255u ? 0u : E);
     }
@@ -108,9 +117,9 @@ __device__ __forceinline__ void emax_block(const float* __restrict__ w, uint32_t
 
 __global__ void emax_kernel(const float* __restrict__ w, uint32_t O, uint32_t d, uint32_t norm,
                             uint32_t* __restrict__ e_max, uint32_t* __restrict__ err, uint32_t tag,
-                            uint32_t* __restrict__ rowsum) {
+                            uint32_t* __restrict__ rowsum, uint32_t pbits) {
   pdl_prologue();
-  emax_block(w, O, d, norm, e_max, err, blockIdx.x, gridDim.x, tag, rowsum);
+  emax_block(w, O, d, norm, e_max, err, blockIdx.x, gridDim.x, tag, rowsum, pbits);
 }
 
 struct SampleParams {
@@ -118,6 +127,7 @@ struct SampleParams {
   uint32_t O, Cg, KHKW, d;
   uint32_t rows_per_block, ch_per_block, ch_chunks;
   uint32_t norm, span, level_mask, max_level;
+  uint32_t underflow, pbits, deterministic;   // options of psb_sample_cfg
   uint32_t seed_lo, seed_hi, layer_id;
   uint32_t cpad, kpad, has_planes;
   uint32_t bk, n_cb, n_kb;         // operand tiles of the tensor path: K block bytes, blocks per tap, blocks per row
@@ -135,6 +145,7 @@ __device__ __forceinline__ void sample_block(const SampleParams& p, uint32_t blo
                                              uint32_t seed_hi, float* stage) {
   // the parameters may sit in global memory (batched launch): read the scalars once
   const uint32_t norm = p.norm, span = p.span, level_mask = p.level_mask, max_level = p.max_level;
+  const uint32_t underflow = p.underflow, pbits = p.pbits, deterministic = p.deterministic;
   const uint32_t layer_id = p.layer_id, KHKW = p.KHKW, Cg = p.Cg;
   const uint32_t packed_kw = p.packed_kw, run_pitch = p.run_pitch, has_planes = p.has_planes;
   const uint32_t bk = p.bk, n_cb = p.n_cb, n_kb = p.n_kb;
@@ -181,31 +192,82 @@ __device__ __forceinline__ void sample_block(const SampleParams& p, uint32_t blo
     // biased exponents throughout: e - e_base = E - (Emax - span)
     const int ebase_biased = (int)Emax - (int)span;
     if (tap == 0 && ci == 0) p.e_base[o] = Emax ? ebase_biased - 127 : 0;
-    const bool live = (E != 0u) && (E != 255u) && ((int)E >= ebase_biased);
-    const uint32_t sh = live ? (uint32_t)((int)E - ebase_biased) : 0u;
+    // probability on the grid of 2^pbits points, a p of 1 carried into the exponent (Sec. 4.4)
+    uint32_t Eq = E, pq = m;
+    if (pbits) {
+      pq = (m + (1u << (22u - pbits))) >> (23u - pbits);
+      if (pq == (1u << pbits)) {
+        if (E < 254u) { Eq = E + 1u; pq = 0u; } else pq = (1u << pbits) - 1u;
+      }
+    }
+    // what the weight becomes: W_k = s (base k + c_k) 2^sh, c_k counting draws with Pr[1] = thr / 2^32 (or
+    // thr / 2^pbits).  Inside the window base = 1 (Eq. 8); below it, if asked for, the Bernoulli gate at the
+    // window's floor (Sec. 3.1): base = 0, sh = 0, thr = |w| / 2^e_base
+    bool live = (E != 0u) && (E != 255u);
+    uint32_t base = 1u, sh = 0u, thr = 0u;
+    const int dist = ebase_biased - (int)Eq;
+    if (dist <= 0) {
+      sh = (uint32_t)(-dist);
+      thr = pbits ? pq : pq << 9;
+    } else if (underflow) {
+      base = 0u;
+      if (pbits == 0u) {
+        thr = dist < 42 ? (uint32_t)((((unsigned long long)(0x800000u + pq)) << 9) >> dist) : 0u;
+        live = live && thr != 0u;
+      } else {
+        const unsigned long long mant = (1ull << pbits) + pq;
+        const unsigned long long qv = dist < 40 ? (mant + (1ull << (dist - 1))) >> dist : 0ull;
+        if (qv == (1ull << pbits)) base = 1u;          // rounds to the window's floor itself
+        else { thr = (uint32_t)qv; live = live && qv != 0ull; }
+      }
+    } else {
+      live = false;
+    }
     const bool neg = (u >> 31) != 0u;
 
     // c_k for every level k = 2^l: level l is complete after draw 2^l, i.e. levels 0..2 after the
     // first Philox call, level l >= 2 after call 2^(l-2)
     uint32_t cnt[kMaxLevels] = {0u, 0u, 0u, 0u, 0u, 0u, 0u};
-    if (live && m != 0u) {
-      const uint32_t T = m << 9;
+    if (live && thr != 0u) {
       const uint32_t i_lo = (uint32_t)index, i_hi = (uint32_t)(index >> 32);
       uint32_t rnd[4];
-      philox4x32_10(0u, layer_id, i_lo, i_hi, keys, rnd);
-      cnt[0] = rnd[0] < T ? 1u : 0u;
-      cnt[1] = cnt[0] + (rnd[1] < T ? 1u : 0u);
-      uint32_t c = cnt[1] + (rnd[2] < T ? 1u : 0u) + (rnd[3] < T ? 1u : 0u);
-      cnt[2] = c;
+      if (pbits == 0u) {
+        const uint32_t T = thr;
+        philox4x32_10(0u, layer_id, i_lo, i_hi, keys, rnd);
+        cnt[0] = rnd[0] < T ? 1u : 0u;
+        cnt[1] = cnt[0] + (rnd[1] < T ? 1u : 0u);
+        uint32_t c = cnt[1] + (rnd[2] < T ? 1u : 0u) + (rnd[3] < T ? 1u : 0u);
+        cnt[2] = c;
 #pragma unroll
-      for (int l = 3; l < kMaxLevels; ++l) {
-        if ((uint32_t)l <= max_level) {
-          for (uint32_t q = 1u << (l - 3); q < (1u << (l - 2)); ++q) {
-            philox4x32_10(q, layer_id, i_lo, i_hi, keys, rnd);
-            c += (rnd[0] < T ? 1u : 0u) + (rnd[1] < T ? 1u : 0u) + (rnd[2] < T ? 1u : 0u) + (rnd[3] < T ? 1u : 0u);
+        for (int l = 3; l < kMaxLevels; ++l) {
+          if ((uint32_t)l <= max_level) {
+            for (uint32_t q = 1u << (l - 3); q < (1u << (l - 2)); ++q) {
+              philox4x32_10(q, layer_id, i_lo, i_hi, keys, rnd);
+              c += (rnd[0] < T ? 1u : 0u) + (rnd[1] < T ? 1u : 0u) + (rnd[2] < T ? 1u : 0u) + (rnd[3] < T ? 1u : 0u);
+            }
+            cnt[l] = c;
           }
-          cnt[l] = c;
         }
+      } else if (deterministic) {
+#pragma unroll
+        for (int l = 0; l < kMaxLevels; ++l) cnt[l] = ((thr << l) + (1u << (pbits - 1u))) >> pbits;
+      } else {
+        // pbits-bit comparator, n = 32 / pbits draws per random word: bit j of `drawn` is draw j
+        const uint32_t n = 32u / pbits, per_call = 4u * n, fmask = (1u << pbits) - 1u, kmax = 1u << max_level;
+        unsigned long long drawn = 0ull;
+        for (uint32_t q = 0; q * per_call < kmax; ++q) {
+          philox4x32_10(q, layer_id, i_lo, i_hi, keys, rnd);
+#pragma unroll
+          for (int wd = 0; wd < 4; ++wd) {
+            uint32_t word = rnd[wd], bits = 0u;
+            for (uint32_t f = 0; f < n; ++f, word >>= pbits) bits |= ((word & fmask) < thr ? 1u : 0u) << f;
+            const uint32_t j0 = q * per_call + (uint32_t)wd * n;
+            if (j0 < 64u) drawn |= (unsigned long long)bits << j0;
+          }
+        }
+#pragma unroll
+        for (int l = 0; l < kMaxLevels; ++l)
+          cnt[l] = (uint32_t)__popcll(l == 6 ? drawn : drawn & ((1ull << (1u << l)) - 1ull));
       }
     }
 
@@ -222,7 +284,7 @@ __device__ __forceinline__ void sample_block(const SampleParams& p, uint32_t blo
 #pragma unroll
     for (int l = 0; l < kMaxLevels; ++l) {
       if (!((level_mask >> l) & 1u)) continue;
-      const uint32_t mag = live ? (((1u << l) + cnt[l]) << sh) : 0u;
+      const uint32_t mag = live ? (((base << l) + cnt[l]) << sh) : 0u;
       p.wint[l][wpos] = neg ? -(int32_t)mag : (int32_t)mag;
       if (track) {
         // lanes of a warp mostly share a row: one shared-memory add per row and warp
@@ -284,7 +346,7 @@ __global__ void __launch_bounds__(kThreads) emax_batch_kernel(const BatchEntry* 
   pdl_prologue();
   const BatchEntry& e = entries[find_entry(entries, n, blockIdx.x, true)];
   emax_block(e.p.w, e.p.O, e.p.d, e.p.norm, const_cast<uint32_t*>(e.p.e_max), err,
-             blockIdx.x - e.emax_first, e.emax_blocks, 0u, e.p.rowsum);
+             blockIdx.x - e.emax_first, e.emax_blocks, 0u, e.p.rowsum, e.p.pbits);
 }
 
 __global__ void __launch_bounds__(kThreads) sample_batch_kernel(const BatchEntry* __restrict__ entries, uint32_t n,
@@ -359,6 +421,9 @@ uint32_t fill_sample_params(const float* w_dev, const psb_weights* wt, uint32_t*
   p.norm = wt->cfg.norm;
   p.span = (1u << wt->cfg.exp_bits) - 1u;
   p.level_mask = wt->cfg.level_mask;
+  p.underflow = wt->cfg.underflow;
+  p.pbits = wt->cfg.prob_bits;
+  p.deterministic = wt->cfg.deterministic;
   p.max_level = 0;
   for (uint32_t l = 0; l < (uint32_t)kMaxLevels; ++l)
     if ((p.level_mask >> l) & 1u) p.max_level = l;
@@ -402,7 +467,7 @@ cudaError_t launch_sampler(const float* w_dev, psb_weights* wt, uint32_t* err_de
     wt->e_calls = 1u;
   }
   launch_pdl(emax_kernel, emax_blocks_for(O, wt->d, wt->cfg.norm), kThreads, 0, s, w_dev, O, wt->d, wt->cfg.norm,
-             wt->e_max, err_dev, wt->e_calls << 8, wt->rowsum256); note_launch();
+             wt->e_max, err_dev, wt->e_calls << 8, wt->rowsum256, wt->cfg.prob_bits); note_launch();
   SampleParams p;
   const uint32_t blocks = fill_sample_params(w_dev, wt, wt->e_max, p);
   p.e_tag = wt->e_calls;
@@ -580,6 +645,7 @@ extern "C" psb_status psb_sample_level_static(const float* w_dev, const psb_wsha
   if (log2k >= (uint32_t)kMaxLevels) return PSB_ERR_BAD_K;
   const uint32_t exp_bits = cfg->exp_bits ? cfg->exp_bits : 4u;
   if (exp_bits > 4 || cfg->norm > 1) return PSB_ERR_INVALID_ARG;
+  if (cfg->underflow || cfg->prob_bits || cfg->deterministic) return PSB_ERR_UNSUPPORTED;
   // the static scratch holds one word per output channel: larger filters are refused
   if (shape->out_ch > kStaticMaxOutCh) return PSB_ERR_UNSUPPORTED;
   const uint64_t d64 = (uint64_t)shape->in_ch_per_group * shape->kh * shape->kw;
@@ -605,12 +671,12 @@ extern "C" psb_status psb_sample_level_static(const float* w_dev, const psb_wsha
   // the array keeps the previous call's maxima: the reduction must start from zero
   if (cudaMemsetAsync(e_max, 0, sizeof(uint32_t) * O, s) != cudaSuccess) return PSB_ERR_CUDA;
   if (cfg->norm) {
-    emax_kernel<<<O, kThreads, 0, s>>>(w_dev, O, d, 1, e_max, err_sink, 0u, nullptr); note_launch();
+    emax_kernel<<<O, kThreads, 0, s>>>(w_dev, O, d, 1, e_max, err_sink, 0u, nullptr, 0u); note_launch();
   } else {
     size_t total = (size_t)O * d;
     uint32_t blocks = (uint32_t)((total + kThreads * 8 - 1) / (kThreads * 8));
     blocks = blocks < 1 ? 1 : (blocks > 1184 ? 1184 : blocks);
-    emax_kernel<<<blocks, kThreads, 0, s>>>(w_dev, O, d, 0, e_max, err_sink, 0u, nullptr); note_launch();
+    emax_kernel<<<blocks, kThreads, 0, s>>>(w_dev, O, d, 0, e_max, err_sink, 0u, nullptr, 0u); note_launch();
   }
   size_t total = (size_t)O * d;
   uint32_t blocks = (uint32_t)((total + kThreads - 1) / kThreads);

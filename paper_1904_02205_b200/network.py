@@ -11,9 +11,11 @@ from . import binding as B
 
 class Network:
     def __init__(self, ctx, layers, net, batch, level_mask, kmaps=None, uniform_log2k=3, fc_log2k=None,
-                 path=B.PSB_PATH_AUTO):
-        """layers/net: from workloads.build_network; kmaps: {resolution: u8 [batch, res, res]} or None."""
+                 path=B.PSB_PATH_AUTO, sample_opts=None):
+        """layers/net: from workloads.build_network; kmaps: {resolution: u8 [batch, res, res]} or None;
+        sample_opts: keyword options of Context.sample_weights (exp_bits, underflow, prob_bits, ...)."""
         self.ctx, self.layers, self.batch, self.level_mask, self.path = ctx, layers, batch, level_mask, path
+        self.sample_opts = dict(sample_opts or {})
         self.uniform_log2k = uniform_log2k
         self.fc_log2k = uniform_log2k if fc_log2k is None else fc_log2k
         dev = ctx.device
@@ -55,7 +57,7 @@ class Network:
             pr = self.params[l["name"]]
             self.weights[l["name"]] = self.ctx.sample_weights(
                 pr["w"], groups=l["groups"], seed=seed, layer_id=pr["p"]["layer_id"], level_mask=self.level_mask,
-                into=self.weights.get(l["name"]))
+                into=self.weights.get(l["name"]), **self.sample_opts)
         convs = [l["name"] for l in self.layers if l["op"] == "conv"]
         self._batch = self.ctx.sample_batch_create([self.params[n]["w"] for n in convs],
                                                    [self.weights[n] for n in convs])

@@ -5,10 +5,13 @@ import numpy as np
 
 def oracle_layer(orc, w, x, layout, groups, stride, pad, seed, layer_id, levels, kmap, uniform_log2k,
                  scale, bias, relu, inv_step, qmin, qmax, residual=None, res_scale=0.0, exp_bits=4,
-                 norm=0):
+                 norm=0, opts=None):
     Ws, eb = {}, None
     for l in levels:
-        Ws[l], eb, _ = orc.sample_level(w, seed, layer_id, l, exp_bits=exp_bits, norm=norm)
+        if opts:
+            Ws[l], eb = orc.sample_level_ex(w, seed, layer_id, l, exp_bits=exp_bits, norm=norm, **opts)[:2]
+        else:
+            Ws[l], eb, _ = orc.sample_level(w, seed, layer_id, l, exp_bits=exp_bits, norm=norm)
     lay = orc.NCHW if layout == 0 else orc.NHWC
     g = orc.geom(x.shape, lay, orc.U8 if x.dtype == np.uint8 else orc.S8, w.shape, groups, stride, pad)
     acc = orc.conv_acc(x, g, Ws, kmap=kmap, uniform_log2k=uniform_log2k)
@@ -19,7 +22,7 @@ def oracle_layer(orc, w, x, layout, groups, stride, pad, seed, layer_id, levels,
 
 def gpu_layer(psb, ctx, w, x, layout, groups, stride, pad, seed, layer_id, levels, kmap, uniform_log2k,
               scale, bias, relu, inv_step, qmin, qmax, out_dtype, residual=None, res_scale=0.0,
-              exp_bits=4, norm=0, in_max=0, path=0, guard=True, want=("q", "f32", "acc")):
+              exp_bits=4, norm=0, in_max=0, path=0, guard=True, want=("q", "f32", "acc"), opts=None):
     import torch
 
     dev = ctx.device
@@ -28,7 +31,7 @@ def gpu_layer(psb, ctx, w, x, layout, groups, stride, pad, seed, layer_id, level
     for l in levels:
         mask |= 1 << l
     wt = ctx.sample_weights(t(w), groups=groups, seed=seed, layer_id=layer_id, level_mask=mask,
-                            exp_bits=exp_bits, norm=norm)
+                            exp_bits=exp_bits, norm=norm, **(opts or {}))
     exported = {l: tuple(v.cpu().numpy() for v in ctx.weights_export(wt, l)) for l in levels}
     ctx.set_sample_map(None if kmap is None else t(kmap), uniform_log2k)
     O, KH, KW = w.shape[0], w.shape[2], w.shape[3]

@@ -39,14 +39,15 @@ def _layer_inputs(rng, N, C, H, W, O, KH, KW, groups, layout, x_dtype=np.uint8, 
 
 def _both(psb, ctx, oracle, w, x, layout, groups, stride, pad, levels, scale, bias, kmap=None,
           uniform=None, relu=True, inv_step=0.5, qmin=0, qmax=15, out_dtype=0, residual=None,
-          res_scale=0.0, exp_bits=4, norm=0, in_max=0, path=0, seed=5, layer_id=3, want=("q", "f32", "acc")):
+          res_scale=0.0, exp_bits=4, norm=0, in_max=0, path=0, seed=5, layer_id=3, want=("q", "f32", "acc"),
+          opts=None):
     uniform = levels[0] if uniform is None else uniform
     o = oracle_layer(oracle, w, x, layout, groups, stride, pad, seed, layer_id, levels, kmap, uniform,
                      scale, bias, relu, np.float32(inv_step), qmin, qmax, residual, np.float32(res_scale),
-                     exp_bits, norm)
+                     exp_bits, norm, opts=opts)
     g = gpu_layer(psb, ctx, w, x, layout, groups, stride, pad, seed, layer_id, levels, kmap, uniform,
                   scale, bias, relu, np.float32(inv_step), qmin, qmax, out_dtype, residual,
-                  np.float32(res_scale), exp_bits, norm, in_max, path, want=want)
+                  np.float32(res_scale), exp_bits, norm, in_max, path, want=want, opts=opts)
     compare(g, o, levels)
     return g
 
@@ -689,3 +690,70 @@ def test_tensor_path_codes_only_wide_accumulators(psb, ctx, oracle):
     g = _both(psb, ctx, oracle, w, x, 1, 1, 1, 1, [3], scale, bias, inv_step=0.008, qmax=255, in_max=127,
               path=psb.PSB_PATH_TENSOR, want=("q",))
     assert g["q"].max() > 0
+
+
+# ------------------------------------------- sampling options: gate below the window, b-bit probabilities
+
+@pytest.mark.parametrize("opts", [dict(underflow=1), dict(prob_bits=4), dict(prob_bits=6), dict(prob_bits=8),
+                                  dict(prob_bits=3, underflow=1), dict(prob_bits=4, deterministic=1),
+                                  dict(prob_bits=8, underflow=1, deterministic=1), dict(prob_bits=1)])
+@pytest.mark.parametrize("shape,groups,norm", [((64, 64, 3, 3), 1, 0), ((96, 1, 3, 3), 96, 1), ((130, 40, 1, 1), 1, 1),
+                                                ((16, 3, 7, 7), 1, 0)])
+def test_sampler_options_all_levels(psb, ctx, oracle, opts, shape, groups, norm):
+    """The Bernoulli gate at the window floor (Sec. 3.1) and probabilities on a grid with packed draws and the
+    deterministic variant (Sec. 4.4): integer filters of every level and base exponents against the oracle."""
+    import torch
+
+    rng = np.random.default_rng(abs(hash((shape, norm, tuple(sorted(opts.items()))))) % 2 ** 31)
+    w = (rng.normal(0, 0.1, size=shape) * 2.0 ** rng.integers(-9, 1, size=shape)).astype(np.float32)
+    flat = w.reshape(-1)
+    flat[rng.random(flat.size) < 0.05] = 0.0
+    flat[:6] = [0.5, -0.25, 1e-41, 3e-9, 0.99999994, -1.9999999]   # powers of two, sub-normal, tiny, p rounding to 1
+    for exp_bits in (4, 3, 2):
+        wt = ctx.sample_weights(torch.from_numpy(w).cuda(), groups=groups, seed=2 ** 41 + 3, layer_id=4,
+                                level_mask=0x7F, exp_bits=exp_bits, norm=norm, **opts)
+        for l in range(7):
+            Wg, ebg = (v.cpu().numpy() for v in ctx.weights_export(wt, l))
+            Wo, ebo = oracle.sample_level_ex(w, 2 ** 41 + 3, 4, l, exp_bits=exp_bits, norm=norm, **opts)[:2]
+            assert np.array_equal(ebg, ebo), (exp_bits, l)
+            assert np.array_equal(Wg.astype(np.int64), Wo), (shape, norm, exp_bits, l, opts)
+        assert ctx.device_status() == 0
+        wt.free()
+
+
+@pytest.mark.parametrize("exp_bits,opts", [(3, dict(underflow=1)), (2, dict(underflow=1)), (3, dict(underflow=1, prob_bits=4)),
+                                           (4, dict(prob_bits=4))])
+@pytest.mark.parametrize("case", [(2, 64, 14, 13, 80, 3, 1, 1), (3, 128, 9, 11, 64, 3, 1, 0), (2, 256, 9, 9, 128, 1, 0, 1),
+                                  (2, 3, 21, 21, 32, 7, 3, 1)])
+def test_layers_with_sampling_options(psb, ctx, oracle, exp_bits, opts, case):
+    """Whole layers under the sampling options, all outputs and codes only: narrow windows with the gate run
+    on two digit planes or one."""
+    N, C, H, W, O, K, pad, layout = case
+    rng = np.random.default_rng(abs(hash((case, exp_bits))) % 2 ** 31)
+    w, x, scale, bias = _layer_inputs(rng, N, C, H, W, O, K, K, 1, layout, x_hi=16 if C >= 32 else 256)
+    for want in (("q", "f32", "acc"), ("q",)):
+        g = _both(psb, ctx, oracle, w, x, layout, 1, 1, pad, [3], scale, bias, inv_step=0.5 if C >= 32 else 0.02,
+                  qmax=15 if C >= 32 else 255, exp_bits=exp_bits, in_max=15 if C >= 32 else 0,
+                  path=psb.PSB_PATH_TENSOR, want=want, opts=opts)
+        assert g["path"] == psb.PSB_PATH_TENSOR
+
+
+def test_depthwise_and_fc_with_sampling_options(psb, ctx, oracle):
+    rng = np.random.default_rng(61)
+    C = 48
+    w, x, scale, bias = _layer_inputs(rng, 2, C, 12, 10, C, 3, 3, C, 1, x_hi=256)
+    _both(psb, ctx, oracle, w, x, 1, C, 1, 1, [4], scale, bias, inv_step=0.03, qmax=255, exp_bits=3, want=("q",),
+          opts=dict(underflow=1, prob_bits=4))
+    w, x, scale, bias = _layer_inputs(rng, 16, 256, 1, 1, 128, 1, 1, 1, 1)
+    _both(psb, ctx, oracle, w, x, 1, 1, 1, 0, [2], scale, bias, inv_step=0.3, qmax=255, exp_bits=3, in_max=15,
+          path=psb.PSB_PATH_SHIFT_ADD, opts=dict(underflow=1))
+
+
+def test_bad_sampling_options_are_refused(psb, ctx):
+    import torch
+
+    w = torch.randn(16, 16, 1, 1, device=ctx.device)
+    for bad in (dict(prob_bits=9), dict(deterministic=1), dict(underflow=2)):
+        with pytest.raises(psb.PsbError) as e:
+            ctx.sample_weights(w, level_mask=1, **bad)
+        assert e.value.status == psb.PSB_ERR_INVALID_ARG

@@ -111,11 +111,12 @@ class ConvWorkload:
     name = "conv3x3_c64_56x56_b32_nchw"
     oracle_images = 16
 
-    def __init__(self, k, rank=0):
+    def __init__(self, k, rank=0, sample_opts=None):
         from workloads import config2_conv
 
         self.k = k
         self.log2k = int(np.log2(k))
+        self.sample_opts = dict(sample_opts or {})
         self.cfg = config2_conv(seed=1 + 100 * rank)
         self.macs = self.cfg["macs"]
         self.images = self.cfg["x"].shape[0]
@@ -129,7 +130,7 @@ class ConvWorkload:
         self.x_nhwc = self.x.permute(0, 2, 3, 1).contiguous()
         self.scale = torch.from_numpy(c["scale"]).to(dev)
         self.bias = torch.from_numpy(c["bias"]).to(dev)
-        self.wt = ctx.sample_weights(self.w, seed=c["seed"], layer_id=0, level_mask=1 << self.log2k)
+        self.wt = ctx.sample_weights(self.w, seed=c["seed"], layer_id=0, level_mask=1 << self.log2k, **self.sample_opts)
         ctx.set_sample_map(None, self.log2k)
         self.out = {"q": torch.empty((32, 64, 56, 56), dtype=torch.uint8, device=dev)}
         self.out_nhwc = {"q": torch.empty((32, 56, 56, 64), dtype=torch.uint8, device=dev)}
@@ -137,12 +138,13 @@ class ConvWorkload:
         self.x_host = torch.from_numpy(c["x"]).pin_memory()
         self.q_host = torch.empty((32, 64, 56, 56), dtype=torch.uint8).pin_memory()
         self.x_stage = torch.empty_like(self.x)
-        span = 15 + self.log2k + 2
+        span = (1 << self.sample_opts.get("exp_bits", 4)) - 1 + self.log2k + 2
         self.planes = (span + 6) // 7
 
     def step(self, i):
         c, psb = self.cfg, self.psb
-        self.ctx.sample_weights(self.w, seed=c["seed"] + i, layer_id=0, level_mask=1 << self.log2k, into=self.wt)
+        self.ctx.sample_weights(self.w, seed=c["seed"] + i, layer_id=0, level_mask=1 << self.log2k, into=self.wt,
+                                **self.sample_opts)
         self.ctx.conv2d(self.wt, self.x, psb.PSB_LAYOUT_NCHW, 1, 1, self.scale, self.bias, True,
                         c["inv_step"], 0, 15, in_max=15, out=self.out)
 
@@ -155,7 +157,8 @@ class ConvWorkload:
     def e2e_step(self, i):
         self.x_stage.copy_(self.x_host, non_blocking=True)
         c, psb = self.cfg, self.psb
-        self.ctx.sample_weights(self.w, seed=c["seed"] + i, layer_id=0, level_mask=1 << self.log2k, into=self.wt)
+        self.ctx.sample_weights(self.w, seed=c["seed"] + i, layer_id=0, level_mask=1 << self.log2k, into=self.wt,
+                                **self.sample_opts)
         self.ctx.conv2d(self.wt, self.x_stage, psb.PSB_LAYOUT_NCHW, 1, 1, self.scale, self.bias, True,
                         c["inv_step"], 0, 15, in_max=15, out=self.out)
         self.q_host.copy_(self.out["q"], non_blocking=True)
@@ -185,7 +188,7 @@ class ConvWorkload:
         c = self.cfg
         x = np.ascontiguousarray(c["x"][:n_images])
         t0 = time.perf_counter()
-        W, eb, _ = orc.sample_level(c["w"], c["seed"], 0, self.log2k)
+        W, eb = orc.sample_level_ex(c["w"], c["seed"], 0, self.log2k, **self.sample_opts)[:2]
         g = orc.geom(x.shape, orc.NCHW, orc.U8, c["w"].shape, 1, 1, 1)
         acc = orc.conv_acc(x, g, {self.log2k: W}, uniform_log2k=self.log2k)
         orc.epilogue(acc, g, c["scale"], c["bias"], eb, True, c["inv_step"], 0, 15, uniform_log2k=self.log2k)
@@ -267,10 +270,11 @@ class NetWorkload:
     """Network-shaped workloads: every conv / FC layer is a PSB layer, activations stay in HBM."""
     oracle_images = 1
 
-    def __init__(self, kind, k, rank=0, batch=0):
+    def __init__(self, kind, k, rank=0, batch=0, sample_opts=None):
         from workloads import mobilenetv2_layers, network_macs, resnet50_layers
 
         self.kind, self.k, self.rank = kind, k, rank
+        self.sample_opts = dict(sample_opts or {})
         self.log2k = int(np.log2(k))
         if kind == "mobilenetv2":
             self.layers, self.batch, self.qu, self.qs, self.prune, self.seed = mobilenetv2_layers(), batch or 64, 255, 127, 0.5, 3
@@ -294,7 +298,7 @@ class NetWorkload:
         self.kmaps = saliency_kmaps(self.batch, [112, 56, 28, 14, 7], self.seed) if self.adaptive else None
         mask = 0b11111 if self.adaptive else 1 << self.log2k
         self.nw = Network(ctx, self.layers, self.net, self.batch, mask, kmaps=self.kmaps, uniform_log2k=self.log2k,
-                          fc_log2k=4 if self.adaptive else None)
+                          fc_log2k=4 if self.adaptive else None, sample_opts=self.sample_opts)
         self.nw.sample(self.seed)
         self.image_host = torch.from_numpy(self.net["image"]).pin_memory()
         self.image_dev = self.image_host.to(ctx.device)
@@ -328,7 +332,7 @@ class NetWorkload:
     def roofline(self, _kernel_ms, peaks):
         """All launches of the tensor-core contraction in one forward pass, from per-layer events."""
         psb = self.psb
-        span_bits = 15 + (4 if self.adaptive else self.log2k) + 2
+        span_bits = (1 << self.sample_opts.get("exp_bits", 4)) - 1 + (4 if self.adaptive else self.log2k) + 2
         planes = (span_bits + 6) // 7
         t_ops, t_ms, s_ms, rows = 0.0, 0.0, 0.0, []
         for l in self.layers:
@@ -448,12 +452,23 @@ def default_run_extras(args, ctx, psb, torch, timed):
     return out
 
 
+def sample_options(args):
+    opts = {}
+    if args.exp_bits != 4:
+        opts["exp_bits"] = args.exp_bits
+    if args.underflow:
+        opts["underflow"] = 1
+    if args.prob_bits:
+        opts["prob_bits"] = args.prob_bits
+    return opts
+
+
 def make_workload(args, rank):
     if args.workload == "conv3x3":
-        return ConvWorkload(args.k, rank)
+        return ConvWorkload(args.k, rank, sample_options(args))
     if args.workload == "fc":
         return FcWorkload(args.k, rank)
-    return NetWorkload(args.workload, args.k, rank, batch=args.batch)
+    return NetWorkload(args.workload, args.k, rank, batch=args.batch, sample_opts=sample_options(args))
 
 
 # --------------------------------------------------------------------------- timing helpers
@@ -529,6 +544,9 @@ def main():
     ap.add_argument("--workload", default="conv3x3", choices=["conv3x3", "fc", "resnet50", "mobilenetv2", "resnet50_adaptive"])
     ap.add_argument("--k", type=int, default=8)
     ap.add_argument("--batch", type=int, default=0)
+    ap.add_argument("--exp-bits", type=int, default=4, help="octaves of the exponent window: 2^exp_bits (Sec. 4.4)")
+    ap.add_argument("--underflow", action="store_true", help="Bernoulli gate below the window instead of flushing (Sec. 3.1)")
+    ap.add_argument("--prob-bits", type=int, default=0, help="probabilities on a grid of 2^b points, packed draws (Sec. 4.4)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-extras", action="store_true",
                     help="default workload only: skip the draw-count sweep, the int8 probe and the network record")
@@ -628,7 +646,8 @@ def main():
     line = dict(metric=METRIC, value=value, unit=UNIT, n_gpus=world, steps=args.steps, warmup=args.warmup,
                 ms_per_step=sec * 1e3 / args.steps, higher_is_better=True, scaling="weak", vs_baseline=None,
                 dtype="int8 digits, int64 accumulators", data="synthetic",
-                config=dict(workload=wl.name, k=args.k, l2="flushed between steps (1 GiB memset, untimed)",
+                config=dict(workload=wl.name, k=args.k, sampling=sample_options(args) or "defaults",
+                            l2="flushed between steps (1 GiB memset, untimed)",
                             images_per_step=wl.images * world, sampler="inside the timed step, fresh seed per step"),
                 images_per_s=wl.images * world * args.steps / sec,
                 gated_add_equiv_per_s=units * getattr(wl, "mean_k", args.k) / sec,

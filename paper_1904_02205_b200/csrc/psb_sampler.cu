@@ -59,6 +59,63 @@ __device__ __forceinline__ void philox4x32_10(uint32_t c0, uint32_t c1, uint32_t
   philox4x32_10(c0, c1, c2, c3, key, out);
 }
 
+// Counts with a B-bit comparator (Sec. 4.4; supplement, "Stochastic multiplier"): draw j is bit field
+// (j mod n) of word ((j / n) mod 4) of Philox call j / (4 n), n = 32 / B; cnt[l] = ones among the first 2^l
+// draws.  Every index is a compile-time constant here, so the loops unroll into one extract / compare / add
+// per draw.
+template <int B>
+__device__ __forceinline__ void packed_counts(uint32_t thr, uint32_t max_level, uint32_t layer_id, uint32_t i_lo,
+                                              uint32_t i_hi, const PhiloxKeys& keys, uint32_t (&cnt)[kMaxLevels]) {
+  constexpr int n = 32 / B, per_call = 4 * n, calls = (64 + per_call - 1) / per_call;
+  const uint32_t kmax = 1u << max_level;
+  uint32_t c = 0;
+#pragma unroll
+  for (int q = 0; q < calls; ++q) {
+    if ((uint32_t)(q * per_call) < kmax) {
+      uint32_t rnd[4];
+      philox4x32_10((uint32_t)q, layer_id, i_lo, i_hi, keys, rnd);
+#pragma unroll
+      for (int wd = 0; wd < 4; ++wd) {
+#pragma unroll
+        for (int f = 0; f < n; ++f) {
+          constexpr uint32_t fmask = (1u << B) - 1u;
+          const int j = q * per_call + wd * n + f;
+          if (j < 64) {
+            c += ((rnd[wd] >> (f * B)) & fmask) < thr ? 1u : 0u;
+            if (((j + 1) & j) == 0) {           // j + 1 is a power of two: a level is complete
+              const int l = j + 1 == 1 ? 0 : j + 1 == 2 ? 1 : j + 1 == 4 ? 2 : j + 1 == 8 ? 3 : j + 1 == 16 ? 4 : j + 1 == 32 ? 5 : 6;
+              cnt[l] = c;
+            }
+          }
+        }
+      }
+    }
+  }
+}
+
+// The same for any width 1..8, indices at run time.
+__device__ __forceinline__ void packed_counts_any(uint32_t pbits, uint32_t thr, uint32_t max_level, uint32_t layer_id,
+                                               uint32_t i_lo, uint32_t i_hi, const PhiloxKeys& keys,
+                                               uint32_t (&cnt)[kMaxLevels]) {
+  const uint32_t n = 32u / pbits, per_call = 4u * n, fmask = (1u << pbits) - 1u, kmax = 1u << max_level;
+  unsigned long long drawn = 0ull;      // bit j = draw j
+  for (uint32_t q = 0; q * per_call < kmax && q * per_call < 64u; ++q) {
+    uint32_t rnd[4];
+    philox4x32_10(q, layer_id, i_lo, i_hi, keys, rnd);
+#pragma unroll
+    for (int wd = 0; wd < 4; ++wd) {
+      uint32_t word = rnd[wd];
+      unsigned long long bits = 0ull;
+      for (uint32_t f = 0; f < n; ++f, word >>= pbits) bits |= (unsigned long long)((word & fmask) < thr ? 1u : 0u) << f;
+      const uint32_t j0 = q * per_call + (uint32_t)wd * n;
+      if (j0 < 64u) drawn |= bits << j0;
+    }
+  }
+#pragma unroll
+  for (int l = 0; l < kMaxLevels; ++l)
+    cnt[l] = (uint32_t)__popcll(l == 6 ? drawn : drawn & ((1ull << (1u << l)) - 1ull));
+}
+
 // Division of a small number (< 2^16) by a block-uniform divisor (< 2^16): q = umulhi(t, magic)
 // with magic = floor((2^32 - 1) / d) + 1 is exact in that range.
 __device__ __forceinline__ uint32_t small_div_magic(uint32_t d) { return 0xFFFFFFFFu / d + 1u; }
@@ -252,22 +309,13 @@ __device__ __forceinline__ void sample_block(const SampleParams& p, uint32_t blo
 #pragma unroll
         for (int l = 0; l < kMaxLevels; ++l) cnt[l] = ((thr << l) + (1u << (pbits - 1u))) >> pbits;
       } else {
-        // pbits-bit comparator, n = 32 / pbits draws per random word: bit j of `drawn` is draw j
-        const uint32_t n = 32u / pbits, per_call = 4u * n, fmask = (1u << pbits) - 1u, kmax = 1u << max_level;
-        unsigned long long drawn = 0ull;
-        for (uint32_t q = 0; q * per_call < kmax; ++q) {
-          philox4x32_10(q, layer_id, i_lo, i_hi, keys, rnd);
-#pragma unroll
-          for (int wd = 0; wd < 4; ++wd) {
-            uint32_t word = rnd[wd], bits = 0u;
-            for (uint32_t f = 0; f < n; ++f, word >>= pbits) bits |= ((word & fmask) < thr ? 1u : 0u) << f;
-            const uint32_t j0 = q * per_call + (uint32_t)wd * n;
-            if (j0 < 64u) drawn |= (unsigned long long)bits << j0;
-          }
+        // pbits-bit comparator, n = 32 / pbits draws per random word
+        switch (pbits) {
+          case 4: packed_counts<4>(thr, max_level, layer_id, i_lo, i_hi, keys, cnt); break;
+          case 6: packed_counts<6>(thr, max_level, layer_id, i_lo, i_hi, keys, cnt); break;
+          case 8: packed_counts<8>(thr, max_level, layer_id, i_lo, i_hi, keys, cnt); break;
+          default: packed_counts_any(pbits, thr, max_level, layer_id, i_lo, i_hi, keys, cnt); break;
         }
-#pragma unroll
-        for (int l = 0; l < kMaxLevels; ++l)
-          cnt[l] = (uint32_t)__popcll(l == 6 ? drawn : drawn & ((1ull << (1u << l)) - 1ull));
       }
     }
 

@@ -176,14 +176,39 @@ psb_status run_layer(psb_ctx* ctx, const psb_weights* wt, const void* x_dev, uin
         if (wt->level[l].corr128 && (ctx->kmap || l == ctx->uniform_log2k))
           if (launch_corr128(wt, l, s) != cudaSuccess) return PSB_ERR_CUDA;
     }
+    SortedRows sorted;
     if (a.kmap) {
-      // one byte per row tile: strips of 128 locations, or 8 x 16 patches (a few more of them)
-      const size_t strips = ((size_t)a.N * a.OH * a.OW + 127) / 128;
-      const size_t patches = (size_t)((a.OW + 7) / 8) * (((size_t)a.OH * a.N + 15) / 16);
-      st = ensure_scratch(ctx, 2, strips > patches ? strips : patches);
+      // per-location draw counts: sort the locations by level (once per map), gather the activation rows in
+      // that order, contract the matrix with one level per tile, scatter the rows back in the output stage
+      const uint32_t tiles = sorted_tiles_bound(M);
+      const size_t ctl_bytes = (sort_ctl_bytes() + 255u) & ~(size_t)255u;
+      const size_t perm_bytes = (size_t)tiles * 128u * sizeof(uint32_t);
+      if (ctx->scratch_bytes[2] < ctl_bytes + perm_bytes + tiles) ctx->sorted_rows = 0;    // the buffer moves
+      st = ensure_scratch(ctx, 2, ctl_bytes + perm_bytes + tiles);
       if (st != PSB_OK) return st;
+      uint8_t* base = (uint8_t*)ctx->scratch[2];
+      uint32_t* perm = (uint32_t*)(base + ctl_bytes);
+      uint8_t* tile_mask = base + ctl_bytes + perm_bytes;
+      if (ctx->sorted_map != a.kmap || ctx->sorted_rows != (uint32_t)M) {
+        if (launch_level_sort(a.kmap, (uint32_t)M, base, perm, tile_mask, s) != cudaSuccess) return PSB_ERR_CUDA;
+        ctx->sorted_map = a.kmap;
+        ctx->sorted_rows = (uint32_t)M;
+      }
+      // the matrix: K index (kh * KW + kw) * cpad + ci, cpad = channel blocks of the filter's plane layout
+      const uint32_t cpad = wt->packed_k ? wt->n_cb * wt->bk : ((a.C + wt->bk - 1) / wt->bk) * wt->bk;
+      const size_t row_bytes = (size_t)a.KH * a.KW * cpad;
+      st = ensure_scratch(ctx, 3, (size_t)tiles * 128u * row_bytes);
+      if (st != PSB_OK) return st;
+      if (launch_gather_sorted(a, perm, base, cpad, (uint8_t*)ctx->scratch[3], s) != cudaSuccess) return PSB_ERR_CUDA;
+      a.x = ctx->scratch[3];
+      a.C = (uint32_t)row_bytes;
+      a.H = oh; a.W = ow;
+      a.KH = 1; a.KW = 1; a.stride = 1; a.pad = 0;
+      sorted.perm = perm;
+      sorted.tile_mask = tile_mask;
+      sorted.tiles = tiles;
     }
-    st = launch_tensor(ctx, wt, a, amax, add_corr, s);
+    st = launch_tensor(ctx, wt, a, amax, add_corr, a.kmap ? &sorted : nullptr, s);
     if (st != PSB_OK) return st;
     ctx->last_path = PSB_PATH_TENSOR;
     return PSB_OK;
@@ -242,7 +267,7 @@ psb_status psb_destroy(psb_ctx* ctx) {
   if (!ctx) return PSB_ERR_INVALID_ARG;
   cudaSetDevice(ctx->device);
   cudaDeviceSynchronize();
-  for (int i = 0; i < 3; ++i)
+  for (int i = 0; i < 4; ++i)
     if (ctx->scratch[i]) cudaFree(ctx->scratch[i]);
   if (ctx->err_dev) cudaFree(ctx->err_dev);
   for (int i = 0; i < psb_ctx::kTimedLaunches; ++i) {
@@ -401,6 +426,7 @@ psb_status psb_weights_free(psb_ctx* ctx, psb_weights* weights) {
 psb_status psb_set_sample_map(psb_ctx* ctx, const uint8_t* log2k_dev, uint32_t n, uint32_t oh,
                               uint32_t ow, uint32_t uniform_log2k) {
   if (!ctx) return PSB_ERR_INVALID_ARG;
+  ctx->sorted_rows = 0;      // whatever was derived from an earlier map is dropped
   if (log2k_dev) {
     if (!n || !oh || !ow) return PSB_ERR_INVALID_ARG;
     ctx->kmap = log2k_dev;
@@ -515,12 +541,19 @@ psb_status psb_run(psb_ctx* ctx, const psb_op* ops, uint32_t n_ops, void* stream
     psb_status st;
     switch (op.kind) {
       case PSB_OP_CONV2D:
-      case PSB_OP_GEMM:
+      case PSB_OP_GEMM: {
+        // within one list a map that several operations name is sorted by level once (the maps must not
+        // change while the list runs); psb_set_sample_map drops the sorted order, so it is kept across it
+        const uint8_t* kept_map = ctx->sorted_map;
+        const uint32_t kept_rows = i ? ctx->sorted_rows : 0u;
         st = psb_set_sample_map(ctx, op.map_dev, op.map_n, op.map_oh, op.map_ow, op.uniform_log2k);
         if (st != PSB_OK) return st;
+        ctx->sorted_map = kept_map;
+        ctx->sorted_rows = kept_rows;
         st = op.kind == PSB_OP_CONV2D ? psb_conv2d(ctx, op.weights, op.x_dev, &op.conv, stream)
                                       : psb_gemm(ctx, op.weights, op.x_dev, &op.gemm, stream);
         break;
+      }
       case PSB_OP_MAXPOOL:
         st = psb_maxpool2d_u8(ctx, (const uint8_t*)op.x_dev, op.conv.layout, op.conv.n, op.conv.c, op.conv.h,
                               op.conv.w, op.pool_k, op.conv.stride, op.conv.pad, op.pool_out_dev, stream);

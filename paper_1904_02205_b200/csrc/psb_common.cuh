@@ -85,8 +85,13 @@ struct psb_ctx {
   const uint8_t* kmap = nullptr;    // borrowed
   uint32_t map_n = 0, map_oh = 0, map_ow = 0;
   uint32_t uniform_log2k = 0;
-  void* scratch[3] = {nullptr, nullptr, nullptr};   // layout conversion buffers
-  size_t scratch_bytes[3] = {0, 0, 0};
+  // scratch: [0] layout conversion, [1] gathered / offset activation matrix, [2] level-sorted order of the
+  // current draw-count map (control block, permutation, tile levels), [3] activation rows in that order
+  void* scratch[4] = {nullptr, nullptr, nullptr, nullptr};
+  size_t scratch_bytes[4] = {0, 0, 0, 0};
+  // the sorted order in scratch[2] belongs to this map (pointer and dimensions); 0 rows = none
+  const uint8_t* sorted_map = nullptr;
+  uint32_t sorted_rows = 0;
   int32_t last_path = 0;
   int sm_count = 0;
   unsigned long long wait_limit_cycles = psb::kDefaultWaitLimitCycles;   // bound of every device-side wait
@@ -237,8 +242,22 @@ cudaError_t launch_avgpool(const uint8_t* x, uint32_t nchw, uint32_t N, uint32_t
                            cudaStream_t s);
 // tensor path: returns PSB_ERR_UNSUPPORTED if the shape does not fit it
 psb_status tensor_supported(const psb_ctx* ctx, const psb_weights* wt, const ConvArgs& a);
+// sorted != null: the activation matrix is in level-sorted row order (psb_sort.cu)
+struct SortedRows {
+  const uint32_t* perm;       // [tiles * 128] location of every sorted row, 0xFFFFFFFF = padding
+  const uint8_t* tile_mask;   // [tiles] the level of every tile as a one-bit mask (0 = unused tile)
+  uint32_t tiles;             // upper bound of the tiles in use
+};
 psb_status launch_tensor(psb_ctx* ctx, const psb_weights* wt, const ConvArgs& a, uint32_t amax,
-                         bool add_corr128, cudaStream_t s);
+                         bool add_corr128, const SortedRows* sorted, cudaStream_t s);
+
+// level-sorted rows for draw-count maps (psb_sort.cu)
+size_t sort_ctl_bytes();
+uint32_t sorted_tiles_bound(uint64_t M);
+cudaError_t launch_level_sort(const uint8_t* kmap, uint32_t M, void* ctl, uint32_t* perm, uint8_t* tile_mask,
+                              cudaStream_t s);
+cudaError_t launch_gather_sorted(const ConvArgs& a, const uint32_t* perm, const void* ctl, uint32_t cpad, uint8_t* dst,
+                                 cudaStream_t s);
 
 // int8 tensor-core issue-rate probe (psb_probe.cu)
 psb_status int8_mma_probe(psb_ctx* ctx, uint32_t n_cols, uint32_t groups, double* mac_per_clk_per_sm,

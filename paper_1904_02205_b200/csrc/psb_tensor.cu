@@ -21,8 +21,9 @@
 //   warps 4-19 epilogue: TMEM -> registers, recombine planes, dequantise, bias,
 //            shortcut, ReLU, re-quantise, vectorised stores; overlaps the next
 //            tile's MMAs through two TMEM accumulator buffers
-// Per-location draw counts (Sec. 4.5): a tile is contracted once per level present
-// among its 128 rows; the epilogue of each pass stores only the rows of that level.
+// Per-location draw counts (Sec. 4.5): the caller sorts the output locations by level and
+// gathers the activation rows in that order (psb_sort.cu); every tile then has one level, and
+// the epilogue scatters each row back to its location.
 // Every wait is bounded; on a timeout the kernel raises the device error word and
 // leaves through the common exit that frees TMEM.
 #include <cuda.h>
@@ -86,12 +87,9 @@ struct TensorParams {
   uint32_t tpi;         // tiles per image: ceil(OH * Wp / 128)
   uint32_t band_rows;   // padded input rows per band
   uint32_t band_bytes;  // stage size (band_rows * Wp * C rounded up to 1024)
-  // Patch mode (plain GEMM layers under a per-location map): a tile is a patch of 8 x 16 locations
-  // (x by y, y running over the rows of all images) instead of a strip of 128 consecutive ones, so
-  // that fewer levels of a smooth map meet in one tile; one 3-D tiled copy per K block.  Row r of the
-  // tile is location (tx * 8 + r % 8, ty * 16 + r / 8).  Used where the image width is a multiple of 8.
-  uint32_t patch;       // 1: patch mode
-  uint32_t tiles_x;     // patches per image row: ceil(OW / 8)
+  // Per-location draw counts: the rows of the activation matrix are sorted by level (psb_sort.cu), every tile
+  // has one level (tile_mask holds one bit), and row r of the matrix is output location perm[r]
+  const uint32_t* perm;  // or null
   uint32_t Wp_magic, tpi_magic;   // ceil(2^32 / Wp), ceil(2^32 / tpi): quotients by multiply-high (exact in the
                                   // ranges band mode is restricted to)
   unsigned long long wait_limit;  // bound of every wait in SM clocks
@@ -172,14 +170,6 @@ __device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_
   asm volatile(
       "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
       ::"r"(dst), "l"(src), "r"(bytes), "r"(bar)
-      : "memory");
-}
-
-__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c, int x, int y) {
-  asm volatile(
-      "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes"
-      " [%0], [%1, {%3, %4, %5}], [%2];"
-      ::"r"(dst), "l"(map), "r"(bar), "r"(c), "r"(x), "r"(y)
       : "memory");
 }
 
@@ -283,40 +273,11 @@ __device__ __forceinline__ uint32_t smem_desc_hi(uint32_t bk) {
   return ((8u * bk) >> 4) | (1u << 14) | (layout << 29);
 }
 
-// Levels (log2 k) present among the 128 rows of a tile, as a bit mask: one byte per row tile,
-// written by tile_levels_kernel just before the contraction kernel.
+// Levels (log2 k) of a tile as a bit mask: one byte per row tile, written by the level sort just before the
+// contraction kernel (rows are sorted by level, so exactly one bit is set).
 __device__ __forceinline__ uint32_t tile_levels(const TensorParams& p, uint32_t m_tile) {
   if (!p.tile_mask) return 1u << p.a.uniform_log2k;
   return (uint32_t)p.tile_mask[m_tile];
-}
-
-constexpr uint32_t kPatchW = 8, kPatchH = kTileM / kPatchW;
-
-// Linear location index of row `row` of patch `m_tile` (rows of all images stacked: y < rows_all), and
-// whether it is a real location.
-__device__ __forceinline__ uint32_t patch_row_index(uint32_t m_tile, uint32_t row, uint32_t tiles_x, uint32_t OW,
-                                                    uint32_t rows_all, bool* valid) {
-  const uint32_t ty = m_tile / tiles_x, tx = m_tile - ty * tiles_x;
-  const uint32_t x = tx * kPatchW + (row % kPatchW), y = ty * kPatchH + row / kPatchW;
-  *valid = x < OW && y < rows_all;
-  return y * OW + x;
-}
-
-__global__ void tile_levels_kernel(const uint8_t* __restrict__ kmap, uint32_t M, uint32_t m_tiles,
-                                   uint8_t* __restrict__ tile_mask, uint32_t patch_tiles_x, uint32_t OW,
-                                   uint32_t rows_all) {
-  const uint32_t tile = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31u;
-  if (tile >= m_tiles) return;
-  uint32_t mask = 0;
-#pragma unroll
-  for (int r = 0; r < 4; ++r) {
-    uint32_t m = tile * kTileM + r * 32u + lane;
-    bool ok = m < M;
-    if (patch_tiles_x) m = patch_row_index(tile, r * 32u + lane, patch_tiles_x, OW, rows_all, &ok);
-    if (ok) mask |= 1u << min((uint32_t)kmap[m], 7u);   // levels >= 7 are invalid: bit 7, flagged by the epilogue
-  }
-  mask = __reduce_or_sync(0xFFFFFFFFu, mask);
-  if (lane == 0) tile_mask[tile] = (uint8_t)mask;
 }
 
 // Walks the tiles of this CTA without divisions in the loop.  Resident mode: the CTA owns one
@@ -584,8 +545,18 @@ __device__ __noinline__ void epilogue_chunk(const TensorParams& p, uint32_t tadd
 __device__ __forceinline__ bool uniform_epilogue(const TensorParams& p) {
   const ConvArgs& a = p.a;
   const bool q_only = a.q_out && !a.f32_out && !a.acc_out && (p.vec_ok || a.out_nchw) && a.inv_step > 0.0f;
+  if (a.kmap) {
+    // rows sorted by level: the same loop serves if every sampled level has the same number of digit planes
+    uint32_t P0 = 0;
+    for (uint32_t lv = 0; lv < (uint32_t)kMaxLevels; ++lv)
+      if ((a.level_mask >> lv) & 1u) {
+        if (P0 && p.planes[lv] != P0) return false;
+        P0 = p.planes[lv];
+      }
+    return p.perm && q_only && P0 >= 2u && P0 <= 4u;
+  }
   const uint32_t P0 = p.planes[a.uniform_log2k < (uint32_t)kMaxLevels ? a.uniform_log2k : 0u];
-  return !a.kmap && q_only && P0 >= 2u && P0 <= 4u;
+  return q_only && P0 >= 2u && P0 <= 4u;
 }
 
 // Linear output index (n * OH + oy) * OW + ox of row `row` of row tile `m_tile`, and whether the
@@ -661,6 +632,26 @@ __device__ __forceinline__ bool fits_32_bits(const TensorParams& p, uint32_t l) 
   return (unsigned long long)best * 256ull * (unsigned long long)p.amax < (1ull << 31) && best < (1u << 24);
 }
 
+// Rows sorted by level (per-location draw counts): row r of the matrix is location perm[r].
+struct RowMapSorted {
+  static constexpr int kTag = 2;
+  const uint32_t* perm;
+  uint32_t O, ohow, planar;
+  __device__ __forceinline__ void init(const TensorParams& p) {
+    perm = p.perm; O = p.a.O; ohow = p.a.OH * p.a.OW; planar = p.a.out_nchw;
+  }
+  __device__ __forceinline__ uint32_t row_index(uint32_t m_tile, uint32_t row, bool* valid) const {
+    const uint32_t m = __ldg(perm + (size_t)m_tile * kTileM + row);
+    *valid = m != 0xFFFFFFFFu;
+    return m;
+  }
+  __device__ __forceinline__ size_t offset(uint32_t m, uint32_t o_base) const {
+    if (!planar) return (size_t)m * O + o_base;
+    const uint32_t n = m / ohow;
+    return ((size_t)n * O + o_base) * ohow + (m - n * ohow);
+  }
+};
+
 // Epilogue loop of one warp for the common case: one draw count for the whole layer, only
 // re-quantised bytes wanted.  The warp owns 32 rows (its TMEM lane quarter) x 16 channels of
 // every tile.  Per tile: wait for the accumulator, pull the chunk into registers, hand the TMEM
@@ -676,8 +667,9 @@ __device__ __noinline__ bool epilogue_uniform(const TensorParams& p, SharedCtl* 
   const ConvArgs& a = p.a;
   const uint32_t quarter = ew & 3u, sub = ew >> 2;
   const uint32_t row = quarter * 32u + lane;
-  const uint32_t l = a.uniform_log2k;
-  const bool use_corr = p.corr[l] != nullptr;
+  constexpr bool kSorted = RM::kTag == 2;      // one level per tile, taken from the tile's mask
+  uint32_t l = a.uniform_log2k;
+  const bool use_corr = p.corr[kSorted ? (uint32_t)__ffs((int)(a.level_mask & 0x7Fu)) - 1u : l] != nullptr;
   WaitCtl* abort = &ctl->wait;
   const uint8_t* const res_base = (const uint8_t*)a.residual;
   uint8_t* const q_base = (uint8_t*)a.q_out;
@@ -705,8 +697,27 @@ __device__ __noinline__ bool epilogue_uniform(const TensorParams& p, SharedCtl* 
     const uint32_t o_tile = ti.o_tile;
     const uint32_t o_base = o_tile * kTileN + sub * 16u;
     const bool active = o_base < rm.O;          // warp-uniform
+    if (kSorted) {
+      // the tile's level; a tile without a sampled level gets no pass from the other roles either
+      const uint32_t levels = tile_levels(p, ti.m_tile);
+      if (!(levels & a.level_mask & 0x7Fu)) {
+        if (row_valid) atomicOr(a.err, kDevErrBadLevel);     // a location asks for a level that was not sampled
+        ti.next();
+        if (HAS_RES && ti.valid()) {
+          bool ok_row;
+          const uint32_t mn = rm.row_index(ti.m_tile, row, &ok_row), ob = ti.o_tile * kTileN + sub * 16u;
+          r_next = make_uint4(0, 0, 0, 0);
+          if (ok_row && ob < rm.O) {
+            const uint8_t* src = res_base + rm.offset(mn, ob);
+            r_next = planar ? load_planar16<TAG>(src, ohow, rm.O - ob) : load_row16(src, vec16, ob + 16u <= rm.O);
+          }
+        }
+        continue;
+      }
+      l = (uint32_t)__ffs((int)(levels & a.level_mask & 0x7Fu)) - 1u;
+    }
     ti.next();
-    if (o_tile != cur_o_tile) {
+    if ((kSorted ? o_tile * 8u + l : o_tile) != cur_o_tile) {
       // per-channel constants of this channel tile: the warp keeps its own copy of its 16 channels
       __syncwarp();
       if (lane < 16u) {
@@ -721,7 +732,7 @@ __device__ __noinline__ bool epilogue_uniform(const TensorParams& p, SharedCtl* 
         ctl->scb[ew][lane] = sb;
         ctl->corr[ew][lane] = cr;
       }
-      cur_o_tile = o_tile;
+      cur_o_tile = kSorted ? o_tile * 8u + l : o_tile;
       __syncwarp();
     }
     const uint4 r_cur = r_next;
@@ -765,6 +776,9 @@ __device__ __forceinline__ bool uniform_dispatch_tail(const TensorParams& p, Sha
   if (p.band)
     return fast_u8 ? epilogue_uniform<P, W32, RES, true, RowMapBand>(p, ctl, tmem_base, ew, lane, c)
                    : epilogue_uniform<P, W32, RES, false, RowMapBand>(p, ctl, tmem_base, ew, lane, c);
+  if (p.perm)
+    return fast_u8 ? epilogue_uniform<P, W32, RES, true, RowMapSorted>(p, ctl, tmem_base, ew, lane, c)
+                   : epilogue_uniform<P, W32, RES, false, RowMapSorted>(p, ctl, tmem_base, ew, lane, c);
   return fast_u8 ? epilogue_uniform<P, W32, RES, true, RowMap>(p, ctl, tmem_base, ew, lane, c)
                  : epilogue_uniform<P, W32, RES, false, RowMap>(p, ctl, tmem_base, ew, lane, c);
 }
@@ -1090,9 +1104,6 @@ psb_mma_kernel(const __grid_constant__ TmapSet maps, const __grid_constant__ Ten
               const uint32_t dst = ring_addr + s * stage_bytes + lane * sub_bytes;
               if (p.im2col)
                 tma_load_im2col_4d(dst, &maps.a, bar, (int)(cb * BK), w0, h0, (int)n0, (uint16_t)kw, (uint16_t)kh);
-              else if (p.patch)
-                tma_load_3d(dst, &maps.a, bar, (int)(cb * BK), (int)((m_tile % p.tiles_x) * kPatchW),
-                            (int)((m_tile / p.tiles_x) * kPatchH));
               else
                 tma_load_2d(dst, &maps.a, bar, (int)(cb * BK), (int)m0);
               if (!p.resident) bulk_load(dst + p.stage_bytes_a, b_tiles + (size_t)kb * blk, blk, bar);
@@ -1133,7 +1144,8 @@ psb_mma_kernel(const __grid_constant__ TmapSet maps, const __grid_constant__ Ten
     // unsigned codes from 0 up: the byte saturation of the packing instruction is the lower clamp
     const bool fast_u8 = a.out_dtype == PSB_DT_U8 && a.qmin == 0;
     const uint32_t res_kind = !a.residual ? 0u : (a.residual_dtype == PSB_DT_S8 ? 2u : 1u);
-    const uint32_t P0 = p.planes[a.uniform_log2k < (uint32_t)kMaxLevels ? a.uniform_log2k : 0u];
+    uint32_t P0 = p.planes[a.uniform_log2k < (uint32_t)kMaxLevels ? a.uniform_log2k : 0u];
+    if (a.kmap) P0 = p.planes[(uint32_t)__ffs((int)(a.level_mask & 0x7Fu)) - 1u];
     if (p.resident && lane == 0) {
       // the digit planes of this CTA's channel tile, all K blocks, once: the epilogue warps have
       // nothing else to do yet, and sixteen threads get the copies under way sooner than one
@@ -1148,7 +1160,13 @@ psb_mma_kernel(const __grid_constant__ TmapSet maps, const __grid_constant__ Ten
       }
     }
     if (uniform_epilogue(p)) {
-      const bool w32 = fits_32_bits(p, a.uniform_log2k);
+      bool w32 = true;
+      if (a.kmap) {          // every level a tile may have must fit
+        for (uint32_t lv = 0; lv < (uint32_t)kMaxLevels; ++lv)
+          if ((a.level_mask >> lv) & 1u) w32 = fits_32_bits(p, lv) && w32;
+      } else {
+        w32 = fits_32_bits(p, a.uniform_log2k);
+      }
       if (P0 == 4u) failed = uniform_dispatch<4>(p, ctl, tmem_base, ew, lane, ec, fast_u8, w32, res_kind);
       else if (P0 == 3u) failed = uniform_dispatch<3>(p, ctl, tmem_base, ew, lane, ec, fast_u8, w32, res_kind);
       else failed = uniform_dispatch<2>(p, ctl, tmem_base, ew, lane, ec, fast_u8, w32, res_kind);
@@ -1167,7 +1185,10 @@ psb_mma_kernel(const __grid_constant__ TmapSet maps, const __grid_constant__ Ten
         const uint32_t levels = tile_levels(p, ti.m_tile) & a.level_mask;
         uint32_t m = m0 + row;
         bool in_range = m < p.M;
-        if (p.patch) m = patch_row_index(ti.m_tile, row, p.tiles_x, a.OW, a.OH * a.N, &in_range);
+        if (p.perm) {           // rows sorted by level: the location of this row
+          m = p.perm[m0 + row];
+          in_range = m != 0xFFFFFFFFu;
+        }
         const uint32_t my_level = in_range ? (a.kmap ? (uint32_t)a.kmap[m] : a.uniform_log2k) : 0xFFu;
         if (in_range && (my_level >= (uint32_t)kMaxLevels || !((a.level_mask >> my_level) & 1u)))
           atomicOr(a.err, kDevErrBadLevel);
@@ -1331,7 +1352,7 @@ psb_status tensor_supported(const psb_ctx* ctx, const psb_weights* wt, const Con
 }
 
 psb_status launch_tensor(psb_ctx* ctx, const psb_weights* wt, const ConvArgs& a, uint32_t amax,
-                         bool add_corr128, cudaStream_t s) {
+                         bool add_corr128, const SortedRows* sorted, cudaStream_t s) {
   TmapSet maps;
   TensorParams p;
   p.a = a;
@@ -1362,14 +1383,12 @@ psb_status launch_tensor(psb_ctx* ctx, const psb_weights* wt, const ConvArgs& a,
   p.vec_ok = 0u;
   if (!a.out_nchw && a.O % 16u == 0u && !(out_ptrs & 15u)) p.vec_ok = 2u;
   else if (!a.out_nchw && a.O % 8u == 0u && !(out_ptrs & 7u)) p.vec_ok = 1u;
-  p.patch = 0;
-  p.tiles_x = 0;
-  // (image widths that are not a multiple of the patch width would compute dropped columns: at 28, 14
-  // and 7 that costs what the fewer levels per tile save, so those keep strips)
-  if (a.kmap && !p.im2col && !a.out_nchw && a.OW % kPatchW == 0u) {
-    p.patch = 1;
-    p.tiles_x = (a.OW + kPatchW - 1) / kPatchW;
-    p.m_tiles = p.tiles_x * ((a.OH * a.N + kPatchH - 1) / kPatchH);
+  p.perm = nullptr;
+  if (a.kmap) {
+    // the caller has sorted the rows by level and gathered the matrix in that order
+    if (!sorted || p.im2col) return PSB_ERR_INVALID_ARG;
+    p.perm = sorted->perm;
+    p.m_tiles = sorted->tiles;
   }
   if (!a.kmap) {
     const uint32_t P = p.planes[a.uniform_log2k];
@@ -1455,17 +1474,8 @@ psb_status launch_tensor(psb_ctx* ctx, const psb_weights* wt, const ConvArgs& a,
                    lower, upper, bk, kTileM, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, swz,
                    CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
       return PSB_ERR_CUDA;
-  } else if (p.patch) {
-    cuuint64_t dims[3] = {a.C, a.W, (cuuint64_t)a.H * a.N};
-    cuuint64_t strides[2] = {(cuuint64_t)a.C, (cuuint64_t)a.C * a.W};
-    cuuint32_t box[3] = {bk, kPatchW, kPatchH};
-    cuuint32_t estr[3] = {1, 1, 1};
-    if (enc_tiled(&maps.a, CU_TENSOR_MAP_DATA_TYPE_UINT8, 3, const_cast<void*>(a.x), dims, strides, box, estr,
-                  CU_TENSOR_MAP_INTERLEAVE_NONE, swz, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
-                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
-      return PSB_ERR_CUDA;
   } else {
-    cuuint64_t dims[2] = {a.C, p.M};
+    cuuint64_t dims[2] = {a.C, a.kmap ? (cuuint64_t)p.m_tiles * kTileM : (cuuint64_t)p.M};
     cuuint64_t strides[1] = {(cuuint64_t)a.C};
     cuuint32_t box[2] = {bk, kTileM};
     cuuint32_t estr[2] = {1, 1};
@@ -1476,16 +1486,7 @@ psb_status launch_tensor(psb_ctx* ctx, const psb_weights* wt, const ConvArgs& a,
   }
   for (int l = 0; l < kMaxLevels; ++l) p.planes_ptr[l] = wt->level[l].planes;
 
-  p.tile_mask = nullptr;
-  if (a.kmap) {
-    // the caller has sized the third scratch buffer for one byte per row tile
-    if (!ctx->scratch[2] || ctx->scratch_bytes[2] < p.m_tiles) return PSB_ERR_INVALID_ARG;
-    tile_levels_kernel<<<(p.m_tiles * 32u + 255u) / 256u, 256, 0, s>>>(a.kmap, p.M, p.m_tiles,
-                                                                      (uint8_t*)ctx->scratch[2],
-                                                                      p.patch ? p.tiles_x : 0u, a.OW, a.OH * a.N);
-    note_launch();
-    p.tile_mask = (const uint8_t*)ctx->scratch[2];
-  }
+  p.tile_mask = a.kmap ? sorted->tile_mask : nullptr;
   const uint32_t n_tiles = p.m_tiles * p.o_tiles;
   const uint32_t grid = p.resident ? p.o_tiles * p.ctas_per_otile
                                    : (n_tiles < (uint32_t)ctx->sm_count ? n_tiles : (uint32_t)ctx->sm_count);

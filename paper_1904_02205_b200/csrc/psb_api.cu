@@ -215,7 +215,7 @@ psb_status run_layer(psb_ctx* ctx, const psb_weights* wt, const void* x_dev, uin
   }
   WintTable tab;
   for (int l = 0; l < kMaxLevels; ++l) tab.w[l] = wt->level[l].wint;
-  if (launch_shift_add(a, tab, s) != cudaSuccess) return PSB_ERR_CUDA;
+  if (launch_shift_add(a, tab, wt->rowsum256, amax, s) != cudaSuccess) return PSB_ERR_CUDA;
   ctx->last_path = PSB_PATH_SHIFT_ADD;
   return PSB_OK;
 }
@@ -373,8 +373,7 @@ psb_status psb_sample_weights(psb_ctx* ctx, const float* w_dev, const psb_wshape
     w->n_kb = w->packed_k ? w->n_cb : shape->kh * shape->kw * w->n_cb;
     bool ok = cudaMalloc(&w->e_base, sizeof(int32_t) * shape->out_ch) == cudaSuccess &&
               cudaMalloc(&w->e_max, sizeof(uint32_t) * shape->out_ch) == cudaSuccess &&
-              (!w->has_planes ||
-               cudaMalloc(&w->rowsum256, sizeof(uint32_t) * kMaxLevels * shape->out_ch) == cudaSuccess) &&
+              cudaMalloc(&w->rowsum256, sizeof(uint32_t) * kMaxLevels * shape->out_ch) == cudaSuccess &&
               cudaMemsetAsync(w->e_max, 0, sizeof(uint32_t) * shape->out_ch, s) == cudaSuccess;
     for (uint32_t l = 0; ok && l < (uint32_t)kMaxLevels; ++l) {
       if (!((cfg.level_mask >> l) & 1u)) continue;

@@ -75,7 +75,7 @@ struct psb_weights {
   uint32_t e_calls = 0;        // sampling calls made on this handle, modulo 2^24
   uint32_t* rowsum256 = nullptr;  // [kMaxLevels][O] row sums of |W_k| of the last sampling, in units of 256 (each
                                   // weight rounded up): the contraction derives from them whether its accumulators
-                                  // fit 32 bits; kept for filters with digit planes only
+                                  // fit 32 bits
   int device;
 };
 
@@ -218,7 +218,9 @@ psb_status sample_batch_run(psb_ctx* ctx, psb_sample_batch* b, uint64_t seed, cu
 void sample_batch_free(psb_sample_batch* b);
 cudaError_t launch_export(const psb_weights* wt, uint32_t level, int32_t* wint_out,
                           int32_t* e_base_out, cudaStream_t s);
-cudaError_t launch_shift_add(const ConvArgs& a, const WintTable& wt, cudaStream_t s);
+// rowsum256: [level][O] row sums of |W_k| / 256 kept by the sampler; amax: largest activation magnitude
+cudaError_t launch_shift_add(const ConvArgs& a, const WintTable& wt, const uint32_t* rowsum256, uint32_t amax,
+                             cudaStream_t s);
 // gathers [M][kpad] signed bytes (x - offset; zero padding becomes -offset, K padding 0); row kh of the
 // filter window occupies bytes [kh * run_pitch, kh * run_pitch + kw * c) of a matrix row
 cudaError_t launch_im2col_s8(const ConvArgs& a, uint32_t kpad, uint32_t run_pitch, uint32_t offset, int8_t* dst,

@@ -20,7 +20,7 @@ namespace {
 
 constexpr int kThreads = 256;
 constexpr int kStage = 2048;  // weights staged in shared memory per block
-constexpr int kRowSumRows = 128;   // filter rows per block for which the sampler keeps sums of |W_k|
+constexpr int kRowSumRows = 256;   // filter rows per block for which the sampler keeps sums of |W_k|
 
 // Philox4x32-10 (Salmon et al., SC'11): ten rounds of two 32x32->64 multiplies and
 // xors; the key advances by the two Weyl constants after every round.  The ten round keys

@@ -275,6 +275,131 @@ __global__ void __launch_bounds__(256, 2) dwconv3x3_row_kernel(const ConvArgs a,
   }
 }
 
+// The same layer class with the arithmetic cut down to what the bytes need.  The integer sum x * W_k over the
+// nine taps (Eq. 9 summed over the draws) fits 32 bits whenever (largest activation) x (sum of |W_k| of the
+// channel) stays below 2^31; the sampler keeps those sums, so a thread knows per channel whether 32-bit
+// multiply-adds are exact and falls back to 64-bit ones where they are not.  A thread owns 4 channels and kOut
+// consecutive outputs of one row and works channel by channel: the bytes of the 3 x kCols input words are
+// extracted once per row and channel and serve up to three outputs each, one multiply-add per tap; the output
+// stage is dequant()/requant() with conversion-unit instructions (one int -> float, one float -> int, both
+// round to nearest even as the definitions ask).  About 20 instructions per output where the 64-bit kernel
+// above needs about 70.
+template <typename Acc>
+__device__ __forceinline__ float dw_acc_to_float(Acc acc);
+template <>
+__device__ __forceinline__ float dw_acc_to_float<int>(int acc) { return __int2float_rn(acc); }
+template <>
+__device__ __forceinline__ float dw_acc_to_float<long long>(long long acc) { return acc_to_float(acc); }
+
+template <int S, bool kSignedIn, typename Acc>
+__device__ __forceinline__ void dw_channel(const uint32_t (&raw)[3][DwSeg<S>::kCols], int j, const int32_t* __restrict__ wch,
+                                           float sc, float bi, bool has_res, const uint32_t (&rv)[DwSeg<S>::kOut],
+                                           bool res_signed, float res_scale, float relu_floor, float inv_step,
+                                           float lo_f, float hi_f, uint32_t n_out, uint32_t (&qw)[DwSeg<S>::kOut]) {
+  constexpr int L = DwSeg<S>::kOut, NC = DwSeg<S>::kCols;
+  Acc acc[L];
+#pragma unroll
+  for (int i = 0; i < L; ++i) acc[i] = 0;
+#pragma unroll
+  for (int r = 0; r < 3; ++r) {
+    const int w0 = __ldg(wch + r * 3), w1 = __ldg(wch + r * 3 + 1), w2 = __ldg(wch + r * 3 + 2);
+    int xb[NC];
+#pragma unroll
+    for (int cidx = 0; cidx < NC; ++cidx) {
+      const uint32_t b = (raw[r][cidx] >> (8 * j)) & 0xFFu;
+      xb[cidx] = kSignedIn ? (int)(signed char)b : (int)b;
+    }
+#pragma unroll
+    for (int i = 0; i < L; ++i) {
+      acc[i] += (Acc)xb[i * S] * (Acc)w0;
+      acc[i] += (Acc)xb[i * S + 1] * (Acc)w1;
+      acc[i] += (Acc)xb[i * S + 2] * (Acc)w2;
+    }
+  }
+#pragma unroll
+  for (int i = 0; i < L; ++i) {
+    if ((uint32_t)i >= n_out) break;
+    float y = __fmaf_rn(dw_acc_to_float<Acc>(acc[i]), sc, bi);
+    if (has_res) {
+      const uint32_t rb = (rv[i] >> (8 * j)) & 0xFFu;
+      y = __fmaf_rn(res_signed ? (float)(int)(signed char)rb : (float)rb, res_scale, y);
+    }
+    y = fmaxf(y, relu_floor);
+    const float t = fminf(fmaxf(__fmul_rn(y, inv_step), lo_f), hi_f);
+    const uint32_t q = (uint32_t)__float2int_rn(t) & 0xFFu;
+    qw[i] |= q << (8 * j);
+  }
+}
+
+template <int S, bool kSignedIn>
+__global__ void __launch_bounds__(256, 2) dwconv3x3_row32_kernel(const ConvArgs a, const int32_t* __restrict__ wint,
+                                                                 const uint32_t* __restrict__ rowsum256,
+                                                                 uint32_t amax) {
+  pdl_prologue();
+  constexpr int L = DwSeg<S>::kOut, NC = DwSeg<S>::kCols;
+  const uint32_t C = a.C, G = C / 4u;
+  const uint32_t segs = (a.OW + L - 1) / L;
+  const uint32_t total = a.N * a.OH * segs * G;   // the launcher keeps this below 2^32
+  const uint32_t idx = blockIdx.x * blockDim.x + threadIdx.x;
+  if (idx >= total) return;
+  uint32_t t = idx / G;
+  const uint32_t c0 = (idx - t * G) * 4u;
+  const uint32_t seg = t % segs; t /= segs;
+  const uint32_t oy = t % a.OH, n = t / a.OH;
+  const uint32_t ox0 = seg * L;
+
+  // band of input: rows iy0..iy0+2, columns ix0..ix0+NC-1, every word = 4 channels of one position
+  const int iy0 = (int)(oy * S) - (int)a.pad, ix0 = (int)(ox0 * S) - (int)a.pad;
+  const uint32_t last_ox = min(ox0 + (uint32_t)L, a.OW) - 1u;
+  const int ix_end = (int)(last_ox * S) - (int)a.pad + 2;     // last column any output of the segment reads
+  uint32_t raw[3][NC];
+#pragma unroll
+  for (int r = 0; r < 3; ++r) {
+    const int iy = iy0 + r;
+    const bool row_in = (unsigned)iy < a.H;
+    const uint8_t* rp = (const uint8_t*)a.x + ((size_t)(n * a.H + (row_in ? iy : 0)) * a.W) * C + c0;
+#pragma unroll
+    for (int cidx = 0; cidx < NC; ++cidx) {
+      const int ix = ix0 + cidx;
+      raw[r][cidx] = 0u;
+      if (row_in && (unsigned)ix < a.W && ix <= ix_end)
+        raw[r][cidx] = __ldg(reinterpret_cast<const uint32_t*>(rp + (size_t)ix * C));
+    }
+  }
+  const bool has_res = a.residual != nullptr;
+  const size_t obase = ((size_t)(n * a.OH + oy) * a.OW + ox0) * C + c0;
+  const uint32_t n_out = last_ox - ox0 + 1u;
+  uint32_t rv[L], qw[L];
+#pragma unroll
+  for (int i = 0; i < L; ++i) {
+    qw[i] = 0u;
+    rv[i] = 0u;
+    if (has_res && (uint32_t)i < n_out)
+      rv[i] = __ldg(reinterpret_cast<const uint32_t*>((const uint8_t*)a.residual + obase + (size_t)i * C));
+  }
+  const float relu_floor = a.relu ? 0.0f : __int_as_float(0xFF800000);
+  const float lo_f = (float)a.qmin, hi_f = (float)a.qmax;
+  const bool res_signed = a.residual_dtype == PSB_DT_S8;
+  const uint32_t level = a.uniform_log2k;
+#pragma unroll
+  for (int j = 0; j < 4; ++j) {
+    const uint32_t o = c0 + j;
+    const float sc = ldexpf(a.scale[o], a.e_base[o] - (int)level), bi = a.bias[o];
+    const int32_t* wch = wint + (size_t)o * 9u;
+    // (a sum marked unknown, 0xFFFFFFFF, fails the test like a large one)
+    const unsigned long long bound = (unsigned long long)__ldg(rowsum256 + (size_t)level * a.O + o) * 256ull * amax;
+    if (bound < (1ull << 31))
+      dw_channel<S, kSignedIn, int>(raw, j, wch, sc, bi, has_res, rv, res_signed, a.residual_scale, relu_floor,
+                                    a.inv_step, lo_f, hi_f, n_out, qw);
+    else
+      dw_channel<S, kSignedIn, long long>(raw, j, wch, sc, bi, has_res, rv, res_signed, a.residual_scale, relu_floor,
+                                          a.inv_step, lo_f, hi_f, n_out, qw);
+  }
+#pragma unroll
+  for (int i = 0; i < L; ++i)
+    if ((uint32_t)i < n_out) *reinterpret_cast<uint32_t*>((uint8_t*)a.q_out + obase + (size_t)i * C) = qw[i];
+}
+
 // x ^ 0x80 over a whole tensor: unsigned bytes become (x - 128) as signed bytes, 16 per thread.
 __global__ void offset128_kernel(const uint4* __restrict__ src, uint4* __restrict__ dst, size_t n16, uint32_t limit,
                                  uint32_t* __restrict__ err) {
@@ -560,7 +685,8 @@ cudaError_t launch_range_check(const void* x, size_t bytes, uint32_t is_signed, 
   return cudaGetLastError();
 }
 
-cudaError_t launch_shift_add(const ConvArgs& a, const WintTable& wt, cudaStream_t s) {
+cudaError_t launch_shift_add(const ConvArgs& a, const WintTable& wt, const uint32_t* rowsum256, uint32_t amax,
+                             cudaStream_t s) {
   size_t total = (size_t)a.N * a.OH * a.OW * a.O;
   // depthwise, channels-last, one draw count, only codes wanted: the vectorised kernel
   const size_t dw_smem = (size_t)a.KH * a.KW * a.C * sizeof(int32_t);
@@ -581,7 +707,15 @@ cudaError_t launch_shift_add(const ConvArgs& a, const WintTable& wt, cudaStream_
         const uint32_t blocks = (uint32_t)((threads + 255u) / 256u);
         const int32_t* wl = wt.w[a.uniform_log2k];
         const bool sg = a.in_dtype == PSB_DT_S8;
-        if (a.stride == 1) {
+        if (rowsum256) {
+          if (a.stride == 1) {
+            if (sg) launch_pdl(dwconv3x3_row32_kernel<1, true>, blocks, 256, 0, s, a, wl, rowsum256, amax);
+            else launch_pdl(dwconv3x3_row32_kernel<1, false>, blocks, 256, 0, s, a, wl, rowsum256, amax);
+          } else {
+            if (sg) launch_pdl(dwconv3x3_row32_kernel<2, true>, blocks, 256, 0, s, a, wl, rowsum256, amax);
+            else launch_pdl(dwconv3x3_row32_kernel<2, false>, blocks, 256, 0, s, a, wl, rowsum256, amax);
+          }
+        } else if (a.stride == 1) {
           if (sg) launch_pdl(dwconv3x3_row_kernel<1, true>, blocks, 256, 0, s, a, wl);
           else launch_pdl(dwconv3x3_row_kernel<1, false>, blocks, 256, 0, s, a, wl);
         } else {

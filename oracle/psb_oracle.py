@@ -300,3 +300,36 @@ def run_network(layers, net, images, seed, uniform_log2k=3, fc_log2k=None, kmaps
             q, logits = q.reshape(q.shape[0], -1), y.reshape(y.shape[0], -1)
         acts[l["dst"]] = q
     return acts, logits
+
+
+# ---- attention proposal (Sec. 4.5, "Computational Attention") ---------------------------------
+# Plain numpy in float64, written out from the definitions.
+
+def attention_entropy(codes, step):
+    """Pixelwise entropy of the softmax over the channels of a layer's activations a = codes * step
+    (channels-last [n, h, w, c]):  h_xy = - sum_c softmax(a_xy)_c * log softmax(a_xy)_c."""
+    a = np.asarray(codes, dtype=np.float64) * float(step)
+    a = a - a.max(axis=-1, keepdims=True)
+    e = np.exp(a)
+    sm = e / e.sum(axis=-1, keepdims=True)
+    with np.errstate(divide="ignore", invalid="ignore"):
+        t = np.where(sm > 0, sm * np.log(sm), 0.0)
+    return -t.sum(axis=-1)
+
+
+def attention_maps(entropy, lo_log2k, hi_log2k, resolutions):
+    """Hard threshold at the mean entropy of each image: locations above it get the higher draw count.  The
+    mask of the layer's own resolution serves every other resolution by nearest-neighbour sampling:
+    location (y, x) of an r x r map reads mask[floor(y * h / r), floor(x * w / r)].
+    Returns ({r: uint8 [n, r, r] of log2 k}, mean entropy per image)."""
+    h = np.asarray(entropy, dtype=np.float64)
+    n, H, W = h.shape
+    mean = h.reshape(n, -1).mean(axis=1)
+    mask = h > mean[:, None, None]
+    out = {}
+    for r in resolutions:
+        ys = (np.arange(r) * H) // r
+        xs = (np.arange(r) * W) // r
+        m = mask[:, ys][:, :, xs]
+        out[r] = np.where(m, hi_log2k, lo_log2k).astype(np.uint8)
+    return out, mean

@@ -463,7 +463,67 @@ def sample_options(args):
     return opts
 
 
+class AttentionWorkload(NetWorkload):
+    """The two-pass scheme of Sec. 4.5 on the ResNet-50-shaped network: a first pass with k = 8 everywhere, the
+    pixelwise entropy of its last convolutional layer thresholded at the image mean, a second pass with k = 16
+    inside the mask and k = 8 outside (psb8/16).  Both passes use one set of draws (levels share draws)."""
+
+    def __init__(self, k, rank=0, batch=0, sample_opts=None):
+        NetWorkload.__init__(self, "resnet50", 8, rank, batch=batch or 64, sample_opts=sample_opts)
+        self.name = "resnet50_attention_b%d" % self.batch
+        self.macs = 2 * self.macs_per_image * self.batch           # two passes
+        self.mean_k = 8.0
+
+    def setup(self, ctx, psb, torch):
+        from paper_1904_02205_b200.network import Network
+        from workloads import build_network
+
+        self.ctx, self.psb, self.torch = ctx, psb, torch
+        self.net = build_network(self.layers, 224, self.batch, self.seed + 100 * self.rank, self.qu, self.qs)
+        res = [112, 56, 28, 14, 7]
+        self.maps = {r: torch.full((self.batch, r, r), 3, dtype=torch.uint8, device=ctx.device) for r in res}
+        self.first = Network(ctx, self.layers, self.net, self.batch, 0b11000, uniform_log2k=3, sample_opts=self.sample_opts)
+        self.nw = Network(ctx, self.layers, self.net, self.batch, 0b11000, kmaps={r: m.cpu().numpy() for r, m in self.maps.items()},
+                          uniform_log2k=3, fc_log2k=4, sample_opts=self.sample_opts, weights_from=self.first)
+        self.nw.kmaps = self.maps                                  # the maps the producer writes, in place
+        self.last = [l for l in self.layers if l["op"] == "conv" and l["hout"] == 7][-1]["dst"]
+        self.last_step = float(self.net["steps"][self.last])
+        self.entropy = torch.empty((self.batch, 7, 7), dtype=torch.float32, device=ctx.device)
+        self.first.sample(self.seed)
+        self.image_host = torch.from_numpy(self.net["image"]).pin_memory()
+        self.image_dev = self.image_host.to(ctx.device)
+        self.logits_host = torch.empty((self.batch, self.layers[-1]["cout"]), dtype=torch.float32).pin_memory()
+        self.first.forward(self.image_dev)
+        self.nw.acts["image"] = self.first.acts["image"]
+        self._propose()
+        self.nw.forward(self.image_dev)
+        self.e2e_h2d = self.image_host.numel()
+        self.e2e_d2h = self.logits_host.numel() * 4
+        self.layer_ms = None
+
+    def _propose(self):
+        self.ctx.attention_entropy(self.first.acts[self.last], self.last_step, out=self.entropy)
+        self.ctx.attention_maps(self.entropy, 3, 4, [112, 56, 28, 14, 7], out=self.maps)
+
+    def step(self, i):
+        self.first.sample(self.seed + i)
+        self.first.forward()
+        self._propose()
+        self.nw.forward()
+
+    def e2e_step(self, i):
+        self.first.acts["image"].copy_(self.image_host, non_blocking=True)
+        self.step(i)
+        self.logits_host.copy_(self.nw.logits, non_blocking=True)
+
+    def kernel_only(self):
+        self.refined = float((self.maps[7] == 4).float().mean().item())
+        NetWorkload.kernel_only(self)
+
+
 def make_workload(args, rank):
+    if args.workload == "resnet50_attention":
+        return AttentionWorkload(args.k, rank, batch=args.batch, sample_opts=sample_options(args))
     if args.workload == "conv3x3":
         return ConvWorkload(args.k, rank, sample_options(args))
     if args.workload == "fc":
@@ -541,7 +601,7 @@ def main():
     ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="psb")
-    ap.add_argument("--workload", default="conv3x3", choices=["conv3x3", "fc", "resnet50", "mobilenetv2", "resnet50_adaptive"])
+    ap.add_argument("--workload", default="conv3x3", choices=["conv3x3", "fc", "resnet50", "mobilenetv2", "resnet50_adaptive", "resnet50_attention"])
     ap.add_argument("--k", type=int, default=8)
     ap.add_argument("--batch", type=int, default=0)
     ap.add_argument("--exp-bits", type=int, default=4, help="octaves of the exponent window: 2^exp_bits (Sec. 4.4)")
@@ -671,6 +731,8 @@ def main():
     for key in ("k_sweep", "resnet50_b64_k8"):
         if key in extras:
             line[key] = extras[key]
+    if hasattr(wl, "refined"):
+        line["config"]["refined_fraction"] = wl.refined      # share of the locations the mask sends to k = 16
     if not args.no_cpu_baseline and world == 1:
         dt, macs, sample = wl.oracle_sample(getattr(wl, "oracle_images", 4))
         line["cpu_baseline"] = dict(value=macs / dt / 1e9, unit=UNIT, cores=1, kind="oracle", sample=sample)

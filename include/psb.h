@@ -305,6 +305,23 @@ psb_status psb_global_avgpool_u8(psb_ctx* ctx, const uint8_t* x_dev, uint32_t la
                                  uint32_t c, uint32_t h, uint32_t w, float pool_mul, int32_t qmin,
                                  int32_t qmax, uint8_t* out_dev, void* stream);
 
+/* Attention proposal (Sec. 4.5, "Computational Attention"): from a cheap pass with few draws everywhere,
+ * find the regions that deserve more.
+ * psb_attention_entropy: pixelwise entropy of the softmax over the channels of a layer's activations
+ *   a = code * step (the paper uses the last convolutional layer):
+ *   h[n][y][x] = - sum_c softmax(a[n][y][x][.])_c * log softmax(a[n][y][x][.])_c,  fp32.
+ *   act_dev: channels-last codes [n][h][w][c] of in_dtype; entropy_dev: float [n][h][w].
+ * psb_attention_maps: hard threshold at the mean entropy of each image; locations above it get
+ *   hi_log2k, the others lo_log2k.  The mask serves every layer resolution by nearest-neighbour
+ *   sampling: location (y, x) of map i reads the mask at (floor(y * h / res[i]), floor(x * w / res[i])).
+ *   res (host): n_res <= 8 resolutions; maps_dev (host array of device pointers): u8 [n][res[i]][res[i]],
+ *   ready for psb_set_sample_map; mean_dev: float [n], the thresholds, may be NULL. */
+psb_status psb_attention_entropy(psb_ctx* ctx, const void* act_dev, uint32_t in_dtype, uint32_t n, uint32_t h,
+                                 uint32_t w, uint32_t c, float step, float* entropy_dev, void* stream);
+psb_status psb_attention_maps(psb_ctx* ctx, const float* entropy_dev, uint32_t n, uint32_t h, uint32_t w,
+                              uint32_t lo_log2k, uint32_t hi_log2k, uint32_t n_res, const uint32_t* res,
+                              uint8_t* const* maps_dev, float* mean_dev, void* stream);
+
 /* Whole networks with few host calls.
  *
  * psb_sample_batch_*: re-sample many layers at once.  The handles must exist already (created

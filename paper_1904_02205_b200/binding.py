@@ -26,7 +26,8 @@ EXPORTS = ["psb_create", "psb_destroy", "psb_status_string", "psb_device_status"
            "psb_last_path", "psb_maxpool2d_u8", "psb_global_avgpool_u8", "psb_sample_level_static",
            "psb_sample_batch_create", "psb_sample_batch_run", "psb_sample_batch_free", "psb_run",
            "psb_launch_count", "psb_int8_mma_probe", "psb_contraction_timing", "psb_contraction_time",
-           "psb_set_checks", "psb_set_wait_limit", "psb_wait_selftest", "psb_contraction_times"]
+           "psb_set_checks", "psb_set_wait_limit", "psb_wait_selftest", "psb_contraction_times",
+           "psb_attention_entropy", "psb_attention_maps"]
 
 
 class psb_wshape(C.Structure):
@@ -100,6 +101,8 @@ def load_library():
     lib.psb_set_checks.argtypes = [vp, u32]
     lib.psb_set_wait_limit.argtypes = [vp, C.c_uint64]
     lib.psb_wait_selftest.argtypes = [vp, vp]
+    lib.psb_attention_entropy.argtypes = [vp, vp, u32, u32, u32, u32, u32, C.c_float, vp, vp]
+    lib.psb_attention_maps.argtypes = [vp, vp, u32, u32, u32, u32, u32, u32, C.POINTER(u32), C.POINTER(vp), vp, vp]
     lib.psb_launch_count.argtypes = []
     lib.psb_launch_count.restype = C.c_uint64
     lib.psb_maxpool2d_u8.argtypes = [vp, vp, u32, u32, u32, u32, u32, u32, u32, u32, vp, vp]
@@ -340,6 +343,29 @@ class Context:
         _check(self.lib.psb_gemm(self.handle, weights.handle, _ptr(x), C.byref(d), _stream(stream)),
                "psb_gemm")
         return out
+
+    # -- attention proposal (Sec. 4.5) -----------------------------------------
+    def attention_entropy(self, act, step, out=None, stream=None):
+        """act: uint8/int8 CUDA tensor [n, h, w, c] of codes; returns float32 [n, h, w]."""
+        assert act.is_cuda and act.is_contiguous() and act.dim() == 4
+        n, h, w, c = act.shape
+        if out is None:
+            out = torch.empty((n, h, w), dtype=torch.float32, device=self.device)
+        _check(self.lib.psb_attention_entropy(self.handle, _ptr(act), _dt_of(act), n, h, w, c, float(step), _ptr(out),
+                                              _stream(stream)), "psb_attention_entropy")
+        return out
+
+    def attention_maps(self, entropy, lo_log2k, hi_log2k, resolutions, out=None, stream=None):
+        """entropy: float32 CUDA tensor [n, h, w]; returns ({res: uint8 [n, res, res]}, mean float32 [n])."""
+        n, h, w = entropy.shape
+        res = list(resolutions)
+        maps = out or {r: torch.empty((n, r, r), dtype=torch.uint8, device=self.device) for r in res}
+        mean = torch.empty((n,), dtype=torch.float32, device=self.device)
+        ra = (C.c_uint32 * len(res))(*res)
+        pa = (C.c_void_p * len(res))(*[maps[r].data_ptr() for r in res])
+        _check(self.lib.psb_attention_maps(self.handle, _ptr(entropy), n, h, w, lo_log2k, hi_log2k, len(res), ra, pa,
+                                           _ptr(mean), _stream(stream)), "psb_attention_maps")
+        return maps, mean
 
     # -- whole networks -------------------------------------------------------
     def sample_batch_create(self, filters, weights):

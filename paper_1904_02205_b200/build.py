@@ -7,7 +7,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libpsb_b200.so")
-SOURCES = ["psb_api.cu", "psb_sampler.cu", "psb_shiftadd.cu", "psb_tensor.cu", "psb_probe.cu", "psb_sort.cu"]
+SOURCES = ["psb_api.cu", "psb_sampler.cu", "psb_shiftadd.cu", "psb_tensor.cu", "psb_probe.cu", "psb_sort.cu", "psb_attention.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "-I" + os.path.join(ROOT, "include"), "-I" + CSRC]
 

@@ -570,6 +570,30 @@ psb_status psb_run(psb_ctx* ctx, const psb_op* ops, uint32_t n_ops, void* stream
   return PSB_OK;
 }
 
+psb_status psb_attention_entropy(psb_ctx* ctx, const void* act_dev, uint32_t in_dtype, uint32_t n, uint32_t h,
+                                 uint32_t w, uint32_t c, float step, float* entropy_dev, void* stream) {
+  if (!ctx || !act_dev || !entropy_dev || !n || !h || !w || !c) return PSB_ERR_INVALID_ARG;
+  if (in_dtype != PSB_DT_U8 && in_dtype != PSB_DT_S8) return PSB_ERR_INVALID_ARG;
+  if (!(step > 0.0f) || ((uintptr_t)entropy_dev & 3u)) return PSB_ERR_INVALID_ARG;
+  if ((uint64_t)n * h * w >= (1ull << 31)) return PSB_ERR_UNSUPPORTED;
+  if (launch_entropy(act_dev, in_dtype == PSB_DT_S8, n * h * w, c, step, entropy_dev, (cudaStream_t)stream) != cudaSuccess)
+    return PSB_ERR_CUDA;
+  return PSB_OK;
+}
+
+psb_status psb_attention_maps(psb_ctx* ctx, const float* entropy_dev, uint32_t n, uint32_t h, uint32_t w,
+                              uint32_t lo_log2k, uint32_t hi_log2k, uint32_t n_res, const uint32_t* res,
+                              uint8_t* const* maps_dev, float* mean_dev, void* stream) {
+  if (!ctx || !entropy_dev || !n || !h || !w || !n_res || n_res > 8u || !res || !maps_dev) return PSB_ERR_INVALID_ARG;
+  if (!pow2_level_ok(lo_log2k) || !pow2_level_ok(hi_log2k)) return PSB_ERR_BAD_K;
+  for (uint32_t i = 0; i < n_res; ++i)
+    if (!res[i] || !maps_dev[i] || (uint64_t)res[i] * res[i] >= (1ull << 31)) return PSB_ERR_INVALID_ARG;
+  if (launch_attention_maps(entropy_dev, n, h, w, lo_log2k, hi_log2k, n_res, res, maps_dev, mean_dev,
+                            (cudaStream_t)stream) != cudaSuccess)
+    return PSB_ERR_CUDA;
+  return PSB_OK;
+}
+
 psb_status psb_maxpool2d_u8(psb_ctx* ctx, const uint8_t* x_dev, uint32_t layout, uint32_t n,
                             uint32_t c, uint32_t h, uint32_t w, uint32_t k, uint32_t stride,
                             uint32_t pad, uint8_t* out_dev, void* stream) {

@@ -261,6 +261,13 @@ cudaError_t launch_level_sort(const uint8_t* kmap, uint32_t M, void* ctl, uint32
 cudaError_t launch_gather_sorted(const ConvArgs& a, const uint32_t* perm, const void* ctl, uint32_t cpad, uint8_t* dst,
                                  cudaStream_t s);
 
+// attention proposal (psb_attention.cu)
+cudaError_t launch_entropy(const void* act, uint32_t is_signed, uint32_t locations, uint32_t C, float step,
+                           float* entropy, cudaStream_t s);
+cudaError_t launch_attention_maps(const float* entropy, uint32_t N, uint32_t H, uint32_t W, uint32_t lo_log2k,
+                                  uint32_t hi_log2k, uint32_t n_res, const uint32_t* res, uint8_t* const* maps,
+                                  float* mean_out, cudaStream_t s);
+
 // int8 tensor-core issue-rate probe (psb_probe.cu)
 psb_status int8_mma_probe(psb_ctx* ctx, uint32_t n_cols, uint32_t groups, double* mac_per_clk_per_sm,
                           double* tera_ops_per_s, cudaStream_t s);

@@ -11,9 +11,11 @@ from . import binding as B
 
 class Network:
     def __init__(self, ctx, layers, net, batch, level_mask, kmaps=None, uniform_log2k=3, fc_log2k=None,
-                 path=B.PSB_PATH_AUTO, sample_opts=None):
+                 path=B.PSB_PATH_AUTO, sample_opts=None, weights_from=None):
         """layers/net: from workloads.build_network; kmaps: {resolution: u8 [batch, res, res]} or None;
-        sample_opts: keyword options of Context.sample_weights (exp_bits, underflow, prob_bits, ...)."""
+        sample_opts: keyword options of Context.sample_weights (exp_bits, underflow, prob_bits, ...);
+        weights_from: another Network over the same layers whose sampled filters this one uses (two passes of one
+        network with different draw counts share one set of draws)."""
         self.ctx, self.layers, self.batch, self.level_mask, self.path = ctx, layers, batch, level_mask, path
         self.sample_opts = dict(sample_opts or {})
         self.uniform_log2k = uniform_log2k
@@ -44,10 +46,15 @@ class Network:
         self.paths = {}
         self._batch = None
         self._ops = None
+        self._shared = weights_from
+        if weights_from is not None:
+            self.weights = weights_from.weights
 
     def sample(self, seed):
         """Fresh draws for every layer.  The first call creates the handles layer by layer
         (psb_sample_weights); later calls re-sample all layers in one psb_sample_batch_run."""
+        if self._shared is not None:
+            return self._shared.sample(seed)
         if self._batch is not None:
             self.ctx.sample_batch_run(self._batch, seed)
             return
@@ -161,6 +168,9 @@ class Network:
         return self.logits
 
     def free(self):
+        if self._shared is not None:
+            self.weights = {}
+            return
         if self._batch is not None:
             self.ctx.sample_batch_free(self._batch)
             self._batch = None

@@ -757,3 +757,44 @@ def test_bad_sampling_options_are_refused(psb, ctx):
         with pytest.raises(psb.PsbError) as e:
             ctx.sample_weights(w, level_mask=1, **bad)
         assert e.value.status == psb.PSB_ERR_INVALID_ARG
+
+
+# ------------------------------------------------------------- attention proposal (Sec. 4.5)
+
+@pytest.mark.parametrize("case", [(3, 7, 7, 2048, np.uint8, 15, 0.21), (2, 5, 9, 37, np.uint8, 255, 0.03),
+                                  (2, 4, 4, 96, np.int8, 15, 0.4), (1, 14, 14, 1000, np.uint8, 15, 1.3)])
+def test_attention_entropy_and_maps(psb, ctx, oracle, case):
+    """Pixelwise entropy of the softmax over channels (fp32 on the device, float64 in the oracle: sums of up to
+    2048 terms, so 2e-5 relative + 2e-5 absolute), the threshold at the image mean and the maps of every resolution.
+    The threshold decides an integer from a floating-point value: locations whose entropy lies within 1e-4 of the
+    mean may fall on either side; everywhere else the maps must be identical."""
+    import torch
+
+    N, H, W, C, dt, hi, step = case
+    rng = np.random.default_rng(abs(hash(case[:4])) % 2 ** 31)
+    lo = 0 if dt == np.uint8 else -hi
+    q = rng.integers(lo, hi + 1, size=(N, H, W, C)).astype(dt)
+    q[0, 0, 0] = q[0, 0, 0, 0]                   # equal activations: log C
+    q[-1, -1, -1] = lo
+    q[-1, -1, -1, C // 2] = hi                   # one dominant channel
+    h_gpu = ctx.attention_entropy(torch.from_numpy(q).to(ctx.device), step)
+    res = [H, 2 * H, 3, 11]
+    maps, mean = ctx.attention_maps(h_gpu, 2, 4, res)
+    assert ctx.device_status() == 0
+    h_ref = oracle.attention_entropy(q, step)
+    hg = h_gpu.cpu().numpy()
+    assert np.allclose(hg, h_ref, rtol=2e-5, atol=2e-5)
+    ref_maps, ref_mean = oracle.attention_maps(h_ref, 2, 4, res)
+    assert np.allclose(mean.cpu().numpy(), ref_mean, rtol=2e-5, atol=2e-5)
+    sure = np.abs(h_ref - ref_mean[:, None, None]) > 1e-4
+    for r in res:
+        got = maps[r].cpu().numpy()
+        assert got.shape == (N, r, r) and set(np.unique(got)) <= {2, 4}
+        ys, xs = (np.arange(r) * H) // r, (np.arange(r) * W) // r
+        s = sure[:, ys][:, :, xs]
+        assert np.array_equal(got[s], ref_maps[r][s])
+        # and the map is what the device's own entropies and mean say
+        own = np.where(hg[:, ys][:, :, xs] > mean.cpu().numpy()[:, None, None], 4, 2)
+        assert np.array_equal(got, own)
+    with pytest.raises(psb.PsbError):
+        ctx.attention_maps(h_gpu, 2, 9, res)

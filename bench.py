@@ -154,6 +154,29 @@ class ConvWorkload:
         self.ctx.conv2d(self.wt, self.x_nhwc, psb.PSB_LAYOUT_NHWC, 1, 1, self.scale, self.bias, True,
                         c["inv_step"], 0, 15, in_max=15, out=self.out_nhwc)
 
+    def back_to_back(self, n_sets=24, rounds=4):
+        """The dominant kernel launched back to back on a rotating set of input / output tensors larger than L2
+        (24 x 12.8 MB): average device time per launch between one pair of events, i.e. without the gaps that a
+        pair of events and an L2 flush put around a single launch."""
+        c, psb, torch = self.cfg, self.psb, self.torch
+        if not hasattr(self, "x_sets"):
+            self.x_sets = [self.x_nhwc.clone() for _ in range(n_sets)]
+            self.out_sets = [{"q": torch.empty_like(self.out_nhwc["q"])} for _ in range(n_sets)]
+        def one(j):
+            self.ctx.conv2d(self.wt, self.x_sets[j], psb.PSB_LAYOUT_NHWC, 1, 1, self.scale, self.bias, True,
+                            c["inv_step"], 0, 15, in_max=15, out=self.out_sets[j])
+        for j in range(n_sets):
+            one(j)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        e0.record()
+        for _ in range(rounds):
+            for j in range(n_sets):
+                one(j)
+        e1.record()
+        e1.synchronize()
+        return e0.elapsed_time(e1) / (rounds * n_sets)
+
     def e2e_step(self, i):
         self.x_stage.copy_(self.x_host, non_blocking=True)
         c, psb = self.cfg, self.psb
@@ -666,6 +689,7 @@ def main():
         dist.barrier()
     kern_ms = timed(lambda i: wl.kernel_only(), max(args.steps, 10) if args.workload in ("conv3x3", "fc") else 4)
     in_step_ms = []
+    b2b_ms = wl.back_to_back() if args.workload == "conv3x3" else None
     if args.workload == "conv3x3":
         # the same steps once more with the library's own pair of events around the contraction kernel:
         # its duration inside the step (filters and converted input just written, output planar)
@@ -721,6 +745,12 @@ def main():
         r = line["roofline"]
         r["kernel_ms_in_step_planar_out"] = statistics.mean(in_step_ms)
         r["frac_in_step"] = r["frac"] * r["kernel_ms"] / r["kernel_ms_in_step_planar_out"]
+    if b2b_ms:
+        # the same kernel launched back to back on inputs that rotate through more than the L2 holds
+        r = line["roofline"]
+        r["kernel_ms_back_to_back"] = b2b_ms
+        r["frac_back_to_back"] = r["frac"] * r["kernel_ms"] / b2b_ms
+        r["back_to_back_note"] = "24 input/output sets of 12.8 MB in rotation (> L2), one pair of events around 96 launches"
     if clk.get("sm_mhz"):
         # kernel time x the SM clock sampled under load: comparable across runs whatever the clock was
         line["roofline"]["kernel_clocks"] = line["roofline"].get("kernel_ms", 0.0) * 1e-3 * clk["sm_mhz"] * 1e6

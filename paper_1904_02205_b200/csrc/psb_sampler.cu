@@ -206,6 +206,7 @@ __device__ __forceinline__ void sample_block(const SampleParams& p, uint32_t blo
   const uint32_t layer_id = p.layer_id, KHKW = p.KHKW, Cg = p.Cg;
   const uint32_t packed_kw = p.packed_kw, run_pitch = p.run_pitch, has_planes = p.has_planes;
   const uint32_t bk = p.bk, n_cb = p.n_cb, n_kb = p.n_kb;
+  const uint32_t bk_shift = 31u - (uint32_t)__clz((int)bk), bk_mask = bk - 1u;     // bk is a power of two (32, 64, 128)
   const PhiloxKeys keys(seed_lo, seed_hi);
   // Row sums of |W_k| (in units of 256, each weight rounded up) for the bound that lets the contraction
   // recombine its digit planes in 32 bits: gathered per block in shared memory, then added to the layer's words
@@ -321,12 +322,12 @@ __device__ __forceinline__ void sample_block(const SampleParams& p, uint32_t blo
 
     const size_t wpos = ((size_t)o * KHKW + tap) * Cg + ci;
     // K block and column inside it (bk is a power of two)
-    uint32_t kb = tap * n_cb + ci / bk, kin = ci % bk;
+    uint32_t kb = tap * n_cb + (ci >> bk_shift), kin = ci & bk_mask;
     if (packed_kw) {
       const uint32_t kh = tap / packed_kw;
       const uint32_t kcol = kh * run_pitch + (tap - kh * packed_kw) * Cg + ci;
-      kb = kcol / bk;
-      kin = kcol % bk;
+      kb = kcol >> bk_shift;
+      kin = kcol & bk_mask;
     }
     const uint32_t jt = o / kTileN, on = o % kTileN;
 #pragma unroll
@@ -335,18 +336,26 @@ __device__ __forceinline__ void sample_block(const SampleParams& p, uint32_t blo
       const uint32_t mag = live ? (((base << l) + cnt[l]) << sh) : 0u;
       p.wint[l][wpos] = neg ? -(int32_t)mag : (int32_t)mag;
       if (track) {
-        // lanes of a warp mostly share a row: one shared-memory add per row and warp
+        // lanes of a warp mostly share a row: then one reduction and one shared-memory add per warp
         const uint32_t lanes = __activemask();
-        const uint32_t peers = __match_any_sync(lanes, r);
-        const uint32_t sum = __reduce_add_sync(peers, (mag + 255u) >> 8);
-        if ((threadIdx.x & 31u) == (uint32_t)__ffs((int)peers) - 1u && sum) atomicAdd(&row_sum[l][r], sum);
+        const uint32_t r_first = __shfl_sync(lanes, r, (int)__ffs((int)lanes) - 1);
+        const uint32_t part = (mag + 255u) >> 8;
+        if (__all_sync(lanes, r == r_first)) {
+          const uint32_t sum = __reduce_add_sync(lanes, part);
+          if ((threadIdx.x & 31u) == (uint32_t)__ffs((int)lanes) - 1u && sum) atomicAdd(&row_sum[l][r], sum);
+        } else if (part) {
+          atomicAdd(&row_sum[l][r], part);
+        }
       }
       if (has_planes) {
         const int P = p.planes_count[l];
-        int8_t* tile = p.planes[l] + ((size_t)jt * n_kb + kb) * ((size_t)P * kTileN * bk);
+        int8_t* tile = p.planes[l] + (((size_t)jt * n_kb + kb) * (size_t)P << (6u + bk_shift));   // P * 64 * bk per tile
+        // byte offset of (row, kin) in the swizzled tile (plane_offset), advanced by 64 rows per plane
+        const uint32_t lin0 = (on << bk_shift) + kin, sw_mask = (bk >> 4) - 1u;
         for (int pl = 0; pl < P; ++pl) {
           const int digit = (int)((mag >> (kDigitBits * pl)) & 0x7Fu);
-          tile[plane_offset((uint32_t)pl * kTileN + on, kin, bk)] = (int8_t)(neg ? -digit : digit);
+          const uint32_t lin = lin0 + ((uint32_t)pl << (6u + bk_shift));
+          tile[lin ^ (((lin >> 7) & sw_mask) << 4)] = (int8_t)(neg ? -digit : digit);
         }
       }
     }

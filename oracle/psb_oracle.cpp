@@ -29,7 +29,7 @@
 //     q = |w| / 2^e_base, the plain Bernoulli gate of Eq. 2-3; unbiased, no "+ 1" term.
 //   * optional (Sec. 4.4): probabilities stored with b bits on the regular grid {0, 1/2^b, ...,
 //     1 - 1/2^b}; p is rounded to the nearest grid point, and a p that rounds to 1 becomes p = 0 at the
-//     next exponent ("the right boundary would result in a higher exponent").  The comparator then has
+//     next exponent (the grid leaves 1 out because it belongs there).  The comparator then has
 //     b bits (supplement, "Stochastic multiplier") and one Philox word serves floor(32 / b) draws.
 //     The deterministic variant of Sec. 4.4 uses the upper shift in round(p_q * k) of the k cases.
 //   * the random stream is Philox4x32-10 (Salmon, Moraes, Dror, Shaw, SC'11),

@@ -20,6 +20,8 @@ namespace {
 
 constexpr int kThreads = 256;
 constexpr int kStage = 2048;  // weights staged in shared memory per block
+constexpr int kEmaxRows = kThreads / 32;   // output channels per block of the exponent pass (norm == 1, short rows)
+constexpr int kEmaxLongRow = 1024;         // rows longer than this get a block each
 constexpr int kRowSumRows = 256;   // filter rows per block for which the sampler keeps sums of |W_k|
 
 // Philox4x32-10 (Salmon et al., SC'11): ten rounds of two 32x32->64 multiplies and
@@ -123,7 +125,7 @@ __device__ __forceinline__ uint32_t small_div(uint32_t t, uint32_t magic) { retu
 
 // Largest biased exponent of the finite weights of each exponent group; flags Inf/NaN (which
 // contribute nothing: the finite weights of the group keep the window they would have without it).
-// norm == 1: one block per output channel.  norm == 0: grid-stride over the layer.
+// norm == 1: one warp (short rows) or one block per output channel.  norm == 0: grid-stride over the layer.
 // Biased exponent of a weight after its probability has been rounded to `pbits` bits (Sec. 4.4): a
 // probability that rounds to 1 is the next power of two.  pbits == 0: the exponent as it is.
 __device__ __forceinline__ uint32_t quantised_exponent(uint32_t u, uint32_t pbits) {
@@ -145,18 +147,63 @@ __device__ __forceinline__ void emax_block(const float* __restrict__ w, uint32_t
   uint32_t best = 0;
   bool bad = false;
   if (norm) {
-    const float* row = w + (size_t)block * d;
-    for (uint32_t i = threadIdx.x; i < d; i += blockDim.x) {
-      uint32_t E = quantised_exponent(__float_as_uint(row[i]), pbits);
-      bad |= (E == 255u);
-      best = max(best, E == 255u ? 0u : E);     // Inf/NaN is flagged and takes no part in the window
+    // short rows: one warp per output channel, kEmaxRows channels per block; long rows: one block per
+    // channel.  16-byte loads where the row allows, several in flight per lane.
+    const bool per_warp = d <= (uint32_t)kEmaxLongRow;
+    const uint32_t o = per_warp ? block * (uint32_t)kEmaxRows + (threadIdx.x >> 5) : block;
+    const uint32_t lane = per_warp ? (threadIdx.x & 31u) : threadIdx.x, lanes = per_warp ? 32u : blockDim.x;
+    if (o < O) {
+      const float* row = w + (size_t)o * d;
+      if ((((uintptr_t)row) & 15u) == 0u && (d & 3u) == 0u) {
+#pragma unroll 4
+        for (uint32_t i = lane * 4u; i < d; i += lanes * 4u) {
+          const uint4 v = __ldg(reinterpret_cast<const uint4*>(row + i));
+          const uint32_t u4[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+          for (int j = 0; j < 4; ++j) {
+            const uint32_t E = quantised_exponent(u4[j], pbits);
+            bad |= (E == 255u);
+            best = max(best, E == 255u ? 0u : E);     // Inf/NaN is flagged and takes no part in the window
+          }
+        }
+      } else {
+#pragma unroll 4
+        for (uint32_t i = lane; i < d; i += lanes) {
+          const uint32_t E = quantised_exponent(__float_as_uint(__ldg(row + i)), pbits);
+          bad |= (E == 255u);
+          best = max(best, E == 255u ? 0u : E);
+        }
+      }
+    }
+    if (per_warp) {
+      if (o >= O) return;                                   // warp-uniform; no block-wide barrier on this path
+      if (__any_sync(0xFFFFFFFFu, bad) && lane == 0u) atomicOr(err, kDevErrNonFinite);
+      best = __reduce_max_sync(0xFFFFFFFFu, best);
+      // `tag` (a call number in the bits above the exponent) distinguishes this call's maxima from whatever
+      // an earlier call left in the word
+      if (lane == 0u) e_max[o] = tag | best;
+      return;
     }
   } else {
-    size_t total = (size_t)O * d;
-    for (size_t i = (size_t)block * blockDim.x + threadIdx.x; i < total; i += (size_t)blocks * blockDim.x) {
-      uint32_t E = quantised_exponent(__float_as_uint(w[i]), pbits);
-      bad |= (E == 255u);
-      best = max(best, E == 255u ? 0u : E);
+    const size_t total = (size_t)O * d;
+    if ((((uintptr_t)w) & 15u) == 0u && (total & 3u) == 0u) {
+#pragma unroll 4
+      for (size_t i = ((size_t)block * blockDim.x + threadIdx.x) * 4u; i < total; i += (size_t)blocks * blockDim.x * 4u) {
+        const uint4 v = __ldg(reinterpret_cast<const uint4*>(w + i));
+        const uint32_t u4[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          const uint32_t E = quantised_exponent(u4[j], pbits);
+          bad |= (E == 255u);
+          best = max(best, E == 255u ? 0u : E);
+        }
+      }
+    } else {
+      for (size_t i = (size_t)block * blockDim.x + threadIdx.x; i < total; i += (size_t)blocks * blockDim.x) {
+        const uint32_t E = quantised_exponent(__float_as_uint(__ldg(w + i)), pbits);
+        bad |= (E == 255u);
+        best = max(best, E == 255u ? 0u : E);
+      }
     }
   }
   if (__any_sync(0xFFFFFFFFu, bad) && (threadIdx.x & 31) == 0) atomicOr(err, kDevErrNonFinite);
@@ -177,6 +224,96 @@ __global__ void emax_kernel(const float* __restrict__ w, uint32_t O, uint32_t d,
                             uint32_t* __restrict__ rowsum, uint32_t pbits) {
   pdl_prologue();
   emax_block(w, O, d, norm, e_max, err, blockIdx.x, gridDim.x, tag, rowsum, pbits);
+}
+
+// What one weight becomes at every level: W_k = s (base k + c_k) 2^sh with c_k = cnt[log2 k]; a weight that is
+// not live becomes 0.  `u` is the weight's bit pattern, `index` its canonical index (the Philox counter),
+// `ebase_biased` the biased exponent of the window's floor.
+struct Drawn {
+  uint32_t cnt[kMaxLevels];
+  uint32_t base, sh;
+  bool live;
+};
+
+__device__ __forceinline__ void draw_weight(uint32_t u, uint64_t index, int ebase_biased, uint32_t pbits,
+                                            uint32_t underflow, uint32_t deterministic, uint32_t max_level,
+                                            uint32_t layer_id, const PhiloxKeys& keys, Drawn& out) {
+  const uint32_t E = (u >> 23) & 0xFFu;
+  const uint32_t m = u & 0x7FFFFFu;
+  uint32_t (&cnt)[kMaxLevels] = out.cnt;
+#pragma unroll
+  for (int l = 0; l < kMaxLevels; ++l) cnt[l] = 0u;
+  // probability on the grid of 2^pbits points, a p of 1 carried into the exponent (Sec. 4.4)
+  uint32_t Eq = E, pq = m;
+  if (pbits) {
+    pq = (m + (1u << (22u - pbits))) >> (23u - pbits);
+    if (pq == (1u << pbits)) {
+      if (E < 254u) { Eq = E + 1u; pq = 0u; } else pq = (1u << pbits) - 1u;
+    }
+  }
+  // what the weight becomes: W_k = s (base k + c_k) 2^sh, c_k counting draws with Pr[1] = thr / 2^32 (or
+  // thr / 2^pbits).  Inside the window base = 1 (Eq. 8); below it, if asked for, the Bernoulli gate at the
+  // window's floor (Sec. 3.1): base = 0, sh = 0, thr = |w| / 2^e_base
+  bool live = (E != 0u) && (E != 255u);
+  uint32_t base = 1u, sh = 0u, thr = 0u;
+  const int dist = ebase_biased - (int)Eq;
+  if (dist <= 0) {
+    sh = (uint32_t)(-dist);
+    thr = pbits ? pq : pq << 9;
+  } else if (underflow) {
+    base = 0u;
+    if (pbits == 0u) {
+      thr = dist < 42 ? (uint32_t)((((unsigned long long)(0x800000u + pq)) << 9) >> dist) : 0u;
+      live = live && thr != 0u;
+    } else {
+      const unsigned long long mant = (1ull << pbits) + pq;
+      const unsigned long long qv = dist < 40 ? (mant + (1ull << (dist - 1))) >> dist : 0ull;
+      if (qv == (1ull << pbits)) base = 1u;          // rounds to the window's floor itself
+      else { thr = (uint32_t)qv; live = live && qv != 0ull; }
+    }
+  } else {
+    live = false;
+  }
+
+  // c_k for every level k = 2^l: level l is complete after draw 2^l, i.e. levels 0..2 after the
+  // first Philox call, level l >= 2 after call 2^(l-2)
+  if (live && thr != 0u) {
+    const uint32_t i_lo = (uint32_t)index, i_hi = (uint32_t)(index >> 32);
+    uint32_t rnd[4];
+    if (pbits == 0u) {
+      const uint32_t T = thr;
+      philox4x32_10(0u, layer_id, i_lo, i_hi, keys, rnd);
+      cnt[0] = rnd[0] < T ? 1u : 0u;
+      cnt[1] = cnt[0] + (rnd[1] < T ? 1u : 0u);
+      uint32_t c = cnt[1] + (rnd[2] < T ? 1u : 0u) + (rnd[3] < T ? 1u : 0u);
+      cnt[2] = c;
+#pragma unroll
+      for (int l = 3; l < kMaxLevels; ++l) {
+        if ((uint32_t)l <= max_level) {
+          for (uint32_t q = 1u << (l - 3); q < (1u << (l - 2)); ++q) {
+            philox4x32_10(q, layer_id, i_lo, i_hi, keys, rnd);
+            c += (rnd[0] < T ? 1u : 0u) + (rnd[1] < T ? 1u : 0u) + (rnd[2] < T ? 1u : 0u) + (rnd[3] < T ? 1u : 0u);
+          }
+          cnt[l] = c;
+        }
+      }
+    } else if (deterministic) {
+#pragma unroll
+      for (int l = 0; l < kMaxLevels; ++l) cnt[l] = ((thr << l) + (1u << (pbits - 1u))) >> pbits;
+    } else {
+      // pbits-bit comparator, n = 32 / pbits draws per random word
+      switch (pbits) {
+        case 4: packed_counts<4>(thr, max_level, layer_id, i_lo, i_hi, keys, cnt); break;
+        case 6: packed_counts<6>(thr, max_level, layer_id, i_lo, i_hi, keys, cnt); break;
+        case 8: packed_counts<8>(thr, max_level, layer_id, i_lo, i_hi, keys, cnt); break;
+        default: packed_counts_any(pbits, thr, max_level, layer_id, i_lo, i_hi, keys, cnt); break;
+      }
+    }
+  }
+
+  out.base = base;
+  out.sh = sh;
+  out.live = live;
 }
 
 struct SampleParams {
@@ -225,100 +362,120 @@ __device__ __forceinline__ void sample_block(const SampleParams& p, uint32_t blo
   const uint32_t per_row = cc * p.KHKW;     // canonical elements of one row in this block
   const uint32_t count = rows * per_row;
 
-  // count <= kStage = 2048 and the divisors are block-uniform: divisions by multiply-high
-  const uint32_t per_row_magic = small_div_magic(per_row), cc_magic = small_div_magic(cc);
-  // stage the canonical (channel-major) slice with coalesced loads
-  for (uint32_t t = threadIdx.x; t < count; t += blockDim.x) {
-    const uint32_t r = small_div(t, per_row_magic), rem = t - r * per_row;
-    stage[t] = p.w[(size_t)(o0 + r) * p.d + (size_t)c0 * p.KHKW + rem];
+  // The slice is one contiguous run of the weight tensor (whole rows, or a channel range of one row): stage it
+  // with 16-byte loads where the run allows.
+  {
+    const float* src = p.w + (size_t)o0 * p.d + (size_t)c0 * p.KHKW;
+    if ((((uintptr_t)src) & 15u) == 0u && (count & 3u) == 0u) {
+#pragma unroll 2
+      for (uint32_t t = threadIdx.x * 4u; t < count; t += blockDim.x * 4u)
+        *reinterpret_cast<float4*>(stage + t) = __ldg(reinterpret_cast<const float4*>(src + t));
+    } else {
+#pragma unroll 4
+      for (uint32_t t = threadIdx.x; t < count; t += blockDim.x) stage[t] = __ldg(src + t);
+    }
   }
   __syncthreads();
 
-  // walk the slice in output order (row, tap, channel) so that stores coalesce
+  const uint32_t d = p.d, e_tag = p.e_tag;
+  const uint32_t* const e_max = p.e_max;
+  int32_t* const e_base_out = p.e_base;
+  // count <= kStage and the divisors are block-uniform: divisions by multiply-high.  The slice is walked in
+  // output order (row, tap, channel) so that stores coalesce.
+  if (!packed_kw && has_planes && ((cc | Cg | c0) & 3u) == 0u) {
+    // Four consecutive channels per thread: one 16-byte store of the integer weights and one 4-byte store per
+    // digit plane and level.  Between the draws and the stores the four weights' counts travel as the bytes of
+    // one word per level (c_k <= 64), and (sh, base, sign) as one byte per weight.
+    const uint32_t cc4 = cc >> 2, per_row4 = per_row >> 2;
+    const uint32_t per_row4_magic = small_div_magic(per_row4), cc4_magic = small_div_magic(cc4);
+    for (uint32_t t = threadIdx.x; t < (count >> 2); t += blockDim.x) {
+      const uint32_t r = small_div(t, per_row4_magic), rem = t - r * per_row4;
+      const uint32_t tap = small_div(rem, cc4_magic), cl = (rem - tap * cc4) << 2;
+      const uint32_t o = o0 + r, ci = c0 + cl;
+      // a word written by an earlier call (other tag) means this call found no live weight in the group
+      const uint32_t e_word = e_max[norm ? o : 0];
+      const uint32_t Emax = (e_word >> 8) == e_tag ? (e_word & 0xFFu) : 0u;
+      // biased exponents throughout: e - e_base = E - (Emax - span)
+      const int ebase_biased = (int)Emax - (int)span;
+      if (tap == 0 && ci == 0) e_base_out[o] = Emax ? ebase_biased - 127 : 0;
+      uint32_t cntpk[kMaxLevels] = {0u, 0u, 0u, 0u, 0u, 0u, 0u};
+      uint32_t meta = 0u;
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        const uint32_t u = __float_as_uint(stage[r * per_row + (cl + (uint32_t)j) * KHKW + tap]);
+        const uint64_t index = (uint64_t)o * d + (uint64_t)(ci + (uint32_t)j) * KHKW + tap;  // canonical
+        Drawn dw;
+        draw_weight(u, index, ebase_biased, pbits, underflow, deterministic, max_level, layer_id, keys, dw);
+        if (dw.live) {
+#pragma unroll
+          for (int l = 0; l < kMaxLevels; ++l) cntpk[l] |= dw.cnt[l] << (8 * j);
+          meta |= (dw.sh | (dw.base << 4) | ((u >> 31) << 5)) << (8 * j);
+        }
+      }
+      const size_t wpos = ((size_t)o * KHKW + tap) * Cg + ci;
+      const uint32_t kb = tap * n_cb + (ci >> bk_shift), kin = ci & bk_mask;
+      const uint32_t jt = o / kTileN, on = o % kTileN;
+#pragma unroll
+      for (int l = 0; l < kMaxLevels; ++l) {
+        if (!((level_mask >> l) & 1u)) continue;
+        uint32_t mag[4];
+        int wv[4];
+        uint32_t part = 0u;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          const uint32_t m8 = meta >> (8 * j), c = (cntpk[l] >> (8 * j)) & 0xFFu;
+          mag[j] = ((((m8 >> 4) & 1u) << l) + c) << (m8 & 15u);
+          wv[j] = ((m8 >> 5) & 1u) ? -(int32_t)mag[j] : (int32_t)mag[j];
+          part += (mag[j] + 255u) >> 8;
+        }
+        *reinterpret_cast<int4*>(p.wint[l] + wpos) = make_int4(wv[0], wv[1], wv[2], wv[3]);
+        if (track) {
+          // lanes of a warp mostly share a row: then one reduction and one shared-memory add per warp
+          const uint32_t lanes = __activemask();
+          const uint32_t r_first = __shfl_sync(lanes, r, (int)__ffs((int)lanes) - 1);
+          if (__all_sync(lanes, r == r_first)) {
+            const uint32_t sum = __reduce_add_sync(lanes, part);
+            if ((threadIdx.x & 31u) == (uint32_t)__ffs((int)lanes) - 1u && sum) atomicAdd(&row_sum[l][r], sum);
+          } else if (part) {
+            atomicAdd(&row_sum[l][r], part);
+          }
+        }
+        const int P = p.planes_count[l];
+        int8_t* tile = p.planes[l] + (((size_t)jt * n_kb + kb) * (size_t)P << (6u + bk_shift));   // P * 64 * bk per tile
+        // byte offset of (row, kin) in the swizzled tile (plane_offset), advanced by 64 rows per plane; the four
+        // bytes share a 16-byte piece
+        const uint32_t lin0 = (on << bk_shift) + kin, sw_mask = (bk >> 4) - 1u;
+        for (int pl = 0; pl < P; ++pl) {
+          uint32_t word = 0u;
+#pragma unroll
+          for (int j = 0; j < 4; ++j) {
+            const int digit = (int)((mag[j] >> (kDigitBits * pl)) & 0x7Fu);
+            word |= (uint32_t)((wv[j] < 0 ? -digit : digit) & 0xFF) << (8 * j);
+          }
+          const uint32_t lin = lin0 + ((uint32_t)pl << (6u + bk_shift));
+          *reinterpret_cast<uint32_t*>(tile + (lin ^ (((lin >> 7) & sw_mask) << 4))) = word;
+        }
+      }
+    }
+  } else {
+  const uint32_t per_row_magic = small_div_magic(per_row), cc_magic = small_div_magic(cc);
   for (uint32_t t = threadIdx.x; t < count; t += blockDim.x) {
     const uint32_t r = small_div(t, per_row_magic), rem = t - r * per_row;
     const uint32_t tap = small_div(rem, cc_magic), cl = rem - tap * cc;
     const uint32_t o = o0 + r, ci = c0 + cl;
-    const uint32_t u = __float_as_uint(stage[r * per_row + cl * p.KHKW + tap]);
-    const uint64_t index = (uint64_t)o * p.d + (uint64_t)ci * p.KHKW + tap;  // canonical
-
-    const uint32_t E = (u >> 23) & 0xFFu;
-    const uint32_t m = u & 0x7FFFFFu;
+    const uint32_t u = __float_as_uint(stage[r * per_row + cl * KHKW + tap]);
+    const uint64_t index = (uint64_t)o * d + (uint64_t)ci * KHKW + tap;  // canonical
     // a word written by an earlier call (other tag) means this call found no live weight in the group
-    const uint32_t e_word = p.e_max[norm ? o : 0];
-    const uint32_t Emax = (e_word >> 8) == p.e_tag ? (e_word & 0xFFu) : 0u;
+    const uint32_t e_word = e_max[norm ? o : 0];
+    const uint32_t Emax = (e_word >> 8) == e_tag ? (e_word & 0xFFu) : 0u;
     // biased exponents throughout: e - e_base = E - (Emax - span)
     const int ebase_biased = (int)Emax - (int)span;
-    if (tap == 0 && ci == 0) p.e_base[o] = Emax ? ebase_biased - 127 : 0;
-    // probability on the grid of 2^pbits points, a p of 1 carried into the exponent (Sec. 4.4)
-    uint32_t Eq = E, pq = m;
-    if (pbits) {
-      pq = (m + (1u << (22u - pbits))) >> (23u - pbits);
-      if (pq == (1u << pbits)) {
-        if (E < 254u) { Eq = E + 1u; pq = 0u; } else pq = (1u << pbits) - 1u;
-      }
-    }
-    // what the weight becomes: W_k = s (base k + c_k) 2^sh, c_k counting draws with Pr[1] = thr / 2^32 (or
-    // thr / 2^pbits).  Inside the window base = 1 (Eq. 8); below it, if asked for, the Bernoulli gate at the
-    // window's floor (Sec. 3.1): base = 0, sh = 0, thr = |w| / 2^e_base
-    bool live = (E != 0u) && (E != 255u);
-    uint32_t base = 1u, sh = 0u, thr = 0u;
-    const int dist = ebase_biased - (int)Eq;
-    if (dist <= 0) {
-      sh = (uint32_t)(-dist);
-      thr = pbits ? pq : pq << 9;
-    } else if (underflow) {
-      base = 0u;
-      if (pbits == 0u) {
-        thr = dist < 42 ? (uint32_t)((((unsigned long long)(0x800000u + pq)) << 9) >> dist) : 0u;
-        live = live && thr != 0u;
-      } else {
-        const unsigned long long mant = (1ull << pbits) + pq;
-        const unsigned long long qv = dist < 40 ? (mant + (1ull << (dist - 1))) >> dist : 0ull;
-        if (qv == (1ull << pbits)) base = 1u;          // rounds to the window's floor itself
-        else { thr = (uint32_t)qv; live = live && qv != 0ull; }
-      }
-    } else {
-      live = false;
-    }
-    const bool neg = (u >> 31) != 0u;
-
-    // c_k for every level k = 2^l: level l is complete after draw 2^l, i.e. levels 0..2 after the
-    // first Philox call, level l >= 2 after call 2^(l-2)
-    uint32_t cnt[kMaxLevels] = {0u, 0u, 0u, 0u, 0u, 0u, 0u};
-    if (live && thr != 0u) {
-      const uint32_t i_lo = (uint32_t)index, i_hi = (uint32_t)(index >> 32);
-      uint32_t rnd[4];
-      if (pbits == 0u) {
-        const uint32_t T = thr;
-        philox4x32_10(0u, layer_id, i_lo, i_hi, keys, rnd);
-        cnt[0] = rnd[0] < T ? 1u : 0u;
-        cnt[1] = cnt[0] + (rnd[1] < T ? 1u : 0u);
-        uint32_t c = cnt[1] + (rnd[2] < T ? 1u : 0u) + (rnd[3] < T ? 1u : 0u);
-        cnt[2] = c;
-#pragma unroll
-        for (int l = 3; l < kMaxLevels; ++l) {
-          if ((uint32_t)l <= max_level) {
-            for (uint32_t q = 1u << (l - 3); q < (1u << (l - 2)); ++q) {
-              philox4x32_10(q, layer_id, i_lo, i_hi, keys, rnd);
-              c += (rnd[0] < T ? 1u : 0u) + (rnd[1] < T ? 1u : 0u) + (rnd[2] < T ? 1u : 0u) + (rnd[3] < T ? 1u : 0u);
-            }
-            cnt[l] = c;
-          }
-        }
-      } else if (deterministic) {
-#pragma unroll
-        for (int l = 0; l < kMaxLevels; ++l) cnt[l] = ((thr << l) + (1u << (pbits - 1u))) >> pbits;
-      } else {
-        // pbits-bit comparator, n = 32 / pbits draws per random word
-        switch (pbits) {
-          case 4: packed_counts<4>(thr, max_level, layer_id, i_lo, i_hi, keys, cnt); break;
-          case 6: packed_counts<6>(thr, max_level, layer_id, i_lo, i_hi, keys, cnt); break;
-          case 8: packed_counts<8>(thr, max_level, layer_id, i_lo, i_hi, keys, cnt); break;
-          default: packed_counts_any(pbits, thr, max_level, layer_id, i_lo, i_hi, keys, cnt); break;
-        }
-      }
-    }
+    if (tap == 0 && ci == 0) e_base_out[o] = Emax ? ebase_biased - 127 : 0;
+    Drawn dw;
+    draw_weight(u, index, ebase_biased, pbits, underflow, deterministic, max_level, layer_id, keys, dw);
+    const bool live = dw.live, neg = (u >> 31) != 0u;
+    const uint32_t base = dw.base, sh = dw.sh;
+    const uint32_t (&cnt)[kMaxLevels] = dw.cnt;
 
     const size_t wpos = ((size_t)o * KHKW + tap) * Cg + ci;
     // K block and column inside it (bk is a power of two)
@@ -359,6 +516,7 @@ __device__ __forceinline__ void sample_block(const SampleParams& p, uint32_t blo
         }
       }
     }
+  }
   }
   if (rowsum) {
     __syncthreads();
@@ -447,26 +605,29 @@ __global__ void export_kernel(const int32_t* __restrict__ wint, int32_t* __restr
 namespace {
 
 uint32_t emax_blocks_for(uint32_t O, uint32_t d, uint32_t norm) {
-  if (norm) return O;
+  if (norm) return d <= (uint32_t)kEmaxLongRow ? (O + (uint32_t)kEmaxRows - 1u) / (uint32_t)kEmaxRows : O;
   size_t total = (size_t)O * d;
-  // two weights per thread: the loads of a small layer are all in flight at once
-  uint32_t blocks = (uint32_t)((total + kThreads * 2 - 1) / (kThreads * 2));
+  // sixteen weights per thread (four 16-byte loads in flight)
+  uint32_t blocks = (uint32_t)((total + kThreads * 16 - 1) / (kThreads * 16));
   return blocks < 1 ? 1 : (blocks > 1184 ? 1184 : blocks);
 }
 
 // Parameters of one layer's sampling pass; returns the number of blocks it needs.
-uint32_t fill_sample_params(const float* w_dev, const psb_weights* wt, uint32_t* e_max, SampleParams& p) {
+uint32_t fill_sample_params(const float* w_dev, const psb_weights* wt, uint32_t* e_max, SampleParams& p,
+                            bool batched) {
   const psb_wshape& sh = wt->shape;
   const uint32_t O = sh.out_ch, Cg = sh.in_ch_per_group, KHKW = sh.kh * sh.kw, d = wt->d;
   p.w = w_dev;
   p.O = O; p.Cg = Cg; p.KHKW = KHKW; p.d = d;
-  // weights per block: the whole staging buffer for large layers, less for small ones so that
-  // the layer still spreads over a few hundred blocks
+  // weights per block: the whole staging buffer for large layers; a layer sampled by a launch of its own
+  // gets less if it is small, so that it still spreads over a few hundred blocks (in a batched launch the
+  // other layers' blocks fill the machine)
   const uint64_t total = (uint64_t)O * d;
-  uint32_t budget = (uint32_t)std::min<uint64_t>((uint64_t)kStage, std::max<uint64_t>(256u, total / 296u));
+  uint32_t budget = batched ? (uint32_t)kStage
+                            : (uint32_t)std::min<uint64_t>((uint64_t)kStage, std::max<uint64_t>(256u, total / 296u));
   if (budget < KHKW) budget = KHKW;   // at least one channel (host validation keeps kh*kw <= kStage)
   if (d <= budget) {
-    p.rows_per_block = budget / d;
+    p.rows_per_block = std::min<uint32_t>(budget / d, (uint32_t)kRowSumRows);   // the rows a block keeps sums for
     p.ch_per_block = Cg;
     p.ch_chunks = 1;
   } else {
@@ -526,7 +687,7 @@ cudaError_t launch_sampler(const float* w_dev, psb_weights* wt, uint32_t* err_de
   launch_pdl(emax_kernel, emax_blocks_for(O, wt->d, wt->cfg.norm), kThreads, 0, s, w_dev, O, wt->d, wt->cfg.norm,
              wt->e_max, err_dev, wt->e_calls << 8, wt->rowsum256, wt->cfg.prob_bits); note_launch();
   SampleParams p;
-  const uint32_t blocks = fill_sample_params(w_dev, wt, wt->e_max, p);
+  const uint32_t blocks = fill_sample_params(w_dev, wt, wt->e_max, p, false);
   p.e_tag = wt->e_calls;
   launch_pdl(sample_kernel, blocks, kThreads, 0, s, p); note_launch();
   return cudaGetLastError();
@@ -564,7 +725,7 @@ psb_status sample_batch_create(psb_ctx* ctx, uint32_t n, const float* const* w_d
     for (uint32_t i = 0; i < n; ++i) {
       const psb_weights* wt = weights[i];
       BatchEntry& e = host[i];
-      e.sample_blocks = fill_sample_params(w_dev[i], wt, b->e_max_pool + off, e.p);
+      e.sample_blocks = fill_sample_params(w_dev[i], wt, b->e_max_pool + off, e.p, true);
       e.emax_blocks = emax_blocks_for(wt->shape.out_ch, wt->d, wt->cfg.norm);
       e.emax_first = eb;
       e.sample_first = sb;
@@ -728,7 +889,7 @@ extern "C" psb_status psb_sample_level_static(const float* w_dev, const psb_wsha
   // the array keeps the previous call's maxima: the reduction must start from zero
   if (cudaMemsetAsync(e_max, 0, sizeof(uint32_t) * O, s) != cudaSuccess) return PSB_ERR_CUDA;
   if (cfg->norm) {
-    emax_kernel<<<O, kThreads, 0, s>>>(w_dev, O, d, 1, e_max, err_sink, 0u, nullptr, 0u); note_launch();
+    emax_kernel<<<emax_blocks_for(O, d, 1), kThreads, 0, s>>>(w_dev, O, d, 1, e_max, err_sink, 0u, nullptr, 0u); note_launch();
   } else {
     size_t total = (size_t)O * d;
     uint32_t blocks = (uint32_t)((total + kThreads * 8 - 1) / (kThreads * 8));

@@ -26,11 +26,11 @@ constexpr int kRowSumRows = 256;   // filter rows per block for which the sample
 
 // Philox4x32-10 (Salmon et al., SC'11): ten rounds of two 32x32->64 multiplies and
 // xors; the key advances by the two Weyl constants after every round.  The ten round keys
-// depend on the seed only, so a thread computes them once (PhiloxKeys) and reuses them for
-// every weight.
+// depend on the seed only: the host computes them once per launch (PhiloxKeys) and hands them to the kernel as a
+// parameter, so every round reads its key straight from the constant bank and no register holds one.
 struct PhiloxKeys {
   uint32_t k0[10], k1[10];
-  __device__ __forceinline__ PhiloxKeys(uint32_t seed_lo, uint32_t seed_hi) {
+  __host__ __device__ __forceinline__ PhiloxKeys(uint32_t seed_lo, uint32_t seed_hi) {
 #pragma unroll
     for (int r = 0; r < 10; ++r) {
       k0[r] = seed_lo + (uint32_t)r * 0x9E3779B9u;
@@ -335,8 +335,8 @@ struct SampleParams {
   int planes_count[kMaxLevels];
 };
 
-__device__ __forceinline__ void sample_block(const SampleParams& p, uint32_t block, uint32_t seed_lo,
-                                             uint32_t seed_hi, float* stage) {
+__device__ __forceinline__ void sample_block(const SampleParams& p, uint32_t block, const PhiloxKeys& keys,
+                                             float* stage) {
   // the parameters may sit in global memory (batched launch): read the scalars once
   const uint32_t norm = p.norm, span = p.span, level_mask = p.level_mask, max_level = p.max_level;
   const uint32_t underflow = p.underflow, pbits = p.pbits, deterministic = p.deterministic;
@@ -344,7 +344,6 @@ __device__ __forceinline__ void sample_block(const SampleParams& p, uint32_t blo
   const uint32_t packed_kw = p.packed_kw, run_pitch = p.run_pitch, has_planes = p.has_planes;
   const uint32_t bk = p.bk, n_cb = p.n_cb, n_kb = p.n_kb;
   const uint32_t bk_shift = 31u - (uint32_t)__clz((int)bk), bk_mask = bk - 1u;     // bk is a power of two (32, 64, 128)
-  const PhiloxKeys keys(seed_lo, seed_hi);
   // Row sums of |W_k| (in units of 256, each weight rounded up) for the bound that lets the contraction
   // recombine its digit planes in 32 bits: gathered per block in shared memory, then added to the layer's words
   __shared__ uint32_t row_sum[kMaxLevels][kRowSumRows];
@@ -532,10 +531,11 @@ __device__ __forceinline__ void sample_block(const SampleParams& p, uint32_t blo
   }
 }
 
-__global__ void __launch_bounds__(kThreads) sample_kernel(const SampleParams p) {
+__global__ void __launch_bounds__(kThreads) sample_kernel(const __grid_constant__ SampleParams p,
+                                                          const __grid_constant__ PhiloxKeys keys) {
   pdl_prologue();
   __shared__ float stage[kStage];
-  sample_block(p, blockIdx.x, p.seed_lo, p.seed_hi, stage);
+  sample_block(p, blockIdx.x, keys, stage);
 }
 
 // All layers of a network in two launches.  Entry i owns blocks [first, first + count) of each
@@ -565,11 +565,11 @@ __global__ void __launch_bounds__(kThreads) emax_batch_kernel(const BatchEntry* 
 }
 
 __global__ void __launch_bounds__(kThreads) sample_batch_kernel(const BatchEntry* __restrict__ entries, uint32_t n,
-                                                                uint32_t seed_lo, uint32_t seed_hi) {
+                                                                const __grid_constant__ PhiloxKeys keys) {
   pdl_prologue();
   __shared__ float stage[kStage];
   const BatchEntry& e = entries[find_entry(entries, n, blockIdx.x, false)];
-  sample_block(e.p, blockIdx.x - e.sample_first, seed_lo, seed_hi, stage);
+  sample_block(e.p, blockIdx.x - e.sample_first, keys, stage);
 }
 
 // 128 * (sum of each filter row): the constant that restores sum x*W from sum (x-128)*W when
@@ -689,7 +689,7 @@ cudaError_t launch_sampler(const float* w_dev, psb_weights* wt, uint32_t* err_de
   SampleParams p;
   const uint32_t blocks = fill_sample_params(w_dev, wt, wt->e_max, p, false);
   p.e_tag = wt->e_calls;
-  launch_pdl(sample_kernel, blocks, kThreads, 0, s, p); note_launch();
+  launch_pdl(sample_kernel, blocks, kThreads, 0, s, p, PhiloxKeys(p.seed_lo, p.seed_hi)); note_launch();
   return cudaGetLastError();
 }
 
@@ -760,8 +760,8 @@ psb_status sample_batch_run(psb_ctx* ctx, psb_sample_batch* b, uint64_t seed, cu
     return PSB_ERR_CUDA;
   launch_pdl(emax_batch_kernel, b->emax_grid, kThreads, 0, s, (const BatchEntry*)b->entries_dev, b->n, ctx->err_dev);
   note_launch();
-  launch_pdl(sample_batch_kernel, b->sample_grid, kThreads, 0, s, (const BatchEntry*)b->entries_dev, b->n, (uint32_t)seed,
-             (uint32_t)(seed >> 32));
+  launch_pdl(sample_batch_kernel, b->sample_grid, kThreads, 0, s, (const BatchEntry*)b->entries_dev, b->n,
+             PhiloxKeys((uint32_t)seed, (uint32_t)(seed >> 32)));
   note_launch();
   return cudaGetLastError() == cudaSuccess ? PSB_OK : PSB_ERR_CUDA;
 }

@@ -223,6 +223,7 @@ cudaError_t launch_shift_add(const ConvArgs& a, const WintTable& wt, const uint3
                              cudaStream_t s);
 // gathers [M][kpad] signed bytes (x - offset; zero padding becomes -offset, K padding 0); row kh of the
 // filter window occupies bytes [kh * run_pitch, kh * run_pitch + kw * c) of a matrix row
+size_t im2col_s8_smem(const ConvArgs& a, uint32_t run_pitch);   // shared memory the gather kernel needs
 cudaError_t launch_im2col_s8(const ConvArgs& a, uint32_t kpad, uint32_t run_pitch, uint32_t offset, int8_t* dst,
                              uint32_t limit, cudaStream_t s);
 cudaError_t launch_corr128(const psb_weights* wt, uint32_t level, cudaStream_t s);

@@ -443,63 +443,101 @@ __global__ void range_check_kernel(const uint8_t* __restrict__ x, size_t bytes, 
 // [kh * run_pitch, kh * run_pitch + KW * C) of it, which in a channels-last image is one
 // contiguous run of the input row iy0 + kh; the rest of the matrix row is zero.  Values are
 // stored minus `offset` (0 or 128) as signed bytes; a padded input position is the value 0, i.e.
-// -offset.  A block handles kIm2colPix consecutive output locations of one output row: the KH
-// input-row spans they touch are staged in shared memory (contiguous copies, no index
-// arithmetic per byte), then each thread copies whole runs: aligned shared-memory words, a
-// funnel shift by the byte misalignment, 8-byte stores.
-constexpr uint32_t kIm2colPix = 32;
+// -offset.  A block handles a strip of up to kIm2colPix consecutive output locations of
+// kIm2colRows consecutive output rows: the input-row spans they touch are staged in shared
+// memory, each at the byte offset that keeps its 16-byte pieces aligned with global memory
+// (whole-piece copies; single bytes only at the image's edges), then each thread copies whole
+// runs: aligned shared-memory words, a funnel shift by the byte misalignment, 8-byte stores.
+constexpr uint32_t kIm2colPix = 128;
+constexpr uint32_t kIm2colRows = 2;
+
+__host__ __device__ __forceinline__ uint32_t im2col_span_pitch(uint32_t stride, uint32_t C, uint32_t run_pitch) {
+  // alignment shift (< 16) + the last pixel's run, read up to run_pitch + 7 bytes past its start in whole words
+  return (15u + (kIm2colPix - 1u) * stride * C + run_pitch + 12u + 15u) & ~15u;
+}
 
 __global__ void __launch_bounds__(256) im2col_s8_kernel(const ConvArgs a, uint32_t kpad, uint32_t run_pitch,
-                                                       uint32_t offset, uint32_t span_bytes, uint32_t span_pitch,
-                                                       uint32_t limit, int8_t* __restrict__ dst) {
+                                                       uint32_t offset, uint32_t limit, int8_t* __restrict__ dst) {
   pdl_prologue();
   bool bad = false;
-  extern __shared__ uint32_t im2col_smem[];                   // [KH][span_pitch / 4] words
+  extern __shared__ __align__(16) uint32_t im2col_smem[];     // [staged rows][span_pitch / 4] words
+  __shared__ uint32_t row_adj[(kIm2colRows - 1u) * 8u + 128u];   // per staged row: byte offset of the span's start
   uint8_t* rows = reinterpret_cast<uint8_t*>(im2col_smem);
+  const uint32_t span_pitch = im2col_span_pitch(a.stride, a.C, run_pitch);
   const uint32_t strips = (a.OW + kIm2colPix - 1) / kIm2colPix;
+  const uint32_t row_groups = (a.OH + kIm2colRows - 1) / kIm2colRows;
   const uint32_t strip = blockIdx.x % strips;
-  const uint32_t oy = (blockIdx.x / strips) % a.OH;
-  const uint32_t n = blockIdx.x / (strips * a.OH);
+  const uint32_t oy0 = ((blockIdx.x / strips) % row_groups) * kIm2colRows;
+  const uint32_t n = blockIdx.x / (strips * row_groups);
+  const uint32_t nrows = min(kIm2colRows, a.OH - oy0);
   const uint32_t ox0 = strip * kIm2colPix;
   const uint32_t npix = min(kIm2colPix, a.OW - ox0);
   const int ix0 = (int)(ox0 * a.stride) - (int)a.pad;         // leftmost input column of the strip
-  const int iy0 = (int)(oy * a.stride) - (int)a.pad;
+  const int iy0 = (int)(oy0 * a.stride) - (int)a.pad;         // topmost input row
+  const uint32_t staged = (nrows - 1u) * a.stride + a.KH;     // input rows the block touches
+  const uint32_t span_bytes = ((npix - 1u) * a.stride + a.KW) * a.C;
   const uint8_t* x = (const uint8_t*)a.x;
-  const uint8_t flip = (uint8_t)offset;                       // 0 or 0x80: v - 128 == v ^ 0x80 as a byte
-  const uint8_t fill = (uint8_t)(0u - offset);
+  const uint32_t flip = offset ? 0x80808080u : 0u;            // v - 128 == v ^ 0x80 as a byte
+  const uint32_t fill = (0u - offset) & 0xFFu;
+  const uint32_t fill4 = fill * 0x01010101u;
+  const uint32_t is_signed = a.in_dtype == PSB_DT_S8 ? 1u : 0u;
   // bytes [lo_b, hi_b) of a span lie inside the image row
   const int lo_b = ix0 < 0 ? -ix0 * (int)a.C : 0;
   const int hi_b = min((int)span_bytes, ((int)a.W - ix0) * (int)a.C);
-  for (uint32_t kh = threadIdx.x >> 6; kh < a.KH; kh += 4u) {
-    const int iy = iy0 + (int)kh;
+  const uint32_t pieces = span_pitch / 16u;
+  const uint32_t warp = threadIdx.x >> 5, lane = threadIdx.x & 31u;
+  for (uint32_t sr = warp; sr < staged; sr += 8u) {
+    const int iy = iy0 + (int)sr;
     const bool row_in = iy >= 0 && iy < (int)a.H;
     const uint8_t* src = x + (((size_t)n * a.H + (row_in ? iy : 0)) * a.W) * a.C + (ptrdiff_t)ix0 * (int)a.C;
-    for (uint32_t b = threadIdx.x & 63u; b < span_pitch; b += 64u) {
-      uint8_t v = fill;
-      if (row_in && (int)b >= lo_b && (int)b < hi_b) {
-        const uint8_t raw = src[b];
-        bad |= bytes_beyond((uint32_t)raw, a.in_dtype == PSB_DT_S8 ? 1u : 0u, limit);
-        v = (uint8_t)(raw ^ flip);
+    const uint32_t adj = (uint32_t)((uintptr_t)src & 15u);    // span byte b sits at shared byte adj + b
+    if (lane == 0) row_adj[sr] = adj;
+    const uint8_t* src16 = src - adj;                          // 16-byte aligned
+    uint32_t* out_row = im2col_smem + sr * (span_pitch / 4u);
+    for (uint32_t pc = lane; pc < pieces; pc += 32u) {
+      const int b0 = (int)(pc * 16u) - (int)adj;               // span byte of the piece's first byte
+      uint4 v;
+      if (row_in && b0 >= lo_b && b0 + 16 <= hi_b) {
+        v = __ldg(reinterpret_cast<const uint4*>(src16 + pc * 16u));
+        bad |= bytes_beyond(v.x, is_signed, limit) | bytes_beyond(v.y, is_signed, limit) |
+               bytes_beyond(v.z, is_signed, limit) | bytes_beyond(v.w, is_signed, limit);
+        v.x ^= flip; v.y ^= flip; v.z ^= flip; v.w ^= flip;
+      } else {
+        uint32_t wv[4] = {fill4, fill4, fill4, fill4};
+        if (row_in && b0 + 16 > lo_b && b0 < hi_b) {
+          for (int j = 0; j < 16; ++j) {
+            const int b = b0 + j;
+            if (b >= lo_b && b < hi_b) {
+              const uint32_t raw = src[b];
+              bad |= bytes_beyond(raw, is_signed, limit);
+              wv[j >> 2] = (wv[j >> 2] & ~(0xFFu << (8 * (j & 3)))) | (((raw ^ offset) & 0xFFu) << (8 * (j & 3)));
+            }
+          }
+        }
+        v = make_uint4(wv[0], wv[1], wv[2], wv[3]);
       }
-      rows[kh * span_pitch + b] = v;
+      *reinterpret_cast<uint4*>(out_row + pc * 4u) = v;
     }
   }
   if (bad) atomicOr(a.err, kDevErrRange);
   __syncthreads();
-  const size_t m0 = ((size_t)n * a.OH + oy) * a.OW + ox0;
   const uint32_t run = a.KW * a.C;                            // bytes of one filter row
   const uint32_t words = run_pitch / 4u;
   const uint32_t tail0 = a.KH * run_pitch;                    // zero bytes [tail0, kpad)
   const uint32_t items = a.KH + (kpad > tail0 ? 1u : 0u);
-  for (uint32_t t = threadIdx.x; t < npix * items; t += blockDim.x) {
-    const uint32_t px = t / items, kh = t - px * items;
-    int8_t* out = dst + (m0 + px) * kpad + kh * run_pitch;
+  const uint32_t per_row = npix * items;
+  for (uint32_t t = threadIdx.x; t < nrows * per_row; t += blockDim.x) {
+    const uint32_t ry = t / per_row, t1 = t - ry * per_row;
+    const uint32_t px = t1 / items, kh = t1 - px * items;
+    const size_t m = ((size_t)n * a.OH + oy0 + ry) * a.OW + ox0 + px;
+    int8_t* out = dst + m * kpad + kh * run_pitch;
     if (kh == a.KH) {
       for (uint32_t b = 0; b < kpad - tail0; b += 8u) *reinterpret_cast<uint2*>(out + b) = make_uint2(0u, 0u);
       continue;
     }
-    const uint32_t o = px * a.stride * a.C;                   // byte offset of the run in the staged span
-    const uint32_t* wsrc = im2col_smem + kh * (span_pitch / 4u) + (o >> 2);
+    const uint32_t sr = ry * a.stride + kh;
+    const uint32_t o = row_adj[sr] + px * a.stride * a.C;     // byte offset of the run in the staged row
+    const uint32_t* wsrc = im2col_smem + sr * (span_pitch / 4u) + (o >> 2);
     const uint32_t sh = (o & 3u) * 8u;
     uint32_t lo = wsrc[0];
     for (uint32_t w = 0; w < words; w += 2u) {
@@ -740,18 +778,19 @@ cudaError_t launch_shift_add(const ConvArgs& a, const WintTable& wt, const uint3
   return cudaGetLastError();
 }
 
+size_t im2col_s8_smem(const ConvArgs& a, uint32_t run_pitch) {
+  return (size_t)((kIm2colRows - 1u) * a.stride + a.KH) * im2col_span_pitch(a.stride, a.C, run_pitch);
+}
+
 cudaError_t launch_im2col_s8(const ConvArgs& a, uint32_t kpad, uint32_t run_pitch, uint32_t offset, int8_t* dst,
                              uint32_t limit, cudaStream_t s) {
   const uint32_t strips = (a.OW + kIm2colPix - 1) / kIm2colPix;
-  const uint32_t span_bytes = ((kIm2colPix - 1) * a.stride + a.KW) * a.C;
-  // a run may be read up to run_pitch + 7 bytes past its start (whole words, two at a time)
-  const uint32_t span_pitch = round_up((kIm2colPix - 1) * a.stride * a.C + run_pitch + 12u, 4u);
-  const size_t smem = (size_t)a.KH * span_pitch;
-  if (smem > 48 * 1024 || (uint64_t)a.N * a.OH * strips >= (1ull << 31) || run_pitch % 8u || kpad % 16u ||
-      (offset != 0u && offset != 128u) || a.KH * run_pitch > kpad)
+  const uint32_t row_groups = (a.OH + kIm2colRows - 1) / kIm2colRows;
+  const size_t smem = im2col_s8_smem(a, run_pitch);
+  if (smem > 48 * 1024 || (uint64_t)a.N * row_groups * strips >= (1ull << 31) || run_pitch % 8u || kpad % 16u ||
+      (offset != 0u && offset != 128u) || a.KH * run_pitch > kpad || (kIm2colRows - 1u) * a.stride + a.KH > 128u)
     return cudaErrorInvalidValue;
-  launch_pdl(im2col_s8_kernel, a.N * a.OH * strips, 256, smem, s, a, kpad, run_pitch, offset, span_bytes, span_pitch, limit,
-             dst);
+  launch_pdl(im2col_s8_kernel, a.N * row_groups * strips, 256, smem, s, a, kpad, run_pitch, offset, limit, dst);
   note_launch();
   return cudaGetLastError();
 }

@@ -1341,9 +1341,8 @@ psb_status tensor_supported(const psb_ctx* ctx, const psb_weights* wt, const Con
   // each plane accumulates in 32 bits: |digit| <= 127, |x| <= 128
   if ((uint64_t)wt->d * 127ull * 128ull >= (1ull << 31)) return PSB_ERR_UNSUPPORTED;
   if (wt->packed_k) {
-    // the gather kernel stages KH input-row segments of a 32-pixel strip in 48 KB of shared memory
-    const uint64_t stage = (uint64_t)a.KH * (31ull * a.stride * a.C + wt->run_pitch + 16u);
-    return stage > 48u * 1024u ? PSB_ERR_UNSUPPORTED : PSB_OK;
+    // the gather kernel stages the input-row segments of a strip of output locations in 48 KB of shared memory
+    return (a.KH > 120u || im2col_s8_smem(a, wt->run_pitch) > 48u * 1024u) ? PSB_ERR_UNSUPPORTED : PSB_OK;
   }
   if (a.C % 16u || a.C < 32u) return PSB_ERR_UNSUPPORTED;
   if ((uintptr_t)a.x & 15u) return PSB_ERR_UNSUPPORTED;

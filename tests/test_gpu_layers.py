@@ -161,6 +161,8 @@ def test_tensor_path_layers(psb, ctx, oracle, case):
     dict(N=2, C=3, H=30, W=30, O=32, K=3, stride=2, pad=1, dtype=np.uint8, hi=256),   # 27 -> 32 columns
     dict(N=2, C=24, H=13, W=13, O=40, K=1, stride=1, pad=0, dtype=np.int8, hi=128),   # 24 channels, signed
     dict(N=2, C=20, H=11, W=9, O=70, K=3, stride=1, pad=1, dtype=np.uint8, hi=256),   # ragged everything
+    dict(N=1, C=3, H=21, W=300, O=16, K=5, stride=2, pad=2, dtype=np.uint8, hi=256),  # two strips of output columns, odd row count
+    dict(N=2, C=5, H=9, W=140, O=16, K=3, stride=1, pad=1, dtype=np.int8, hi=128),    # rows that start at odd byte addresses
 ])
 def test_tensor_path_few_input_channels_full_range_bytes(psb, ctx, oracle, case):
     """Filters whose input-channel count is not a multiple of 16 run on the tensor cores through an

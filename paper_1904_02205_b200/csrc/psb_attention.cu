@@ -15,7 +15,7 @@ namespace {
 // 256 (u8) / 511 (s8 differences) arguments: a table in shared memory, exp(-j * step) for j = 0.., filled
 // once per block; the two sums of a location are then table look-ups and multiply-adds:
 //   z_c = (q_c - q_max) * step <= 0,  S = sum exp(z_c),  T = sum z_c exp(z_c),  h = log S - T / S.
-__global__ void __launch_bounds__(256) entropy_kernel(const uint8_t* __restrict__ act, uint32_t is_signed,
+__global__ void __launch_bounds__(256) entropy_kernel(const uint8_t* act, uint32_t is_signed,
                                                       uint32_t locations, uint32_t C, float step,
                                                       float* __restrict__ entropy) {
   pdl_prologue();
@@ -55,7 +55,7 @@ struct MapTable {
 };
 
 // One block per image: mean entropy (fixed summation order), threshold, maps of every resolution.
-__global__ void __launch_bounds__(256) attention_maps_kernel(const float* __restrict__ entropy, uint32_t H, uint32_t W,
+__global__ void __launch_bounds__(256) attention_maps_kernel(const float* entropy, uint32_t H, uint32_t W,
                                                              uint32_t lo_log2k, uint32_t hi_log2k, uint32_t n_res,
                                                              const MapTable maps, float* __restrict__ mean_out) {
   pdl_prologue();

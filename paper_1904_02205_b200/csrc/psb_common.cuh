@@ -185,6 +185,14 @@ __device__ __forceinline__ float acc_to_float_small(long long acc) {
 // kernel before it in the stream is still running; it must call pdl_prologue() before it touches
 // global memory, which waits for the earlier grids to complete (and lets the kernel after it be
 // scheduled in turn).  What is saved is the launch latency between the many short kernels of a step.
+//
+// Rule for such kernels: whatever an earlier kernel of the stream may have written (activations, integer
+// filters and their row sums, the sorted order of a draw-count map, scratch matrices) is read with ordinary
+// loads (plain, __ldca, __ldcg), never through the read-only path (__ldg, or a const __restrict__ kernel
+// parameter, which the compiler turns into the same instruction).  That path promises data that does not
+// change during the kernel's lifetime, which here begins before the earlier kernel has finished: the compiler
+// may move such a load above the wait in pdl_prologue().  (Seen once: a gather that read the number of sorted
+// tiles before the sorting kernel had written it.)
 #ifdef __CUDACC__
 __device__ __forceinline__ void pdl_prologue() {
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");

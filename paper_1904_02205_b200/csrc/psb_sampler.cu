@@ -574,7 +574,7 @@ __global__ void __launch_bounds__(kThreads) sample_batch_kernel(const BatchEntry
 
 // 128 * (sum of each filter row): the constant that restores sum x*W from sum (x-128)*W when
 // unsigned activations are fed to the signed MMA with an offset of 128.  One warp per row.
-__global__ void corr128_kernel(const int32_t* __restrict__ wint, uint32_t O, uint32_t d,
+__global__ void corr128_kernel(const int32_t* wint, uint32_t O, uint32_t d,
                                long long* __restrict__ corr) {
   pdl_prologue();
   const uint32_t row = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31u;

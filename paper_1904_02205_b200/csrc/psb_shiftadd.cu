@@ -57,7 +57,7 @@ __global__ void __launch_bounds__(256) conv_direct_kernel(const ConvArgs a, cons
       atomicOr(a.err, kDevErrBadLevel);
       continue;
     }
-    const int32_t* __restrict__ w = wt.w[level] + (size_t)o * a.KH * a.KW * Cg;
+    const int32_t* w = wt.w[level] + (size_t)o * a.KH * a.KW * Cg;
     const uint32_t cbase = (o / Og) * Cg;
     long long acc = 0;
     for (uint32_t kh = 0; kh < a.KH; ++kh) {
@@ -70,7 +70,7 @@ __global__ void __launch_bounds__(256) conv_direct_kernel(const ConvArgs a, cons
         const int32_t* wr = w + (size_t)(kh * a.KW + kw) * Cg;
         for (uint32_t ci = 0; ci < Cg; ++ci) {
           int xv = load_act(a.x, a.in_dtype, xoff + ci);
-          acc += (long long)xv * (long long)__ldg(wr + ci);
+          acc += (long long)xv * (long long)__ldca(wr + ci);
         }
       }
     }
@@ -96,11 +96,11 @@ __global__ void __launch_bounds__(256) gemv_warp_kernel(const ConvArgs a, const 
       if (lane == 0) atomicOr(a.err, kDevErrBadLevel);
       continue;
     }
-    const int32_t* __restrict__ w = wt.w[level] + (size_t)o * a.C;
+    const int32_t* w = wt.w[level] + (size_t)o * a.C;
     const size_t xoff = (size_t)n * a.C;
     long long acc = 0;
     for (uint32_t ci = lane; ci < a.C; ci += 32u)
-      acc += (long long)load_act(a.x, a.in_dtype, xoff + ci) * (long long)__ldg(w + ci);
+      acc += (long long)load_act(a.x, a.in_dtype, xoff + ci) * (long long)__ldca(w + ci);
 #pragma unroll
     for (int d = 16; d > 0; d >>= 1) acc += __shfl_down_sync(0xFFFFFFFFu, acc, d);
     if (lane == 0) store_outputs(a, idx, o, level, acc);
@@ -111,7 +111,7 @@ __global__ void __launch_bounds__(256) gemv_warp_kernel(const ConvArgs a, const 
 // the layer: a thread owns 8 consecutive channels of one output location.  The block keeps the
 // layer's integer filter in shared memory as [tap][channel]; activations come in 8-byte loads;
 // the integer sum x * W_k over the taps is Eq. 9 summed over the draws.  Writes 8 codes at once.
-__global__ void __launch_bounds__(256) dwconv_nhwc8_kernel(const ConvArgs a, const int32_t* __restrict__ wint) {
+__global__ void __launch_bounds__(256) dwconv_nhwc8_kernel(const ConvArgs a, const int32_t* wint) {
   pdl_prologue();
   extern __shared__ int32_t dw_w[];   // [KH*KW][C]
   const uint32_t taps = a.KH * a.KW, C = a.C;
@@ -135,7 +135,7 @@ __global__ void __launch_bounds__(256) dwconv_nhwc8_kernel(const ConvArgs a, con
       for (uint32_t kw = 0; kw < a.KW; ++kw) {
         const int ix = (int)(ox * a.stride + kw) - (int)a.pad;
         if (ix < 0 || ix >= (int)a.W) continue;
-        const uint2 xv = __ldg(reinterpret_cast<const uint2*>(
+        const uint2 xv = __ldcg(reinterpret_cast<const uint2*>(
             (const uint8_t*)a.x + (((size_t)n * a.H + iy) * a.W + ix) * C + c0));
         const int32_t* wr = dw_w + (kh * a.KW + kw) * C + c0;
         const int4 w0 = *reinterpret_cast<const int4*>(wr), w1 = *reinterpret_cast<const int4*>(wr + 4);
@@ -152,7 +152,7 @@ __global__ void __launch_bounds__(256) dwconv_nhwc8_kernel(const ConvArgs a, con
     const size_t oidx = pix * C + c0;
     uint32_t rw[2] = {0, 0};
     if (has_res) {
-      const uint2 rv = __ldg(reinterpret_cast<const uint2*>((const uint8_t*)a.residual + oidx));
+      const uint2 rv = __ldcg(reinterpret_cast<const uint2*>((const uint8_t*)a.residual + oidx));
       rw[0] = rv.x; rw[1] = rv.y;
     }
     uint32_t qw[2] = {0, 0};
@@ -182,7 +182,7 @@ template <int S>
 struct DwSeg { static constexpr int kOut = S == 1 ? 8 : 4; static constexpr int kCols = (kOut - 1) * S + 3; };
 
 template <int S, bool kSignedIn>
-__global__ void __launch_bounds__(256, 2) dwconv3x3_row_kernel(const ConvArgs a, const int32_t* __restrict__ wint) {
+__global__ void __launch_bounds__(256, 2) dwconv3x3_row_kernel(const ConvArgs a, const int32_t* wint) {
   pdl_prologue();
   constexpr int L = DwSeg<S>::kOut, NC = DwSeg<S>::kCols;
   const uint32_t C = a.C, G = C / 4u;
@@ -211,7 +211,7 @@ __global__ void __launch_bounds__(256, 2) dwconv3x3_row_kernel(const ConvArgs a,
       const int ix = ix0 + cidx;
       raw[r][cidx] = 0u;
       if (row_in && (unsigned)ix < a.W && ix <= ix_end)
-        raw[r][cidx] = __ldg(reinterpret_cast<const uint32_t*>(rp + (size_t)ix * C));
+        raw[r][cidx] = __ldcg(reinterpret_cast<const uint32_t*>(rp + (size_t)ix * C));
     }
   }
   // filter [channel][tap] and output constants of the 4 channels
@@ -220,7 +220,7 @@ __global__ void __launch_bounds__(256, 2) dwconv3x3_row_kernel(const ConvArgs a,
     const int4* wp = reinterpret_cast<const int4*>(wint + (size_t)c0 * 9u);
 #pragma unroll
     for (int i = 0; i < 9; ++i) {
-      const int4 v = __ldg(wp + i);
+      const int4 v = __ldca(wp + i);
       w[4 * i] = v.x; w[4 * i + 1] = v.y; w[4 * i + 2] = v.z; w[4 * i + 3] = v.w;
     }
   }
@@ -242,7 +242,7 @@ __global__ void __launch_bounds__(256, 2) dwconv3x3_row_kernel(const ConvArgs a,
     if (ox0 + i > last_ox) break;
     const size_t oidx = obase + (size_t)i * C;
     uint32_t rv = 0u;
-    if (has_res) rv = __ldg(reinterpret_cast<const uint32_t*>((const uint8_t*)a.residual + oidx));
+    if (has_res) rv = __ldcg(reinterpret_cast<const uint32_t*>((const uint8_t*)a.residual + oidx));
     long long acc[4] = {0, 0, 0, 0};
 #pragma unroll
     for (int r = 0; r < 3; ++r) {
@@ -292,7 +292,7 @@ template <>
 __device__ __forceinline__ float dw_acc_to_float<long long>(long long acc) { return acc_to_float(acc); }
 
 template <int S, bool kSignedIn, typename Acc>
-__device__ __forceinline__ void dw_channel(const uint32_t (&raw)[3][DwSeg<S>::kCols], int j, const int32_t* __restrict__ wch,
+__device__ __forceinline__ void dw_channel(const uint32_t (&raw)[3][DwSeg<S>::kCols], int j, const int32_t* wch,
                                            float sc, float bi, bool has_res, const uint32_t (&rv)[DwSeg<S>::kOut],
                                            bool res_signed, float res_scale, float relu_floor, float inv_step,
                                            float lo_f, float hi_f, uint32_t n_out, uint32_t (&qw)[DwSeg<S>::kOut]) {
@@ -302,7 +302,7 @@ __device__ __forceinline__ void dw_channel(const uint32_t (&raw)[3][DwSeg<S>::kC
   for (int i = 0; i < L; ++i) acc[i] = 0;
 #pragma unroll
   for (int r = 0; r < 3; ++r) {
-    const int w0 = __ldg(wch + r * 3), w1 = __ldg(wch + r * 3 + 1), w2 = __ldg(wch + r * 3 + 2);
+    const int w0 = __ldca(wch + r * 3), w1 = __ldca(wch + r * 3 + 1), w2 = __ldca(wch + r * 3 + 2);
     int xb[NC];
 #pragma unroll
     for (int cidx = 0; cidx < NC; ++cidx) {
@@ -332,8 +332,8 @@ __device__ __forceinline__ void dw_channel(const uint32_t (&raw)[3][DwSeg<S>::kC
 }
 
 template <int S, bool kSignedIn>
-__global__ void __launch_bounds__(256, 2) dwconv3x3_row32_kernel(const ConvArgs a, const int32_t* __restrict__ wint,
-                                                                 const uint32_t* __restrict__ rowsum256,
+__global__ void __launch_bounds__(256, 2) dwconv3x3_row32_kernel(const ConvArgs a, const int32_t* wint,
+                                                                 const uint32_t* rowsum256,
                                                                  uint32_t amax) {
   pdl_prologue();
   constexpr int L = DwSeg<S>::kOut, NC = DwSeg<S>::kCols;
@@ -363,7 +363,7 @@ __global__ void __launch_bounds__(256, 2) dwconv3x3_row32_kernel(const ConvArgs 
       const int ix = ix0 + cidx;
       raw[r][cidx] = 0u;
       if (row_in && (unsigned)ix < a.W && ix <= ix_end)
-        raw[r][cidx] = __ldg(reinterpret_cast<const uint32_t*>(rp + (size_t)ix * C));
+        raw[r][cidx] = __ldcg(reinterpret_cast<const uint32_t*>(rp + (size_t)ix * C));
     }
   }
   const bool has_res = a.residual != nullptr;
@@ -375,7 +375,7 @@ __global__ void __launch_bounds__(256, 2) dwconv3x3_row32_kernel(const ConvArgs 
     qw[i] = 0u;
     rv[i] = 0u;
     if (has_res && (uint32_t)i < n_out)
-      rv[i] = __ldg(reinterpret_cast<const uint32_t*>((const uint8_t*)a.residual + obase + (size_t)i * C));
+      rv[i] = __ldcg(reinterpret_cast<const uint32_t*>((const uint8_t*)a.residual + obase + (size_t)i * C));
   }
   const float relu_floor = a.relu ? 0.0f : __int_as_float(0xFF800000);
   const float lo_f = (float)a.qmin, hi_f = (float)a.qmax;
@@ -387,7 +387,7 @@ __global__ void __launch_bounds__(256, 2) dwconv3x3_row32_kernel(const ConvArgs 
     const float sc = ldexpf(a.scale[o], a.e_base[o] - (int)level), bi = a.bias[o];
     const int32_t* wch = wint + (size_t)o * 9u;
     // (a sum marked unknown, 0xFFFFFFFF, fails the test like a large one)
-    const unsigned long long bound = (unsigned long long)__ldg(rowsum256 + (size_t)level * a.O + o) * 256ull * amax;
+    const unsigned long long bound = (unsigned long long)__ldca(rowsum256 + (size_t)level * a.O + o) * 256ull * amax;
     if (bound < (1ull << 31))
       dw_channel<S, kSignedIn, int>(raw, j, wch, sc, bi, has_res, rv, res_signed, a.residual_scale, relu_floor,
                                     a.inv_step, lo_f, hi_f, n_out, qw);
@@ -401,12 +401,12 @@ __global__ void __launch_bounds__(256, 2) dwconv3x3_row32_kernel(const ConvArgs 
 }
 
 // x ^ 0x80 over a whole tensor: unsigned bytes become (x - 128) as signed bytes, 16 per thread.
-__global__ void offset128_kernel(const uint4* __restrict__ src, uint4* __restrict__ dst, size_t n16, uint32_t limit,
+__global__ void offset128_kernel(const uint4* src, uint4* dst, size_t n16, uint32_t limit,
                                  uint32_t* __restrict__ err) {
   pdl_prologue();
   bool bad = false;
   for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n16; i += (size_t)gridDim.x * blockDim.x) {
-    uint4 v = __ldg(src + i);
+    uint4 v = __ldcg(src + i);
     if (limit < 255u)
       bad |= bytes_beyond(v.x, 0u, limit) | bytes_beyond(v.y, 0u, limit) | bytes_beyond(v.z, 0u, limit) |
              bytes_beyond(v.w, 0u, limit);
@@ -418,7 +418,7 @@ __global__ void offset128_kernel(const uint4* __restrict__ src, uint4* __restric
 
 // Largest byte magnitude of a tensor against the bound the caller gave (PSB_CHECK_RANGE): 16 bytes per
 // thread and iteration, the ragged tail byte by byte.
-__global__ void range_check_kernel(const uint8_t* __restrict__ x, size_t bytes, uint32_t is_signed, uint32_t limit,
+__global__ void range_check_kernel(const uint8_t* x, size_t bytes, uint32_t is_signed, uint32_t limit,
                                    uint32_t* __restrict__ err) {
   pdl_prologue();
   bool bad = false;
@@ -426,7 +426,7 @@ __global__ void range_check_kernel(const uint8_t* __restrict__ x, size_t bytes, 
   const size_t n16 = (bytes - head) / 16u;
   const uint4* x16 = reinterpret_cast<const uint4*>(x + head);
   for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n16; i += (size_t)gridDim.x * blockDim.x) {
-    const uint4 v = __ldg(x16 + i);
+    const uint4 v = __ldcg(x16 + i);
     bad |= bytes_beyond(v.x, is_signed, limit) | bytes_beyond(v.y, is_signed, limit) |
            bytes_beyond(v.z, is_signed, limit) | bytes_beyond(v.w, is_signed, limit);
   }
@@ -498,7 +498,7 @@ __global__ void __launch_bounds__(256) im2col_s8_kernel(const ConvArgs a, uint32
       const int b0 = (int)(pc * 16u) - (int)adj;               // span byte of the piece's first byte
       uint4 v;
       if (row_in && b0 >= lo_b && b0 + 16 <= hi_b) {
-        v = __ldg(reinterpret_cast<const uint4*>(src16 + pc * 16u));
+        v = __ldcg(reinterpret_cast<const uint4*>(src16 + pc * 16u));
         bad |= bytes_beyond(v.x, is_signed, limit) | bytes_beyond(v.y, is_signed, limit) |
                bytes_beyond(v.z, is_signed, limit) | bytes_beyond(v.w, is_signed, limit);
         v.x ^= flip; v.y ^= flip; v.z ^= flip; v.w ^= flip;
@@ -554,7 +554,7 @@ __global__ void __launch_bounds__(256) im2col_s8_kernel(const ConvArgs a, uint32
 }
 
 // [N][C][HW] -> [N][HW][C], elements of 1 byte, through a 32x33 tile.
-__global__ void nchw_to_nhwc_u8_kernel(const uint8_t* __restrict__ src, uint8_t* __restrict__ dst,
+__global__ void nchw_to_nhwc_u8_kernel(const uint8_t* src, uint8_t* dst,
                                        uint32_t C, uint32_t HW, uint32_t is_signed, uint32_t limit,
                                        uint32_t* __restrict__ err) {
   pdl_prologue();
@@ -584,7 +584,7 @@ __global__ void nchw_to_nhwc_u8_kernel(const uint8_t* __restrict__ src, uint8_t*
 // per location, 4 channels each) in shared memory with one 16-byte store.  Then 8 consecutive
 // lanes write the 32 channel bytes of one location: whole 32-byte sectors, no bank conflicts
 // (row pitch 132 words: bank = 4 * quad + location).
-__global__ void __launch_bounds__(256) nchw_to_nhwc_u8x4_kernel(const uint8_t* __restrict__ src,
+__global__ void __launch_bounds__(256) nchw_to_nhwc_u8x4_kernel(const uint8_t* src,
                                                                uint8_t* __restrict__ dst, uint32_t C,
                                                                uint32_t HW, uint32_t is_signed, uint32_t limit,
                                                                uint32_t* __restrict__ err) {
@@ -599,7 +599,7 @@ __global__ void __launch_bounds__(256) nchw_to_nhwc_u8x4_kernel(const uint8_t* _
     if (c < C && p < HW) {
 #pragma unroll
       for (int k = 0; k < 4; ++k)
-        r[k] = __ldg(reinterpret_cast<const uint32_t*>(src + base + (size_t)(c + k) * HW + p));
+        r[k] = __ldcg(reinterpret_cast<const uint32_t*>(src + base + (size_t)(c + k) * HW + p));
       if (bytes_beyond(r[0], is_signed, limit) | bytes_beyond(r[1], is_signed, limit) |
           bytes_beyond(r[2], is_signed, limit) | bytes_beyond(r[3], is_signed, limit))
         atomicOr(err, kDevErrRange);
@@ -620,7 +620,7 @@ __global__ void __launch_bounds__(256) nchw_to_nhwc_u8x4_kernel(const uint8_t* _
   }
 }
 
-__global__ void maxpool_kernel(const uint8_t* __restrict__ x, uint32_t nchw, uint32_t N, uint32_t C,
+__global__ void maxpool_kernel(const uint8_t* x, uint32_t nchw, uint32_t N, uint32_t C,
                                uint32_t H, uint32_t W, uint32_t k, uint32_t stride, uint32_t pad,
                                uint32_t OH, uint32_t OW, uint8_t* __restrict__ out) {
   pdl_prologue();
@@ -652,7 +652,7 @@ __global__ void maxpool_kernel(const uint8_t* __restrict__ x, uint32_t nchw, uin
 }
 
 // Channels-last max-pooling, 16 channels per thread: 16-byte loads, byte-wise maxima.
-__global__ void __launch_bounds__(256) maxpool_nhwc16_kernel(const uint8_t* __restrict__ x, uint32_t N, uint32_t C,
+__global__ void __launch_bounds__(256) maxpool_nhwc16_kernel(const uint8_t* x, uint32_t N, uint32_t C,
                                                             uint32_t H, uint32_t W, uint32_t k, uint32_t stride,
                                                             uint32_t pad, uint32_t OH, uint32_t OW,
                                                             uint8_t* __restrict__ out) {
@@ -672,7 +672,7 @@ __global__ void __launch_bounds__(256) maxpool_nhwc16_kernel(const uint8_t* __re
       for (uint32_t kw = 0; kw < k; ++kw) {
         const int ix = (int)(ox * stride + kw) - (int)pad;
         if (ix < 0 || ix >= (int)W) continue;
-        const uint4 v = __ldg(reinterpret_cast<const uint4*>(x + (((size_t)n * H + iy) * W + ix) * C + g * 16u));
+        const uint4 v = __ldcg(reinterpret_cast<const uint4*>(x + (((size_t)n * H + iy) * W + ix) * C + g * 16u));
         best.x = __vmaxu4(best.x, v.x); best.y = __vmaxu4(best.y, v.y);
         best.z = __vmaxu4(best.z, v.z); best.w = __vmaxu4(best.w, v.w);
       }
@@ -682,7 +682,7 @@ __global__ void __launch_bounds__(256) maxpool_nhwc16_kernel(const uint8_t* __re
 }
 
 // One warp per (n, c): integer sum over H*W, then one re-quantisation.
-__global__ void avgpool_kernel(const uint8_t* __restrict__ x, uint32_t nchw, uint32_t N, uint32_t C,
+__global__ void avgpool_kernel(const uint8_t* x, uint32_t nchw, uint32_t N, uint32_t C,
                                uint32_t HW, float pool_mul, int qmin, int qmax,
                                uint8_t* __restrict__ out) {
   pdl_prologue();

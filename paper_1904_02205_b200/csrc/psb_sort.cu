@@ -31,7 +31,7 @@ namespace {
 
 // Histogram of the map; the last block to finish turns it into the padded run starts.  Also marks the whole
 // permutation as padding, which the scatter pass then overwrites where a location lands.
-__global__ void __launch_bounds__(256) level_count_kernel(const uint8_t* __restrict__ kmap, uint32_t M,
+__global__ void __launch_bounds__(256) level_count_kernel(const uint8_t* kmap, uint32_t M,
                                                           SortCtl* __restrict__ ctl, uint32_t* __restrict__ perm,
                                                           uint32_t perm_words) {
   pdl_prologue();
@@ -66,7 +66,7 @@ __global__ void __launch_bounds__(256) level_count_kernel(const uint8_t* __restr
 // perm[sorted row] = location.  Lanes of a warp that share a level take consecutive slots, so the order of
 // the locations is kept within a warp (neighbouring locations stay neighbours in memory).  Also writes the
 // level of every tile as a one-bit mask (0 for tiles beyond the last run).
-__global__ void __launch_bounds__(256) level_scatter_kernel(const uint8_t* __restrict__ kmap, uint32_t M,
+__global__ void __launch_bounds__(256) level_scatter_kernel(const uint8_t* kmap, uint32_t M,
                                                             SortCtl* __restrict__ ctl, uint32_t* __restrict__ perm,
                                                             uint8_t* __restrict__ tile_mask, uint32_t max_tiles) {
   pdl_prologue();
@@ -93,33 +93,56 @@ __global__ void __launch_bounds__(256) level_scatter_kernel(const uint8_t* __res
 
 // Activation rows in sorted order: row r of the matrix is the patch of location perm[r], K index
 // (kh * KW + kw) * cpad + ci (cpad >= C bytes per tap, the rest zero); positions outside the image are zero.
-// A group of `lanes_per_item` lanes copies the C bytes of one (row, tap) in 16-byte pieces.
-__global__ void __launch_bounds__(256) gather_sorted_kernel(const ConvArgs a, const uint32_t* __restrict__ perm,
-                                                            const SortCtl* __restrict__ ctl, uint32_t cpad,
-                                                            uint32_t lanes_per_item, uint8_t* __restrict__ dst) {
+// A group of `lanes_per_row` lanes copies the patches of kGatherRows rows at a time, tap by tap, in 16-byte
+// pieces: the loads of the rows are issued together, then their stores (a copy with one load in flight per
+// thread, behind the lookup of its row, reached a third of the memory bandwidth).
+constexpr int kGatherRows = 4;
+
+__global__ void __launch_bounds__(256) gather_sorted_kernel(const ConvArgs a, const uint32_t* perm,
+                                                            const SortCtl* ctl, uint32_t cpad,
+                                                            uint32_t lanes_per_row, uint8_t* __restrict__ dst) {
   pdl_prologue();
   const uint32_t taps = a.KH * a.KW, pitch = taps * cpad;
-  const uint32_t rows = ctl->tiles * kTileRows;
-  const uint32_t items_per_block = blockDim.x / lanes_per_item;
-  const uint32_t sub = threadIdx.x % lanes_per_item, slot = threadIdx.x / lanes_per_item;
-  const unsigned long long items = (unsigned long long)rows * taps;
+  const uint32_t rows = __ldcg(&ctl->tiles) * kTileRows;
+  const uint32_t slots = blockDim.x / lanes_per_row;
+  const uint32_t sub = threadIdx.x % lanes_per_row, slot = threadIdx.x / lanes_per_row;
   const uint32_t ohow = a.OH * a.OW;
   const uint8_t* x = (const uint8_t*)a.x;
-  for (unsigned long long it = (unsigned long long)blockIdx.x * items_per_block + slot; it < items;
-       it += (unsigned long long)gridDim.x * items_per_block) {
-    const uint32_t r = (uint32_t)(it / taps), tap = (uint32_t)(it - (unsigned long long)r * taps);
-    const uint32_t m = perm[r];
-    if (m == 0xFFFFFFFFu) continue;                     // padding row: never stored by the output stage
-    const uint32_t n = m / ohow, pix = m - n * ohow, oy = pix / a.OW, ox = pix - oy * a.OW;
-    const uint32_t kh = tap / a.KW, kw = tap - kh * a.KW;
-    const int iy = (int)(oy * a.stride + kh) - (int)a.pad, ix = (int)(ox * a.stride + kw) - (int)a.pad;
-    const bool inside = (unsigned)iy < a.H && (unsigned)ix < a.W;
-    const uint8_t* src = x + (((size_t)n * a.H + (inside ? iy : 0)) * a.W + (inside ? ix : 0)) * a.C;
-    uint8_t* out = dst + (size_t)r * pitch + (size_t)tap * cpad;
-    for (uint32_t b = sub * 16u; b < cpad; b += lanes_per_item * 16u) {
-      uint4 v = make_uint4(0u, 0u, 0u, 0u);
-      if (inside && b < a.C) v = __ldg(reinterpret_cast<const uint4*>(src + b));
-      *reinterpret_cast<uint4*>(out + b) = v;
+  const uint32_t step = gridDim.x * slots;              // rows between the rows of one thread
+  for (uint32_t r0 = blockIdx.x * slots + slot; r0 < rows; r0 += step * (uint32_t)kGatherRows) {
+    // the rows of this round: image base, input coordinates of the filter's first tap, whether the row is real
+    const uint8_t* img[kGatherRows];
+    uint8_t* out[kGatherRows];
+    int y0[kGatherRows], x0[kGatherRows];
+    bool live[kGatherRows];
+#pragma unroll
+    for (int u = 0; u < kGatherRows; ++u) {
+      const uint32_t r = r0 + (uint32_t)u * step;
+      const uint32_t m = r < rows ? __ldcg(perm + r) : 0xFFFFFFFFu;
+      live[u] = m != 0xFFFFFFFFu;                       // padding rows are never stored by the output stage
+      const uint32_t mm = live[u] ? m : 0u;
+      const uint32_t n = mm / ohow, pix = mm - n * ohow, oy = pix / a.OW, ox = pix - oy * a.OW;
+      img[u] = x + (size_t)n * a.H * a.W * a.C;
+      y0[u] = (int)(oy * a.stride) - (int)a.pad;
+      x0[u] = (int)(ox * a.stride) - (int)a.pad;
+      out[u] = dst + (size_t)(live[u] ? r : 0u) * pitch;
+    }
+    uint32_t kh = 0, kw = 0;
+    for (uint32_t tap = 0; tap < taps; ++tap) {
+      for (uint32_t b = sub * 16u; b < cpad; b += lanes_per_row * 16u) {
+        uint4 v[kGatherRows];
+#pragma unroll
+        for (int u = 0; u < kGatherRows; ++u) {
+          const int iy = y0[u] + (int)kh, ix = x0[u] + (int)kw;
+          const bool inside = live[u] && (unsigned)iy < a.H && (unsigned)ix < a.W && b < a.C;
+          v[u] = make_uint4(0u, 0u, 0u, 0u);
+          if (inside) v[u] = __ldcg(reinterpret_cast<const uint4*>(img[u] + ((size_t)iy * a.W + (uint32_t)ix) * a.C + b));
+        }
+#pragma unroll
+        for (int u = 0; u < kGatherRows; ++u)
+          if (live[u]) *reinterpret_cast<uint4*>(out[u] + (size_t)tap * cpad + b) = v[u];
+      }
+      if (++kw == a.KW) { kw = 0; ++kh; }
     }
   }
 }
@@ -148,8 +171,9 @@ cudaError_t launch_gather_sorted(const ConvArgs& a, const uint32_t* perm, const 
                                  cudaStream_t s) {
   uint32_t lanes = 1;
   while (lanes < 32u && lanes * 16u < cpad) lanes *= 2u;
-  const uint64_t items = (uint64_t)sorted_tiles_bound((uint64_t)a.N * a.OH * a.OW) * kTileRows * a.KH * a.KW;
-  uint64_t blocks = (items * lanes + 255u) / 256u;
+  const uint64_t rows = (uint64_t)sorted_tiles_bound((uint64_t)a.N * a.OH * a.OW) * kTileRows;
+  const uint32_t rows_per_block = (256u / lanes) * (uint32_t)kGatherRows;
+  uint64_t blocks = (rows + rows_per_block - 1) / rows_per_block;
   if (blocks > 148u * 16u) blocks = 148u * 16u;
   if (blocks < 1u) blocks = 1u;
   launch_pdl(gather_sorted_kernel, (uint32_t)blocks, 256, 0, s, a, perm, (const SortCtl*)ctl, cpad, lanes, dst);

@@ -438,7 +438,7 @@ __device__ __noinline__ uint4 load_planar16(const uint8_t* src, size_t plane, ui
   uint32_t w[4] = {0u, 0u, 0u, 0u};
 #pragma unroll
   for (int j = 0; j < 16; ++j)
-    if ((uint32_t)j < count) w[j >> 2] |= (uint32_t)__ldg(src + (size_t)j * plane) << (8 * (j & 3));
+    if ((uint32_t)j < count) w[j >> 2] |= (uint32_t)__ldcg(src + (size_t)j * plane) << (8 * (j & 3));
   return make_uint4(w[0], w[1], w[2], w[3]);
 }
 template <int TAG>
@@ -641,7 +641,7 @@ struct RowMapSorted {
     perm = p.perm; O = p.a.O; ohow = p.a.OH * p.a.OW; planar = p.a.out_nchw;
   }
   __device__ __forceinline__ uint32_t row_index(uint32_t m_tile, uint32_t row, bool* valid) const {
-    const uint32_t m = __ldg(perm + (size_t)m_tile * kTileM + row);
+    const uint32_t m = __ldcg(perm + (size_t)m_tile * kTileM + row);
     *valid = m != 0xFFFFFFFFu;
     return m;
   }

@@ -332,7 +332,7 @@ __device__ __forceinline__ void dw_channel(const uint32_t (&raw)[3][DwSeg<S>::kC
 }
 
 template <int S, bool kSignedIn>
-__global__ void __launch_bounds__(256, 2) dwconv3x3_row32_kernel(const ConvArgs a, const int32_t* wint,
+__global__ void __launch_bounds__(256, 3) dwconv3x3_row32_kernel(const ConvArgs a, const int32_t* wint,
                                                                  const uint32_t* rowsum256,
                                                                  uint32_t amax) {
   pdl_prologue();
@@ -682,6 +682,33 @@ __global__ void __launch_bounds__(256) maxpool_nhwc16_kernel(const uint8_t* x, u
 }
 
 // One warp per (n, c): integer sum over H*W, then one re-quantisation.
+// Channels-last, 16 channels per thread: every load is 16 bytes, neighbouring threads read neighbouring
+// channel groups of the same position.
+__global__ void __launch_bounds__(128) avgpool_nhwc16_kernel(const uint8_t* x, uint32_t N, uint32_t C, uint32_t HW,
+                                                             float pool_mul, int qmin, int qmax, uint8_t* __restrict__ out) {
+  pdl_prologue();
+  const uint32_t groups = C / 16u;
+  const uint32_t idx = blockIdx.x * blockDim.x + threadIdx.x;
+  if (idx >= N * groups) return;
+  const uint32_t n = idx / groups, g = idx - n * groups;
+  const uint8_t* src = x + (size_t)n * HW * C + g * 16u;
+  int sum[16];
+#pragma unroll
+  for (int j = 0; j < 16; ++j) sum[j] = 0;
+#pragma unroll 4
+  for (uint32_t p = 0; p < HW; ++p) {
+    const uint4 v = __ldcg(reinterpret_cast<const uint4*>(src + (size_t)p * C));
+    const uint32_t w4[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+    for (int j = 0; j < 16; ++j) sum[j] += (int)((w4[j >> 2] >> (8 * (j & 3))) & 0xFFu);
+  }
+  uint32_t q[4] = {0u, 0u, 0u, 0u};
+#pragma unroll
+  for (int j = 0; j < 16; ++j)
+    q[j >> 2] |= ((uint32_t)requant((float)sum[j], pool_mul, qmin, qmax) & 0xFFu) << (8 * (j & 3));
+  *reinterpret_cast<uint4*>(out + (size_t)n * C + g * 16u) = make_uint4(q[0], q[1], q[2], q[3]);
+}
+
 __global__ void avgpool_kernel(const uint8_t* x, uint32_t nchw, uint32_t N, uint32_t C,
                                uint32_t HW, float pool_mul, int qmin, int qmax,
                                uint8_t* __restrict__ out) {
@@ -828,6 +855,12 @@ cudaError_t launch_maxpool(const uint8_t* x, uint32_t nchw, uint32_t N, uint32_t
 cudaError_t launch_avgpool(const uint8_t* x, uint32_t nchw, uint32_t N, uint32_t C, uint32_t H,
                            uint32_t W, float pool_mul, int32_t qmin, int32_t qmax, uint8_t* out,
                            cudaStream_t s) {
+  if (!nchw && C % 16u == 0 && !(((uintptr_t)x | (uintptr_t)out) & 15u) && (uint64_t)N * (C / 16u) < (1ull << 31)) {
+    const uint32_t threads = N * (C / 16u);
+    launch_pdl(avgpool_nhwc16_kernel, (threads + 127u) / 128u, 128, 0, s, x, N, C, H * W, pool_mul, qmin, qmax, out);
+    note_launch();
+    return cudaGetLastError();
+  }
   size_t warps = (size_t)N * C;
   uint32_t blocks = (uint32_t)((warps * 32 + 255) / 256);
   launch_pdl(avgpool_kernel, blocks, 256, 0, s, x, nchw, N, C, H * W, pool_mul, qmin, qmax, out); note_launch();

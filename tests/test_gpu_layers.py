@@ -454,6 +454,12 @@ def test_pooling_kernels(psb, ctx, oracle):
                               oracle.maxpool_u8(x, layout, 3, 2, 1))
         assert np.array_equal(ctx.global_avgpool_u8(xd, layout, 0.0123, 0, 255).cpu().numpy(),
                               oracle.global_avgpool_u8(x, layout, np.float32(0.0123), 0, 255))
+    # channels-last with whole 16-channel groups: the vectorised kernels
+    x = rng.integers(0, 256, size=(5, 7, 7, 48), dtype=np.uint8)
+    xd = torch.from_numpy(x).to(ctx.device)
+    assert np.array_equal(ctx.maxpool2d_u8(xd, 1, 3, 2, 1).cpu().numpy(), oracle.maxpool_u8(x, 1, 3, 2, 1))
+    assert np.array_equal(ctx.global_avgpool_u8(xd, 1, 0.0201, 0, 15).cpu().numpy(),
+                          oracle.global_avgpool_u8(x, 1, np.float32(0.0201), 0, 15))
 
 
 def test_contraction_timing_hook(psb, oracle):

@@ -399,7 +399,7 @@ __device__ __forceinline__ void sample_block(const SampleParams& p, uint32_t blo
       if (tap == 0 && ci == 0) e_base_out[o] = Emax ? ebase_biased - 127 : 0;
       uint32_t cntpk[kMaxLevels] = {0u, 0u, 0u, 0u, 0u, 0u, 0u};
       uint32_t meta = 0u;
-#pragma unroll
+#pragma unroll 1       // one copy of the drawing code: unrolled four times it no longer fits the instruction cache
       for (int j = 0; j < 4; ++j) {
         const uint32_t u = __float_as_uint(stage[r * per_row + (cl + (uint32_t)j) * KHKW + tap]);
         const uint64_t index = (uint64_t)o * d + (uint64_t)(ci + (uint32_t)j) * KHKW + tap;  // canonical

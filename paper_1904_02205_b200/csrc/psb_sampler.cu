@@ -335,6 +335,9 @@ struct SampleParams {
   int planes_count[kMaxLevels];
 };
 
+// kVec: whether the instance contains the four-weights-per-thread loop at all (a launch whose items are all
+// small carries only the one-weight loop: with the L2 cold, what a short kernel costs is mostly its code)
+template <bool kVec>
 __device__ __forceinline__ void sample_block(const SampleParams& p, uint32_t block, const PhiloxKeys& keys,
                                              float* stage) {
   // the parameters may sit in global memory (batched launch): read the scalars once
@@ -381,9 +384,9 @@ __device__ __forceinline__ void sample_block(const SampleParams& p, uint32_t blo
   int32_t* const e_base_out = p.e_base;
   // count <= kStage and the divisors are block-uniform: divisions by multiply-high.  The slice is walked in
   // output order (row, tap, channel) so that stores coalesce.
-  if (!packed_kw && has_planes && ((cc | Cg | c0) & 3u) == 0u) {
-    // Four consecutive channels per thread: one 16-byte store of the integer weights and one 4-byte store per
-    // digit plane and level.  Between the draws and the stores the four weights' counts travel as the bytes of
+  if (kVec && !packed_kw && has_planes && ((cc | Cg | c0) & 3u) == 0u && count >= 4u * blockDim.x) {
+    // Items that give every thread at least four weights: four consecutive channels per thread, one 16-byte
+    // store of the integer weights and one 4-byte store per digit plane and level.  Between the draws and the stores the four weights' counts travel as the bytes of
     // one word per level (c_k <= 64), and (sh, base, sign) as one byte per weight.
     const uint32_t cc4 = cc >> 2, per_row4 = per_row >> 2;
     const uint32_t per_row4_magic = small_div_magic(per_row4), cc4_magic = small_div_magic(cc4);
@@ -531,11 +534,12 @@ __device__ __forceinline__ void sample_block(const SampleParams& p, uint32_t blo
   }
 }
 
+template <bool kVec>
 __global__ void __launch_bounds__(kThreads) sample_kernel(const __grid_constant__ SampleParams p,
                                                           const __grid_constant__ PhiloxKeys keys) {
   pdl_prologue();
   __shared__ float stage[kStage];
-  sample_block(p, blockIdx.x, keys, stage);
+  sample_block<kVec>(p, blockIdx.x, keys, stage);
 }
 
 // All layers of a network in two launches.  Entry i owns blocks [first, first + count) of each
@@ -569,7 +573,7 @@ __global__ void __launch_bounds__(kThreads) sample_batch_kernel(const BatchEntry
   pdl_prologue();
   __shared__ float stage[kStage];
   const BatchEntry& e = entries[find_entry(entries, n, blockIdx.x, false)];
-  sample_block(e.p, blockIdx.x - e.sample_first, keys, stage);
+  sample_block<true>(e.p, blockIdx.x - e.sample_first, keys, stage);
 }
 
 // 128 * (sum of each filter row): the constant that restores sum x*W from sum (x-128)*W when
@@ -607,8 +611,9 @@ namespace {
 uint32_t emax_blocks_for(uint32_t O, uint32_t d, uint32_t norm) {
   if (norm) return d <= (uint32_t)kEmaxLongRow ? (O + (uint32_t)kEmaxRows - 1u) / (uint32_t)kEmaxRows : O;
   size_t total = (size_t)O * d;
-  // sixteen weights per thread (four 16-byte loads in flight)
+  // sixteen weights per thread (four 16-byte loads in flight) once that still fills the machine, four otherwise
   uint32_t blocks = (uint32_t)((total + kThreads * 16 - 1) / (kThreads * 16));
+  if (blocks < 296u) blocks = (uint32_t)std::min<size_t>(296u, (total + kThreads * 4 - 1) / (kThreads * 4));
   return blocks < 1 ? 1 : (blocks > 1184 ? 1184 : blocks);
 }
 
@@ -689,7 +694,13 @@ cudaError_t launch_sampler(const float* w_dev, psb_weights* wt, uint32_t* err_de
   SampleParams p;
   const uint32_t blocks = fill_sample_params(w_dev, wt, wt->e_max, p, false);
   p.e_tag = wt->e_calls;
-  launch_pdl(sample_kernel, blocks, kThreads, 0, s, p, PhiloxKeys(p.seed_lo, p.seed_hi)); note_launch();
+  // items of fewer than four weights per thread never take the four-weights loop: launch the instance without it
+  const uint64_t item_weights = (uint64_t)p.rows_per_block * std::min<uint64_t>(p.ch_per_block, p.Cg) * p.KHKW;
+  if (item_weights >= 4u * (uint64_t)kThreads)
+    launch_pdl(sample_kernel<true>, blocks, kThreads, 0, s, p, PhiloxKeys(p.seed_lo, p.seed_hi));
+  else
+    launch_pdl(sample_kernel<false>, blocks, kThreads, 0, s, p, PhiloxKeys(p.seed_lo, p.seed_hi));
+  note_launch();
   return cudaGetLastError();
 }
 

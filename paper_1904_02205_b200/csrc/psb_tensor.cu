@@ -542,7 +542,7 @@ __device__ __noinline__ void epilogue_chunk(const TensorParams& p, uint32_t tadd
 }
 
 // True when the layer takes the specialised epilogue loop below.
-__device__ __forceinline__ bool uniform_epilogue(const TensorParams& p) {
+__host__ __device__ __forceinline__ bool uniform_epilogue(const TensorParams& p) {
   const ConvArgs& a = p.a;
   const bool q_only = a.q_out && !a.f32_out && !a.acc_out && (p.vec_ok || a.out_nchw) && a.inv_step > 0.0f;
   if (a.kmap) {
@@ -977,7 +977,9 @@ __device__ __noinline__ bool mma_role_band(const TensorParams& p, SharedCtl* ctl
   return false;
 }
 
-template <int BK>
+// kGeneral: which output stage the instance carries, the loop for the common case (uniform_epilogue) or the
+// general one; the host picks the instance, so neither drags the other's code and registers along.
+template <int BK, bool kGeneral>
 __global__ void __launch_bounds__(kThreadsTensor, 1)
 psb_mma_kernel(const __grid_constant__ TmapSet maps, const __grid_constant__ TensorParams p) {
   extern __shared__ uint8_t smem_raw[];
@@ -1159,7 +1161,7 @@ psb_mma_kernel(const __grid_constant__ TmapSet maps, const __grid_constant__ Ten
                   bar);
       }
     }
-    if (uniform_epilogue(p)) {
+    if (!kGeneral) {
       bool w32 = true;
       if (a.kmap) {          // every level a tile may have must fit
         for (uint32_t lv = 0; lv < (uint32_t)kMaxLevels; ++lv)
@@ -1501,10 +1503,17 @@ psb_status launch_tensor(psb_ctx* ctx, const psb_weights* wt, const ConvArgs& a,
   cfg.attrs = attr;
   cfg.numAttrs = 1;
 #define PSB_LAUNCH(BKV)                                                                              \
-  e = cudaFuncSetAttribute(psb_mma_kernel<BKV>, cudaFuncAttributeMaxDynamicSharedMemorySize,         \
-                           (int)smem_bytes);                                                         \
-  if (e == cudaSuccess) e = cudaLaunchKernelEx(&cfg, psb_mma_kernel<BKV>, maps, p);                  \
+  if (general) {                                                                                     \
+    e = cudaFuncSetAttribute(psb_mma_kernel<BKV, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, \
+                             (int)smem_bytes);                                                       \
+    if (e == cudaSuccess) e = cudaLaunchKernelEx(&cfg, psb_mma_kernel<BKV, true>, maps, p);          \
+  } else {                                                                                           \
+    e = cudaFuncSetAttribute(psb_mma_kernel<BKV, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,\
+                             (int)smem_bytes);                                                       \
+    if (e == cudaSuccess) e = cudaLaunchKernelEx(&cfg, psb_mma_kernel<BKV, false>, maps, p);         \
+  }                                                                                                  \
   note_launch();
+  const bool general = !uniform_epilogue(p);
   const bool timed = ctx->time_contraction && ctx->t_begin[0] && ctx->timed_launches < psb_ctx::kTimedLaunches;
   if (timed) cudaEventRecord(ctx->t_begin[ctx->timed_launches], s);
   if (bk == 128) { PSB_LAUNCH(128) } else if (bk == 64) { PSB_LAUNCH(64) } else { PSB_LAUNCH(32) }

@@ -282,7 +282,7 @@ __global__ void __launch_bounds__(256, 2) dwconv3x3_row_kernel(const ConvArgs a,
 // consecutive outputs of one row and works channel by channel: the bytes of the 3 x kCols input words are
 // extracted once per row and channel and serve up to three outputs each, one multiply-add per tap; the output
 // stage is dequant()/requant() with conversion-unit instructions (one int -> float, one float -> int, both
-// round to nearest even as the definitions ask).  About 20 instructions per output where the 64-bit kernel
+// round to nearest even as the definitions ask).  About 25 instructions per output where the 64-bit kernel
 // above needs about 70.
 template <typename Acc>
 __device__ __forceinline__ float dw_acc_to_float(Acc acc);

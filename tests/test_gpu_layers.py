@@ -308,13 +308,13 @@ def test_tensor_path_per_location_draw_counts(psb, ctx, oracle):
 
 @pytest.mark.parametrize("case", [(3, 64, 10, 16, 64, False), (2, 128, 7, 24, 72, True), (5, 32, 9, 8, 64, True)])
 def test_tensor_path_per_location_draw_counts_1x1_patch_tiles(psb, ctx, oracle, case):
-    """1x1 layers under a per-location map on channels-last tensors whose width is a multiple of 8 are tiled
-    in 8 x 16 patches (rows of all images stacked): ragged last patch rows, patches across image borders."""
+    """1x1 layers under a per-location map on channels-last tensors (rows sorted by level, gathered, scattered back
+    in the output stage): ragged sizes, a smooth region with a single level, with and without a shortcut."""
     N, C, H, W, O, with_res = case
     rng = np.random.default_rng(abs(hash(case)) % 2 ** 31)
     w, x, scale, bias = _layer_inputs(rng, N, C, H, W, O, 1, 1, 1, 1)
     kmap = rng.choice([0, 1, 2, 3, 4], size=(N, H, W)).astype(np.uint8)
-    kmap[0, : H // 2] = 2                       # a smooth region: patches with a single level
+    kmap[0, : H // 2] = 2                       # a smooth region: whole tiles of one level
     res = rng.integers(0, 16, size=(N, H, W, O)).astype(np.uint8) if with_res else None
     g = _both(psb, ctx, oracle, w, x, 1, 1, 1, 0, [0, 1, 2, 3, 4], scale, bias, kmap=kmap, inv_step=0.5,
               residual=res, res_scale=0.2 if with_res else 0.0, in_max=15, path=psb.PSB_PATH_TENSOR)

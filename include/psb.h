@@ -19,9 +19,14 @@
  *   - Every pointer named *_dev is DEVICE memory owned by the caller unless said
  *     otherwise; everything else is host memory.  Sizes are in elements.
  *   - `stream` is a cudaStream_t passed as void*.  All compute calls are
- *     asynchronous on that stream and never synchronise the device; only
- *     psb_create, psb_destroy, the first psb_sample_weights for a handle,
- *     psb_weights_free and psb_device_status may block.
+ *     asynchronous on that stream and do not synchronise the device, with one
+ *     exception: a call that needs a larger internal scratch buffer than any
+ *     call before it on this context (layout conversion, gathered matrices,
+ *     the sorted order of a draw-count map) frees and allocates device
+ *     memory, which waits for the device; after one pass over a network's
+ *     shapes no call grows anything.  Otherwise only psb_create, psb_destroy,
+ *     the first psb_sample_weights for a handle, psb_weights_free and
+ *     psb_device_status may block.
  *   - Every function returns a psb_status: 0 on success, negative on error.
  *     Arguments are validated on the host before anything is launched; a call
  *     that returns an error has launched nothing.  There is no CPU fallback: if

@@ -713,8 +713,6 @@ struct psb_sample_batch {
   uint32_t* e_max_pool = nullptr;     // one word per output channel of every layer
   size_t e_max_words = 0;
   uint32_t emax_grid = 0, sample_grid = 0;
-  psb_weights** packed = nullptr;     // layers that need the offset correction recomputed
-  uint32_t n_packed = 0;
   int device = 0;
 };
 
@@ -724,8 +722,7 @@ psb_status sample_batch_create(psb_ctx* ctx, uint32_t n, const float* const* w_d
                                psb_weights* const* weights, psb_sample_batch** out) {
   psb_sample_batch* b = new (std::nothrow) psb_sample_batch();
   BatchEntry* host = new (std::nothrow) BatchEntry[n];
-  psb_weights** packed = new (std::nothrow) psb_weights*[n];
-  if (!b || !host || !packed) { delete b; delete[] host; delete[] packed; return PSB_ERR_ALLOC; }
+  if (!b || !host) { delete b; delete[] host; return PSB_ERR_ALLOC; }
   size_t words = 0;
   for (uint32_t i = 0; i < n; ++i) words += weights[i]->shape.out_ch;
   bool ok = cudaMalloc(&b->e_max_pool, sizeof(uint32_t) * words) == cudaSuccess &&
@@ -743,7 +740,6 @@ psb_status sample_batch_create(psb_ctx* ctx, uint32_t n, const float* const* w_d
       eb += e.emax_blocks;
       sb += e.sample_blocks;
       off += wt->shape.out_ch;
-      if (wt->packed_k) packed[b->n_packed++] = weights[i];
     }
     b->emax_grid = eb;
     b->sample_grid = sb;
@@ -754,13 +750,11 @@ psb_status sample_batch_create(psb_ctx* ctx, uint32_t n, const float* const* w_d
     cudaGetLastError();
     if (b->e_max_pool) cudaFree(b->e_max_pool);
     if (b->entries_dev) cudaFree(b->entries_dev);
-    delete[] packed;
     delete b;
     return PSB_ERR_ALLOC;
   }
   b->n = n;
   b->e_max_words = words;
-  b->packed = packed;
   b->device = ctx->device;
   *out = b;
   return PSB_OK;
@@ -780,7 +774,6 @@ psb_status sample_batch_run(psb_ctx* ctx, psb_sample_batch* b, uint64_t seed, cu
 void sample_batch_free(psb_sample_batch* b) {
   if (b->e_max_pool) cudaFree(b->e_max_pool);
   if (b->entries_dev) cudaFree(b->entries_dev);
-  delete[] b->packed;
   delete b;
 }
 

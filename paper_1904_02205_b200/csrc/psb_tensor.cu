@@ -1328,6 +1328,7 @@ bool is_plain_gemm(const ConvArgs& a) {
 }
 
 constexpr size_t kSmemBudget = 227 * 1024;
+constexpr int kMaxDevicesForAttr = 64;
 
 }  // namespace
 
@@ -1502,22 +1503,28 @@ psb_status launch_tensor(psb_ctx* ctx, const psb_weights* wt, const ConvArgs& a,
   cfg.stream = s;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-#define PSB_LAUNCH(BKV)                                                                              \
-  if (general) {                                                                                     \
-    e = cudaFuncSetAttribute(psb_mma_kernel<BKV, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, \
-                             (int)smem_bytes);                                                       \
-    if (e == cudaSuccess) e = cudaLaunchKernelEx(&cfg, psb_mma_kernel<BKV, true>, maps, p);          \
-  } else {                                                                                           \
-    e = cudaFuncSetAttribute(psb_mma_kernel<BKV, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,\
-                             (int)smem_bytes);                                                       \
-    if (e == cudaSuccess) e = cudaLaunchKernelEx(&cfg, psb_mma_kernel<BKV, false>, maps, p);         \
-  }                                                                                                  \
+  // the shared-memory limit of an instance is raised once per device, to the most a launch can ask for
+#define PSB_LAUNCH_INST(BKV, GEN, SLOT)                                                              \
+  {                                                                                                  \
+    static bool raised[kMaxDevicesForAttr][6];                                                       \
+    const int dv = ctx->device;                                                                      \
+    e = cudaSuccess;                                                                                 \
+    if (dv < 0 || dv >= kMaxDevicesForAttr || !raised[dv][SLOT]) {                                   \
+      e = cudaFuncSetAttribute(psb_mma_kernel<BKV, GEN>, cudaFuncAttributeMaxDynamicSharedMemorySize,\
+                               (int)kSmemBudget);                                                    \
+      if (e == cudaSuccess && dv >= 0 && dv < kMaxDevicesForAttr) raised[dv][SLOT] = true;           \
+    }                                                                                                \
+    if (e == cudaSuccess) e = cudaLaunchKernelEx(&cfg, psb_mma_kernel<BKV, GEN>, maps, p);           \
+  }
+#define PSB_LAUNCH(BKV, SLOT)                                                                        \
+  if (general) PSB_LAUNCH_INST(BKV, true, SLOT) else PSB_LAUNCH_INST(BKV, false, SLOT + 1)           \
   note_launch();
   const bool general = !uniform_epilogue(p);
   const bool timed = ctx->time_contraction && ctx->t_begin[0] && ctx->timed_launches < psb_ctx::kTimedLaunches;
   if (timed) cudaEventRecord(ctx->t_begin[ctx->timed_launches], s);
-  if (bk == 128) { PSB_LAUNCH(128) } else if (bk == 64) { PSB_LAUNCH(64) } else { PSB_LAUNCH(32) }
+  if (bk == 128) { PSB_LAUNCH(128, 0) } else if (bk == 64) { PSB_LAUNCH(64, 2) } else { PSB_LAUNCH(32, 4) }
 #undef PSB_LAUNCH
+#undef PSB_LAUNCH_INST
   if (timed) {
     cudaEventRecord(ctx->t_end[ctx->timed_launches], s);
     ++ctx->timed_launches;

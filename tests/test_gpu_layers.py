@@ -729,6 +729,39 @@ def test_sampler_options_all_levels(psb, ctx, oracle, opts, shape, groups, norm)
         wt.free()
 
 
+@pytest.mark.parametrize("opts", [dict(), dict(underflow=1), dict(prob_bits=4), dict(prob_bits=5, underflow=1),
+                                  dict(prob_bits=8, deterministic=1)])
+@pytest.mark.parametrize("shape,norm", [((320, 1280, 1, 1), 0), ((320, 1280, 1, 1), 1), ((256, 192, 3, 3), 1)])
+def test_large_layer_sampled_by_its_own_launch(psb, ctx, oracle, opts, shape, norm):
+    """A layer large enough that a launch of its own gives every thread four weights (the sampler's vectorised
+    loop, otherwise reached through the batched launch of a network only): integer filters of every level against
+    the oracle under every option, and the digit planes through a contraction on a few locations."""
+    import torch
+
+    rng = np.random.default_rng(abs(hash((shape, norm, tuple(sorted(opts.items()))))) % 2 ** 31)
+    w = (rng.normal(0, 0.05, size=shape) * 2.0 ** rng.integers(-7, 1, size=shape)).astype(np.float32)
+    flat = w.reshape(-1)
+    flat[rng.random(flat.size) < 0.05] = 0.0
+    flat[:6] = [0.5, -0.25, 1e-41, 3e-9, 0.99999994, -1.9999999]
+    for exp_bits in (4, 3):
+        wt = ctx.sample_weights(torch.from_numpy(w).cuda(), seed=2 ** 33 + 9, layer_id=6, level_mask=0x7F,
+                                exp_bits=exp_bits, norm=norm, **opts)
+        for l in range(7):
+            Wg, ebg = (v.cpu().numpy() for v in ctx.weights_export(wt, l))
+            Wo, ebo = oracle.sample_level_ex(w, 2 ** 33 + 9, 6, l, exp_bits=exp_bits, norm=norm, **opts)[:2]
+            assert np.array_equal(ebg, ebo), (exp_bits, l)
+            assert np.array_equal(Wg.astype(np.int64), Wo), (shape, norm, exp_bits, l, opts)
+        assert ctx.device_status() == 0
+        wt.free()
+    O, C, K, _ = shape
+    x = rng.integers(0, 16, size=(1, 12, 11, C)).astype(np.uint8)
+    scale = rng.uniform(0.5, 1.5, size=O).astype(np.float32)
+    bias = rng.normal(0, 0.1, size=O).astype(np.float32)
+    g = _both(psb, ctx, oracle, w, x, 1, 1, 1, K // 2, [3], scale, bias, inv_step=0.3, in_max=15, norm=norm,
+              path=psb.PSB_PATH_TENSOR, opts=opts or None)
+    assert g["path"] == psb.PSB_PATH_TENSOR
+
+
 @pytest.mark.parametrize("exp_bits,opts", [(3, dict(underflow=1)), (2, dict(underflow=1)), (3, dict(underflow=1, prob_bits=4)),
                                            (4, dict(prob_bits=4))])
 @pytest.mark.parametrize("case", [(2, 64, 14, 13, 80, 3, 1, 1), (3, 128, 9, 11, 64, 3, 1, 0), (2, 256, 9, 9, 128, 1, 0, 1),

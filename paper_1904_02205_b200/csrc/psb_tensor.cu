@@ -683,29 +683,48 @@ __device__ __noinline__ bool epilogue_uniform(const TensorParams& p, SharedCtl* 
   ti.init(p);
   uint32_t pass = 0, cur_o_tile = 0xFFFFFFFFu;
   uint4 r_next = make_uint4(0, 0, 0, 0);
+  // Sorted rows: the location of this thread's row and the tile's level are lookups in global memory.  They are
+  // made one tile ahead (nx_*) and the shortcut fetch of the next tile, whose address depends on them, is issued
+  // after the accumulator wait instead of before it, so that no address waits for a lookup.
+  // (Without a shortcut nothing but the final store depends on the row's location, and looking ahead only
+  // costs registers: measured slower.)
+  constexpr bool kAhead = kSorted && HAS_RES;
+  uint32_t nx_m = 0, nx_levels = 0;
+  bool nx_ok = false;
+  if (kAhead && ti.valid()) {
+    nx_m = rm.row_index(ti.m_tile, row, &nx_ok);
+    nx_levels = tile_levels(p, ti.m_tile);
+  }
   if (HAS_RES && ti.valid()) {
     bool ok_row;
-    const uint32_t m = rm.row_index(ti.m_tile, row, &ok_row), ob = ti.o_tile * kTileN + sub * 16u;
+    uint32_t m = nx_m;
+    if (kAhead) ok_row = nx_ok; else m = rm.row_index(ti.m_tile, row, &ok_row);
+    const uint32_t ob = ti.o_tile * kTileN + sub * 16u;
     if (ok_row && ob < rm.O) {
       const uint8_t* src = res_base + rm.offset(m, ob);
       r_next = planar ? load_planar16<TAG>(src, ohow, rm.O - ob) : load_row16(src, vec16, ob + 16u <= rm.O);
     }
   }
   while (ti.valid()) {
-    bool row_valid;
-    const uint32_t m = rm.row_index(ti.m_tile, row, &row_valid);
+    bool row_valid = nx_ok;
+    uint32_t m = nx_m;
+    if (!kAhead) m = rm.row_index(ti.m_tile, row, &row_valid);
     const uint32_t o_tile = ti.o_tile;
     const uint32_t o_base = o_tile * kTileN + sub * 16u;
     const bool active = o_base < rm.O;          // warp-uniform
     if (kSorted) {
       // the tile's level; a tile without a sampled level gets no pass from the other roles either
-      const uint32_t levels = tile_levels(p, ti.m_tile);
+      const uint32_t levels = kAhead ? nx_levels : tile_levels(p, ti.m_tile);
       if (!(levels & a.level_mask & 0x7Fu)) {
         if (row_valid) atomicOr(a.err, kDevErrBadLevel);     // a location asks for a level that was not sampled
         ti.next();
+        if (kAhead && ti.valid()) {
+          nx_m = rm.row_index(ti.m_tile, row, &nx_ok);
+          nx_levels = tile_levels(p, ti.m_tile);
+        }
         if (HAS_RES && ti.valid()) {
-          bool ok_row;
-          const uint32_t mn = rm.row_index(ti.m_tile, row, &ok_row), ob = ti.o_tile * kTileN + sub * 16u;
+          const bool ok_row = nx_ok;
+          const uint32_t mn = nx_m, ob = ti.o_tile * kTileN + sub * 16u;
           r_next = make_uint4(0, 0, 0, 0);
           if (ok_row && ob < rm.O) {
             const uint8_t* src = res_base + rm.offset(mn, ob);
@@ -717,6 +736,10 @@ __device__ __noinline__ bool epilogue_uniform(const TensorParams& p, SharedCtl* 
       l = (uint32_t)__ffs((int)(levels & a.level_mask & 0x7Fu)) - 1u;
     }
     ti.next();
+    if (kAhead && ti.valid()) {
+      nx_m = rm.row_index(ti.m_tile, row, &nx_ok);
+      nx_levels = tile_levels(p, ti.m_tile);
+    }
     if ((kSorted ? o_tile * 8u + l : o_tile) != cur_o_tile) {
       // per-channel constants of this channel tile: the warp keeps its own copy of its 16 channels
       __syncwarp();
@@ -736,7 +759,7 @@ __device__ __noinline__ bool epilogue_uniform(const TensorParams& p, SharedCtl* 
       __syncwarp();
     }
     const uint4 r_cur = r_next;
-    if (HAS_RES && ti.valid()) {
+    if (HAS_RES && !kAhead && ti.valid()) {
       bool ok_row;
       const uint32_t mn = rm.row_index(ti.m_tile, row, &ok_row), ob = ti.o_tile * kTileN + sub * 16u;
       r_next = make_uint4(0, 0, 0, 0);
@@ -758,6 +781,14 @@ __device__ __noinline__ bool epilogue_uniform(const TensorParams& p, SharedCtl* 
     tc_fence_before();
     __syncwarp();
     if (lane == 0) mbar_arrive(smem_u32(&ctl->acc_empty[buf]));
+    if (kAhead && ti.valid()) {
+      const uint32_t ob = ti.o_tile * kTileN + sub * 16u;
+      r_next = make_uint4(0, 0, 0, 0);
+      if (nx_ok && ob < rm.O) {
+        const uint8_t* src = res_base + rm.offset(nx_m, ob);
+        r_next = planar ? load_planar16<TAG>(src, ohow, rm.O - ob) : load_row16(src, vec16, ob + 16u <= rm.O);
+      }
+    }
     if (active && row_valid) {
       const uint4 q16 = chunk_math<P, W32, RES, FAST_U8>(v, r_cur, scb, corr, c);
       uint8_t* dst = q_base + rm.offset(m, o_base);

@@ -691,8 +691,8 @@ __device__ __noinline__ bool epilogue_uniform(const TensorParams& p, SharedCtl* 
   constexpr bool kAhead = kSorted && HAS_RES;
   uint32_t nx_m = 0, nx_levels = 0;
   bool nx_ok = false;
-  if (kAhead && ti.valid()) {
-    nx_m = rm.row_index(ti.m_tile, row, &nx_ok);
+  if (kSorted && ti.valid()) {
+    if (kAhead) nx_m = rm.row_index(ti.m_tile, row, &nx_ok);
     nx_levels = tile_levels(p, ti.m_tile);
   }
   if (HAS_RES && ti.valid()) {
@@ -714,12 +714,12 @@ __device__ __noinline__ bool epilogue_uniform(const TensorParams& p, SharedCtl* 
     const bool active = o_base < rm.O;          // warp-uniform
     if (kSorted) {
       // the tile's level; a tile without a sampled level gets no pass from the other roles either
-      const uint32_t levels = kAhead ? nx_levels : tile_levels(p, ti.m_tile);
+      const uint32_t levels = nx_levels;
       if (!(levels & a.level_mask & 0x7Fu)) {
         if (row_valid) atomicOr(a.err, kDevErrBadLevel);     // a location asks for a level that was not sampled
         ti.next();
-        if (kAhead && ti.valid()) {
-          nx_m = rm.row_index(ti.m_tile, row, &nx_ok);
+        if (ti.valid()) {
+          if (kAhead) nx_m = rm.row_index(ti.m_tile, row, &nx_ok);
           nx_levels = tile_levels(p, ti.m_tile);
         }
         if (HAS_RES && ti.valid()) {
@@ -736,8 +736,8 @@ __device__ __noinline__ bool epilogue_uniform(const TensorParams& p, SharedCtl* 
       l = (uint32_t)__ffs((int)(levels & a.level_mask & 0x7Fu)) - 1u;
     }
     ti.next();
-    if (kAhead && ti.valid()) {
-      nx_m = rm.row_index(ti.m_tile, row, &nx_ok);
+    if (kSorted && ti.valid()) {
+      if (kAhead) nx_m = rm.row_index(ti.m_tile, row, &nx_ok);
       nx_levels = tile_levels(p, ti.m_tile);
     }
     if ((kSorted ? o_tile * 8u + l : o_tile) != cur_o_tile) {

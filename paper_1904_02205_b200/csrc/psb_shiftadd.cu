@@ -462,7 +462,6 @@ __global__ void __launch_bounds__(256) im2col_s8_kernel(const ConvArgs a, uint32
   bool bad = false;
   extern __shared__ __align__(16) uint32_t im2col_smem[];     // [staged rows][span_pitch / 4] words
   __shared__ uint32_t row_adj[(kIm2colRows - 1u) * 8u + 128u];   // per staged row: byte offset of the span's start
-  uint8_t* rows = reinterpret_cast<uint8_t*>(im2col_smem);
   const uint32_t span_pitch = im2col_span_pitch(a.stride, a.C, run_pitch);
   const uint32_t strips = (a.OW + kIm2colPix - 1) / kIm2colPix;
   const uint32_t row_groups = (a.OH + kIm2colRows - 1) / kIm2colRows;

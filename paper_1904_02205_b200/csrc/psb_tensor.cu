@@ -204,16 +204,6 @@ __device__ __forceinline__ void tc_commit(uint32_t bar) {
                : "memory");
 }
 
-__device__ __forceinline__ void tc_mma_i8(uint32_t d_tmem, uint64_t desc_a, uint64_t desc_b,
-                                          uint32_t idesc, uint32_t accumulate) {
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "setp.ne.b32 p, %4, 0;\n\t"
-      "tcgen05.mma.cta_group::1.kind::i8 [%0], %1, %2, %3, p;\n\t}"
-      ::"r"(d_tmem), "l"(desc_a), "l"(desc_b), "r"(idesc), "r"(accumulate)
-      : "memory");
-}
-
 // The same instruction for the issue loops: accumulate always, descriptors given as (low word, high word),
 // no memory clobber (the loop's own loads of descriptor offsets may then be scheduled ahead of it; the
 // operands are written by the copy engine and ordered by the barrier waits, which keep their clobbers).
@@ -249,19 +239,6 @@ __device__ __forceinline__ void tc_ld16(uint32_t taddr, uint32_t (&v)[16]) {
 }
 __device__ __forceinline__ void tc_wait_ld() {
   asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-}
-
-// Shared-memory matrix descriptor of a K-major tile whose rows are `bk` bytes wide
-// and swizzled with the matching TMA mode; groups of 8 rows are 8*bk bytes apart.
-__device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t bk) {
-  const uint64_t layout = bk == 128 ? 2ull : (bk == 64 ? 4ull : 6ull);
-  uint64_t d = 0;
-  d |= (uint64_t)((addr & 0x3FFFFu) >> 4);
-  d |= (uint64_t)1 << 16;                       // leading byte offset (unused for swizzled K-major)
-  d |= (uint64_t)((8u * bk) >> 4) << 32;        // stride byte offset between 8-row groups
-  d |= (uint64_t)1 << 46;                       // descriptor version of this architecture
-  d |= layout << 61;
-  return d;
 }
 
 // The two words of that descriptor.  Only the low word depends on the address (bits 0..13 = address / 16;
@@ -449,13 +426,6 @@ __device__ __noinline__ void store_planar16(uint8_t* dst, size_t plane, uint32_t
     if ((uint32_t)j < count) dst[(size_t)j * plane] = (uint8_t)(w[j >> 2] >> (8 * (j & 3)));
 }
 
-// Offset of (row m, channel o_base) in the output tensor, either layout.
-__device__ __forceinline__ size_t out_offset(const ConvArgs& a, uint32_t ohow, uint32_t m, uint32_t o_base) {
-  if (!a.out_nchw) return (size_t)m * a.O + o_base;
-  const uint32_t n = m / ohow;
-  return ((size_t)n * a.O + o_base) * ohow + (m - n * ohow);
-}
-
 // The P plane sums of a 16-channel chunk, TMEM -> registers.  With 32-bit recombination the planes are
 // folded as they arrive (v0 + 2^7 v1 + ..., what chunk_math computes first anyway): 32 registers at the
 // peak instead of 16 P, which is what the loop around it was spilling.  The folded planes are left as
@@ -557,22 +527,6 @@ __host__ __device__ __forceinline__ bool uniform_epilogue(const TensorParams& p)
   }
   const uint32_t P0 = p.planes[a.uniform_log2k < (uint32_t)kMaxLevels ? a.uniform_log2k : 0u];
   return q_only && P0 >= 2u && P0 <= 4u;
-}
-
-// Linear output index (n * OH + oy) * OW + ox of row `row` of row tile `m_tile`, and whether the
-// row is a real output.  Plain mode: rows are consecutive outputs.  Band mode: rows are
-// padded-linear positions of one image.
-__device__ __forceinline__ uint32_t tile_row_index(const TensorParams& p, uint32_t m_tile, uint32_t row, bool* valid) {
-  if (!p.band) {
-    const uint32_t m = m_tile * kTileM + row;
-    *valid = m < p.M;
-    return m;
-  }
-  const uint32_t n = __umulhi(m_tile, p.tpi_magic);
-  const uint32_t t = (m_tile - n * p.tpi) * kTileM + row;
-  const uint32_t oy = __umulhi(t, p.Wp_magic), ox = t - oy * p.Wp;
-  *valid = oy < p.a.OH && ox < p.a.OW;
-  return (n * p.a.OH + oy) * p.a.OW + ox;
 }
 
 // The same two functions on register copies of the few parameters they need.  Inside an out-of-line
